@@ -1,0 +1,222 @@
+"""Pins for the oracle's state update (Eqs. 7, 12), the multi-anchor estimate and
+gate (Eqs. 8-11) and the state-size bookkeeping (Sec. 3.1 memory example).
+
+The factorisation is checked against library SVDs (numpy / torch, fp64), the
+Eckart-Young optimum and closed-form eigenproblems -- none of which is the
+oracle's own Jacobi routine.
+"""
+import math
+import os
+
+import numpy as np
+import torch
+
+from oracle import kvc_oracle as orc
+
+
+def _bits(x):
+    t = torch.as_tensor(np.asarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16).copy()
+
+
+def _val(bits):
+    return torch.from_numpy(np.asarray(bits).view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+
+
+def test_jacobi_closed_forms():
+    # 2x2: [[2,1],[1,2]] has eigenvalues 1 and 3 with eigenvectors (1,-1)/sqrt2, (1,1)/sqrt2
+    w, V = orc.jacobi_eigh(np.array([[2.0, 1.0], [1.0, 2.0]]))
+    order = np.argsort(w)
+    assert np.allclose(w[order], [1.0, 3.0], atol=1e-14)
+    assert np.allclose(np.abs(V[:, order[1]]), [1 / math.sqrt(2)] * 2, atol=1e-14)
+    # second-difference matrix tridiag(-1, 2, -1) of order n: eigenvalues 2 - 2 cos(k pi/(n+1))
+    n = 12
+    A = 2 * np.eye(n) - np.eye(n, k=1) - np.eye(n, k=-1)
+    w, V = orc.jacobi_eigh(A)
+    exp = 2 - 2 * np.cos(np.arange(1, n + 1) * math.pi / (n + 1))
+    assert np.allclose(np.sort(w), np.sort(exp), atol=1e-13)
+    assert np.allclose(V.T @ V, np.eye(n), atol=1e-13)
+    assert np.allclose(A @ V, V * w, atol=1e-12)
+
+
+def test_fit_matches_library_svd_and_eckart_young():
+    rng = np.random.default_rng(0)
+    T, d, r = 90, 24, 6
+    delta = rng.standard_normal((T, d)) @ np.diag(np.linspace(3.0, 0.1, d)) @ rng.standard_normal((d, d))
+    B, w = orc.fit_basis(delta, r)
+    A = orc.project(delta, B)
+    U, S, Vt = np.linalg.svd(delta, full_matrices=False)
+    S_t = torch.linalg.svdvals(torch.from_numpy(delta)).numpy()
+    # eigenvalues of the Gram matrix are the squared singular values, sorted descending
+    assert np.allclose(w, S ** 2, rtol=1e-10)
+    assert np.allclose(w, S_t ** 2, rtol=1e-10)
+    # B rows orthonormal, equal to the top right singular vectors up to sign
+    assert np.allclose(B @ B.T, np.eye(r), atol=1e-12)
+    assert np.allclose(np.abs(np.sum(B * Vt[:r], axis=1)), 1.0, atol=1e-9)
+    # sign convention: the largest-magnitude entry of each row is positive
+    assert np.all(B[np.arange(r), np.argmax(np.abs(B), axis=1)] > 0)
+    # A = U_r Sigma_r: columns orthogonal with norms sigma_1 >= ... >= sigma_r
+    Gm = A.T @ A
+    assert np.allclose(Gm, np.diag(S[:r] ** 2), atol=1e-8 * S[0] ** 2)
+    assert np.allclose(np.abs(A), np.abs(U[:, :r] * S[:r]), atol=1e-8 * S[0])
+    # Eckart-Young: the residual is the tail energy
+    res = np.sum((delta - A @ B) ** 2)
+    assert math.isclose(res, np.sum(S[r:] ** 2), rel_tol=1e-9)
+    # and no other rank-r projection does better (random subspaces)
+    for _ in range(5):
+        Q = np.linalg.qr(rng.standard_normal((d, r)))[0].T
+        assert np.sum((delta - (delta @ Q.T) @ Q) ** 2) >= res * (1 - 1e-12)
+
+
+def test_exact_rank_r_deviation_is_reconstructed_to_rounding():
+    # a deviation built exactly rank r (coeff x orthonormal basis) comes back to fp64 rounding
+    rng = np.random.default_rng(1)
+    T, d, r = 256, 64, 8
+    c = rng.standard_normal((T, r))
+    Bt = np.linalg.qr(rng.standard_normal((d, r)))[0].T
+    delta = c @ Bt
+    B, w = orc.fit_basis(delta, r)
+    A = orc.project(delta, B)
+    assert np.max(np.abs(A @ B - delta)) < 1e-12
+    assert np.all(np.abs(w[r:]) < 1e-12 * w[0])
+    # same subspace as the construction
+    assert np.allclose(B.T @ B, Bt.T @ Bt, atol=1e-10)
+    # full rank r = d reconstructs anything
+    delta = rng.standard_normal((40, 16))
+    B, _ = orc.fit_basis(delta, 16)
+    assert np.max(np.abs(orc.project(delta, B) @ B - delta)) < 1e-12
+
+
+def test_rank_limits_and_selection_basis():
+    rng = np.random.default_rng(2)
+    # fewer rows than the requested rank: rows beyond T are zero
+    delta = rng.standard_normal((3, 8))
+    B, w = orc.fit_basis(delta, 5)
+    assert np.allclose(B[3:], 0) and np.allclose(B[:3] @ B[:3].T, np.eye(3), atol=1e-12)
+    # projecting on unit rows picks channels
+    delta = rng.standard_normal((7, 8))
+    sel = np.eye(8)[[5, 0, 2]]
+    assert np.array_equal(orc.project(delta, sel), delta[:, [5, 0, 2]])
+
+
+def test_state_update_then_apply_round_trip():
+    # target = Align(src) + exact rank-r deviation (kept in float64, not re-quantised):
+    # FIT then the unrounded apply reproduces it to rounding; the first hop of a chain.
+    rng = np.random.default_rng(3)
+    L, H, T, d, r, s = 1, 2, 48, 16, 4, 16
+    f = orc.rope_inv_freq(d, 10000.0)
+    src = orc.Cache(_bits(rng.standard_normal((L, H, T, d))), _bits(rng.standard_normal((L, H, T, d))))
+    for l in range(L):
+        for h in range(H):
+            c = rng.standard_normal((T, r))
+            Bt = np.linalg.qr(rng.standard_normal((d, r)))[0].T
+            aligned = orc.rope_shift(_val(src.k[l, h]), s, f)
+            target = aligned + c @ Bt
+            dlt = target - aligned
+            B, _ = orc.fit_basis(dlt, r)
+            out = orc.chain_unrounded_slab(_val(src.k[l, h]), [0, s], [orc.project(dlt, B)], [B], f, True)[0]
+            assert np.max(np.abs(out - target)) < 1e-12
+
+
+def test_state_update_deviation_uses_aligned_source():
+    # Eq. 12: Delta = C_j - Align(C_i).  If the target is exactly the re-aligned source the
+    # key deviation vanishes; values ignore the shift.
+    rng = np.random.default_rng(4)
+    d, T, s = 8, 5, 11
+    f = orc.rope_inv_freq(d, 10000.0)
+    src = _bits(rng.standard_normal((T, d)))
+    aligned = orc.rope_shift(_val(src), s, f)
+    dk = orc.deviation(src, src, s, f, is_key=True)
+    assert np.allclose(dk, _val(src) - aligned, atol=1e-15) and np.max(np.abs(dk)) > 0.1
+    assert np.array_equal(orc.deviation(src, src, s, f, is_key=False), np.zeros((T, d)))
+    # src None: factorise the cache itself
+    assert np.array_equal(orc.deviation(None, src, s, f, is_key=True), _val(src))
+
+
+def test_state_update_project_mode_full():
+    rng = np.random.default_rng(5)
+    L, H, T, d, r, s = 2, 1, 12, 8, 3, -4
+    f = orc.rope_inv_freq(d, 10000.0)
+    src = orc.Cache(_bits(rng.standard_normal((L, H, T, d))), _bits(rng.standard_normal((L, H, T, d))))
+    tgt = orc.Cache(_bits(rng.standard_normal((L, H, T, d))), _bits(rng.standard_normal((L, H, T, d))))
+    bk = rng.standard_normal((L, H, r, d)).astype(np.float32)
+    bv = rng.standard_normal((L, H, r, d)).astype(np.float32)
+    st, _ = orc.state_update(src, tgt, s, f, mode=orc.PROJECT, basis_k=bk, basis_v=bv)
+    assert st.coeff_k.dtype == np.float32 and st.coeff_k.shape == (L, H, T, r)
+    # scalar re-derivation of a few entries
+    for (l, t, q) in ((0, 0, 0), (1, 7, 2), (1, 11, 1)):
+        acc_k = acc_v = 0.0
+        ks, kt = _val(src.k[l, 0, t]), _val(tgt.k[l, 0, t])
+        for c in range(d):
+            k = c % (d // 2)
+            ang = s * 10000.0 ** (-2.0 * k / d)
+            rot = (ks[k] * math.cos(ang) - ks[k + d // 2] * math.sin(ang)) if c < d // 2 else \
+                  (ks[k] * math.sin(ang) + ks[k + d // 2] * math.cos(ang))
+            acc_k += (kt[c] - rot) * float(bk[l, 0, q, c])
+            acc_v += (_val(tgt.v[l, 0, t])[c] - _val(src.v[l, 0, t])[c]) * float(bv[l, 0, q, c])
+        assert math.isclose(float(st.coeff_k[l, 0, t, q]), acc_k, rel_tol=1e-6, abs_tol=1e-6)
+        assert math.isclose(float(st.coeff_v[l, 0, t, q]), acc_v, rel_tol=1e-6, abs_tol=1e-6)
+
+
+# ---- gate and multi-anchor estimate (Eqs. 8-11) -----------------------------
+
+
+def test_entropy_limits():
+    for n in (2, 5, 10):
+        assert math.isclose(orc.normalized_entropy(np.full(n, 1.0 / n)), 1.0, rel_tol=1e-12)
+        one_hot = np.zeros(n)
+        one_hot[1] = 1.0
+        assert orc.normalized_entropy(one_hot) == 0.0
+    # two anchors, weights (1/4, 3/4): H = 2 - (3/4) log2 3
+    assert math.isclose(orc.normalized_entropy(np.array([0.25, 0.75])), 2 - 0.75 * math.log2(3), rel_tol=1e-12)
+    try:
+        orc.normalized_entropy(np.array([1.0]))
+        assert False, "a single anchor has no gate value"
+    except ValueError:
+        pass
+
+
+def test_gate_weights_and_distance():
+    g = orc.gate_weights(np.array([1.0, 1.0, 1.0]))
+    assert np.allclose(g, 1 / 3)
+    g = orc.gate_weights(np.array([0.0, math.log(3.0)]))        # exp(0) : exp(-ln 3) = 3 : 1
+    assert np.allclose(g, [0.75, 0.25])
+    # distance: two layers, prefix k = 2; differences 3 and 4 in single entries -> 5
+    a = [np.zeros((3, 2)), np.zeros((3, 2))]
+    b = [np.array([[3.0, 0], [0, 0], [9, 9]]), np.array([[0, 0], [0, 4.0], [9, 9]])]
+    assert math.isclose(orc.gate_distance(a, b, 2), 5.0)
+
+
+def test_multi_anchor_is_apply_at_stacked_rank():
+    rng = np.random.default_rng(6)
+    V, T, r, d = 3, 10, 4, 8
+    w = rng.random((V, T))
+    w /= w.sum(0, keepdims=True)
+    As = [rng.standard_normal((T, r)) for _ in range(V)]
+    Bs = [rng.standard_normal((r, d)) for _ in range(V)]
+    est = orc.multi_anchor_delta(w, As, Bs)
+    # scalar definition of Eq. 8 for one entry
+    t, c = 4, 5
+    ref = sum(w[v, t] * sum(As[v][t, q] * Bs[v][q, c] for q in range(r)) for v in range(V))
+    assert math.isclose(est[t, c], ref, rel_tol=1e-12)
+    cs, bs = orc.stack_anchors(w, As, Bs)
+    assert cs.shape == (T, V * r) and bs.shape == (V * r, d)
+    assert np.allclose(cs @ bs, est, atol=1e-12)
+    # a single anchor with weight one is the plain correction
+    assert np.allclose(orc.multi_anchor_delta(np.ones((1, T)), As[:1], Bs[:1]), As[0] @ Bs[0])
+
+
+# ---- bookkeeping --------------------------------------------------------------
+
+
+def test_memory_example_from_the_paper():
+    path = os.path.join(os.path.dirname(__file__), "golden", "memory_example.txt")
+    row = [ln for ln in open(path) if ln.strip() and not ln.startswith("#")][0].split()
+    L, Hkv, hd, bpe, tok, V, N = (int(x) for x in row[:7])
+    expect, tol = float(row[7]), float(row[8])
+    got = orc.full_state_bytes(V, N, tok, L, Hkv, hd, bpe) / 2.0 ** 30
+    assert abs(got - expect) <= tol
+    # the low-rank pool is O(V N r (L_seg + D)) per matrix
+    lr = orc.lowrank_state_bytes(V, N, tok, L, Hkv, hd, r=32)
+    per_matrix = 32 * (tok + hd) * 4
+    assert lr == V * (1 + N) * 2 * L * Hkv * per_matrix
