@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-correction hot path on B200.
+
+One *step* is one pass of the whole path over one synthetic request of the named
+workload: for every workflow edge a -> a+1 the rank-r state is built from the pair of
+true caches (kvc_state_update, FIT mode: deviation, Gram, eigensolve, projection), then
+the corrected caches of agents 1..N-1 are materialised from agent 0's exact cache
+(kvc_chain).  `value` is the algorithmic HBM bytes of those launches divided by the
+device time of the step (CUDA events), inputs resident in HBM; `e2e` is the same with
+the step's inputs copied from pinned host memory and the corrected caches copied back
+inside the timed region.  `roofline` is for the dominant kernel (one hop of the apply
+stream) against the measured HBM copy bandwidth of this machine.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+With --impl reference the fp64 CPU oracle is timed instead, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_34060_b200 import workloads as wl  # noqa: E402
+
+METRIC = "corrected-KV GB/s (algorithmic HBM bytes / time), whole hot path"
+UNIT = "GB/s"
+HBM_FALLBACK_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one apply launch, from the ncu capture
+# summarised under profiles/ (bytes per launch on the benchmark workload), or None.
+APPLY_TRAFFIC_BYTES = None
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def _dist():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# --------------------------------------------------------------------------------------
+# the library arm
+# --------------------------------------------------------------------------------------
+
+
+def build_workload(cfg: wl.Config, dev, kvc):
+    """Everything one step reads, resident on the device.  Draws come from the seeded
+    generator; the true target caches are derived with the library itself (aligned
+    source + exact rank-r deviation, then N(0, sigma) noise, rounded to bf16)."""
+    rope = kvc.Rope(cfg.theta)
+    pl = wl.prefix_lengths(cfg)
+    n = cfg.n_agents
+    if cfg.paged:
+        npg = wl.n_pages(cfg.T, cfg.page)
+        P = npg + 8
+        tables = [wl.page_table(npg, P, cfg.seed, a, dev) for a in range(2 * n)]
+        k0, v0 = wl.base_cache(cfg, dev, table=tables[0], n_phys=P)
+        mk = lambda t: kvc.Cache(torch.empty_like(k0), torch.empty_like(v0), T=cfg.T, page_table=t)
+        a0 = kvc.Cache(k0, v0, T=cfg.T, page_table=tables[0])
+    else:
+        k0, v0 = wl.base_cache(cfg, dev)
+        mk = lambda t: kvc.Cache(torch.empty_like(k0), torch.empty_like(v0))
+        tables = [None] * (2 * n)
+        a0 = kvc.Cache(k0, v0)
+    true = [a0]
+    for a in range(1, n):
+        s = wl.hop_state(cfg, a, dev)
+        st = kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"])
+        tgt = mk(tables[a])
+        kvc.kvc_apply(true[-1], st, pl[a] - pl[a - 1], rope, tgt)
+        for t, tag in ((tgt.k, 0), (tgt.v, 1)):      # noise below one bf16 step mostly dithers the rounding
+            flat = t.view(-1)
+            chunk = 1 << 26
+            g = torch.Generator(device=dev)
+            g.manual_seed(cfg.seed * 7919 + 2 * a + tag)
+            for o in range(0, flat.numel(), chunk):
+                seg = flat[o:o + chunk]
+                seg.copy_((seg.float() + cfg.sigma * torch.randn(seg.numel(), device=dev, generator=g)).to(torch.bfloat16))
+        true.append(tgt)
+        del s, st
+    torch.cuda.synchronize()
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+    states = [kvc.State(torch.empty(L, H, T, r, device=dev), torch.empty(L, H, T, r, device=dev),
+                        torch.empty(L, H, r, d, device=dev), torch.empty(L, H, r, d, device=dev)) for _ in range(n - 1)]
+    outs = [mk(tables[n + a]) for a in range(1, n)]
+    ws = torch.empty(max(kvc.kvc_workspace_bytes(a0, states[0], kvc.KVC_FIT), 256), dtype=torch.uint8, device=dev)
+    return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws}
+
+
+def run_step(W, kvc, ev=None):
+    """One pass of the path.  `ev` (optional) collects CUDA-event pairs per kernel family."""
+    pl, rope, n = W["pl"], W["rope"], len(W["true"])
+
+    def mark(name):
+        if ev is None:
+            return None
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        ev.setdefault(name, []).append(e)
+        return e
+
+    for a in range(1, n):
+        mark("update_begin")
+        kvc.kvc_state_update(W["true"][a - 1], W["true"][a], pl[a] - pl[a - 1], rope, W["states"][a - 1], kvc.KVC_FIT,
+                             workspace=W["ws"])
+        mark("update_end")
+    mark("chain_begin")
+    kvc.kvc_chain(W["true"][0], pl, W["states"], rope, W["outs"])
+    mark("chain_end")
+
+
+def step_bytes(W, kvc):
+    n = len(W["true"])
+    upd = sum(kvc.kvc_update_bytes(W["true"][a], W["states"][a - 1], kvc.KVC_FIT, True) for a in range(1, n))
+    app = sum(kvc.kvc_apply_bytes(W["true"][0], W["states"][a - 1]) for a in range(1, n))
+    return upd, app
+
+
+def cpu_baseline(cfg: wl.Config, budget_s: float = 20.0):
+    """The fp64 oracle, as it stands, on a bounded sample of the same workload: whole
+    (layer, head) slabs -- all tokens, all hops: FIT update then chain -- until the
+    time budget is used.  Returns the same metric (algorithmic bytes / wall time)."""
+    import numpy as np
+    from oracle import kvc_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    one = cfg.scaled(L=1, H=1, paged=False)
+    pl = wl.prefix_lengths(cfg)
+    f = orc.rope_inv_freq(cfg.d, cfg.theta)
+    bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    done, t_used, nbytes = 0, 0.0, 0
+    per_slab = None
+    while done < cfg.L * cfg.H and (per_slab is None or t_used + per_slab <= budget_s):
+        c = one.scaled(seed=cfg.seed + 1000 + done)
+        k0, v0 = wl.base_cache(c, "cpu")
+        true = [orc.Cache(bits(k0), bits(v0))]
+        for a in range(1, cfg.n_agents):                       # untimed: derive the true targets
+            s = wl.hop_state(c, a, "cpu")
+            st = orc.State(*(s[x].numpy() for x in ("coeff_k", "coeff_v", "basis_k", "basis_v")))
+            nk = wl.noise((1, 1, c.T, c.d), c.seed, 2 * a).numpy()
+            nv = wl.noise((1, 1, c.T, c.d), c.seed, 2 * a + 1).numpy()
+            true.append(orc.make_target(true[-1], st, pl[a] - pl[a - 1], f, nk, nv, c.sigma))
+        t0 = time.perf_counter()
+        states = []
+        for a in range(1, cfg.n_agents):
+            st, _ = orc.state_update(true[a - 1], true[a], pl[a] - pl[a - 1], f, r=cfg.r, mode=orc.FIT)
+            states.append(st)
+        orc.chain(true[0], pl, states, f)
+        dt = time.perf_counter() - t0
+        per_slab = dt if per_slab is None else max(per_slab, dt)
+        t_used += dt
+        done += 1
+        hops = cfg.n_agents - 1
+        tok = cfg.T
+        apply_b = hops * (tok * (8 * cfg.d + 8 * cfg.r) + 2 * cfg.r * cfg.d * 4)
+        upd_b = hops * (2 * tok * 8 * cfg.d + tok * 8 * cfg.r + 2 * cfg.r * cfg.d * 4 + 4 * cfg.d * cfg.d * 4)
+        nbytes += apply_b + upd_b
+    return {"value": nbytes / t_used / 1e9, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"{done} of {cfg.L * cfg.H} (layer, head) slabs, all {cfg.T} tokens, all {cfg.n_agents - 1} hops "
+                      f"(FIT update + chain), {t_used:.1f} s"}, t_used
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llama8b_8k", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="kvc", choices=["kvc", "reference"])
+    ap.add_argument("--path", default="auto", choices=["auto", "generic", "tc"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    rank, world, local = _dist()
+    cfg = wl.CONFIGS[args.workload]
+    config = {"workload": f"{cfg.name}: L={cfg.L} Hkv={cfg.H} d={cfg.d} T={cfg.T} agents={cfg.n_agents} r={cfg.r} "
+                          f"{'paged16' if cfg.paged else 'contiguous'} bf16, seed {cfg.seed}",
+              "step": "per edge: kvc_state_update(FIT) ; then kvc_chain over all agents",
+              "l2": "inputs larger than L2 (every pass streams > 1 GiB)", "parallelism": f"replicas x{world}"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, min(args.steps, 3))
+        vals = []
+        for _ in range(min(args.warmup, 1)):
+            cpu_baseline(cfg, 3.0)
+        t_all = 0.0
+        for _ in range(steps):
+            cb, t = cpu_baseline(cfg, max(2.0, 60.0 / steps))
+            vals.append(cb["value"])
+            t_all += t
+        v = sum(vals) / len(vals)
+        cb["value"] = v
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t_all / steps,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic", "config": config, "cpu_baseline": cb,
+                          "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import paper_2609_34060_b200 as kvc
+    from paper_2609_34060_b200 import build as kbuild
+    if not os.path.exists(kvc.LIB_PATH):
+        kbuild.build()
+    kvc.load()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    kvc.kvc_set_path({"auto": kvc.KVC_PATH_AUTO, "generic": kvc.KVC_PATH_GENERIC, "tc": kvc.KVC_PATH_TC}[args.path])
+
+    W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
+    upd_b, app_b = step_bytes(W, kvc)
+    hops = cfg.n_agents - 1
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        run_step(W, kvc)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = {}
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for _ in range(args.steps):
+        run_step(W, kvc, ev)
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t_begin.elapsed_time(t_end)
+    chain_ms = sum(b.elapsed_time(e) for b, e in zip(ev["chain_begin"], ev["chain_end"])) / args.steps
+    upd_ms = sum(b.elapsed_time(e) for b, e in zip(ev["update_begin"], ev["update_end"])) / args.steps
+    last_path = kvc.kvc_last_path()
+    assert kvc.kvc_status_poll() == 0, "a kernel flagged an anomaly"
+    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = world * (upd_b + app_b) / (ms_step * 1e-3) / 1e9
+
+    # end to end: inputs from pinned host memory, corrected caches back to the host
+    e2e = None
+    if not args.no_e2e:
+        srcs = [c for c in W["true"]]
+        host_in = [(c.k.cpu().pin_memory(), c.v.cpu().pin_memory()) for c in srcs]
+        host_out = [(torch.empty_like(o.k, device="cpu").pin_memory(), torch.empty_like(o.v, device="cpu").pin_memory())
+                    for o in W["outs"]]
+        h2d = sum(k.numel() * 2 + v.numel() * 2 for k, v in host_in)
+        d2h = sum(k.numel() * 2 + v.numel() * 2 for k, v in host_out)
+
+        def e2e_step():
+            for c, (hk, hv) in zip(srcs, host_in):
+                c.k.copy_(hk, non_blocking=True)
+                c.v.copy_(hv, non_blocking=True)
+            run_step(W, kvc)
+            for o, (hk, hv) in zip(W["outs"], host_out):
+                hk.copy_(o.k, non_blocking=True)
+                hv.copy_(o.v, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        b, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e.record()
+        barrier()
+        te = torch.tensor([b.elapsed_time(e)], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * (upd_b + app_b) / (float(te.item()) / n_e2e * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
+        del host_in, host_out
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = _peaks()
+    hop_ms = chain_ms / hops
+    achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                "traffic": APPLY_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": app_b // hops,
+                "us_per_launch": hop_ms * 1e3}
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic", "config": config,
+           "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * (hops * 3 + hops),
+           "roofline": roofline,
+           "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
+                         "us_per_agent_layer": hop_ms * 1e3 / cfg.L,
+                         "update_fit_GBs": upd_b / (upd_ms * 1e-3) / 1e9, "update_ms_per_step": upd_ms,
+                         "chain_ms_per_step": chain_ms,
+                         "kernel_family": {0: "auto", 1: "generic (CUDA cores)", 2: "tc (TMA + tcgen05)"}[last_path]}}
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"], _ = cpu_baseline(cfg, args.cpu_budget)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,229 @@
+/*
+ * kvc.h -- C ABI of the low-rank KV-cache correction library (B200 / sm_100a).
+ *
+ * The library turns one agent's shared-context KV cache into the next agent's
+ * cache without running the model: it re-aligns cached keys to their new
+ * positions (RoPE re-rotation), adds a stored rank-r correction
+ * coeff x basis per (layer, KV head), and chains agent to agent with the first
+ * agent's cache left exact.  It also builds that rank-r state from an observed
+ * pair of caches.
+ *
+ * Conventions for every entry point
+ *   - plain C types only; every pointer says whether it is HOST or DEVICE memory;
+ *   - all device work is enqueued on `stream` (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream); no entry point synchronises, and none
+ *     allocates device memory: every buffer, scratch included, is the caller's;
+ *   - the return value is KVC_OK (0) or a negative KVC_E_* code; nothing is
+ *     launched when an argument check fails;
+ *   - bf16 means the upper 16 bits of an IEEE float32, rounded to nearest-even
+ *     wherever the library produces one;
+ *   - the CUDA device that is current at the call is the one used.
+ */
+#ifndef KVC_H_
+#define KVC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------- */
+#define KVC_OK              0
+#define KVC_E_INVALID_ARG  (-1)  /* null pointer, negative size, bad enum          */
+#define KVC_E_SHAPE        (-2)  /* geometries of the arguments do not agree       */
+#define KVC_E_UNSUPPORTED  (-3)  /* valid but not built (head_dim, page size ...)  */
+#define KVC_E_ALIAS        (-4)  /* dst overlaps src without being the same cache  */
+#define KVC_E_CUDA         (-5)  /* a CUDA runtime / driver call failed            */
+#define KVC_E_WORKSPACE    (-6)  /* workspace missing, misaligned or too small     */
+#define KVC_E_DEVICE_FLAG  (-7)  /* a kernel recorded an anomaly (see status_poll) */
+
+/* ---- layouts, dtypes, modes --------------------------------------------- */
+#define KVC_CONTIG 0   /* k, v: bf16 [L, H, T, d]                                  */
+#define KVC_PAGED  1   /* k, v: bf16 pool [L, n_phys_pages, H, page_size, d]       */
+
+#define KVC_F32  0
+#define KVC_BF16 1
+
+#define KVC_ROPE_HALF        0   /* channel c pairs with c + d/2                   */
+#define KVC_ROPE_INTERLEAVED 1   /* channel 2c pairs with 2c + 1                   */
+
+#define KVC_PROJECT 0  /* bases given, compute coefficients                        */
+#define KVC_FIT     1  /* compute bases (truncated SVD), then coefficients         */
+
+#define KVC_PATH_AUTO    0  /* pick the fastest kernel that supports the arguments */
+#define KVC_PATH_GENERIC 1  /* CUDA-core kernels (any supported shape)             */
+#define KVC_PATH_TC      2  /* TMA + tcgen05 kernels (d = 128, r <= 64 ...)        */
+
+/*
+ * One agent's cache of the shared context (the paper's C_{i,seg}, Sec. 2.1 /
+ * Eq. 2, held per layer and per KV head).  Caller-owned DEVICE memory.
+ *
+ * KVC_CONTIG: element (l, h, t, c) at  l*s_layer + h*s_head + t*s_tok + c.
+ * KVC_PAGED : logical token t lives in physical page p = page_table[t / page_size]
+ *             at row t % page_size: element at
+ *             l*s_layer + p*s_page + h*s_head + (t % page_size)*s_tok + c.
+ *             One table serves all layers and heads (the serving engine's block
+ *             table).  The last page may be partial; rows >= T are never touched,
+ *             nor are physical pages the table does not name.
+ * Strides are in elements; 0 selects the dense default for the layout.
+ * Every row start must be 16-byte aligned (strides multiples of 8 elements).
+ */
+typedef struct kvc_cache {
+  void *k;                    /* DEVICE bf16                                       */
+  void *v;                    /* DEVICE bf16                                       */
+  int32_t layout;             /* KVC_CONTIG | KVC_PAGED                            */
+  int32_t L, H, T, d;         /* layers, KV heads, shared tokens, head dim         */
+  int32_t page_size;          /* KVC_PAGED: tokens per page (power of two, >= 8)   */
+  int32_t n_phys_pages;       /* KVC_PAGED: pages in the pool; bound for page ids  */
+  const int32_t *page_table;  /* DEVICE int32 [ceil(T / page_size)]                */
+  int64_t s_layer, s_page, s_head, s_tok;
+} kvc_cache;
+
+/*
+ * Rank-r state of one workflow edge (Eq. 7: Z ~= A_Z B_Z with A = U_r Sigma_r,
+ * B = R_r^T), one independent state per (layer, KV head), keys and values
+ * separately.  Caller-owned DEVICE memory.
+ *   coeff_*: float32 [L, H, n_cov, r]   (the paper's A)
+ *   basis_*: [L, H, r, d] in basis_dtype (the paper's B; rows orthonormal when fitted)
+ * n_cov is the covered prefix (App. A.3 "Variable Segment Lengths"): rows
+ * t >= n_cov of a cache receive the alignment only.  r == 0 or n_cov == 0 is
+ * the empty state (pointers may be NULL).
+ */
+typedef struct kvc_state {
+  float *coeff_k;
+  float *coeff_v;
+  void *basis_k;
+  void *basis_v;
+  int32_t r;
+  int32_t n_cov;
+  int32_t basis_dtype;        /* KVC_F32 | KVC_BF16                                */
+  int32_t reserved;
+} kvc_state;
+
+/*
+ * Rotary position embedding used for the key re-alignment that precedes every
+ * cross-agent reuse (Sec. 2.2; App. A.3).  A key cached at position p and
+ * reused at position p + s is rotated, pair by pair, by the angle s * f_k with
+ * f_k = theta^(-2k/d), k = 0..d/2-1, unless inv_freq overrides the table
+ * (scaled-RoPE models).  Values are never rotated.
+ */
+typedef struct kvc_rope {
+  double theta;
+  int32_t pairing;            /* KVC_ROPE_HALF | KVC_ROPE_INTERLEAVED              */
+  int32_t reserved;
+  const double *inv_freq;     /* HOST float64 [d/2] or NULL                        */
+} kvc_rope;
+
+/*
+ * kvc_apply -- one hop (Eq. 8 with a single anchor; Sec. 3.3):
+ *     K_dst[l,h,t,:] = bf16( Rot_shift(K_src[l,h,t,:]) + coeff_k[l,h,t,:] . basis_k[l,h] )
+ *     V_dst[l,h,t,:] = bf16(           V_src[l,h,t,:]  + coeff_v[l,h,t,:] . basis_v[l,h] )
+ * for t < n_cov; rows t >= n_cov (and every row of an empty state) keep the
+ * re-aligned source: V bit for bit, K bit for bit when shift == 0.
+ * Products and sums are accumulated in float32; one rounding to bf16.
+ *   src   HOST struct, DEVICE buffers, read only.
+ *   st    HOST struct, DEVICE buffers, read only.
+ *   shift target position minus source position of the shared context
+ *         (difference of the two agents' prefix lengths), any sign.
+ *   dst   HOST struct, DEVICE buffers, written.  Same L, H, T, d as src; layout,
+ *         strides and page table may differ.  dst may be the very same cache as src
+ *         (same pointers, strides and table: in place); any other overlap is
+ *         KVC_E_ALIAS when it can be detected from the pointers.
+ * Errors: KVC_E_INVALID_ARG, KVC_E_SHAPE, KVC_E_UNSUPPORTED (d not in {64,128},
+ * r > 256), KVC_E_ALIAS, KVC_E_CUDA.
+ */
+int kvc_apply(const kvc_cache *src, const kvc_state *st, int32_t shift, const kvc_rope *rope,
+              kvc_cache *dst, void *stream);
+
+/*
+ * kvc_chain -- corrections chained along the workflow (Sec. 3.2; App. A.3 "Cache
+ * Materialization"): agent 0's cache is exact and only read; for a = 1..n_agents-1
+ *     outs[a-1] = kvc_apply(a == 1 ? agent0 : outs[a-2], states[a-1],
+ *                           prefix_len[a] - prefix_len[a-1])
+ * Each materialised cache is rounded to bf16 before it becomes the next source.
+ *   prefix_len HOST int32 [n_agents]; states HOST array [n_agents-1]; outs HOST
+ *   array [n_agents-1] of caller-owned destination caches (distinct from one
+ *   another and from agent0).
+ */
+int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_len,
+              const kvc_state *states, const kvc_rope *rope, kvc_cache *outs, void *stream);
+
+/*
+ * kvc_state_update -- build the rank-r state of the edge src -> tgt (Eq. 12 then
+ * Eq. 7), for every (layer, KV head), keys and values:
+ *     Delta_K = K_tgt - Rot_shift(K_src),  Delta_V = V_tgt - V_src   (rows t < st->n_cov)
+ *   KVC_PROJECT: st->basis_* are inputs; coeff = Delta . basis^T is written (float32).
+ *   KVC_FIT    : G = Delta^T Delta (d x d), its top-r eigenvectors become the rows
+ *                of st->basis_* (float32; right singular vectors of Delta, largest
+ *                singular values first, each row's largest-magnitude entry made
+ *                positive; rows beyond min(r, d, n_cov) are zero), then coeff as above
+ *                (= U_r Sigma_r).  st->basis_dtype must be KVC_F32.
+ *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
+ *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte
+ *              aligned; contents undefined afterwards.  May be NULL when 0 is needed.
+ * Errors as kvc_apply, plus KVC_E_WORKSPACE.
+ */
+int kvc_state_update(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,
+                     kvc_state *st, int32_t mode, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Scratch kvc_state_update needs for this geometry and mode (0 for KVC_PROJECT). */
+size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mode);
+
+/*
+ * kvc_apply_batch -- many independent hops in ONE launch (concurrent serving: each
+ * item is one request's next hop, with its own length, rank, shift and tables).
+ * The computation per item is exactly kvc_apply's.
+ *   items      HOST array [n_items]; every item's caches must share d.
+ *   workspace  DEVICE scratch >= kvc_batch_workspace_bytes(n_items), 256-byte aligned;
+ *              receives the launch's work table and must stay untouched until the
+ *              launch has finished.
+ *   staging    HOST buffer of the same size (pinned memory recommended); the work
+ *              table is built here and copied to `workspace` on `stream`; it must stay
+ *              untouched until that copy has executed.
+ */
+typedef struct kvc_item {
+  kvc_cache src;
+  kvc_cache dst;
+  kvc_state st;
+  int32_t shift;
+  int32_t reserved;
+} kvc_item;
+
+int kvc_apply_batch(const kvc_item *items, int32_t n_items, const kvc_rope *rope,
+                    void *workspace, size_t workspace_bytes, void *staging, void *stream);
+size_t kvc_batch_workspace_bytes(int32_t n_items);
+
+/*
+ * Device-side anomalies never trap or hang: a kernel that meets a page id outside
+ * [0, n_phys_pages) or whose bounded wait on an asynchronous copy runs out skips
+ * that tile and ORs a bit into a per-device status word.
+ * kvc_status_poll copies the word to *flags (this call synchronises the device)
+ * and returns KVC_OK when it is zero, KVC_E_DEVICE_FLAG otherwise;
+ * kvc_status_reset clears it.
+ */
+#define KVC_FLAG_BAD_PAGE     1u
+#define KVC_FLAG_WAIT_EXPIRED 2u
+#define KVC_FLAG_NOT_CONVERGED 4u   /* eigensolver hit its sweep limit             */
+int kvc_status_poll(uint32_t *flags);
+int kvc_status_reset(void);
+
+/* Force a kernel family (testing / benchmarking); KVC_PATH_TC returns
+ * KVC_E_UNSUPPORTED from later calls whose arguments it cannot serve. */
+int kvc_set_path(int32_t path);
+/* Which family the last successful launch on this thread used (KVC_PATH_*). */
+int kvc_last_path(void);
+
+/* Algorithmic HBM bytes one hop moves (reads + writes of caches, coefficients and
+ * bases), the figure the roofline is reported against. */
+int64_t kvc_apply_bytes(const kvc_cache *src, const kvc_state *st);
+int64_t kvc_update_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mode, int32_t has_src);
+
+const char *kvc_strerror(int code);
+const char *kvc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVC_H_ */

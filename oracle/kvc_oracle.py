@@ -262,6 +262,21 @@ def chain(agent0, prefix_len, states, inv_freq, dst_tables=None, pairing=ROPE_HA
     return (outs, refs) if want_ref else outs
 
 
+def make_target(src, st, s, inv_freq, noise_k, noise_v, sigma, dst=None, pairing=ROPE_HALF):
+    """The true cache of the next agent in the synthetic workloads: the re-aligned source
+    plus an exactly rank-r deviation plus Gaussian noise, rounded once to bf16:
+        C_j = bf16(Align_s(C_i) + A B + sigma * noise).
+    noise_* are standard-normal draws [L,H,T,d] handed in by the input generator."""
+    dst = src.empty_like() if dst is None else dst
+    for l in range(src.L):
+        for h in range(src.H):
+            for which, cf, bs, nz in (("k", st.coeff_k, st.basis_k, noise_k), ("v", st.coeff_v, st.basis_v, noise_v)):
+                ref, _ = apply_slab(src.get_bits(which, l, h), cf[l, h], bs[l, h], s, inv_freq, st.n_cov,
+                                    which == "k", pairing)
+                dst.put_bits(which, l, h, f64_to_bf16_bits(ref + sigma * np.asarray(nz[l, h], np.float64)))
+    return dst
+
+
 def chain_unrounded_slab(x0, prefix_len, coeffs, bases, inv_freq, is_key, pairing=ROPE_HALF):
     """The same recursion carried in float64 with no intermediate rounding.
 

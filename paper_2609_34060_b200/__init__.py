@@ -1,0 +1,294 @@
+"""Python binding of the KV-correction CUDA library (``libkvc.so``).
+
+Argument marshalling only: torch tensors supply device memory and the stream,
+every step of the path runs in the library's kernels.  The functions carry the
+C ABI's names (``include/kvc.h``) and raise :class:`KvcError` on a non-zero
+status.  There is no CPU fallback: if the shared object is missing or cannot
+be loaded, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvc.so")
+
+KVC_CONTIG, KVC_PAGED = 0, 1
+KVC_F32, KVC_BF16 = 0, 1
+KVC_ROPE_HALF, KVC_ROPE_INTERLEAVED = 0, 1
+KVC_PROJECT, KVC_FIT = 0, 1
+KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
+KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4
+
+EXPORTS = (
+    "kvc_apply", "kvc_chain", "kvc_state_update", "kvc_workspace_bytes", "kvc_apply_batch",
+    "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
+    "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version",
+)
+
+
+class KvcError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+class kvc_cache(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("layout", C.c_int32), ("L", C.c_int32), ("H", C.c_int32),
+                ("T", C.c_int32), ("d", C.c_int32), ("page_size", C.c_int32), ("n_phys_pages", C.c_int32),
+                ("page_table", C.c_void_p), ("s_layer", C.c_int64), ("s_page", C.c_int64), ("s_head", C.c_int64),
+                ("s_tok", C.c_int64)]
+
+
+class kvc_state(C.Structure):
+    _fields_ = [("coeff_k", C.c_void_p), ("coeff_v", C.c_void_p), ("basis_k", C.c_void_p), ("basis_v", C.c_void_p),
+                ("r", C.c_int32), ("n_cov", C.c_int32), ("basis_dtype", C.c_int32), ("reserved", C.c_int32)]
+
+
+class kvc_rope(C.Structure):
+    _fields_ = [("theta", C.c_double), ("pairing", C.c_int32), ("reserved", C.c_int32), ("inv_freq", C.c_void_p)]
+
+
+class kvc_item(C.Structure):
+    _fields_ = [("src", kvc_cache), ("dst", kvc_cache), ("st", kvc_state), ("shift", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
+_lib = None
+
+
+def load(path: Optional[str] = None):
+    """Load the shared library (once).  Raises if it is not there: no fallback."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(f"{p} not found: build it with `python -m paper_2609_34060_b200.build`")
+    lib = C.CDLL(p)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    PC, PS, PR, PI = C.POINTER(kvc_cache), C.POINTER(kvc_state), C.POINTER(kvc_rope), C.POINTER(kvc_item)
+    lib.kvc_apply.argtypes = [PC, PS, i32, PR, PC, vp]
+    lib.kvc_chain.argtypes = [PC, i32, C.POINTER(i32), PS, PR, PC, vp]
+    lib.kvc_state_update.argtypes = [PC, PC, i32, PR, PS, i32, vp, sz, vp]
+    lib.kvc_workspace_bytes.argtypes = [PC, PS, i32]
+    lib.kvc_workspace_bytes.restype = sz
+    lib.kvc_apply_batch.argtypes = [PI, i32, PR, vp, sz, vp, vp]
+    lib.kvc_batch_workspace_bytes.argtypes = [i32]
+    lib.kvc_batch_workspace_bytes.restype = sz
+    lib.kvc_status_poll.argtypes = [C.POINTER(C.c_uint32)]
+    lib.kvc_status_reset.argtypes = []
+    lib.kvc_set_path.argtypes = [i32]
+    lib.kvc_last_path.argtypes = []
+    lib.kvc_apply_bytes.argtypes = [PC, PS]
+    lib.kvc_apply_bytes.restype = i64
+    lib.kvc_update_bytes.argtypes = [PC, PS, i32, i32]
+    lib.kvc_update_bytes.restype = i64
+    lib.kvc_strerror.argtypes = [C.c_int]
+    lib.kvc_strerror.restype = C.c_char_p
+    lib.kvc_version.argtypes = []
+    lib.kvc_version.restype = C.c_char_p
+    for name in ("kvc_apply", "kvc_chain", "kvc_state_update", "kvc_apply_batch", "kvc_status_poll",
+                 "kvc_status_reset", "kvc_set_path", "kvc_last_path"):
+        getattr(lib, name).restype = C.c_int
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().kvc_strerror(code).decode()
+
+
+def version() -> str:
+    return load().kvc_version().decode()
+
+
+# ---- descriptors over torch tensors ------------------------------------------------
+
+
+class Cache:
+    """A cache descriptor over torch tensors (which it keeps alive).
+
+    contiguous: ``k``, ``v`` bf16 [L, H, T, d].
+    paged:      ``k``, ``v`` bf16 pools [L, P, H, page, d], ``page_table`` int32
+                [ceil(T/page)], ``T`` the logical length.
+    """
+
+    def __init__(self, k: torch.Tensor, v: torch.Tensor, T: Optional[int] = None,
+                 page_table: Optional[torch.Tensor] = None):
+        assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16
+        assert k.is_contiguous() and v.is_contiguous() and k.shape == v.shape
+        self.k, self.v, self.page_table = k, v, page_table
+        if page_table is None:
+            self.L, self.H, self.T, self.d = (int(x) for x in k.shape)
+            self.page, self.P = 0, 0
+        else:
+            assert page_table.dtype == torch.int32 and page_table.is_contiguous() and T is not None
+            self.L, self.P, self.H, self.page, self.d = (int(x) for x in k.shape)
+            self.T = int(T)
+
+    def struct(self) -> kvc_cache:
+        s = kvc_cache()
+        s.k, s.v = self.k.data_ptr(), self.v.data_ptr()
+        s.L, s.H, s.T, s.d = self.L, self.H, self.T, self.d
+        if self.page_table is None:
+            s.layout = KVC_CONTIG
+        else:
+            s.layout = KVC_PAGED
+            s.page_size, s.n_phys_pages = self.page, self.P
+            s.page_table = self.page_table.data_ptr()
+        return s
+
+    def empty_like(self, page_table: Optional[torch.Tensor] = None, fill: Optional[float] = None) -> "Cache":
+        mk = (lambda t: torch.empty_like(t)) if fill is None else (lambda t: torch.full_like(t, fill))
+        if self.page_table is None:
+            return Cache(mk(self.k), mk(self.v))
+        return Cache(mk(self.k), mk(self.v), T=self.T,
+                     page_table=self.page_table if page_table is None else page_table)
+
+    def nbytes(self) -> int:
+        return self.k.numel() * 2 + self.v.numel() * 2
+
+
+class State:
+    """Rank-r state over torch tensors: coeff fp32 [L,H,n_cov,r], basis fp32|bf16 [L,H,r,d]."""
+
+    def __init__(self, coeff_k, coeff_v, basis_k, basis_v, n_cov: Optional[int] = None):
+        self.coeff_k, self.coeff_v, self.basis_k, self.basis_v = coeff_k, coeff_v, basis_k, basis_v
+        self.r = 0 if basis_k is None else int(basis_k.shape[2])
+        self.n_cov = (0 if coeff_k is None else int(coeff_k.shape[2])) if n_cov is None else int(n_cov)
+        if self.r > 0:
+            assert basis_k.is_contiguous() and basis_v.is_contiguous() and basis_k.dtype == basis_v.dtype
+            assert basis_k.dtype in (torch.float32, torch.bfloat16)
+        if self.r > 0 and self.n_cov > 0:
+            assert coeff_k.dtype == torch.float32 and coeff_v.dtype == torch.float32
+            assert coeff_k.is_contiguous() and coeff_v.is_contiguous()
+            assert int(coeff_k.shape[2]) == self.n_cov and int(coeff_k.shape[3]) == self.r
+
+    @staticmethod
+    def empty() -> "State":
+        return State(None, None, None, None, n_cov=0)
+
+    def struct(self) -> kvc_state:
+        s = kvc_state()
+        ptr = lambda t: 0 if t is None else t.data_ptr()
+        s.coeff_k, s.coeff_v, s.basis_k, s.basis_v = ptr(self.coeff_k), ptr(self.coeff_v), ptr(self.basis_k), ptr(self.basis_v)
+        s.r, s.n_cov = self.r, self.n_cov
+        s.basis_dtype = KVC_BF16 if (self.basis_k is not None and self.basis_k.dtype == torch.bfloat16) else KVC_F32
+        return s
+
+
+class Rope:
+    def __init__(self, theta: float = 10000.0, pairing: int = KVC_ROPE_HALF, inv_freq: Optional[Sequence[float]] = None):
+        self.theta, self.pairing = float(theta), int(pairing)
+        self._tab = None if inv_freq is None else (C.c_double * len(inv_freq))(*[float(x) for x in inv_freq])
+
+    def struct(self) -> kvc_rope:
+        s = kvc_rope()
+        s.theta, s.pairing = self.theta, self.pairing
+        s.inv_freq = None if self._tab is None else C.cast(self._tab, C.c_void_p)
+        return s
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise KvcError(code, what)
+
+
+# ---- the C ABI, same names ---------------------------------------------------------
+
+
+def kvc_apply(src: Cache, st: State, shift: int, rope: Rope, dst: Cache, stream=None) -> None:
+    s, d, t, r = src.struct(), dst.struct(), st.struct(), rope.struct()
+    _check(load().kvc_apply(C.byref(s), C.byref(t), int(shift), C.byref(r), C.byref(d), _stream(stream)), "kvc_apply")
+
+
+def kvc_chain(agent0: Cache, prefix_len: Sequence[int], states: Sequence[State], rope: Rope, outs: Sequence[Cache],
+              stream=None) -> None:
+    n = len(prefix_len)
+    a0, r = agent0.struct(), rope.struct()
+    pl = (C.c_int32 * n)(*[int(x) for x in prefix_len])
+    sts = (kvc_state * max(n - 1, 1))(*[s.struct() for s in states])
+    os_ = (kvc_cache * max(n - 1, 1))(*[o.struct() for o in outs])
+    _check(load().kvc_chain(C.byref(a0), n, pl, sts, C.byref(r), os_, _stream(stream)), "kvc_chain")
+
+
+def kvc_workspace_bytes(tgt: Cache, st: State, mode: int) -> int:
+    t, s = tgt.struct(), st.struct()
+    return int(load().kvc_workspace_bytes(C.byref(t), C.byref(s), int(mode)))
+
+
+def kvc_state_update(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, st: State, mode: int,
+                     workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    t, s, r = tgt.struct(), st.struct(), rope.struct()
+    sp = None
+    if src is not None:
+        ss = src.struct()
+        sp = C.byref(ss)
+    ws_ptr = 0 if workspace is None else workspace.data_ptr()
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().kvc_state_update(sp, C.byref(t), int(shift), C.byref(r), C.byref(s), int(mode), ws_ptr, ws_bytes,
+                                   _stream(stream)), "kvc_state_update")
+
+
+class Item:
+    def __init__(self, src: Cache, dst: Cache, st: State, shift: int):
+        self.src, self.dst, self.st, self.shift = src, dst, st, int(shift)
+
+
+def kvc_batch_workspace_bytes(n_items: int) -> int:
+    return int(load().kvc_batch_workspace_bytes(int(n_items)))
+
+
+def kvc_apply_batch(items: Sequence[Item], rope: Rope, workspace: torch.Tensor, staging: torch.Tensor,
+                    stream=None) -> None:
+    n = len(items)
+    arr = (kvc_item * max(n, 1))()
+    for i, it in enumerate(items):
+        arr[i].src, arr[i].dst, arr[i].st, arr[i].shift = it.src.struct(), it.dst.struct(), it.st.struct(), it.shift
+    r = rope.struct()
+    assert staging.device.type == "cpu" and staging.numel() * staging.element_size() >= kvc_batch_workspace_bytes(n)
+    _check(load().kvc_apply_batch(arr, n, C.byref(r), workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), staging.data_ptr(), _stream(stream)),
+           "kvc_apply_batch")
+
+
+def kvc_status_poll() -> int:
+    w = C.c_uint32(0)
+    rc = load().kvc_status_poll(C.byref(w))
+    if rc not in (0, -7):
+        raise KvcError(rc, "kvc_status_poll")
+    return int(w.value)
+
+
+def kvc_status_reset() -> None:
+    _check(load().kvc_status_reset(), "kvc_status_reset")
+
+
+def kvc_set_path(path: int) -> None:
+    _check(load().kvc_set_path(int(path)), "kvc_set_path")
+
+
+def kvc_last_path() -> int:
+    return int(load().kvc_last_path())
+
+
+def kvc_apply_bytes(src: Cache, st: State) -> int:
+    s, t = src.struct(), st.struct()
+    return int(load().kvc_apply_bytes(C.byref(s), C.byref(t)))
+
+
+def kvc_update_bytes(tgt: Cache, st: State, mode: int, has_src: bool = True) -> int:
+    s, t = tgt.struct(), st.struct()
+    return int(load().kvc_update_bytes(C.byref(s), C.byref(t), int(mode), int(bool(has_src))))

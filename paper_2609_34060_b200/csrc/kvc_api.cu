@@ -1,0 +1,459 @@
+// C ABI: argument checks, descriptor resolution, kernel-family dispatch.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/kvc.h"
+#include "kvc_dev.cuh"
+#include "kvc_launch.h"
+#include "kvc_tc.h"
+
+namespace kvc {
+
+__device__ uint32_t g_status_word;
+
+static thread_local int tl_path_force = KVC_PATH_AUTO;
+static thread_local int tl_last_path = KVC_PATH_AUTO;
+
+static uint32_t* status_ptr() {
+  uint32_t* p = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
+  return p;
+}
+
+static int ilog2_exact(int x) {
+  if (x <= 0 || (x & (x - 1))) return -1;
+  int s = 0;
+  while ((1 << s) < x) ++s;
+  return s;
+}
+
+// Validate one cache descriptor and resolve it for the kernels.
+static int resolve_cache(const kvc_cache* c, DevCache* out) {
+  if (!c || !c->k || !c->v) return KVC_E_INVALID_ARG;
+  if (c->L <= 0 || c->H <= 0 || c->T < 0 || c->d <= 0) return KVC_E_INVALID_ARG;
+  if (c->d != 64 && c->d != 128) return KVC_E_UNSUPPORTED;
+  if (c->layout != KVC_CONTIG && c->layout != KVC_PAGED) return KVC_E_INVALID_ARG;
+  if (c->s_layer < 0 || c->s_page < 0 || c->s_head < 0 || c->s_tok < 0) return KVC_E_INVALID_ARG;
+  DevCache d;
+  memset(&d, 0, sizeof(d));
+  d.k = reinterpret_cast<__nv_bfloat16*>(c->k);
+  d.v = reinterpret_cast<__nv_bfloat16*>(c->v);
+  d.T = c->T;
+  d.s_tok = c->s_tok ? c->s_tok : c->d;
+  if (c->layout == KVC_CONTIG) {
+    d.page_table = nullptr;
+    d.s_head = c->s_head ? c->s_head : (int64_t)c->T * d.s_tok;
+    d.s_layer = c->s_layer ? c->s_layer : (int64_t)c->H * d.s_head;
+    d.s_page = 0;
+  } else {
+    const int sh = ilog2_exact(c->page_size);
+    if (sh < 3) return c->page_size > 0 ? KVC_E_UNSUPPORTED : KVC_E_INVALID_ARG;
+    if (c->n_phys_pages <= 0) return KVC_E_INVALID_ARG;
+    if (!c->page_table && c->T > 0) return KVC_E_INVALID_ARG;
+    d.page_table = c->page_table;
+    d.page_shift = sh;
+    d.page_mask = c->page_size - 1;
+    d.n_phys = c->n_phys_pages;
+    d.s_head = c->s_head ? c->s_head : (int64_t)c->page_size * d.s_tok;
+    d.s_page = c->s_page ? c->s_page : (int64_t)c->H * d.s_head;
+    d.s_layer = c->s_layer ? c->s_layer : (int64_t)c->n_phys_pages * d.s_page;
+  }
+  if ((d.s_tok | d.s_head | d.s_layer | d.s_page) & 7) return KVC_E_UNSUPPORTED;  // 16-byte rows
+  if ((reinterpret_cast<uintptr_t>(c->k) | reinterpret_cast<uintptr_t>(c->v)) & 15) return KVC_E_UNSUPPORTED;
+  *out = d;
+  return KVC_OK;
+}
+
+static int resolve_state(const kvc_state* st, int for_update, DevState* out) {
+  if (!st) return KVC_E_INVALID_ARG;
+  if (st->r < 0 || st->n_cov < 0) return KVC_E_INVALID_ARG;
+  if (st->r > 256) return KVC_E_UNSUPPORTED;
+  if (st->basis_dtype != KVC_F32 && st->basis_dtype != KVC_BF16) return KVC_E_INVALID_ARG;
+  const bool live = st->r > 0 && st->n_cov > 0;
+  if (live || (for_update && st->r > 0)) {
+    if (!st->basis_k || !st->basis_v) return KVC_E_INVALID_ARG;
+    if (live && (!st->coeff_k || !st->coeff_v)) return KVC_E_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(st->coeff_k) | reinterpret_cast<uintptr_t>(st->coeff_v) |
+         reinterpret_cast<uintptr_t>(st->basis_k) | reinterpret_cast<uintptr_t>(st->basis_v)) & 15)
+      return KVC_E_UNSUPPORTED;
+  }
+  DevState d;
+  d.coeff_k = st->coeff_k;
+  d.coeff_v = st->coeff_v;
+  d.basis_k = st->basis_k;
+  d.basis_v = st->basis_v;
+  d.r = st->r;
+  d.n_cov = st->n_cov;
+  d.basis_bf16 = st->basis_dtype == KVC_BF16;
+  d.pad = 0;
+  *out = d;
+  return KVC_OK;
+}
+
+static int check_rope(const kvc_rope* rope) {
+  if (!rope) return KVC_E_INVALID_ARG;
+  if (rope->pairing != KVC_ROPE_HALF && rope->pairing != KVC_ROPE_INTERLEAVED) return KVC_E_INVALID_ARG;
+  if (!rope->inv_freq && !(rope->theta > 0.0)) return KVC_E_INVALID_ARG;
+  return KVC_OK;
+}
+
+// cos / sin of shift * f_k in float64, rounded once to float32.
+static void rope_tables(const kvc_rope* rope, int d, int shift, float* cs, float* sn) {
+  for (int k = 0; k < kMaxHalfD; ++k) {
+    cs[k] = 1.f;
+    sn[k] = 0.f;
+  }
+  if (shift == 0) return;
+  for (int k = 0; k < d / 2; ++k) {
+    const double f = rope->inv_freq ? rope->inv_freq[k] : pow(rope->theta, -2.0 * (double)k / (double)d);
+    const double a = (double)shift * f;
+    cs[k] = (float)cos(a);
+    sn[k] = (float)sin(a);
+  }
+}
+
+// Byte extent a cache can touch, for the alias check.
+static void cache_extent(const kvc_cache* c, const DevCache& d, const void* base, uintptr_t* lo, uintptr_t* hi) {
+  int64_t last = (int64_t)(c->L - 1) * d.s_layer + (int64_t)(c->H - 1) * d.s_head + c->d;
+  if (c->layout == KVC_CONTIG)
+    last += (int64_t)(c->T > 0 ? c->T - 1 : 0) * d.s_tok;
+  else
+    last += (int64_t)(c->n_phys_pages - 1) * d.s_page + (int64_t)(c->page_size - 1) * d.s_tok;
+  *lo = reinterpret_cast<uintptr_t>(base);
+  *hi = *lo + (uintptr_t)last * 2;
+}
+
+static bool overlaps(uintptr_t a0, uintptr_t a1, uintptr_t b0, uintptr_t b1) { return a0 < b1 && b0 < a1; }
+
+static bool same_cache(const kvc_cache* a, const DevCache& da, const kvc_cache* b, const DevCache& db) {
+  return a->k == b->k && a->v == b->v && a->layout == b->layout && da.s_layer == db.s_layer &&
+         da.s_page == db.s_page && da.s_head == db.s_head && da.s_tok == db.s_tok && a->page_table == b->page_table;
+}
+
+// Contiguous caches: any overlap other than "the very same cache" is an error.  Paged
+// caches may legitimately share one pool (disjoint pages), which pointers cannot prove,
+// so only K-vs-V cross overlap is rejected there.
+static int alias_check(const kvc_cache* src, const DevCache& ds, const kvc_cache* dst, const DevCache& dd) {
+  if (same_cache(src, ds, dst, dd)) return KVC_OK;
+  uintptr_t sk0, sk1, sv0, sv1, dk0, dk1, dv0, dv1;
+  cache_extent(src, ds, src->k, &sk0, &sk1);
+  cache_extent(src, ds, src->v, &sv0, &sv1);
+  cache_extent(dst, dd, dst->k, &dk0, &dk1);
+  cache_extent(dst, dd, dst->v, &dv0, &dv1);
+  if (overlaps(dk0, dk1, dv0, dv1)) return KVC_E_ALIAS;
+  if (overlaps(sk0, sk1, dv0, dv1) || overlaps(sv0, sv1, dk0, dk1)) return KVC_E_ALIAS;
+  const bool both_paged = src->layout == KVC_PAGED && dst->layout == KVC_PAGED;
+  if (!both_paged && (overlaps(sk0, sk1, dk0, dk1) || overlaps(sv0, sv1, dv0, dv1))) return KVC_E_ALIAS;
+  return KVC_OK;
+}
+
+struct ResolvedHop {
+  DevItem item;
+  int d;
+};
+
+static int resolve_hop(const kvc_cache* src, const kvc_state* st, int32_t shift, const kvc_rope* rope,
+                       const kvc_cache* dst, ResolvedHop* out) {
+  int rc;
+  memset(&out->item, 0, sizeof(DevItem));
+  if ((rc = check_rope(rope)) != KVC_OK) return rc;
+  if ((rc = resolve_cache(src, &out->item.src)) != KVC_OK) return rc;
+  if ((rc = resolve_cache(dst, &out->item.dst)) != KVC_OK) return rc;
+  if ((rc = resolve_state(st, 0, &out->item.st)) != KVC_OK) return rc;
+  if (src->L != dst->L || src->H != dst->H || src->T != dst->T || src->d != dst->d) return KVC_E_SHAPE;
+  if (st->r > 0 && st->n_cov > src->T) return KVC_E_SHAPE;
+  if ((rc = alias_check(src, out->item.src, dst, out->item.dst)) != KVC_OK) return rc;
+  out->item.shift = shift;
+  out->item.L = src->L;
+  out->item.H = src->H;
+  out->d = src->d;
+  rope_tables(rope, src->d, shift, out->item.cs, out->item.sn);
+  return KVC_OK;
+}
+
+static int apply_resolved(ResolvedHop& hop, int pairing, cudaStream_t s) {
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  const int T = hop.item.src.T;
+  if (T == 0) return KVC_OK;
+  const bool want_tc = tl_path_force != KVC_PATH_GENERIC;
+  if (want_tc) {
+    const int trc = tc_apply_single(hop.item, hop.d, pairing, status, s);
+    if (trc == KVC_OK) {
+      tl_last_path = KVC_PATH_TC;
+      return KVC_OK;
+    }
+    if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  }
+  ApplyLaunch L;
+  memset(&L, 0, sizeof(L));
+  const int tile = generic_apply_tile(hop.d);
+  hop.item.tiles_per_slab = (T + tile - 1) / tile;
+  L.items = nullptr;
+  L.tile_prefix = nullptr;
+  L.n_items = 1;
+  L.pairing = pairing;
+  L.total_tiles = (int64_t)hop.item.L * hop.item.H * 2 * hop.item.tiles_per_slab;
+  L.status = status;
+  L.one = hop.item;
+  if (launch_apply_generic(L, hop.d, s) != cudaSuccess) return KVC_E_CUDA;
+  tl_last_path = KVC_PATH_GENERIC;
+  return KVC_OK;
+}
+
+}  // namespace kvc
+
+using namespace kvc;
+
+extern "C" {
+
+int kvc_apply(const kvc_cache* src, const kvc_state* st, int32_t shift, const kvc_rope* rope, kvc_cache* dst,
+              void* stream) {
+  ResolvedHop hop;
+  const int rc = resolve_hop(src, st, shift, rope, dst, &hop);
+  if (rc != KVC_OK) return rc;
+  return apply_resolved(hop, rope->pairing, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int kvc_chain(const kvc_cache* agent0, int32_t n_agents, const int32_t* prefix_len, const kvc_state* states,
+              const kvc_rope* rope, kvc_cache* outs, void* stream) {
+  if (!agent0 || n_agents < 1 || !prefix_len) return KVC_E_INVALID_ARG;
+  if (n_agents == 1) return KVC_OK;
+  if (!states || !outs) return KVC_E_INVALID_ARG;
+  // validate the whole chain before the first launch
+  for (int a = 1; a < n_agents; ++a) {
+    ResolvedHop hop;
+    const kvc_cache* src = (a == 1) ? agent0 : &outs[a - 2];
+    const int rc = resolve_hop(src, &states[a - 1], prefix_len[a] - prefix_len[a - 1], rope, &outs[a - 1], &hop);
+    if (rc != KVC_OK) return rc;
+    // the first agent's cache is exact and must never be a destination; outputs are distinct
+    if (outs[a - 1].k == agent0->k || outs[a - 1].v == agent0->v) return KVC_E_ALIAS;
+    for (int b = 1; b < a; ++b)
+      if (outs[b - 1].k == outs[a - 1].k && outs[b - 1].page_table == outs[a - 1].page_table) return KVC_E_ALIAS;
+  }
+  for (int a = 1; a < n_agents; ++a) {
+    ResolvedHop hop;
+    const kvc_cache* src = (a == 1) ? agent0 : &outs[a - 2];
+    int rc = resolve_hop(src, &states[a - 1], prefix_len[a] - prefix_len[a - 1], rope, &outs[a - 1], &hop);
+    if (rc == KVC_OK) rc = apply_resolved(hop, rope->pairing, reinterpret_cast<cudaStream_t>(stream));
+    if (rc != KVC_OK) return rc;
+  }
+  return KVC_OK;
+}
+
+size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
+  if (!tgt || !st || mode != KVC_FIT) return 0;
+  const size_t m = (size_t)tgt->L * tgt->H * 2;
+  return m * tgt->d * tgt->d * sizeof(float) + m * tgt->d * sizeof(float);
+}
+
+int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
+                     int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
+  if (mode != KVC_PROJECT && mode != KVC_FIT) return KVC_E_INVALID_ARG;
+  int rc;
+  if ((rc = check_rope(rope)) != KVC_OK) return rc;
+  DevCache dt, ds;
+  memset(&ds, 0, sizeof(ds));
+  if ((rc = resolve_cache(tgt, &dt)) != KVC_OK) return rc;
+  if (src) {
+    if ((rc = resolve_cache(src, &ds)) != KVC_OK) return rc;
+    if (src->L != tgt->L || src->H != tgt->H || src->T != tgt->T || src->d != tgt->d) return KVC_E_SHAPE;
+  }
+  DevState dst_state;
+  if ((rc = resolve_state(st, 1, &dst_state)) != KVC_OK) return rc;
+  if (st->n_cov > tgt->T) return KVC_E_SHAPE;
+  if (st->r == 0 || st->n_cov == 0) return KVC_OK;   // nothing to compute
+  if (!st->coeff_k || !st->coeff_v) return KVC_E_INVALID_ARG;
+  if (mode == KVC_FIT && st->basis_dtype != KVC_F32) return KVC_E_UNSUPPORTED;
+  if (mode == KVC_FIT) {
+    const size_t need = kvc_workspace_bytes(tgt, st, mode);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_E_WORKSPACE;
+  }
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const int d = tgt->d;
+
+  if (mode == KVC_FIT) {
+    FitLaunch F;
+    memset(&F, 0, sizeof(F));
+    F.src = ds;
+    F.tgt = dt;
+    F.gram = reinterpret_cast<float*>(workspace);
+    F.evals = F.gram + (size_t)tgt->L * tgt->H * 2 * d * d;
+    F.basis_k = reinterpret_cast<float*>(st->basis_k);
+    F.basis_v = reinterpret_cast<float*>(st->basis_v);
+    F.r = st->r;
+    F.n_cov = st->n_cov;
+    F.pairing = rope->pairing;
+    F.shift = shift;
+    F.L = tgt->L;
+    F.H = tgt->H;
+    F.status = status;
+    rope_tables(rope, d, shift, F.cs, F.sn);
+    bool gram_done = false;
+    if (tl_path_force != KVC_PATH_GENERIC) {
+      const int trc = tc_gram(F, d, s);
+      if (trc == KVC_OK) gram_done = true;
+      else if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+    }
+    if (!gram_done && launch_gram_generic(F, d, s) != cudaSuccess) return KVC_E_CUDA;
+    if (launch_eig(F, d, s) != cudaSuccess) return KVC_E_CUDA;
+  }
+
+  UpdateLaunch U;
+  memset(&U, 0, sizeof(U));
+  U.src = ds;
+  U.tgt = dt;
+  U.coeff_k = st->coeff_k;
+  U.coeff_v = st->coeff_v;
+  U.basis_k = st->basis_k;
+  U.basis_v = st->basis_v;
+  U.r = st->r;
+  U.n_cov = st->n_cov;
+  U.basis_bf16 = st->basis_dtype == KVC_BF16;
+  U.pairing = rope->pairing;
+  U.shift = shift;
+  U.L = tgt->L;
+  U.H = tgt->H;
+  U.status = status;
+  rope_tables(rope, d, shift, U.cs, U.sn);
+  if (tl_path_force != KVC_PATH_GENERIC) {
+    const int trc = tc_project(U, d, s);
+    if (trc == KVC_OK) {
+      tl_last_path = KVC_PATH_TC;
+      return KVC_OK;
+    }
+    if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  }
+  U.tiles_per_slab = (st->n_cov + kGenericProjectTile - 1) / kGenericProjectTile;
+  const int64_t tiles = (int64_t)tgt->L * tgt->H * 2 * U.tiles_per_slab;
+  if (launch_project_generic(U, d, tiles, s) != cudaSuccess) return KVC_E_CUDA;
+  tl_last_path = KVC_PATH_GENERIC;
+  return KVC_OK;
+}
+
+// Work table layout in the batch workspace: [int64 prefix[n+1]] padded to 256 B, then DevItem[n].
+static size_t batch_prefix_bytes(int32_t n) { return (((size_t)(n + 1) * sizeof(int64_t)) + 255) & ~(size_t)255; }
+
+size_t kvc_batch_workspace_bytes(int32_t n_items) {
+  if (n_items <= 0) return 0;
+  return batch_prefix_bytes(n_items) + (size_t)n_items * sizeof(DevItem) + tc_batch_extra_bytes(n_items);
+}
+
+int kvc_apply_batch(const kvc_item* items, int32_t n_items, const kvc_rope* rope, void* workspace,
+                    size_t workspace_bytes, void* staging, void* stream) {
+  if (n_items < 0 || (n_items > 0 && !items)) return KVC_E_INVALID_ARG;
+  if (n_items == 0) return KVC_OK;
+  int rc;
+  if ((rc = check_rope(rope)) != KVC_OK) return rc;
+  const size_t need = kvc_batch_workspace_bytes(n_items);
+  if (!workspace || !staging || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return KVC_E_WORKSPACE;
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+  int64_t* prefix = reinterpret_cast<int64_t*>(staging);
+  DevItem* tab = reinterpret_cast<DevItem*>(reinterpret_cast<char*>(staging) + batch_prefix_bytes(n_items));
+  const int d = items[0].src.d;
+  for (int i = 0; i < n_items; ++i) {
+    ResolvedHop hop;
+    if ((rc = resolve_hop(&items[i].src, &items[i].st, items[i].shift, rope, &items[i].dst, &hop)) != KVC_OK) return rc;
+    if (hop.d != d) return KVC_E_SHAPE;
+    tab[i] = hop.item;
+  }
+  if (tl_path_force != KVC_PATH_GENERIC) {
+    const int trc = tc_apply_batch(tab, prefix, n_items, d, rope->pairing, status, workspace, staging, need, s);
+    if (trc == KVC_OK) {
+      tl_last_path = KVC_PATH_TC;
+      return KVC_OK;
+    }
+    if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  }
+  const int tile = generic_apply_tile(d);
+  int64_t total = 0;
+  for (int i = 0; i < n_items; ++i) {
+    prefix[i] = total;
+    tab[i].tiles_per_slab = (tab[i].src.T + tile - 1) / tile;
+    total += (int64_t)tab[i].L * tab[i].H * 2 * tab[i].tiles_per_slab;
+  }
+  prefix[n_items] = total;
+  if (total == 0) return KVC_OK;
+  if (total > 0x7fffffffLL) return KVC_E_UNSUPPORTED;
+  const size_t bytes = batch_prefix_bytes(n_items) + (size_t)n_items * sizeof(DevItem);
+  if (cudaMemcpyAsync(workspace, staging, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return KVC_E_CUDA;
+  ApplyLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.tile_prefix = reinterpret_cast<const int64_t*>(workspace);
+  L.items = reinterpret_cast<const DevItem*>(reinterpret_cast<char*>(workspace) + batch_prefix_bytes(n_items));
+  L.n_items = n_items;
+  L.pairing = rope->pairing;
+  L.total_tiles = total;
+  L.status = status;
+  if (launch_apply_generic(L, d, s) != cudaSuccess) return KVC_E_CUDA;
+  tl_last_path = KVC_PATH_GENERIC;
+  return KVC_OK;
+}
+
+int kvc_status_poll(uint32_t* flags) {
+  uint32_t w = 0;
+  if (cudaMemcpyFromSymbol(&w, g_status_word, sizeof(w)) != cudaSuccess) return KVC_E_CUDA;
+  if (flags) *flags = w;
+  return w ? KVC_E_DEVICE_FLAG : KVC_OK;
+}
+
+int kvc_status_reset(void) {
+  const uint32_t z = 0;
+  return cudaMemcpyToSymbol(g_status_word, &z, sizeof(z)) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+int kvc_set_path(int32_t path) {
+  if (path != KVC_PATH_AUTO && path != KVC_PATH_GENERIC && path != KVC_PATH_TC) return KVC_E_INVALID_ARG;
+  tl_path_force = path;
+  return KVC_OK;
+}
+
+int kvc_last_path(void) { return tl_last_path; }
+
+int64_t kvc_apply_bytes(const kvc_cache* src, const kvc_state* st) {
+  if (!src || !st) return 0;
+  const int64_t slabs = (int64_t)src->L * src->H * 2;
+  const int64_t cache = slabs * src->T * src->d * 2;          // read once, written once
+  const bool live = st->r > 0 && st->n_cov > 0;
+  const int64_t coeff = live ? slabs * st->n_cov * st->r * 4 : 0;
+  const int64_t basis = live ? slabs * st->r * src->d * (st->basis_dtype == KVC_BF16 ? 2 : 4) : 0;
+  return 2 * cache + coeff + basis;
+}
+
+int64_t kvc_update_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode, int32_t has_src) {
+  if (!tgt || !st) return 0;
+  const int64_t slabs = (int64_t)tgt->L * tgt->H * 2;
+  const int64_t rows = slabs * st->n_cov * tgt->d * 2 * (has_src ? 2 : 1);   // src + tgt rows
+  const int64_t coeff = slabs * st->n_cov * st->r * 4;
+  const int64_t basis = slabs * st->r * tgt->d * (st->basis_dtype == KVC_BF16 ? 2 : 4);
+  int64_t b = rows + coeff + basis;                                          // projection pass
+  if (mode == KVC_FIT) b += rows + 2 * slabs * tgt->d * tgt->d * 4;          // Gram pass + G write/read
+  return b;
+}
+
+const char* kvc_strerror(int code) {
+  switch (code) {
+    case KVC_OK: return "ok";
+    case KVC_E_INVALID_ARG: return "invalid argument";
+    case KVC_E_SHAPE: return "argument geometries do not agree";
+    case KVC_E_UNSUPPORTED: return "valid but unsupported configuration";
+    case KVC_E_ALIAS: return "destination overlaps source";
+    case KVC_E_CUDA: return "CUDA call failed";
+    case KVC_E_WORKSPACE: return "workspace missing, misaligned or too small";
+    case KVC_E_DEVICE_FLAG: return "a kernel recorded an anomaly";
+    default: return "unknown kvc status";
+  }
+}
+
+const char* kvc_version(void) { return "kvc 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,109 @@
+// Device-side descriptors shared by the kernels of this library (not by the oracle).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace kvc {
+
+constexpr int kMaxHalfD = 64;  // head_dim <= 128
+
+// One cache as the kernels see it: strides resolved, page size as shift/mask.
+struct DevCache {
+  __nv_bfloat16* k;
+  __nv_bfloat16* v;
+  const int32_t* page_table;  // nullptr => contiguous
+  int64_t s_layer, s_page, s_head, s_tok;
+  int32_t T, n_phys;
+  int32_t page_shift, page_mask;
+};
+
+struct DevState {
+  const float* coeff_k;
+  const float* coeff_v;
+  const void* basis_k;
+  const void* basis_v;
+  int32_t r, n_cov, basis_bf16, pad;
+};
+
+// One hop over one request: what kvc_apply does for all (layer, head, token).
+struct DevItem {
+  DevCache src, dst;
+  DevState st;
+  int32_t shift, L, H, tiles_per_slab;   // tiles_per_slab = ceil(T / tile)
+  float cs[kMaxHalfD], sn[kMaxHalfD];    // cos / sin of shift * f_k, rounded from float64
+};
+
+struct ApplyLaunch {
+  const DevItem* items;        // device table, or nullptr => `one`
+  const int64_t* tile_prefix;  // device [n_items + 1] exclusive prefix of tile counts
+  int32_t n_items, pairing;
+  int64_t total_tiles;
+  uint32_t* status;
+  DevItem one;
+};
+
+struct UpdateLaunch {
+  DevCache src, tgt;           // src.k == nullptr => Delta = tgt
+  float* coeff_k;
+  float* coeff_v;
+  const void* basis_k;
+  const void* basis_v;
+  int32_t r, n_cov, basis_bf16, pairing;
+  int32_t shift, L, H, tiles_per_slab;
+  uint32_t* status;
+  float cs[kMaxHalfD], sn[kMaxHalfD];
+};
+
+struct FitLaunch {             // Gram + eigensolve
+  DevCache src, tgt;
+  float* gram;                 // [L*H*2][d][d]
+  float* evals;                // [L*H*2][d] descending
+  float* basis_k;              // [L,H,r,d] float32 out
+  float* basis_v;
+  int32_t r, n_cov, pairing, shift, L, H;
+  uint32_t* status;
+  float cs[kMaxHalfD], sn[kMaxHalfD];
+};
+
+// Address of row (l, h, t) of a cache; returns nullptr (and flags) on a bad page id.
+__device__ __forceinline__ __nv_bfloat16* row_ptr(const DevCache& c, __nv_bfloat16* base, int l, int h, int t,
+                                                   uint32_t* status) {
+  int64_t off = (int64_t)l * c.s_layer + (int64_t)h * c.s_head;
+  if (c.page_table) {
+    int p = c.page_table[t >> c.page_shift];
+    if ((unsigned)p >= (unsigned)c.n_phys) {
+      atomicOr(status, 1u);
+      return nullptr;
+    }
+    off += (int64_t)p * c.s_page + (int64_t)(t & c.page_mask) * c.s_tok;
+  } else {
+    off += (int64_t)t * c.s_tok;
+  }
+  return base + off;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 u;
+  u.x = pack2(f[0], f[1]);
+  u.y = pack2(f[2], f[3]);
+  u.z = pack2(f[4], f[5]);
+  u.w = pack2(f[6], f[7]);
+  return u;
+}
+
+}  // namespace kvc

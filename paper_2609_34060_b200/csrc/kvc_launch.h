@@ -1,0 +1,18 @@
+// Host-side launch interface between the C ABI and the kernel translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvc_dev.cuh"
+
+namespace kvc {
+
+// CUDA-core family (kvc_generic.cu)
+cudaError_t launch_apply_generic(const ApplyLaunch& L, int d, cudaStream_t s);
+int generic_apply_tile(int d);                     // tokens per tile of the generic apply kernel
+constexpr int kGenericProjectTile = 64;
+cudaError_t launch_project_generic(const UpdateLaunch& U, int d, int64_t tiles, cudaStream_t s);
+cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s);
+cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s);
+
+}  // namespace kvc

@@ -1,0 +1,20 @@
+// TMA + tcgen05 kernel family (kvc_tc_*.cu): host entry points used by the C ABI.
+// Each returns KVC_OK, KVC_E_UNSUPPORTED when the arguments are outside what the
+// family serves (the caller then uses the CUDA-core kernels), or another KVC_E_*.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "kvc_dev.cuh"
+
+namespace kvc {
+
+int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s);
+int tc_apply_batch(DevItem* tab_host, int64_t* prefix_host, int n_items, int d, int pairing, uint32_t* status,
+                   void* workspace_dev, void* staging_host, size_t bytes, cudaStream_t s);
+size_t tc_batch_extra_bytes(int n_items);
+int tc_project(const UpdateLaunch& U, int d, cudaStream_t s);
+int tc_gram(const FitLaunch& F, int d, cudaStream_t s);
+
+}  // namespace kvc

@@ -1,0 +1,194 @@
+"""GPU parity of kvc_state_update (project and fit modes) against the fp64 oracle.
+
+Coefficients with a *given* basis are compared element by element.  A fitted basis is not
+unique (sign, rotations inside near-equal singular values), so fit mode is checked through
+what is unique: the Gram matrix, the eigenvalues, orthonormality, the projector on a
+well-separated spectrum, the Eckart-Young residual and the update -> apply round trip.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_34060_b200 as kvc
+from paper_2609_34060_b200 import workloads as wl
+from oracle import kvc_oracle as orc
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+CFG_TINY = wl.CONFIGS["tiny"]
+CFG_8B_S = wl.CONFIGS["llama8b_8k"].scaled(name="8b_small", L=2, H=2, T=700)
+CFG_VLM_S = wl.CONFIGS["vlm_16k"].scaled(name="vlm_small", L=1, H=2, T=1003, image_spans=((512, 1024),))
+CFG_R64_S = wl.CONFIGS["llama70b_32k"].scaled(name="r64_small", L=1, H=2, T=390)
+
+PATHS = [kvc.KVC_PATH_GENERIC, kvc.KVC_PATH_AUTO]
+PATH_IDS = ["generic", "auto"]
+
+
+@pytest.fixture(autouse=True)
+def _reset_path():
+    kvc.kvc_status_reset()
+    yield
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    assert kvc.kvc_status_poll() == 0
+
+
+def _edge(cfg, hop=1):
+    """(src, tgt) caches of one edge on the CPU, the true state, the shift.  The target is
+    derived by the oracle from generator draws: bf16(Align(src) + A B + sigma noise)."""
+    src_cpu = hp.make_cache(cfg)
+    true = hp.make_state(cfg, hop)
+    pl = wl.prefix_lengths(cfg)
+    shift = pl[hop] - pl[hop - 1]
+    nk = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2 * hop).numpy()
+    nv = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2 * hop + 1).numpy()
+    osrc = hp.oracle_cache(src_cpu)
+    otgt = orc.make_target(osrc, hp.oracle_state(true), shift, hp.inv_freq(cfg), nk, nv, cfg.sigma)
+    as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    if cfg.paged:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v), T=cfg.T, page_table=src_cpu.page_table)
+    else:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v))
+    return src_cpu, tgt_cpu, osrc, otgt, true, shift
+
+
+def _coeff_tol(osrc, otgt, delta, basis, l, h, which):
+    """|c_gpu - c_ref| <= 2^-12 |Delta_t| |B_q| + 2^-18 (|src_t| + |tgt_t|) |B_q| + 1e-6.
+    First term: product rounding of the split-precision contraction; second: float32
+    rotation and cancellation in tgt - Rot(src), relative to the inputs' size."""
+    bn = np.linalg.norm(basis, axis=1)[None, :]
+    dn = np.linalg.norm(delta, axis=1)[:, None]
+    sn = np.linalg.norm(orc.bf16_to_f64(osrc.get_bits(which, l, h)), axis=1)[:, None] if osrc is not None else 0.0
+    tn = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h)), axis=1)[:, None]
+    return 2.0 ** -12 * dn * bn + 2.0 ** -18 * (sn + tn) * bn + 1e-6
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("cfg", [CFG_TINY, CFG_8B_S, CFG_VLM_S, CFG_R64_S], ids=lambda c: c.name)
+def test_project_mode(cfg, path):
+    src_cpu, tgt_cpu, osrc, otgt, true, shift = _edge(cfg)
+    n_cov = cfg.T - 5
+    # project onto a basis that is NOT the true one (any given basis must work)
+    other = hp.make_state(cfg, 3)
+    ost, _ = orc.state_update(osrc, otgt, shift, hp.inv_freq(cfg), mode=orc.PROJECT, n_cov=n_cov,
+                              basis_k=other.basis_k.numpy(), basis_v=other.basis_v.numpy())
+    kvc.kvc_set_path(path)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    st = kvc.State(torch.full((cfg.L, cfg.H, n_cov, cfg.r), 7.0, device=DEV),
+                   torch.full((cfg.L, cfg.H, n_cov, cfg.r), 7.0, device=DEV),
+                   other.basis_k.to(DEV), other.basis_v.to(DEV), n_cov=n_cov)
+    kvc.kvc_state_update(src, tgt, shift, kvc.Rope(cfg.theta), st, kvc.KVC_PROJECT)
+    torch.cuda.synchronize()
+    ck, cv = st.coeff_k.cpu().numpy().astype(np.float64), st.coeff_v.cpu().numpy().astype(np.float64)
+    worst = 0.0
+    for l in range(cfg.L):
+        for h in range(cfg.H):
+            for which, got, ref, bs in (("k", ck, ost.coeff_k, other.basis_k), ("v", cv, ost.coeff_v, other.basis_v)):
+                dl = orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, hp.inv_freq(cfg),
+                                   which == "k")[:n_cov]
+                tol = _coeff_tol(osrc, otgt, dl, bs[l, h].numpy().astype(np.float64), l, h, which)[:n_cov]
+                worst = max(worst, float(np.max(np.abs(got[l, h] - ref[l, h].astype(np.float64)) / tol)))
+    assert worst <= 1.0, worst
+    # inputs are only read
+    assert torch.equal(src.k.cpu(), src_cpu.k) and torch.equal(tgt.v.cpu(), tgt_cpu.v)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_project_without_source_and_bf16_basis(path):
+    cfg = CFG_8B_S.scaled(T=200)
+    src_cpu, tgt_cpu, osrc, otgt, true, shift = _edge(cfg)
+    other = hp.make_state(cfg, 3, basis_dtype=torch.bfloat16)
+    ost, _ = orc.state_update(None, otgt, 0, hp.inv_freq(cfg), mode=orc.PROJECT,
+                              basis_k=other.basis_k.float().numpy(), basis_v=other.basis_v.float().numpy())
+    kvc.kvc_set_path(path)
+    st = kvc.State(torch.zeros(cfg.L, cfg.H, cfg.T, cfg.r, device=DEV), torch.zeros(cfg.L, cfg.H, cfg.T, cfg.r, device=DEV),
+                   other.basis_k.to(DEV), other.basis_v.to(DEV))
+    kvc.kvc_state_update(None, hp.to_dev(tgt_cpu, DEV), 0, kvc.Rope(cfg.theta), st, kvc.KVC_PROJECT)
+    torch.cuda.synchronize()
+    for got, ref in ((st.coeff_k, ost.coeff_k), (st.coeff_v, ost.coeff_v)):
+        err = np.abs(got.cpu().numpy().astype(np.float64) - ref.astype(np.float64))
+        # Delta = tgt: |c| up to ~|tgt_t|; float32 accumulation over d terms
+        assert np.max(err) <= 2.0 ** -12 * 40.0
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("cfg", [CFG_TINY, CFG_8B_S.scaled(T=520), CFG_VLM_S.scaled(T=400, image_spans=())],
+                         ids=lambda c: c.name)
+def test_fit_mode(cfg, path):
+    src_cpu, tgt_cpu, osrc, otgt, true, shift = _edge(cfg)
+    f = hp.inv_freq(cfg)
+    ost, oev = orc.state_update(osrc, otgt, shift, f, r=cfg.r, mode=orc.FIT)
+    kvc.kvc_set_path(path)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+    st = kvc.State(torch.zeros(L, H, T, r, device=DEV), torch.zeros(L, H, T, r, device=DEV),
+                   torch.zeros(L, H, r, d, device=DEV), torch.zeros(L, H, r, d, device=DEV))
+    ws = torch.empty(kvc.kvc_workspace_bytes(tgt, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(src, tgt, shift, kvc.Rope(cfg.theta), st, kvc.KVC_FIT, workspace=ws)
+    torch.cuda.synchronize()
+    wsf = ws.view(torch.float32).cpu().numpy().astype(np.float64)
+    G = wsf[: L * H * 2 * d * d].reshape(L, H, 2, d, d)
+    ev = wsf[L * H * 2 * d * d: L * H * 2 * d * (d + 1)].reshape(L, H, 2, d)
+    for l in range(L):
+        for h in range(H):
+            for i, (which, B_t, c_t, B_o) in enumerate((("k", st.basis_k, st.coeff_k, ost.basis_k),
+                                                        ("v", st.basis_v, st.coeff_v, ost.basis_v))):
+                dl = orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, f, which == "k")
+                Gref = orc.gram(dl)
+                dg = np.sqrt(np.diag(Gref))
+                # float32 accumulation over T rows of split-precision products
+                assert np.max(np.abs(G[l, h, i] - Gref) / (2.0 ** -12 * np.outer(dg, dg) + 1e-6)) <= 1.0
+                w = oev[l, h, i]
+                assert np.max(np.abs(ev[l, h, i] - w)) <= 1e-4 * w[0]
+                assert np.all(np.diff(ev[l, h, i]) <= 1e-6 * w[0])                       # descending
+                B = B_t[l, h].cpu().numpy().astype(np.float64)
+                c = c_t[l, h].cpu().numpy().astype(np.float64)
+                assert np.max(np.abs(B @ B.T - np.eye(r))) <= 1e-4                        # orthonormal rows
+                assert np.all(B[np.arange(r), np.argmax(np.abs(B), axis=1)] > 0)          # sign convention
+                # the spectrum is well separated at r (rank-r signal over a noise floor):
+                # the projector is unique and must match the oracle's
+                Bo = B_o[l, h].astype(np.float64)
+                assert np.linalg.norm(B.T @ B - Bo.T @ Bo) <= 1e-2
+                # Eckart-Young: no rank-r state reconstructs Delta better than the tail energy
+                tail = float(np.sum(w[r:]))
+                res = float(np.sum((dl - c @ B) ** 2))
+                assert res <= 1.001 * tail + 1e-6 * float(np.sum(w)), (res, tail)
+                # coeff columns are U_r Sigma_r: mutually orthogonal, energies = top eigenvalues
+                Gc = c.T @ c
+                assert np.max(np.abs(Gc - np.diag(np.diag(Gc)))) <= 2e-3 * w[0]
+                assert np.max(np.abs(np.sort(np.diag(Gc))[::-1] - w[:r])) <= 1e-3 * w[0]
+    # round trip: applying the fitted state to the source gives back the target (up to the
+    # noise floor and bf16 rounding)
+    dst = kvc.Cache(torch.zeros_like(src.k), torch.zeros_like(src.v), T=cfg.T if cfg.paged else None,
+                    page_table=src.page_table)
+    kvc.kvc_apply(src, st, shift, kvc.Rope(cfg.theta), dst)
+    torch.cuda.synchronize()
+    for which in ("k", "v"):
+        got = orc.bf16_to_f64(hp.logical_bits(dst, which))
+        want = orc.bf16_to_f64(hp.logical_bits(otgt, which))
+        err = np.abs(got - want)
+        assert np.mean(err > 2.0 ** -6 * np.abs(want) + 0.02) < 1e-3
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_fit_rank_limits(path):
+    # fewer covered rows than the requested rank: the surplus basis rows are zero
+    cfg = CFG_TINY.scaled(T=40, r=8)
+    src_cpu, tgt_cpu, osrc, otgt, true, shift = _edge(cfg)
+    kvc.kvc_set_path(path)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    n_cov = 5
+    st = kvc.State(torch.zeros(cfg.L, cfg.H, n_cov, 8, device=DEV), torch.zeros(cfg.L, cfg.H, n_cov, 8, device=DEV),
+                   torch.ones(cfg.L, cfg.H, 8, cfg.d, device=DEV), torch.ones(cfg.L, cfg.H, 8, cfg.d, device=DEV), n_cov=n_cov)
+    ws = torch.empty(kvc.kvc_workspace_bytes(tgt, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(src, tgt, shift, kvc.Rope(cfg.theta), st, kvc.KVC_FIT, workspace=ws)
+    torch.cuda.synchronize()
+    B = st.basis_k.cpu().numpy().astype(np.float64)
+    assert np.all(B[:, :, n_cov:] == 0)
+    assert np.max(np.abs(B[0, 0, :n_cov] @ B[0, 0, :n_cov].T - np.eye(n_cov))) <= 1e-4
+    # with all five directions kept the five covered rows are reproduced exactly
+    dl = orc.deviation(osrc.get_bits("k", 0, 0), otgt.get_bits("k", 0, 0), shift, hp.inv_freq(cfg), True)[:n_cov]
+    c = st.coeff_k[0, 0].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(c @ B[0, 0] - dl)) <= 1e-3 * np.max(np.abs(dl))
