@@ -310,7 +310,8 @@ def main():
     chain_ms = sum(b.elapsed_time(e) for b, e in zip(ev["chain_begin"], ev["chain_end"])) / args.steps
     upd_ms = sum(b.elapsed_time(e) for b, e in zip(ev["update_begin"], ev["update_end"])) / args.steps
     last_path = kvc.kvc_last_path()
-    assert kvc.kvc_status_poll() == 0, "a kernel flagged an anomaly"
+    flags = kvc.kvc_status_poll()
+    assert flags == 0, f"a kernel flagged an anomaly: {flags}"
     t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)

@@ -58,10 +58,11 @@ def _coeff_tol(osrc, otgt, delta, basis, l, h, which):
     """|c_gpu - c_ref| <= 2^-12 |Delta_t| |B_q| + 2^-18 (|src_t| + |tgt_t|) |B_q| + 1e-6.
     First term: product rounding of the split-precision contraction; second: float32
     rotation and cancellation in tgt - Rot(src), relative to the inputs' size."""
+    n = delta.shape[0]
     bn = np.linalg.norm(basis, axis=1)[None, :]
     dn = np.linalg.norm(delta, axis=1)[:, None]
-    sn = np.linalg.norm(orc.bf16_to_f64(osrc.get_bits(which, l, h)), axis=1)[:, None] if osrc is not None else 0.0
-    tn = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h)), axis=1)[:, None]
+    sn = np.linalg.norm(orc.bf16_to_f64(osrc.get_bits(which, l, h)), axis=1)[:n, None] if osrc is not None else 0.0
+    tn = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h)), axis=1)[:n, None]
     return 2.0 ** -12 * dn * bn + 2.0 ** -18 * (sn + tn) * bn + 1e-6
 
 
@@ -88,7 +89,7 @@ def test_project_mode(cfg, path):
             for which, got, ref, bs in (("k", ck, ost.coeff_k, other.basis_k), ("v", cv, ost.coeff_v, other.basis_v)):
                 dl = orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, hp.inv_freq(cfg),
                                    which == "k")[:n_cov]
-                tol = _coeff_tol(osrc, otgt, dl, bs[l, h].numpy().astype(np.float64), l, h, which)[:n_cov]
+                tol = _coeff_tol(osrc, otgt, dl, bs[l, h].numpy().astype(np.float64), l, h, which)
                 worst = max(worst, float(np.max(np.abs(got[l, h] - ref[l, h].astype(np.float64)) / tol)))
     assert worst <= 1.0, worst
     # inputs are only read
