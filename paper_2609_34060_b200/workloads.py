@@ -132,10 +132,15 @@ def base_cache(cfg: Config, device="cpu", table: Optional[torch.Tensor] = None, 
                 k[:, :, a:b, :] += off_k[:, :, None, :]
                 v[:, :, a:b, :] += off_v[:, :, None, :]
             else:
-                assert a % cfg.page == 0 and b % cfg.page == 0
-                phys = table[a // cfg.page: b // cfg.page].to(torch.int64).to(dev)
+                assert a % cfg.page == 0
+                full = b // cfg.page
+                phys = table[a // cfg.page: full].to(torch.int64).to(dev)
                 k[:, phys] += off_k[:, None, :, None, :]
                 v[:, phys] += off_v[:, None, :, None, :]
+                if b % cfg.page:                          # the span ends inside a page
+                    last = int(table[full])
+                    k[:, last, :, : b % cfg.page] += off_k[:, :, None, :]
+                    v[:, last, :, : b % cfg.page] += off_v[:, :, None, :]
     return k.to(torch.bfloat16), v.to(torch.bfloat16)
 
 
