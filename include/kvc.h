@@ -12,7 +12,8 @@
  *   - plain C types only; every pointer says whether it is HOST or DEVICE memory;
  *   - all device work is enqueued on `stream` (a cudaStream_t passed as void*;
  *     NULL = the legacy default stream); no entry point synchronises, and none
- *     allocates device memory: every buffer, scratch included, is the caller's;
+ *     allocates device memory: every buffer, scratch included, is the caller's
+ *     (kvc_state_update_noalloc alone uses scratch built into the library);
  *   - the return value is KVC_OK (0) or a negative KVC_E_* code; nothing is
  *     launched when an argument check fails;
  *   - bf16 means the upper 16 bits of an IEEE float32, rounded to nearest-even
@@ -38,6 +39,7 @@ extern "C" {
 #define KVC_E_CUDA         (-5)  /* a CUDA runtime / driver call failed            */
 #define KVC_E_WORKSPACE    (-6)  /* workspace missing, misaligned or too small     */
 #define KVC_E_DEVICE_FLAG  (-7)  /* a kernel recorded an anomaly (see status_poll) */
+#define KVC_E_TOO_LARGE    (-8)  /* problem needs more than the built-in scratch   */
 
 /* ---- layouts, dtypes, modes --------------------------------------------- */
 #define KVC_CONTIG 0   /* k, v: bf16 [L, H, T, d]                                  */
@@ -170,6 +172,36 @@ int kvc_state_update(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, 
 
 /* Scratch kvc_state_update needs for this geometry and mode (0 for KVC_PROJECT). */
 size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mode);
+
+/*
+ * kvc_state_update_noalloc -- kvc_state_update without a workspace argument.
+ * (No counterpart in the paper: this exists for integration only.)
+ *
+ * Some callers cannot obtain device memory at the point where they need a state
+ * update: code that runs inside a serving engine whose memory pool was sized and handed
+ * out at start-up, plugins that are forbidden to call cudaMalloc because an allocation
+ * synchronises the device and would stall the engine's other streams, and processes
+ * whose GPU memory is already fully committed to the KV pool.  For them the FIT-mode
+ * scratch lives in a fixed array inside the library image (KVC_STATIC_SCRATCH_BYTES on
+ * every GPU that loads the library, held until the process exits).  The call performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine; inputs and outputs are
+ * still the caller's buffers, with the same meaning as in kvc_state_update.
+ *
+ *  - Capacity: kvc_workspace_bytes(tgt, st, mode) must not exceed
+ *    KVC_STATIC_SCRATCH_BYTES, i.e. L*H <= 64 at d = 128 (L*H <= 254 at d = 64) in FIT
+ *    mode; larger problems return KVC_E_TOO_LARGE and launch nothing (split them by
+ *    layer, or use kvc_state_update with your own workspace).  KVC_PROJECT needs no
+ *    scratch and is never rejected for size.
+ *  - The first call on each device looks up the array's device address (with that
+ *    device current).  Make that first call before any stream capture begins.
+ *  - All calls on one device share the one array, and it keeps the previous call's
+ *    contents: the entry point clears the part it is about to use on `stream` first.
+ *    Two calls whose device work can overlap (different streams, or different host
+ *    threads on different streams) race on the array: serialise them.
+ */
+#define KVC_STATIC_SCRATCH_BYTES (128 * (128 * 128 + 128) * 4)
+int kvc_state_update_noalloc(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,
+                             kvc_state *st, int32_t mode, void *stream);
 
 /*
  * kvc_apply_batch -- many independent hops in ONE launch (concurrent serving: each

@@ -25,7 +25,7 @@ KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
 KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4
 
 EXPORTS = (
-    "kvc_apply", "kvc_chain", "kvc_state_update", "kvc_workspace_bytes", "kvc_apply_batch",
+    "kvc_apply", "kvc_chain", "kvc_state_update", "kvc_state_update_noalloc", "kvc_workspace_bytes", "kvc_apply_batch",
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version",
 )
@@ -75,6 +75,8 @@ def load(path: Optional[str] = None):
     lib.kvc_apply.argtypes = [PC, PS, i32, PR, PC, vp]
     lib.kvc_chain.argtypes = [PC, i32, C.POINTER(i32), PS, PR, PC, vp]
     lib.kvc_state_update.argtypes = [PC, PC, i32, PR, PS, i32, vp, sz, vp]
+    lib.kvc_state_update_noalloc.argtypes = [PC, PC, i32, PR, PS, i32, vp]
+    lib.kvc_state_update_noalloc.restype = C.c_int
     lib.kvc_workspace_bytes.argtypes = [PC, PS, i32]
     lib.kvc_workspace_bytes.restype = sz
     lib.kvc_apply_batch.argtypes = [PI, i32, PR, vp, sz, vp, vp]
@@ -240,6 +242,26 @@ def kvc_state_update(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, s
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().kvc_state_update(sp, C.byref(t), int(shift), C.byref(r), C.byref(s), int(mode), ws_ptr, ws_bytes,
                                    _stream(stream)), "kvc_state_update")
+
+
+KVC_STATIC_SCRATCH_BYTES = 128 * (128 * 128 + 128) * 4
+
+
+def kvc_state_update_noalloc(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, st: State, mode: int,
+                             stream=None) -> None:
+    """kvc_state_update for callers that may not allocate device memory (an engine plugin
+    working inside a pre-sized pool, a process whose memory is all committed to the KV
+    pool): FIT-mode scratch is a fixed array inside the library, so there is no workspace
+    argument.  Raises KvcError(-8) when the problem needs more than
+    KVC_STATIC_SCRATCH_BYTES (L*H > 64 at d = 128).  Calls that may overlap on the GPU must
+    be serialised by the caller: they share the one array."""
+    t, s, r = tgt.struct(), st.struct(), rope.struct()
+    sp = None
+    if src is not None:
+        ss = src.struct()
+        sp = C.byref(ss)
+    _check(load().kvc_state_update_noalloc(sp, C.byref(t), int(shift), C.byref(r), C.byref(s), int(mode),
+                                           _stream(stream)), "kvc_state_update_noalloc")
 
 
 class Item:

@@ -450,6 +450,7 @@ const char* kvc_strerror(int code) {
     case KVC_E_CUDA: return "CUDA call failed";
     case KVC_E_WORKSPACE: return "workspace missing, misaligned or too small";
     case KVC_E_DEVICE_FLAG: return "a kernel recorded an anomaly";
+    case KVC_E_TOO_LARGE: return "problem needs more scratch than the built-in array holds (KVC_STATIC_SCRATCH_BYTES)";
     default: return "unknown kvc status";
   }
 }
