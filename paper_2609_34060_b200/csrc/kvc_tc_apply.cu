@@ -1,0 +1,872 @@
+// apply / chain / batch on the Blackwell data path: TMA-staged tiles, the rank-r
+// contraction coeff . basis on tcgen05 tensor cores with fp32 accumulators in TMEM, RoPE
+// re-alignment and the add in registers, results written back through TMA.
+//
+// One persistent CTA per SM walks a contiguous range of tiles; a tile is 128 tokens of one
+// (layer, head, K|V) slab.  Warp roles:
+//   warp 0      TMA producer (one lane): base tile (bf16 128 x 128) + fp32 coefficient tile
+//   warp 1      MMA issuer (one lane) and TMEM owner
+//   warp 2      basis stager: basis[r][d] -> K-major, 128B-swizzled bf16 hi/lo operand
+//   warp 3      idle
+//   warps 4-7, 8-11   two epilogue groups; a group owns every other tile of the CTA:
+//               convert its coefficient rows to bf16 hi/lo in place, wait for the MMA, read the
+//               accumulator row from TMEM, rotate/add/round, write the row back in place, and
+//               one lane issues the TMA store and releases the stage.
+// Precision: c = c1 + c2 and B = B1 + B2 with bf16 terms; c.B ~= c1.B1 + c2.B1 + c1.B2
+// (relative error about 2^-16 per product), accumulated in fp32.
+// Every wait is bounded; on expiry the CTA records KVC_FLAG_WAIT_EXPIRED, drains and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <string.h>
+
+#include <cstddef>
+
+#include "../../include/kvc.h"
+#include "kvc_dev.cuh"
+#include "kvc_tc.h"
+
+namespace kvc {
+namespace tc {
+
+constexpr int kTileTok = 128;
+constexpr int kThreads = 384;
+constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a base tile (bf16)
+constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
+constexpr int kCoeffBlkBytes = kTileTok * 128;    // 128 tokens x 32 fp32 (one rank block)
+constexpr int kBasisBlkBytes = 128 * 128;         // 128 channels x (32 hi + 32 lo) bf16
+constexpr long long kWaitLimitCycles = 3000000000LL;   // about 1.5 s
+
+struct alignas(64) ItemMaps {
+  CUtensorMap src_k, src_v, dst_k, dst_v, coeff_k, coeff_v;
+};
+
+struct ApplyTcLaunch {
+  const DevItem* items;        // device table or nullptr => `one`
+  const ItemMaps* maps;        // device table or nullptr => `one_maps`
+  const int64_t* tile_prefix;  // device [n_items + 1]
+  int32_t n_items, pairing;
+  int64_t total_tiles;
+  uint32_t* status;
+  DevItem one;
+  ItemMaps one_maps;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another thread already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+// Bounded wait used while draining after an abort: ignores the abort flag, shorter limit.
+__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return;
+    if ((it & 63u) == 0u && clock64() - t0 > kWaitLimitCycles / 8) return;
+  }
+}
+// Named barrier over n threads that also ORs a predicate: every thread gets the same answer.
+__device__ __forceinline__ bool named_bar_or(int id, int n, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(n), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled shared-memory operand: 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                               // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset: next 8-row group
+  d |= (uint64_t)1 << 46;                               // descriptor version (sm_100)
+  d |= (uint64_t)2 << 61;                               // SWIZZLE_128B
+  return d;
+}
+// kind::f16, A = B = bf16, D = f32, both K-major, M = 128, N = 128
+constexpr uint32_t kIdescBf16M128N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+// ------------------------------------------------------------------ tile bookkeeping
+struct Tile {
+  const DevItem* it;
+  const ItemMaps* mp;
+  int item, slab, is_v, t0, l, h;
+  bool has_coeff;    // the tile holds covered rows of a live state
+  bool uses_basis;   // its slab has a live state (basis staged for the slab)
+};
+
+struct TileWalker {
+  const ApplyTcLaunch* p;
+  int64_t tile, end;
+  int item;
+  int64_t item_lo, item_hi;
+
+  __device__ void init(const ApplyTcLaunch* pp, int64_t begin, int64_t end_) {
+    p = pp;
+    tile = begin;
+    end = end_;
+    item = 0;
+    if (p->items) {
+      int lo = 0, hi = p->n_items;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (begin >= p->tile_prefix[mid]) lo = mid; else hi = mid;
+      }
+      item = lo;
+      item_lo = p->tile_prefix[item];
+      item_hi = p->tile_prefix[item + 1];
+    } else {
+      item_lo = 0;
+      item_hi = p->total_tiles;
+    }
+  }
+  __device__ bool done() const { return tile >= end; }
+  __device__ void get(Tile& t) {
+    while (tile >= item_hi) {   // items with zero tiles are skipped
+      ++item;
+      item_lo = item_hi;
+      item_hi = p->tile_prefix[item + 1];
+    }
+    const DevItem* it = p->items ? p->items + item : &p->one;
+    t.it = it;
+    t.mp = p->maps ? p->maps + item : &p->one_maps;
+    t.item = item;
+    const int64_t local = tile - item_lo;
+    const int tt = (int)(local % it->tiles_per_slab);
+    const int64_t sk = local / it->tiles_per_slab;
+    t.is_v = (int)(sk & 1);
+    t.slab = (int)(sk >> 1);
+    t.l = t.slab / it->H;
+    t.h = t.slab % it->H;
+    t.t0 = tt * kTileTok;
+    t.uses_basis = it->st.r > 0 && it->st.n_cov > 0;
+    t.has_coeff = t.uses_basis && t.t0 < it->st.n_cov;
+  }
+  __device__ void next() { ++tile; }
+};
+
+__device__ __forceinline__ bool same_slab(const Tile& a, const Tile& b) {
+  return a.item == b.item && a.slab == b.slab && a.is_v == b.is_v;
+}
+
+// Shared-memory control block (after the tiles)
+template <int NSTAGE, int NB>
+struct Ctrl {
+  uint64_t full[NSTAGE], conv[NSTAGE], empty[NSTAGE];
+  uint64_t mma_done[2], acc_empty[2];
+  uint64_t basis_full[NB], basis_empty[NB];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// ------------------------------------------------------------------ the kernel
+template <int RB, int NSTAGE, int NB>
+__global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
+  constexpr int kStageBytes = kBaseBytes + RB * kCoeffBlkBytes;
+  constexpr int kBasisSlotBytes = RB * kBasisBlkBytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t stages = base;
+  const uint32_t bases = base + NSTAGE * kStageBytes;
+  Ctrl<NSTAGE, NB>* ctrl = reinterpret_cast<Ctrl<NSTAGE, NB>*>(smem + NSTAGE * kStageBytes + NB * kBasisSlotBytes);
+  volatile int* abort_flag = &ctrl->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t n = p.total_tiles;
+  const int64_t tile_begin = n * blockIdx.x / gridDim.x;
+  const int64_t tile_end = n * (blockIdx.x + 1) / gridDim.x;
+
+  if (tid == 0) {
+    for (int s = 0; s < NSTAGE; ++s) {
+      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->conv[s]), 128);
+      mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
+      mbar_init(smem_u32(&ctrl->acc_empty[g]), 128);
+    }
+    for (int b = 0; b < NB; ++b) {
+      mbar_init(smem_u32(&ctrl->basis_full[b]), 1);
+      mbar_init(smem_u32(&ctrl->basis_empty[b]), 1);
+    }
+    mbar_init(smem_u32(&ctrl->drain), 1);
+    ctrl->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctrl->tmem_base), 256);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+
+  if (warp == 0) {
+    // =============================================================== TMA producer
+    if (lane == 0) {
+      TileWalker w;
+      w.init(&p, tile_begin, tile_end);
+      uint32_t i = 0;
+      for (; !w.done(); w.next(), ++i) {
+        Tile t;
+        w.get(t);
+        const int s = i % NSTAGE;
+        const uint32_t use = i / NSTAGE;
+        if (!mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag)) break;
+        const DevItem& it = *t.it;
+        const uint32_t st_base = stages + s * kStageBytes;
+        const uint32_t bar = smem_u32(&ctrl->full[s]);
+        const CUtensorMap* smap = t.is_v ? &t.mp->src_v : &t.mp->src_k;
+        uint32_t bytes = t.has_coeff ? RB * kCoeffBlkBytes : 0;
+        if (!it.src.page_table) {
+          bytes += kBaseBytes;
+          mbar_expect_tx(bar, bytes);
+          tma_load_5d(st_base, smap, bar, 0, t.t0, t.h, 0, t.l);
+          tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t.t0, t.h, 0, t.l);
+        } else {
+          const int page = it.src.page_mask + 1;
+          const int per_tile = kTileTok >> it.src.page_shift;
+          const int first = t.t0 >> it.src.page_shift;
+          const int n_pages = min(per_tile, ((it.src.T + page - 1) >> it.src.page_shift) - first);
+          int ids[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) ids[u] = (u < n_pages) ? it.src.page_table[first + u] : -1;
+          int n_ok = 0;
+#pragma unroll
+          for (int u = 0; u < 16; ++u) n_ok += (u < n_pages) && ((unsigned)ids[u] < (unsigned)it.src.n_phys);
+          bytes += n_ok * page * 256;
+          mbar_expect_tx(bar, bytes);
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            if (u < n_pages) {
+              if ((unsigned)ids[u] < (unsigned)it.src.n_phys) {
+                tma_load_5d(st_base + u * page * 128, smap, bar, 0, 0, t.h, ids[u], t.l);
+                tma_load_5d(st_base + kHalfBytes + u * page * 128, smap, bar, 64, 0, t.h, ids[u], t.l);
+              } else {
+                atomicOr(p.status, KVC_FLAG_BAD_PAGE);
+              }
+            }
+          }
+        }
+        if (t.has_coeff) {
+          const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
+#pragma unroll
+          for (int b = 0; b < RB; ++b) tma_load_3d(st_base + kBaseBytes + b * kCoeffBlkBytes, cmap, bar, 32 * b, t.t0, t.slab);
+        }
+      }
+      // drain: every load that was issued must have landed before the CTA may exit
+      const uint32_t issued = i;
+      for (uint32_t k = (issued > NSTAGE ? issued - NSTAGE : 0); k < issued; ++k)
+        mbar_wait_drain(smem_u32(&ctrl->full[k % NSTAGE]), (k / NSTAGE) & 1u);
+    }
+  } else if (warp == 1) {
+    // =============================================================== MMA issuer
+    if (lane == 0) {
+      TileWalker w;
+      w.init(&p, tile_begin, tile_end);
+      uint32_t i = 0, slabs = 0;
+      bool have_prev = false, in_slab = false;
+      Tile prev;
+      int slot = 0;
+      for (; !w.done(); w.next(), ++i) {
+        Tile t;
+        w.get(t);
+        const int s = i % NSTAGE, g = i & 1;
+        const uint32_t use = i / NSTAGE, acc_use = i >> 1;
+        const bool new_slab = !have_prev || !same_slab(prev, t);
+        if (new_slab) {
+          if (in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));   // all MMAs of the old slab done => slot free
+          in_slab = false;
+          if (t.uses_basis) {
+            slot = slabs % NB;
+            if (!mbar_wait(smem_u32(&ctrl->basis_full[slot]), (slabs / NB) & 1u, abort_flag)) break;
+            ++slabs;
+            in_slab = true;
+          }
+        }
+        prev = t;
+        have_prev = true;
+        if (!mbar_wait(smem_u32(&ctrl->conv[s]), use & 1u, abort_flag)) break;
+        if (!mbar_wait(smem_u32(&ctrl->acc_empty[g]), (acc_use & 1u) ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        if (t.has_coeff) {
+          const uint32_t d_tmem = tmem_base + g * 128;
+          const uint32_t a0 = stages + s * kStageBytes + kBaseBytes;
+          const uint32_t b0 = bases + slot * kBasisSlotBytes;
+          uint32_t acc = 0;
+#pragma unroll
+          for (int b = 0; b < RB; ++b) {
+            const uint64_t ad = umma_desc_sw128(a0 + b * kCoeffBlkBytes);
+            const uint64_t bd = umma_desc_sw128(b0 + b * kBasisBlkBytes);
+            // byte offsets inside the 128-byte row: c1 | c2 for A, B1 | B2 for B; 16 bf16 = 32 B per k-step
+            const int aoff[6] = {0, 32, 64, 96, 0, 32};
+            const int boff[6] = {0, 32, 0, 32, 64, 96};
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+              umma_bf16(d_tmem, ad + (uint64_t)(aoff[k] >> 4), bd + (uint64_t)(boff[k] >> 4), kIdescBf16M128N128, acc);
+              acc = 1;
+            }
+          }
+        }
+        umma_commit(smem_u32(&ctrl->mma_done[g]));
+      }
+      if (in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));
+      umma_commit(smem_u32(&ctrl->drain));
+      mbar_wait_drain(smem_u32(&ctrl->drain), 0);
+    }
+  } else if (warp == 2) {
+    // =============================================================== basis stager
+    TileWalker w;
+    w.init(&p, tile_begin, tile_end);
+    bool have_prev = false;
+    Tile prev;
+    uint32_t slabs = 0;
+    for (; !w.done(); w.next()) {
+      Tile t;
+      w.get(t);
+      const bool new_slab = !have_prev || !same_slab(prev, t);
+      prev = t;
+      have_prev = true;
+      if (!new_slab || !t.uses_basis) continue;
+      const int slot = slabs % NB;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->basis_empty[slot]), ((slabs / NB) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      ++slabs;
+      const DevItem& it = *t.it;
+      const int r = it.st.r;
+      const void* basis = t.is_v ? it.st.basis_v : it.st.basis_k;
+      uint8_t* slot_ptr = smem + NSTAGE * kStageBytes + slot * kBasisSlotBytes;
+      for (int b = 0; b < RB; ++b) {
+        for (int pass = 0; pass < 4; ++pass) {
+          const int ch = pass * 32 + lane;                 // operand row = channel
+          uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
+#pragma unroll
+          for (int k8 = 0; k8 < 4; ++k8) {
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int q = 32 * b + 8 * k8 + e;
+              float x = 0.f;
+              if (q < r) {
+                const int64_t off = ((int64_t)t.slab * r + q) * 128 + ch;
+                x = it.st.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
+                                     : reinterpret_cast<const float*>(basis)[off];
+              }
+              v[e] = x;
+            }
+            uint4 hi, lo;
+            uint32_t* hp = reinterpret_cast<uint32_t*>(&hi);
+            uint32_t* lp = reinterpret_cast<uint32_t*>(&lo);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * e]), h1 = __float2bfloat16_rn(v[2 * e + 1]);
+              const __nv_bfloat16 l0 = __float2bfloat16_rn(v[2 * e] - __bfloat162float(h0));
+              const __nv_bfloat16 l1 = __float2bfloat16_rn(v[2 * e + 1] - __bfloat162float(h1));
+              hp[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+              lp[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            }
+            *reinterpret_cast<uint4*>(row + (((k8) ^ (ch & 7)) << 4)) = hi;
+            *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
+          }
+        }
+      }
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
+    }
+  } else if (warp >= 4) {
+    // =============================================================== epilogue groups
+    const int g = (warp - 4) >> 2;                 // group 0: warps 4-7, group 1: warps 8-11
+    const int q = warp & 3;                        // TMEM lane quadrant of this warp
+    const int m = q * 32 + lane;                   // row of the tile = token
+    const int gt = tid - 128 - g * 128;            // thread index inside the group
+    const int bar_id = 1 + g;
+    const uint32_t sw = (uint32_t)(m & 7);
+    TileWalker w;
+    w.init(&p, tile_begin, tile_end);
+    uint32_t i = 0;
+    for (; !w.done(); w.next(), ++i) {
+      if ((int)(i & 1u) != g) continue;
+      Tile t;
+      w.get(t);
+      const int s = i % NSTAGE;
+      const uint32_t use = i / NSTAGE, acc_use = i >> 1;
+      const DevItem& it = *t.it;
+      uint8_t* st_ptr = smem + s * kStageBytes;
+
+      // ---- 1. tile landed
+      const bool ok1 = mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag);
+      if (named_bar_or(bar_id, 128, !ok1 || *abort_flag != 0)) break;
+
+      // ---- 2. coefficients: fp32 row -> bf16 [c1 | c2], in place
+      if (t.has_coeff) {
+#pragma unroll
+        for (int b = 0; b < RB; ++b) {
+          uint8_t* row = st_ptr + kBaseBytes + b * kCoeffBlkBytes + m * 128;
+          float c[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4*>(c + 4 * j) = *reinterpret_cast<const float4*>(row + ((j ^ sw) << 4));
+          uint32_t hi[16], lo[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(c[2 * e]), h1 = __float2bfloat16_rn(c[2 * e + 1]);
+            const __nv_bfloat16 l0 = __float2bfloat16_rn(c[2 * e] - __bfloat162float(h0));
+            const __nv_bfloat16 l1 = __float2bfloat16_rn(c[2 * e + 1] - __bfloat162float(h1));
+            hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            *reinterpret_cast<uint4*>(row + ((j ^ sw) << 4)) = make_uint4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+            *reinterpret_cast<uint4*>(row + (((4 + j) ^ sw) << 4)) = make_uint4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+          }
+        }
+        fence_proxy_async();
+      }
+      mbar_arrive(smem_u32(&ctrl->conv[s]));
+
+      // ---- 3. accumulator ready
+      const bool ok3 = mbar_wait(smem_u32(&ctrl->mma_done[g]), acc_use & 1u, abort_flag);
+      if (named_bar_or(bar_id, 128, !ok3 || *abort_flag != 0)) break;
+      tc_fence_after();
+
+      // ---- 4. rotate, add, round: row m, in place
+      const int tok = t.t0 + m;
+      const bool in_range = tok < it.src.T;
+      const bool covered = t.has_coeff && tok < it.st.n_cov;
+      const bool rotate = !t.is_v && it.shift != 0;
+      const bool work = in_range && (covered || rotate);
+      const uint32_t t_acc = tmem_base + g * 128 + ((uint32_t)(q * 32) << 16);
+      uint8_t* row0 = st_ptr + m * 128;
+      uint8_t* row1 = row0 + kHalfBytes;
+#pragma unroll
+      for (int pass = 0; pass < 2; ++pass) {
+        float a0[32], a1[32];
+        if (t.has_coeff) {
+          if (p.pairing == 0) {
+            tmem_ld32(t_acc + 32 * pass, a0);           // channels 32p .. 32p+31
+            tmem_ld32(t_acc + 64 + 32 * pass, a1);      // channels 64+32p ..
+          } else {
+            tmem_ld32(t_acc + 64 * pass, a0);           // channels 64p .. 64p+31
+            tmem_ld32(t_acc + 64 * pass + 32, a1);      // channels 64p+32 ..
+          }
+          tmem_ld_wait();
+        }
+        if (work) {
+          if (p.pairing == 0) {
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+              const int j = 4 * pass + jj;               // chunk of 8 channels inside each half
+              uint4* p0 = reinterpret_cast<uint4*>(row0 + ((j ^ sw) << 4));
+              uint4* p1 = reinterpret_cast<uint4*>(row1 + ((j ^ sw) << 4));
+              float x[16];
+              unpack8(*p0, x);
+              unpack8(*p1, x + 8);
+              if (rotate) {
+                const float4 c0 = *reinterpret_cast<const float4*>(it.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
+                const float4 s0 = *reinterpret_cast<const float4*>(it.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
+                const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const float u = x[e], v = x[8 + e];
+                  x[e] = u * cs[e] - v * sn[e];
+                  x[8 + e] = u * sn[e] + v * cs[e];
+                }
+              }
+              if (covered) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  x[e] += a0[8 * jj + e];
+                  x[8 + e] += a1[8 * jj + e];
+                }
+              }
+              *p0 = pack8(x);
+              *p1 = pack8(x + 8);
+            }
+          } else {
+            // interleaved pairs (2k, 2k+1): a0 / a1 hold 64 consecutive channels starting at 64*pass
+            uint8_t* rowp = pass == 0 ? row0 : row1;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              uint4* pp = reinterpret_cast<uint4*>(rowp + ((j ^ sw) << 4));
+              float x[8];
+              unpack8(*pp, x);
+              if (rotate) {
+                const int f0 = 32 * pass + 4 * j;        // pair index of the chunk's first pair
+                const float4 c0 = *reinterpret_cast<const float4*>(it.cs + f0);
+                const float4 s0 = *reinterpret_cast<const float4*>(it.sn + f0);
+                const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
+                const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float u = x[2 * e], v = x[2 * e + 1];
+                  x[2 * e] = u * cs[e] - v * sn[e];
+                  x[2 * e + 1] = u * sn[e] + v * cs[e];
+                }
+              }
+              if (covered) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) x[e] += (j < 4) ? a0[8 * j + e] : a1[8 * (j - 4) + e];
+              }
+              *pp = pack8(x);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
+
+      // ---- 5. rows of a partial last page go out with plain stores (rows >= T stay untouched)
+      const bool dst_paged = it.dst.page_table != nullptr;
+      const int dpage = it.dst.page_mask + 1;
+      const int last_pg = dst_paged ? ((it.dst.T - 1) >> it.dst.page_shift) : -1;
+      const bool last_partial = dst_paged && (it.dst.T & it.dst.page_mask) != 0;
+      if (last_partial && in_range && (tok >> it.dst.page_shift) == last_pg) {
+        __nv_bfloat16* drow = row_ptr(it.dst, t.is_v ? it.dst.v : it.dst.k, t.l, t.h, tok, p.status);
+        bool src_ok = true;
+        if (it.src.page_table) src_ok = (unsigned)it.src.page_table[tok >> it.src.page_shift] < (unsigned)it.src.n_phys;
+        if (drow && src_ok) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            *reinterpret_cast<uint4*>(drow + 8 * j) = *reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4));
+            *reinterpret_cast<uint4*>(drow + 64 + 8 * j) = *reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4));
+          }
+        }
+      }
+
+      // ---- 6. hand the finished tile to the TMA store, then release the stage
+      fence_proxy_async();
+      named_bar_sync(bar_id, 128);
+      if (gt == 0) {
+        const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
+        const uint32_t st_base = stages + s * kStageBytes;
+        if (!dst_paged) {
+          tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
+          tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
+        } else {
+          const int per_tile = kTileTok >> it.dst.page_shift;
+          const int first = t.t0 >> it.dst.page_shift;
+          const int n_pages = min(per_tile, ((it.dst.T + dpage - 1) >> it.dst.page_shift) - first);
+          int ids[16], sids[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            ids[u] = (u < n_pages) ? it.dst.page_table[first + u] : -1;
+            sids[u] = 0;
+          }
+          if (it.src.page_table) {
+            // a source page that could not be loaded must not be stored
+            const int sper = dpage >> it.src.page_shift;       // source pages per destination page (>= 1 when equal sizes)
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+              if (u < n_pages) {
+                const int tk = t.t0 + u * dpage;
+                const int np = max(sper, 1);
+                for (int e = 0; e < np; ++e) {
+                  const int spi = (tk >> it.src.page_shift) + e;
+                  if ((spi << it.src.page_shift) < it.src.T && (unsigned)it.src.page_table[spi] >= (unsigned)it.src.n_phys) sids[u] = 1;
+                }
+              }
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            if (u < n_pages) {
+              const bool partial = last_partial && (first + u) == last_pg;
+              if ((unsigned)ids[u] >= (unsigned)it.dst.n_phys) {
+                atomicOr(p.status, KVC_FLAG_BAD_PAGE);
+              } else if (!partial && !sids[u]) {
+                tma_store_5d(dmap, st_base + u * dpage * 128, 0, 0, t.h, ids[u], t.l);
+                tma_store_5d(dmap, st_base + kHalfBytes + u * dpage * 128, 64, 0, t.h, ids[u], t.l);
+              }
+            }
+          }
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(smem_u32(&ctrl->empty[s]));
+      }
+    }
+  }
+
+  // =============================================================== teardown
+  __syncthreads();
+  if (tid == 0 && *abort_flag) atomicOr(p.status, KVC_FLAG_WAIT_EXPIRED);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  }
+  return fn;
+}
+
+// 5-D view of a cache: (channel, token-in-unit, head, unit, layer); unit = page (paged) or the whole sequence.
+static bool encode_cache(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base, int L, int H) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const bool paged = c.page_table != nullptr;
+  const cuuint64_t rows = paged ? (cuuint64_t)(c.page_mask + 1) : (cuuint64_t)c.T;
+  const cuuint64_t units = paged ? (cuuint64_t)c.n_phys : 1;
+  const cuuint64_t dims[5] = {128, rows, (cuuint64_t)H, units, (cuuint64_t)L};
+  const cuuint64_t unit_stride = paged ? (cuuint64_t)c.s_page * 2 : (cuuint64_t)c.s_layer * 2;
+  const cuuint64_t strides[4] = {(cuuint64_t)c.s_tok * 2, (cuuint64_t)c.s_head * 2, unit_stride, (cuuint64_t)c.s_layer * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)(paged ? (c.page_mask + 1) : kTileTok), 1, 1, 1};
+  const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static bool encode_coeff(CUtensorMap* m, const float* coeff, int r, int n_cov, int slabs) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)r, (cuuint64_t)n_cov, (cuuint64_t)slabs};
+  const cuuint64_t strides[2] = {(cuuint64_t)r * 4, (cuuint64_t)r * 4 * (cuuint64_t)n_cov};
+  const cuuint32_t box[3] = {32, kTileTok, 1};
+  const cuuint32_t es[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(coeff), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Can this item run on the tensor-core path?
+static bool item_supported(const DevItem& it, int d) {
+  if (d != 128) return false;
+  if (it.st.r <= 0 || it.st.n_cov <= 0) return false;       // empty state: a copy / rotate, CUDA-core kernel
+  if (it.st.r > 64 || (it.st.r & 3)) return false;
+  for (const DevCache* c : {&it.src, &it.dst}) {
+    if (c->page_table) {
+      const int page = c->page_mask + 1;
+      if (page > 128) return false;
+    }
+    if (c->T >= (1 << 30)) return false;
+  }
+  if (it.src.page_table && it.dst.page_table && it.src.page_mask != it.dst.page_mask) return false;
+  return true;
+}
+
+static bool build_maps(const DevItem& it, ItemMaps* mp) {
+  bool ok = encode_cache(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
+            encode_cache(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
+  ok = ok && encode_coeff(&mp->coeff_k, it.st.coeff_k, it.st.r, it.st.n_cov, it.L * it.H) &&
+       encode_coeff(&mp->coeff_v, it.st.coeff_v, it.st.r, it.st.n_cov, it.L * it.H);
+  return ok;
+}
+
+template <int RB, int NSTAGE, int NB>
+static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
+  const size_t smem = 1024 + (size_t)NSTAGE * (kBaseBytes + RB * kCoeffBlkBytes) + (size_t)NB * RB * kBasisBlkBytes +
+                      sizeof(Ctrl<NSTAGE, NB>);
+  static bool set = false;
+  if (!set) {
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    set = true;
+  }
+  apply_tc_kernel<RB, NSTAGE, NB><<<grid, kThreads, smem, s>>>(L);
+  return cudaGetLastError();
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s) {
+  const int sms = sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+  cudaError_t e = (max_r <= 32) ? launch_t<1, 4, 2>(L, grid, s) : launch_t<2, 3, 1>(L, grid, s);
+  return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+}  // namespace tc
+
+static_assert(offsetof(DevItem, cs) % 16 == 0 && offsetof(DevItem, sn) % 16 == 0, "rope tables must be 16-byte aligned");
+
+int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s) {
+  if (!tc::item_supported(item, d) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  tc::ApplyTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.one = item;
+  L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
+  if (!tc::build_maps(L.one, &L.one_maps)) return KVC_E_CUDA;
+  L.n_items = 1;
+  L.pairing = pairing;
+  L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
+  L.status = status;
+  if (L.total_tiles == 0) return KVC_OK;
+  return tc::launch(L, item.st.r, s);
+}
+
+size_t tc_batch_extra_bytes(int n_items) { return 256 + (size_t)n_items * sizeof(tc::ItemMaps); }
+
+int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int d, int pairing, uint32_t* status, void* workspace,
+                   void* staging, size_t bytes, cudaStream_t s) {
+  if (!tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  int max_r = 0;
+  for (int i = 0; i < n_items; ++i) {
+    if (!tc::item_supported(tab[i], d)) return KVC_E_UNSUPPORTED;
+    max_r = tab[i].st.r > max_r ? tab[i].st.r : max_r;
+  }
+  // maps live after the item table, 256-byte aligned, at the same offset in staging and workspace
+  const size_t tab_off = reinterpret_cast<char*>(tab) - reinterpret_cast<char*>(staging);
+  const size_t maps_off = (tab_off + (size_t)n_items * sizeof(DevItem) + 255) & ~(size_t)255;
+  if (maps_off + (size_t)n_items * sizeof(tc::ItemMaps) > bytes) return KVC_E_WORKSPACE;
+  tc::ItemMaps* maps = reinterpret_cast<tc::ItemMaps*>(reinterpret_cast<char*>(staging) + maps_off);
+  int64_t total = 0;
+  for (int i = 0; i < n_items; ++i) {
+    prefix[i] = total;
+    tab[i].tiles_per_slab = (tab[i].src.T + tc::kTileTok - 1) / tc::kTileTok;
+    total += (int64_t)tab[i].L * tab[i].H * 2 * tab[i].tiles_per_slab;
+    if (!tc::build_maps(tab[i], &maps[i])) return KVC_E_CUDA;
+  }
+  prefix[n_items] = total;
+  if (total == 0) return KVC_OK;
+  const size_t copy = maps_off + (size_t)n_items * sizeof(tc::ItemMaps);
+  if (cudaMemcpyAsync(workspace, staging, copy, cudaMemcpyHostToDevice, s) != cudaSuccess) return KVC_E_CUDA;
+  tc::ApplyTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.tile_prefix = reinterpret_cast<const int64_t*>(workspace);
+  L.items = reinterpret_cast<const DevItem*>(reinterpret_cast<char*>(workspace) + tab_off);
+  L.maps = reinterpret_cast<const tc::ItemMaps*>(reinterpret_cast<char*>(workspace) + maps_off);
+  L.n_items = n_items;
+  L.pairing = pairing;
+  L.total_tiles = total;
+  L.status = status;
+  return tc::launch(L, max_r, s);
+}
+
+}  // namespace kvc

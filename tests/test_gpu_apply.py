@@ -43,6 +43,8 @@ def _run_hop(cfg, src_cpu, st_cpu, shift, path, dst_fill=None, in_place=False, p
     st = hp.state_to_dev(st_cpu, DEV)
     kvc.kvc_apply(src, st, shift, rope, dst)
     torch.cuda.synchronize()
+    if path == kvc.KVC_PATH_AUTO and cfg.d == 128 and 0 < st.r <= 64 and st.n_cov > 0 and cfg.T > 0:
+        assert kvc.kvc_last_path() == kvc.KVC_PATH_TC, "the TMA + tcgen05 kernels should have served this call"
     return src, dst
 
 
@@ -56,9 +58,11 @@ def _assert_parity(dst, ref_k, ref_v, odst):
     gk, gv = hp.logical_bits(dst, "k"), hp.logical_bits(dst, "v")
     rk, rv = hp.tol_ratio(gk, ref_k), hp.tol_ratio(gv, ref_v)
     assert rk <= 1.0 and rv <= 1.0, (rk, rv)
-    # almost every element is the oracle's own rounding
-    assert hp.ulp_mismatch_fraction(gk, hp.logical_bits(odst, "k")) < 2e-3
-    assert hp.ulp_mismatch_fraction(gv, hp.logical_bits(odst, "v")) < 2e-3
+    # sanity beside the tolerance: almost every element is the oracle's own rounding (the
+    # split-precision tensor-core contraction differs from float64 by ~1e-5, which flips a
+    # bf16 rounding in a few elements per thousand at rank 64)
+    assert hp.ulp_mismatch_fraction(gk, hp.logical_bits(odst, "k")) < 1e-2
+    assert hp.ulp_mismatch_fraction(gv, hp.logical_bits(odst, "v")) < 1e-2
 
 
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
