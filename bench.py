@@ -110,7 +110,7 @@ def _dist():
 # --------------------------------------------------------------------------------------
 
 
-def build_workload(cfg: wl.Config, dev, kvc):
+def build_workload(cfg: wl.Config, dev, kvc, only="all"):
     """Everything one step reads, resident on the device.  Draws come from the seeded
     generator; the true target caches are derived with the library itself (aligned
     source + exact rank-r deviation, then N(0, sigma) noise, rounded to bf16)."""
@@ -130,6 +130,14 @@ def build_workload(cfg: wl.Config, dev, kvc):
         tables = [None] * (2 * n)
         a0 = kvc.Cache(k0, v0)
     true = [a0]
+    if only == "apply":
+        # the chain alone: the generator's states are applied directly, no targets needed
+        states = []
+        for a in range(1, n):
+            s = wl.hop_state(cfg, a, dev)
+            states.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
+        outs = [mk(tables[n + a]) for a in range(1, n)]
+        return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": None, "only": only}
     for a in range(1, n):
         s = wl.hop_state(cfg, a, dev)
         st = kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"])
@@ -151,7 +159,7 @@ def build_workload(cfg: wl.Config, dev, kvc):
                         torch.empty(L, H, r, d, device=dev), torch.empty(L, H, r, d, device=dev)) for _ in range(n - 1)]
     outs = [mk(tables[n + a]) for a in range(1, n)]
     ws = torch.empty(max(kvc.kvc_workspace_bytes(a0, states[0], kvc.KVC_FIT), 256), dtype=torch.uint8, device=dev)
-    return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws}
+    return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws, "only": only}
 
 
 def run_step(W, kvc, ev=None):
@@ -166,20 +174,25 @@ def run_step(W, kvc, ev=None):
         ev.setdefault(name, []).append(e)
         return e
 
-    for a in range(1, n):
-        mark("update_begin")
-        kvc.kvc_state_update(W["true"][a - 1], W["true"][a], pl[a] - pl[a - 1], rope, W["states"][a - 1], kvc.KVC_FIT,
-                             workspace=W["ws"])
-        mark("update_end")
-    mark("chain_begin")
-    kvc.kvc_chain(W["true"][0], pl, W["states"], rope, W["outs"])
-    mark("chain_end")
+    only = W.get("only", "all")
+    if only != "apply":
+        for a in range(1, n):
+            mark("update_begin")
+            kvc.kvc_state_update(W["true"][a - 1], W["true"][a], pl[a] - pl[a - 1], rope, W["states"][a - 1],
+                                 kvc.KVC_FIT, workspace=W["ws"])
+            mark("update_end")
+    if only != "update":
+        mark("chain_begin")
+        kvc.kvc_chain(W["true"][0], pl, W["states"], rope, W["outs"])
+        mark("chain_end")
 
 
 def step_bytes(W, kvc):
-    n = len(W["true"])
-    upd = sum(kvc.kvc_update_bytes(W["true"][a], W["states"][a - 1], kvc.KVC_FIT, True) for a in range(1, n))
-    app = sum(kvc.kvc_apply_bytes(W["true"][0], W["states"][a - 1]) for a in range(1, n))
+    n = len(W["states"]) + 1
+    only = W.get("only", "all")
+    upd = 0 if only == "apply" else sum(kvc.kvc_update_bytes(W["true"][0], W["states"][a - 1], kvc.KVC_FIT, True)
+                                         for a in range(1, n))
+    app = 0 if only == "update" else sum(kvc.kvc_apply_bytes(W["true"][0], W["states"][a - 1]) for a in range(1, n))
     return upd, app
 
 
@@ -241,13 +254,19 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
+    ap.add_argument("--only", default="all", choices=["all", "apply", "update"],
+                    help="profiling aid: time only the chain or only the state updates")
     args = ap.parse_args()
     rank, world, local = _dist()
     cfg = wl.CONFIGS[args.workload]
+    if args.layers > 0:
+        cfg = cfg.scaled(L=args.layers)
     config = {"workload": f"{cfg.name}: L={cfg.L} Hkv={cfg.H} d={cfg.d} T={cfg.T} agents={cfg.n_agents} r={cfg.r} "
                           f"{'paged16' if cfg.paged else 'contiguous'} bf16, seed {cfg.seed}",
               "step": "per edge: kvc_state_update(FIT) ; then kvc_chain over all agents",
-              "l2": "inputs larger than L2 (every pass streams > 1 GiB)", "parallelism": f"replicas x{world}"}
+              "l2": "inputs larger than L2 (126 MB): no flush between iterations", "parallelism": f"replicas x{world}",
+              "only": args.only}
 
     if args.impl == "reference":
         if rank != 0:
@@ -282,7 +301,9 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     kvc.kvc_set_path({"auto": kvc.KVC_PATH_AUTO, "generic": kvc.KVC_PATH_GENERIC, "tc": kvc.KVC_PATH_TC}[args.path])
 
-    W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
+    W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only)
+    if args.only != "all":
+        args.no_e2e = True
     upd_b, app_b = step_bytes(W, kvc)
     hops = cfg.n_agents - 1
 
@@ -307,8 +328,9 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms_total = t_begin.elapsed_time(t_end)
-    chain_ms = sum(b.elapsed_time(e) for b, e in zip(ev["chain_begin"], ev["chain_end"])) / args.steps
-    upd_ms = sum(b.elapsed_time(e) for b, e in zip(ev["update_begin"], ev["update_end"])) / args.steps
+    chain_ms = sum(b.elapsed_time(e) for b, e in zip(ev.get("chain_begin", []), ev.get("chain_end", []))) / args.steps
+    upd_ms = sum(b.elapsed_time(e) for b, e in zip(ev.get("update_begin", []), ev.get("update_end", []))) / args.steps
+    chain_ms, upd_ms = max(chain_ms, 1e-9), max(upd_ms, 1e-9)
     last_path = kvc.kvc_last_path()
     flags = kvc.kvc_status_poll()
     assert flags == 0, f"a kernel flagged an anomaly: {flags}"

@@ -27,7 +27,9 @@ struct DevState {
 };
 
 // One hop over one request: what kvc_apply does for all (layer, head, token).
-struct DevItem {
+// 16-byte aligned so that the cos / sin tables can be read as float4 wherever the
+// struct sits (kernel parameter space or a device table).
+struct alignas(16) DevItem {
   DevCache src, dst;
   DevState st;
   int32_t shift, L, H, tiles_per_slab;   // tiles_per_slab = ceil(T / tile)

@@ -30,7 +30,8 @@ namespace kvc {
 namespace tc {
 
 constexpr int kTileTok = 128;
-constexpr int kThreads = 384;
+constexpr int kThreads = 640;
+constexpr int kTeamThreads = 512;
 constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a base tile (bf16)
 constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
 constexpr int kCoeffBlkBytes = kTileTok * 128;    // 128 tokens x 32 fp32 (one rank block)
@@ -187,6 +188,15 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
 // kind::f16, A = B = bf16, D = f32, both K-major, M = 128, N = 128
 constexpr uint32_t kIdescBf16M128N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi), for two values, packed as bf16x2 words
+__device__ __forceinline__ void split2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+  const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+  const __nv_bfloat16 l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+
 // ------------------------------------------------------------------ tile bookkeeping
 struct Tile {
   const DevItem* it;
@@ -253,7 +263,7 @@ __device__ __forceinline__ bool same_slab(const Tile& a, const Tile& b) {
 // Shared-memory control block (after the tiles)
 template <int NSTAGE, int NB>
 struct Ctrl {
-  uint64_t full[NSTAGE], conv[NSTAGE], empty[NSTAGE];
+  uint64_t full[NSTAGE], conv[NSTAGE], ready[NSTAGE], empty[NSTAGE];
   uint64_t mma_done[2], acc_empty[2];
   uint64_t basis_full[NB], basis_empty[NB];
   uint64_t drain;
@@ -261,7 +271,21 @@ struct Ctrl {
   int abort_flag;
 };
 
+// 16 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
 // ------------------------------------------------------------------ the kernel
+// Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 basis stager, 3 store warp, 4..19 the team.
+// Team warp e (0..15): TMEM lane quadrant e & 3 (rows 32q..32q+31), channel quarter e >> 2.
 template <int RB, int NSTAGE, int NB>
 __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
   constexpr int kStageBytes = kBaseBytes + RB * kCoeffBlkBytes;
@@ -283,12 +307,13 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
   if (tid == 0) {
     for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(smem_u32(&ctrl->full[s]), 1);
-      mbar_init(smem_u32(&ctrl->conv[s]), 128);
+      mbar_init(smem_u32(&ctrl->conv[s]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->ready[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
-      mbar_init(smem_u32(&ctrl->acc_empty[g]), 128);
+      mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
     }
     for (int b = 0; b < NB; ++b) {
       mbar_init(smem_u32(&ctrl->basis_full[b]), 1);
@@ -309,59 +334,57 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
   const uint32_t tmem_base = ctrl->tmem_base;
 
   if (warp == 0) {
-    // =============================================================== TMA producer
-    if (lane == 0) {
-      TileWalker w;
-      w.init(&p, tile_begin, tile_end);
-      uint32_t i = 0;
-      for (; !w.done(); w.next(), ++i) {
-        Tile t;
-        w.get(t);
-        const int s = i % NSTAGE;
-        const uint32_t use = i / NSTAGE;
-        if (!mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag)) break;
-        const DevItem& it = *t.it;
-        const uint32_t st_base = stages + s * kStageBytes;
-        const uint32_t bar = smem_u32(&ctrl->full[s]);
-        const CUtensorMap* smap = t.is_v ? &t.mp->src_v : &t.mp->src_k;
-        uint32_t bytes = t.has_coeff ? RB * kCoeffBlkBytes : 0;
-        if (!it.src.page_table) {
-          bytes += kBaseBytes;
-          mbar_expect_tx(bar, bytes);
+    // =============================================================== TMA producer (whole warp)
+    TileWalker w;
+    w.init(&p, tile_begin, tile_end);
+    uint32_t i = 0;
+    for (; !w.done(); w.next(), ++i) {
+      Tile t;
+      w.get(t);
+      const int s = i % NSTAGE;
+      const uint32_t use = i / NSTAGE;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const DevItem& it = *t.it;
+      const uint32_t st_base = stages + s * kStageBytes;
+      const uint32_t bar = smem_u32(&ctrl->full[s]);
+      const CUtensorMap* smap = t.is_v ? &t.mp->src_v : &t.mp->src_k;
+      const uint32_t cbytes = t.has_coeff ? RB * kCoeffBlkBytes : 0;
+      if (!it.src.page_table) {
+        if (lane == 0) {
+          mbar_expect_tx(bar, cbytes + kBaseBytes);
           tma_load_5d(st_base, smap, bar, 0, t.t0, t.h, 0, t.l);
           tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t.t0, t.h, 0, t.l);
-        } else {
-          const int page = it.src.page_mask + 1;
-          const int per_tile = kTileTok >> it.src.page_shift;
-          const int first = t.t0 >> it.src.page_shift;
-          const int n_pages = min(per_tile, ((it.src.T + page - 1) >> it.src.page_shift) - first);
-          int ids[16];
-#pragma unroll
-          for (int u = 0; u < 16; ++u) ids[u] = (u < n_pages) ? it.src.page_table[first + u] : -1;
-          int n_ok = 0;
-#pragma unroll
-          for (int u = 0; u < 16; ++u) n_ok += (u < n_pages) && ((unsigned)ids[u] < (unsigned)it.src.n_phys);
-          bytes += n_ok * page * 256;
-          mbar_expect_tx(bar, bytes);
-#pragma unroll
-          for (int u = 0; u < 16; ++u) {
-            if (u < n_pages) {
-              if ((unsigned)ids[u] < (unsigned)it.src.n_phys) {
-                tma_load_5d(st_base + u * page * 128, smap, bar, 0, 0, t.h, ids[u], t.l);
-                tma_load_5d(st_base + kHalfBytes + u * page * 128, smap, bar, 64, 0, t.h, ids[u], t.l);
-              } else {
-                atomicOr(p.status, KVC_FLAG_BAD_PAGE);
-              }
-            }
-          }
         }
-        if (t.has_coeff) {
-          const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
-#pragma unroll
-          for (int b = 0; b < RB; ++b) tma_load_3d(st_base + kBaseBytes + b * kCoeffBlkBytes, cmap, bar, 32 * b, t.t0, t.slab);
+      } else {
+        // one lane per page of the tile
+        const int page = it.src.page_mask + 1;
+        const int per_tile = kTileTok >> it.src.page_shift;
+        const int first = t.t0 >> it.src.page_shift;
+        const int n_pages = min(per_tile, ((it.src.T + page - 1) >> it.src.page_shift) - first);
+        int id = -1;
+        if (lane < n_pages) id = it.src.page_table[first + lane];
+        const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.src.n_phys;
+        if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
+        const int n_ok = __popc(__ballot_sync(0xffffffffu, valid));
+        if (lane == 0) mbar_expect_tx(bar, cbytes + (uint32_t)(n_ok * page * 256));
+        __syncwarp();
+        if (valid) {
+          tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, t.h, id, t.l);
+          tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, t.h, id, t.l);
         }
       }
-      // drain: every load that was issued must have landed before the CTA may exit
+      if (t.has_coeff && lane == 0) {
+        const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
+#pragma unroll
+        for (int b = 0; b < RB; ++b) tma_load_3d(st_base + kBaseBytes + b * kCoeffBlkBytes, cmap, bar, 32 * b, t.t0, t.slab);
+      }
+      __syncwarp();
+    }
+    // drain: every load that was issued must have landed before the CTA may exit
+    if (lane == 0) {
       const uint32_t issued = i;
       for (uint32_t k = (issued > NSTAGE ? issued - NSTAGE : 0); k < issued; ++k)
         mbar_wait_drain(smem_u32(&ctrl->full[k % NSTAGE]), (k / NSTAGE) & 1u);
@@ -467,13 +490,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             uint32_t* hp = reinterpret_cast<uint32_t*>(&hi);
             uint32_t* lp = reinterpret_cast<uint32_t*>(&lo);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * e]), h1 = __float2bfloat16_rn(v[2 * e + 1]);
-              const __nv_bfloat16 l0 = __float2bfloat16_rn(v[2 * e] - __bfloat162float(h0));
-              const __nv_bfloat16 l1 = __float2bfloat16_rn(v[2 * e + 1] - __bfloat162float(h1));
-              hp[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-              lp[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-            }
+            for (int e = 0; e < 4; ++e) split2(v[2 * e], v[2 * e + 1], hp[e], lp[e]);
             *reinterpret_cast<uint4*>(row + (((k8) ^ (ch & 7)) << 4)) = hi;
             *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
           }
@@ -483,219 +500,233 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
     }
-  } else if (warp >= 4) {
-    // =============================================================== epilogue groups
-    const int g = (warp - 4) >> 2;                 // group 0: warps 4-7, group 1: warps 8-11
-    const int q = warp & 3;                        // TMEM lane quadrant of this warp
-    const int m = q * 32 + lane;                   // row of the tile = token
-    const int gt = tid - 128 - g * 128;            // thread index inside the group
-    const int bar_id = 1 + g;
-    const uint32_t sw = (uint32_t)(m & 7);
+  } else if (warp == 3) {
+    // =============================================================== store warp
     TileWalker w;
     w.init(&p, tile_begin, tile_end);
     uint32_t i = 0;
     for (; !w.done(); w.next(), ++i) {
-      if ((int)(i & 1u) != g) continue;
       Tile t;
       w.get(t);
       const int s = i % NSTAGE;
-      const uint32_t use = i / NSTAGE, acc_use = i >> 1;
+      const uint32_t use = i / NSTAGE;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), use & 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
       const DevItem& it = *t.it;
+      const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
+      const uint32_t st_base = stages + s * kStageBytes;
       uint8_t* st_ptr = smem + s * kStageBytes;
+      if (!it.dst.page_table) {
+        bool src_ok = true;   // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
+        if (lane == 0 && src_ok) {
+          tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
+          tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
+        }
+      } else {
+        // one lane per destination page; the last, partial page goes out row by row so that
+        // rows >= T stay untouched; pages whose source could not be loaded are skipped
+        const int dpage = it.dst.page_mask + 1;
+        const int per_tile = kTileTok >> it.dst.page_shift;
+        const int first = t.t0 >> it.dst.page_shift;
+        const int n_pages = min(per_tile, ((it.dst.T + dpage - 1) >> it.dst.page_shift) - first);
+        const int last_pg = (it.dst.T - 1) >> it.dst.page_shift;
+        const bool last_partial = (it.dst.T & it.dst.page_mask) != 0;
+        int id = -1;
+        bool src_ok = true;
+        if (lane < n_pages) {
+          id = it.dst.page_table[first + lane];
+          if (it.src.page_table) {
+            const int tk0 = t.t0 + lane * dpage;
+            const int tk1 = min(tk0 + dpage, it.src.T);
+            for (int sp = tk0 >> it.src.page_shift; (sp << it.src.page_shift) < tk1; ++sp)
+              if ((unsigned)it.src.page_table[sp] >= (unsigned)it.src.n_phys) src_ok = false;
+          }
+        }
+        const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.dst.n_phys;
+        if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
+        const bool partial = last_partial && (first + lane) == last_pg;
+        if (valid && src_ok && !partial) {
+          tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, t.h, id, t.l);
+          tma_store_5d(dmap, st_base + kHalfBytes + lane * dpage * 128, 64, 0, t.h, id, t.l);
+        }
+        // the partial page, if this tile holds it: which lane owns it, is it storable
+        const unsigned pm = __ballot_sync(0xffffffffu, valid && src_ok && partial);
+        if (pm) {
+          const int u = __ffs(pm) - 1;
+          const int rows = it.dst.T & it.dst.page_mask;
+          __nv_bfloat16* dbase = t.is_v ? it.dst.v : it.dst.k;
+          for (int c = lane; c < rows * 16; c += 32) {
+            const int row = u * dpage + (c >> 4), half = (c >> 3) & 1, j = c & 7;
+            __nv_bfloat16* drow = row_ptr(it.dst, dbase, t.l, t.h, t.t0 + row, p.status);
+            if (drow)
+              *reinterpret_cast<uint4*>(drow + half * 64 + j * 8) =
+                  *reinterpret_cast<const uint4*>(st_ptr + half * kHalfBytes + row * 128 + ((j ^ (row & 7)) << 4));
+          }
+        }
+      }
+      tma_store_commit();
+      tma_store_wait_read();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[s]));
+    }
+  } else {
+    // =============================================================== the team (16 warps)
+    const int e = warp - 4;
+    const int q = e & 3;                           // TMEM lane quadrant (== hardware warp id & 3)
+    const int cq = e >> 2;                         // channel quarter
+    const int m = q * 32 + lane;                   // epilogue row = token of the tile
+    const uint32_t sw = (uint32_t)(m & 7);
+    // conversion mapping: the four threads of a coefficient row sit in one warp
+    const int crow = e * 8 + (lane >> 2), cpart = lane & 3;
+    const uint32_t csw = (uint32_t)(crow & 7);
 
-      // ---- 1. tile landed
-      const bool ok1 = mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag);
-      if (named_bar_or(bar_id, 128, !ok1 || *abort_flag != 0)) break;
+    TileWalker w;
+    w.init(&p, tile_begin, tile_end);
+    TileWalker wn = w;                              // runs one tile ahead (conversion)
+    uint32_t i = 0;
+    bool alive = true;
 
-      // ---- 2. coefficients: fp32 row -> bf16 [c1 | c2], in place
+    // conversion of tile index `ci` held by walker `cw`
+    auto convert = [&](TileWalker& cw, uint32_t ci) {
+      Tile t;
+      cw.get(t);
+      const int s = ci % NSTAGE;
+      const uint32_t use = ci / NSTAGE;
+      bool ok = mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return false;
       if (t.has_coeff) {
+        uint8_t* st_ptr = smem + s * kStageBytes;
 #pragma unroll
         for (int b = 0; b < RB; ++b) {
-          uint8_t* row = st_ptr + kBaseBytes + b * kCoeffBlkBytes + m * 128;
-          float c[32];
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<float4*>(c + 4 * j) = *reinterpret_cast<const float4*>(row + ((j ^ sw) << 4));
-          uint32_t hi[16], lo[16];
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const __nv_bfloat16 h0 = __float2bfloat16_rn(c[2 * e]), h1 = __float2bfloat16_rn(c[2 * e + 1]);
-            const __nv_bfloat16 l0 = __float2bfloat16_rn(c[2 * e] - __bfloat162float(h0));
-            const __nv_bfloat16 l1 = __float2bfloat16_rn(c[2 * e + 1] - __bfloat162float(h1));
-            hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-            lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            *reinterpret_cast<uint4*>(row + ((j ^ sw) << 4)) = make_uint4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
-            *reinterpret_cast<uint4*>(row + (((4 + j) ^ sw) << 4)) = make_uint4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
-          }
+          uint8_t* row = st_ptr + kBaseBytes + b * kCoeffBlkBytes + crow * 128;
+          // this thread's 8 coefficients: fp32 chunks 2*cpart, 2*cpart+1 of the row
+          const float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
+          const float4 f1 = *reinterpret_cast<const float4*>(row + (((2 * cpart + 1) ^ csw) << 4));
+          uint4 hi, lo;
+          split2(f0.x, f0.y, hi.x, lo.x);
+          split2(f0.z, f0.w, hi.y, lo.y);
+          split2(f1.x, f1.y, hi.z, lo.z);
+          split2(f1.z, f1.w, hi.w, lo.w);
+          __syncwarp();                               // all four threads of the row have read
+          *reinterpret_cast<uint4*>(row + ((cpart ^ csw) << 4)) = hi;         // c1: chunks 0..3
+          *reinterpret_cast<uint4*>(row + (((4 + cpart) ^ csw) << 4)) = lo;   // c2: chunks 4..7
         }
         fence_proxy_async();
       }
       mbar_arrive(smem_u32(&ctrl->conv[s]));
+      return true;
+    };
 
-      // ---- 3. accumulator ready
-      const bool ok3 = mbar_wait(smem_u32(&ctrl->mma_done[g]), acc_use & 1u, abort_flag);
-      if (named_bar_or(bar_id, 128, !ok3 || *abort_flag != 0)) break;
+    if (!w.done()) alive = convert(wn, 0);
+    for (; alive && !w.done(); w.next(), ++i) {
+      // ---- 1. get the next tile's coefficients converted and its MMA going
+      wn.next();
+      if (!wn.done()) {
+        if (!convert(wn, i + 1)) break;
+      }
+      Tile t;
+      w.get(t);
+      const int s = i % NSTAGE, g = i & 1;
+      const uint32_t acc_use = i >> 1;
+      const DevItem& it = *t.it;
+      uint8_t* st_ptr = smem + s * kStageBytes;
+
+      // ---- 2. accumulator of this tile ready
+      bool ok = mbar_wait(smem_u32(&ctrl->mma_done[g]), acc_use & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
 
-      // ---- 4. rotate, add, round: row m, in place
+      // ---- 3. rotate, add, round: row m, this warp's channel quarter, in place
       const int tok = t.t0 + m;
       const bool in_range = tok < it.src.T;
       const bool covered = t.has_coeff && tok < it.st.n_cov;
       const bool rotate = !t.is_v && it.shift != 0;
       const bool work = in_range && (covered || rotate);
       const uint32_t t_acc = tmem_base + g * 128 + ((uint32_t)(q * 32) << 16);
-      uint8_t* row0 = st_ptr + m * 128;
-      uint8_t* row1 = row0 + kHalfBytes;
-#pragma unroll
-      for (int pass = 0; pass < 2; ++pass) {
-        float a0[32], a1[32];
-        if (t.has_coeff) {
-          if (p.pairing == 0) {
-            tmem_ld32(t_acc + 32 * pass, a0);           // channels 32p .. 32p+31
-            tmem_ld32(t_acc + 64 + 32 * pass, a1);      // channels 64+32p ..
-          } else {
-            tmem_ld32(t_acc + 64 * pass, a0);           // channels 64p .. 64p+31
-            tmem_ld32(t_acc + 64 * pass + 32, a1);      // channels 64p+32 ..
-          }
-          tmem_ld_wait();
+      float a0[16], a1[16];
+      if (t.has_coeff) {
+        if (p.pairing == 0) {
+          tmem_ld16(t_acc + 16 * cq, a0);             // channels 16cq .. 16cq+15
+          tmem_ld16(t_acc + 64 + 16 * cq, a1);        // channels 64+16cq ..
+        } else {
+          tmem_ld16(t_acc + 32 * cq, a0);             // channels 32cq .. 32cq+15
+          tmem_ld16(t_acc + 32 * cq + 16, a1);        // channels 32cq+16 ..
         }
-        if (work) {
-          if (p.pairing == 0) {
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-              const int j = 4 * pass + jj;               // chunk of 8 channels inside each half
-              uint4* p0 = reinterpret_cast<uint4*>(row0 + ((j ^ sw) << 4));
-              uint4* p1 = reinterpret_cast<uint4*>(row1 + ((j ^ sw) << 4));
-              float x[16];
-              unpack8(*p0, x);
-              unpack8(*p1, x + 8);
-              if (rotate) {
-                const float4 c0 = *reinterpret_cast<const float4*>(it.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
-                const float4 s0 = *reinterpret_cast<const float4*>(it.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
-                const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-                const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const float u = x[e], v = x[8 + e];
-                  x[e] = u * cs[e] - v * sn[e];
-                  x[8 + e] = u * sn[e] + v * cs[e];
-                }
-              }
-              if (covered) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  x[e] += a0[8 * jj + e];
-                  x[8 + e] += a1[8 * jj + e];
-                }
-              }
-              *p0 = pack8(x);
-              *p1 = pack8(x + 8);
-            }
-          } else {
-            // interleaved pairs (2k, 2k+1): a0 / a1 hold 64 consecutive channels starting at 64*pass
-            uint8_t* rowp = pass == 0 ? row0 : row1;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              uint4* pp = reinterpret_cast<uint4*>(rowp + ((j ^ sw) << 4));
-              float x[8];
-              unpack8(*pp, x);
-              if (rotate) {
-                const int f0 = 32 * pass + 4 * j;        // pair index of the chunk's first pair
-                const float4 c0 = *reinterpret_cast<const float4*>(it.cs + f0);
-                const float4 s0 = *reinterpret_cast<const float4*>(it.sn + f0);
-                const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
-                const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float u = x[2 * e], v = x[2 * e + 1];
-                  x[2 * e] = u * cs[e] - v * sn[e];
-                  x[2 * e + 1] = u * sn[e] + v * cs[e];
-                }
-              }
-              if (covered) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) x[e] += (j < 4) ? a0[8 * j + e] : a1[8 * (j - 4) + e];
-              }
-              *pp = pack8(x);
-            }
-          }
-        }
+        tmem_ld_wait();
       }
       tc_fence_before();
       mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
-
-      // ---- 5. rows of a partial last page go out with plain stores (rows >= T stay untouched)
-      const bool dst_paged = it.dst.page_table != nullptr;
-      const int dpage = it.dst.page_mask + 1;
-      const int last_pg = dst_paged ? ((it.dst.T - 1) >> it.dst.page_shift) : -1;
-      const bool last_partial = dst_paged && (it.dst.T & it.dst.page_mask) != 0;
-      if (last_partial && in_range && (tok >> it.dst.page_shift) == last_pg) {
-        __nv_bfloat16* drow = row_ptr(it.dst, t.is_v ? it.dst.v : it.dst.k, t.l, t.h, tok, p.status);
-        bool src_ok = true;
-        if (it.src.page_table) src_ok = (unsigned)it.src.page_table[tok >> it.src.page_shift] < (unsigned)it.src.n_phys;
-        if (drow && src_ok) {
+      if (work) {
+        if (p.pairing == 0) {
+          uint8_t* row0 = st_ptr + m * 128;
+          uint8_t* row1 = row0 + kHalfBytes;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            *reinterpret_cast<uint4*>(drow + 8 * j) = *reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4));
-            *reinterpret_cast<uint4*>(drow + 64 + 8 * j) = *reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4));
+          for (int jj = 0; jj < 2; ++jj) {
+            const int j = 2 * cq + jj;                 // chunk of 8 channels inside each half
+            uint4* p0 = reinterpret_cast<uint4*>(row0 + ((j ^ sw) << 4));
+            uint4* p1 = reinterpret_cast<uint4*>(row1 + ((j ^ sw) << 4));
+            float x[16];
+            unpack8(*p0, x);
+            unpack8(*p1, x + 8);
+            if (rotate) {
+              const float4 c0 = *reinterpret_cast<const float4*>(it.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
+              const float4 s0 = *reinterpret_cast<const float4*>(it.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
+              const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+              const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const float u = x[k], v = x[8 + k];
+                x[k] = u * cs[k] - v * sn[k];
+                x[8 + k] = u * sn[k] + v * cs[k];
+              }
+            }
+            if (covered) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                x[k] += a0[8 * jj + k];
+                x[8 + k] += a1[8 * jj + k];
+              }
+            }
+            *p0 = pack8(x);
+            *p1 = pack8(x + 8);
           }
-        }
-      }
-
-      // ---- 6. hand the finished tile to the TMA store, then release the stage
-      fence_proxy_async();
-      named_bar_sync(bar_id, 128);
-      if (gt == 0) {
-        const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
-        const uint32_t st_base = stages + s * kStageBytes;
-        if (!dst_paged) {
-          tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
-          tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
         } else {
-          const int per_tile = kTileTok >> it.dst.page_shift;
-          const int first = t.t0 >> it.dst.page_shift;
-          const int n_pages = min(per_tile, ((it.dst.T + dpage - 1) >> it.dst.page_shift) - first);
-          int ids[16], sids[16];
+          // interleaved pairs (2k, 2k+1): 32 consecutive channels 32cq .. 32cq+31
+          uint8_t* rowp = st_ptr + (cq >> 1) * kHalfBytes + m * 128;
 #pragma unroll
-          for (int u = 0; u < 16; ++u) {
-            ids[u] = (u < n_pages) ? it.dst.page_table[first + u] : -1;
-            sids[u] = 0;
-          }
-          if (it.src.page_table) {
-            // a source page that could not be loaded must not be stored
-            const int sper = dpage >> it.src.page_shift;       // source pages per destination page (>= 1 when equal sizes)
+          for (int jj = 0; jj < 4; ++jj) {
+            const int j = 4 * (cq & 1) + jj;           // chunk inside the half
+            uint4* pp = reinterpret_cast<uint4*>(rowp + ((j ^ sw) << 4));
+            float x[8];
+            unpack8(*pp, x);
+            if (rotate) {
+              const int f0 = 16 * cq + 4 * jj;         // pair index of the chunk's first pair
+              const float4 c0 = *reinterpret_cast<const float4*>(it.cs + f0);
+              const float4 s0 = *reinterpret_cast<const float4*>(it.sn + f0);
+              const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
+              const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
-              if (u < n_pages) {
-                const int tk = t.t0 + u * dpage;
-                const int np = max(sper, 1);
-                for (int e = 0; e < np; ++e) {
-                  const int spi = (tk >> it.src.page_shift) + e;
-                  if ((spi << it.src.page_shift) < it.src.T && (unsigned)it.src.page_table[spi] >= (unsigned)it.src.n_phys) sids[u] = 1;
-                }
+              for (int k = 0; k < 4; ++k) {
+                const float u = x[2 * k], v = x[2 * k + 1];
+                x[2 * k] = u * cs[k] - v * sn[k];
+                x[2 * k + 1] = u * sn[k] + v * cs[k];
               }
             }
-          }
+            if (covered) {
 #pragma unroll
-          for (int u = 0; u < 16; ++u) {
-            if (u < n_pages) {
-              const bool partial = last_partial && (first + u) == last_pg;
-              if ((unsigned)ids[u] >= (unsigned)it.dst.n_phys) {
-                atomicOr(p.status, KVC_FLAG_BAD_PAGE);
-              } else if (!partial && !sids[u]) {
-                tma_store_5d(dmap, st_base + u * dpage * 128, 0, 0, t.h, ids[u], t.l);
-                tma_store_5d(dmap, st_base + kHalfBytes + u * dpage * 128, 64, 0, t.h, ids[u], t.l);
-              }
+              for (int k = 0; k < 8; ++k) x[k] += (jj < 2) ? a0[8 * jj + k] : a1[8 * (jj - 2) + k];
             }
+            *pp = pack8(x);
           }
         }
-        tma_store_commit();
-        tma_store_wait_read();
-        mbar_arrive(smem_u32(&ctrl->empty[s]));
       }
+      // ---- 4. the tile is final in shared memory: hand it to the store warp
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&ctrl->ready[s]));
     }
   }
 
@@ -768,7 +799,6 @@ static bool item_supported(const DevItem& it, int d) {
     }
     if (c->T >= (1 << 30)) return false;
   }
-  if (it.src.page_table && it.dst.page_table && it.src.page_mask != it.dst.page_mask) return false;
   return true;
 }
 
@@ -815,6 +845,9 @@ static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s) {
 }  // namespace tc
 
 static_assert(offsetof(DevItem, cs) % 16 == 0 && offsetof(DevItem, sn) % 16 == 0, "rope tables must be 16-byte aligned");
+static_assert(alignof(DevItem) >= 16 && sizeof(DevItem) % 16 == 0, "items in a table keep the alignment");
+static_assert(offsetof(tc::ApplyTcLaunch, one) % 16 == 0, "the by-value item must keep the alignment");
+static_assert(offsetof(tc::ApplyTcLaunch, one_maps) % 64 == 0, "tensor maps need 64-byte alignment");
 
 int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s) {
   if (!tc::item_supported(item, d) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
