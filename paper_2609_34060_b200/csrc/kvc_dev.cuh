@@ -54,7 +54,8 @@ struct UpdateLaunch {
   int32_t r, n_cov, basis_bf16, pairing;
   int32_t shift, L, H, tiles_per_slab;
   uint32_t* status;
-  float cs[kMaxHalfD], sn[kMaxHalfD];
+  alignas(16) float cs[kMaxHalfD];
+  alignas(16) float sn[kMaxHalfD];
 };
 
 struct FitLaunch {             // Gram + eigensolve
@@ -65,7 +66,8 @@ struct FitLaunch {             // Gram + eigensolve
   float* basis_v;
   int32_t r, n_cov, pairing, shift, L, H;
   uint32_t* status;
-  float cs[kMaxHalfD], sn[kMaxHalfD];
+  alignas(16) float cs[kMaxHalfD];
+  alignas(16) float sn[kMaxHalfD];
 };
 
 // Address of row (l, h, t) of a cache; returns nullptr (and flags) on a bad page id.

@@ -1,0 +1,69 @@
+// Host-side construction of the TMA tensor maps used by the tensor-core kernels.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "kvc_dev.cuh"
+
+namespace kvc {
+namespace tc {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  }
+  return fn;
+}
+
+// 5-D view of a cache: (channel, token-in-unit, head, unit, layer); unit = page (paged) or the whole sequence.
+inline bool encode_cache(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base, int L, int H) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const bool paged = c.page_table != nullptr;
+  const cuuint64_t rows = paged ? (cuuint64_t)(c.page_mask + 1) : (cuuint64_t)c.T;
+  const cuuint64_t units = paged ? (cuuint64_t)c.n_phys : 1;
+  const cuuint64_t dims[5] = {128, rows, (cuuint64_t)H, units, (cuuint64_t)L};
+  const cuuint64_t unit_stride = paged ? (cuuint64_t)c.s_page * 2 : (cuuint64_t)c.s_layer * 2;
+  const cuuint64_t strides[4] = {(cuuint64_t)c.s_tok * 2, (cuuint64_t)c.s_head * 2, unit_stride, (cuuint64_t)c.s_layer * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)(paged ? (c.page_mask + 1) : 128), 1, 1, 1};
+  const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool encode_coeff(CUtensorMap* m, const float* coeff, int r, int n_cov, int slabs) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)r, (cuuint64_t)n_cov, (cuuint64_t)slabs};
+  const cuuint64_t strides[2] = {(cuuint64_t)r * 4, (cuuint64_t)r * 4 * (cuuint64_t)n_cov};
+  const cuuint32_t box[3] = {32, 128, 1};
+  const cuuint32_t es[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(coeff), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+
+inline int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+}  // namespace tc
+}  // namespace kvc

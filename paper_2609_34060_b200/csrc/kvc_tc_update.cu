@@ -1,0 +1,448 @@
+// State update on the Blackwell data path.
+//
+// project:  coeff[t, :] = (tgt[t, :] - Rot(src[t, :])) . basis^T     (Eq. 12 then Eq. 7's A = Delta B^T)
+//
+// The projection is linear and a rotation is orthogonal, so
+//     coeff = tgt . B^T  +  src . Bs^T      with   Bs = -Rot_{-shift}(B)
+// i.e. the BASIS is rotated once per (layer, head) instead of every source token.  The cache
+// tiles then go from TMA straight into the tensor cores as they are (bf16, exact): no per-token
+// arithmetic, no rewriting of operands.  One persistent CTA per SM walks tiles of 128 tokens:
+//   warp 0      TMA producer: target tile and source tile (bf16 128 x 128 each)
+//   warp 1      MMA issuer + TMEM owner
+//   warp 3      store warp: coefficient tile (fp32 128 x r) out through TMA, releases the stage
+//   warps 4-19  the team: stages B and Bs as K-major 128B-swizzled bf16 hi/lo operands whenever the
+//               slab changes; per tile reads the accumulator row from TMEM and writes the
+//               coefficient tile into the (by then free) stage.
+// Precision: B = B1 + B2, Bs = S1 + S2 (bf16 terms, residual 2^-18 relative); tiles are exact;
+// fp32 accumulation.  The two products cancel down to Delta . B^T, so the absolute error scales
+// with |src| + |tgt| (about 2^-18 (|src_t| + |tgt_t|) |B_q|), not with |Delta|.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <string.h>
+
+#include <cstddef>
+
+#include "../../include/kvc.h"
+#include "kvc_dev.cuh"
+#include "kvc_tc.h"
+#include "kvc_tc_maps.h"
+#include "kvc_tc_ptx.cuh"
+
+namespace kvc {
+namespace tcu {
+
+using namespace kvc::tc;
+
+constexpr int kTileTok = 128;
+constexpr int kThreads = 640;
+constexpr int kTeamThreads = 512;
+constexpr int kHalfBytes = kTileTok * 128;     // 64 channels x 128 tokens, bf16
+constexpr int kTileBytes = 2 * kHalfBytes;     // one cache tile
+constexpr int kStageBytes = 2 * kTileBytes;    // target tile, then source tile
+
+struct alignas(64) UpdMaps {
+  CUtensorMap src_k, src_v, tgt_k, tgt_v, coeff_k, coeff_v;
+};
+
+struct ProjectTcLaunch {
+  UpdateLaunch u;
+  int64_t total_tiles;
+  int32_t has_src, pad;
+  UpdMaps maps;
+};
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+
+struct PTile {
+  int slab, is_v, t0, l, h;
+};
+__device__ __forceinline__ PTile decode(const UpdateLaunch& u, int64_t tile) {
+  PTile t;
+  const int tt = (int)(tile % u.tiles_per_slab);
+  const int64_t sk = tile / u.tiles_per_slab;
+  t.is_v = (int)(sk & 1);
+  t.slab = (int)(sk >> 1);
+  t.l = t.slab / u.H;
+  t.h = t.slab % u.H;
+  t.t0 = tt * kTileTok;
+  return t;
+}
+
+template <int NS>
+struct Ctrl {
+  uint64_t full[NS], ready[NS], empty[NS];
+  uint64_t mma_done[2], acc_empty[2];
+  uint64_t basis_full;
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// Bytes one cache tile will deliver (for expect_tx) and, for paged caches, this lane's page.
+// Must be called by the whole warp.
+__device__ __forceinline__ uint32_t tile_bytes(const DevCache& c, int t0, int lane, int& id, bool& valid,
+                                               uint32_t* status) {
+  if (!c.page_table) {
+    id = 0;
+    valid = lane == 0;
+    return kTileBytes;
+  }
+  const int page = c.page_mask + 1;
+  const int per_tile = kTileTok >> c.page_shift;
+  const int first = t0 >> c.page_shift;
+  const int n_pages = min(per_tile, ((c.T + page - 1) >> c.page_shift) - first);
+  id = -1;
+  if (lane < n_pages) id = c.page_table[first + lane];
+  valid = lane < n_pages && (unsigned)id < (unsigned)c.n_phys;
+  if (lane < n_pages && !valid) atomicOr(status, KVC_FLAG_BAD_PAGE);
+  return (uint32_t)(__popc(__ballot_sync(0xffffffffu, valid)) * page * 256);
+}
+__device__ __forceinline__ void tile_issue(const DevCache& c, const CUtensorMap* map, uint32_t dst, uint32_t bar,
+                                           const PTile& t, int lane, int id, bool valid) {
+  if (!valid) return;
+  if (!c.page_table) {
+    tma_load_5d(dst, map, bar, 0, t.t0, t.h, 0, t.l);
+    tma_load_5d(dst + kHalfBytes, map, bar, 64, t.t0, t.h, 0, t.l);
+  } else {
+    const int page = c.page_mask + 1;
+    tma_load_5d(dst + lane * page * 128, map, bar, 0, 0, t.h, id, t.l);
+    tma_load_5d(dst + kHalfBytes + lane * page * 128, map, bar, 64, 0, t.h, id, t.l);
+  }
+}
+
+// RB = rank blocks of 32 (accumulator columns = 32 RB), NS = stages
+template <int RB, int NS>
+__global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_constant__ ProjectTcLaunch p) {
+  constexpr int RN = 32 * RB;
+  constexpr int kBlk = RN * 128;                 // RN basis rows x 64 channels, bf16
+  constexpr int kSlotBytes = 8 * kBlk;           // {B, Bs} x {hi, lo} x {channels 0-63, 64-127}
+  // kind::f16, bf16 x bf16 -> f32, K-major operands, M = 128, N = 32
+  constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t stages = base;
+  const uint32_t slot = base + NS * kStageBytes;
+  uint8_t* slot_ptr = smem + NS * kStageBytes;
+  Ctrl<NS>* ctrl = reinterpret_cast<Ctrl<NS>*>(smem + NS * kStageBytes + kSlotBytes);
+  volatile int* abort_flag = &ctrl->abort_flag;
+  const UpdateLaunch& u = p.u;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t n = p.total_tiles;
+  const int64_t tile_begin = n * blockIdx.x / gridDim.x;
+  const int64_t tile_end = n * (blockIdx.x + 1) / gridDim.x;
+  const uint32_t n_my = (uint32_t)(tile_end - tile_begin);
+
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->ready[s]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
+      mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
+    }
+    mbar_init(smem_u32(&ctrl->basis_full), kTeamThreads);
+    mbar_init(smem_u32(&ctrl->drain), 1);
+    ctrl->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctrl->tmem_base), 128);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+
+  if (warp == 0) {
+    // =============================================================== TMA producer
+    uint32_t i = 0;
+    for (; i < n_my; ++i) {
+      const PTile t = decode(u, tile_begin + i);
+      const int s = i % NS;
+      const uint32_t use = i / NS;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const uint32_t st_base = stages + s * kStageBytes;
+      const uint32_t bar = smem_u32(&ctrl->full[s]);
+      int id_t, id_s = 0;
+      bool ok_t, ok_s = false;
+      uint32_t bytes = tile_bytes(u.tgt, t.t0, lane, id_t, ok_t, u.status);
+      if (p.has_src) bytes += tile_bytes(u.src, t.t0, lane, id_s, ok_s, u.status);
+      if (lane == 0) mbar_expect_tx(bar, bytes);
+      __syncwarp();
+      tile_issue(u.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
+      if (p.has_src) tile_issue(u.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
+      __syncwarp();
+    }
+    if (lane == 0) {
+      for (uint32_t k = (i > NS ? i - NS : 0); k < i; ++k) mbar_wait_drain(smem_u32(&ctrl->full[k % NS]), (k / NS) & 1u);
+    }
+  } else if (warp == 1) {
+    // =============================================================== MMA issuer
+    if (lane == 0) {
+      uint32_t slabs = 0;
+      int prev_key = -1;
+      for (uint32_t i = 0; i < n_my; ++i) {
+        const PTile t = decode(u, tile_begin + i);
+        const int s = i % NS, g = i & 1;
+        const uint32_t use = i / NS, acc_use = i >> 1;
+        const int key = t.slab * 2 + t.is_v;
+        if (key != prev_key) {                                    // the team stages the operands of a new slab
+          if (!mbar_wait(smem_u32(&ctrl->basis_full), slabs & 1u, abort_flag)) break;
+          ++slabs;
+          prev_key = key;
+        }
+        if (!mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag)) break;
+        if (!mbar_wait(smem_u32(&ctrl->acc_empty[g]), (acc_use & 1u) ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a_t = stages + s * kStageBytes;            // target tile
+        const uint32_t a_s = a_t + kTileBytes;                    // source tile
+#pragma unroll
+        for (int nb = 0; nb < RB; ++nb) {                         // N = 32 per instruction
+          const uint32_t d_tmem = tmem_base + g * 64 + 32 * nb;
+          uint32_t acc = 0;
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb) {                        // two 64-channel K blocks
+            const uint64_t at = umma_desc_sw128(a_t + kb * kHalfBytes), as = umma_desc_sw128(a_s + kb * kHalfBytes);
+            const uint32_t bo = slot + kb * kBlk + nb * 32 * 128;
+            const uint64_t b_hi = umma_desc_sw128(bo), b_lo = umma_desc_sw128(bo + 2 * kBlk);
+            const uint64_t s_hi = umma_desc_sw128(bo + 4 * kBlk), s_lo = umma_desc_sw128(bo + 6 * kBlk);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {                         // 16 channels = 32 bytes per step
+              umma_bf16(d_tmem, at + 2 * k, b_hi + 2 * k, kIdesc, acc);
+              acc = 1;
+              umma_bf16(d_tmem, at + 2 * k, b_lo + 2 * k, kIdesc, 1);
+              if (p.has_src) {
+                umma_bf16(d_tmem, as + 2 * k, s_hi + 2 * k, kIdesc, 1);
+                umma_bf16(d_tmem, as + 2 * k, s_lo + 2 * k, kIdesc, 1);
+              }
+            }
+          }
+        }
+        umma_commit(smem_u32(&ctrl->mma_done[g]));
+      }
+      umma_commit(smem_u32(&ctrl->drain));
+      mbar_wait_drain(smem_u32(&ctrl->drain), 0);
+    }
+  } else if (warp == 3) {
+    // =============================================================== store warp
+    for (uint32_t i = 0; i < n_my; ++i) {
+      const PTile t = decode(u, tile_begin + i);
+      const int s = i % NS;
+      const uint32_t use = i / NS;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), use & 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane == 0) {
+        const CUtensorMap* cmap = t.is_v ? &p.maps.coeff_v : &p.maps.coeff_k;
+        const uint32_t st_base = stages + s * kStageBytes;
+#pragma unroll
+        for (int b = 0; b < RB; ++b) tma_store_3d(cmap, st_base + b * kHalfBytes, 32 * b, t.t0, t.slab);
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(smem_u32(&ctrl->empty[s]));
+      }
+      __syncwarp();
+    }
+  } else if (warp >= 4) {
+    // =============================================================== the team (16 warps)
+    const int e = warp - 4;
+    const int q = e & 3;                           // TMEM lane quadrant
+    const int cq = e >> 2;                         // coefficient quarter
+    const int m = q * 32 + lane;                   // row of the tile = token
+    const int tt = tid - 128;                      // 0..511
+    const uint32_t sw = (uint32_t)(m & 7);
+
+    // B and Bs = -Rot_{-shift}(B) of one slab as swizzled K-major bf16 hi/lo operands
+    auto stage_basis = [&](const PTile& t) {
+      const void* basis = t.is_v ? u.basis_v : u.basis_k;
+      const bool rotate = u.shift != 0 && !t.is_v;
+      for (int task = tt; task < RN * 16; task += kTeamThreads) {
+        const int row = task >> 4, jj = task & 15;                // basis row, chunk of 8 channels
+        float v[8], w[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = w[k] = 0.f;
+        if (row < u.r) {
+          const int64_t off = ((int64_t)t.slab * u.r + row) * 128;
+          auto load8 = [&](int chunk, float* o) {
+            if (u.basis_bf16) {
+              unpack8(*reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(basis) + off + 8 * chunk), o);
+            } else {
+              const float* b = reinterpret_cast<const float*>(basis) + off + 8 * chunk;
+              *reinterpret_cast<float4*>(o) = *reinterpret_cast<const float4*>(b);
+              *reinterpret_cast<float4*>(o + 4) = *reinterpret_cast<const float4*>(b + 4);
+            }
+          };
+          load8(jj, v);
+          if (rotate && u.pairing == 0) load8(jj ^ 8, w);          // the pair partners of this chunk
+        }
+        float sneg[8];                                             // -Rot_{-shift}(b) on this chunk
+        if (!rotate) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) sneg[k] = -v[k];
+        } else if (u.pairing == 0) {
+          const int f0 = 8 * (jj & 7);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float c = u.cs[f0 + k], sn = u.sn[f0 + k];
+            // first half: b[k] c + b[k+64] s ; second half: -b[k] s + b[k+64] c   (then negated)
+            sneg[k] = (jj < 8) ? -(v[k] * c + w[k] * sn) : -(v[k] * c - w[k] * sn);
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float c = u.cs[4 * jj + k], sn = u.sn[4 * jj + k];
+            sneg[2 * k] = -(v[2 * k] * c + v[2 * k + 1] * sn);
+            sneg[2 * k + 1] = -(v[2 * k + 1] * c - v[2 * k] * sn);
+          }
+        }
+        uint4 bh, bl, sh, sl;
+        split2(v[0], v[1], bh.x, bl.x);
+        split2(v[2], v[3], bh.y, bl.y);
+        split2(v[4], v[5], bh.z, bl.z);
+        split2(v[6], v[7], bh.w, bl.w);
+        split2(sneg[0], sneg[1], sh.x, sl.x);
+        split2(sneg[2], sneg[3], sh.y, sl.y);
+        split2(sneg[4], sneg[5], sh.z, sl.z);
+        split2(sneg[6], sneg[7], sh.w, sl.w);
+        const int kb = jj >> 3, j = jj & 7;
+        uint8_t* o = slot_ptr + kb * kBlk + row * 128 + ((j ^ (row & 7)) << 4);
+        *reinterpret_cast<uint4*>(o) = bh;
+        *reinterpret_cast<uint4*>(o + 2 * kBlk) = bl;
+        *reinterpret_cast<uint4*>(o + 4 * kBlk) = sh;
+        *reinterpret_cast<uint4*>(o + 6 * kBlk) = sl;
+      }
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&ctrl->basis_full));
+    };
+
+    int prev_key = -1;
+    if (n_my > 0) {
+      const PTile t0 = decode(u, tile_begin);
+      stage_basis(t0);
+      prev_key = t0.slab * 2 + t0.is_v;
+    }
+    for (uint32_t i = 0; i < n_my; ++i) {
+      const int s = i % NS, g = i & 1;
+      const uint32_t acc_use = i >> 1;
+      bool ok = mbar_wait(smem_u32(&ctrl->mma_done[g]), acc_use & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      // The MMAs of tile i are complete.  If tile i + 1 opens a new slab, tile i was the last
+      // reader of the operand slot: restage it now so that the next MMA can start early.
+      if (i + 1 < n_my) {
+        const PTile tn = decode(u, tile_begin + i + 1);
+        const int key = tn.slab * 2 + tn.is_v;
+        if (key != prev_key) {
+          stage_basis(tn);
+          prev_key = key;
+        }
+      }
+      const uint32_t t_acc = tmem_base + g * 64 + ((uint32_t)(q * 32) << 16);
+      float c[8 * RB];
+      if constexpr (RB == 1) {
+        tmem_ld8(t_acc + 8 * cq, c);
+      } else {
+        tmem_ld16(t_acc + 16 * cq, c);
+      }
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
+      // the operands of this tile have been consumed: its first RB * 16 KB become the coefficient tile
+      uint8_t* st_ptr = smem + s * kStageBytes;
+      if constexpr (RB == 1) {
+        uint8_t* row = st_ptr + m * 128;
+        *reinterpret_cast<float4*>(row + (((2 * cq) ^ sw) << 4)) = make_float4(c[0], c[1], c[2], c[3]);
+        *reinterpret_cast<float4*>(row + (((2 * cq + 1) ^ sw) << 4)) = make_float4(c[4], c[5], c[6], c[7]);
+      } else {
+        uint8_t* row = st_ptr + (cq >> 1) * kHalfBytes + m * 128;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          *reinterpret_cast<float4*>(row + (((4 * (cq & 1) + k) ^ sw) << 4)) = make_float4(c[4 * k], c[4 * k + 1], c[4 * k + 2], c[4 * k + 3]);
+      }
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&ctrl->ready[s]));
+    }
+  }
+
+  __syncthreads();
+  if (tid == 0 && *abort_flag) atomicOr(u.status, KVC_FLAG_WAIT_EXPIRED);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 128);
+  }
+}
+
+template <int RB, int NS>
+static cudaError_t launch_project_t(const ProjectTcLaunch& L, int grid, cudaStream_t s) {
+  const size_t smem = 1024 + (size_t)NS * kStageBytes + (size_t)8 * (32 * RB) * 128 + sizeof(Ctrl<NS>);
+  static bool set = false;
+  if (!set) {
+    cudaError_t e = cudaFuncSetAttribute(project_tc_kernel<RB, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    set = true;
+  }
+  project_tc_kernel<RB, NS><<<grid, kThreads, smem, s>>>(L);
+  return cudaGetLastError();
+}
+
+static bool cache_ok(const DevCache& c) {
+  if (c.page_table && (c.page_mask + 1) > 128) return false;
+  return c.T < (1 << 30);
+}
+
+}  // namespace tcu
+
+static_assert(offsetof(UpdateLaunch, cs) % 16 == 0 && offsetof(UpdateLaunch, sn) % 16 == 0, "rope tables: float4 reads");
+static_assert(offsetof(tcu::ProjectTcLaunch, maps) % 64 == 0, "tensor maps need 64-byte alignment");
+
+int tc_project(const UpdateLaunch& U, int d, cudaStream_t s) {
+  using namespace tcu;
+  if (d != 128 || U.r <= 0 || U.r > 64 || (U.r & 3) || U.n_cov <= 0) return KVC_E_UNSUPPORTED;
+  if (!cache_ok(U.tgt) || (U.src.k && !cache_ok(U.src)) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  ProjectTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.u = U;
+  L.u.tiles_per_slab = (U.n_cov + kTileTok - 1) / kTileTok;
+  L.total_tiles = (int64_t)U.L * U.H * 2 * L.u.tiles_per_slab;
+  L.has_src = U.src.k != nullptr;
+  bool ok = tc::encode_cache(&L.maps.tgt_k, U.tgt, U.tgt.k, U.L, U.H) && tc::encode_cache(&L.maps.tgt_v, U.tgt, U.tgt.v, U.L, U.H);
+  if (L.has_src)
+    ok = ok && tc::encode_cache(&L.maps.src_k, U.src, U.src.k, U.L, U.H) && tc::encode_cache(&L.maps.src_v, U.src, U.src.v, U.L, U.H);
+  ok = ok && tc::encode_coeff(&L.maps.coeff_k, U.coeff_k, U.r, U.n_cov, U.L * U.H) &&
+       tc::encode_coeff(&L.maps.coeff_v, U.coeff_v, U.r, U.n_cov, U.L * U.H);
+  if (!ok) return KVC_E_CUDA;
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+  const cudaError_t e = (U.r <= 32) ? launch_project_t<1, 3>(L, grid, s) : launch_project_t<2, 2>(L, grid, s);
+  return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+int tc_gram(const FitLaunch&, int, cudaStream_t) { return KVC_E_UNSUPPORTED; }
+
+}  // namespace kvc

@@ -82,6 +82,8 @@ def test_project_mode(cfg, path):
                    other.basis_k.to(DEV), other.basis_v.to(DEV), n_cov=n_cov)
     kvc.kvc_state_update(src, tgt, shift, kvc.Rope(cfg.theta), st, kvc.KVC_PROJECT)
     torch.cuda.synchronize()
+    if path == kvc.KVC_PATH_AUTO and cfg.d == 128:
+        assert kvc.kvc_last_path() == kvc.KVC_PATH_TC, "the TMA + tcgen05 kernels should have served this call"
     ck, cv = st.coeff_k.cpu().numpy().astype(np.float64), st.coeff_v.cpu().numpy().astype(np.float64)
     worst = 0.0
     for l in range(cfg.L):
