@@ -164,7 +164,9 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                (= U_r Sigma_r).  st->basis_dtype must be KVC_F32.
  *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
  *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte
- *              aligned; contents undefined afterwards.  May be NULL when 0 is needed.
+ *              aligned.  May be NULL when 0 is needed.  After a KVC_FIT call it holds, as
+ *              float32: the Gram matrices [L, H, 2, d, d] (2 = K, V), then scratch of the
+ *              same size, then the eigenvalues [L, H, 2, d] in descending order.
  * Errors as kvc_apply, plus KVC_E_WORKSPACE.
  */
 int kvc_state_update(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,
@@ -188,7 +190,7 @@ size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mo
  * still the caller's buffers, with the same meaning as in kvc_state_update.
  *
  *  - Capacity: kvc_workspace_bytes(tgt, st, mode) must not exceed
- *    KVC_STATIC_SCRATCH_BYTES, i.e. L*H <= 64 at d = 128 (L*H <= 254 at d = 64) in FIT
+ *    KVC_STATIC_SCRATCH_BYTES, i.e. L*H <= 64 at d = 128 (L*H <= 255 at d = 64) in FIT
  *    mode; larger problems return KVC_E_TOO_LARGE and launch nothing (split them by
  *    layer, or use kvc_state_update with your own workspace).  KVC_PROJECT needs no
  *    scratch and is never rejected for size.
@@ -199,7 +201,7 @@ size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mo
  *    Two calls whose device work can overlap (different streams, or different host
  *    threads on different streams) race on the array: serialise them.
  */
-#define KVC_STATIC_SCRATCH_BYTES (128 * (128 * 128 + 128) * 4)
+#define KVC_STATIC_SCRATCH_BYTES (128 * (2 * 128 * 128 + 128) * 4)
 int kvc_state_update_noalloc(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,
                              kvc_state *st, int32_t mode, void *stream);
 

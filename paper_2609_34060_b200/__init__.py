@@ -244,7 +244,7 @@ def kvc_state_update(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, s
                                    _stream(stream)), "kvc_state_update")
 
 
-KVC_STATIC_SCRATCH_BYTES = 128 * (128 * 128 + 128) * 4
+KVC_STATIC_SCRATCH_BYTES = 128 * (2 * 128 * 128 + 128) * 4
 
 
 def kvc_state_update_noalloc(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, st: State, mode: int,

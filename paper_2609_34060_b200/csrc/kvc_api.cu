@@ -247,7 +247,7 @@ int kvc_chain(const kvc_cache* agent0, int32_t n_agents, const int32_t* prefix_l
 size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
   if (!tgt || !st || mode != KVC_FIT) return 0;
   const size_t m = (size_t)tgt->L * tgt->H * 2;
-  return m * tgt->d * tgt->d * sizeof(float) + m * tgt->d * sizeof(float);
+  return 2 * m * tgt->d * tgt->d * sizeof(float) + m * tgt->d * sizeof(float);   // two partial Grams + eigenvalues
 }
 
 int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
@@ -283,7 +283,8 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
     F.src = ds;
     F.tgt = dt;
     F.gram = reinterpret_cast<float*>(workspace);
-    F.evals = F.gram + (size_t)tgt->L * tgt->H * 2 * d * d;
+    F.evals = F.gram + 2 * (size_t)tgt->L * tgt->H * 2 * d * d;
+    F.n_parts = 1;
     F.basis_k = reinterpret_cast<float*>(st->basis_k);
     F.basis_v = reinterpret_cast<float*>(st->basis_v);
     F.r = st->r;
@@ -297,7 +298,10 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
     bool gram_done = false;
     if (tl_path_force != KVC_PATH_GENERIC) {
       const int trc = tc_gram(F, d, s);
-      if (trc == KVC_OK) gram_done = true;
+      if (trc == KVC_OK) {
+        gram_done = true;
+        F.n_parts = 2;
+      }
       else if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
     }
     if (!gram_done && launch_gram_generic(F, d, s) != cudaSuccess) return KVC_E_CUDA;

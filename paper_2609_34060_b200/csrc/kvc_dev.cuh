@@ -60,11 +60,12 @@ struct UpdateLaunch {
 
 struct FitLaunch {             // Gram + eigensolve
   DevCache src, tgt;
-  float* gram;                 // [L*H*2][d][d]
+  float* gram;                 // [n_parts][L*H*2][d][d] partial sums in, [L*H*2][d][d] final out
   float* evals;                // [L*H*2][d] descending
   float* basis_k;              // [L,H,r,d] float32 out
   float* basis_v;
   int32_t r, n_cov, pairing, shift, L, H;
+  int32_t n_parts, pad;
   uint32_t* status;
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];

@@ -375,13 +375,19 @@ __global__ void __launch_bounds__(256) eig_jacobi_kernel(const __grid_constant__
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sk = blockIdx.x;
   const int is_v = sk & 1, slab = sk >> 1;
-  const float* G = p.gram + (int64_t)sk * n * n;
+  float* G = p.gram + (int64_t)sk * n * n;
+  const int64_t part_stride = (int64_t)p.L * p.H * 2 * n * n;
   for (int i = tid; i < n * n; i += 256) {
     const int rr = i / n, cc = i % n;
-    // symmetrise what the Gram kernel wrote (it is symmetric up to summation order)
-    A[i] = 0.5f * (G[i] + G[cc * n + rr]);
+    // sum the partial Grams in a fixed order and symmetrise (the split-precision tensor-core
+    // product leaves its L^T H term to this transpose-average)
+    float a = 0.f;
+    for (int pt = 0; pt < p.n_parts; ++pt) a += G[pt * part_stride + i] + G[pt * part_stride + cc * n + rr];
+    A[i] = 0.5f * a;
     VT[i] = (rr == cc) ? 1.f : 0.f;
   }
+  __syncthreads();
+  for (int i = tid; i < n * n; i += 256) G[i] = A[i];   // the final Gram matrix stays readable
   if (tid == 0) done = 0;
   __syncthreads();
 

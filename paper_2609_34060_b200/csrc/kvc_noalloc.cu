@@ -9,7 +9,8 @@
 
 namespace {
 
-// Built-in scratch: 128 matrices of 128 x 128 float32 plus their 128 eigenvalues each.
+// Built-in scratch: room for 128 Gram problems of 128 x 128 float32 (two partial sums each)
+// plus their 128 eigenvalues each.
 // Every GPU that loads the library holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[KVC_STATIC_SCRATCH_BYTES];
 

@@ -68,6 +68,15 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
 struct PTile {
   int slab, is_v, t0, l, h;
 };
+
+// hi = bf16(x), lo2 = bf16(2 (x - hi)) for two values, packed as bf16x2 words
+__device__ __forceinline__ void split2x(float x0, float x1, uint32_t& hi, uint32_t& lo2) {
+  const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+  const __nv_bfloat16 l0 = __float2bfloat16_rn(2.f * (x0 - __bfloat162float(h0)));
+  const __nv_bfloat16 l1 = __float2bfloat16_rn(2.f * (x1 - __bfloat162float(h1)));
+  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+  lo2 = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
 __device__ __forceinline__ PTile decode(const UpdateLaunch& u, int64_t tile) {
   PTile t;
   const int tt = (int)(tile % u.tiles_per_slab);
@@ -410,6 +419,337 @@ static cudaError_t launch_project_t(const ProjectTcLaunch& L, int grid, cudaStre
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Gram:  G = Delta^T Delta  per (layer, head, K|V)   (Eq. 7: the d x d matrix whose top-r eigenvectors
+// are the basis).  Delta has to be explicit here (its Gram is quadratically small against the
+// inputs'), so the team forms Delta = tgt - Rot(src) in fp32, and writes H = bf16(Delta) over the
+// target tile and 2 (Delta - H) over the source tile.  The tensor cores accumulate
+//     P = H^T H + H^T (2 L)
+// with both operands read MN-major straight from the token-major tiles; the eigensolver's
+// symmetrisation (P + P^T) / 2 = H^T H + H^T L + L^T H completes the split product.
+// Work unit = half of a slab's tokens (fixed split, so partial sums combine in a fixed order).
+// ---------------------------------------------------------------------------------------------
+struct GramTcLaunch {
+  FitLaunch f;
+  int64_t total_units;
+  int32_t tiles_per_slab, tiles_per_unit, has_src, pad;
+  UpdMaps maps;
+};
+
+struct GUnit {
+  int slab, is_v, part, l, h, tile0, n_tiles;
+};
+__device__ __forceinline__ GUnit gdecode(const GramTcLaunch& p, int64_t unit) {
+  GUnit g;
+  g.part = (int)(unit & 1);
+  const int64_t sk = unit >> 1;
+  g.is_v = (int)(sk & 1);
+  g.slab = (int)(sk >> 1);
+  g.l = g.slab / p.f.H;
+  g.h = g.slab % p.f.H;
+  g.tile0 = g.part * p.tiles_per_unit;
+  g.n_tiles = max(0, min(p.tiles_per_unit, p.tiles_per_slab - g.tile0));
+  return g;
+}
+
+template <int NS>
+struct GCtrl {
+  uint64_t full[NS], conv[NS], empty[NS];
+  uint64_t acc_full[2], acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// MN-major, 128-byte-swizzled operand: 64 channels x 8 tokens per 1 KB atom; atoms of the other 64
+// channels 16 KB further (leading offset), atoms of the next 8 tokens 1 KB further (stride offset).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(kHalfBytes >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcLaunch p) {
+  // kind::f16, bf16 x bf16 -> f32, both operands MN-major, M = 128, N = 128
+  constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t stages = base;
+  GCtrl<NS>* ctrl = reinterpret_cast<GCtrl<NS>*>(smem + NS * kStageBytes);
+  volatile int* abort_flag = &ctrl->abort_flag;
+  const FitLaunch& f = p.f;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t nu = p.total_units;
+  const int64_t unit_begin = nu * blockIdx.x / gridDim.x;
+  const int64_t unit_end = nu * (blockIdx.x + 1) / gridDim.x;
+
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->conv[s]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&ctrl->acc_full[g]), 1);
+      mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
+    }
+    mbar_init(smem_u32(&ctrl->drain), 1);
+    ctrl->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctrl->tmem_base), 256);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+
+  if (warp == 0) {
+    // =============================================================== TMA producer
+    uint32_t i = 0;
+    bool dead = false;
+    for (int64_t un = unit_begin; un < unit_end && !dead; ++un) {
+      const GUnit g = gdecode(p, un);
+      for (int k = 0; k < g.n_tiles; ++k, ++i) {
+        PTile t;
+        t.slab = g.slab;
+        t.is_v = g.is_v;
+        t.l = g.l;
+        t.h = g.h;
+        t.t0 = (g.tile0 + k) * kTileTok;
+        const int s = i % NS;
+        const uint32_t use = i / NS;
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) {
+          dead = true;
+          break;
+        }
+        const uint32_t st_base = stages + s * kStageBytes;
+        const uint32_t bar = smem_u32(&ctrl->full[s]);
+        int id_t, id_s = 0;
+        bool ok_t, ok_s = false;
+        uint32_t bytes = tile_bytes(f.tgt, t.t0, lane, id_t, ok_t, f.status);
+        if (p.has_src) bytes += tile_bytes(f.src, t.t0, lane, id_s, ok_s, f.status);
+        if (lane == 0) mbar_expect_tx(bar, bytes);
+        __syncwarp();
+        tile_issue(f.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
+        if (p.has_src) tile_issue(f.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
+        __syncwarp();
+      }
+    }
+    if (lane == 0) {
+      for (uint32_t k = (i > NS ? i - NS : 0); k < i; ++k) mbar_wait_drain(smem_u32(&ctrl->full[k % NS]), (k / NS) & 1u);
+    }
+  } else if (warp == 1) {
+    // =============================================================== MMA issuer
+    if (lane == 0) {
+      uint32_t i = 0, ui = 0;
+      bool dead = false;
+      for (int64_t un = unit_begin; un < unit_end && !dead; ++un, ++ui) {
+        const GUnit g = gdecode(p, un);
+        const int a = ui & 1;
+        if (!mbar_wait(smem_u32(&ctrl->acc_empty[a]), ((ui >> 1) & 1u) ^ 1u, abort_flag)) break;
+        const uint32_t d_tmem = tmem_base + a * 128;
+        uint32_t acc = 0;
+        for (int k = 0; k < g.n_tiles; ++k, ++i) {
+          const int s = i % NS;
+          const uint32_t use = i / NS;
+          if (!mbar_wait(smem_u32(&ctrl->conv[s]), use & 1u, abort_flag)) {
+            dead = true;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t hb = stages + s * kStageBytes;          // H over the target tile
+          const uint32_t lb = hb + kTileBytes;                    // 2 L over the source tile
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {                        // 16 tokens = two 1 KB atoms per step
+            const uint64_t hd = umma_desc_mn_sw128(hb + ks * 2048);
+            umma_bf16(d_tmem, hd, hd, kIdesc, acc);
+            acc = 1;
+            if (p.has_src) umma_bf16(d_tmem, hd, umma_desc_mn_sw128(lb + ks * 2048), kIdesc, 1);
+          }
+          umma_commit(smem_u32(&ctrl->empty[s]));                  // operands consumed => stage free
+        }
+        if (dead) break;
+        umma_commit(smem_u32(&ctrl->acc_full[a]));
+      }
+      umma_commit(smem_u32(&ctrl->drain));
+      mbar_wait_drain(smem_u32(&ctrl->drain), 0);
+    }
+  } else if (warp >= 4) {
+    // =============================================================== the team (16 warps)
+    const int e = warp - 4;
+    const int q = e & 3;
+    const int cq = e >> 2;
+    const int m = q * 32 + lane;                   // token row (conversion) / Gram row (flush)
+    const uint32_t sw = (uint32_t)(m & 7);
+    const bool rot_any = f.shift != 0;
+
+    auto flush = [&](const GUnit& g, uint32_t ui) {
+      const int a = ui & 1;
+      bool ok = mbar_wait(smem_u32(&ctrl->acc_full[a]), (ui >> 1) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return false;
+      tc_fence_after();
+      const uint32_t t_acc = tmem_base + a * 128 + ((uint32_t)(q * 32) << 16);
+      float c0[16], c1[16];
+      tmem_ld16(t_acc + 32 * cq, c0);
+      tmem_ld16(t_acc + 32 * cq + 16, c1);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->acc_empty[a]));
+      const int64_t mats = (int64_t)f.L * f.H * 2;
+      float* G = f.gram + ((int64_t)g.part * mats + (int64_t)g.slab * 2 + g.is_v) * 128 * 128 + (int64_t)m * 128 + 32 * cq;
+      if (g.n_tiles == 0) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) c0[k] = c1[k] = 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        *reinterpret_cast<float4*>(G + 4 * k) = make_float4(c0[4 * k], c0[4 * k + 1], c0[4 * k + 2], c0[4 * k + 3]);
+        *reinterpret_cast<float4*>(G + 16 + 4 * k) = make_float4(c1[4 * k], c1[4 * k + 1], c1[4 * k + 2], c1[4 * k + 3]);
+      }
+      return true;
+    };
+
+    uint32_t i = 0, ui = 0;
+    bool alive = true, have_prev = false;
+    GUnit prev;
+    for (int64_t un = unit_begin; un < unit_end && alive; ++un, ++ui) {
+      const GUnit g = gdecode(p, un);
+      for (int k = 0; k < g.n_tiles && alive; ++k, ++i) {
+        const int s = i % NS;
+        const uint32_t use = i / NS;
+        bool ok = mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+          alive = false;
+          break;
+        }
+        uint8_t* tg = smem + s * kStageBytes;
+        uint8_t* sr = tg + kTileBytes;
+        const int tok = (g.tile0 + k) * kTileTok + m;
+        const bool live = tok < f.n_cov;
+        const bool rotate = rot_any && !g.is_v;
+        if (p.has_src || !live) {
+          if (f.pairing == 0) {
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+              const int j = 2 * cq + jj;
+              const uint32_t o = (uint32_t)(m * 128 + ((j ^ sw) << 4));
+              uint4* t0p = reinterpret_cast<uint4*>(tg + o);
+              uint4* t1p = reinterpret_cast<uint4*>(tg + kHalfBytes + o);
+              uint4* s0p = reinterpret_cast<uint4*>(sr + o);
+              uint4* s1p = reinterpret_cast<uint4*>(sr + kHalfBytes + o);
+              uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
+              if (live) {
+                float x[16], y[16];
+                unpack8(*s0p, x);
+                unpack8(*s1p, x + 8);
+                unpack8(*t0p, y);
+                unpack8(*t1p, y + 8);
+                if (rotate) {
+                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(f.cs + 8 * j + 4);
+                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(f.sn + 8 * j + 4);
+                  const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                  const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                  for (int z = 0; z < 8; ++z) {
+                    const float a = x[z], b = x[8 + z];
+                    x[z] = a * cs[z] - b * sn[z];
+                    x[8 + z] = a * sn[z] + b * cs[z];
+                  }
+                }
+                uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
+                uint32_t* hp1 = reinterpret_cast<uint32_t*>(&h1);
+                uint32_t* lp0 = reinterpret_cast<uint32_t*>(&l0);
+                uint32_t* lp1 = reinterpret_cast<uint32_t*>(&l1);
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  split2x(y[2 * z] - x[2 * z], y[2 * z + 1] - x[2 * z + 1], hp0[z], lp0[z]);
+                  split2x(y[8 + 2 * z] - x[8 + 2 * z], y[9 + 2 * z] - x[9 + 2 * z], hp1[z], lp1[z]);
+                }
+              }
+              *t0p = h0;
+              *t1p = h1;
+              if (p.has_src) {
+                *s0p = l0;
+                *s1p = l1;
+              }
+            }
+          } else {
+            const uint32_t hb = (uint32_t)((cq >> 1) * kHalfBytes);
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+              const int j = 4 * (cq & 1) + jj;
+              const uint32_t o = hb + (uint32_t)(m * 128 + ((j ^ sw) << 4));
+              uint4* tp = reinterpret_cast<uint4*>(tg + o);
+              uint4* sp = reinterpret_cast<uint4*>(sr + o);
+              uint4 h = make_uint4(0, 0, 0, 0), l = h;
+              if (live) {
+                float x[8], y[8];
+                unpack8(*sp, x);
+                unpack8(*tp, y);
+                if (rotate) {
+                  const int f0 = 16 * cq + 4 * jj;
+                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + f0);
+                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + f0);
+                  const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
+                  const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
+#pragma unroll
+                  for (int z = 0; z < 4; ++z) {
+                    const float a = x[2 * z], b = x[2 * z + 1];
+                    x[2 * z] = a * cs[z] - b * sn[z];
+                    x[2 * z + 1] = a * sn[z] + b * cs[z];
+                  }
+                }
+                uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
+                uint32_t* lp = reinterpret_cast<uint32_t*>(&l);
+#pragma unroll
+                for (int z = 0; z < 4; ++z) split2x(y[2 * z] - x[2 * z], y[2 * z + 1] - x[2 * z + 1], hp[z], lp[z]);
+              }
+              *tp = h;
+              if (p.has_src) *sp = l;
+            }
+          }
+          fence_proxy_async();
+        }
+        mbar_arrive(smem_u32(&ctrl->conv[s]));
+        // the previous unit's accumulator is complete by now (its MMAs were issued a tile ago)
+        if (k == 0 && have_prev) {
+          alive = flush(prev, ui - 1);
+          have_prev = false;
+        }
+      }
+      if (have_prev && alive) alive = flush(prev, ui - 1);   // the unit before this one had no successor tile yet
+      prev = g;
+      have_prev = true;
+    }
+    if (have_prev && alive) flush(prev, ui - 1);
+  }
+
+  __syncthreads();
+  if (tid == 0 && *abort_flag) atomicOr(f.status, KVC_FLAG_WAIT_EXPIRED);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
 static bool cache_ok(const DevCache& c) {
   if (c.page_table && (c.page_mask + 1) > 128) return false;
   return c.T < (1 << 30);
@@ -443,6 +783,37 @@ int tc_project(const UpdateLaunch& U, int d, cudaStream_t s) {
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
-int tc_gram(const FitLaunch&, int, cudaStream_t) { return KVC_E_UNSUPPORTED; }
+static_assert(offsetof(FitLaunch, cs) % 16 == 0 && offsetof(FitLaunch, sn) % 16 == 0, "rope tables: float4 reads");
+static_assert(offsetof(tcu::GramTcLaunch, maps) % 64 == 0, "tensor maps need 64-byte alignment");
+
+// Writes two partial Gram matrices per (layer, head, K|V): part p at F.gram + p * (L*H*2) * d * d.
+int tc_gram(const FitLaunch& F, int d, cudaStream_t s) {
+  using namespace tcu;
+  if (d != 128 || F.n_cov <= 0) return KVC_E_UNSUPPORTED;
+  if (!cache_ok(F.tgt) || (F.src.k && !cache_ok(F.src)) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  GramTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.f = F;
+  L.tiles_per_slab = (F.n_cov + kTileTok - 1) / kTileTok;
+  L.tiles_per_unit = (L.tiles_per_slab + 1) / 2;
+  L.total_units = (int64_t)F.L * F.H * 2 * 2;
+  L.has_src = F.src.k != nullptr;
+  bool ok = tc::encode_cache(&L.maps.tgt_k, F.tgt, F.tgt.k, F.L, F.H) && tc::encode_cache(&L.maps.tgt_v, F.tgt, F.tgt.v, F.L, F.H);
+  if (L.has_src)
+    ok = ok && tc::encode_cache(&L.maps.src_k, F.src, F.src.k, F.L, F.H) && tc::encode_cache(&L.maps.src_v, F.src, F.src.v, F.L, F.H);
+  if (!ok) return KVC_E_CUDA;
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(L.total_units < sms ? L.total_units : sms);
+  constexpr int NS = 3;
+  const size_t smem = 1024 + (size_t)NS * kStageBytes + sizeof(GCtrl<NS>);
+  static bool set = false;
+  if (!set) {
+    if (cudaFuncSetAttribute(gram_tc_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+    set = true;
+  }
+  gram_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
+  return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
 
 }  // namespace kvc

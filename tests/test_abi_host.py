@@ -100,7 +100,7 @@ def test_chain_and_update_argument_errors(lib):
     assert upd(5, None, 0) == -1
     assert upd(kvc.KVC_FIT, None, 0) == -6                            # FIT needs scratch
     need = lib.kvc_workspace_bytes(C.byref(tgt), C.byref(st), kvc.KVC_FIT)
-    assert need == 2 * 2 * 2 * (128 * 128 + 128) * 4
+    assert need == 2 * 2 * 2 * (2 * 128 * 128 + 128) * 4
     assert lib.kvc_workspace_bytes(C.byref(tgt), C.byref(st), kvc.KVC_PROJECT) == 0
     assert upd(kvc.KVC_FIT, 0x7000100, need - 1) == -6                # too small
     assert upd(kvc.KVC_FIT, 0x7000101, need) == -6                    # misaligned

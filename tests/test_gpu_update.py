@@ -133,7 +133,7 @@ def test_fit_mode(cfg, path):
     torch.cuda.synchronize()
     wsf = ws.view(torch.float32).cpu().numpy().astype(np.float64)
     G = wsf[: L * H * 2 * d * d].reshape(L, H, 2, d, d)
-    ev = wsf[L * H * 2 * d * d: L * H * 2 * d * (d + 1)].reshape(L, H, 2, d)
+    ev = wsf[2 * L * H * 2 * d * d: 2 * L * H * 2 * d * d + L * H * 2 * d].reshape(L, H, 2, d)
     for l in range(L):
         for h in range(H):
             for i, (which, B_t, c_t, B_o) in enumerate((("k", st.basis_k, st.coeff_k, ost.basis_k),
