@@ -161,7 +161,8 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                of st->basis_* (float32; right singular vectors of Delta, largest
  *                singular values first, each row's largest-magnitude entry made
  *                positive; rows beyond min(r, d, n_cov) are zero), then coeff as above
- *                (= U_r Sigma_r).  st->basis_dtype must be KVC_F32.
+ *                (= U_r Sigma_r).  st->basis_dtype must be KVC_F32 and r <= 64 (else
+ *                KVC_E_UNSUPPORTED).
  *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
  *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte
  *              aligned.  May be NULL when 0 is needed.  After a KVC_FIT call it holds, as

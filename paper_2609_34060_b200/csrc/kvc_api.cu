@@ -267,7 +267,7 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   if (st->n_cov > tgt->T) return KVC_E_SHAPE;
   if (st->r == 0 || st->n_cov == 0) return KVC_OK;   // nothing to compute
   if (!st->coeff_k || !st->coeff_v) return KVC_E_INVALID_ARG;
-  if (mode == KVC_FIT && st->basis_dtype != KVC_F32) return KVC_E_UNSUPPORTED;
+  if (mode == KVC_FIT && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
   if (mode == KVC_FIT) {
     const size_t need = kvc_workspace_bytes(tgt, st, mode);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_E_WORKSPACE;

@@ -358,167 +358,300 @@ __global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant
 }
 
 // ---------------------------------------------------------------------------------
-// Symmetric eigensolver: parallel cyclic Jacobi (round-robin pairing), one block per
-// matrix, A and V^T in shared memory.  Writes eigenvalues (descending) and the top-r
-// eigenvectors as basis rows, each with its largest-magnitude entry positive.
+// Symmetric eigensolver for the top-r eigenpairs of the d x d Gram matrices (Eq. 7: the basis
+// rows are the right singular vectors of Delta for its largest r singular values).
+// One block per matrix, everything in shared memory, float32:
+//   1. Householder reduction to tridiagonal form T = Q^T G Q (reflectors kept in place);
+//   2. all eigenvalues of T by bisection on Sturm counts (one thread per eigenvalue);
+//   3. eigenvectors of T for the r largest by inverse iteration (tridiagonal LU with partial
+//      pivoting, one thread per vector), re-orthogonalised (Gram-Schmidt, twice) after each of
+//      two iterations so that equal or close eigenvalues still give an orthonormal set;
+//   4. back-transformation by the reflectors, sign convention, output.
+// The input is the sum of the partial Gram matrices, symmetrised; it is written back so that
+// the final Gram matrix stays readable in the workspace.
 // ---------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) eig_jacobi_kernel(const __grid_constant__ FitLaunch p, int n) {
+constexpr int kEigThreads = 256;
+constexpr int kEigMaxR = 64;
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+__global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int n, int zs) {
   extern __shared__ __align__(16) float smem[];
-  float* A = smem;              // [n][n]
-  float* VT = smem + n * n;     // [n][n]  row i = eigenvector i
-  __shared__ float rot_c[kMaxHalfD], rot_s[kMaxHalfD];
-  __shared__ int rot_p[kMaxHalfD], rot_q[kMaxHalfD];
-  __shared__ float red[2][8];
-  __shared__ int order[2 * kMaxHalfD];
-  __shared__ int done;
+  float* A = smem;                    // [n][n]   symmetric; row k right of the diagonal later holds reflector k
+  float* Zt = A + n * n;              // [n][zs]  Zt[i][j] = component i of eigenvector j  (zs = r_eff + 1, odd)
+  float* vv = Zt + n * zs;            // [n] current reflector
+  float* pp = vv + n;                 // [n] beta * A v
+  float* dd = pp + n;                 // [n] diagonal of T
+  float* ee = dd + n;                 // [n] off-diagonal of T (ee[i] couples i and i+1)
+  float* e2 = ee + n;                 // [n] squares of ee
+  float* bet = e2 + n;                // [n] reflector scalars
+  float* lam = bet + n;               // [n] eigenvalues, descending
+  float* shf = lam + n;               // [kEigMaxR] perturbed shifts for inverse iteration
+  float* red = shf + kEigMaxR;        // [16] reductions
+  float* cdot = red + 16;             // [kEigMaxR] Gram-Schmidt coefficients
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NW = kEigThreads / 32;
   const int sk = blockIdx.x;
   const int is_v = sk & 1, slab = sk >> 1;
   float* G = p.gram + (int64_t)sk * n * n;
   const int64_t part_stride = (int64_t)p.L * p.H * 2 * n * n;
-  for (int i = tid; i < n * n; i += 256) {
-    const int rr = i / n, cc = i % n;
-    // sum the partial Grams in a fixed order and symmetrise (the split-precision tensor-core
-    // product leaves its L^T H term to this transpose-average)
+
+  // ---- load: fixed-order sum of the partial Grams, symmetrised
+  for (int i = tid; i < n * n; i += kEigThreads) {
+    const int rr = i / n, cc = i - rr * n;
     float a = 0.f;
     for (int pt = 0; pt < p.n_parts; ++pt) a += G[pt * part_stride + i] + G[pt * part_stride + cc * n + rr];
     A[i] = 0.5f * a;
-    VT[i] = (rr == cc) ? 1.f : 0.f;
   }
   __syncthreads();
-  for (int i = tid; i < n * n; i += 256) G[i] = A[i];   // the final Gram matrix stays readable
-  if (tid == 0) done = 0;
-  __syncthreads();
+  for (int i = tid; i < n * n; i += kEigThreads) G[i] = A[i];
 
-  const int half = n / 2, m = n - 1;
-  const int max_sweeps = 30;
-  int sweep = 0;
-  for (; sweep < max_sweeps; ++sweep) {
-    // off-diagonal and total energy
-    float off = 0.f, tot = 0.f;
-    for (int i = tid; i < n * n; i += 256) {
-      const float x = A[i];
-      const float x2 = x * x;
-      tot += x2;
-      if (i / n != i % n) off += x2;
+  // ---- 1. Householder tridiagonalisation
+  for (int k = 0; k < n - 2; ++k) {
+    const int m = n - k - 1;                      // order of the trailing block; x = A[k][k+1 .. n-1]
+    const float* x = A + k * n + k + 1;
+    if (warp == 0) {
+      float s2 = 0.f;
+      for (int i = lane; i < m; i += 32) s2 += x[i] * x[i];
+      s2 = warp_sum(s2);
+      const float x0 = x[0];
+      const float tail = s2 - x0 * x0;            // energy below the sub-diagonal entry
+      float alpha = x0, beta = 0.f, v0 = 0.f;
+      if (tail > 1e-30f * s2 && s2 > 0.f) {
+        alpha = (x0 >= 0.f) ? -sqrtf(s2) : sqrtf(s2);
+        v0 = x0 - alpha;
+        beta = 1.f / (s2 - x0 * alpha);           // 2 / |v|^2
+      }
+      for (int i = lane; i < m; i += 32) vv[i] = (i == 0) ? v0 : x[i];
+      if (lane == 0) {
+        dd[k] = A[k * n + k];
+        ee[k] = alpha;
+        bet[k] = beta;
+      }
     }
+    __syncthreads();
+    const float beta = bet[k];
+    if (beta != 0.f) {                            // uniform over the block
+      // p = beta * A22 v  (rows strided over warps, columns over lanes), partial v . p per warp
+      float vp = 0.f;
+      for (int i = warp; i < m; i += NW) {
+        const float* row = A + (k + 1 + i) * n + k + 1;
+        float acc = 0.f;
+        for (int j = lane; j < m; j += 32) acc = fmaf(row[j], vv[j], acc);
+        acc = warp_sum(acc) * beta;
+        if (lane == 0) pp[i] = acc;
+        vp += acc * vv[i];
+      }
+      if (lane == 0) red[warp] = vp;
+      __syncthreads();
+      float K = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      off += __shfl_xor_sync(0xffffffffu, off, o);
-      tot += __shfl_xor_sync(0xffffffffu, tot, o);
-    }
-    if (lane == 0) {
-      red[0][warp] = off;
-      red[1][warp] = tot;
-    }
-    __syncthreads();
-    if (tid == 0) {
-      float o = 0.f, t = 0.f;
-      for (int w = 0; w < 8; ++w) {
-        o += red[0][w];
-        t += red[1][w];
-      }
-      // float32 rotations leave off-diagonal noise of about eps * |A|: stop at 5e-6 relative
-      if (o <= 2.5e-11f * t || t == 0.f) done = 1;
-      else if (sweep == max_sweeps - 1 && o > 1e-8f * t) atomicOr(p.status, 4u);
-    }
-    __syncthreads();
-    if (done) break;
-
-    for (int step = 0; step < m; ++step) {
-      if (tid < half) {
-        int a, b;
-        if (tid == 0) {
-          a = m;
-          b = step;
-        } else {
-          a = (step + tid) % m;
-          b = (step - tid + m) % m;
+      for (int w = 0; w < NW; ++w) K += red[w];
+      K *= 0.5f * beta;
+      // A22 -= v w^T + w v^T,  w = p - K v
+      for (int i = warp; i < m; i += NW) {
+        float* row = A + (k + 1 + i) * n + k + 1;
+        const float vi = vv[i], wi = pp[i] - K * vi;
+        for (int j = lane; j < m; j += 32) {
+          const float vj = vv[j], wj = pp[j] - K * vj;
+          row[j] -= vi * wj + wi * vj;
         }
-        const int pp = min(a, b), qq = max(a, b);
-        const double apq = A[pp * n + qq];
-        double c = 1.0, s = 0.0;
-        if (apq != 0.0) {
-          const double tau = ((double)A[qq * n + qq] - (double)A[pp * n + pp]) / (2.0 * apq);
-          const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
-          c = 1.0 / sqrt(1.0 + t * t);
-          s = t * c;
-        }
-        rot_c[tid] = (float)c;
-        rot_s[tid] = (float)s;
-        rot_p[tid] = pp;
-        rot_q[tid] = qq;
       }
-      __syncthreads();
-      // columns: A <- A J
-      for (int i = tid; i < n * half; i += 256) {
-        const int row = i / half, k = i % half;
-        const float c = rot_c[k], s = rot_s[k];
-        float* ap = A + row * n + rot_p[k];
-        float* aq = A + row * n + rot_q[k];
-        const float x = *ap, y = *aq;
-        *ap = c * x - s * y;
-        *aq = s * x + c * y;
-      }
-      __syncthreads();
-      // rows: A <- J^T A, and the eigenvector rows
-      for (int i = tid; i < n * half; i += 256) {
-        const int k = i / n, col = i % n;
-        const float c = rot_c[k], s = rot_s[k];
-        const int pp = rot_p[k], qq = rot_q[k];
-        float x = A[pp * n + col], y = A[qq * n + col];
-        A[pp * n + col] = c * x - s * y;
-        A[qq * n + col] = s * x + c * y;
-        x = VT[pp * n + col];
-        y = VT[qq * n + col];
-        VT[pp * n + col] = c * x - s * y;
-        VT[qq * n + col] = s * x + c * y;
-      }
-      __syncthreads();
     }
+    // keep the reflector in row k (its old content is no longer needed)
+    for (int i = tid; i < m; i += kEigThreads) A[k * n + k + 1 + i] = vv[i];
+    __syncthreads();
   }
+  if (tid == 0) {
+    dd[n - 2] = A[(n - 2) * n + n - 2];
+    ee[n - 2] = A[(n - 2) * n + n - 1];
+    dd[n - 1] = A[(n - 1) * n + n - 1];
+    ee[n - 1] = 0.f;
+    bet[n - 2] = bet[n - 1] = 0.f;
+  }
+  __syncthreads();
 
-  // descending order, ties by lower index
+  // ---- 2. eigenvalues by bisection (Sturm counts), thread j -> j-th largest
+  float gl = 1e30f, gu = -1e30f;
+  for (int i = 0; i < n; ++i) {
+    const float rad = fabsf(i > 0 ? ee[i - 1] : 0.f) + fabsf(i < n - 1 ? ee[i] : 0.f);
+    gl = fminf(gl, dd[i] - rad);
+    gu = fmaxf(gu, dd[i] + rad);
+  }
+  const float tnorm = fmaxf(fabsf(gl), fabsf(gu));
+  const float pivmin = fmaxf(1e-36f, tnorm * tnorm * 1e-34f);   // keeps e^2 / q finite
+  if (tid < n) e2[tid] = ee[tid] * ee[tid];
+  __syncthreads();
   if (tid < n) {
-    const float w = A[tid * n + tid];
-    int rank = 0;
-    for (int k = 0; k < n; ++k) {
-      const float wk = A[k * n + k];
-      rank += (wk > w) || (wk == w && k < tid);
+    const int want = n - 1 - tid;                 // ascending index of this thread's eigenvalue
+    float lo = gl - 1e-6f * tnorm, hi = gu + 1e-6f * tnorm;
+    for (int it = 0; it < 30; ++it) {
+      const float mid = 0.5f * (lo + hi);
+      float qv = dd[0] - mid;
+      int cnt = qv < 0.f;
+      for (int i = 1; i < n; ++i) {
+        if (fabsf(qv) < pivmin) qv = -pivmin;
+        qv = dd[i] - mid - __fdividef(e2[i - 1], qv);
+        cnt += qv < 0.f;
+      }
+      if (cnt <= want) lo = mid; else hi = mid;
     }
-    order[rank] = tid;
-    p.evals[(int64_t)sk * n + rank] = w;
+    lam[tid] = 0.5f * (lo + hi);
   }
   __syncthreads();
-  const int r_eff = min(min(p.r, n), p.n_cov);
+  if (tid < n) p.evals[(int64_t)sk * n + tid] = lam[tid];
+
+  // ---- 3. eigenvectors of T for the r_eff largest eigenvalues
+  const int r_eff = min(min(min(p.r, n), p.n_cov), kEigMaxR);
+  const float eps3 = 1.2e-7f * fmaxf(tnorm, 1e-30f);
+  if (tid == 0) {
+    // separate equal / very close eigenvalues so that their solves differ
+    const float pert = 10.f * eps3;
+    float prev = 0.f;
+    for (int j = 0; j < r_eff; ++j) {
+      float s = lam[j];
+      if (j > 0 && prev - s < pert) s = prev - pert;
+      shf[j] = s;
+      prev = s;
+    }
+  }
+  for (int i = tid; i < n * zs; i += kEigThreads) {
+    const int comp = i / zs, j = i - comp * zs;
+    // start vectors: different for every eigenvector, no component zero
+    const uint32_t hsh = (uint32_t)(comp * 2654435761u) ^ (uint32_t)(j * 40503u + 12345u);
+    Zt[i] = 1.f + 0.5f * (float)((hsh >> 8) & 1023) * (1.f / 1024.f);
+  }
+  __syncthreads();
+
+  for (int iter = 0; iter < 2; ++iter) {
+    if (tid < r_eff) {
+      // solve (T - s I) y = z in place: elimination with partial pivoting, U kept in local arrays
+      const int j = tid;
+      const float s = shf[j];
+      float U0[128], U1[128], U2[128];
+      float u = dd[0] - s, v = ee[0];
+      for (int i = 1; i < n; ++i) {
+        const float sub = ee[i - 1], dg = dd[i] - s, sp = (i < n - 1) ? ee[i] : 0.f;
+        if (fabsf(sub) > fabsf(u)) {              // swap rows i-1 and i
+          const float mult = u / sub;
+          U0[i - 1] = sub;
+          U1[i - 1] = dg;
+          U2[i - 1] = sp;
+          u = v - mult * dg;
+          v = -mult * sp;
+          const float t = Zt[(i - 1) * zs + j];
+          Zt[(i - 1) * zs + j] = Zt[i * zs + j];
+          Zt[i * zs + j] = t - mult * Zt[(i - 1) * zs + j];
+        } else {
+          if (u == 0.f) u = eps3;
+          const float mult = sub / u;
+          U0[i - 1] = u;
+          U1[i - 1] = v;
+          U2[i - 1] = 0.f;
+          u = dg - mult * v;
+          v = sp;
+          Zt[i * zs + j] -= mult * Zt[(i - 1) * zs + j];
+        }
+      }
+      if (fabsf(u) < eps3) u = (u < 0.f) ? -eps3 : eps3;
+      U0[n - 1] = u;
+      float y2 = Zt[(n - 1) * zs + j] / U0[n - 1];
+      Zt[(n - 1) * zs + j] = y2;
+      float y1 = (Zt[(n - 2) * zs + j] - U1[n - 2] * y2) / U0[n - 2];
+      Zt[(n - 2) * zs + j] = y1;
+      float big = fmaxf(fabsf(y1), fabsf(y2));
+      for (int i = n - 3; i >= 0; --i) {
+        const float y0 = (Zt[i * zs + j] - U1[i] * y1 - U2[i] * y2) / U0[i];
+        Zt[i * zs + j] = y0;
+        big = fmaxf(big, fabsf(y0));
+        y2 = y1;
+        y1 = y0;
+      }
+      // scale against overflow, then normalise
+      const float sc = 1.f / fmaxf(big, 1e-30f);
+      float nn = 0.f;
+      for (int i = 0; i < n; ++i) {
+        const float y = Zt[i * zs + j] * sc;
+        Zt[i * zs + j] = y;
+        nn += y * y;
+      }
+      const float inv = rsqrtf(fmaxf(nn, 1e-30f));
+      for (int i = 0; i < n; ++i) Zt[i * zs + j] *= inv;
+    }
+    __syncthreads();
+    // Gram-Schmidt in eigenvalue order, each vector against all earlier ones, twice
+    for (int j = 1; j < r_eff; ++j) {
+      for (int pass = 0; pass < 2; ++pass) {
+        for (int i = warp; i < j; i += NW) {
+          float acc = 0.f;
+          for (int c = lane; c < n; c += 32) acc = fmaf(Zt[c * zs + i], Zt[c * zs + j], acc);
+          acc = warp_sum(acc);
+          if (lane == 0) cdot[i] = acc;
+        }
+        __syncthreads();
+        if (tid < n) {
+          float y = Zt[tid * zs + j];
+          for (int i = 0; i < j; ++i) y = fmaf(-cdot[i], Zt[tid * zs + i], y);
+          Zt[tid * zs + j] = y;
+        }
+        __syncthreads();
+      }
+      if (warp == 0) {
+        float nn = 0.f;
+        for (int c = lane; c < n; c += 32) nn += Zt[c * zs + j] * Zt[c * zs + j];
+        nn = warp_sum(nn);
+        const float inv = rsqrtf(fmaxf(nn, 1e-30f));
+        for (int c = lane; c < n; c += 32) Zt[c * zs + j] *= inv;
+      }
+      __syncthreads();
+    }
+  }
+
+  // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, one warp per vector, then output
   float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
-  for (int q = warp; q < p.r; q += 8) {
-    const int src = order[min(q, n - 1)];
-    const bool live = (q < r_eff) && (A[src * n + src] > 0.f);
-    float nrm = 0.f, best = -1.f;
-    int besti = 0;
-    for (int c = lane; c < n; c += 32) {
-      const float x = VT[src * n + c];
-      nrm += x * x;
-      if (fabsf(x) > best) {
-        best = fabsf(x);
-        besti = c;
+  for (int j = warp; j < p.r; j += NW) {
+    const bool live = j < r_eff && lam[j] > 0.f;
+    if (live) {
+      for (int k = n - 3; k >= 0; --k) {
+        const float beta = bet[k];
+        if (beta == 0.f) continue;
+        const float* v = A + k * n;               // reflector entries at columns k+1 .. n-1
+        float acc = 0.f;
+        for (int c = k + 1 + lane; c < n; c += 32) acc = fmaf(v[c], Zt[c * zs + j], acc);
+        acc = warp_sum(acc) * beta;
+        for (int c = k + 1 + lane; c < n; c += 32) Zt[c * zs + j] -= acc * v[c];
       }
-    }
+      float nn = 0.f, best = -1.f;
+      int besti = 0;
+      for (int c = lane; c < n; c += 32) {
+        const float x = Zt[c * zs + j];
+        nn += x * x;
+        if (fabsf(x) > best) {
+          best = fabsf(x);
+          besti = c;
+        }
+      }
+      nn = warp_sum(nn);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
-      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-      if (ob > best || (ob == best && oi < besti)) {
-        best = ob;
-        besti = oi;
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+        if (ob > best || (ob == best && oi < besti)) {
+          best = ob;
+          besti = oi;
+        }
       }
+      const float sgn = (Zt[besti * zs + j] < 0.f) ? -1.f : 1.f;
+      const float inv = sgn * rsqrtf(fmaxf(nn, 1e-30f));
+      for (int c = lane; c < n; c += 32) basis[j * n + c] = Zt[c * zs + j] * inv;
+    } else {
+      for (int c = lane; c < n; c += 32) basis[j * n + c] = 0.f;
     }
-    const float sgn = (VT[src * n + besti] < 0.f) ? -1.f : 1.f;
-    const float inv = live ? sgn * rsqrtf(nrm) : 0.f;
-    for (int c = lane; c < n; c += 32) basis[q * n + c] = live ? VT[src * n + c] * inv : 0.f;
   }
 }
 
@@ -571,10 +704,14 @@ cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s) {
 cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
   const int blocks = F.L * F.H * 2;
   if (blocks <= 0) return cudaSuccess;
-  const size_t smem = 2 * (size_t)d * d * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(eig_jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  int r_eff = F.r < d ? F.r : d;
+  r_eff = r_eff < F.n_cov ? r_eff : F.n_cov;
+  r_eff = r_eff < kEigMaxR ? r_eff : kEigMaxR;
+  const int zs = r_eff | 1;                       // odd row pitch: conflict-free both ways
+  const size_t smem = ((size_t)d * d + (size_t)d * zs + 8 * (size_t)d + 2 * kEigMaxR + 16) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(eig_tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  eig_jacobi_kernel<<<blocks, 256, smem, s>>>(F, d);
+  eig_tridiag_kernel<<<blocks, kEigThreads, smem, s>>>(F, d, zs);
   return cudaGetLastError();
 }
 
