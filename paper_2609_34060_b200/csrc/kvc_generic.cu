@@ -381,8 +381,9 @@ __device__ __forceinline__ float warp_sum(float x) {
 
 __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int n, int zs) {
   extern __shared__ __align__(16) float smem[];
-  float* A = smem;                    // [n][n]   symmetric; row k right of the diagonal later holds reflector k
-  float* Zt = A + n * n;              // [n][zs]  Zt[i][j] = component i of eigenvector j  (zs = r_eff + 1, odd)
+  const int np = n + 1;               // row pitch of A: a thread can walk its own row without bank conflicts
+  float* A = smem;                    // [n][np]  symmetric; row k right of the diagonal later holds reflector k
+  float* Zt = A + n * np;              // [n][zs]  Zt[i][j] = component i of eigenvector j  (zs = r_eff + 1, odd)
   float* vv = Zt + n * zs;            // [n] current reflector
   float* pp = vv + n;                 // [n] beta * A v
   float* dd = pp + n;                 // [n] diagonal of T
@@ -406,71 +407,87 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
     const int rr = i / n, cc = i - rr * n;
     float a = 0.f;
     for (int pt = 0; pt < p.n_parts; ++pt) a += G[pt * part_stride + i] + G[pt * part_stride + cc * n + rr];
-    A[i] = 0.5f * a;
+    A[rr * np + cc] = 0.5f * a;
   }
   __syncthreads();
-  for (int i = tid; i < n * n; i += kEigThreads) G[i] = A[i];
+  for (int i = tid; i < n * n; i += kEigThreads) G[i] = A[(i / n) * np + (i % n)];
 
-  // ---- 1. Householder tridiagonalisation
-  for (int k = 0; k < n - 2; ++k) {
-    const int m = n - k - 1;                      // order of the trailing block; x = A[k][k+1 .. n-1]
-    const float* x = A + k * n + k + 1;
-    if (warp == 0) {
-      float s2 = 0.f;
-      for (int i = lane; i < m; i += 32) s2 += x[i] * x[i];
-      s2 = warp_sum(s2);
-      const float x0 = x[0];
-      const float tail = s2 - x0 * x0;            // energy below the sub-diagonal entry
-      float alpha = x0, beta = 0.f, v0 = 0.f;
-      if (tail > 1e-30f * s2 && s2 > 0.f) {
-        alpha = (x0 >= 0.f) ? -sqrtf(s2) : sqrtf(s2);
-        v0 = x0 - alpha;
-        beta = 1.f / (s2 - x0 * alpha);           // 2 / |v|^2
-      }
-      for (int i = lane; i < m; i += 32) vv[i] = (i == 0) ? v0 : x[i];
-      if (lane == 0) {
-        dd[k] = A[k * n + k];
-        ee[k] = alpha;
-        bet[k] = beta;
-      }
-    }
-    __syncthreads();
-    const float beta = bet[k];
-    if (beta != 0.f) {                            // uniform over the block
-      // p = beta * A22 v  (rows strided over warps, columns over lanes), partial v . p per warp
-      float vp = 0.f;
-      for (int i = warp; i < m; i += NW) {
-        const float* row = A + (k + 1 + i) * n + k + 1;
-        float acc = 0.f;
-        for (int j = lane; j < m; j += 32) acc = fmaf(row[j], vv[j], acc);
-        acc = warp_sum(acc) * beta;
-        if (lane == 0) pp[i] = acc;
-        vp += acc * vv[i];
-      }
-      if (lane == 0) red[warp] = vp;
-      __syncthreads();
-      float K = 0.f;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) K += red[w];
-      K *= 0.5f * beta;
-      // A22 -= v w^T + w v^T,  w = p - K v
-      for (int i = warp; i < m; i += NW) {
-        float* row = A + (k + 1 + i) * n + k + 1;
-        const float vi = vv[i], wi = pp[i] - K * vi;
-        for (int j = lane; j < m; j += 32) {
-          const float vj = vv[j], wj = pp[j] - K * vj;
-          row[j] -= vi * wj + wi * vj;
+  // ---- 1. Householder tridiagonalisation.  Thread (row, half) owns half of one row of the
+  // trailing block in the matrix-vector product and in the rank-2 update: no shuffles, the
+  // loads of a row are independent and pipeline.
+  {
+    const int trow = tid >> 1, thalf = tid & 1;   // kEigThreads = 2 * 128 rows
+    for (int k = 0; k < n - 2; ++k) {
+      const int m = n - k - 1;                    // order of the trailing block; x = A[k][k+1 .. n-1]
+      const float* x = A + k * np + k + 1;
+      if (warp == 0) {
+        float s2 = 0.f;
+        for (int i = lane; i < m; i += 32) s2 += x[i] * x[i];
+        s2 = warp_sum(s2);
+        const float x0 = x[0];
+        const float tail = s2 - x0 * x0;          // energy below the sub-diagonal entry
+        float alpha = x0, beta = 0.f, v0 = 0.f;
+        if (tail > 1e-30f * s2 && s2 > 0.f) {
+          alpha = (x0 >= 0.f) ? -sqrtf(s2) : sqrtf(s2);
+          v0 = x0 - alpha;
+          beta = 1.f / (s2 - x0 * alpha);         // 2 / |v|^2
+        }
+        for (int i = lane; i < m; i += 32) vv[i] = (i == 0) ? v0 : x[i];
+        if (lane == 0) {
+          dd[k] = A[k * np + k];
+          ee[k] = alpha;
+          bet[k] = beta;
         }
       }
+      __syncthreads();
+      const float beta = bet[k];
+      if (beta != 0.f) {                          // uniform over the block
+        const int j0 = thalf ? (m >> 1) : 0, j1 = thalf ? m : (m >> 1);
+        float* row = A + (k + 1 + trow) * np + k + 1;
+        // p = beta * A22 v : two partial sums per row
+        {
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          if (trow < m) {
+            int j = j0;
+            for (; j + 3 < j1; j += 4) {
+              a0 = fmaf(row[j], vv[j], a0);
+              a1 = fmaf(row[j + 1], vv[j + 1], a1);
+              a2 = fmaf(row[j + 2], vv[j + 2], a2);
+              a3 = fmaf(row[j + 3], vv[j + 3], a3);
+            }
+            for (; j < j1; ++j) a0 = fmaf(row[j], vv[j], a0);
+          }
+          float acc = (a0 + a1) + (a2 + a3);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 1);   // the row's other half sits in the next lane
+          if (thalf == 0 && trow < m) pp[trow] = acc * beta;
+        }
+        __syncthreads();
+        if (warp == 0) {
+          float vp = 0.f;
+          for (int i = lane; i < m; i += 32) vp += vv[i] * pp[i];
+          vp = warp_sum(vp);
+          if (lane == 0) red[0] = 0.5f * beta * vp;
+        }
+        __syncthreads();
+        const float K = red[0];
+        // A22 -= v w^T + w v^T,  w = p - K v
+        if (trow < m) {
+          const float vi = vv[trow], wi = pp[trow] - K * vi;
+          for (int j = j0; j < j1; ++j) {
+            const float vj = vv[j], wj = pp[j] - K * vj;
+            row[j] -= vi * wj + wi * vj;
+          }
+        }
+      }
+      // keep the reflector in row k (its old content is no longer needed)
+      for (int i = tid; i < m; i += kEigThreads) A[k * np + k + 1 + i] = vv[i];
+      __syncthreads();
     }
-    // keep the reflector in row k (its old content is no longer needed)
-    for (int i = tid; i < m; i += kEigThreads) A[k * n + k + 1 + i] = vv[i];
-    __syncthreads();
   }
   if (tid == 0) {
-    dd[n - 2] = A[(n - 2) * n + n - 2];
-    ee[n - 2] = A[(n - 2) * n + n - 1];
-    dd[n - 1] = A[(n - 1) * n + n - 1];
+    dd[n - 2] = A[(n - 2) * np + n - 2];
+    ee[n - 2] = A[(n - 2) * np + n - 1];
+    dd[n - 1] = A[(n - 1) * np + n - 1];
     ee[n - 1] = 0.f;
     bet[n - 2] = bet[n - 1] = 0.f;
   }
@@ -492,12 +509,26 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
     float lo = gl - 1e-6f * tnorm, hi = gu + 1e-6f * tnorm;
     for (int it = 0; it < 30; ++it) {
       const float mid = 0.5f * (lo + hi);
-      float qv = dd[0] - mid;
-      int cnt = qv < 0.f;
+      // Sturm sequence p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}: the eigenvalues below x are
+      // the sign changes.  Division-free; rescaled every four terms against over/underflow.
+      float p0 = 1.f, p1 = dd[0] - mid;
+      int cnt = p1 < 0.f;
       for (int i = 1; i < n; ++i) {
-        if (fabsf(qv) < pivmin) qv = -pivmin;
-        qv = dd[i] - mid - __fdividef(e2[i - 1], qv);
-        cnt += qv < 0.f;
+        float pn = fmaf(dd[i] - mid, p1, -e2[i - 1] * p0);
+        if (pn == 0.f) pn = (p1 < 0.f) ? pivmin : -pivmin;     // a zero counts as a sign change
+        cnt += (pn < 0.f) != (p1 < 0.f);
+        p0 = p1;
+        p1 = pn;
+        if ((i & 3) == 3) {
+          const float mag = fmaxf(fabsf(p0), fabsf(p1));
+          if (mag > 1e12f) {
+            p0 *= 1e-12f;
+            p1 *= 1e-12f;
+          } else if (mag < 1e-12f) {
+            p0 *= 1e12f;
+            p1 *= 1e12f;
+          }
+        }
       }
       if (cnt <= want) lo = mid; else hi = mid;
     }
@@ -614,18 +645,47 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
 
   // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, one warp per vector, then output
   float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
+  // every warp carries up to four of its vectors through the reflectors together (independent
+  // reduction chains overlap)
+  for (int jb = warp * 4; jb < ((r_eff + 3) & ~3); jb += NW * 4) {
+    for (int k = n - 3; k >= 0; --k) {
+      const float beta = bet[k];
+      if (beta == 0.f) continue;
+      const float* v = A + k * np;                // reflector entries at columns k+1 .. n-1
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      for (int c = k + 1 + lane; c < n; c += 32) {
+        const float vc = v[c];
+        const float* z = Zt + c * zs + jb;
+        a0 = fmaf(vc, z[0], a0);
+        if (jb + 1 < r_eff) a1 = fmaf(vc, z[1], a1);
+        if (jb + 2 < r_eff) a2 = fmaf(vc, z[2], a2);
+        if (jb + 3 < r_eff) a3 = fmaf(vc, z[3], a3);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+        a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+        a2 += __shfl_xor_sync(0xffffffffu, a2, o);
+        a3 += __shfl_xor_sync(0xffffffffu, a3, o);
+      }
+      a0 *= beta;
+      a1 *= beta;
+      a2 *= beta;
+      a3 *= beta;
+      for (int c = k + 1 + lane; c < n; c += 32) {
+        const float vc = v[c];
+        float* z = Zt + c * zs + jb;
+        z[0] -= a0 * vc;
+        if (jb + 1 < r_eff) z[1] -= a1 * vc;
+        if (jb + 2 < r_eff) z[2] -= a2 * vc;
+        if (jb + 3 < r_eff) z[3] -= a3 * vc;
+      }
+    }
+  }
+  __syncthreads();
   for (int j = warp; j < p.r; j += NW) {
     const bool live = j < r_eff && lam[j] > 0.f;
     if (live) {
-      for (int k = n - 3; k >= 0; --k) {
-        const float beta = bet[k];
-        if (beta == 0.f) continue;
-        const float* v = A + k * n;               // reflector entries at columns k+1 .. n-1
-        float acc = 0.f;
-        for (int c = k + 1 + lane; c < n; c += 32) acc = fmaf(v[c], Zt[c * zs + j], acc);
-        acc = warp_sum(acc) * beta;
-        for (int c = k + 1 + lane; c < n; c += 32) Zt[c * zs + j] -= acc * v[c];
-      }
       float nn = 0.f, best = -1.f;
       int besti = 0;
       for (int c = lane; c < n; c += 32) {
@@ -708,7 +768,7 @@ cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
   r_eff = r_eff < F.n_cov ? r_eff : F.n_cov;
   r_eff = r_eff < kEigMaxR ? r_eff : kEigMaxR;
   const int zs = r_eff | 1;                       // odd row pitch: conflict-free both ways
-  const size_t smem = ((size_t)d * d + (size_t)d * zs + 8 * (size_t)d + 2 * kEigMaxR + 16) * sizeof(float);
+  const size_t smem = ((size_t)d * (d + 1) + (size_t)d * (zs + 3) + 8 * (size_t)d + 2 * kEigMaxR + 16) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(eig_tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   eig_tridiag_kernel<<<blocks, kEigThreads, smem, s>>>(F, d, zs);
