@@ -501,38 +501,34 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
     gu = fmaxf(gu, dd[i] + rad);
   }
   const float tnorm = fmaxf(fabsf(gl), fabsf(gu));
-  const float pivmin = fmaxf(1e-36f, tnorm * tnorm * 1e-34f);   // keeps e^2 / q finite
-  if (tid < n) e2[tid] = ee[tid] * ee[tid];
+  // bisection runs on T / |T| (entries of magnitude <= 1): pivots and their guard are then
+  // independent of the data's scale; vv / pp are free after step 1
+  const float tscale = fmaxf(tnorm, 1e-30f), tinv = 1.f / tscale;
+  float* ds = vv;                     // scaled diagonal
+  float* es2 = pp;                    // scaled squared off-diagonal
+  if (tid < n) {
+    ds[tid] = dd[tid] * tinv;
+    const float es = ee[tid] * tinv;
+    es2[tid] = es * es;
+    e2[tid] = ee[tid] * ee[tid];
+  }
   __syncthreads();
   if (tid < n) {
     const int want = n - 1 - tid;                 // ascending index of this thread's eigenvalue
-    float lo = gl - 1e-6f * tnorm, hi = gu + 1e-6f * tnorm;
+    float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
     for (int it = 0; it < 30; ++it) {
       const float mid = 0.5f * (lo + hi);
-      // Sturm sequence p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}: the eigenvalues below x are
-      // the sign changes.  Division-free; rescaled every four terms against over/underflow.
-      float p0 = 1.f, p1 = dd[0] - mid;
-      int cnt = p1 < 0.f;
+      // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots
+      float qv = ds[0] - mid;
+      int cnt = qv < 0.f;
       for (int i = 1; i < n; ++i) {
-        float pn = fmaf(dd[i] - mid, p1, -e2[i - 1] * p0);
-        if (pn == 0.f) pn = (p1 < 0.f) ? pivmin : -pivmin;     // a zero counts as a sign change
-        cnt += (pn < 0.f) != (p1 < 0.f);
-        p0 = p1;
-        p1 = pn;
-        if ((i & 3) == 3) {
-          const float mag = fmaxf(fabsf(p0), fabsf(p1));
-          if (mag > 1e12f) {
-            p0 *= 1e-12f;
-            p1 *= 1e-12f;
-          } else if (mag < 1e-12f) {
-            p0 *= 1e12f;
-            p1 *= 1e12f;
-          }
-        }
+        if (fabsf(qv) < 1e-30f) qv = -1e-30f;
+        qv = ds[i] - mid - __fdividef(es2[i - 1], qv);
+        cnt += qv < 0.f;
       }
       if (cnt <= want) lo = mid; else hi = mid;
     }
-    lam[tid] = 0.5f * (lo + hi);
+    lam[tid] = 0.5f * (lo + hi) * tscale;
   }
   __syncthreads();
   if (tid < n) p.evals[(int64_t)sk * n + tid] = lam[tid];
