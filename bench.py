@@ -162,9 +162,65 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all"):
     return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws, "only": only}
 
 
+def build_ring(cfg: wl.Config, dev, kvc):
+    """Long-context chain that does not fit with every agent's cache resident (config 5): agent 0's
+    cache, two output buffers used in turn, one coefficient set shared by all hops (the shift still
+    differs per hop).  Apply only: there are no resident true targets to fit states from."""
+    rope = kvc.Rope(cfg.theta)
+    pl = wl.prefix_lengths(cfg)
+    npg = wl.n_pages(cfg.T, cfg.page)
+    P = npg + 8
+    tables = [wl.page_table(npg, P, cfg.seed, a, dev) for a in range(3)]
+    k0, v0 = wl.base_cache(cfg, dev, table=tables[0], n_phys=P)
+    a0 = kvc.Cache(k0, v0, T=cfg.T, page_table=tables[0])
+    ring = [kvc.Cache(torch.empty_like(k0), torch.empty_like(v0), T=cfg.T, page_table=tables[1 + i]) for i in range(2)]
+    s = wl.hop_state(cfg, 1, dev)
+    st = kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"])
+    return {"kind": "ring", "rope": rope, "pl": pl, "a0": a0, "ring": ring, "st": st, "true": [a0], "states": [st] * (cfg.n_agents - 1),
+            "only": "apply"}
+
+
+def build_serving(n_requests: int, dev, kvc, seed=0, L=32, H=8, d=128, page=16, theta=500000.0):
+    """Config 4: a ragged serving batch.  One shared page pool holds two copies of every request's
+    cache (source and destination of a hop round alternate); hop round h is ONE kvc_apply_batch
+    over all requests that have more than h agents."""
+    reqs = wl.serving_batch(n_requests, seed=seed)
+    rope = kvc.Rope(theta)
+    pages = [wl.n_pages(r.T, page) for r in reqs]
+    P = 2 * sum(pages) + 16
+    perm = wl.page_table(P, P, seed, 900, "cpu")
+    pool_k = torch.empty((L, P, H, page, d), dtype=torch.bfloat16, device=dev)
+    pool_v = torch.empty((L, P, H, page, d), dtype=torch.bfloat16, device=dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed * 7919 + 4)
+    for t in (pool_k, pool_v):
+        for l in range(L):
+            t[l].normal_(generator=g)
+    caches, states, off = [], [], 0
+    for i, r in enumerate(reqs):
+        ta = perm[off: off + pages[i]].contiguous().to(dev)
+        tb = perm[off + pages[i]: off + 2 * pages[i]].contiguous().to(dev)
+        off += 2 * pages[i]
+        caches.append((kvc.Cache(pool_k, pool_v, T=r.T, page_table=ta), kvc.Cache(pool_k, pool_v, T=r.T, page_table=tb)))
+        c = wl.Config(f"rq{i}", L=L, H=H, d=d, T=r.T, n_agents=r.n_agents, r=r.r, theta=theta, seed=seed * 1000 + i)
+        s = wl.hop_state(c, 1, dev)
+        states.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
+    rounds = []
+    for h in range(1, max(r.n_agents for r in reqs)):
+        items = [kvc.Item(caches[i][(h - 1) % 2], caches[i][h % 2], states[i], r.prefix[h] - r.prefix[h - 1])
+                 for i, r in enumerate(reqs) if r.n_agents > h]
+        rounds.append(items)
+    nb = kvc.kvc_batch_workspace_bytes(n_requests)
+    ws = [torch.empty(nb, dtype=torch.uint8, device=dev) for _ in rounds]
+    staging = [torch.empty(nb, dtype=torch.uint8).pin_memory() for _ in rounds]
+    app = sum(kvc.kvc_apply_bytes(it.src, it.st) for items in rounds for it in items)
+    return {"kind": "serving", "rope": rope, "rounds": rounds, "ws": ws, "staging": staging, "reqs": reqs, "apply_bytes": app,
+            "only": "apply", "launches": len(rounds), "tokens": sum(r.T for r in reqs)}
+
+
 def run_step(W, kvc, ev=None):
     """One pass of the path.  `ev` (optional) collects CUDA-event pairs per kernel family."""
-    pl, rope, n = W["pl"], W["rope"], len(W["true"])
+    pl, rope, n = W.get("pl"), W["rope"], len(W.get("true", []))
 
     def mark(name):
         if ev is None:
@@ -175,6 +231,21 @@ def run_step(W, kvc, ev=None):
         return e
 
     only = W.get("only", "all")
+    if W.get("kind") == "ring":
+        mark("chain_begin")
+        cur = W["a0"]
+        for a in range(1, len(pl)):
+            dst = W["ring"][a % 2]
+            kvc.kvc_apply(cur, W["st"], pl[a] - pl[a - 1], rope, dst)
+            cur = dst
+        mark("chain_end")
+        return
+    if W.get("kind") == "serving":
+        mark("chain_begin")
+        for items, ws, stg in zip(W["rounds"], W["ws"], W["staging"]):
+            kvc.kvc_apply_batch(items, rope, ws, stg)
+        mark("chain_end")
+        return
     if only != "apply":
         for a in range(1, n):
             mark("update_begin")
@@ -188,6 +259,8 @@ def run_step(W, kvc, ev=None):
 
 
 def step_bytes(W, kvc):
+    if W.get("kind") == "serving":
+        return 0, W["apply_bytes"]
     n = len(W["states"]) + 1
     only = W.get("only", "all")
     upd = 0 if only == "apply" else sum(kvc.kvc_update_bytes(W["true"][0], W["states"][a - 1], kvc.KVC_FIT, True)
@@ -233,7 +306,7 @@ def cpu_baseline(cfg: wl.Config, budget_s: float = 20.0):
         per_slab = dt if per_slab is None else max(per_slab, dt)
         t_used += dt
         done += 1
-        hops = cfg.n_agents - 1
+        hops = W["launches"] if serving else cfg.n_agents - 1
         tok = cfg.T
         apply_b = hops * (tok * (8 * cfg.d + 8 * cfg.r) + 2 * cfg.r * cfg.d * 4)
         upd_b = hops * (2 * tok * 8 * cfg.d + tok * 8 * cfg.r + 2 * cfg.r * cfg.d * 4 + 4 * cfg.d * cfg.d * 4)
@@ -248,7 +321,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="llama8b_8k", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default="llama8b_8k", choices=sorted(wl.CONFIGS) + ["serve64"])
+    ap.add_argument("--requests", type=int, default=64, help="serve64: number of concurrent requests")
     ap.add_argument("--impl", default="kvc", choices=["kvc", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "generic", "tc"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -259,11 +333,18 @@ def main():
                     help="profiling aid: time only the chain or only the state updates")
     args = ap.parse_args()
     rank, world, local = _dist()
-    cfg = wl.CONFIGS[args.workload]
+    serving = args.workload == "serve64"
+    cfg = wl.CONFIGS["llama8b_8k" if serving else args.workload]
     if args.layers > 0:
         cfg = cfg.scaled(L=args.layers)
-    config = {"workload": f"{cfg.name}: L={cfg.L} Hkv={cfg.H} d={cfg.d} T={cfg.T} agents={cfg.n_agents} r={cfg.r} "
-                          f"{'paged16' if cfg.paged else 'contiguous'} bf16, seed {cfg.seed}",
+    ring = (not serving) and cfg.paged and cfg.n_agents * cfg.L * cfg.H * cfg.T * cfg.d * 8 > 100e9
+    if serving or ring:
+        args.only, args.no_e2e, args.no_cpu_baseline = "apply", True, True
+    wname = (f"serve64: {args.requests} requests, L={cfg.L} Hkv={cfg.H} d={cfg.d}, T lognormal(median 4096) in [1k,32k], "
+             f"3-6 agents, r in {{16,32,64}}, paged16, one ragged launch per hop round" if serving else
+             f"{cfg.name}: L={cfg.L} Hkv={cfg.H} d={cfg.d} T={cfg.T} agents={cfg.n_agents} r={cfg.r} "
+             f"{'paged16' if cfg.paged else 'contiguous'} bf16, seed {cfg.seed}" + (" (two output buffers in turn)" if ring else ""))
+    config = {"workload": wname,
               "step": "per edge: kvc_state_update(FIT) ; then kvc_chain over all agents",
               "l2": "inputs larger than L2 (126 MB): no flush between iterations", "parallelism": f"replicas x{world}",
               "only": args.only}
@@ -301,11 +382,16 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     kvc.kvc_set_path({"auto": kvc.KVC_PATH_AUTO, "generic": kvc.KVC_PATH_GENERIC, "tc": kvc.KVC_PATH_TC}[args.path])
 
-    W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only)
+    if serving:
+        W = build_serving(args.requests, dev, kvc, seed=rank, L=cfg.L)
+    elif ring:
+        W = build_ring(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
+    else:
+        W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only)
     if args.only != "all":
         args.no_e2e = True
     upd_b, app_b = step_bytes(W, kvc)
-    hops = cfg.n_agents - 1
+    hops = W["launches"] if serving else cfg.n_agents - 1
 
     def barrier():
         torch.cuda.synchronize()
@@ -389,7 +475,8 @@ def main():
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic", "config": config,
-           "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * (hops * 3 + hops),
+           "clocks": clocks, "e2e": e2e,
+           "gpu_launches": args.steps * (hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
            "roofline": roofline,
            "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
                          "us_per_agent_layer": hop_ms * 1e3 / cfg.L,

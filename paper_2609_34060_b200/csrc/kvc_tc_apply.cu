@@ -6,8 +6,8 @@
 // (layer, head, K|V) slab.  Warp roles:
 //   warp 0      TMA producer (one lane): base tile (bf16 128 x 128) + fp32 coefficient tile
 //   warp 1      MMA issuer (one lane) and TMEM owner
-//   warp 2      basis stager: basis[r][d] -> K-major, 128B-swizzled bf16 hi/lo operand
-//   warp 3      idle
+//   warp 2      basis stager (two operand slots, r <= 32); with one slot (r = 64) the team stages
+//   warp 3      store warp: TMA stores of finished tiles, releases the stage
 //   warps 4-7, 8-11   two epilogue groups; a group owns every other tile of the CTA:
 //               convert its coefficient rows to bf16 hi/lo in place, wait for the MMA, read the
 //               accumulator row from TMEM, rotate/add/round, write the row back in place, and
@@ -59,21 +59,31 @@ struct Tile {
   const DevItem* it;
   const ItemMaps* mp;
   int item, slab, is_v, t0, l, h;
+  bool first;        // first tile of its slab within this walk (the slab's operands must be staged)
   bool has_coeff;    // the tile holds covered rows of a live state
   bool uses_basis;   // its slab has a live state (basis staged for the slab)
 };
 
+// Walks a contiguous range of global tiles.  All divisions happen once in init(); stepping to
+// the next tile is a few increments (every role of the CTA steps through every tile).
 struct TileWalker {
   const ApplyTcLaunch* p;
-  int64_t tile, end;
-  int item;
-  int64_t item_lo, item_hi;
+  int64_t remaining;
+  int item, slab2, n_slab2, tt, tps, l, h;
+  bool first;
+  const DevItem* it;
 
+  __device__ void load_item() {
+    it = p->items ? p->items + item : &p->one;
+    tps = it->tiles_per_slab;
+    n_slab2 = it->L * it->H * 2;
+  }
   __device__ void init(const ApplyTcLaunch* pp, int64_t begin, int64_t end_) {
     p = pp;
-    tile = begin;
-    end = end_;
+    remaining = end_ - begin;
     item = 0;
+    first = true;
+    int64_t local = begin;
     if (p->items) {
       int lo = 0, hi = p->n_items;
       while (hi - lo > 1) {
@@ -81,41 +91,59 @@ struct TileWalker {
         if (begin >= p->tile_prefix[mid]) lo = mid; else hi = mid;
       }
       item = lo;
-      item_lo = p->tile_prefix[item];
-      item_hi = p->tile_prefix[item + 1];
-    } else {
-      item_lo = 0;
-      item_hi = p->total_tiles;
+      local = begin - p->tile_prefix[item];
+    }
+    load_item();
+    if (remaining > 0) {
+      while (tps == 0 || n_slab2 == 0) {          // items without tiles hold no global tile index
+        ++item;
+        load_item();
+        local = 0;
+      }
+      tt = (int)(local % tps);
+      slab2 = (int)(local / tps);
+      const int slab = slab2 >> 1;
+      l = slab / it->H;
+      h = slab - l * it->H;
     }
   }
-  __device__ bool done() const { return tile >= end; }
-  __device__ void get(Tile& t) {
-    while (tile >= item_hi) {   // items with zero tiles are skipped
-      ++item;
-      item_lo = item_hi;
-      item_hi = p->tile_prefix[item + 1];
-    }
-    const DevItem* it = p->items ? p->items + item : &p->one;
+  __device__ bool done() const { return remaining <= 0; }
+  __device__ void get(Tile& t) const {
     t.it = it;
     t.mp = p->maps ? p->maps + item : &p->one_maps;
     t.item = item;
-    const int64_t local = tile - item_lo;
-    const int tt = (int)(local % it->tiles_per_slab);
-    const int64_t sk = local / it->tiles_per_slab;
-    t.is_v = (int)(sk & 1);
-    t.slab = (int)(sk >> 1);
-    t.l = t.slab / it->H;
-    t.h = t.slab % it->H;
+    t.first = first;
+    t.is_v = slab2 & 1;
+    t.slab = slab2 >> 1;
+    t.l = l;
+    t.h = h;
     t.t0 = tt * kTileTok;
     t.uses_basis = it->st.r > 0 && it->st.n_cov > 0;
     t.has_coeff = t.uses_basis && t.t0 < it->st.n_cov;
   }
-  __device__ void next() { ++tile; }
+  __device__ void next() {
+    if (--remaining <= 0) return;
+    first = false;
+    if (++tt < tps) return;
+    first = true;
+    tt = 0;
+    ++slab2;
+    if ((slab2 & 1) == 0) {                       // K and V of one (layer, head) are adjacent
+      if (++h == it->H) {
+        h = 0;
+        ++l;
+      }
+    }
+    if (slab2 == n_slab2) {
+      do {
+        ++item;
+        load_item();
+      } while (tps == 0 || n_slab2 == 0);
+      slab2 = 0;
+      l = h = 0;
+    }
+  }
 };
-
-__device__ __forceinline__ bool same_slab(const Tile& a, const Tile& b) {
-  return a.item == b.item && a.slab == b.slab && a.is_v == b.is_v;
-}
 
 // Shared-memory control block (after the tiles)
 template <int NSTAGE, int NB>
@@ -127,6 +155,38 @@ struct Ctrl {
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// basis[r][d] of one slab -> K-major, 128B-swizzled bf16 operand: row = channel, [B1 | B2] along the
+// row (hi and lo parts of 32 basis vectors per rank block).  Tasks are strided over the callers.
+template <int RB>
+__device__ __forceinline__ void stage_basis(const Tile& t, uint8_t* slot_ptr, int first, int stride) {
+  const DevItem& it = *t.it;
+  const int r = it.st.r;
+  const void* basis = t.is_v ? it.st.basis_v : it.st.basis_k;
+  for (int task = first; task < RB * 512; task += stride) {
+    const int b = task >> 9, ch = task & 127, k8 = (task >> 7) & 3;
+    float v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int q = 32 * b + 8 * k8 + e;
+      float x = 0.f;
+      if (q < r) {
+        const int64_t off = ((int64_t)t.slab * r + q) * 128 + ch;
+        x = it.st.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
+                             : reinterpret_cast<const float*>(basis)[off];
+      }
+      v[e] = x;
+    }
+    uint4 hi, lo;
+    split2(v[0], v[1], hi.x, lo.x);
+    split2(v[2], v[3], hi.y, lo.y);
+    split2(v[4], v[5], hi.z, lo.z);
+    split2(v[6], v[7], hi.w, lo.w);
+    uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
+    *reinterpret_cast<uint4*>(row + ((k8 ^ (ch & 7)) << 4)) = hi;
+    *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
+  }
+}
 
 // ------------------------------------------------------------------ the kernel
 // Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 basis stager, 3 store warp, 4..19 the team.
@@ -161,7 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
     }
     for (int b = 0; b < NB; ++b) {
-      mbar_init(smem_u32(&ctrl->basis_full[b]), 1);
+      mbar_init(smem_u32(&ctrl->basis_full[b]), NB == 1 ? kTeamThreads : 1);   // who stages: team or stager warp
       mbar_init(smem_u32(&ctrl->basis_empty[b]), 1);
     }
     mbar_init(smem_u32(&ctrl->drain), 1);
@@ -240,17 +300,15 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       TileWalker w;
       w.init(&p, tile_begin, tile_end);
       uint32_t i = 0, slabs = 0;
-      bool have_prev = false, in_slab = false;
-      Tile prev;
+      bool in_slab = false;
       int slot = 0;
       for (; !w.done(); w.next(), ++i) {
         Tile t;
         w.get(t);
         const int s = i % NSTAGE, g = i & 1;
         const uint32_t use = i / NSTAGE, acc_use = i >> 1;
-        const bool new_slab = !have_prev || !same_slab(prev, t);
-        if (new_slab) {
-          if (in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));   // all MMAs of the old slab done => slot free
+        if (t.first) {
+          if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));   // all MMAs of the old slab done => slot free
           in_slab = false;
           if (t.uses_basis) {
             slot = slabs % NB;
@@ -259,8 +317,6 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             in_slab = true;
           }
         }
-        prev = t;
-        have_prev = true;
         if (!mbar_wait(smem_u32(&ctrl->conv[s]), use & 1u, abort_flag)) break;
         if (!mbar_wait(smem_u32(&ctrl->acc_empty[g]), (acc_use & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
@@ -285,65 +341,31 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         }
         umma_commit(smem_u32(&ctrl->mma_done[g]));
       }
-      if (in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));
+      if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));
       umma_commit(smem_u32(&ctrl->drain));
       mbar_wait_drain(smem_u32(&ctrl->drain), 0);
     }
   } else if (warp == 2) {
-    // =============================================================== basis stager
-    TileWalker w;
-    w.init(&p, tile_begin, tile_end);
-    bool have_prev = false;
-    Tile prev;
-    uint32_t slabs = 0;
-    for (; !w.done(); w.next()) {
-      Tile t;
-      w.get(t);
-      const bool new_slab = !have_prev || !same_slab(prev, t);
-      prev = t;
-      have_prev = true;
-      if (!new_slab || !t.uses_basis) continue;
-      const int slot = slabs % NB;
-      int ok = 1;
-      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->basis_empty[slot]), ((slabs / NB) & 1u) ^ 1u, abort_flag) ? 1 : 0;
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      ++slabs;
-      const DevItem& it = *t.it;
-      const int r = it.st.r;
-      const void* basis = t.is_v ? it.st.basis_v : it.st.basis_k;
-      uint8_t* slot_ptr = smem + NSTAGE * kStageBytes + slot * kBasisSlotBytes;
-      for (int b = 0; b < RB; ++b) {
-        for (int pass = 0; pass < 4; ++pass) {
-          const int ch = pass * 32 + lane;                 // operand row = channel
-          uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
-#pragma unroll
-          for (int k8 = 0; k8 < 4; ++k8) {
-            float v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int q = 32 * b + 8 * k8 + e;
-              float x = 0.f;
-              if (q < r) {
-                const int64_t off = ((int64_t)t.slab * r + q) * 128 + ch;
-                x = it.st.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
-                                     : reinterpret_cast<const float*>(basis)[off];
-              }
-              v[e] = x;
-            }
-            uint4 hi, lo;
-            uint32_t* hp = reinterpret_cast<uint32_t*>(&hi);
-            uint32_t* lp = reinterpret_cast<uint32_t*>(&lo);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) split2(v[2 * e], v[2 * e + 1], hp[e], lp[e]);
-            *reinterpret_cast<uint4*>(row + (((k8) ^ (ch & 7)) << 4)) = hi;
-            *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
-          }
-        }
+    // =============================================================== basis stager (two-slot variant only)
+    if constexpr (NB > 1) {
+      TileWalker w;
+      w.init(&p, tile_begin, tile_end);
+      uint32_t slabs = 0;
+      for (; !w.done(); w.next()) {
+        Tile t;
+        w.get(t);
+        if (!t.first || !t.uses_basis) continue;
+        const int slot = slabs % NB;
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->basis_empty[slot]), ((slabs / NB) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        ++slabs;
+        stage_basis<RB>(t, smem + NSTAGE * kStageBytes + slot * kBasisSlotBytes, lane, 32);
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
       }
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
     }
   } else if (warp == 3) {
     // =============================================================== store warp
@@ -465,6 +487,18 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       return true;
     };
 
+    const int tt = tid - 128;                       // 0 .. 511
+    if constexpr (NB == 1) {                         // single operand slot: the team stages it
+      if (!w.done()) {
+        Tile t0;
+        w.get(t0);
+        if (t0.uses_basis) {
+          stage_basis<RB>(t0, smem + NSTAGE * kStageBytes, tt, kTeamThreads);
+          fence_proxy_async();
+          mbar_arrive(smem_u32(&ctrl->basis_full[0]));
+        }
+      }
+    }
     if (!w.done()) alive = convert(wn, 0);
     for (; alive && !w.done(); w.next(), ++i) {
       // ---- 1. get the next tile's coefficients converted and its MMA going
@@ -484,6 +518,19 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      if constexpr (NB == 1) {
+        // The MMAs of tile i are complete.  If tile i + 1 opens a new slab, tile i was the last
+        // reader of the operand slot: restage it now (512 threads: about a microsecond).
+        if (!wn.done()) {
+          Tile tn;
+          wn.get(tn);
+          if (tn.uses_basis && tn.first) {
+            stage_basis<RB>(tn, smem + NSTAGE * kStageBytes, tt, kTeamThreads);
+            fence_proxy_async();
+            mbar_arrive(smem_u32(&ctrl->basis_full[0]));
+          }
+        }
+      }
 
       // ---- 3. rotate, add, round: row m, this warp's channel quarter, in place
       const int tok = t.t0 + m;
