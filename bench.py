@@ -31,14 +31,17 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2609_34060_b200 import dist_util  # noqa: E402
 from paper_2609_34060_b200 import workloads as wl  # noqa: E402
 
 METRIC = "corrected-KV GB/s (algorithmic HBM bytes / time), whole hot path"
 UNIT = "GB/s"
 HBM_FALLBACK_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one apply launch, from the ncu capture
-# summarised under profiles/ (bytes per launch on the benchmark workload), or None.
-APPLY_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one apply launch on the 8K workload, from the ncu
+# capture summarised in profiles/apply_tc_kernel_dram_traffic_L16.md: measured at L = 16
+# (812.65 MB read + 492.24 MB written per launch) and scaled by 2 to L = 32 (traffic is
+# proportional to the token-slabs processed).  None for other workloads.
+APPLY_TRAFFIC_BYTES_LLAMA8B_8K = 2 * (812_650_000 + 492_240_000)
 
 
 def _peaks():
@@ -306,7 +309,7 @@ def cpu_baseline(cfg: wl.Config, budget_s: float = 20.0):
         per_slab = dt if per_slab is None else max(per_slab, dt)
         t_used += dt
         done += 1
-        hops = W["launches"] if serving else cfg.n_agents - 1
+        hops = cfg.n_agents - 1
         tok = cfg.T
         apply_b = hops * (tok * (8 * cfg.d + 8 * cfg.r) + 2 * cfg.r * cfg.d * 4)
         upd_b = hops * (2 * tok * 8 * cfg.d + tok * 8 * cfg.r + 2 * cfg.r * cfg.d * 4 + 4 * cfg.d * cfg.d * 4)
@@ -383,7 +386,7 @@ def main():
     kvc.kvc_set_path({"auto": kvc.KVC_PATH_AUTO, "generic": kvc.KVC_PATH_GENERIC, "tc": kvc.KVC_PATH_TC}[args.path])
 
     if serving:
-        W = build_serving(args.requests, dev, kvc, seed=rank, L=cfg.L)
+        W = build_serving(args.requests, dev, kvc, seed=rank, L=cfg.L)      # each rank serves its own batch
     elif ring:
         W = build_ring(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
     else:
@@ -420,10 +423,7 @@ def main():
     last_path = kvc.kvc_last_path()
     flags = kvc.kvc_status_poll()
     assert flags == 0, f"a kernel flagged an anomaly: {flags}"
-    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = dist_util.max_over_ranks(ms_total, dev) / args.steps
     value = world * (upd_b + app_b) / (ms_step * 1e-3) / 1e9
 
     # end to end: inputs from pinned host memory, corrected caches back to the host
@@ -454,10 +454,8 @@ def main():
             e2e_step()
         e.record()
         barrier()
-        te = torch.tensor([b.elapsed_time(e)], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * (upd_b + app_b) / (float(te.item()) / n_e2e * 1e-3) / 1e9, "unit": UNIT,
+        te = dist_util.max_over_ranks(b.elapsed_time(e), dev)
+        e2e = {"value": world * (upd_b + app_b) / (te / n_e2e * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
         del host_in, host_out
 
@@ -470,7 +468,8 @@ def main():
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": APPLY_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": app_b // hops,
+                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0) else None,
+                "algorithmic_bytes_per_launch": app_b // hops,
                 "us_per_launch": hop_ms * 1e3}
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
