@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant
 // The input is the sum of the partial Gram matrices, symmetrised; it is written back so that
 // the final Gram matrix stays readable in the workspace.
 // ---------------------------------------------------------------------------------
-constexpr int kEigThreads = 256;
+constexpr int kEigThreads = 512;
 constexpr int kEigMaxR = 64;
 
 __device__ __forceinline__ float warp_sum(float x) {
@@ -381,7 +381,7 @@ __device__ __forceinline__ float warp_sum(float x) {
 
 __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int n, int zs) {
   extern __shared__ __align__(16) float smem[];
-  const int np = n + 1;               // row pitch of A: a thread can walk its own row without bank conflicts
+  const int np = n + 4;               // row pitch of A = 4 (mod 32): four threads per row, eight rows per warp, no bank conflicts
   float* A = smem;                    // [n][np]  symmetric; row k right of the diagonal later holds reflector k
   float* Zt = A + n * np;              // [n][zs]  Zt[i][j] = component i of eigenvector j  (zs = r_eff + 1, odd)
   float* vv = Zt + n * zs;            // [n] current reflector
@@ -402,85 +402,110 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
   float* G = p.gram + (int64_t)sk * n * n;
   const int64_t part_stride = (int64_t)p.L * p.H * 2 * n * n;
 
-  // ---- load: fixed-order sum of the partial Grams, symmetrised
+  // ---- load: fixed-order sum of the partial Grams (coalesced), then symmetrise in place
   for (int i = tid; i < n * n; i += kEigThreads) {
     const int rr = i / n, cc = i - rr * n;
     float a = 0.f;
-    for (int pt = 0; pt < p.n_parts; ++pt) a += G[pt * part_stride + i] + G[pt * part_stride + cc * n + rr];
-    A[rr * np + cc] = 0.5f * a;
+    for (int pt = 0; pt < p.n_parts; ++pt) a += G[pt * part_stride + i];
+    A[rr * np + cc] = a;
+  }
+  __syncthreads();
+  for (int i = tid; i < n * n; i += kEigThreads) {
+    const int rr = i / n, cc = i - rr * n;
+    if (cc > rr) {                                 // one thread per unordered pair
+      const float m2 = 0.5f * (A[rr * np + cc] + A[cc * np + rr]);
+      A[rr * np + cc] = m2;
+      A[cc * np + rr] = m2;
+    }
   }
   __syncthreads();
   for (int i = tid; i < n * n; i += kEigThreads) G[i] = A[(i / n) * np + (i % n)];
 
-  // ---- 1. Householder tridiagonalisation.  Thread (row, half) owns half of one row of the
-  // trailing block in the matrix-vector product and in the rank-2 update: no shuffles, the
-  // loads of a row are independent and pipeline.
+  // ---- 1. Householder tridiagonalisation.  Four threads own one row of the trailing block
+  // (columns interleaved), in the matrix-vector product and in the rank-2 update.  Reflector k
+  // lives in row k right of the diagonal (v0 written over x0), so it is never copied; the
+  // threads that own the next pivot row compute its norm and (alpha, beta, v0) at the end of
+  // the update, which leaves two block barriers per step.
   {
-    const int trow = tid >> 1, thalf = tid & 1;   // kEigThreads = 2 * 128 rows
+    const int trow = tid >> 2, tq = tid & 3;
+    // scalar set-up of step k from the row's squared norm s2 (x = A[k][k+1 ..]); one thread
+    auto setup = [&](int k, float s2) {
+      float* x = A + k * np + k + 1;
+      const float x0 = x[0];
+      const float tail = s2 - x0 * x0;            // energy below the sub-diagonal entry
+      float alpha = x0, beta = 0.f, v0 = 0.f;
+      if (tail > 1e-30f * s2 && s2 > 0.f) {
+        alpha = (x0 >= 0.f) ? -sqrtf(s2) : sqrtf(s2);
+        v0 = x0 - alpha;
+        beta = 1.f / (s2 - x0 * alpha);           // 2 / |v|^2
+      }
+      dd[k] = A[k * np + k];
+      ee[k] = alpha;
+      bet[k] = beta;
+      x[0] = v0;                                  // row k now holds the reflector
+      red[k & 1] = 0.f;                           // accumulates v . p of step k (the other slot may still be read)
+    };
+    if (warp == 0) {
+      float s2 = 0.f;
+      for (int i = 1 + lane; i < n; i += 32) s2 += A[i] * A[i];
+      s2 = warp_sum(s2);
+      if (lane == 0) setup(0, s2);
+    }
+    __syncthreads();
     for (int k = 0; k < n - 2; ++k) {
-      const int m = n - k - 1;                    // order of the trailing block; x = A[k][k+1 .. n-1]
-      const float* x = A + k * np + k + 1;
-      if (warp == 0) {
-        float s2 = 0.f;
-        for (int i = lane; i < m; i += 32) s2 += x[i] * x[i];
-        s2 = warp_sum(s2);
-        const float x0 = x[0];
-        const float tail = s2 - x0 * x0;          // energy below the sub-diagonal entry
-        float alpha = x0, beta = 0.f, v0 = 0.f;
-        if (tail > 1e-30f * s2 && s2 > 0.f) {
-          alpha = (x0 >= 0.f) ? -sqrtf(s2) : sqrtf(s2);
-          v0 = x0 - alpha;
-          beta = 1.f / (s2 - x0 * alpha);         // 2 / |v|^2
-        }
-        for (int i = lane; i < m; i += 32) vv[i] = (i == 0) ? v0 : x[i];
-        if (lane == 0) {
-          dd[k] = A[k * np + k];
-          ee[k] = alpha;
-          bet[k] = beta;
-        }
-      }
-      __syncthreads();
+      const int m = n - k - 1;                    // order of the trailing block
+      const float* v = A + k * np + k + 1;        // reflector k, entries 0 .. m-1
       const float beta = bet[k];
+      float* row = A + (k + 1 + trow) * np + k + 1;
+      float K = 0.f;
       if (beta != 0.f) {                          // uniform over the block
-        const int j0 = thalf ? (m >> 1) : 0, j1 = thalf ? m : (m >> 1);
-        float* row = A + (k + 1 + trow) * np + k + 1;
-        // p = beta * A22 v : two partial sums per row
-        {
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          if (trow < m) {
-            int j = j0;
-            for (; j + 3 < j1; j += 4) {
-              a0 = fmaf(row[j], vv[j], a0);
-              a1 = fmaf(row[j + 1], vv[j + 1], a1);
-              a2 = fmaf(row[j + 2], vv[j + 2], a2);
-              a3 = fmaf(row[j + 3], vv[j + 3], a3);
-            }
-            for (; j < j1; ++j) a0 = fmaf(row[j], vv[j], a0);
-          }
-          float acc = (a0 + a1) + (a2 + a3);
-          acc += __shfl_xor_sync(0xffffffffu, acc, 1);   // the row's other half sits in the next lane
-          if (thalf == 0 && trow < m) pp[trow] = acc * beta;
-        }
-        __syncthreads();
-        if (warp == 0) {
-          float vp = 0.f;
-          for (int i = lane; i < m; i += 32) vp += vv[i] * pp[i];
-          vp = warp_sum(vp);
-          if (lane == 0) red[0] = 0.5f * beta * vp;
-        }
-        __syncthreads();
-        const float K = red[0];
-        // A22 -= v w^T + w v^T,  w = p - K v
+        // p = beta * A22 v : four partial sums per row, combined by two shuffles
+        float a0 = 0.f, a1 = 0.f;
         if (trow < m) {
-          const float vi = vv[trow], wi = pp[trow] - K * vi;
-          for (int j = j0; j < j1; ++j) {
-            const float vj = vv[j], wj = pp[j] - K * vj;
-            row[j] -= vi * wj + wi * vj;
+          int j = tq;
+          for (; j + 4 < m; j += 8) {
+            a0 = fmaf(row[j], v[j], a0);
+            a1 = fmaf(row[j + 4], v[j + 4], a1);
           }
+          if (j < m) a0 = fmaf(row[j], v[j], a0);
+        }
+        float acc = a0 + a1;
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        float vp = 0.f;
+        if (tq == 0 && trow < m) {
+          acc *= beta;
+          pp[trow] = acc;
+          vp = acc * v[trow];
+        }
+        vp = warp_sum(vp);                        // 8 rows per warp
+        if (lane == 0 && vp != 0.f) atomicAdd(&red[k & 1], vp);
+        __syncthreads();
+        K = 0.5f * beta * red[k & 1];
+      }
+      // A22 -= v w^T + w v^T,  w = p - K v ; the owners of the next pivot row also sum its squares
+      float s2n = 0.f;
+      if (trow < m) {
+        if (beta != 0.f) {
+          const float vi = v[trow], wi = pp[trow] - K * vi;
+#pragma unroll 4
+          for (int j = tq; j < m; j += 4) {
+            const float vj = v[j], wj = pp[j] - K * vj;
+            const float a = row[j] - (vi * wj + wi * vj);
+            row[j] = a;
+            if (trow == 0 && j >= 1) s2n = fmaf(a, a, s2n);
+          }
+        } else if (trow == 0) {
+          for (int j = tq; j < m; j += 4)
+            if (j >= 1) s2n = fmaf(row[j], row[j], s2n);
         }
       }
-      // keep the reflector in row k (its old content is no longer needed)
-      for (int i = tid; i < m; i += kEigThreads) A[k * np + k + 1 + i] = vv[i];
+      if (warp == 0) {                            // rows 0 .. 7 of the trailing block; row 0 = next pivot row
+        s2n += __shfl_xor_sync(0xffffffffu, s2n, 1);
+        s2n += __shfl_xor_sync(0xffffffffu, s2n, 2);
+        __syncwarp();
+        if (lane == 0 && k + 1 < n - 2) setup(k + 1, s2n);
+      }
       __syncthreads();
     }
   }
@@ -516,7 +541,7 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
   if (tid < n) {
     const int want = n - 1 - tid;                 // ascending index of this thread's eigenvalue
     float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
-    for (int it = 0; it < 30; ++it) {
+    for (int it = 0; it < 26; ++it) {             // interval 2 |T| -> 2^-25 |T|: float32 resolution
       const float mid = 0.5f * (lo + hi);
       // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots
       float qv = ds[0] - mid;
@@ -560,40 +585,46 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
       // solve (T - s I) y = z in place: elimination with partial pivoting, U kept in local arrays
       const int j = tid;
       const float s = shf[j];
-      float U0[128], U1[128], U2[128];
+      // U of the pivoted LU kept in local arrays: reciprocal pivot, first super-diagonal; the second
+      // super-diagonal is e[i+1] where rows were swapped (one bit per row), else zero
+      float R0[128], U1[128];
+      uint32_t swp[4] = {0u, 0u, 0u, 0u};
       float u = dd[0] - s, v = ee[0];
+      float xp = Zt[j];                           // running right-hand side entry of the pivot row
       for (int i = 1; i < n; ++i) {
         const float sub = ee[i - 1], dg = dd[i] - s, sp = (i < n - 1) ? ee[i] : 0.f;
+        const float xi = Zt[i * zs + j];
         if (fabsf(sub) > fabsf(u)) {              // swap rows i-1 and i
-          const float mult = u / sub;
-          U0[i - 1] = sub;
+          const float rs = 1.f / sub;
+          const float mult = u * rs;
+          R0[i - 1] = rs;
           U1[i - 1] = dg;
-          U2[i - 1] = sp;
+          swp[(i - 1) >> 5] |= 1u << ((i - 1) & 31);
           u = v - mult * dg;
           v = -mult * sp;
-          const float t = Zt[(i - 1) * zs + j];
-          Zt[(i - 1) * zs + j] = Zt[i * zs + j];
-          Zt[i * zs + j] = t - mult * Zt[(i - 1) * zs + j];
+          Zt[(i - 1) * zs + j] = xi;
+          xp = xp - mult * xi;
         } else {
           if (u == 0.f) u = eps3;
-          const float mult = sub / u;
-          U0[i - 1] = u;
+          const float ru = 1.f / u;
+          const float mult = sub * ru;
+          R0[i - 1] = ru;
           U1[i - 1] = v;
-          U2[i - 1] = 0.f;
           u = dg - mult * v;
           v = sp;
-          Zt[i * zs + j] -= mult * Zt[(i - 1) * zs + j];
+          Zt[(i - 1) * zs + j] = xp;
+          xp = xi - mult * xp;
         }
       }
       if (fabsf(u) < eps3) u = (u < 0.f) ? -eps3 : eps3;
-      U0[n - 1] = u;
-      float y2 = Zt[(n - 1) * zs + j] / U0[n - 1];
+      float y2 = xp / u;
       Zt[(n - 1) * zs + j] = y2;
-      float y1 = (Zt[(n - 2) * zs + j] - U1[n - 2] * y2) / U0[n - 2];
+      float y1 = (Zt[(n - 2) * zs + j] - U1[n - 2] * y2) * R0[n - 2];
       Zt[(n - 2) * zs + j] = y1;
       float big = fmaxf(fabsf(y1), fabsf(y2));
       for (int i = n - 3; i >= 0; --i) {
-        const float y0 = (Zt[i * zs + j] - U1[i] * y1 - U2[i] * y2) / U0[i];
+        const float u2 = ((swp[i >> 5] >> (i & 31)) & 1u) ? ee[i + 1] : 0.f;
+        const float y0 = (Zt[i * zs + j] - U1[i] * y1 - u2 * y2) * R0[i];
         Zt[i * zs + j] = y0;
         big = fmaxf(big, fabsf(y0));
         y2 = y1;
@@ -764,7 +795,7 @@ cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
   r_eff = r_eff < F.n_cov ? r_eff : F.n_cov;
   r_eff = r_eff < kEigMaxR ? r_eff : kEigMaxR;
   const int zs = r_eff | 1;                       // odd row pitch: conflict-free both ways
-  const size_t smem = ((size_t)d * (d + 1) + (size_t)d * (zs + 3) + 8 * (size_t)d + 2 * kEigMaxR + 16) * sizeof(float);
+  const size_t smem = ((size_t)d * (d + 4) + (size_t)d * (zs + 3) + 8 * (size_t)d + 2 * kEigMaxR + 16) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(eig_tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   eig_tridiag_kernel<<<blocks, kEigThreads, smem, s>>>(F, d, zs);
