@@ -538,22 +538,34 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
     e2[tid] = ee[tid] * ee[tid];
   }
   __syncthreads();
-  if (tid < n) {
-    const int want = n - 1 - tid;                 // ascending index of this thread's eigenvalue
+  {
+    // four threads per eigenvalue: each round tests four interior points, the interval shrinks 5x
+    const int ev = tid >> 2, sub = tid & 3;        // kEigThreads = 4 * 128
+    const int want = n - 1 - ev;                   // ascending index of this group's eigenvalue
     float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
-    for (int it = 0; it < 26; ++it) {             // interval 2 |T| -> 2^-25 |T|: float32 resolution
-      const float mid = 0.5f * (lo + hi);
+    for (int it = 0; it < 12; ++it) {              // 5^12 = 2.4e8 > 2^26
+      const float step = (hi - lo) * 0.2f;
+      const float mid = lo + step * (float)(sub + 1);
       // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots
-      float qv = ds[0] - mid;
-      int cnt = qv < 0.f;
-      for (int i = 1; i < n; ++i) {
-        if (fabsf(qv) < 1e-30f) qv = -1e-30f;
-        qv = ds[i] - mid - __fdividef(es2[i - 1], qv);
-        cnt += qv < 0.f;
+      int cnt = 0;
+      if (ev < n) {
+        float qv = ds[0] - mid;
+        cnt = qv < 0.f;
+        for (int i = 1; i < n; ++i) {
+          if (fabsf(qv) < 1e-30f) qv = -1e-30f;
+          qv = ds[i] - mid - __fdividef(es2[i - 1], qv);
+          cnt += qv < 0.f;
+        }
       }
-      if (cnt <= want) lo = mid; else hi = mid;
+      const bool below = cnt <= want;              // the eigenvalue is at or above this point
+      // the four points are ordered: new lo = last point with `below`, new hi = first without
+      const unsigned grp = __ballot_sync(0xffffffffu, below) >> (lane & ~3) & 0xFu;
+      const int nb = __popc(grp);                  // points 0 .. nb-1 are below (monotone up to rounding)
+      const float nlo = lo + step * (float)nb, nhi = (nb < 4) ? lo + step * (float)(nb + 1) : hi;
+      lo = nlo;
+      hi = nhi;
     }
-    lam[tid] = 0.5f * (lo + hi) * tscale;
+    if (ev < n && sub == 0) lam[ev] = 0.5f * (lo + hi) * tscale;
   }
   __syncthreads();
   if (tid < n) p.evals[(int64_t)sk * n + tid] = lam[tid];
@@ -580,6 +592,10 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
   }
   __syncthreads();
 
+  // scratch for the r_eff x r_eff Gram matrix of the vectors: the lower-left quadrant of A is
+  // free after the reduction (reflectors live right of the diagonal) when r_eff <= n / 2
+  float* S = (2 * r_eff <= n) ? A + (n / 2) * np : cdot + kEigMaxR;
+  const int sp = (2 * r_eff <= n) ? np : (r_eff | 1);
   for (int iter = 0; iter < 2; ++iter) {
     if (tid < r_eff) {
       // solve (T - s I) y = z in place: elimination with partial pivoting, U kept in local arrays
@@ -642,29 +658,48 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
       for (int i = 0; i < n; ++i) Zt[i * zs + j] *= inv;
     }
     __syncthreads();
-    // Gram-Schmidt in eigenvalue order, each vector against all earlier ones, twice
-    for (int j = 1; j < r_eff; ++j) {
-      for (int pass = 0; pass < 2; ++pass) {
-        for (int i = warp; i < j; i += NW) {
+    // Re-orthonormalise all r_eff vectors at once: S = Z^T Z (close to the identity), S = L L^T,
+    // Z <- Z L^-T.  Equivalent to Gram-Schmidt in eigenvalue order, without its r_eff sequential
+    // rounds; S is well conditioned because inverse iteration already separates the vectors.
+    {
+      for (int t2 = tid; t2 < r_eff * r_eff; t2 += kEigThreads) {
+        const int i = t2 / r_eff, j = t2 - i * r_eff;
+        if (j <= i) {
           float acc = 0.f;
-          for (int c = lane; c < n; c += 32) acc = fmaf(Zt[c * zs + i], Zt[c * zs + j], acc);
-          acc = warp_sum(acc);
-          if (lane == 0) cdot[i] = acc;
+          for (int c = 0; c < n; ++c) acc = fmaf(Zt[c * zs + i], Zt[c * zs + j], acc);
+          S[i * sp + j] = acc;
         }
-        __syncthreads();
-        if (tid < n) {
-          float y = Zt[tid * zs + j];
-          for (int i = 0; i < j; ++i) y = fmaf(-cdot[i], Zt[tid * zs + i], y);
-          Zt[tid * zs + j] = y;
-        }
-        __syncthreads();
       }
+      __syncthreads();
       if (warp == 0) {
-        float nn = 0.f;
-        for (int c = lane; c < n; c += 32) nn += Zt[c * zs + j] * Zt[c * zs + j];
-        nn = warp_sum(nn);
-        const float inv = rsqrtf(fmaxf(nn, 1e-30f));
-        for (int c = lane; c < n; c += 32) Zt[c * zs + j] *= inv;
+        for (int j = 0; j < r_eff; ++j) {
+          float dsum = 0.f;
+          for (int k = lane; k < j; k += 32) dsum = fmaf(S[j * sp + k], S[j * sp + k], dsum);
+          dsum = warp_sum(dsum);
+          float piv = S[j * sp + j] - dsum;
+          if (piv < 1e-6f) {                      // (nearly) dependent vectors: keep going, flag it
+            piv = 1e-6f;
+            if (lane == 0) atomicOr(p.status, 4u);
+          }
+          const float ljj = sqrtf(piv), rl = 1.f / ljj;
+          __syncwarp();
+          for (int i = j + 1 + lane; i < r_eff; i += 32) {
+            float acc = S[i * sp + j];
+            for (int k = 0; k < j; ++k) acc = fmaf(-S[i * sp + k], S[j * sp + k], acc);
+            S[i * sp + j] = acc * rl;
+          }
+          if (lane == 0) S[j * sp + j] = rl;      // keep the reciprocal of the diagonal
+          __syncwarp();
+        }
+      }
+      __syncthreads();
+      if (tid < n) {                              // row tid of Z:  x L^T = z  (forward substitution)
+        float* z = Zt + tid * zs;
+        for (int j = 0; j < r_eff; ++j) {
+          float acc = z[j];
+          for (int k = 0; k < j; ++k) acc = fmaf(-z[k], S[j * sp + k], acc);
+          z[j] = acc * S[j * sp + j];
+        }
       }
       __syncthreads();
     }
@@ -795,7 +830,8 @@ cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
   r_eff = r_eff < F.n_cov ? r_eff : F.n_cov;
   r_eff = r_eff < kEigMaxR ? r_eff : kEigMaxR;
   const int zs = r_eff | 1;                       // odd row pitch: conflict-free both ways
-  const size_t smem = ((size_t)d * (d + 4) + (size_t)d * (zs + 3) + 8 * (size_t)d + 2 * kEigMaxR + 16) * sizeof(float);
+  const size_t extra = (2 * r_eff <= d) ? 0 : (size_t)r_eff * (r_eff | 1);   // Gram scratch when A has no free quadrant
+  const size_t smem = ((size_t)d * (d + 4) + (size_t)d * (zs + 3) + 8 * (size_t)d + 2 * kEigMaxR + 16 + extra) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(eig_tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   eig_tridiag_kernel<<<blocks, kEigThreads, smem, s>>>(F, d, zs);
