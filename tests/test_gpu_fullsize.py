@@ -158,3 +158,73 @@ def test_state_update_full_size_sampled_slabs(name):
             assert np.max(np.abs(B @ B.T - np.eye(r))) <= 1e-4
             res = float(np.sum((dl - c @ B) ** 2))
             assert res <= 1.001 * float(np.sum(w[r:])) + 1e-6 * float(np.sum(w)), (res, float(np.sum(w[r:])))
+
+
+def _free_gb():
+    free, _ = torch.cuda.mem_get_info()
+    return free / 2 ** 30
+
+
+def test_serving_batch_full_size_sampled_slabs():
+    """Config 4 as bench.py launches it: 64 ragged requests, one kvc_apply_batch per hop round."""
+    import bench
+    if _free_gb() < 120:
+        pytest.skip("needs about 110 GB of device memory")
+    kvc.kvc_status_reset()
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    W = bench.build_serving(64, DEV, kvc, seed=0)
+    f = orc.rope_inv_freq(128, 500000.0)
+    items = W["rounds"][0]                         # hop round 1: every request takes part
+    g = np.random.default_rng(5)
+    picks = [(int(g.integers(len(items))), int(g.integers(32)), int(g.integers(8))) for _ in range(5)]
+    picks += [(int(np.argmin([it.src.T for it in items])), 31, 7), (int(np.argmax([it.src.T for it in items])), 0, 0)]
+    before = {}
+    for (i, l, h) in picks:                        # the source slabs, read before the launch
+        for which in ("k", "v"):
+            before[(i, l, h, which)] = _slab_bits(items[i].src, which, l, h)
+    kvc.kvc_apply_batch(items, W["rope"], W["ws"][0], W["staging"][0])
+    torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+    assert kvc.kvc_status_poll() == 0
+    for (i, l, h) in picks:
+        it = items[i]
+        for which in ("k", "v"):
+            c = (it.st.coeff_k if which == "k" else it.st.coeff_v)[l, h].cpu().numpy()
+            b = (it.st.basis_k if which == "k" else it.st.basis_v)[l, h].cpu().numpy()
+            ref, exp = orc.apply_slab(before[(i, l, h, which)], c, b, it.shift, f, it.src.T, which == "k")
+            got = _slab_bits(it.dst, which, l, h)
+            assert hp.tol_ratio(got, ref) <= 1.0, (i, l, h, which, it.src.T, it.st.r)
+            assert hp.ulp_mismatch_fraction(got, exp) < 1e-2
+            # the source pages are only read
+            assert np.array_equal(_slab_bits(it.src, which, l, h), before[(i, l, h, which)])
+
+
+def test_long_context_full_size_sampled_slabs():
+    """Config 5 as bench.py launches it: L=80, T=32768, r=64, paged, two output buffers in turn."""
+    import bench
+    if _free_gb() < 60:
+        pytest.skip("needs about 50 GB of device memory")
+    cfg = wl.CONFIGS["llama70b_32k"]
+    kvc.kvc_status_reset()
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    W = bench.build_ring(cfg, DEV, kvc)
+    pl, rope, st = W["pl"], W["rope"], W["st"]
+    f = hp.inv_freq(cfg)
+    kvc.kvc_apply(W["a0"], st, pl[1] - pl[0], rope, W["ring"][1])
+    kvc.kvc_apply(W["ring"][1], st, pl[2] - pl[1], rope, W["ring"][0])
+    torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+    assert kvc.kvc_status_poll() == 0
+    for (l, h) in [(0, 0), (79, 7), (41, 3)]:
+        for which in ("k", "v"):
+            c = (st.coeff_k if which == "k" else st.coeff_v)[l, h].cpu().numpy()
+            b = (st.basis_k if which == "k" else st.basis_v)[l, h].cpu().numpy()
+            src = _slab_bits(W["a0"], which, l, h)
+            ref1, exp1 = orc.apply_slab(src, c, b, pl[1] - pl[0], f, cfg.T, which == "k")
+            got1 = _slab_bits(W["ring"][1], which, l, h)
+            assert hp.tol_ratio(got1, ref1) <= 1.0
+            assert hp.ulp_mismatch_fraction(got1, exp1) < 1e-2
+            ref2, _ = orc.apply_slab(exp1, c, b, pl[2] - pl[1], f, cfg.T, which == "k")
+            gv = orc.bf16_to_f64(_slab_bits(W["ring"][0], which, l, h))
+            bad = np.abs(gv - ref2) > hp.BF16_REL * np.abs(ref2) + hp.BF16_ABS
+            assert bad.mean() < 2e-3
