@@ -332,6 +332,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
+    ap.add_argument("--rank", type=int, default=0, help="override the rank r (experiments)")
+    ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
     ap.add_argument("--only", default="all", choices=["all", "apply", "update"],
                     help="profiling aid: time only the chain or only the state updates")
     args = ap.parse_args()
@@ -340,6 +342,10 @@ def main():
     cfg = wl.CONFIGS["llama8b_8k" if serving else args.workload]
     if args.layers > 0:
         cfg = cfg.scaled(L=args.layers)
+    if args.rank > 0:
+        cfg = cfg.scaled(r=args.rank)
+    if args.paged >= 0:
+        cfg = cfg.scaled(paged=bool(args.paged), image_spans=())
     ring = (not serving) and cfg.paged and cfg.n_agents * cfg.L * cfg.H * cfg.T * cfg.d * 8 > 100e9
     if serving or ring:
         args.only, args.no_e2e, args.no_cpu_baseline = "apply", True, True
@@ -468,7 +474,7 @@ def main():
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0) else None,
+                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0) else None,
                 "algorithmic_bytes_per_launch": app_b // hops,
                 "us_per_launch": hop_ms * 1e3}
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

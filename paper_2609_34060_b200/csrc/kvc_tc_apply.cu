@@ -248,29 +248,33 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       w.get(t);
       const int s = i % NSTAGE;
       const uint32_t use = i / NSTAGE;
+      const DevItem& it = *t.it;
+      // paged source: one lane per page of the tile; the ids are fetched BEFORE waiting for the
+      // stage, so that their global-memory latency hides behind the wait
+      const bool paged = it.src.page_table != nullptr;
+      const int page = it.src.page_mask + 1;
+      int id = -1, n_pages = 0;
+      if (paged) {
+        const int per_tile = kTileTok >> it.src.page_shift;
+        const int first = t.t0 >> it.src.page_shift;
+        n_pages = min(per_tile, ((it.src.T + page - 1) >> it.src.page_shift) - first);
+        if (lane < n_pages) id = it.src.page_table[first + lane];
+      }
       int ok = 1;
       if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      const DevItem& it = *t.it;
       const uint32_t st_base = stages + s * kStageBytes;
       const uint32_t bar = smem_u32(&ctrl->full[s]);
       const CUtensorMap* smap = t.is_v ? &t.mp->src_v : &t.mp->src_k;
       const uint32_t cbytes = t.has_coeff ? RB * kCoeffBlkBytes : 0;
-      if (!it.src.page_table) {
+      if (!paged) {
         if (lane == 0) {
           mbar_expect_tx(bar, cbytes + kBaseBytes);
           tma_load_5d(st_base, smap, bar, 0, t.t0, t.h, 0, t.l);
           tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t.t0, t.h, 0, t.l);
         }
       } else {
-        // one lane per page of the tile
-        const int page = it.src.page_mask + 1;
-        const int per_tile = kTileTok >> it.src.page_shift;
-        const int first = t.t0 >> it.src.page_shift;
-        const int n_pages = min(per_tile, ((it.src.T + page - 1) >> it.src.page_shift) - first);
-        int id = -1;
-        if (lane < n_pages) id = it.src.page_table[first + lane];
         const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.src.n_phys;
         if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
         const int n_ok = __popc(__ballot_sync(0xffffffffu, valid));
@@ -377,31 +381,17 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       w.get(t);
       const int s = i % NSTAGE;
       const uint32_t use = i / NSTAGE;
-      int ok = 1;
-      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), use & 1u, abort_flag) ? 1 : 0;
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
       const DevItem& it = *t.it;
-      const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
-      const uint32_t st_base = stages + s * kStageBytes;
-      uint8_t* st_ptr = smem + s * kStageBytes;
-      if (!it.dst.page_table) {
-        bool src_ok = true;   // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
-        if (lane == 0 && src_ok) {
-          tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
-          tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
-        }
-      } else {
-        // one lane per destination page; the last, partial page goes out row by row so that
-        // rows >= T stay untouched; pages whose source could not be loaded are skipped
-        const int dpage = it.dst.page_mask + 1;
+      // paged destination: one lane per page; ids (and the validity of the matching source pages)
+      // are fetched before waiting for the tile
+      const bool dpaged = it.dst.page_table != nullptr;
+      const int dpage = it.dst.page_mask + 1;
+      int id = -1, n_pages = 0, first = 0;
+      bool src_ok = true;
+      if (dpaged) {
         const int per_tile = kTileTok >> it.dst.page_shift;
-        const int first = t.t0 >> it.dst.page_shift;
-        const int n_pages = min(per_tile, ((it.dst.T + dpage - 1) >> it.dst.page_shift) - first);
-        const int last_pg = (it.dst.T - 1) >> it.dst.page_shift;
-        const bool last_partial = (it.dst.T & it.dst.page_mask) != 0;
-        int id = -1;
-        bool src_ok = true;
+        first = t.t0 >> it.dst.page_shift;
+        n_pages = min(per_tile, ((it.dst.T + dpage - 1) >> it.dst.page_shift) - first);
         if (lane < n_pages) {
           id = it.dst.page_table[first + lane];
           if (it.src.page_table) {
@@ -411,6 +401,24 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
               if ((unsigned)it.src.page_table[sp] >= (unsigned)it.src.n_phys) src_ok = false;
           }
         }
+      }
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), use & 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
+      const uint32_t st_base = stages + s * kStageBytes;
+      uint8_t* st_ptr = smem + s * kStageBytes;
+      if (!dpaged) {
+        if (lane == 0) {          // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
+          tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
+          tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
+        }
+      } else {
+        // the last, partial page goes out row by row so that rows >= T stay untouched; pages whose
+        // source could not be loaded are skipped
+        const int last_pg = (it.dst.T - 1) >> it.dst.page_shift;
+        const bool last_partial = (it.dst.T & it.dst.page_mask) != 0;
         const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.dst.n_phys;
         if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
         const bool partial = last_partial && (first + lane) == last_pg;
@@ -418,7 +426,6 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, t.h, id, t.l);
           tma_store_5d(dmap, st_base + kHalfBytes + lane * dpage * 128, 64, 0, t.h, id, t.l);
         }
-        // the partial page, if this tile holds it: which lane owns it, is it storable
         const unsigned pm = __ballot_sync(0xffffffffu, valid && src_ok && partial);
         if (pm) {
           const int u = __ffs(pm) - 1;
