@@ -146,9 +146,10 @@ struct TileWalker {
 };
 
 // Shared-memory control block (after the tiles)
-template <int NSTAGE, int NB>
+template <int NSTAGE, int NSC, int NB>
 struct Ctrl {
-  uint64_t full[NSTAGE], conv[NSTAGE], ready[NSTAGE], empty[NSTAGE];
+  uint64_t full[NSTAGE], ready[NSTAGE], empty[NSTAGE];      // base-tile ring
+  uint64_t cfull[NSC], conv[NSC], cempty[NSC];              // coefficient ring
   uint64_t mma_done[2], acc_empty[2];
   uint64_t basis_full[NB], basis_empty[NB];
   uint64_t drain;
@@ -191,17 +192,24 @@ __device__ __forceinline__ void stage_basis(const Tile& t, uint8_t* slot_ptr, in
 // ------------------------------------------------------------------ the kernel
 // Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 basis stager, 3 store warp, 4..19 the team.
 // Team warp e (0..15): TMEM lane quadrant e & 3 (rows 32q..32q+31), channel quarter e >> 2.
-template <int RB, int NSTAGE, int NB>
+//
+// Two rings of shared-memory slots: NSTAGE base tiles (alive from the load until the TMA store has
+// read them) and NSC coefficient tiles (alive only until the tile's MMAs have completed), so that
+// the short-lived operand does not hold a long-lived slot.
+template <int RB, int NSTAGE, int NSC, int NB>
 __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
-  constexpr int kStageBytes = kBaseBytes + RB * kCoeffBlkBytes;
+  constexpr int kStageBytes = kBaseBytes;
+  constexpr int kCoeffSlotBytes = RB * kCoeffBlkBytes;
   constexpr int kBasisSlotBytes = RB * kBasisBlkBytes;
+  constexpr int kOperandOff = NSTAGE * kStageBytes + NSC * kCoeffSlotBytes;   // basis slots start here
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t stages = base;
-  const uint32_t bases = base + NSTAGE * kStageBytes;
-  Ctrl<NSTAGE, NB>* ctrl = reinterpret_cast<Ctrl<NSTAGE, NB>*>(smem + NSTAGE * kStageBytes + NB * kBasisSlotBytes);
+  const uint32_t coeffs = base + NSTAGE * kStageBytes;
+  const uint32_t bases = base + kOperandOff;
+  Ctrl<NSTAGE, NSC, NB>* ctrl = reinterpret_cast<Ctrl<NSTAGE, NSC, NB>*>(smem + kOperandOff + NB * kBasisSlotBytes);
   volatile int* abort_flag = &ctrl->abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -212,9 +220,13 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
   if (tid == 0) {
     for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(smem_u32(&ctrl->full[s]), 1);
-      mbar_init(smem_u32(&ctrl->conv[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->ready[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int c = 0; c < NSC; ++c) {
+      mbar_init(smem_u32(&ctrl->cfull[c]), 1);
+      mbar_init(smem_u32(&ctrl->conv[c]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->cempty[c]), 1);
     }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
@@ -242,7 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     // =============================================================== TMA producer (whole warp)
     TileWalker w;
     w.init(&p, tile_begin, tile_end);
-    uint32_t i = 0;
+    uint32_t i = 0, c_issued = 0;
     for (; !w.done(); w.next(), ++i) {
       Tile t;
       w.get(t);
@@ -260,17 +272,32 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         n_pages = min(per_tile, ((it.src.T + page - 1) >> it.src.page_shift) - first);
         if (lane < n_pages) id = it.src.page_table[first + lane];
       }
+      // coefficient tile first: its slot turns over quickly
+      const int c = i % NSC;
       int ok = 1;
-      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
+      if (lane == 0) {
+        ok = mbar_wait(smem_u32(&ctrl->cempty[c]), ((i / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+        if (ok) {
+          const uint32_t cbar = smem_u32(&ctrl->cfull[c]);
+          mbar_expect_tx(cbar, t.has_coeff ? (uint32_t)kCoeffSlotBytes : 0u);
+          if (t.has_coeff) {
+            const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
+#pragma unroll
+            for (int b = 0; b < RB; ++b)
+              tma_load_3d(coeffs + c * kCoeffSlotBytes + b * kCoeffBlkBytes, cmap, cbar, 32 * b, t.t0, t.slab);
+          }
+          ++c_issued;
+          ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
+        }
+      }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       const uint32_t st_base = stages + s * kStageBytes;
       const uint32_t bar = smem_u32(&ctrl->full[s]);
       const CUtensorMap* smap = t.is_v ? &t.mp->src_v : &t.mp->src_k;
-      const uint32_t cbytes = t.has_coeff ? RB * kCoeffBlkBytes : 0;
       if (!paged) {
         if (lane == 0) {
-          mbar_expect_tx(bar, cbytes + kBaseBytes);
+          mbar_expect_tx(bar, kBaseBytes);
           tma_load_5d(st_base, smap, bar, 0, t.t0, t.h, 0, t.l);
           tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t.t0, t.h, 0, t.l);
         }
@@ -278,17 +305,12 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.src.n_phys;
         if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
         const int n_ok = __popc(__ballot_sync(0xffffffffu, valid));
-        if (lane == 0) mbar_expect_tx(bar, cbytes + (uint32_t)(n_ok * page * 256));
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_ok * page * 256));
         __syncwarp();
         if (valid) {
           tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, t.h, id, t.l);
           tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, t.h, id, t.l);
         }
-      }
-      if (t.has_coeff && lane == 0) {
-        const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
-#pragma unroll
-        for (int b = 0; b < RB; ++b) tma_load_3d(st_base + kBaseBytes + b * kCoeffBlkBytes, cmap, bar, 32 * b, t.t0, t.slab);
       }
       __syncwarp();
     }
@@ -297,6 +319,8 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const uint32_t issued = i;
       for (uint32_t k = (issued > NSTAGE ? issued - NSTAGE : 0); k < issued; ++k)
         mbar_wait_drain(smem_u32(&ctrl->full[k % NSTAGE]), (k / NSTAGE) & 1u);
+      for (uint32_t k = (c_issued > NSC ? c_issued - NSC : 0); k < c_issued; ++k)
+        mbar_wait_drain(smem_u32(&ctrl->cfull[k % NSC]), (k / NSC) & 1u);
     }
   } else if (warp == 1) {
     // =============================================================== MMA issuer
@@ -309,8 +333,8 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       for (; !w.done(); w.next(), ++i) {
         Tile t;
         w.get(t);
-        const int s = i % NSTAGE, g = i & 1;
-        const uint32_t use = i / NSTAGE, acc_use = i >> 1;
+        const int c = i % NSC, g = i & 1;
+        const uint32_t use = i / NSC, acc_use = i >> 1;
         if (t.first) {
           if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));   // all MMAs of the old slab done => slot free
           in_slab = false;
@@ -321,12 +345,12 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             in_slab = true;
           }
         }
-        if (!mbar_wait(smem_u32(&ctrl->conv[s]), use & 1u, abort_flag)) break;
+        if (!mbar_wait(smem_u32(&ctrl->conv[c]), use & 1u, abort_flag)) break;
         if (!mbar_wait(smem_u32(&ctrl->acc_empty[g]), (acc_use & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
         if (t.has_coeff) {
           const uint32_t d_tmem = tmem_base + g * 128;
-          const uint32_t a0 = stages + s * kStageBytes + kBaseBytes;
+          const uint32_t a0 = coeffs + c * kCoeffSlotBytes;
           const uint32_t b0 = bases + slot * kBasisSlotBytes;
           uint32_t acc = 0;
 #pragma unroll
@@ -344,6 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           }
         }
         umma_commit(smem_u32(&ctrl->mma_done[g]));
+        umma_commit(smem_u32(&ctrl->cempty[c]));      // the coefficient slot may be refilled
       }
       if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));
       umma_commit(smem_u32(&ctrl->drain));
@@ -365,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         ++slabs;
-        stage_basis<RB>(t, smem + NSTAGE * kStageBytes + slot * kBasisSlotBytes, lane, 32);
+        stage_basis<RB>(t, smem + kOperandOff + slot * kBasisSlotBytes, lane, 32);
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
@@ -466,16 +491,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     auto convert = [&](TileWalker& cw, uint32_t ci) {
       Tile t;
       cw.get(t);
-      const int s = ci % NSTAGE;
-      const uint32_t use = ci / NSTAGE;
-      bool ok = mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag);
+      const int c = ci % NSC;
+      const uint32_t use = ci / NSC;
+      bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), use & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return false;
       if (t.has_coeff) {
-        uint8_t* st_ptr = smem + s * kStageBytes;
+        uint8_t* c_ptr = smem + NSTAGE * kStageBytes + c * kCoeffSlotBytes;
 #pragma unroll
         for (int b = 0; b < RB; ++b) {
-          uint8_t* row = st_ptr + kBaseBytes + b * kCoeffBlkBytes + crow * 128;
+          uint8_t* row = c_ptr + b * kCoeffBlkBytes + crow * 128;
           // this thread's 8 coefficients: fp32 chunks 2*cpart, 2*cpart+1 of the row
           const float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
           const float4 f1 = *reinterpret_cast<const float4*>(row + (((2 * cpart + 1) ^ csw) << 4));
@@ -490,7 +515,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         }
         fence_proxy_async();
       }
-      mbar_arrive(smem_u32(&ctrl->conv[s]));
+      mbar_arrive(smem_u32(&ctrl->conv[c]));
       return true;
     };
 
@@ -500,7 +525,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         Tile t0;
         w.get(t0);
         if (t0.uses_basis) {
-          stage_basis<RB>(t0, smem + NSTAGE * kStageBytes, tt, kTeamThreads);
+          stage_basis<RB>(t0, smem + kOperandOff, tt, kTeamThreads);
           fence_proxy_async();
           mbar_arrive(smem_u32(&ctrl->basis_full[0]));
         }
@@ -532,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           Tile tn;
           wn.get(tn);
           if (tn.uses_basis && tn.first) {
-            stage_basis<RB>(tn, smem + NSTAGE * kStageBytes, tt, kTeamThreads);
+            stage_basis<RB>(tn, smem + kOperandOff, tt, kTeamThreads);
             fence_proxy_async();
             mbar_arrive(smem_u32(&ctrl->basis_full[0]));
           }
@@ -540,6 +565,9 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       }
 
       // ---- 3. rotate, add, round: row m, this warp's channel quarter, in place
+      ok = mbar_wait(smem_u32(&ctrl->full[s]), (i / NSTAGE) & 1u, abort_flag);   // the base tile has landed
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       const int tok = t.t0 + m;
       const bool in_range = tok < it.src.T;
       const bool covered = t.has_coeff && tok < it.st.n_cov;
@@ -663,17 +691,19 @@ static bool build_maps(const DevItem& it, ItemMaps* mp) {
   return ok;
 }
 
-template <int RB, int NSTAGE, int NB>
+template <int RB, int NSTAGE, int NSC, int NB>
 static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
-  const size_t smem = 1024 + (size_t)NSTAGE * (kBaseBytes + RB * kCoeffBlkBytes) + (size_t)NB * RB * kBasisBlkBytes +
-                      sizeof(Ctrl<NSTAGE, NB>);
+  const size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)NB * RB * kBasisBlkBytes +
+                      sizeof(Ctrl<NSTAGE, NSC, NB>);
+  static_assert(1024 + NSTAGE * kBaseBytes + NSC * RB * kCoeffBlkBytes + NB * RB * kBasisBlkBytes + sizeof(Ctrl<NSTAGE, NSC, NB>) <= 232448,
+                "exceeds the shared memory of one CTA");
   static bool set = false;
   if (!set) {
-    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     set = true;
   }
-  apply_tc_kernel<RB, NSTAGE, NB><<<grid, kThreads, smem, s>>>(L);
+  apply_tc_kernel<RB, NSTAGE, NSC, NB><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError();
 }
 
@@ -681,7 +711,7 @@ static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s) {
   const int sms = sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
-  cudaError_t e = (max_r <= 32) ? launch_t<1, 4, 2>(L, grid, s) : launch_t<2, 3, 1>(L, grid, s);
+  cudaError_t e = (max_r <= 32) ? launch_t<1, 5, 2, 2>(L, grid, s) : launch_t<2, 4, 2, 1>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
