@@ -47,6 +47,7 @@ struct ApplyTcLaunch {
   const DevItem* items;        // device table or nullptr => `one`
   const ItemMaps* maps;        // device table or nullptr => `one_maps`
   const int64_t* tile_prefix;  // device [n_items + 1]
+  const int64_t* cta_bounds;   // device [grid + 1] first tile of every CTA, or nullptr => equal tile counts
   int32_t n_items, pairing;
   int64_t total_tiles;
   uint32_t* status;
@@ -59,6 +60,7 @@ struct Tile {
   const DevItem* it;
   const ItemMaps* mp;
   int item, slab, is_v, t0, l, h;
+  int nb;            // rank blocks of 32 the item's state really has
   bool first;        // first tile of its slab within this walk (the slab's operands must be staged)
   bool has_coeff;    // the tile holds covered rows of a live state
   bool uses_basis;   // its slab has a live state (basis staged for the slab)
@@ -118,6 +120,7 @@ struct TileWalker {
     t.l = l;
     t.h = h;
     t.t0 = tt * kTileTok;
+    t.nb = (it->st.r + 31) >> 5;
     t.uses_basis = it->st.r > 0 && it->st.n_cov > 0;
     t.has_coeff = t.uses_basis && t.t0 < it->st.n_cov;
   }
@@ -158,34 +161,64 @@ struct Ctrl {
 };
 
 // basis[r][d] of one slab -> K-major, 128B-swizzled bf16 operand: row = channel, [B1 | B2] along the
-// row (hi and lo parts of 32 basis vectors per rank block).  Tasks are strided over the callers.
-template <int RB>
+// row (hi and lo parts of 32 basis vectors per rank block).
+// A task is (rank block b, group of 8 basis vectors k8, group of 4 channels): 8 vector loads of 4
+// channels each, then per channel one 16-byte chunk of hi parts and one of lo parts.  Tasks are
+// strided over the callers; consecutive callers take the 4 k8 groups of 8 channel groups, which keeps
+// both the global loads (128-byte segments) and the swizzled stores (all 8 chunk columns) spread out.
+// kFly tasks are in flight per caller so that one warp alone stages a slab in a few load latencies.
+__device__ __forceinline__ float4 load_basis4(const void* basis, int bf16, int64_t off) {
+  if (bf16) {
+    const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(basis) + off);
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xffff0000u));
+  }
+  return *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(basis) + off);
+}
+
+template <int RB, int kFly>
 __device__ __forceinline__ void stage_basis(const Tile& t, uint8_t* slot_ptr, int first, int stride) {
   const DevItem& it = *t.it;
   const int r = it.st.r;
+  const int bf16 = it.st.basis_bf16;
   const void* basis = t.is_v ? it.st.basis_v : it.st.basis_k;
-  for (int task = first; task < RB * 512; task += stride) {
-    const int b = task >> 9, ch = task & 127, k8 = (task >> 7) & 3;
-    float v[8];
+  const int64_t slab_off = (int64_t)t.slab * r * 128;
+  const int n_task = (t.nb < RB ? t.nb : RB) * 128;
+  for (int task0 = first; task0 < n_task; task0 += kFly * stride) {
+    float4 v[kFly][8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int q = 32 * b + 8 * k8 + e;
-      float x = 0.f;
-      if (q < r) {
-        const int64_t off = ((int64_t)t.slab * r + q) * 128 + ch;
-        x = it.st.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
-                             : reinterpret_cast<const float*>(basis)[off];
+    for (int f = 0; f < kFly; ++f) {
+      const int task = task0 + f * stride;
+      // task = ((b * 4 + chg_hi) * 4 + k8) * 8 + chg_lo
+      const int k8 = (task >> 3) & 3, chg = ((task >> 5) & 3) * 8 + (task & 7), b = task >> 7;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int q = 32 * b + 8 * k8 + e;
+        v[f][e] = (task < n_task && q < r) ? load_basis4(basis, bf16, slab_off + (int64_t)q * 128 + 4 * chg)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
       }
-      v[e] = x;
     }
-    uint4 hi, lo;
-    split2(v[0], v[1], hi.x, lo.x);
-    split2(v[2], v[3], hi.y, lo.y);
-    split2(v[4], v[5], hi.z, lo.z);
-    split2(v[6], v[7], hi.w, lo.w);
-    uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
-    *reinterpret_cast<uint4*>(row + ((k8 ^ (ch & 7)) << 4)) = hi;
-    *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
+#pragma unroll
+    for (int f = 0; f < kFly; ++f) {
+      const int task = task0 + f * stride;
+      if (task >= n_task) break;
+      const int k8 = (task >> 3) & 3, chg = ((task >> 5) & 3) * 8 + (task & 7), b = task >> 7;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int ch = 4 * chg + j;
+        float x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = j == 0 ? v[f][e].x : j == 1 ? v[f][e].y : j == 2 ? v[f][e].z : v[f][e].w;
+        uint4 hi, lo;
+        split2(x[0], x[1], hi.x, lo.x);
+        split2(x[2], x[3], hi.y, lo.y);
+        split2(x[4], x[5], hi.z, lo.z);
+        split2(x[6], x[7], hi.w, lo.w);
+        uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
+        *reinterpret_cast<uint4*>(row + ((k8 ^ (ch & 7)) << 4)) = hi;
+        *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
+      }
+    }
   }
 }
 
@@ -214,8 +247,8 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int64_t n = p.total_tiles;
-  const int64_t tile_begin = n * blockIdx.x / gridDim.x;
-  const int64_t tile_end = n * (blockIdx.x + 1) / gridDim.x;
+  const int64_t tile_begin = p.cta_bounds ? p.cta_bounds[blockIdx.x] : n * blockIdx.x / gridDim.x;
+  const int64_t tile_end = p.cta_bounds ? p.cta_bounds[blockIdx.x + 1] : n * (blockIdx.x + 1) / gridDim.x;
 
   if (tid == 0) {
     for (int s = 0; s < NSTAGE; ++s) {
@@ -279,12 +312,12 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         ok = mbar_wait(smem_u32(&ctrl->cempty[c]), ((i / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
         if (ok) {
           const uint32_t cbar = smem_u32(&ctrl->cfull[c]);
-          mbar_expect_tx(cbar, t.has_coeff ? (uint32_t)kCoeffSlotBytes : 0u);
+          mbar_expect_tx(cbar, t.has_coeff ? (uint32_t)((t.nb < RB ? t.nb : RB) * kCoeffBlkBytes) : 0u);
           if (t.has_coeff) {
             const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
 #pragma unroll
             for (int b = 0; b < RB; ++b)
-              tma_load_3d(coeffs + c * kCoeffSlotBytes + b * kCoeffBlkBytes, cmap, cbar, 32 * b, t.t0, t.slab);
+              if (b < t.nb) tma_load_3d(coeffs + c * kCoeffSlotBytes + b * kCoeffBlkBytes, cmap, cbar, 32 * b, t.t0, t.slab);
           }
           ++c_issued;
           ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
@@ -355,6 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           uint32_t acc = 0;
 #pragma unroll
           for (int b = 0; b < RB; ++b) {
+            if (b >= t.nb) break;
             const uint64_t ad = umma_desc_sw128(a0 + b * kCoeffBlkBytes);
             const uint64_t bd = umma_desc_sw128(b0 + b * kBasisBlkBytes);
             // byte offsets inside the 128-byte row: c1 | c2 for A, B1 | B2 for B; 16 bf16 = 32 B per k-step
@@ -390,7 +424,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         ++slabs;
-        stage_basis<RB>(t, smem + kOperandOff + slot * kBasisSlotBytes, lane, 32);
+        stage_basis<RB, 2>(t, smem + kOperandOff + slot * kBasisSlotBytes, lane, 32);
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
@@ -500,6 +534,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         uint8_t* c_ptr = smem + NSTAGE * kStageBytes + c * kCoeffSlotBytes;
 #pragma unroll
         for (int b = 0; b < RB; ++b) {
+          if (b >= t.nb) break;                       // uniform over the CTA
           uint8_t* row = c_ptr + b * kCoeffBlkBytes + crow * 128;
           // this thread's 8 coefficients: fp32 chunks 2*cpart, 2*cpart+1 of the row
           const float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
@@ -525,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         Tile t0;
         w.get(t0);
         if (t0.uses_basis) {
-          stage_basis<RB>(t0, smem + kOperandOff, tt, kTeamThreads);
+          stage_basis<RB, 1>(t0, smem + kOperandOff, tt, kTeamThreads);
           fence_proxy_async();
           mbar_arrive(smem_u32(&ctrl->basis_full[0]));
         }
@@ -557,7 +592,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           Tile tn;
           wn.get(tn);
           if (tn.uses_basis && tn.first) {
-            stage_basis<RB>(tn, smem + kOperandOff, tt, kTeamThreads);
+            stage_basis<RB, 1>(tn, smem + kOperandOff, tt, kTeamThreads);
             fence_proxy_async();
             mbar_arrive(smem_u32(&ctrl->basis_full[0]));
           }
@@ -673,6 +708,7 @@ static bool item_supported(const DevItem& it, int d) {
   if (d != 128) return false;
   if (it.st.r <= 0 || it.st.n_cov <= 0) return false;       // empty state: a copy / rotate, CUDA-core kernel
   if (it.st.r > 64 || (it.st.r & 3)) return false;
+  if ((reinterpret_cast<uintptr_t>(it.st.basis_k) | reinterpret_cast<uintptr_t>(it.st.basis_v)) & 15) return false;   // vector loads
   for (const DevCache* c : {&it.src, &it.dst}) {
     if (c->page_table) {
       const int page = c->page_mask + 1;
@@ -707,10 +743,12 @@ static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s) {
-  const int sms = sm_count();
-  if (sms <= 0) return KVC_E_CUDA;
-  const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s, int grid = 0) {
+  if (grid <= 0) {
+    const int sms = sm_count();
+    if (sms <= 0) return KVC_E_CUDA;
+    grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+  }
   cudaError_t e = (max_r <= 32) ? launch_t<1, 5, 2, 2>(L, grid, s) : launch_t<2, 4, 2, 1>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
@@ -737,7 +775,12 @@ int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, c
   return tc::launch(L, item.st.r, s);
 }
 
-size_t tc_batch_extra_bytes(int n_items) { return 256 + (size_t)n_items * sizeof(tc::ItemMaps); }
+namespace tc {
+constexpr int kMaxGrid = 1024;   // CTA boundaries of a ragged launch are tabulated up to this grid size
+}
+size_t tc_batch_extra_bytes(int n_items) {
+  return 256 + (size_t)n_items * sizeof(tc::ItemMaps) + 8 * (size_t)(tc::kMaxGrid + 1);
+}
 
 int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int d, int pairing, uint32_t* status, void* workspace,
                    void* staging, size_t bytes, cudaStream_t s) {
@@ -761,7 +804,36 @@ int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int d, int pairin
   }
   prefix[n_items] = total;
   if (total == 0) return KVC_OK;
-  const size_t copy = maps_off + (size_t)n_items * sizeof(tc::ItemMaps);
+  // CTA boundaries: equal BYTES per CTA, not equal tile counts - a tile of a rank-64 state moves a
+  // third more than one of a rank-16 state (per token 4 d bytes of cache in and out, 4 r of coefficients)
+  const size_t bounds_off = maps_off + (size_t)n_items * sizeof(tc::ItemMaps);
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(total < sms ? total : (sms < tc::kMaxGrid ? sms : tc::kMaxGrid));
+  if (bounds_off + 8 * (size_t)(grid + 1) > bytes) return KVC_E_WORKSPACE;
+  int64_t* bounds = reinterpret_cast<int64_t*>(reinterpret_cast<char*>(staging) + bounds_off);
+  {
+    double w_total = 0;
+    for (int i = 0; i < n_items; ++i) w_total += (double)(prefix[i + 1] - prefix[i]) * (4 * d + 4 * tab[i].st.r);
+    int it = 0;
+    double w_before = 0;   // weight of items [0, it)
+    bounds[0] = 0;
+    for (int b = 1; b < grid; ++b) {
+      const double target = w_total * b / grid;
+      while (it < n_items) {
+        const double w_item = (double)(prefix[it + 1] - prefix[it]) * (4 * d + 4 * tab[it].st.r);
+        if (w_before + w_item > target || it == n_items - 1) break;
+        w_before += w_item;
+        ++it;
+      }
+      int64_t tile = prefix[it] + (int64_t)((target - w_before) / (4 * d + 4 * tab[it].st.r));
+      if (tile > prefix[it + 1]) tile = prefix[it + 1];
+      if (tile < bounds[b - 1]) tile = bounds[b - 1];
+      bounds[b] = tile;
+    }
+    bounds[grid] = total;
+  }
+  const size_t copy = bounds_off + 8 * (size_t)(grid + 1);
   if (cudaMemcpyAsync(workspace, staging, copy, cudaMemcpyHostToDevice, s) != cudaSuccess) return KVC_E_CUDA;
   tc::ApplyTcLaunch L;
   memset(&L, 0, sizeof(L));
@@ -770,9 +842,10 @@ int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int d, int pairin
   L.maps = reinterpret_cast<const tc::ItemMaps*>(reinterpret_cast<char*>(workspace) + maps_off);
   L.n_items = n_items;
   L.pairing = pairing;
+  L.cta_bounds = reinterpret_cast<const int64_t*>(reinterpret_cast<char*>(workspace) + bounds_off);
   L.total_tiles = total;
   L.status = status;
-  return tc::launch(L, max_r, s);
+  return tc::launch(L, max_r, s, grid);
 }
 
 }  // namespace kvc
