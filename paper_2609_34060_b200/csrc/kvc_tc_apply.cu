@@ -222,6 +222,46 @@ __device__ __forceinline__ void stage_basis(const Tile& t, uint8_t* slot_ptr, in
   }
 }
 
+// The same operand built from a RAW copy of the slab's basis in shared memory (rows of d values,
+// fp32 or bf16, as they sit in global memory), which a bulk copy brought in ahead of time.
+template <int RB>
+__device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_ptr, int r, int bf16, int first, int stride) {
+  const int nb = (r + 31) >> 5;
+  const int n_task = (nb < RB ? nb : RB) * 128;
+  for (int task = first; task < n_task; task += stride) {
+    const int k8 = (task >> 3) & 3, chg = ((task >> 5) & 3) * 8 + (task & 7), b = task >> 7;
+    float4 v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int q = 32 * b + 8 * k8 + e;
+      if (q >= r) {
+        v[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+      } else if (bf16) {
+        const uint2 u = *reinterpret_cast<const uint2*>(raw + q * 256 + chg * 8);
+        v[e] = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                           __uint_as_float(u.y & 0xffff0000u));
+      } else {
+        v[e] = *reinterpret_cast<const float4*>(raw + q * 512 + chg * 16);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int ch = 4 * chg + j;
+      float x[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) x[e] = j == 0 ? v[e].x : j == 1 ? v[e].y : j == 2 ? v[e].z : v[e].w;
+      uint4 hi, lo;
+      split2(x[0], x[1], hi.x, lo.x);
+      split2(x[2], x[3], hi.y, lo.y);
+      split2(x[4], x[5], hi.z, lo.z);
+      split2(x[6], x[7], hi.w, lo.w);
+      uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
+      *reinterpret_cast<uint4*>(row + ((k8 ^ (ch & 7)) << 4)) = hi;
+      *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
+    }
+  }
+}
+
 // ------------------------------------------------------------------ the kernel
 // Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 basis stager, 3 store warp, 4..19 the team.
 // Team warp e (0..15): TMEM lane quadrant e & 3 (rows 32q..32q+31), channel quarter e >> 2.
@@ -287,13 +327,18 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     // =============================================================== TMA producer (whole warp)
     TileWalker w;
     w.init(&p, tile_begin, tile_end);
-    uint32_t i = 0, c_issued = 0;
+    uint32_t i = 0, cpos = 0;                       // cpos: position in the coefficient ring
     for (; !w.done(); w.next(), ++i) {
       Tile t;
       w.get(t);
       const int s = i % NSTAGE;
       const uint32_t use = i / NSTAGE;
       const DevItem& it = *t.it;
+      // single operand slot: the slab's raw basis travels through the coefficient ring, one entry
+      // ahead of the slab's first coefficient tile, and the team turns it into the operand
+      uint32_t bpos = cpos;
+      const bool raw_basis = NB == 1 && t.first && t.uses_basis;
+      if (raw_basis) ++cpos;
       // paged source: one lane per page of the tile; the ids are fetched BEFORE waiting for the
       // stage, so that their global-memory latency hides behind the wait
       const bool paged = it.src.page_table != nullptr;
@@ -306,10 +351,22 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         if (lane < n_pages) id = it.src.page_table[first + lane];
       }
       // coefficient tile first: its slot turns over quickly
-      const int c = i % NSC;
+      const int c = cpos % NSC;
       int ok = 1;
       if (lane == 0) {
-        ok = mbar_wait(smem_u32(&ctrl->cempty[c]), ((i / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+        if (raw_basis) {
+          const int bc = bpos % NSC;
+          ok = mbar_wait(smem_u32(&ctrl->cempty[bc]), ((bpos / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+          if (ok) {
+            const uint32_t row_bytes = it.st.basis_bf16 ? 256u : 512u;
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(t.is_v ? it.st.basis_v : it.st.basis_k) +
+                                 (size_t)t.slab * it.st.r * row_bytes;
+            const uint32_t bbar = smem_u32(&ctrl->cfull[bc]);
+            mbar_expect_tx(bbar, it.st.r * row_bytes);
+            bulk_load_1d(coeffs + bc * kCoeffSlotBytes, src, it.st.r * row_bytes, bbar);
+          }
+        }
+        if (ok) ok = mbar_wait(smem_u32(&ctrl->cempty[c]), ((cpos / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
         if (ok) {
           const uint32_t cbar = smem_u32(&ctrl->cfull[c]);
           mbar_expect_tx(cbar, t.has_coeff ? (uint32_t)((t.nb < RB ? t.nb : RB) * kCoeffBlkBytes) : 0u);
@@ -319,12 +376,12 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             for (int b = 0; b < RB; ++b)
               if (b < t.nb) tma_load_3d(coeffs + c * kCoeffSlotBytes + b * kCoeffBlkBytes, cmap, cbar, 32 * b, t.t0, t.slab);
           }
-          ++c_issued;
           ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
+      if (!ok) break;        // an expired wait: whatever was issued before it has landed or lands in the drain below
+      ++cpos;
       const uint32_t st_base = stages + s * kStageBytes;
       const uint32_t bar = smem_u32(&ctrl->full[s]);
       const CUtensorMap* smap = t.is_v ? &t.mp->src_v : &t.mp->src_k;
@@ -352,7 +409,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const uint32_t issued = i;
       for (uint32_t k = (issued > NSTAGE ? issued - NSTAGE : 0); k < issued; ++k)
         mbar_wait_drain(smem_u32(&ctrl->full[k % NSTAGE]), (k / NSTAGE) & 1u);
-      for (uint32_t k = (c_issued > NSC ? c_issued - NSC : 0); k < c_issued; ++k)
+      for (uint32_t k = (cpos > NSC ? cpos - NSC : 0); k < cpos; ++k)
         mbar_wait_drain(smem_u32(&ctrl->cfull[k % NSC]), (k / NSC) & 1u);
     }
   } else if (warp == 1) {
@@ -360,24 +417,34 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     if (lane == 0) {
       TileWalker w;
       w.init(&p, tile_begin, tile_end);
-      uint32_t i = 0, slabs = 0;
+      uint32_t i = 0, slabs = 0, cpos = 0;
       bool in_slab = false;
       int slot = 0;
       for (; !w.done(); w.next(), ++i) {
         Tile t;
         w.get(t);
-        const int c = i % NSC, g = i & 1;
-        const uint32_t use = i / NSC, acc_use = i >> 1;
+        const int g = i & 1;
+        const uint32_t acc_use = i >> 1;
         if (t.first) {
           if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));   // all MMAs of the old slab done => slot free
           in_slab = false;
           if (t.uses_basis) {
+            if constexpr (NB == 1) {
+              // ring entry of the slab's raw basis: once the team has consumed it, hand the slot back
+              const int bc = cpos % NSC;
+              if (!mbar_wait(smem_u32(&ctrl->conv[bc]), (cpos / NSC) & 1u, abort_flag)) break;
+              umma_commit(smem_u32(&ctrl->cempty[bc]));
+              ++cpos;
+            }
             slot = slabs % NB;
             if (!mbar_wait(smem_u32(&ctrl->basis_full[slot]), (slabs / NB) & 1u, abort_flag)) break;
             ++slabs;
             in_slab = true;
           }
         }
+        const int c = cpos % NSC;
+        const uint32_t use = cpos / NSC;
+        ++cpos;
         if (!mbar_wait(smem_u32(&ctrl->conv[c]), use & 1u, abort_flag)) break;
         if (!mbar_wait(smem_u32(&ctrl->acc_empty[g]), (acc_use & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
@@ -521,7 +588,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     uint32_t i = 0;
     bool alive = true;
 
-    // conversion of tile index `ci` held by walker `cw`
+    // conversion of the coefficient tile held by walker `cw`, at ring position `ci`
     auto convert = [&](TileWalker& cw, uint32_t ci) {
       Tile t;
       cw.get(t);
@@ -555,23 +622,43 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     };
 
     const int tt = tid - 128;                       // 0 .. 511
-    if constexpr (NB == 1) {                         // single operand slot: the team stages it
-      if (!w.done()) {
+    uint32_t cpos = 0;                              // ring position of the next entry the team consumes
+    // single operand slot: the raw basis of a slab sits in ring entry `pos`; build the operand from it
+    auto take_basis = [&](const Tile& tb, uint32_t pos) {
+      const int bc = pos % NSC;
+      bool ok = mbar_wait(smem_u32(&ctrl->cfull[bc]), (pos / NSC) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return false;
+      convert_basis<RB>(smem + NSTAGE * kStageBytes + bc * kCoeffSlotBytes, smem + kOperandOff, tb.it->st.r,
+                        tb.it->st.basis_bf16, tt, kTeamThreads);
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&ctrl->basis_full[0]));
+      mbar_arrive(smem_u32(&ctrl->conv[bc]));       // the issuer hands the ring slot back
+      return true;
+    };
+    uint32_t pending_basis = 0;                     // ring position of a raw basis not yet consumed
+    bool have_pending = false;
+    if (!w.done()) {
+      if constexpr (NB == 1) {
         Tile t0;
         w.get(t0);
-        if (t0.uses_basis) {
-          stage_basis<RB, 1>(t0, smem + kOperandOff, tt, kTeamThreads);
-          fence_proxy_async();
-          mbar_arrive(smem_u32(&ctrl->basis_full[0]));
-        }
+        if (t0.uses_basis) alive = take_basis(t0, cpos++);
       }
+      if (alive) alive = convert(wn, cpos++);
     }
-    if (!w.done()) alive = convert(wn, 0);
     for (; alive && !w.done(); w.next(), ++i) {
       // ---- 1. get the next tile's coefficients converted and its MMA going
       wn.next();
       if (!wn.done()) {
-        if (!convert(wn, i + 1)) break;
+        if constexpr (NB == 1) {
+          Tile tn;
+          wn.get(tn);
+          have_pending = tn.uses_basis && tn.first;
+          if (have_pending) pending_basis = cpos++;
+        }
+        if (!convert(wn, cpos++)) break;
+      } else {
+        have_pending = false;
       }
       Tile t;
       w.get(t);
@@ -588,14 +675,10 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       if constexpr (NB == 1) {
         // The MMAs of tile i are complete.  If tile i + 1 opens a new slab, tile i was the last
         // reader of the operand slot: restage it now (512 threads: about a microsecond).
-        if (!wn.done()) {
+        if (have_pending) {
           Tile tn;
           wn.get(tn);
-          if (tn.uses_basis && tn.first) {
-            stage_basis<RB, 1>(tn, smem + kOperandOff, tt, kTeamThreads);
-            fence_proxy_async();
-            mbar_arrive(smem_u32(&ctrl->basis_full[0]));
-          }
+          if (!take_basis(tn, pending_basis)) break;
         }
       }
 
