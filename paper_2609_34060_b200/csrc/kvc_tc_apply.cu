@@ -2,16 +2,22 @@
 // contraction coeff . basis on tcgen05 tensor cores with fp32 accumulators in TMEM, RoPE
 // re-alignment and the add in registers, results written back through TMA.
 //
-// One persistent CTA per SM walks a contiguous range of tiles; a tile is 128 tokens of one
-// (layer, head, K|V) slab.  Warp roles:
-//   warp 0      TMA producer (one lane): base tile (bf16 128 x 128) + fp32 coefficient tile
-//   warp 1      MMA issuer (one lane) and TMEM owner
-//   warp 2      basis stager (two operand slots, r <= 32); with one slot (r = 64) the team stages
-//   warp 3      store warp: TMA stores of finished tiles, releases the stage
-//   warps 4-7, 8-11   two epilogue groups; a group owns every other tile of the CTA:
-//               convert its coefficient rows to bf16 hi/lo in place, wait for the MMA, read the
-//               accumulator row from TMEM, rotate/add/round, write the row back in place, and
-//               one lane issues the TMA store and releases the stage.
+// One persistent CTA per SM walks a contiguous range of tiles (ranges of equal bytes); a tile is
+// 128 tokens of one (layer, head, K|V) slab.  Shared memory holds two rings and one operand slot:
+//   base ring         bf16 128 x 128 cache tiles, alive from the load until the TMA store has read them
+//   coefficient ring  fp32 coefficient tiles, alive until the tile's MMAs have completed; the raw
+//                     basis of a slab travels through the same ring, one entry ahead of the slab's
+//                     first coefficient tile
+//   operand slot      the slab's basis as a K-major swizzled bf16 hi/lo operand
+// Warp roles:
+//   warp 0      TMA producer: base tile (one lane, or one lane per page of a paged cache),
+//               coefficient tile, raw basis at the start of a slab
+//   warp 1      MMA issuer (one lane) and TMEM owner (two accumulators of 128 columns)
+//   warp 2      spare
+//   warp 3      store warp: TMA stores of finished tiles, releases the base slot
+//   warps 4-19  the team: converts the next tile's coefficient rows to bf16 hi/lo in place, rebuilds
+//               the operand slot when a slab starts, and for the current tile reads the accumulator
+//               row from TMEM, rotates, adds, rounds and writes the row back in place.
 // Precision: c = c1 + c2 and B = B1 + B2 with bf16 terms; c.B ~= c1.B1 + c2.B1 + c1.B2
 // (relative error about 2^-16 per product), accumulated in fp32.
 // Every wait is bounded; on expiry the CTA records KVC_FLAG_WAIT_EXPIRED, drains and returns.
@@ -149,81 +155,25 @@ struct TileWalker {
 };
 
 // Shared-memory control block (after the tiles)
-template <int NSTAGE, int NSC, int NB>
+template <int NSTAGE, int NSC>
 struct Ctrl {
   uint64_t full[NSTAGE], ready[NSTAGE], empty[NSTAGE];      // base-tile ring
   uint64_t cfull[NSC], conv[NSC], cempty[NSC];              // coefficient ring
   uint64_t mma_done[2], acc_empty[2];
-  uint64_t basis_full[NB], basis_empty[NB];
+  uint64_t basis_full;                                      // the slab's operand is staged
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
 };
 
 // basis[r][d] of one slab -> K-major, 128B-swizzled bf16 operand: row = channel, [B1 | B2] along the
-// row (hi and lo parts of 32 basis vectors per rank block).
+// row (hi and lo parts of 32 basis vectors per rank block).  The operand is built from a RAW copy of
+// the slab's basis in shared memory (rows of d values, fp32 or bf16, as they sit in global memory),
+// which a bulk copy brought in ahead of time.
 // A task is (rank block b, group of 8 basis vectors k8, group of 4 channels): 8 vector loads of 4
-// channels each, then per channel one 16-byte chunk of hi parts and one of lo parts.  Tasks are
-// strided over the callers; consecutive callers take the 4 k8 groups of 8 channel groups, which keeps
-// both the global loads (128-byte segments) and the swizzled stores (all 8 chunk columns) spread out.
-// kFly tasks are in flight per caller so that one warp alone stages a slab in a few load latencies.
-__device__ __forceinline__ float4 load_basis4(const void* basis, int bf16, int64_t off) {
-  if (bf16) {
-    const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(basis) + off);
-    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-                       __uint_as_float(u.y & 0xffff0000u));
-  }
-  return *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(basis) + off);
-}
-
-template <int RB, int kFly>
-__device__ __forceinline__ void stage_basis(const Tile& t, uint8_t* slot_ptr, int first, int stride) {
-  const DevItem& it = *t.it;
-  const int r = it.st.r;
-  const int bf16 = it.st.basis_bf16;
-  const void* basis = t.is_v ? it.st.basis_v : it.st.basis_k;
-  const int64_t slab_off = (int64_t)t.slab * r * 128;
-  const int n_task = (t.nb < RB ? t.nb : RB) * 128;
-  for (int task0 = first; task0 < n_task; task0 += kFly * stride) {
-    float4 v[kFly][8];
-#pragma unroll
-    for (int f = 0; f < kFly; ++f) {
-      const int task = task0 + f * stride;
-      // task = ((b * 4 + chg_hi) * 4 + k8) * 8 + chg_lo
-      const int k8 = (task >> 3) & 3, chg = ((task >> 5) & 3) * 8 + (task & 7), b = task >> 7;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int q = 32 * b + 8 * k8 + e;
-        v[f][e] = (task < n_task && q < r) ? load_basis4(basis, bf16, slab_off + (int64_t)q * 128 + 4 * chg)
-                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-    }
-#pragma unroll
-    for (int f = 0; f < kFly; ++f) {
-      const int task = task0 + f * stride;
-      if (task >= n_task) break;
-      const int k8 = (task >> 3) & 3, chg = ((task >> 5) & 3) * 8 + (task & 7), b = task >> 7;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int ch = 4 * chg + j;
-        float x[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] = j == 0 ? v[f][e].x : j == 1 ? v[f][e].y : j == 2 ? v[f][e].z : v[f][e].w;
-        uint4 hi, lo;
-        split2(x[0], x[1], hi.x, lo.x);
-        split2(x[2], x[3], hi.y, lo.y);
-        split2(x[4], x[5], hi.z, lo.z);
-        split2(x[6], x[7], hi.w, lo.w);
-        uint8_t* row = slot_ptr + b * kBasisBlkBytes + ch * 128;
-        *reinterpret_cast<uint4*>(row + ((k8 ^ (ch & 7)) << 4)) = hi;
-        *reinterpret_cast<uint4*>(row + (((4 + k8) ^ (ch & 7)) << 4)) = lo;
-      }
-    }
-  }
-}
-
-// The same operand built from a RAW copy of the slab's basis in shared memory (rows of d values,
-// fp32 or bf16, as they sit in global memory), which a bulk copy brought in ahead of time.
+// channels each, then per channel one 16-byte chunk of hi parts and one of lo parts.  Consecutive
+// callers take the 4 k8 groups of 8 channel groups, which spreads both the loads and the swizzled
+// stores over all banks.
 template <int RB>
 __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_ptr, int r, int bf16, int first, int stride) {
   const int nb = (r + 31) >> 5;
@@ -263,13 +213,13 @@ __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_
 }
 
 // ------------------------------------------------------------------ the kernel
-// Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 basis stager, 3 store warp, 4..19 the team.
+// Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 spare, 3 store warp, 4..19 the team.
 // Team warp e (0..15): TMEM lane quadrant e & 3 (rows 32q..32q+31), channel quarter e >> 2.
 //
 // Two rings of shared-memory slots: NSTAGE base tiles (alive from the load until the TMA store has
 // read them) and NSC coefficient tiles (alive only until the tile's MMAs have completed), so that
 // the short-lived operand does not hold a long-lived slot.
-template <int RB, int NSTAGE, int NSC, int NB>
+template <int RB, int NSTAGE, int NSC>
 __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
   constexpr int kStageBytes = kBaseBytes;
   constexpr int kCoeffSlotBytes = RB * kCoeffBlkBytes;
@@ -282,7 +232,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
   const uint32_t stages = base;
   const uint32_t coeffs = base + NSTAGE * kStageBytes;
   const uint32_t bases = base + kOperandOff;
-  Ctrl<NSTAGE, NSC, NB>* ctrl = reinterpret_cast<Ctrl<NSTAGE, NSC, NB>*>(smem + kOperandOff + NB * kBasisSlotBytes);
+  Ctrl<NSTAGE, NSC>* ctrl = reinterpret_cast<Ctrl<NSTAGE, NSC>*>(smem + kOperandOff + kBasisSlotBytes);
   volatile int* abort_flag = &ctrl->abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -305,10 +255,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
       mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
     }
-    for (int b = 0; b < NB; ++b) {
-      mbar_init(smem_u32(&ctrl->basis_full[b]), NB == 1 ? kTeamThreads : 1);   // who stages: team or stager warp
-      mbar_init(smem_u32(&ctrl->basis_empty[b]), 1);
-    }
+    mbar_init(smem_u32(&ctrl->basis_full), kTeamThreads);
     mbar_init(smem_u32(&ctrl->drain), 1);
     ctrl->abort_flag = 0;
     fence_barrier_init();
@@ -337,7 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       // single operand slot: the slab's raw basis travels through the coefficient ring, one entry
       // ahead of the slab's first coefficient tile, and the team turns it into the operand
       uint32_t bpos = cpos;
-      const bool raw_basis = NB == 1 && t.first && t.uses_basis;
+      const bool raw_basis = t.first && t.uses_basis;
       if (raw_basis) ++cpos;
       // paged source: one lane per page of the tile; the ids are fetched BEFORE waiting for the
       // stage, so that their global-memory latency hides behind the wait
@@ -418,29 +365,19 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       TileWalker w;
       w.init(&p, tile_begin, tile_end);
       uint32_t i = 0, slabs = 0, cpos = 0;
-      bool in_slab = false;
-      int slot = 0;
       for (; !w.done(); w.next(), ++i) {
         Tile t;
         w.get(t);
         const int g = i & 1;
         const uint32_t acc_use = i >> 1;
-        if (t.first) {
-          if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));   // all MMAs of the old slab done => slot free
-          in_slab = false;
-          if (t.uses_basis) {
-            if constexpr (NB == 1) {
-              // ring entry of the slab's raw basis: once the team has consumed it, hand the slot back
-              const int bc = cpos % NSC;
-              if (!mbar_wait(smem_u32(&ctrl->conv[bc]), (cpos / NSC) & 1u, abort_flag)) break;
-              umma_commit(smem_u32(&ctrl->cempty[bc]));
-              ++cpos;
-            }
-            slot = slabs % NB;
-            if (!mbar_wait(smem_u32(&ctrl->basis_full[slot]), (slabs / NB) & 1u, abort_flag)) break;
-            ++slabs;
-            in_slab = true;
-          }
+        if (t.first && t.uses_basis) {
+          // ring entry of the slab's raw basis: once the team has consumed it, hand the slot back
+          const int bc = cpos % NSC;
+          if (!mbar_wait(smem_u32(&ctrl->conv[bc]), (cpos / NSC) & 1u, abort_flag)) break;
+          umma_commit(smem_u32(&ctrl->cempty[bc]));
+          ++cpos;
+          if (!mbar_wait(smem_u32(&ctrl->basis_full), slabs & 1u, abort_flag)) break;
+          ++slabs;
         }
         const int c = cpos % NSC;
         const uint32_t use = cpos / NSC;
@@ -451,7 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         if (t.has_coeff) {
           const uint32_t d_tmem = tmem_base + g * 128;
           const uint32_t a0 = coeffs + c * kCoeffSlotBytes;
-          const uint32_t b0 = bases + slot * kBasisSlotBytes;
+          const uint32_t b0 = bases;
           uint32_t acc = 0;
 #pragma unroll
           for (int b = 0; b < RB; ++b) {
@@ -471,32 +408,11 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         umma_commit(smem_u32(&ctrl->mma_done[g]));
         umma_commit(smem_u32(&ctrl->cempty[c]));      // the coefficient slot may be refilled
       }
-      if (NB > 1 && in_slab) umma_commit(smem_u32(&ctrl->basis_empty[slot]));
       umma_commit(smem_u32(&ctrl->drain));
       mbar_wait_drain(smem_u32(&ctrl->drain), 0);
     }
   } else if (warp == 2) {
-    // =============================================================== basis stager (two-slot variant only)
-    if constexpr (NB > 1) {
-      TileWalker w;
-      w.init(&p, tile_begin, tile_end);
-      uint32_t slabs = 0;
-      for (; !w.done(); w.next()) {
-        Tile t;
-        w.get(t);
-        if (!t.first || !t.uses_basis) continue;
-        const int slot = slabs % NB;
-        int ok = 1;
-        if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->basis_empty[slot]), ((slabs / NB) & 1u) ^ 1u, abort_flag) ? 1 : 0;
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;
-        ++slabs;
-        stage_basis<RB, 2>(t, smem + kOperandOff + slot * kBasisSlotBytes, lane, 32);
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctrl->basis_full[slot]));
-      }
-    }
+    // spare warp: keeps the team's warps aligned with the TMEM lane quadrants (warp id & 3)
   } else if (warp == 3) {
     // =============================================================== store warp
     TileWalker w;
@@ -632,30 +548,26 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       convert_basis<RB>(smem + NSTAGE * kStageBytes + bc * kCoeffSlotBytes, smem + kOperandOff, tb.it->st.r,
                         tb.it->st.basis_bf16, tt, kTeamThreads);
       fence_proxy_async();
-      mbar_arrive(smem_u32(&ctrl->basis_full[0]));
+      mbar_arrive(smem_u32(&ctrl->basis_full));
       mbar_arrive(smem_u32(&ctrl->conv[bc]));       // the issuer hands the ring slot back
       return true;
     };
     uint32_t pending_basis = 0;                     // ring position of a raw basis not yet consumed
     bool have_pending = false;
     if (!w.done()) {
-      if constexpr (NB == 1) {
-        Tile t0;
-        w.get(t0);
-        if (t0.uses_basis) alive = take_basis(t0, cpos++);
-      }
+      Tile t0;
+      w.get(t0);
+      if (t0.uses_basis) alive = take_basis(t0, cpos++);
       if (alive) alive = convert(wn, cpos++);
     }
     for (; alive && !w.done(); w.next(), ++i) {
       // ---- 1. get the next tile's coefficients converted and its MMA going
       wn.next();
       if (!wn.done()) {
-        if constexpr (NB == 1) {
-          Tile tn;
-          wn.get(tn);
-          have_pending = tn.uses_basis && tn.first;
-          if (have_pending) pending_basis = cpos++;
-        }
+        Tile tn;
+        wn.get(tn);
+        have_pending = tn.uses_basis && tn.first;
+        if (have_pending) pending_basis = cpos++;
         if (!convert(wn, cpos++)) break;
       } else {
         have_pending = false;
@@ -672,14 +584,12 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      if constexpr (NB == 1) {
-        // The MMAs of tile i are complete.  If tile i + 1 opens a new slab, tile i was the last
-        // reader of the operand slot: restage it now (512 threads: about a microsecond).
-        if (have_pending) {
-          Tile tn;
-          wn.get(tn);
-          if (!take_basis(tn, pending_basis)) break;
-        }
+      // The MMAs of tile i are complete.  If tile i + 1 opens a new slab, tile i was the last
+      // reader of the operand slot: rebuild it now from the raw basis that waits in the ring.
+      if (have_pending) {
+        Tile tn;
+        wn.get(tn);
+        if (!take_basis(tn, pending_basis)) break;
       }
 
       // ---- 3. rotate, add, round: row m, this warp's channel quarter, in place
@@ -810,19 +720,18 @@ static bool build_maps(const DevItem& it, ItemMaps* mp) {
   return ok;
 }
 
-template <int RB, int NSTAGE, int NSC, int NB>
+template <int RB, int NSTAGE, int NSC>
 static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
-  const size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)NB * RB * kBasisBlkBytes +
-                      sizeof(Ctrl<NSTAGE, NSC, NB>);
-  static_assert(1024 + NSTAGE * kBaseBytes + NSC * RB * kCoeffBlkBytes + NB * RB * kBasisBlkBytes + sizeof(Ctrl<NSTAGE, NSC, NB>) <= 232448,
-                "exceeds the shared memory of one CTA");
+  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
+                          sizeof(Ctrl<NSTAGE, NSC>);
+  static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
   static bool set = false;
   if (!set) {
-    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     set = true;
   }
-  apply_tc_kernel<RB, NSTAGE, NSC, NB><<<grid, kThreads, smem, s>>>(L);
+  apply_tc_kernel<RB, NSTAGE, NSC><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError();
 }
 
@@ -832,7 +741,7 @@ static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s, int grid = 
     if (sms <= 0) return KVC_E_CUDA;
     grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
   }
-  cudaError_t e = (max_r <= 32) ? launch_t<1, 5, 2, 2>(L, grid, s) : launch_t<2, 4, 2, 1>(L, grid, s);
+  cudaError_t e = (max_r <= 32) ? launch_t<1, 5, 3>(L, grid, s) : launch_t<2, 4, 2>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
