@@ -213,12 +213,14 @@ def build_serving(n_requests: int, dev, kvc, seed=0, L=32, H=8, d=128, page=16, 
         items = [kvc.Item(caches[i][(h - 1) % 2], caches[i][h % 2], states[i], r.prefix[h] - r.prefix[h - 1])
                  for i, r in enumerate(reqs) if r.n_agents > h]
         rounds.append(items)
+    # a round runs as one kernel per rank class present (r <= 32, r > 32)
+    kernels = sum(len({r.r <= 32 for r in reqs if r.n_agents > h}) for h in range(1, max(r.n_agents for r in reqs)))
     nb = kvc.kvc_batch_workspace_bytes(n_requests)
     ws = [torch.empty(nb, dtype=torch.uint8, device=dev) for _ in rounds]
     staging = [torch.empty(nb, dtype=torch.uint8).pin_memory() for _ in rounds]
     app = sum(kvc.kvc_apply_bytes(it.src, it.st) for items in rounds for it in items)
     return {"kind": "serving", "rope": rope, "rounds": rounds, "ws": ws, "staging": staging, "reqs": reqs, "apply_bytes": app,
-            "only": "apply", "launches": len(rounds), "tokens": sum(r.T for r in reqs)}
+            "only": "apply", "launches": len(rounds), "kernels": kernels, "tokens": sum(r.T for r in reqs)}
 
 
 def run_step(W, kvc, ev=None):
@@ -481,7 +483,7 @@ def main():
            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic", "config": config,
            "clocks": clocks, "e2e": e2e,
-           "gpu_launches": args.steps * (hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
+           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
            "roofline": roofline,
            "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
                          "us_per_agent_layer": hop_ms * 1e3 / cfg.L,
