@@ -379,13 +379,15 @@ __device__ __forceinline__ float warp_sum(float x) {
   return x;
 }
 
-__global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int n, int zs) {
+template <int N>
+__global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs) {
   extern __shared__ __align__(16) float smem[];
-  const int np = n + 4;               // row pitch of A = 4 (mod 32): four threads per row, eight rows per warp, no bank conflicts
-  float* A = smem;                    // [n][np]  symmetric; row k right of the diagonal later holds reflector k
-  float* Zt = A + n * np;              // [n][zs]  Zt[i][j] = component i of eigenvector j  (zs = r_eff + 1, odd)
-  float* vv = Zt + n * zs;            // [n] current reflector
-  float* pp = vv + n;                 // [n] beta * A v
+  constexpr int n = N;
+  constexpr int np = N + 4;           // row pitch of A = 4 (mod 32)
+  float* A = smem;                    // [n][np]  staging of the input; then row k right of the diagonal holds reflector k
+  float* Zt = A + n * np;             // [n][zs]  Zt[i][j] = component i of eigenvector j  (zs = r_eff + 1, odd)
+  float* vv = Zt + n * zs;            // [n] scratch
+  float* pp = vv + n;                 // [n] beta * A v, indexed by row
   float* dd = pp + n;                 // [n] diagonal of T
   float* ee = dd + n;                 // [n] off-diagonal of T (ee[i] couples i and i+1)
   float* e2 = ee + n;                 // [n] squares of ee
@@ -402,119 +404,163 @@ __global__ void __launch_bounds__(kEigThreads) eig_tridiag_kernel(const __grid_c
   float* G = p.gram + (int64_t)sk * n * n;
   const int64_t part_stride = (int64_t)p.L * p.H * 2 * n * n;
 
-  // ---- load: fixed-order sum of the partial Grams (coalesced), then symmetrise in place
-  for (int i = tid; i < n * n; i += kEigThreads) {
-    const int rr = i / n, cc = i - rr * n;
-    float a = 0.f;
-    for (int pt = 0; pt < p.n_parts; ++pt) a += G[pt * part_stride + i];
-    A[rr * np + cc] = a;
-  }
-  __syncthreads();
-  for (int i = tid; i < n * n; i += kEigThreads) {
-    const int rr = i / n, cc = i - rr * n;
-    if (cc > rr) {                                 // one thread per unordered pair
-      const float m2 = 0.5f * (A[rr * np + cc] + A[cc * np + rr]);
-      A[rr * np + cc] = m2;
-      A[cc * np + rr] = m2;
-    }
-  }
-  __syncthreads();
-  for (int i = tid; i < n * n; i += kEigThreads) G[i] = A[(i / n) * np + (i % n)];
-
-  // ---- 1. Householder tridiagonalisation.  Four threads own one row of the trailing block
-  // (columns interleaved), in the matrix-vector product and in the rank-2 update.  Reflector k
-  // lives in row k right of the diagonal (v0 written over x0), so it is never copied; the
-  // threads that own the next pivot row compute its norm and (alpha, beta, v0) at the end of
-  // the update, which leaves two block barriers per step.
+  // ---- 1. Householder tridiagonalisation with the matrix in REGISTERS.  TPR threads own one row,
+  // in chunks of four columns dealt out round-robin (chunk c of thread tq: columns 4 (c TPR + tq) ..
+  // + 3), so the work of a row stays spread over its threads as the trailing block shrinks.
+  // Reflector k is written to row k of the shared-memory copy (zeros left of the sub-diagonal), where
+  // the back-transformation finds it later.  Two block barriers per step.
+  constexpr int TPR = kEigThreads / N;          // 4 (N = 128) or 8 (N = 64)
+  constexpr int NCH = N / (4 * TPR);            // chunks per thread: 8 or 2
+  static_assert(TPR * N == kEigThreads && NCH * 4 * TPR == N && TPR <= 32, "thread layout");
+  const int trow = tid / TPR, tq = tid % TPR;
+  float a[NCH][4];
   {
-    const int trow = tid >> 2, tq = tid & 3;
-    // scalar set-up of step k from the row's squared norm s2 (x = A[k][k+1 ..]); one thread
-    auto setup = [&](int k, float s2) {
-      float* x = A + k * np + k + 1;
-      const float x0 = x[0];
+    // stage the fixed-order sum of the partial Grams (coalesced), then symmetrise into registers
+    for (int i = tid; i < n * n / 4; i += kEigThreads) {
+      const int rr = i / (n / 4), c4 = i % (n / 4);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int pt = 0; pt < p.n_parts; ++pt) {
+        const float4 g = *reinterpret_cast<const float4*>(G + pt * part_stride + (int64_t)rr * n + 4 * c4);
+        acc.x += g.x;
+        acc.y += g.y;
+        acc.z += g.z;
+        acc.w += g.w;
+      }
+      *reinterpret_cast<float4*>(A + rr * np + 4 * c4) = acc;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const int col0 = 4 * (c * TPR + tq);
+      const float4 own = *reinterpret_cast<const float4*>(A + trow * np + col0);
+      a[c][0] = 0.5f * (own.x + A[(col0 + 0) * np + trow]);
+      a[c][1] = 0.5f * (own.y + A[(col0 + 1) * np + trow]);
+      a[c][2] = 0.5f * (own.z + A[(col0 + 2) * np + trow]);
+      a[c][3] = 0.5f * (own.w + A[(col0 + 3) * np + trow]);
+      *reinterpret_cast<float4*>(G + (int64_t)trow * n + col0) = make_float4(a[c][0], a[c][1], a[c][2], a[c][3]);
+    }
+    if (tid < n) pp[tid] = 0.f;
+    __syncthreads();                              // everybody has read the staging copy
+  }
+  {
+    // sum over the TPR threads of a row (they are neighbouring lanes)
+    auto row_sum = [&](float x, unsigned mask) {
+#pragma unroll
+      for (int o = 1; o < TPR; o <<= 1) x += __shfl_xor_sync(mask, x, o);
+      return x;
+    };
+    const unsigned own_mask = ((TPR == 32) ? 0xffffffffu : ((1u << TPR) - 1u)) << (lane & ~(TPR - 1));   // the lanes of this row
+    // The owners of row k set up step k: reflector into shared row k, scalars into dd / ee / bet.
+    // Called by all TPR owners together (one warp).
+    auto setup = [&](int k) {
+      float s2 = 0.f, x0 = 0.f, dg = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int col = 4 * (c * TPR + tq) + e;
+          if (col > k) s2 = fmaf(a[c][e], a[c][e], s2);
+          if (col == k + 1) x0 = a[c][e];
+          if (col == k) dg = a[c][e];
+        }
+      s2 = row_sum(s2, own_mask);
+      x0 = row_sum(x0, own_mask);
+      dg = row_sum(dg, own_mask);
       const float tail = s2 - x0 * x0;            // energy below the sub-diagonal entry
-      float alpha = x0, beta = 0.f, v0 = 0.f;
+      float alpha = x0, beta = 0.f, v0 = x0;
       if (tail > 1e-30f * s2 && s2 > 0.f) {
         alpha = (x0 >= 0.f) ? -sqrtf(s2) : sqrtf(s2);
         v0 = x0 - alpha;
         beta = 1.f / (s2 - x0 * alpha);           // 2 / |v|^2
       }
-      dd[k] = A[k * np + k];
-      ee[k] = alpha;
-      bet[k] = beta;
-      x[0] = v0;                                  // row k now holds the reflector
-      red[k & 1] = 0.f;                           // accumulates v . p of step k (the other slot may still be read)
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const int col0 = 4 * (c * TPR + tq);
+        if (col0 + 3 > k) {
+          float4 v;
+          v.x = (col0 + 0 > k) ? ((col0 + 0 == k + 1) ? v0 : a[c][0]) : 0.f;
+          v.y = (col0 + 1 > k) ? ((col0 + 1 == k + 1) ? v0 : a[c][1]) : 0.f;
+          v.z = (col0 + 2 > k) ? ((col0 + 2 == k + 1) ? v0 : a[c][2]) : 0.f;
+          v.w = (col0 + 3 > k) ? ((col0 + 3 == k + 1) ? v0 : a[c][3]) : 0.f;
+          *reinterpret_cast<float4*>(A + k * np + col0) = v;
+        }
+      }
+      if (tq == 0) {
+        dd[k] = dg;
+        ee[k] = alpha;
+        bet[k] = beta;
+        red[k & 1] = 0.f;                         // accumulates v . p of step k (the other slot may still be read)
+      }
     };
-    if (warp == 0) {
-      float s2 = 0.f;
-      for (int i = 1 + lane; i < n; i += 32) s2 += A[i] * A[i];
-      s2 = warp_sum(s2);
-      if (lane == 0) setup(0, s2);
-    }
+    if (trow == 0) setup(0);
     __syncthreads();
     for (int k = 0; k < n - 2; ++k) {
-      const int m = n - k - 1;                    // order of the trailing block
-      const float* v = A + k * np + k + 1;        // reflector k, entries 0 .. m-1
+      const float* v = A + k * np;                // reflector k, absolute column index, zero up to column k
       const float beta = bet[k];
-      float* row = A + (k + 1 + trow) * np + k + 1;
-      float K = 0.f;
+      const bool active = trow > k;
+      if (trow == k && tq == 0) pp[k] = 0.f;      // row k takes no further part (its column meets v = 0 from now on)
       if (beta != 0.f) {                          // uniform over the block
-        // p = beta * A22 v : four partial sums per row, combined by two shuffles
-        float a0 = 0.f, a1 = 0.f;
-        if (trow < m) {
-          int j = tq;
-          for (; j + 4 < m; j += 8) {
-            a0 = fmaf(row[j], v[j], a0);
-            a1 = fmaf(row[j + 4], v[j + 4], a1);
+        // p = beta * A v
+        float acc = 0.f;
+        if (active) {
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) {
+            const int col0 = 4 * (c * TPR + tq);
+            if (col0 + 3 > k) {
+              const float4 v4 = *reinterpret_cast<const float4*>(v + col0);
+              acc = fmaf(a[c][0], v4.x, acc);
+              acc = fmaf(a[c][1], v4.y, acc);
+              acc = fmaf(a[c][2], v4.z, acc);
+              acc = fmaf(a[c][3], v4.w, acc);
+            }
           }
-          if (j < m) a0 = fmaf(row[j], v[j], a0);
         }
-        float acc = a0 + a1;
-        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        acc = row_sum(acc, 0xffffffffu);
         float vp = 0.f;
-        if (tq == 0 && trow < m) {
+        if (active && tq == 0) {
           acc *= beta;
           pp[trow] = acc;
           vp = acc * v[trow];
         }
-        vp = warp_sum(vp);                        // 8 rows per warp
+        vp = warp_sum(vp);
         if (lane == 0 && vp != 0.f) atomicAdd(&red[k & 1], vp);
         __syncthreads();
-        K = 0.5f * beta * red[k & 1];
-      }
-      // A22 -= v w^T + w v^T,  w = p - K v ; the owners of the next pivot row also sum its squares
-      float s2n = 0.f;
-      if (trow < m) {
-        if (beta != 0.f) {
-          const float vi = v[trow], wi = pp[trow] - K * vi;
-#pragma unroll 4
-          for (int j = tq; j < m; j += 4) {
-            const float vj = v[j], wj = pp[j] - K * vj;
-            const float a = row[j] - (vi * wj + wi * vj);
-            row[j] = a;
-            if (trow == 0 && j >= 1) s2n = fmaf(a, a, s2n);
+        // A -= v w^T + w v^T with w = p - K v, written as  a_ij -= v_i p_j + (p_i - 2 K v_i) v_j
+        if (active) {
+          const float K = 0.5f * beta * red[k & 1];
+          const float vi = v[trow], ci = pp[trow] - 2.f * K * vi;
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) {
+            const int col0 = 4 * (c * TPR + tq);
+            if (col0 + 3 > k) {
+              const float4 v4 = *reinterpret_cast<const float4*>(v + col0);
+              const float4 p4 = *reinterpret_cast<const float4*>(pp + col0);
+              a[c][0] -= fmaf(vi, p4.x, ci * v4.x);
+              a[c][1] -= fmaf(vi, p4.y, ci * v4.y);
+              a[c][2] -= fmaf(vi, p4.z, ci * v4.z);
+              a[c][3] -= fmaf(vi, p4.w, ci * v4.w);
+            }
           }
-        } else if (trow == 0) {
-          for (int j = tq; j < m; j += 4)
-            if (j >= 1) s2n = fmaf(row[j], row[j], s2n);
         }
       }
-      if (warp == 0) {                            // rows 0 .. 7 of the trailing block; row 0 = next pivot row
-        s2n += __shfl_xor_sync(0xffffffffu, s2n, 1);
-        s2n += __shfl_xor_sync(0xffffffffu, s2n, 2);
-        __syncwarp();
-        if (lane == 0 && k + 1 < n - 2) setup(k + 1, s2n);
-      }
+      // (the set-up of row n - 2 finds nothing below its sub-diagonal: it records d, e and beta = 0)
+      if (trow == k + 1) setup(k + 1);
       __syncthreads();
     }
-  }
-  if (tid == 0) {
-    dd[n - 2] = A[(n - 2) * np + n - 2];
-    ee[n - 2] = A[(n - 2) * np + n - 1];
-    dd[n - 1] = A[(n - 1) * np + n - 1];
-    ee[n - 1] = 0.f;
-    bet[n - 2] = bet[n - 1] = 0.f;
+    if (trow == n - 1) {
+      float dg = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (4 * (c * TPR + tq) + e == n - 1) dg = a[c][e];
+      dg = row_sum(dg, own_mask);
+      if (tq == 0) {
+        dd[n - 1] = dg;
+        ee[n - 1] = 0.f;
+        bet[n - 1] = 0.f;
+      }
+    }
   }
   __syncthreads();
 
@@ -832,9 +878,14 @@ cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
   const int zs = r_eff | 1;                       // odd row pitch: conflict-free both ways
   const size_t extra = (2 * r_eff <= d) ? 0 : (size_t)r_eff * (r_eff | 1);   // Gram scratch when A has no free quadrant
   const size_t smem = ((size_t)d * (d + 4) + (size_t)d * (zs + 3) + 8 * (size_t)d + 2 * kEigMaxR + 16 + extra) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(eig_tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (d != 128 && d != 64) return cudaErrorInvalidValue;
+  cudaError_t e = d == 128 ? cudaFuncSetAttribute(eig_tridiag_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                           : cudaFuncSetAttribute(eig_tridiag_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  eig_tridiag_kernel<<<blocks, kEigThreads, smem, s>>>(F, d, zs);
+  if (d == 128)
+    eig_tridiag_kernel<128><<<blocks, kEigThreads, smem, s>>>(F, zs);
+  else
+    eig_tridiag_kernel<64><<<blocks, kEigThreads, smem, s>>>(F, zs);
   return cudaGetLastError();
 }
 
