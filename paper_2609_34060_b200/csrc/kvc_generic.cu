@@ -444,28 +444,36 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   }
   {
     // sum over the TPR threads of a row (they are neighbouring lanes)
-    auto row_sum = [&](float x, unsigned mask) {
+    auto row_sum = [&](float x) {
 #pragma unroll
-      for (int o = 1; o < TPR; o <<= 1) x += __shfl_xor_sync(mask, x, o);
+      for (int o = 1; o < TPR; o <<= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
       return x;
     };
-    const unsigned own_mask = ((TPR == 32) ? 0xffffffffu : ((1u << TPR) - 1u)) << (lane & ~(TPR - 1));   // the lanes of this row
-    // The owners of row k set up step k: reflector into shared row k, scalars into dd / ee / bet.
-    // Called by all TPR owners together (one warp).
+    float* redw = cdot;                           // [NW] per-warp parts of v . p (cdot is free until step 3)
+    // Set-up of step k, by the WHOLE warp that holds row k (a serial section of the block: kept short).
+    // The row's owners publish it to shared row k; the warp reads it back one float4 per lane, forms
+    // the reflector scalars, and rewrites the row as the reflector (zeros up to column k, v0 at k + 1).
     auto setup = [&](int k) {
-      float s2 = 0.f, x0 = 0.f, dg = 0.f;
+      float* rowk = A + k * np;
+      if (trow == k) {
 #pragma unroll
-      for (int c = 0; c < NCH; ++c)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int col = 4 * (c * TPR + tq) + e;
-          if (col > k) s2 = fmaf(a[c][e], a[c][e], s2);
-          if (col == k + 1) x0 = a[c][e];
-          if (col == k) dg = a[c][e];
+        for (int c = 0; c < NCH; ++c) {
+          const int col0 = 4 * (c * TPR + tq);
+          if (col0 + 3 >= k) *reinterpret_cast<float4*>(rowk + col0) = make_float4(a[c][0], a[c][1], a[c][2], a[c][3]);
         }
-      s2 = row_sum(s2, own_mask);
-      x0 = row_sum(x0, own_mask);
-      dg = row_sum(dg, own_mask);
+      }
+      __syncwarp();
+      const int c0 = 4 * lane;
+      const bool mine = lane < N / 4 && c0 + 3 > k;
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (mine) x = *reinterpret_cast<const float4*>(rowk + c0);
+      if (c0 + 0 <= k) x.x = 0.f;
+      if (c0 + 1 <= k) x.y = 0.f;
+      if (c0 + 2 <= k) x.z = 0.f;
+      if (c0 + 3 <= k) x.w = 0.f;
+      const float x0 = rowk[k + 1], dg = rowk[k];
+      float s2 = warp_sum(fmaf(x.x, x.x, x.y * x.y) + fmaf(x.z, x.z, x.w * x.w));
+      __syncwarp();                               // x0 and dg are read before the row is rewritten
       const float tail = s2 - x0 * x0;            // energy below the sub-diagonal entry
       float alpha = x0, beta = 0.f, v0 = x0;
       if (tail > 1e-30f * s2 && s2 > 0.f) {
@@ -473,26 +481,20 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
         v0 = x0 - alpha;
         beta = 1.f / (s2 - x0 * alpha);           // 2 / |v|^2
       }
-#pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        const int col0 = 4 * (c * TPR + tq);
-        if (col0 + 3 > k) {
-          float4 v;
-          v.x = (col0 + 0 > k) ? ((col0 + 0 == k + 1) ? v0 : a[c][0]) : 0.f;
-          v.y = (col0 + 1 > k) ? ((col0 + 1 == k + 1) ? v0 : a[c][1]) : 0.f;
-          v.z = (col0 + 2 > k) ? ((col0 + 2 == k + 1) ? v0 : a[c][2]) : 0.f;
-          v.w = (col0 + 3 > k) ? ((col0 + 3 == k + 1) ? v0 : a[c][3]) : 0.f;
-          *reinterpret_cast<float4*>(A + k * np + col0) = v;
-        }
+      if (mine) {
+        if (c0 + 0 == k + 1) x.x = v0;
+        if (c0 + 1 == k + 1) x.y = v0;
+        if (c0 + 2 == k + 1) x.z = v0;
+        if (c0 + 3 == k + 1) x.w = v0;
+        *reinterpret_cast<float4*>(rowk + c0) = x;
       }
-      if (tq == 0) {
+      if (lane == 0) {
         dd[k] = dg;
         ee[k] = alpha;
         bet[k] = beta;
-        red[k & 1] = 0.f;                         // accumulates v . p of step k (the other slot may still be read)
       }
     };
-    if (trow == 0) setup(0);
+    if (warp == 0) setup(0);
     __syncthreads();
     for (int k = 0; k < n - 2; ++k) {
       const float* v = A + k * np;                // reflector k, absolute column index, zero up to column k
@@ -501,21 +503,21 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
       if (trow == k && tq == 0) pp[k] = 0.f;      // row k takes no further part (its column meets v = 0 from now on)
       if (beta != 0.f) {                          // uniform over the block
         // p = beta * A v
-        float acc = 0.f;
+        float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
         if (active) {
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             const int col0 = 4 * (c * TPR + tq);
             if (col0 + 3 > k) {
               const float4 v4 = *reinterpret_cast<const float4*>(v + col0);
-              acc = fmaf(a[c][0], v4.x, acc);
-              acc = fmaf(a[c][1], v4.y, acc);
-              acc = fmaf(a[c][2], v4.z, acc);
-              acc = fmaf(a[c][3], v4.w, acc);
+              acc0 = fmaf(a[c][0], v4.x, acc0);
+              acc1 = fmaf(a[c][1], v4.y, acc1);
+              acc2 = fmaf(a[c][2], v4.z, acc2);
+              acc3 = fmaf(a[c][3], v4.w, acc3);
             }
           }
         }
-        acc = row_sum(acc, 0xffffffffu);
+        float acc = row_sum((acc0 + acc1) + (acc2 + acc3));
         float vp = 0.f;
         if (active && tq == 0) {
           acc *= beta;
@@ -523,11 +525,17 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
           vp = acc * v[trow];
         }
         vp = warp_sum(vp);
-        if (lane == 0 && vp != 0.f) atomicAdd(&red[k & 1], vp);
+        if (lane == 0) redw[warp] = vp;
         __syncthreads();
         // A -= v w^T + w v^T with w = p - K v, written as  a_ij -= v_i p_j + (p_i - 2 K v_i) v_j
         if (active) {
-          const float K = 0.5f * beta * red[k & 1];
+          float vdotp = 0.f;
+#pragma unroll
+          for (int w4 = 0; w4 < NW / 4; ++w4) {
+            const float4 r4 = *reinterpret_cast<const float4*>(redw + 4 * w4);
+            vdotp += (r4.x + r4.y) + (r4.z + r4.w);
+          }
+          const float K = 0.5f * beta * vdotp;
           const float vi = v[trow], ci = pp[trow] - 2.f * K * vi;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
@@ -544,19 +552,15 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
         }
       }
       // (the set-up of row n - 2 finds nothing below its sub-diagonal: it records d, e and beta = 0)
-      if (trow == k + 1) setup(k + 1);
+      if (warp == ((k + 1) * TPR) / 32) setup(k + 1);
       __syncthreads();
     }
-    if (trow == n - 1) {
-      float dg = 0.f;
-#pragma unroll
-      for (int c = 0; c < NCH; ++c)
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (4 * (c * TPR + tq) + e == n - 1) dg = a[c][e];
-      dg = row_sum(dg, own_mask);
-      if (tq == 0) {
-        dd[n - 1] = dg;
+    if (warp == ((n - 1) * TPR) / 32) {           // the last diagonal entry, through shared memory like the others
+      float* rowk = A + (n - 1) * np;
+      if (trow == n - 1 && tq == TPR - 1) rowk[n - 1] = a[NCH - 1][3];
+      __syncwarp();
+      if (lane == 0) {
+        dd[n - 1] = rowk[n - 1];
         ee[n - 1] = 0.f;
         bet[n - 1] = 0.f;
       }
