@@ -660,27 +660,20 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
       for (int i = 1; i < n; ++i) {
         const float sub = ee[i - 1], dg = dd[i] - s, sp = (i < n - 1) ? ee[i] : 0.f;
         const float xi = Zt[i * zs + j];
-        if (fabsf(sub) > fabsf(u)) {              // swap rows i-1 and i
-          const float rs = 1.f / sub;
-          const float mult = u * rs;
-          R0[i - 1] = rs;
-          U1[i - 1] = dg;
-          swp[(i - 1) >> 5] |= 1u << ((i - 1) & 31);
-          u = v - mult * dg;
-          v = -mult * sp;
-          Zt[(i - 1) * zs + j] = xi;
-          xp = xp - mult * xi;
-        } else {
-          if (u == 0.f) u = eps3;
-          const float ru = 1.f / u;
-          const float mult = sub * ru;
-          R0[i - 1] = ru;
-          U1[i - 1] = v;
-          u = dg - mult * v;
-          v = sp;
-          Zt[(i - 1) * zs + j] = xp;
-          xp = xi - mult * xp;
-        }
+        // one elimination step, written without branches (the lanes of the warp pivot differently):
+        // swap rows i-1 and i when the sub-diagonal entry is the larger pivot
+        const bool swap = fabsf(sub) > fabsf(u);
+        float piv = swap ? sub : u;
+        if (piv == 0.f) piv = eps3;
+        const float rp = 1.f / piv;
+        const float mult = (swap ? u : sub) * rp;
+        R0[i - 1] = rp;
+        U1[i - 1] = swap ? dg : v;
+        if (swap) swp[(i - 1) >> 5] |= 1u << ((i - 1) & 31);
+        Zt[(i - 1) * zs + j] = swap ? xi : xp;
+        xp = swap ? (xp - mult * xi) : (xi - mult * xp);
+        u = swap ? (v - mult * dg) : (dg - mult * v);
+        v = swap ? (-mult * sp) : sp;
       }
       if (fabsf(u) < eps3) u = (u < 0.f) ? -eps3 : eps3;
       float y2 = xp / u;
