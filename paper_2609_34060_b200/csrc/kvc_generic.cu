@@ -748,42 +748,52 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
     }
   }
 
-  // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, one warp per vector, then output
+  // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, then output
   float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
-  // every warp carries up to four of its vectors through the reflectors together (independent
-  // reduction chains overlap)
-  for (int jb = warp * 4; jb < ((r_eff + 3) & ~3); jb += NW * 4) {
-    for (int k = n - 3; k >= 0; --k) {
-      const float beta = bet[k];
-      if (beta == 0.f) continue;
-      const float* v = A + k * np;                // reflector entries at columns k+1 .. n-1
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-      for (int c = k + 1 + lane; c < n; c += 32) {
-        const float vc = v[c];
-        const float* z = Zt + c * zs + jb;
-        a0 = fmaf(vc, z[0], a0);
-        if (jb + 1 < r_eff) a1 = fmaf(vc, z[1], a1);
-        if (jb + 2 < r_eff) a2 = fmaf(vc, z[2], a2);
-        if (jb + 3 < r_eff) a3 = fmaf(vc, z[3], a3);
-      }
+  // Sixteen threads (half a warp) carry one vector through all reflectors with its entries in
+  // registers: thread `part` holds rows RPT part .. RPT part + RPT-1.  Per reflector: v . z over the
+  // half-warp (four shuffles), then z -= beta (v . z) v.  No block barrier: vectors are independent.
+  {
+    constexpr int RPT = N / 16;                   // rows per thread: 8 (N = 128) or 4 (N = 64)
+    const int part = lane & 15;
+    for (int j0 = 0; j0 < r_eff; j0 += kEigThreads / 16) {
+      const int j = j0 + (tid >> 4);
+      const bool have = j < r_eff;                // uniform over the half-warp
+      float z[RPT];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        a0 += __shfl_xor_sync(0xffffffffu, a0, o);
-        a1 += __shfl_xor_sync(0xffffffffu, a1, o);
-        a2 += __shfl_xor_sync(0xffffffffu, a2, o);
-        a3 += __shfl_xor_sync(0xffffffffu, a3, o);
+      for (int e = 0; e < RPT; ++e) z[e] = have ? Zt[(RPT * part + e) * zs + j] : 0.f;
+      for (int k = n - 3; k >= 0; --k) {
+        const float beta = bet[k];
+        if (beta == 0.f) continue;
+        const float* v = A + k * np + RPT * part;   // reflector entries are zero up to column k
+        float vr[RPT];
+#pragma unroll
+        for (int e4 = 0; e4 < RPT / 4; ++e4) {
+          // a group of four columns that ends at or before column k was never written as part of
+          // the reflector (the set-up rewrites only groups that reach beyond k): it counts as zero
+          float4 t4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (RPT * part + 4 * e4 + 3 > k) t4 = *reinterpret_cast<const float4*>(v + 4 * e4);
+          vr[4 * e4 + 0] = t4.x;
+          vr[4 * e4 + 1] = t4.y;
+          vr[4 * e4 + 2] = t4.z;
+          vr[4 * e4 + 3] = t4.w;
+        }
+        float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+        for (int e = 0; e < RPT; e += 2) {
+          d0 = fmaf(vr[e], z[e], d0);
+          d1 = fmaf(vr[e + 1], z[e + 1], d1);
+        }
+        float dot = d0 + d1;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        dot *= beta;
+#pragma unroll
+        for (int e = 0; e < RPT; ++e) z[e] = fmaf(-dot, vr[e], z[e]);
       }
-      a0 *= beta;
-      a1 *= beta;
-      a2 *= beta;
-      a3 *= beta;
-      for (int c = k + 1 + lane; c < n; c += 32) {
-        const float vc = v[c];
-        float* z = Zt + c * zs + jb;
-        z[0] -= a0 * vc;
-        if (jb + 1 < r_eff) z[1] -= a1 * vc;
-        if (jb + 2 < r_eff) z[2] -= a2 * vc;
-        if (jb + 3 < r_eff) z[3] -= a3 * vc;
+      if (have) {
+#pragma unroll
+        for (int e = 0; e < RPT; ++e) Zt[(RPT * part + e) * zs + j] = z[e];
       }
     }
   }
