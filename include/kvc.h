@@ -231,6 +231,36 @@ int kvc_apply_batch(const kvc_item *items, int32_t n_items, const kvc_rope *rope
 size_t kvc_batch_workspace_bytes(int32_t n_items);
 
 /*
+ * Reliability gate of the anchor pool (App. A.3 "Reliability Gate", Eqs. 9-11).
+ *
+ * kvc_gate_distance (Eq. 9): for every anchor v of a pool,
+ *     dist_sq[v] = sum over layers l, heads h, tokens t < k of
+ *                  || V_src[l,h,t,:] - coeff_v[l,h,t,:] . basis_v[l,h] ||^2 ,
+ * the squared Frobenius distance between the source cache's VALUE states and the value states
+ * anchor v reconstructs from the low-rank factors of its base cache (a state fitted with
+ * kvc_state_update(src = NULL, tgt = the anchor's cache)).  The gate distance of Eq. 9 is
+ * sqrt(dist_sq[v]).  Only coeff_v / basis_v of each state are read; the key factors may be NULL.
+ *   src       source cache (host descriptor, device data), read only
+ *   anchors   host array [n_anchors]; every anchor needs n_cov >= k (anchors whose stored length is
+ *             below the comparison length are not compatible: KVC_E_SHAPE), 0 < r <= 256
+ *   k         comparison prefix length, 0 <= k <= src->T
+ *   dist_sq   DEVICE float64 [n_anchors], overwritten (cleared, then accumulated: the sum's order
+ *             over CTAs is not fixed, which moves the result by float64 rounding only)
+ * Products run in split bf16 with float32 accumulation like kvc_apply; squares are summed in
+ * float32 per 32-channel row segment and in float64 beyond.
+ *
+ * kvc_gate_weights (Eqs. 10-11), on the device so that no host round trip is needed:
+ *     g[v] = softmax_v( -sqrt(dist_sq[v]) / temperature ),   entropy[0] = -sum_v g log2 g / log2 n
+ * in float64 (0 log 0 = 0).  n_anchors < 2 returns KVC_E_INVALID_ARG: the method has no gate value
+ * then and falls back to dense prefill.  dist_sq, g [n_anchors], entropy [1]: DEVICE float64.
+ * The caller accepts the correction when entropy[0] <= tau.
+ */
+int kvc_gate_distance(const kvc_cache *src, const kvc_state *anchors, int32_t n_anchors, int32_t k,
+                      double *dist_sq, void *stream);
+int kvc_gate_weights(const double *dist_sq, int32_t n_anchors, double temperature, double *g,
+                     double *entropy, void *stream);
+
+/*
  * Device-side anomalies never trap or hang: a kernel that meets a page id outside
  * [0, n_phys_pages) or whose bounded wait on an asynchronous copy runs out skips
  * that tile and ORs a bit into a per-device status word.

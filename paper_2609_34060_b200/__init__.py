@@ -23,11 +23,14 @@ KVC_ROPE_HALF, KVC_ROPE_INTERLEAVED = 0, 1
 KVC_PROJECT, KVC_FIT = 0, 1
 KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
 KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4
+KVC_OK = 0
+(KVC_E_INVALID_ARG, KVC_E_SHAPE, KVC_E_UNSUPPORTED, KVC_E_ALIAS, KVC_E_CUDA, KVC_E_WORKSPACE, KVC_E_DEVICE_FLAG,
+ KVC_E_TOO_LARGE) = (-1, -2, -3, -4, -5, -6, -7, -8)
 
 EXPORTS = (
     "kvc_apply", "kvc_chain", "kvc_state_update", "kvc_state_update_noalloc", "kvc_workspace_bytes", "kvc_apply_batch",
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
-    "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version",
+    "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
 )
 
 
@@ -82,6 +85,8 @@ def load(path: Optional[str] = None):
     lib.kvc_apply_batch.argtypes = [PI, i32, PR, vp, sz, vp, vp]
     lib.kvc_batch_workspace_bytes.argtypes = [i32]
     lib.kvc_batch_workspace_bytes.restype = sz
+    lib.kvc_gate_distance.argtypes = [PC, PS, i32, i32, vp, vp]
+    lib.kvc_gate_weights.argtypes = [vp, i32, C.c_double, vp, vp, vp]
     lib.kvc_status_poll.argtypes = [C.POINTER(C.c_uint32)]
     lib.kvc_status_reset.argtypes = []
     lib.kvc_set_path.argtypes = [i32]
@@ -176,12 +181,24 @@ class State:
     def empty() -> "State":
         return State(None, None, None, None, n_cov=0)
 
+    @staticmethod
+    def values_only(coeff_v, basis_v) -> "State":
+        """Value factors alone (what the reliability gate reads); the key pointers are NULL."""
+        s = State.__new__(State)
+        s.coeff_k = s.basis_k = None
+        s.coeff_v, s.basis_v = coeff_v, basis_v
+        s.r, s.n_cov = int(basis_v.shape[2]), int(coeff_v.shape[2])
+        assert coeff_v.dtype == torch.float32 and coeff_v.is_contiguous() and basis_v.is_contiguous()
+        assert basis_v.dtype in (torch.float32, torch.bfloat16) and int(coeff_v.shape[3]) == s.r
+        return s
+
     def struct(self) -> kvc_state:
         s = kvc_state()
         ptr = lambda t: 0 if t is None else t.data_ptr()
         s.coeff_k, s.coeff_v, s.basis_k, s.basis_v = ptr(self.coeff_k), ptr(self.coeff_v), ptr(self.basis_k), ptr(self.basis_v)
         s.r, s.n_cov = self.r, self.n_cov
-        s.basis_dtype = KVC_BF16 if (self.basis_k is not None and self.basis_k.dtype == torch.bfloat16) else KVC_F32
+        b = self.basis_k if self.basis_k is not None else self.basis_v
+        s.basis_dtype = KVC_BF16 if (b is not None and b.dtype == torch.bfloat16) else KVC_F32
         return s
 
 
@@ -284,6 +301,26 @@ def kvc_apply_batch(items: Sequence[Item], rope: Rope, workspace: torch.Tensor, 
     _check(load().kvc_apply_batch(arr, n, C.byref(r), workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), staging.data_ptr(), _stream(stream)),
            "kvc_apply_batch")
+
+
+def kvc_gate_distance(src: Cache, anchors: Sequence[State], k: int, dist_sq: torch.Tensor, stream=None) -> None:
+    """Eq. 9, squared: dist_sq[v] (device float64 [len(anchors)]) for every anchor's value factors."""
+    n = len(anchors)
+    arr = (kvc_state * max(n, 1))()
+    for i, a in enumerate(anchors):
+        arr[i] = a.struct()
+    c = src.struct()
+    assert dist_sq.dtype == torch.float64 and dist_sq.is_cuda and dist_sq.numel() >= n
+    _check(load().kvc_gate_distance(C.byref(c), arr, n, int(k), dist_sq.data_ptr(), _stream(stream)), "kvc_gate_distance")
+
+
+def kvc_gate_weights(dist_sq: torch.Tensor, g: torch.Tensor, entropy: torch.Tensor, temperature: float = 1.0,
+                     stream=None) -> None:
+    """Eqs. 10-11 on the device: g = softmax(-sqrt(dist_sq)/T), entropy[0] = normalised entropy of g."""
+    n = int(dist_sq.numel())
+    assert dist_sq.dtype == g.dtype == entropy.dtype == torch.float64 and g.numel() >= n and entropy.numel() >= 1
+    _check(load().kvc_gate_weights(dist_sq.data_ptr(), n, float(temperature), g.data_ptr(), entropy.data_ptr(),
+                                   _stream(stream)), "kvc_gate_weights")
 
 
 def kvc_status_poll() -> int:

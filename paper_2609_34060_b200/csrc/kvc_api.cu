@@ -403,6 +403,83 @@ int kvc_apply_batch(const kvc_item* items, int32_t n_items, const kvc_rope* rope
   return KVC_OK;
 }
 
+int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_anchors, int32_t k, double* dist_sq,
+                      void* stream) {
+  if (!src || n_anchors < 0 || (n_anchors > 0 && (!anchors || !dist_sq)) || k < 0) return KVC_E_INVALID_ARG;
+  if (n_anchors == 0) return KVC_OK;
+  DevCache dc;
+  int rc;
+  if ((rc = resolve_cache(src, &dc)) != KVC_OK) return rc;
+  if (k > src->T) return KVC_E_SHAPE;
+  for (int v = 0; v < n_anchors; ++v) {
+    const kvc_state& a = anchors[v];
+    if (a.r <= 0 || a.r > 256 || a.n_cov < 0) return KVC_E_INVALID_ARG;
+    if (a.n_cov < k) return KVC_E_SHAPE;            // not compatible at this comparison length
+    if (k > 0 && (!a.coeff_v || !a.basis_v)) return KVC_E_INVALID_ARG;
+    if (a.basis_dtype != KVC_F32 && a.basis_dtype != KVC_BF16) return KVC_E_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a.coeff_v) | reinterpret_cast<uintptr_t>(a.basis_v)) & 15) return KVC_E_UNSUPPORTED;
+  }
+  if (reinterpret_cast<uintptr_t>(dist_sq) & 7) return KVC_E_INVALID_ARG;
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(dist_sq, 0, sizeof(double) * (size_t)n_anchors, s) != cudaSuccess) return KVC_E_CUDA;
+  if (k == 0) return KVC_OK;
+  for (int v = 0; v < n_anchors; ++v) {
+    const kvc_state& a = anchors[v];
+    bool done = false;
+    if (tl_path_force != KVC_PATH_GENERIC) {
+      // the apply kernel's tile walk over the value slabs of the first k tokens
+      DevItem it;
+      memset(&it, 0, sizeof(it));
+      it.src = dc;
+      it.src.T = k;
+      it.dst = it.src;
+      it.st.coeff_k = it.st.coeff_v = a.coeff_v;
+      it.st.basis_k = it.st.basis_v = a.basis_v;
+      it.st.r = a.r;
+      it.st.n_cov = a.n_cov;
+      it.st.basis_bf16 = a.basis_dtype == KVC_BF16;
+      it.L = src->L;
+      it.H = src->H;
+      for (int c = 0; c < kMaxHalfD; ++c) it.cs[c] = 1.f;
+      const int trc = tc_gate_distance(it, src->d, status, dist_sq + v, s);
+      if (trc == KVC_OK) {
+        tl_last_path = KVC_PATH_TC;
+        done = true;
+      } else if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) {
+        return trc;
+      }
+    }
+    if (!done) {
+      GateLaunch g;
+      memset(&g, 0, sizeof(g));
+      g.src = dc;
+      g.coeff = a.coeff_v;
+      g.basis = a.basis_v;
+      g.r = a.r;
+      g.n_cov = a.n_cov;
+      g.basis_bf16 = a.basis_dtype == KVC_BF16;
+      g.k = k;
+      g.L = src->L;
+      g.H = src->H;
+      g.out = dist_sq + v;
+      g.status = status;
+      if (launch_gate_generic(g, src->d, s) != cudaSuccess) return KVC_E_CUDA;
+      tl_last_path = KVC_PATH_GENERIC;
+    }
+  }
+  return KVC_OK;
+}
+
+int kvc_gate_weights(const double* dist_sq, int32_t n_anchors, double temperature, double* g, double* entropy, void* stream) {
+  if (!dist_sq || !g || !entropy || !(temperature > 0.0)) return KVC_E_INVALID_ARG;
+  if (n_anchors < 2) return KVC_E_INVALID_ARG;      // fewer than two compatible anchors: no gate value, dense prefill
+  if (launch_gate_weights(dist_sq, n_anchors, temperature, g, entropy, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return KVC_E_CUDA;
+  return KVC_OK;
+}
+
 int kvc_status_poll(uint32_t* flags) {
   uint32_t w = 0;
   if (cudaMemcpyFromSymbol(&w, g_status_word, sizeof(w)) != cudaSuccess) return KVC_E_CUDA;

@@ -71,6 +71,16 @@ struct FitLaunch {             // Gram + eigensolve
   alignas(16) float sn[kMaxHalfD];
 };
 
+struct GateLaunch {            // Eq. 9 for one anchor, CUDA-core kernel
+  DevCache src;                // values only
+  const float* coeff;          // [L,H,n_cov,r] value coefficients of the anchor's base factorisation
+  const void* basis;           // [L,H,r,d]
+  int32_t r, n_cov, basis_bf16, k;
+  int32_t L, H;
+  double* out;                 // the squared distance is added here
+  uint32_t* status;
+};
+
 // Address of row (l, h, t) of a cache; returns nullptr (and flags) on a bad page id.
 __device__ __forceinline__ __nv_bfloat16* row_ptr(const DevCache& c, __nv_bfloat16* base, int l, int h, int t,
                                                    uint32_t* status) {

@@ -1,0 +1,88 @@
+// Reliability gate (App. A.3, Eqs. 9-11): CUDA-core distance kernel for shapes the tensor-core
+// path does not take, and the softmax / normalised-entropy kernel.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/kvc.h"
+#include "kvc_dev.cuh"
+#include "kvc_launch.h"
+
+namespace kvc {
+
+// Eq. 9, one anchor.  One warp per token of a (layer, head) slab: lane c holds channels c, c + 32, ...
+// of V[t] - coeff[t] . basis; squares summed in float32 per token, float64 across tokens.
+template <int D>
+__global__ void __launch_bounds__(256) gate_generic_kernel(const GateLaunch g) {
+  constexpr int CPL = D / 32;                      // channels per lane
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int slab = blockIdx.y;
+  const int l = slab / g.H, h = slab - l * g.H;
+  const float* coeff = g.coeff + (int64_t)slab * g.n_cov * g.r;
+  double acc = 0.0;
+  for (int t = blockIdx.x * 8 + warp; t < g.k; t += gridDim.x * 8) {
+    const __nv_bfloat16* row = row_ptr(g.src, g.src.v, l, h, t, g.status);
+    if (!row) continue;
+    float x[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) x[c] = __bfloat162float(row[lane + 32 * c]);
+    const float* ct = coeff + (int64_t)t * g.r;
+    for (int q = 0; q < g.r; ++q) {
+      const float cq = ct[q];
+      const int64_t boff = ((int64_t)slab * g.r + q) * D + lane;
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        const float b = g.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(g.basis)[boff + 32 * c])
+                                     : reinterpret_cast<const float*>(g.basis)[boff + 32 * c];
+        x[c] = fmaf(-cq, b, x[c]);
+      }
+    }
+    float sq = 0.f;
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) sq = fmaf(x[c], x[c], sq);
+    acc += (double)sq;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0 && acc != 0.0) atomicAdd(g.out, acc);
+}
+
+cudaError_t launch_gate_generic(const GateLaunch& g, int d, cudaStream_t s) {
+  if (g.k <= 0 || g.L * g.H <= 0) return cudaSuccess;
+  int bx = (g.k + 7) / 8;
+  if (bx > 64) bx = 64;
+  const dim3 grid((unsigned)bx, (unsigned)(g.L * g.H));
+  if (d == 128)
+    gate_generic_kernel<128><<<grid, 256, 0, s>>>(g);
+  else
+    gate_generic_kernel<64><<<grid, 256, 0, s>>>(g);
+  return cudaGetLastError();
+}
+
+// Eqs. 10-11 in float64, one warp: g_v = softmax(-d_v / T), entropy = -sum g log2 g / log2 n.
+__global__ void gate_weights_kernel(const double* dist_sq, int n, double inv_temp, double* gw, double* entropy) {
+  const int lane = threadIdx.x;
+  double zmax = -1e300;
+  for (int v = lane; v < n; v += 32) zmax = fmax(zmax, -sqrt(fmax(dist_sq[v], 0.0)) * inv_temp);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) zmax = fmax(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+  double sum = 0.0;
+  for (int v = lane; v < n; v += 32) sum += exp(-sqrt(fmax(dist_sq[v], 0.0)) * inv_temp - zmax);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  double hsum = 0.0;
+  for (int v = lane; v < n; v += 32) {
+    const double gv = exp(-sqrt(fmax(dist_sq[v], 0.0)) * inv_temp - zmax) / sum;
+    gw[v] = gv;
+    if (gv > 0.0) hsum -= gv * log2(gv);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) hsum += __shfl_xor_sync(0xffffffffu, hsum, o);
+  if (lane == 0) *entropy = hsum / log2((double)n);
+}
+
+cudaError_t launch_gate_weights(const double* dist_sq, int n, double temperature, double* gw, double* entropy, cudaStream_t s) {
+  gate_weights_kernel<<<1, 32, 0, s>>>(dist_sq, n, 1.0 / temperature, gw, entropy);
+  return cudaGetLastError();
+}
+
+}  // namespace kvc

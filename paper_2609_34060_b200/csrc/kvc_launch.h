@@ -15,4 +15,8 @@ cudaError_t launch_project_generic(const UpdateLaunch& U, int d, int64_t tiles, 
 cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s);
 cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s);
 
+// reliability gate (kvc_gate.cu)
+cudaError_t launch_gate_generic(const GateLaunch& g, int d, cudaStream_t s);
+cudaError_t launch_gate_weights(const double* dist_sq, int n, double temperature, double* gw, double* entropy, cudaStream_t s);
+
 }  // namespace kvc

@@ -58,6 +58,7 @@ struct ApplyTcLaunch {
   int32_t n_items, pairing;
   int64_t total_tiles;
   uint32_t* status;
+  double* gate_out;            // gate-distance mode: the squared distance is added here
   DevItem one;
   ItemMaps one_maps;
 };
@@ -75,6 +76,8 @@ struct Tile {
 
 // Walks a contiguous range of global tiles.  All divisions happen once in init(); stepping to
 // the next tile is a few increments (every role of the CTA steps through every tile).
+// VONLY: only the value slabs are walked (gate distance), one slab per (layer, head).
+template <bool VONLY>
 struct TileWalker {
   const ApplyTcLaunch* p;
   int64_t remaining;
@@ -85,7 +88,7 @@ struct TileWalker {
   __device__ void load_item() {
     it = p->items ? p->items + item : &p->one;
     tps = it->tiles_per_slab;
-    n_slab2 = it->L * it->H * 2;
+    n_slab2 = it->L * it->H * (VONLY ? 1 : 2);
   }
   __device__ void init(const ApplyTcLaunch* pp, int64_t begin, int64_t end_) {
     p = pp;
@@ -111,7 +114,7 @@ struct TileWalker {
       }
       tt = (int)(local % tps);
       slab2 = (int)(local / tps);
-      const int slab = slab2 >> 1;
+      const int slab = VONLY ? slab2 : slab2 >> 1;
       l = slab / it->H;
       h = slab - l * it->H;
     }
@@ -122,8 +125,8 @@ struct TileWalker {
     t.mp = p->maps ? p->maps + item : &p->one_maps;
     t.item = item;
     t.first = first;
-    t.is_v = slab2 & 1;
-    t.slab = slab2 >> 1;
+    t.is_v = VONLY ? 1 : slab2 & 1;
+    t.slab = VONLY ? slab2 : slab2 >> 1;
     t.l = l;
     t.h = h;
     t.t0 = tt * kTileTok;
@@ -138,7 +141,7 @@ struct TileWalker {
     first = true;
     tt = 0;
     ++slab2;
-    if ((slab2 & 1) == 0) {                       // K and V of one (layer, head) are adjacent
+    if (VONLY || (slab2 & 1) == 0) {              // K and V of one (layer, head) are adjacent
       if (++h == it->H) {
         h = 0;
         ++l;
@@ -220,7 +223,9 @@ __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_
 // Two rings of shared-memory slots: NSTAGE base tiles (alive from the load until the TMA store has
 // read them) and NSC coefficient tiles (alive only until the tile's MMAs have completed), so that
 // the short-lived operand does not hold a long-lived slot.
-template <int RB, int NSTAGE, int NSC>
+// GATE: gate-distance mode (Eq. 9): value slabs only, nothing is stored; the team accumulates
+// sum (V - c.B)^2 over its rows and the CTA adds its part to *gate_out.
+template <int RB, int NSTAGE, int NSC, bool GATE = false>
 __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
   constexpr int kStageBytes = kBaseBytes;
   constexpr int kCoeffSlotBytes = RB * kCoeffBlkBytes;
@@ -273,7 +278,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
 
   if (warp == 0) {
     // =============================================================== TMA producer (whole warp)
-    TileWalker w;
+    TileWalker<GATE> w;
     w.init(&p, tile_begin, tile_end);
     uint32_t i = 0, cpos = 0;                       // cpos: position in the coefficient ring
     for (; !w.done(); w.next(), ++i) {
@@ -363,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
   } else if (warp == 1) {
     // =============================================================== MMA issuer
     if (lane == 0) {
-      TileWalker w;
+      TileWalker<GATE> w;
       w.init(&p, tile_begin, tile_end);
       uint32_t i = 0, slabs = 0, cpos = 0;
       for (; !w.done(); w.next(), ++i) {
@@ -416,7 +421,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     // spare warp: keeps the team's warps aligned with the TMEM lane quadrants (warp id & 3)
   } else if (warp == 3) {
     // =============================================================== store warp
-    TileWalker w;
+    TileWalker<GATE> w;
     w.init(&p, tile_begin, tile_end);
     uint32_t i = 0;
     for (; !w.done(); w.next(), ++i) {
@@ -452,7 +457,9 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
       const uint32_t st_base = stages + s * kStageBytes;
       uint8_t* st_ptr = smem + s * kStageBytes;
-      if (!dpaged) {
+      if constexpr (GATE) {
+        // nothing to store: the slot goes straight back to the producer
+      } else if (!dpaged) {
         if (lane == 0) {          // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
           tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
           tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
@@ -499,14 +506,15 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     const int crow = e * 8 + (lane >> 2), cpart = lane & 3;
     const uint32_t csw = (uint32_t)(crow & 7);
 
-    TileWalker w;
+    TileWalker<GATE> w;
     w.init(&p, tile_begin, tile_end);
-    TileWalker wn = w;                              // runs one tile ahead (conversion)
+    TileWalker<GATE> wn = w;                              // runs one tile ahead (conversion)
     uint32_t i = 0;
     bool alive = true;
+    double gate_acc = 0.0;                          // gate-distance mode only
 
     // conversion of the coefficient tile held by walker `cw`, at ring position `ci`
-    auto convert = [&](TileWalker& cw, uint32_t ci) {
+    auto convert = [&](TileWalker<GATE>& cw, uint32_t ci) {
       Tile t;
       cw.get(t);
       const int c = ci % NSC;
@@ -605,7 +613,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const uint32_t t_acc = tmem_base + g * 128 + ((uint32_t)(q * 32) << 16);
       float a0[16], a1[16];
       if (t.has_coeff) {
-        if (p.pairing == 0) {
+        if (GATE || p.pairing == 0) {
           tmem_ld16(t_acc + 16 * cq, a0);             // channels 16cq .. 16cq+15
           tmem_ld16(t_acc + 64 + 16 * cq, a1);        // channels 64+16cq ..
         } else {
@@ -616,7 +624,30 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       }
       tc_fence_before();
       mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
-      if (work) {
+      if constexpr (GATE) {
+        // squared distance between the stored values and the anchor's reconstruction, this row and
+        // this warp's 32 channels; fp32 within the tile, float64 across tiles
+        if (in_range) {
+          const uint8_t* row0 = st_ptr + m * 128;
+          const uint8_t* row1 = row0 + kHalfBytes;
+          float sq = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj) {
+            const int j = 2 * cq + jj;
+            float x[16];
+            unpack8(*reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4)), x);
+            unpack8(*reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4)), x + 8);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const float d0 = x[k] - (covered ? a0[8 * jj + k] : 0.f);
+              const float d1 = x[8 + k] - (covered ? a1[8 * jj + k] : 0.f);
+              sq = fmaf(d0, d0, sq);
+              sq = fmaf(d1, d1, sq);
+            }
+          }
+          gate_acc += (double)sq;
+        }
+      } else if (work) {
         if (p.pairing == 0) {
           uint8_t* row0 = st_ptr + m * 128;
           uint8_t* row1 = row0 + kHalfBytes;
@@ -684,6 +715,11 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       fence_proxy_async();
       mbar_arrive(smem_u32(&ctrl->ready[s]));
     }
+    if constexpr (GATE) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) gate_acc += __shfl_xor_sync(0xffffffffu, gate_acc, o);
+      if (lane == 0 && gate_acc != 0.0) atomicAdd(p.gate_out, gate_acc);
+    }
   }
 
   // =============================================================== teardown
@@ -746,6 +782,20 @@ static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s, int grid = 
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
+template <int RB, int NSTAGE, int NSC>
+static cudaError_t launch_gate_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
+  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
+                          sizeof(Ctrl<NSTAGE, NSC>);
+  static bool set = false;
+  if (!set) {
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    set = true;
+  }
+  apply_tc_kernel<RB, NSTAGE, NSC, true><<<grid, kThreads, smem, s>>>(L);
+  return cudaGetLastError();
+}
+
 }  // namespace tc
 
 static_assert(offsetof(DevItem, cs) % 16 == 0 && offsetof(DevItem, sn) % 16 == 0, "rope tables must be 16-byte aligned");
@@ -777,6 +827,27 @@ constexpr int kMaxGrid = 1024;   // CTA boundaries of a ragged launch are tabula
 }
 // Extra workspace of a batch launch after the item table: tensor maps, then per rank class the CTA
 // boundaries, then the tile prefix of the second class.
+// Eq. 9 for one anchor: `item` describes the source cache (src = dst), the anchor's value factors as
+// its state, T = n_cov = k.  The squared distance is ADDED to *out (the caller clears it).
+int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, cudaStream_t s) {
+  if (!tc::item_supported(item, d) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  tc::ApplyTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.one = item;
+  L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
+  if (!tc::build_maps(L.one, &L.one_maps)) return KVC_E_CUDA;
+  L.n_items = 1;
+  L.total_tiles = (int64_t)item.L * item.H * L.one.tiles_per_slab;      // value slabs only
+  L.status = status;
+  L.gate_out = out;
+  if (L.total_tiles == 0) return KVC_OK;
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+  cudaError_t e = (item.st.r <= 32) ? tc::launch_gate_t<1, 5, 3>(L, grid, s) : tc::launch_gate_t<2, 4, 2>(L, grid, s);
+  return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
 size_t tc_batch_extra_bytes(int n_items) {
   return 256 + (size_t)n_items * sizeof(tc::ItemMaps) + 2 * 8 * (size_t)(tc::kMaxGrid + 1) + 8 * (size_t)(n_items + 1);
 }
