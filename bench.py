@@ -133,12 +133,17 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all"):
         tables = [None] * (2 * n)
         a0 = kvc.Cache(k0, v0)
     true = [a0]
-    if only == "apply":
-        # the chain alone: the generator's states are applied directly, no targets needed
+    if only in ("apply", "gate"):
+        # the chain (or the gate) alone: the generator's states are used directly, no targets needed
         states = []
         for a in range(1, n):
             s = wl.hop_state(cfg, a, dev)
             states.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
+        if only == "gate":
+            # the reliability gate over a pool whose anchors are the hop states' value factors
+            f64 = lambda m: torch.empty(m, dtype=torch.float64, device=dev)
+            return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": [], "ws": None, "only": only,
+                    "gate": (f64(n - 1), f64(n - 1), f64(1))}
         outs = [mk(tables[n + a]) for a in range(1, n)]
         return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": None, "only": only}
     for a in range(1, n):
@@ -251,6 +256,13 @@ def run_step(W, kvc, ev=None):
             kvc.kvc_apply_batch(items, rope, ws, stg)
         mark("chain_end")
         return
+    if only == "gate":
+        d2, g, ent = W["gate"]
+        mark("chain_begin")
+        kvc.kvc_gate_distance(W["true"][0], W["states"], W["true"][0].T, d2)
+        kvc.kvc_gate_weights(d2, g, ent)
+        mark("chain_end")
+        return
     if only != "apply":
         for a in range(1, n):
             mark("update_begin")
@@ -268,6 +280,9 @@ def step_bytes(W, kvc):
         return 0, W["apply_bytes"]
     n = len(W["states"]) + 1
     only = W.get("only", "all")
+    if only == "gate":      # per anchor: the source's values (2d B per token-slab) + value coefficients (4r) + basis
+        c = W["true"][0]
+        return 0, sum(c.L * c.H * (c.T * (2 * c.d + 4 * s.r) + 4 * s.r * c.d) for s in W["states"])
     upd = 0 if only == "apply" else sum(kvc.kvc_update_bytes(W["true"][0], W["states"][a - 1], kvc.KVC_FIT, True)
                                          for a in range(1, n))
     app = 0 if only == "update" else sum(kvc.kvc_apply_bytes(W["true"][0], W["states"][a - 1]) for a in range(1, n))
@@ -336,7 +351,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
     ap.add_argument("--rank", type=int, default=0, help="override the rank r (experiments)")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
-    ap.add_argument("--only", default="all", choices=["all", "apply", "update"],
+    ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate"],
                     help="profiling aid: time only the chain or only the state updates")
     args = ap.parse_args()
     rank, world, local = _dist()
@@ -474,16 +489,16 @@ def main():
     peak, peak_kind = _peaks()
     hop_ms = chain_ms / hops
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "gate distance (one anchor, Eq. 9)" if args.only == "gate" else "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0) else None,
+                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0 and args.only != "gate") else None,
                 "algorithmic_bytes_per_launch": app_b // hops,
                 "us_per_launch": hop_ms * 1e3}
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic", "config": config,
            "clocks": clocks, "e2e": e2e,
-           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
+           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (hops + 1 if args.only == "gate" else hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
            "roofline": roofline,
            "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
                          "us_per_agent_layer": hop_ms * 1e3 / cfg.L,

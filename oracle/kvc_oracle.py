@@ -460,6 +460,51 @@ def stack_anchors(weights, coeffs, bases):
     return c, b
 
 
+def token_weights(src_feat, anchor_feats, temperature=1.0):
+    """App. A.3 "Correction Weighting": token-wise interpolation weights.  For token t and anchor v the
+    score is the mean absolute difference between the source cache's features of t and the anchor's
+    reconstructed base features of t (mean over all layers, heads and channels); the weights are the
+    softmax over anchors of minus the score (T = 1).  Keys and values are weighted separately: call
+    once with key features (both sides in canonical positional coordinates) and once with value
+    features.  src_feat [T, F]; anchor_feats list over anchors of [T, F].  Returns [V, T]."""
+    x = np.asarray(src_feat, np.float64)
+    m = np.stack([np.mean(np.abs(x - np.asarray(a, np.float64)), axis=1) for a in anchor_feats])   # [V, T]
+    z = -m / temperature
+    z = z - np.max(z, axis=0, keepdims=True)
+    e = np.exp(z)
+    return e / np.sum(e, axis=0, keepdims=True)
+
+
+def canonical_key_features(bits_slabs, pos, inv_freq, pairing=ROPE_HALF):
+    """Keys of one cache in canonical positional coordinates: every (layer, head) slab [T, d] rotated
+    back by the cache's own position offset `pos`, slabs concatenated along the feature axis."""
+    return np.concatenate([rope_shift(bf16_to_f64(b) if b.dtype == np.uint16 else np.asarray(b, np.float64),
+                                      -pos, inv_freq, pairing) for b in bits_slabs], axis=1)
+
+
+def apply_multi_slab(src_bits, weights, coeffs, bases, n_covs, s, inv_freq, is_key, pairing=ROPE_HALF):
+    """Eq. 8 applied to one (layer, head) slab: C_hat[t] = Align_s(src[t]) + sum_v w_v[t] c_v[t] . B_v,
+    anchor v contributing on its covered rows t < n_cov_v.  weights [V, T] (None: all ones).
+    Returns (ref, out_bits) like apply_slab; rows no anchor covers keep the aligned source."""
+    x = bf16_to_f64(src_bits)
+    T = x.shape[0]
+    shift = s if is_key else 0
+    aligned = rope_shift(x, shift, inv_freq, pairing)
+    ref = np.array(aligned, dtype=np.float64, copy=True)
+    top = 0
+    for v, (c, b, n) in enumerate(zip(coeffs, bases, n_covs)):
+        n = min(int(n), T)
+        if n <= 0 or np.asarray(b).shape[0] == 0:
+            continue
+        w = np.ones(n) if weights is None else np.asarray(weights[v], np.float64)[:n]
+        ref[:n] += w[:, None] * (np.asarray(c[:n], np.float64) @ np.asarray(b, np.float64))
+        top = max(top, n)
+    out = f64_to_bf16_bits(ref)
+    if shift == 0:
+        out[top:] = src_bits[top:]
+    return ref, out
+
+
 # --------------------------------------------------------------------------
 # bookkeeping pinned by the paper's memory example (Sec. 3.1)
 # --------------------------------------------------------------------------

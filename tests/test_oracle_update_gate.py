@@ -220,3 +220,70 @@ def test_memory_example_from_the_paper():
     lr = orc.lowrank_state_bytes(V, N, tok, L, Hkv, hd, r=32)
     per_matrix = 32 * (tok + hd) * 4
     assert lr == V * (1 + N) * 2 * L * Hkv * per_matrix
+
+
+def test_token_weights_pins():
+    rng = np.random.default_rng(3)
+    T, F = 7, 12
+    x = rng.standard_normal((T, F))
+    # identical anchors: uniform weights; a single anchor: all ones
+    a = rng.standard_normal((T, F))
+    w = orc.token_weights(x, [a, a, a])
+    assert np.allclose(w, 1.0 / 3.0)
+    assert np.allclose(orc.token_weights(x, [a]), 1.0)
+    # columns sum to one; hand-computed two-anchor case: scores m0, m1 -> w0 = 1 / (1 + exp(m0 - m1))
+    b = rng.standard_normal((T, F))
+    w = orc.token_weights(x, [a, b])
+    assert np.allclose(w.sum(axis=0), 1.0)
+    m0 = np.abs(x - a).mean(axis=1)
+    m1 = np.abs(x - b).mean(axis=1)
+    assert np.allclose(w[0], 1.0 / (1.0 + np.exp(m0 - m1)))
+    # the anchor that equals the source on a token gets the larger weight there, and almost all of it
+    # when the other is far away
+    far = x + 100.0
+    near = x.copy()
+    w = orc.token_weights(x, [near, far])
+    assert np.all(w[0] > 1.0 - 1e-12)
+    # token-wise: swapping which anchor is near on the second half swaps the weights there
+    mix = np.where(np.arange(T)[:, None] < 3, near, far)
+    mix2 = np.where(np.arange(T)[:, None] < 3, far, near)
+    w = orc.token_weights(x, [mix, mix2])
+    assert np.all(w[0, :3] > 0.999) and np.all(w[1, 3:] > 0.999)
+    # a temperature rescales the scores: T -> infinity gives uniform weights
+    assert np.allclose(orc.token_weights(x, [a, b], temperature=1e12), 0.5, atol=1e-9)
+
+
+def test_apply_multi_slab_pins():
+    rng = np.random.default_rng(4)
+    T, d, r = 9, 8, 3
+    inv = orc.rope_inv_freq(d, 10000.0)
+    src = orc.f64_to_bf16_bits(rng.standard_normal((T, d)))
+    cs = [rng.standard_normal((T, r)) for _ in range(3)]
+    bs = [rng.standard_normal((r, d)) for _ in range(3)]
+    w = rng.random((3, T))
+    w /= w.sum(axis=0, keepdims=True)
+    for is_key, s in ((True, 5), (False, 5), (True, 0)):
+        ref, out = orc.apply_multi_slab(src, w, cs, bs, [T, T, T], s, inv, is_key)
+        # equals the single-state apply at the stacked rank (weights folded into the coefficients)
+        c_st, b_st = orc.stack_anchors(w, cs, bs)
+        ref1, out1 = orc.apply_slab(src, c_st, b_st, s, inv, T, is_key)
+        assert np.allclose(ref, ref1, rtol=0, atol=1e-12) and np.array_equal(out, out1)
+        # and the aligned source plus Eq. 8's estimate
+        base = orc.rope_shift(orc.bf16_to_f64(src), s if is_key else 0, inv)
+        assert np.allclose(ref, base + orc.multi_anchor_delta(w, cs, bs), atol=1e-12)
+    # one anchor, unit weights: the plain apply
+    ref, out = orc.apply_multi_slab(src, None, cs[:1], bs[:1], [T], 3, inv, True)
+    ref1, out1 = orc.apply_slab(src, cs[0], bs[0], 3, inv, T, True)
+    assert np.array_equal(ref, ref1) and np.array_equal(out, out1)
+    # partial coverage per anchor: rows beyond an anchor's length get nothing from it; rows beyond
+    # every anchor keep the source bits at shift 0
+    ref, out = orc.apply_multi_slab(src, w, cs, bs, [4, 6, 0], 0, inv, False)
+    x = orc.bf16_to_f64(src)
+    exp = x.copy()
+    exp[:4] += w[0, :4, None] * (cs[0][:4] @ bs[0])
+    exp[:6] += w[1, :6, None] * (cs[1][:6] @ bs[1])
+    assert np.allclose(ref, exp, atol=1e-12) and np.array_equal(out[6:], src[6:])
+    # canonical key features: rotating a cache forward by p and asking for canonical coordinates undoes it
+    k = rng.standard_normal((T, d))
+    moved = orc.rope_shift(k, 11, inv)
+    assert np.allclose(orc.canonical_key_features([moved], 11, inv), k, atol=1e-12)
