@@ -231,6 +231,31 @@ int kvc_apply_batch(const kvc_item *items, int32_t n_items, const kvc_rope *rope
 size_t kvc_batch_workspace_bytes(int32_t n_items);
 
 /*
+ * Multi-anchor apply (Eq. 8 with the token-wise weights of App. A.3 "Correction Weighting"):
+ *     K_dst[l,h,t,:] = bf16( Rot_shift(K_src[l,h,t,:]) + sum_v w_k[v][t] * coeff_k(v)[l,h,t,:] . basis_k(v)[l,h] )
+ *     V_dst[l,h,t,:] = bf16( V_src[l,h,t,:]            + sum_v w_v[v][t] * coeff_v(v)[l,h,t,:] . basis_v(v)[l,h] )
+ * anchor v contributing on its covered rows t < deltas[v].n_cov; rows no anchor covers keep the
+ * aligned source exactly as in kvc_apply.  This is kvc_apply at the stacked rank sum_v r_v with the
+ * weights folded into the coefficients, computed without building the stacked state.
+ *   deltas     host array [n_anchors] of the anchors' transition corrections (device factors);
+ *              anchors with r = 0 or n_cov = 0 contribute nothing
+ *   w_k, w_v   DEVICE float32 [n_anchors][t_pad], t_pad = KVC_MULTI_TPAD(src->T) (T rounded up to a
+ *              multiple of 128; the padding must hold finite numbers), 16-byte aligned; NULL = all ones
+ *   workspace  DEVICE, kvc_multi_workspace_bytes(...) bytes, 128-byte aligned: the bases rewritten as
+ *              tensor-core operands (rebuilt by every call)
+ * Limits: head_dim 128; every r_v a multiple of 4, at most 64; at most KVC_MULTI_MAX_BLOCKS rank
+ * blocks of 32 in total (sum over anchors of ceil(r_v / 32)), i.e. an effective rank of up to 320.
+ * Arguments outside these limits return KVC_E_UNSUPPORTED: this entry point has no CUDA-core variant.
+ * dst may be src itself (in place).  Precision as kvc_apply.
+ */
+#define KVC_MULTI_MAX_BLOCKS 10
+#define KVC_MULTI_TPAD(T) ((((int64_t)(T)) + 127) / 128 * 128)
+int kvc_apply_multi(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors, const float *w_k,
+                    const float *w_v, int32_t shift, const kvc_rope *rope, kvc_cache *dst, void *workspace,
+                    size_t workspace_bytes, void *stream);
+size_t kvc_multi_workspace_bytes(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors);
+
+/*
  * Reliability gate of the anchor pool (App. A.3 "Reliability Gate", Eqs. 9-11).
  *
  * kvc_gate_distance (Eq. 9): for every anchor v of a pool,

@@ -31,6 +31,7 @@ EXPORTS = (
     "kvc_apply", "kvc_chain", "kvc_state_update", "kvc_state_update_noalloc", "kvc_workspace_bytes", "kvc_apply_batch",
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
+    "kvc_apply_multi", "kvc_multi_workspace_bytes",
 )
 
 
@@ -85,6 +86,9 @@ def load(path: Optional[str] = None):
     lib.kvc_apply_batch.argtypes = [PI, i32, PR, vp, sz, vp, vp]
     lib.kvc_batch_workspace_bytes.argtypes = [i32]
     lib.kvc_batch_workspace_bytes.restype = sz
+    lib.kvc_apply_multi.argtypes = [PC, PS, i32, vp, vp, i32, PR, PC, vp, sz, vp]
+    lib.kvc_multi_workspace_bytes.argtypes = [PC, PS, i32]
+    lib.kvc_multi_workspace_bytes.restype = sz
     lib.kvc_gate_distance.argtypes = [PC, PS, i32, i32, vp, vp]
     lib.kvc_gate_weights.argtypes = [vp, i32, C.c_double, vp, vp, vp]
     lib.kvc_status_poll.argtypes = [C.POINTER(C.c_uint32)]
@@ -301,6 +305,38 @@ def kvc_apply_batch(items: Sequence[Item], rope: Rope, workspace: torch.Tensor, 
     _check(load().kvc_apply_batch(arr, n, C.byref(r), workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), staging.data_ptr(), _stream(stream)),
            "kvc_apply_batch")
+
+
+KVC_MULTI_MAX_BLOCKS = 10
+
+
+def kvc_multi_tpad(T: int) -> int:
+    return (int(T) + 127) // 128 * 128
+
+
+def _state_array(states: Sequence[State]):
+    arr = (kvc_state * max(len(states), 1))()
+    for i, a in enumerate(states):
+        arr[i] = a.struct()
+    return arr
+
+
+def kvc_multi_workspace_bytes(src: Cache, deltas: Sequence[State]) -> int:
+    c = src.struct()
+    return int(load().kvc_multi_workspace_bytes(C.byref(c), _state_array(deltas), len(deltas)))
+
+
+def kvc_apply_multi(src: Cache, deltas: Sequence[State], w_k: Optional[torch.Tensor], w_v: Optional[torch.Tensor],
+                    shift: int, rope: Rope, dst: Cache, workspace: torch.Tensor, stream=None) -> None:
+    """Eq. 8 with token-wise weights [n_anchors, kvc_multi_tpad(T)] fp32 (None: all ones)."""
+    cs, cd, r = src.struct(), dst.struct(), rope.struct()
+    for w in (w_k, w_v):
+        assert w is None or (w.dtype == torch.float32 and w.is_cuda and w.is_contiguous()
+                             and tuple(w.shape) == (len(deltas), kvc_multi_tpad(src.T)))
+    ptr = lambda t: 0 if t is None else t.data_ptr()
+    _check(load().kvc_apply_multi(C.byref(cs), _state_array(deltas), len(deltas), ptr(w_k), ptr(w_v), int(shift),
+                                  C.byref(r), C.byref(cd), workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_apply_multi")
 
 
 def kvc_gate_distance(src: Cache, anchors: Sequence[State], k: int, dist_sq: torch.Tensor, stream=None) -> None:

@@ -403,6 +403,48 @@ int kvc_apply_batch(const kvc_item* items, int32_t n_items, const kvc_rope* rope
   return KVC_OK;
 }
 
+static int multi_blocks(const kvc_state* deltas, int32_t n_anchors) {
+  int nb = 0;
+  for (int v = 0; v < n_anchors; ++v)
+    if (deltas[v].r > 0 && deltas[v].n_cov > 0) nb += (deltas[v].r + 31) / 32;
+  return nb;
+}
+
+size_t kvc_multi_workspace_bytes(const kvc_cache* src, const kvc_state* deltas, int32_t n_anchors) {
+  if (!src || !deltas || n_anchors <= 0) return 0;
+  return tc_multi_workspace_bytes(multi_blocks(deltas, n_anchors), src->L, src->H);
+}
+
+int kvc_apply_multi(const kvc_cache* src, const kvc_state* deltas, int32_t n_anchors, const float* w_k, const float* w_v,
+                    int32_t shift, const kvc_rope* rope, kvc_cache* dst, void* workspace, size_t workspace_bytes,
+                    void* stream) {
+  if (n_anchors < 0 || (n_anchors > 0 && !deltas)) return KVC_E_INVALID_ARG;
+  if (n_anchors > KVC_MULTI_MAX_BLOCKS) return KVC_E_UNSUPPORTED;
+  // geometry, aliasing and the rope tables are checked as for one hop with an empty state
+  kvc_state none;
+  memset(&none, 0, sizeof(none));
+  ResolvedHop hop;
+  int rc = resolve_hop(src, &none, shift, rope, dst, &hop);
+  if (rc != KVC_OK) return rc;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  DevState st[KVC_MULTI_MAX_BLOCKS];
+  int live = 0;
+  for (int v = 0; v < n_anchors; ++v) {
+    if ((rc = resolve_state(&deltas[v], 0, &st[v])) != KVC_OK) return rc;
+    if (deltas[v].r > 0 && deltas[v].n_cov > src->T) return KVC_E_SHAPE;
+    live += deltas[v].r > 0 && deltas[v].n_cov > 0;
+  }
+  if (live == 0) return apply_resolved(hop, rope->pairing, s);       // nothing to add: alignment only
+  if ((reinterpret_cast<uintptr_t>(w_k) | reinterpret_cast<uintptr_t>(w_v)) & 15) return KVC_E_INVALID_ARG;
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  if (src->T == 0) return KVC_OK;
+  rc = tc_apply_multi(hop.item.src, hop.item.dst, src->L, src->H, src->d, st, n_anchors, w_k, w_v, KVC_MULTI_TPAD(src->T),
+                      shift, hop.item.cs, hop.item.sn, rope->pairing, status, workspace, workspace_bytes, s);
+  if (rc == KVC_OK) tl_last_path = KVC_PATH_TC;
+  return rc;
+}
+
 int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_anchors, int32_t k, double* dist_sq,
                       void* stream) {
   if (!src || n_anchors < 0 || (n_anchors > 0 && (!anchors || !dist_sq)) || k < 0) return KVC_E_INVALID_ARG;

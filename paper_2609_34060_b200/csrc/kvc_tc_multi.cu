@@ -1,0 +1,653 @@
+// Multi-anchor apply (Eq. 8 with token-wise weights) on the Blackwell data path:
+//     C_hat[t] = Align_s(src[t]) + sum_v w_v[t] . c_v[t] . B_v ,
+// the sum running over the rank blocks (32 ranks each) of all anchors - up to 10 blocks, i.e. an
+// effective rank of 320 - without materialising a stacked state.
+//
+// Differences from the single-state kernel (kvc_tc_apply.cu), whose skeleton this one shares
+// (persistent CTAs, TMA tiles, tcgen05 MMAs into TMEM, 16-warp team, store warp):
+//   * a tile has a variable number of ring entries, one per rank block that covers it; an entry
+//     holds the fp32 coefficient block of its anchor (converted to bf16 hi/lo in place, scaled by
+//     the anchor's token weights on the way), the block's basis operand and the tile's 128 weights;
+//   * the basis operands are too many to stay resident per slab, so a preparation kernel writes
+//     them once, transposed and split, into a workspace from where TMA drops them into the ring
+//     (L2 traffic, no work for the team);
+//   * all rank blocks of a tile accumulate into one TMEM accumulator.
+// Every wait is bounded; on expiry the CTA records KVC_FLAG_WAIT_EXPIRED, drains and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <string.h>
+
+#include <cstddef>
+
+#include "../../include/kvc.h"
+#include "kvc_dev.cuh"
+#include "kvc_tc.h"
+#include "kvc_tc_ptx.cuh"
+#include "kvc_tc_maps.h"
+
+namespace kvc {
+namespace tcm {
+
+using namespace tc;
+
+constexpr int kTileTok = 128;
+constexpr int kThreads = 640;
+constexpr int kTeamThreads = 512;
+constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a base tile (bf16)
+constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
+constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
+constexpr int kOperandBytes = 128 * 128;          // 128 channels x (32 hi + 32 lo) bf16
+constexpr int kEntryBytes = kCoeffBytes + kOperandBytes;
+constexpr int kWeightBytes = kTileTok * 4;
+constexpr int NSTAGE = 3;                         // base-tile slots
+constexpr int NE = 3;                             // ring entries (rank blocks in flight)
+
+struct Block {                 // one rank block of one anchor
+  const float* w_k;            // token weights of the anchor [T_pad] (nullptr: all ones)
+  const float* w_v;
+  int32_t col0;                // first rank of the block inside the anchor's state
+  int32_t n_cov;               // rows the anchor covers
+  int32_t anchor;              // index of the anchor's coefficient maps
+  int32_t pad;
+};
+
+struct MultiLaunch {
+  DevCache src, dst;
+  int32_t shift, L, H, tps;    // tps = tiles per slab
+  int32_t pairing, n_blocks, cov_max, pad;
+  int64_t total_tiles;
+  uint32_t* status;
+  alignas(16) float cs[kMaxHalfD];
+  alignas(16) float sn[kMaxHalfD];
+  Block blk[KVC_MULTI_MAX_BLOCKS];
+  alignas(64) CUtensorMap src_k, src_v, dst_k, dst_v, operand;
+  CUtensorMap coeff_k[KVC_MULTI_MAX_BLOCKS], coeff_v[KVC_MULTI_MAX_BLOCKS];   // per anchor
+};
+
+struct Ctrl {
+  uint64_t full[NSTAGE], ready[NSTAGE], empty[NSTAGE];      // base-tile ring
+  uint64_t efull[NE], econv[NE], eempty[NE];                // entry ring
+  uint64_t mma_done[2], acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+               : "memory");
+}
+
+// A contiguous range of tiles; tile = (slab2 = 2 (l H + h) + is_v, tt).  Stepping is incremental.
+struct Walker {
+  int64_t remaining;
+  int slab2, tt, tps, H, l, h;
+  __device__ void init(const MultiLaunch& p, int64_t begin, int64_t end_) {
+    remaining = end_ - begin;
+    tps = p.tps;
+    H = p.H;
+    tt = (int)(begin % tps);
+    slab2 = (int)(begin / tps);
+    const int slab = slab2 >> 1;
+    l = slab / H;
+    h = slab - l * H;
+  }
+  __device__ bool done() const { return remaining <= 0; }
+  __device__ void next() {
+    --remaining;
+    if (++tt < tps) return;
+    tt = 0;
+    ++slab2;
+    if ((slab2 & 1) == 0 && ++h == H) {
+      h = 0;
+      ++l;
+    }
+  }
+  __device__ int t0() const { return tt * kTileTok; }
+  __device__ int is_v() const { return slab2 & 1; }
+  __device__ int slab() const { return slab2 >> 1; }
+};
+
+// Writes the basis operands: for block e, K|V, slab: 128 rows (channel) of [32 hi | 32 lo] bf16,
+// ranks col0 .. col0+31 of the anchor's basis (zero beyond its rank).
+struct PrepLaunch {
+  const void* basis_k[KVC_MULTI_MAX_BLOCKS];
+  const void* basis_v[KVC_MULTI_MAX_BLOCKS];
+  int32_t r[KVC_MULTI_MAX_BLOCKS], col0[KVC_MULTI_MAX_BLOCKS], bf16[KVC_MULTI_MAX_BLOCKS];
+  int32_t n_blocks, slabs;
+  __nv_bfloat16* out;
+};
+
+__global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
+  const int slab = blockIdx.x, kv = blockIdx.y, e = blockIdx.z;
+  const void* basis = kv ? p.basis_v[e] : p.basis_k[e];
+  const int r = p.r[e], col0 = p.col0[e];
+  __nv_bfloat16* out = p.out + (((int64_t)e * 2 + kv) * p.slabs + slab) * (128 * 64);
+  for (int i = threadIdx.x; i < 32 * 128; i += 256) {
+    const int q = i >> 7, ch = i & 127;           // coalesced reads along the channel
+    float x = 0.f;
+    if (col0 + q < r) {
+      const int64_t off = ((int64_t)slab * r + col0 + q) * 128 + ch;
+      x = p.bf16[e] ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
+                    : reinterpret_cast<const float*>(basis)[off];
+    }
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    out[ch * 64 + q] = hi;
+    out[ch * 64 + 32 + q] = __float2bfloat16_rn(x - __bfloat162float(hi));
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t stages = base;
+  constexpr int kEntryOff = NSTAGE * kBaseBytes;
+  constexpr int kWeightOff = kEntryOff + NE * kEntryBytes;
+  constexpr int kCtrlOff = kWeightOff + NE * kWeightBytes;
+  const uint32_t entries = base + kEntryOff;
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + kCtrlOff);
+  volatile int* abort_flag = &ctrl->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t n = p.total_tiles;
+  const int64_t tile_begin = n * blockIdx.x / gridDim.x;
+  const int64_t tile_end = n * (blockIdx.x + 1) / gridDim.x;
+
+  if (tid == 0) {
+    for (int s = 0; s < NSTAGE; ++s) {
+      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->ready[s]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int c = 0; c < NE; ++c) {
+      mbar_init(smem_u32(&ctrl->efull[c]), 1);
+      mbar_init(smem_u32(&ctrl->econv[c]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->eempty[c]), 1);
+    }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
+      mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
+    }
+    mbar_init(smem_u32(&ctrl->drain), 1);
+    ctrl->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctrl->tmem_base), 256);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+
+  // does block e take part in a tile that starts at token t0
+  auto active = [&](int e, int t0) { return t0 < p.blk[e].n_cov; };
+
+  if (warp == 0) {
+    // =============================================================== TMA producer (whole warp)
+    Walker w;
+    w.init(p, tile_begin, tile_end);
+    uint32_t i = 0, epos = 0;
+    bool alive = true;
+    for (; alive && !w.done(); w.next(), ++i) {
+      const int s = i % NSTAGE;
+      const int t0 = w.t0(), is_v = w.is_v(), l = w.l, h = w.h;
+      const bool paged = p.src.page_table != nullptr;
+      const int page = p.src.page_mask + 1;
+      int id = -1, n_pages = 0;
+      if (paged) {
+        const int per_tile = kTileTok >> p.src.page_shift;
+        const int first = t0 >> p.src.page_shift;
+        n_pages = min(per_tile, ((p.src.T + page - 1) >> p.src.page_shift) - first);
+        if (lane < n_pages) id = p.src.page_table[first + lane];
+      }
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), ((i / NSTAGE) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const uint32_t st_base = stages + s * kBaseBytes;
+      const uint32_t bar = smem_u32(&ctrl->full[s]);
+      const CUtensorMap* smap = is_v ? &p.src_v : &p.src_k;
+      if (!paged) {
+        if (lane == 0) {
+          mbar_expect_tx(bar, kBaseBytes);
+          tma_load_5d(st_base, smap, bar, 0, t0, h, 0, l);
+          tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t0, h, 0, l);
+        }
+      } else {
+        const bool valid = lane < n_pages && (unsigned)id < (unsigned)p.src.n_phys;
+        if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
+        const int n_ok = __popc(__ballot_sync(0xffffffffu, valid));
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_ok * page * 256));
+        __syncwarp();
+        if (valid) {
+          tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
+          tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
+        }
+      }
+      // the tile's rank blocks
+      for (int e = 0; e < p.n_blocks; ++e) {
+        if (!active(e, t0)) continue;
+        const int c = epos % NE;
+        if (lane == 0) {
+          ok = mbar_wait(smem_u32(&ctrl->eempty[c]), ((epos / NE) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+          if (ok) {
+            const Block& b = p.blk[e];
+            const float* wts = is_v ? b.w_v : b.w_k;
+            const uint32_t ebar = smem_u32(&ctrl->efull[c]);
+            mbar_expect_tx(ebar, (uint32_t)(kEntryBytes + (wts ? kWeightBytes : 0)));
+            const CUtensorMap* cmap = is_v ? &p.coeff_v[b.anchor] : &p.coeff_k[b.anchor];
+            tma_load_3d(entries + c * kEntryBytes, cmap, ebar, b.col0, t0, w.slab());
+            tma_load_2d(entries + c * kEntryBytes + kCoeffBytes, &p.operand, ebar, 0,
+                        ((e * 2 + is_v) * (p.L * p.H) + w.slab()) * 128);
+            if (wts) bulk_load_1d(base + kWeightOff + c * kWeightBytes, wts + t0, kWeightBytes, ebar);
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) {
+          alive = false;
+          break;
+        }
+        ++epos;
+      }
+      __syncwarp();
+    }
+    // drain: every load that was issued must have landed before the CTA may exit
+    if (lane == 0) {
+      for (uint32_t k = (i > NSTAGE ? i - NSTAGE : 0); k < i; ++k)
+        mbar_wait_drain(smem_u32(&ctrl->full[k % NSTAGE]), (k / NSTAGE) & 1u);
+      for (uint32_t k = (epos > NE ? epos - NE : 0); k < epos; ++k)
+        mbar_wait_drain(smem_u32(&ctrl->efull[k % NE]), (k / NE) & 1u);
+    }
+  } else if (warp == 1) {
+    // =============================================================== MMA issuer
+    if (lane == 0) {
+      Walker w;
+      w.init(p, tile_begin, tile_end);
+      uint32_t i = 0, epos = 0;
+      bool alive = true;
+      for (; alive && !w.done(); w.next(), ++i) {
+        const int g = i & 1;
+        const int t0 = w.t0();
+        if (!mbar_wait(smem_u32(&ctrl->acc_empty[g]), ((i >> 1) & 1u) ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + g * 128;
+        uint32_t acc = 0;
+        for (int e = 0; e < p.n_blocks; ++e) {
+          if (!active(e, t0)) continue;
+          const int c = epos % NE;
+          if (!mbar_wait(smem_u32(&ctrl->econv[c]), (epos / NE) & 1u, abort_flag)) {
+            alive = false;
+            break;
+          }
+          tc_fence_after();
+          const uint64_t ad = umma_desc_sw128(entries + c * kEntryBytes);
+          const uint64_t bd = umma_desc_sw128(entries + c * kEntryBytes + kCoeffBytes);
+          // byte offsets inside the 128-byte row: c1 | c2 for A, B1 | B2 for B; 16 bf16 = 32 B per k-step
+          const int aoff[6] = {0, 32, 64, 96, 0, 32};
+          const int boff[6] = {0, 32, 0, 32, 64, 96};
+#pragma unroll
+          for (int k = 0; k < 6; ++k) {
+            umma_bf16(d_tmem, ad + (uint64_t)(aoff[k] >> 4), bd + (uint64_t)(boff[k] >> 4), kIdescBf16M128N128, acc);
+            acc = 1;
+          }
+          umma_commit(smem_u32(&ctrl->eempty[c]));        // the entry may be refilled
+          ++epos;
+        }
+        if (!alive) break;
+        umma_commit(smem_u32(&ctrl->mma_done[g]));
+      }
+      umma_commit(smem_u32(&ctrl->drain));
+      mbar_wait_drain(smem_u32(&ctrl->drain), 0);
+    }
+  } else if (warp == 2) {
+    // spare warp: keeps the team's warps aligned with the TMEM lane quadrants (warp id & 3)
+  } else if (warp == 3) {
+    // =============================================================== store warp
+    Walker w;
+    w.init(p, tile_begin, tile_end);
+    uint32_t i = 0;
+    for (; !w.done(); w.next(), ++i) {
+      const int s = i % NSTAGE;
+      const int t0 = w.t0(), is_v = w.is_v(), l = w.l, h = w.h;
+      const bool dpaged = p.dst.page_table != nullptr;
+      const int dpage = p.dst.page_mask + 1;
+      int id = -1, n_pages = 0, first = 0;
+      bool src_ok = true;
+      if (dpaged) {
+        const int per_tile = kTileTok >> p.dst.page_shift;
+        first = t0 >> p.dst.page_shift;
+        n_pages = min(per_tile, ((p.dst.T + dpage - 1) >> p.dst.page_shift) - first);
+        if (lane < n_pages) {
+          id = p.dst.page_table[first + lane];
+          if (p.src.page_table) {
+            const int tk0 = t0 + lane * dpage;
+            const int tk1 = min(tk0 + dpage, p.src.T);
+            for (int sp = tk0 >> p.src.page_shift; (sp << p.src.page_shift) < tk1; ++sp)
+              if ((unsigned)p.src.page_table[sp] >= (unsigned)p.src.n_phys) src_ok = false;
+          }
+        }
+      }
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), (i / NSTAGE) & 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const CUtensorMap* dmap = is_v ? &p.dst_v : &p.dst_k;
+      const uint32_t st_base = stages + s * kBaseBytes;
+      uint8_t* st_ptr = smem + s * kBaseBytes;
+      if (!dpaged) {
+        if (lane == 0) {          // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
+          tma_store_5d(dmap, st_base, 0, t0, h, 0, l);
+          tma_store_5d(dmap, st_base + kHalfBytes, 64, t0, h, 0, l);
+        }
+      } else {
+        // the last, partial page goes out row by row so that rows >= T stay untouched; pages whose
+        // source could not be loaded are skipped
+        const int last_pg = (p.dst.T - 1) >> p.dst.page_shift;
+        const bool last_partial = (p.dst.T & p.dst.page_mask) != 0;
+        const bool valid = lane < n_pages && (unsigned)id < (unsigned)p.dst.n_phys;
+        if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
+        const bool partial = last_partial && (first + lane) == last_pg;
+        if (valid && src_ok && !partial) {
+          tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, h, id, l);
+          tma_store_5d(dmap, st_base + kHalfBytes + lane * dpage * 128, 64, 0, h, id, l);
+        }
+        const unsigned pm = __ballot_sync(0xffffffffu, valid && src_ok && partial);
+        if (pm) {
+          const int u = __ffs(pm) - 1;
+          const int rows = p.dst.T & p.dst.page_mask;
+          __nv_bfloat16* dbase = is_v ? p.dst.v : p.dst.k;
+          for (int c = lane; c < rows * 16; c += 32) {
+            const int row = u * dpage + (c >> 4), half = (c >> 3) & 1, j = c & 7;
+            __nv_bfloat16* drow = row_ptr(p.dst, dbase, l, h, t0 + row, p.status);
+            if (drow)
+              *reinterpret_cast<uint4*>(drow + half * 64 + j * 8) =
+                  *reinterpret_cast<const uint4*>(st_ptr + half * kHalfBytes + row * 128 + ((j ^ (row & 7)) << 4));
+          }
+        }
+      }
+      tma_store_commit();
+      tma_store_wait_read();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[s]));
+    }
+  } else {
+    // =============================================================== the team (16 warps)
+    const int e16 = warp - 4;
+    const int q = e16 & 3;                         // TMEM lane quadrant (== hardware warp id & 3)
+    const int cq = e16 >> 2;                       // channel quarter
+    const int m = q * 32 + lane;                   // epilogue row = token of the tile
+    const uint32_t sw = (uint32_t)(m & 7);
+    // conversion mapping: the four threads of a coefficient row sit in one warp
+    const int crow = e16 * 8 + (lane >> 2), cpart = lane & 3;
+    const uint32_t csw = (uint32_t)(crow & 7);
+
+    Walker w, wn;
+    w.init(p, tile_begin, tile_end);
+    wn = w;
+    uint32_t i = 0, epos = 0;
+    bool alive = true;
+
+    // converts all entries of the tile the walker points at: fp32 coefficients x token weight ->
+    // bf16 [c1 | c2] in place
+    auto convert_tile = [&](const Walker& cw) {
+      const int t0 = cw.t0(), is_v = cw.is_v();
+      for (int e = 0; e < p.n_blocks; ++e) {
+        if (!active(e, t0)) continue;
+        const int c = epos % NE;
+        bool ok = mbar_wait(smem_u32(&ctrl->efull[c]), (epos / NE) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return false;
+        const bool weighted = (is_v ? p.blk[e].w_v : p.blk[e].w_k) != nullptr;
+        const float wt = weighted ? reinterpret_cast<const float*>(smem + kWeightOff + c * kWeightBytes)[crow] : 1.f;
+        uint8_t* row = smem + kEntryOff + c * kEntryBytes + crow * 128;
+        // this thread's 8 coefficients: fp32 chunks 2*cpart, 2*cpart+1 of the row
+        float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
+        float4 f1 = *reinterpret_cast<const float4*>(row + (((2 * cpart + 1) ^ csw) << 4));
+        uint4 hi, lo;
+        split2(f0.x * wt, f0.y * wt, hi.x, lo.x);
+        split2(f0.z * wt, f0.w * wt, hi.y, lo.y);
+        split2(f1.x * wt, f1.y * wt, hi.z, lo.z);
+        split2(f1.z * wt, f1.w * wt, hi.w, lo.w);
+        __syncwarp();                               // all four threads of the row have read
+        *reinterpret_cast<uint4*>(row + ((cpart ^ csw) << 4)) = hi;         // c1: chunks 0..3
+        *reinterpret_cast<uint4*>(row + (((4 + cpart) ^ csw) << 4)) = lo;   // c2: chunks 4..7
+        fence_proxy_async();
+        mbar_arrive(smem_u32(&ctrl->econv[c]));
+        ++epos;
+      }
+      return true;
+    };
+
+    if (!w.done()) alive = convert_tile(wn);
+    for (; alive && !w.done(); w.next(), ++i) {
+      // ---- 1. get the next tile's rank blocks converted and their MMAs going
+      wn.next();
+      if (!wn.done()) {
+        if (!convert_tile(wn)) break;
+      }
+      const int s = i % NSTAGE, g = i & 1;
+      const int t0 = w.t0(), is_v = w.is_v();
+      uint8_t* st_ptr = smem + s * kBaseBytes;
+      const bool has_coeff = t0 < p.cov_max;
+
+      // ---- 2. accumulator of this tile ready, base tile landed
+      bool ok = mbar_wait(smem_u32(&ctrl->mma_done[g]), (i >> 1) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      ok = mbar_wait(smem_u32(&ctrl->full[s]), (i / NSTAGE) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+
+      // ---- 3. rotate, add, round: row m, this warp's channel quarter, in place
+      const int tok = t0 + m;
+      const bool in_range = tok < p.src.T;
+      const bool covered = has_coeff && tok < p.cov_max;
+      const bool rotate = !is_v && p.shift != 0;
+      const bool work = in_range && (covered || rotate);
+      const uint32_t t_acc = tmem_base + g * 128 + ((uint32_t)(q * 32) << 16);
+      float a0[16], a1[16];
+      if (has_coeff) {
+        if (p.pairing == 0) {
+          tmem_ld16(t_acc + 16 * cq, a0);             // channels 16cq .. 16cq+15
+          tmem_ld16(t_acc + 64 + 16 * cq, a1);        // channels 64+16cq ..
+        } else {
+          tmem_ld16(t_acc + 32 * cq, a0);             // channels 32cq .. 32cq+15
+          tmem_ld16(t_acc + 32 * cq + 16, a1);        // channels 32cq+16 ..
+        }
+        tmem_ld_wait();
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
+      if (work) {
+        if (p.pairing == 0) {
+          uint8_t* row0 = st_ptr + m * 128;
+          uint8_t* row1 = row0 + kHalfBytes;
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj) {
+            const int j = 2 * cq + jj;                 // chunk of 8 channels inside each half
+            uint4* p0 = reinterpret_cast<uint4*>(row0 + ((j ^ sw) << 4));
+            uint4* p1 = reinterpret_cast<uint4*>(row1 + ((j ^ sw) << 4));
+            float x[16];
+            unpack8(*p0, x);
+            unpack8(*p1, x + 8);
+            if (rotate) {
+              const float4 c0 = *reinterpret_cast<const float4*>(p.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(p.cs + 8 * j + 4);
+              const float4 s0 = *reinterpret_cast<const float4*>(p.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(p.sn + 8 * j + 4);
+              const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+              const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const float u = x[k], v = x[8 + k];
+                x[k] = u * cs[k] - v * sn[k];
+                x[8 + k] = u * sn[k] + v * cs[k];
+              }
+            }
+            if (covered) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                x[k] += a0[8 * jj + k];
+                x[8 + k] += a1[8 * jj + k];
+              }
+            }
+            *p0 = pack8(x);
+            *p1 = pack8(x + 8);
+          }
+        } else {
+          // interleaved pairs (2k, 2k+1): 32 consecutive channels 32cq .. 32cq+31
+          uint8_t* rowp = st_ptr + (cq >> 1) * kHalfBytes + m * 128;
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const int j = 4 * (cq & 1) + jj;           // chunk inside the half
+            uint4* pp = reinterpret_cast<uint4*>(rowp + ((j ^ sw) << 4));
+            float x[8];
+            unpack8(*pp, x);
+            if (rotate) {
+              const int f0 = 16 * cq + 4 * jj;         // pair index of the chunk's first pair
+              const float4 c0 = *reinterpret_cast<const float4*>(p.cs + f0);
+              const float4 s0 = *reinterpret_cast<const float4*>(p.sn + f0);
+              const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
+              const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float u = x[2 * k], v = x[2 * k + 1];
+                x[2 * k] = u * cs[k] - v * sn[k];
+                x[2 * k + 1] = u * sn[k] + v * cs[k];
+              }
+            }
+            if (covered) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) x[k] += (jj < 2) ? a0[8 * jj + k] : a1[8 * (jj - 2) + k];
+            }
+            *pp = pack8(x);
+          }
+        }
+      }
+      // ---- 4. the tile is final in shared memory: hand it to the store warp
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&ctrl->ready[s]));
+    }
+  }
+
+  // =============================================================== teardown
+  __syncthreads();
+  if (tid == 0 && *abort_flag) atomicOr(p.status, KVC_FLAG_WAIT_EXPIRED);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+static bool encode_operand(CUtensorMap* m, const __nv_bfloat16* ws, int64_t rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {64, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t es[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(ws), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace tcm
+
+static_assert(offsetof(tcm::MultiLaunch, cs) % 16 == 0 && offsetof(tcm::MultiLaunch, sn) % 16 == 0, "rope tables: float4 reads");
+static_assert(offsetof(tcm::MultiLaunch, src_k) % 64 == 0 && sizeof(CUtensorMap) % 64 == 0, "tensor maps need 64-byte alignment");
+static_assert(sizeof(tcm::MultiLaunch) <= 32000, "kernel parameter space");
+
+size_t tc_multi_workspace_bytes(int n_blocks, int L, int H) {
+  return (size_t)n_blocks * 2 * (size_t)L * H * tcm::kOperandBytes;
+}
+
+// anchors: resolved states (device pointers), weights [n_anchors][t_pad] or nullptr.
+int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d, const DevState* anchors, int n_anchors,
+                   const float* w_k, const float* w_v, int64_t t_pad, int shift, const float* cs, const float* sn, int pairing,
+                   uint32_t* status, void* workspace, size_t ws_bytes, cudaStream_t s) {
+  using namespace tcm;
+  if (d != 128 || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  for (const DevCache* c : {&src, &dst}) {
+    if (c->page_table && c->page_mask + 1 > 128) return KVC_E_UNSUPPORTED;
+    if (c->T >= (1 << 30)) return KVC_E_UNSUPPORTED;
+  }
+  MultiLaunch M;
+  memset(&M, 0, sizeof(M));
+  PrepLaunch P;
+  memset(&P, 0, sizeof(P));
+  int nb = 0, cov_max = 0;
+  if (n_anchors > KVC_MULTI_MAX_BLOCKS) return KVC_E_UNSUPPORTED;
+  for (int v = 0; v < n_anchors; ++v) {
+    const DevState& a = anchors[v];
+    if (a.r <= 0 || a.n_cov <= 0) continue;                     // an empty anchor contributes nothing
+    if (a.r > 64 || (a.r & 3)) return KVC_E_UNSUPPORTED;
+    if (!encode_coeff(&M.coeff_k[v], a.coeff_k, a.r, a.n_cov, L * H) ||
+        !encode_coeff(&M.coeff_v[v], a.coeff_v, a.r, a.n_cov, L * H))
+      return KVC_E_CUDA;
+    for (int col0 = 0; col0 < a.r; col0 += 32) {
+      if (nb == KVC_MULTI_MAX_BLOCKS) return KVC_E_UNSUPPORTED;
+      Block& b = M.blk[nb];
+      b.w_k = w_k ? w_k + (int64_t)v * t_pad : nullptr;
+      b.w_v = w_v ? w_v + (int64_t)v * t_pad : nullptr;
+      b.col0 = col0;
+      b.n_cov = a.n_cov;
+      b.anchor = v;
+      P.basis_k[nb] = a.basis_k;
+      P.basis_v[nb] = a.basis_v;
+      P.r[nb] = a.r;
+      P.col0[nb] = col0;
+      P.bf16[nb] = a.basis_bf16;
+      ++nb;
+    }
+    cov_max = a.n_cov > cov_max ? a.n_cov : cov_max;
+  }
+  if (nb == 0) return KVC_E_UNSUPPORTED;                       // nothing to add: the caller's plain path
+  const size_t need = tc_multi_workspace_bytes(nb, L, H);
+  if (!workspace || ws_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 127)) return KVC_E_WORKSPACE;
+  M.src = src;
+  M.dst = dst;
+  M.shift = shift;
+  M.L = L;
+  M.H = H;
+  M.tps = (src.T + kTileTok - 1) / kTileTok;
+  M.pairing = pairing;
+  M.n_blocks = nb;
+  M.cov_max = cov_max;
+  M.total_tiles = (int64_t)L * H * 2 * M.tps;
+  M.status = status;
+  memcpy(M.cs, cs, sizeof(M.cs));
+  memcpy(M.sn, sn, sizeof(M.sn));
+  if (M.total_tiles == 0) return KVC_OK;
+  __nv_bfloat16* ops = reinterpret_cast<__nv_bfloat16*>(workspace);
+  if (!encode_cache(&M.src_k, src, src.k, L, H) || !encode_cache(&M.src_v, src, src.v, L, H) ||
+      !encode_cache(&M.dst_k, dst, dst.k, L, H) || !encode_cache(&M.dst_v, dst, dst.v, L, H) ||
+      !encode_operand(&M.operand, ops, (int64_t)nb * 2 * L * H * 128))
+    return KVC_E_CUDA;
+  P.n_blocks = nb;
+  P.slabs = L * H;
+  P.out = ops;
+  multi_prep_kernel<<<dim3((unsigned)(L * H), 2, (unsigned)nb), 256, 0, s>>>(P);
+  if (cudaGetLastError() != cudaSuccess) return KVC_E_CUDA;
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(M.total_tiles < sms ? M.total_tiles : sms);
+  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NE * (kEntryBytes + kWeightBytes) + sizeof(Ctrl);
+  static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
+  static bool set = false;
+  if (!set) {
+    if (cudaFuncSetAttribute(apply_multi_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return KVC_E_CUDA;
+    set = true;
+  }
+  apply_multi_tc_kernel<<<grid, kThreads, smem, s>>>(M);
+  return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+}  // namespace kvc
