@@ -248,12 +248,37 @@ size_t kvc_batch_workspace_bytes(int32_t n_items);
  * Arguments outside these limits return KVC_E_UNSUPPORTED: this entry point has no CUDA-core variant.
  * dst may be src itself (in place).  Precision as kvc_apply.
  */
+#define KVC_MAX_ANCHORS 16
 #define KVC_MULTI_MAX_BLOCKS 10
 #define KVC_MULTI_TPAD(T) ((((int64_t)(T)) + 127) / 128 * 128)
 int kvc_apply_multi(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors, const float *w_k,
                     const float *w_v, int32_t shift, const kvc_rope *rope, kvc_cache *dst, void *workspace,
                     size_t workspace_bytes, void *stream);
 size_t kvc_multi_workspace_bytes(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors);
+
+/*
+ * Token-wise interpolation weights (App. A.3 "Correction Weighting and Positional Alignment"):
+ * for token t and anchor v the score is the mean over layers, heads and channels of
+ *     | C_src[l,h,t,c] - coeff(v)[l,h,t,:] . basis(v)[l,h][:,c] | ,
+ * the distance between the source cache and the base cache anchor v reconstructs from its
+ * low-rank factors; keys and values are scored separately, keys after both sides were rotated into
+ * canonical positional coordinates (the source back by src_pos, anchor v's reconstruction back by
+ * anchor_pos[v]).  The weights are the softmax over anchors of -score / temperature:
+ *     w_k[v][t], w_v[v][t] , DEVICE float32 [n_anchors][KVC_MULTI_TPAD(src->T)] ,
+ * the layout kvc_apply_multi consumes.  A token beyond anchor v's coverage (t >= anchors[v].n_cov)
+ * gets weight zero for v and the softmax runs over the anchors that cover it; the padding is zero.
+ *   anchors     host array [n_anchors] of the anchors' BASE factorisations (key and value factors)
+ *   anchor_pos  host int32 [n_anchors]
+ *   workspace   DEVICE, kvc_token_weights_workspace_bytes(src, n_anchors) bytes (the scores:
+ *               float32 [n_anchors][2][t_pad], left readable after the call)
+ * Limits: head_dim 128, 0 < r <= 64 and a multiple of 4, n_anchors <= KVC_MAX_ANCHORS, half-split RoPE
+ * pairing; otherwise KVC_E_UNSUPPORTED (no CUDA-core variant).  Scores are summed with float32
+ * atomics: their last bits depend on the order of the additions.
+ */
+int kvc_token_weights(const kvc_cache *src, int32_t src_pos, const kvc_state *anchors, const int32_t *anchor_pos,
+                      int32_t n_anchors, const kvc_rope *rope, double temperature, float *w_k, float *w_v,
+                      void *workspace, size_t workspace_bytes, void *stream);
+size_t kvc_token_weights_workspace_bytes(const kvc_cache *src, int32_t n_anchors);
 
 /*
  * Reliability gate of the anchor pool (App. A.3 "Reliability Gate", Eqs. 9-11).

@@ -31,7 +31,7 @@ EXPORTS = (
     "kvc_apply", "kvc_chain", "kvc_state_update", "kvc_state_update_noalloc", "kvc_workspace_bytes", "kvc_apply_batch",
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
-    "kvc_apply_multi", "kvc_multi_workspace_bytes",
+    "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
 )
 
 
@@ -89,6 +89,9 @@ def load(path: Optional[str] = None):
     lib.kvc_apply_multi.argtypes = [PC, PS, i32, vp, vp, i32, PR, PC, vp, sz, vp]
     lib.kvc_multi_workspace_bytes.argtypes = [PC, PS, i32]
     lib.kvc_multi_workspace_bytes.restype = sz
+    lib.kvc_token_weights.argtypes = [PC, i32, PS, C.POINTER(i32), i32, PR, C.c_double, vp, vp, vp, sz, vp]
+    lib.kvc_token_weights_workspace_bytes.argtypes = [PC, i32]
+    lib.kvc_token_weights_workspace_bytes.restype = sz
     lib.kvc_gate_distance.argtypes = [PC, PS, i32, i32, vp, vp]
     lib.kvc_gate_weights.argtypes = [vp, i32, C.c_double, vp, vp, vp]
     lib.kvc_status_poll.argtypes = [C.POINTER(C.c_uint32)]
@@ -337,6 +340,28 @@ def kvc_apply_multi(src: Cache, deltas: Sequence[State], w_k: Optional[torch.Ten
     _check(load().kvc_apply_multi(C.byref(cs), _state_array(deltas), len(deltas), ptr(w_k), ptr(w_v), int(shift),
                                   C.byref(r), C.byref(cd), workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_apply_multi")
+
+
+KVC_MAX_ANCHORS = 16
+
+
+def kvc_token_weights_workspace_bytes(src: Cache, n_anchors: int) -> int:
+    c = src.struct()
+    return int(load().kvc_token_weights_workspace_bytes(C.byref(c), int(n_anchors)))
+
+
+def kvc_token_weights(src: Cache, src_pos: int, anchors: Sequence[State], anchor_pos: Sequence[int], rope: Rope,
+                      w_k: torch.Tensor, w_v: torch.Tensor, workspace: torch.Tensor, temperature: float = 1.0,
+                      stream=None) -> None:
+    """App. A.3 token-wise weights [n_anchors, kvc_multi_tpad(T)] fp32 for keys and for values."""
+    n = len(anchors)
+    c, r = src.struct(), rope.struct()
+    pos = (C.c_int32 * max(n, 1))(*[int(x) for x in anchor_pos])
+    for w in (w_k, w_v):
+        assert w.dtype == torch.float32 and w.is_cuda and w.is_contiguous() and tuple(w.shape) == (n, kvc_multi_tpad(src.T))
+    _check(load().kvc_token_weights(C.byref(c), int(src_pos), _state_array(anchors), pos, n, C.byref(r), float(temperature),
+                                    w_k.data_ptr(), w_v.data_ptr(), workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_token_weights")
 
 
 def kvc_gate_distance(src: Cache, anchors: Sequence[State], k: int, dist_sq: torch.Tensor, stream=None) -> None:

@@ -445,6 +445,64 @@ int kvc_apply_multi(const kvc_cache* src, const kvc_state* deltas, int32_t n_anc
   return rc;
 }
 
+size_t kvc_token_weights_workspace_bytes(const kvc_cache* src, int32_t n_anchors) {
+  if (!src || n_anchors <= 0) return 0;
+  return (size_t)n_anchors * 2 * (size_t)KVC_MULTI_TPAD(src->T) * sizeof(float);
+}
+
+int kvc_token_weights(const kvc_cache* src, int32_t src_pos, const kvc_state* anchors, const int32_t* anchor_pos,
+                      int32_t n_anchors, const kvc_rope* rope, double temperature, float* w_k, float* w_v, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  if (!src || !anchors || !anchor_pos || n_anchors <= 0 || !w_k || !w_v || !(temperature > 0.0)) return KVC_E_INVALID_ARG;
+  if (n_anchors > KVC_MAX_ANCHORS) return KVC_E_UNSUPPORTED;
+  int rc;
+  if ((rc = check_rope(rope)) != KVC_OK) return rc;
+  if (rope->pairing != KVC_ROPE_HALF) return KVC_E_UNSUPPORTED;
+  DevCache dc;
+  if ((rc = resolve_cache(src, &dc)) != KVC_OK) return rc;
+  const int64_t t_pad = KVC_MULTI_TPAD(src->T);
+  const size_t need = kvc_token_weights_workspace_bytes(src, n_anchors);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 15)) return KVC_E_WORKSPACE;
+  DevState st[KVC_MAX_ANCHORS];
+  for (int v = 0; v < n_anchors; ++v) {
+    if ((rc = resolve_state(&anchors[v], 0, &st[v])) != KVC_OK) return rc;
+    if (anchors[v].r <= 0 || anchors[v].n_cov < 0 || anchors[v].n_cov > src->T) return KVC_E_SHAPE;
+  }
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  float* scores = reinterpret_cast<float*>(workspace);
+  if (cudaMemsetAsync(scores, 0, need, s) != cudaSuccess) return KVC_E_CUDA;
+  TokenWeightsLaunch q;
+  memset(&q, 0, sizeof(q));
+  for (int v = 0; v < n_anchors; ++v) {
+    q.n_cov[v] = anchors[v].n_cov;
+    if (anchors[v].n_cov == 0) continue;
+    DevItem it;
+    memset(&it, 0, sizeof(it));
+    it.src = dc;
+    it.src.T = anchors[v].n_cov;                    // rows the anchor can be compared on
+    it.dst = it.src;
+    it.st = st[v];
+    it.L = src->L;
+    it.H = src->H;
+    it.shift = -src_pos;
+    rope_tables(rope, src->d, -src_pos, it.cs, it.sn);
+    float cs2[kMaxHalfD], sn2[kMaxHalfD];
+    rope_tables(rope, src->d, -anchor_pos[v], cs2, sn2);
+    rc = tc_row_distance(it, src->d, cs2, sn2, status, scores + (size_t)v * 2 * t_pad, t_pad, s);
+    if (rc != KVC_OK) return rc;
+  }
+  q.w_k = w_k;
+  q.w_v = w_v;
+  q.t_pad = t_pad;
+  q.inv_temp = (float)(1.0 / temperature);
+  q.n = n_anchors;
+  if (launch_token_weights(scores, q, s) != cudaSuccess) return KVC_E_CUDA;
+  tl_last_path = KVC_PATH_TC;
+  return KVC_OK;
+}
+
 int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_anchors, int32_t k, double* dist_sq,
                       void* stream) {
   if (!src || n_anchors < 0 || (n_anchors > 0 && (!anchors || !dist_sq)) || k < 0) return KVC_E_INVALID_ARG;

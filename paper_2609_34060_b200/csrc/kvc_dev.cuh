@@ -81,6 +81,15 @@ struct GateLaunch {            // Eq. 9 for one anchor, CUDA-core kernel
   uint32_t* status;
 };
 
+struct TokenWeightsLaunch {    // softmax over anchors per token
+  float* w_k;
+  float* w_v;
+  int64_t t_pad;
+  float inv_temp;
+  int32_t n;
+  int32_t n_cov[16];
+};
+
 // Address of row (l, h, t) of a cache; returns nullptr (and flags) on a bad page id.
 __device__ __forceinline__ __nv_bfloat16* row_ptr(const DevCache& c, __nv_bfloat16* base, int l, int h, int t,
                                                    uint32_t* status) {

@@ -85,4 +85,32 @@ cudaError_t launch_gate_weights(const double* dist_sq, int n, double temperature
   return cudaGetLastError();
 }
 
+// Token-wise interpolation weights (App. A.3): per token the softmax over the anchors that cover it
+// of minus its score (mean absolute distance), keys and values separately.  scores [n][2][t_pad],
+// w_k / w_v [n][t_pad]; tokens beyond an anchor's coverage, and the padding, get weight zero.
+__global__ void __launch_bounds__(256) token_weights_kernel(const float* scores, TokenWeightsLaunch q) {
+  const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (t >= q.t_pad) return;
+  for (int kv = 0; kv < 2; ++kv) {
+    float* w = kv ? q.w_v : q.w_k;
+    float zmax = -3.0e38f;
+    for (int v = 0; v < q.n; ++v)
+      if (t < q.n_cov[v]) zmax = fmaxf(zmax, -scores[((int64_t)v * 2 + kv) * q.t_pad + t] * q.inv_temp);
+    float sum = 0.f;
+    for (int v = 0; v < q.n; ++v)
+      if (t < q.n_cov[v]) sum += expf(-scores[((int64_t)v * 2 + kv) * q.t_pad + t] * q.inv_temp - zmax);
+    for (int v = 0; v < q.n; ++v) {
+      float x = 0.f;
+      if (t < q.n_cov[v]) x = expf(-scores[((int64_t)v * 2 + kv) * q.t_pad + t] * q.inv_temp - zmax) / sum;
+      w[(int64_t)v * q.t_pad + t] = x;
+    }
+  }
+}
+
+cudaError_t launch_token_weights(const float* scores, const TokenWeightsLaunch& q, cudaStream_t s) {
+  if (q.t_pad <= 0) return cudaSuccess;
+  token_weights_kernel<<<(unsigned)((q.t_pad + 255) / 256), 256, 0, s>>>(scores, q);
+  return cudaGetLastError();
+}
+
 }  // namespace kvc

@@ -12,6 +12,8 @@ namespace kvc {
 
 int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s);
 int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, cudaStream_t s);
+int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* sn2, uint32_t* status, float* row_out,
+                    int64_t t_pad, cudaStream_t s);
 int tc_apply_batch(DevItem* tab_host, int64_t* prefix_host, int n_items, int d, int pairing, uint32_t* status,
                    void* workspace_dev, void* staging_host, size_t bytes, cudaStream_t s);
 size_t tc_batch_extra_bytes(int n_items);

@@ -59,6 +59,12 @@ struct ApplyTcLaunch {
   int64_t total_tiles;
   uint32_t* status;
   double* gate_out;            // gate-distance mode: the squared distance is added here
+  float* row_out;              // row-distance mode: [2][t_pad] sums of |src - reconstruction| per token (K, V)
+  int64_t row_pad;             // t_pad
+  float row_scale;             // 1 / (L H d): the sums become means
+  int32_t pad2;
+  alignas(16) float cs2[kMaxHalfD];   // row-distance mode: rotation of the RECONSTRUCTED keys (the item's own
+  alignas(16) float sn2[kMaxHalfD];   // table rotates the source keys): both sides in canonical coordinates
   DevItem one;
   ItemMaps one_maps;
 };
@@ -223,10 +229,16 @@ __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_
 // Two rings of shared-memory slots: NSTAGE base tiles (alive from the load until the TMA store has
 // read them) and NSC coefficient tiles (alive only until the tile's MMAs have completed), so that
 // the short-lived operand does not hold a long-lived slot.
-// GATE: gate-distance mode (Eq. 9): value slabs only, nothing is stored; the team accumulates
-// sum (V - c.B)^2 over its rows and the CTA adds its part to *gate_out.
-template <int RB, int NSTAGE, int NSC, bool GATE = false>
+// MODE 0: apply.  Modes 1 and 2 store nothing and reduce instead:
+// MODE 1, gate distance (Eq. 9): value slabs only; the team accumulates sum (V - c.B)^2 over its rows
+//         and the CTA adds its part to *gate_out.
+// MODE 2, row distance (token weights of App. A.3): key and value slabs; per token the mean of
+//         |src - c.B| over layers, heads and channels is accumulated in row_out, keys after both
+//         sides were rotated into canonical positional coordinates.
+template <int RB, int NSTAGE, int NSC, int MODE = 0>
 __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
+  constexpr bool GATE = MODE == 1;                // walks value slabs only
+  constexpr bool REDUCE = MODE != 0;              // no stores
   constexpr int kStageBytes = kBaseBytes;
   constexpr int kCoeffSlotBytes = RB * kCoeffBlkBytes;
   constexpr int kBasisSlotBytes = RB * kBasisBlkBytes;
@@ -457,7 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const CUtensorMap* dmap = t.is_v ? &t.mp->dst_v : &t.mp->dst_k;
       const uint32_t st_base = stages + s * kStageBytes;
       uint8_t* st_ptr = smem + s * kStageBytes;
-      if constexpr (GATE) {
+      if constexpr (REDUCE) {
         // nothing to store: the slot goes straight back to the producer
       } else if (!dpaged) {
         if (lane == 0) {          // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
@@ -613,7 +625,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const uint32_t t_acc = tmem_base + g * 128 + ((uint32_t)(q * 32) << 16);
       float a0[16], a1[16];
       if (t.has_coeff) {
-        if (GATE || p.pairing == 0) {
+        if (REDUCE || p.pairing == 0) {
           tmem_ld16(t_acc + 16 * cq, a0);             // channels 16cq .. 16cq+15
           tmem_ld16(t_acc + 64 + 16 * cq, a1);        // channels 64+16cq ..
         } else {
@@ -646,6 +658,34 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             }
           }
           gate_acc += (double)sq;
+        }
+      } else if constexpr (MODE == 2) {
+        // mean absolute distance between the source row and the anchor's reconstruction of it, this
+        // warp's 32 channels (pairs (c, c + 64) sit in one thread): keys are compared after rotating
+        // the source by the item's table and the reconstruction by the second table
+        if (in_range && covered) {
+          const uint8_t* row0 = st_ptr + m * 128;
+          const uint8_t* row1 = row0 + kHalfBytes;
+          float sa = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj) {
+            const int j = 2 * cq + jj;
+            float x[16];
+            unpack8(*reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4)), x);
+            unpack8(*reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4)), x + 8);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              float u = x[k], v = x[8 + k], au = a0[8 * jj + k], av = a1[8 * jj + k];
+              if (!t.is_v) {
+                const float c1 = it.cs[8 * j + k], s1 = it.sn[8 * j + k], c2 = p.cs2[8 * j + k], s2 = p.sn2[8 * j + k];
+                const float ru = u * c1 - v * s1, rv = u * s1 + v * c1;
+                const float bu = au * c2 - av * s2, bv = au * s2 + av * c2;
+                u = ru, v = rv, au = bu, av = bv;
+              }
+              sa += fabsf(u - au) + fabsf(v - av);
+            }
+          }
+          atomicAdd(p.row_out + (int64_t)t.is_v * p.row_pad + tok, sa * p.row_scale);
         }
       } else if (work) {
         if (p.pairing == 0) {
@@ -782,17 +822,17 @@ static int launch(const ApplyTcLaunch& L, int max_r, cudaStream_t s, int grid = 
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
-template <int RB, int NSTAGE, int NSC>
-static cudaError_t launch_gate_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
+template <int RB, int NSTAGE, int NSC, int MODE>
+static cudaError_t launch_reduce_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
                           sizeof(Ctrl<NSTAGE, NSC>);
   static bool set = false;
   if (!set) {
-    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     set = true;
   }
-  apply_tc_kernel<RB, NSTAGE, NSC, true><<<grid, kThreads, smem, s>>>(L);
+  apply_tc_kernel<RB, NSTAGE, NSC, MODE><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError();
 }
 
@@ -844,7 +884,35 @@ int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, 
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
-  cudaError_t e = (item.st.r <= 32) ? tc::launch_gate_t<1, 5, 3>(L, grid, s) : tc::launch_gate_t<2, 4, 2>(L, grid, s);
+  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 5, 3, 1>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 1>(L, grid, s);
+  return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+// Token-weight scores of one anchor (App. A.3): `item` describes the source cache (src = dst, its
+// rope table rotates the source keys into canonical coordinates), the anchor's base factors as its
+// state (T = n_cov of the anchor); cs2 / sn2 rotate the reconstructed keys.  Per-token means are
+// ADDED to row_out[2][t_pad] (the caller clears it).
+int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* sn2, uint32_t* status, float* row_out,
+                    int64_t t_pad, cudaStream_t s) {
+  if (!tc::item_supported(item, d) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  tc::ApplyTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.one = item;
+  L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
+  if (!tc::build_maps(L.one, &L.one_maps)) return KVC_E_CUDA;
+  L.n_items = 1;
+  L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
+  L.status = status;
+  L.row_out = row_out;
+  L.row_pad = t_pad;
+  L.row_scale = 1.f / ((float)item.L * (float)item.H * (float)d);
+  memcpy(L.cs2, cs2, sizeof(L.cs2));
+  memcpy(L.sn2, sn2, sizeof(L.sn2));
+  if (L.total_tiles == 0) return KVC_OK;
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 5, 3, 2>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 2>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

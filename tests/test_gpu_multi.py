@@ -160,3 +160,118 @@ def test_apply_multi_limits_and_empty():
         kvc.kvc_apply(src, kvc.State.empty(), 19, rope, ref)
         torch.cuda.synchronize()
         assert torch.equal(dst.k, ref.k) and torch.equal(dst.v, ref.v)
+
+
+def _oracle_token_weights(cfg, osrc, src_pos, anchors, anchor_pos, temperature=1.0):
+    """App. A.3 with the oracle: features of a token = all (layer, head) slabs side by side; keys in
+    canonical coordinates on both sides."""
+    inv = hp.inv_freq(cfg)
+    slabs = [(l, h) for l in range(cfg.L) for h in range(cfg.H)]
+    out = {}
+    for which in ("k", "v"):
+        if which == "k":
+            src_feat = orc.canonical_key_features([osrc.get_bits("k", l, h) for l, h in slabs], src_pos, inv)
+        else:
+            src_feat = np.concatenate([orc.bf16_to_f64(osrc.get_bits("v", l, h)) for l, h in slabs], axis=1)
+        w = np.zeros((len(anchors), cfg.T))
+        # the softmax runs over the anchors that cover a token: group tokens by the set of covering anchors
+        covs = sorted({a.n_cov for a in anchors} | {0, cfg.T})
+        for lo, hi in zip(covs[:-1], covs[1:]):
+            idx = [v for v, a in enumerate(anchors) if a.n_cov >= hi]
+            if not idx or hi <= lo:
+                continue
+            feats = []
+            for v in idx:
+                a = anchors[v]
+                c = getattr(a, "coeff_" + which).numpy().astype(np.float64)
+                b = getattr(a, "basis_" + which).to(torch.float32).numpy().astype(np.float64)
+                rec = [c[l, h, lo:hi] @ b[l, h] for l, h in slabs]
+                if which == "k":
+                    rec = [orc.rope_shift(x, -anchor_pos[v], inv) for x in rec]
+                feats.append(np.concatenate(rec, axis=1))
+            w[idx, lo:hi] = orc.token_weights(src_feat[lo:hi], feats, temperature)
+        out[which] = w
+    return out["k"], out["v"]
+
+
+@pytest.mark.parametrize("cfg", [CFG_S, CFG_P], ids=lambda c: c.name)
+def test_token_weights_match_the_oracle(cfg):
+    T = cfg.T
+    ranks, covs = (32, 32, 64), (T, T, T - 300)
+    anchors = _anchors(cfg, ranks, covs)
+    anchor_pos = [100, 37, 412]
+    src_pos = 250
+    # the source cache sits close to anchor 0's base on the first half of the tokens and close to
+    # anchor 1's on the second half (oracle arithmetic on generator draws), keys moved to the
+    # source's positions
+    src_cpu = hp.make_cache(cfg)
+    osrc = hp.oracle_cache(src_cpu)
+    inv = hp.inv_freq(cfg)
+    eps = wl.noise((2, cfg.L, cfg.H, T, cfg.d), cfg.seed, 91, "cpu").numpy().astype(np.float64)
+    half = T // 2
+    for l in range(cfg.L):
+        for h in range(cfg.H):
+            for wi, which in enumerate(("k", "v")):
+                rec = []
+                for v in (0, 1):
+                    c = getattr(anchors[v], "coeff_" + which)[l, h].numpy().astype(np.float64)
+                    b = getattr(anchors[v], "basis_" + which)[l, h].numpy().astype(np.float64)
+                    x = c @ b
+                    if which == "k":
+                        x = orc.rope_shift(x, src_pos - anchor_pos[v], inv)
+                    rec.append(x)
+                mix = np.where(np.arange(T)[:, None] < half, rec[0], rec[1]) + 0.3 * eps[wi, l, h]
+                osrc.put_bits(which, l, h, orc.f64_to_bf16_bits(mix))
+    mk = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16)
+    src_cpu = kvc.Cache(mk(osrc.k), mk(osrc.v)) if src_cpu.page_table is None else \
+        kvc.Cache(mk(osrc.k), mk(osrc.v), T=T, page_table=src_cpu.page_table)
+    src = hp.to_dev(src_cpu, DEV)
+    dev_anchors = [hp.state_to_dev(a, DEV) for a in anchors]
+    tp = kvc.kvc_multi_tpad(T)
+    wk = torch.full((3, tp), -1.0, device=DEV)
+    wv = torch.full((3, tp), -1.0, device=DEV)
+    ws = torch.empty(kvc.kvc_token_weights_workspace_bytes(src, 3), dtype=torch.uint8, device=DEV)
+    for temp in (1.0, 0.25):
+        kvc.kvc_token_weights(src, src_pos, dev_anchors, anchor_pos, kvc.Rope(cfg.theta), wk, wv, ws, temperature=temp)
+        torch.cuda.synchronize()
+        rk, rv = _oracle_token_weights(cfg, osrc, src_pos, anchors, anchor_pos, temp)
+        gk, gv = wk.cpu().numpy().astype(np.float64), wv.cpu().numpy().astype(np.float64)
+        # scores are float32 means of ~L*H*d terms with split-precision products: 1e-5 absolute on a weight
+        assert np.max(np.abs(gk[:, :T] - rk)) <= 2e-5 and np.max(np.abs(gv[:, :T] - rv)) <= 2e-5
+        assert np.all(gk[:, T:] == 0) and np.all(gv[:, T:] == 0)               # the padding
+        assert np.all(gk[2, T - 300:T] == 0) and np.all(gv[2, T - 300:T] == 0)   # beyond anchor 2's coverage
+        assert np.allclose(gk[:, :T].sum(axis=0), 1.0, atol=1e-5)
+    # the scenario is token-wise: the first half prefers anchor 0, the second half anchor 1
+    assert rk[0, :half].mean() > 0.5 > rk[0, half:].mean() and rv[1, half:].mean() > 0.5 > rv[1, :half].mean()
+
+
+def test_multi_anchor_pipeline_gate_weights_apply():
+    """Gate, token weights and weighted apply chained on the device against the same chain in the oracle."""
+    cfg = CFG_S.scaled(T=640)
+    T = cfg.T
+    base = _anchors(cfg, (32, 32), (T, T))                       # the anchors' base factorisations
+    delta = [hp.make_state(cfg, hop=v + 5, r=32) for v in range(2)]   # their stored corrections
+    src_cpu = hp.make_cache(cfg)
+    osrc = hp.oracle_cache(src_cpu)
+    src = hp.to_dev(src_cpu, DEV)
+    dev_base = [hp.state_to_dev(a, DEV) for a in base]
+    dev_delta = [hp.state_to_dev(a, DEV) for a in delta]
+    rope = kvc.Rope(cfg.theta)
+    d2 = torch.empty(2, dtype=torch.float64, device=DEV)
+    g = torch.empty(2, dtype=torch.float64, device=DEV)
+    ent = torch.empty(1, dtype=torch.float64, device=DEV)
+    kvc.kvc_gate_distance(src, dev_base, T, d2)
+    kvc.kvc_gate_weights(d2, g, ent)
+    tp = kvc.kvc_multi_tpad(T)
+    wk, wv = torch.empty(2, tp, device=DEV), torch.empty(2, tp, device=DEV)
+    ws = torch.empty(kvc.kvc_token_weights_workspace_bytes(src, 2), dtype=torch.uint8, device=DEV)
+    kvc.kvc_token_weights(src, 0, dev_base, [0, 0], rope, wk, wv, ws)
+    dst = hp.empty_dst(src_cpu, cfg, DEV)
+    ws2 = torch.empty(kvc.kvc_multi_workspace_bytes(src, dev_delta), dtype=torch.uint8, device=DEV)
+    kvc.kvc_apply_multi(src, dev_delta, wk, wv, 48, rope, dst, ws2)
+    torch.cuda.synchronize()
+    assert 0.0 <= ent.item() <= 1.0 + 1e-12
+    ok_, ov_ = _oracle_token_weights(cfg, osrc, 0, base, [0, 0])
+    pad = lambda w: torch.from_numpy(np.pad(w, ((0, 0), (0, tp - T))).astype(np.float32))
+    odst, rk, rv = _oracle(cfg, src_cpu, delta, pad(ok_), pad(ov_), 48)
+    _check(dst, odst, rk, rv)
