@@ -133,7 +133,7 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all"):
         tables = [None] * (2 * n)
         a0 = kvc.Cache(k0, v0)
     true = [a0]
-    if only in ("apply", "gate", "multi"):
+    if only in ("apply", "gate", "multi", "weights"):
         # the chain (or the gate) alone: the generator's states are used directly, no targets needed
         states = []
         for a in range(1, n):
@@ -144,6 +144,12 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all"):
             f64 = lambda m: torch.empty(m, dtype=torch.float64, device=dev)
             return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": [], "ws": None, "only": only,
                     "gate": (f64(n - 1), f64(n - 1), f64(1))}
+        if only == "weights":
+            # App. A.3 token-wise weights: the hop states act as the base factorisations of n - 1 anchors
+            tp = kvc.kvc_multi_tpad(cfg.T)
+            w = [torch.empty(n - 1, tp, device=dev) for _ in range(2)]
+            ws = torch.empty(kvc.kvc_token_weights_workspace_bytes(a0, n - 1), dtype=torch.uint8, device=dev)
+            return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": [], "ws": ws, "only": only, "w": w}
         if only == "multi":
             # Eq. 8: the hop states act as the corrections stored in n - 1 anchors, with seeded token-wise weights
             tp = kvc.kvc_multi_tpad(cfg.T)
@@ -273,6 +279,11 @@ def run_step(W, kvc, ev=None):
         kvc.kvc_gate_weights(d2, g, ent)
         mark("chain_end")
         return
+    if only == "weights":
+        mark("chain_begin")
+        kvc.kvc_token_weights(W["true"][0], pl[0], W["states"], pl[1:], rope, W["w"][0], W["w"][1], W["ws"])
+        mark("chain_end")
+        return
     if only == "multi":
         mark("chain_begin")
         kvc.kvc_apply_multi(W["true"][0], W["states"], W["w"][0], W["w"][1], pl[1] - pl[0], rope, W["outs"][0], W["ws"])
@@ -298,6 +309,9 @@ def step_bytes(W, kvc):
     if only == "gate":      # per anchor: the source's values (2d B per token-slab) + value coefficients (4r) + basis
         c = W["true"][0]
         return 0, sum(c.L * c.H * (c.T * (2 * c.d + 4 * s.r) + 4 * s.r * c.d) for s in W["states"])
+    if only == "weights":   # per anchor: the source cache (4d B per token-slab) + key and value coefficients (8r) + bases
+        c = W["true"][0]
+        return 0, sum(c.L * c.H * (c.T * (4 * c.d + 8 * s.r) + 8 * s.r * c.d) for s in W["states"])
     if only == "multi":     # caches in and out (4d + 4d), every anchor's coefficients (8r) and weights (8 B per token)
         c = W["true"][0]
         return 0, c.L * c.H * c.T * (8 * c.d + sum(8 * s.r for s in W["states"])) + 8 * len(W["states"]) * c.T \
@@ -370,7 +384,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
     ap.add_argument("--rank", type=int, default=0, help="override the rank r (experiments)")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
-    ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi"],
+    ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi", "weights"],
                     help="profiling aid: time only the chain or only the state updates")
     args = ap.parse_args()
     rank, world, local = _dist()
@@ -508,16 +522,16 @@ def main():
     peak, peak_kind = _peaks()
     hop_ms = chain_ms / hops
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "gate distance (one anchor, Eq. 9)" if args.only == "gate" else "multi-anchor apply (Eq. 8)" if args.only == "multi" else "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "gate distance (one anchor, Eq. 9)" if args.only == "gate" else "multi-anchor apply (Eq. 8)" if args.only == "multi" else "token-weight scores (one anchor, App. A.3)" if args.only == "weights" else "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0 and args.only not in ("gate", "multi")) else None,
+                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0 and args.only not in ("gate", "multi", "weights")) else None,
                 "algorithmic_bytes_per_launch": app_b // hops,
                 "us_per_launch": hop_ms * 1e3}
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic", "config": config,
            "clocks": clocks, "e2e": e2e,
-           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (hops + 1 if args.only in ("gate", "multi") else hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
+           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (hops + 1 if args.only in ("gate", "multi", "weights") else hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
            "roofline": roofline,
            "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
                          "us_per_agent_layer": hop_ms * 1e3 / cfg.L,
