@@ -160,3 +160,29 @@ def test_gate_end_to_end_accepts_the_matching_anchor():
     # distances differ by tens of units here, so the weights are one-hot on both sides
     assert int(torch.argmax(g).item()) == int(np.argmax(ref_g)) == 0
     assert g[0].item() > 1.0 - 1e-9 and ent.item() < 1e-6 and orc.normalized_entropy(ref_g) < 1e-6
+
+
+def test_base_factorisation_then_gate_is_the_truncation_residual():
+    """An anchor's base cache factorised by itself (src = NULL, FIT) and compared with itself: the
+    squared gate distance is what a rank-r truncation leaves, sum over value slabs of the
+    eigenvalues of V^T V beyond the r-th (Eckart-Young), computed here by a library eigensolver."""
+    cfg = CFG_8B_S.scaled(L=1, H=2, T=400)
+    r = 32
+    cache_cpu = hp.make_cache(cfg)
+    cache = hp.to_dev(cache_cpu, DEV)
+    L, H, T, d = cfg.L, cfg.H, cfg.T, cfg.d
+    st = kvc.State(torch.empty(L, H, T, r, device=DEV), torch.empty(L, H, T, r, device=DEV),
+                   torch.empty(L, H, r, d, device=DEV), torch.empty(L, H, r, d, device=DEV))
+    ws = torch.empty(kvc.kvc_workspace_bytes(cache, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(None, cache, 0, kvc.Rope(cfg.theta), st, kvc.KVC_FIT, workspace=ws)
+    d2 = torch.empty(1, dtype=torch.float64, device=DEV)
+    kvc.kvc_gate_distance(cache, [st], T, d2)
+    torch.cuda.synchronize()
+    oc = hp.oracle_cache(cache_cpu)
+    expect = 0.0
+    for l in range(L):
+        for h in range(H):
+            v = orc.bf16_to_f64(oc.get_bits("v", l, h))
+            lam = np.linalg.eigvalsh(v.T @ v)[::-1]
+            expect += float(np.sum(lam[r:]))
+    assert abs(d2.item() - expect) <= 2e-3 * expect, (d2.item(), expect)
