@@ -370,7 +370,10 @@ __global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant
 // The input is the sum of the partial Gram matrices, symmetrised; it is written back so that
 // the final Gram matrix stays readable in the workspace.
 // ---------------------------------------------------------------------------------
-constexpr int kEigThreads = 512;
+#ifndef KVC_EIG_THREADS
+#define KVC_EIG_THREADS 256
+#endif
+constexpr int kEigThreads = KVC_EIG_THREADS;
 constexpr int kEigMaxR = 64;
 
 __device__ __forceinline__ float warp_sum(float x) {
@@ -409,7 +412,7 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   // + 3), so the work of a row stays spread over its threads as the trailing block shrinks.
   // Reflector k is written to row k of the shared-memory copy (zeros left of the sub-diagonal), where
   // the back-transformation finds it later.  Two block barriers per step.
-  constexpr int TPR = kEigThreads / N;          // 4 (N = 128) or 8 (N = 64)
+  constexpr int TPR = kEigThreads / N;          // threads per row: 4 (N = 128) or 8 (N = 64) at 512 threads
   constexpr int NCH = N / (4 * TPR);            // chunks per thread: 8 or 2
   static_assert(TPR * N == kEigThreads && NCH * 4 * TPR == N && TPR <= 32, "thread layout");
   const int trow = tid / TPR, tq = tid % TPR;
@@ -589,12 +592,15 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   }
   __syncthreads();
   {
-    // four threads per eigenvalue: each round tests four interior points, the interval shrinks 5x
-    const int ev = tid >> 2, sub = tid & 3;        // kEigThreads = 4 * 128
+    // TPE threads per eigenvalue: each round tests TPE interior points, the interval shrinks (TPE + 1)x
+    constexpr int TPE = kEigThreads / 128;         // 4 at 512 threads, 2 at 256
+    constexpr int kRounds = TPE == 4 ? 12 : 17;    // 5^12 = 2.4e8, 3^17 = 1.3e8: both beyond 2^26
+    static_assert(TPE == 4 || TPE == 2, "multisection layout");
+    const int ev = tid / TPE, sub = tid % TPE;
     const int want = n - 1 - ev;                   // ascending index of this group's eigenvalue
     float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
-    for (int it = 0; it < 12; ++it) {              // 5^12 = 2.4e8 > 2^26
-      const float step = (hi - lo) * 0.2f;
+    for (int it = 0; it < kRounds; ++it) {
+      const float step = (hi - lo) * (1.f / (float)(TPE + 1));
       const float mid = lo + step * (float)(sub + 1);
       // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots
       int cnt = 0;
@@ -608,10 +614,10 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
         }
       }
       const bool below = cnt <= want;              // the eigenvalue is at or above this point
-      // the four points are ordered: new lo = last point with `below`, new hi = first without
-      const unsigned grp = __ballot_sync(0xffffffffu, below) >> (lane & ~3) & 0xFu;
+      // the points are ordered: new lo = last point with `below`, new hi = first without
+      const unsigned grp = __ballot_sync(0xffffffffu, below) >> (lane & ~(TPE - 1)) & ((1u << TPE) - 1u);
       const int nb = __popc(grp);                  // points 0 .. nb-1 are below (monotone up to rounding)
-      const float nlo = lo + step * (float)nb, nhi = (nb < 4) ? lo + step * (float)(nb + 1) : hi;
+      const float nlo = lo + step * (float)nb, nhi = (nb < TPE) ? lo + step * (float)(nb + 1) : hi;
       lo = nlo;
       hi = nhi;
     }
