@@ -228,3 +228,77 @@ def test_long_context_full_size_sampled_slabs():
             gv = orc.bf16_to_f64(_slab_bits(W["ring"][0], which, l, h))
             bad = np.abs(gv - ref2) > hp.BF16_REL * np.abs(ref2) + hp.BF16_ABS
             assert bad.mean() < 2e-3
+
+
+def test_multi_anchor_path_full_size():
+    """Gate distance, token weights and weighted apply at the 8K config's size (3 anchors of rank 32):
+    the oracle walks all 256 slabs for the gate distances and the token scores (two matrix products
+    per slab and anchor); the weighted apply is checked on sampled slabs."""
+    cfg = wl.CONFIGS["llama8b_8k"]
+    rope = kvc.Rope(cfg.theta)
+    f = hp.inv_freq(cfg)
+    kvc.kvc_status_reset()
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    src, tables, mk = _make_full(cfg, DEV)
+    L, H, T, d = cfg.L, cfg.H, cfg.T, cfg.d
+    base, delta = [], []
+    for v in range(3):
+        s = wl.hop_state(cfg, 1 + v, DEV)
+        base.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
+        s = wl.hop_state(cfg, 4 + v, DEV)
+        delta.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
+    tp = kvc.kvc_multi_tpad(T)
+    wk, wv = torch.empty(3, tp, device=DEV), torch.empty(3, tp, device=DEV)
+    ws = torch.empty(kvc.kvc_token_weights_workspace_bytes(src, 3), dtype=torch.uint8, device=DEV)
+    pos = [64, 200, 333]
+    kvc.kvc_token_weights(src, 150, base, pos, rope, wk, wv, ws)
+    d2 = torch.empty(3, dtype=torch.float64, device=DEV)
+    kvc.kvc_gate_distance(src, base, T, d2)
+    dst = mk(None)
+    ws2 = torch.empty(kvc.kvc_multi_workspace_bytes(src, delta), dtype=torch.uint8, device=DEV)
+    shift = -97
+    kvc.kvc_apply_multi(src, delta, wk, wv, shift, rope, dst, ws2)
+    torch.cuda.synchronize()
+    assert kvc.kvc_status_poll() == 0
+    scores = ws.view(torch.float32).view(3, 2, tp).cpu().numpy().astype(np.float64)
+    wk_h, wv_h = wk.cpu().numpy().astype(np.float64), wv.cpu().numpy().astype(np.float64)
+
+    # ---- gate distance: the whole sum, slab by slab in the oracle (values only: 256 slabs of 8192 x 128)
+    total = np.zeros(3)
+    mean_abs = np.zeros((3, 2, T))                       # the token-weight scores, accumulated over all slabs
+    for l in range(L):
+        for h in range(H):
+            vs = orc.bf16_to_f64(_slab_bits(src, "v", l, h))
+            ks = orc.rope_shift(orc.bf16_to_f64(_slab_bits(src, "k", l, h)), -150, f)
+            for v in range(3):
+                rec_v = base[v].coeff_v[l, h].cpu().numpy().astype(np.float64) @ base[v].basis_v[l, h].cpu().numpy().astype(np.float64)
+                total[v] += orc.gate_distance([vs], [rec_v], T) ** 2
+                rec_k = base[v].coeff_k[l, h].cpu().numpy().astype(np.float64) @ base[v].basis_k[l, h].cpu().numpy().astype(np.float64)
+                rec_k = orc.rope_shift(rec_k, -pos[v], f)
+                mean_abs[v, 0] += np.abs(ks - rec_k).sum(axis=1)
+                mean_abs[v, 1] += np.abs(vs - rec_v).sum(axis=1)
+    mean_abs /= L * H * d
+    got = d2.cpu().numpy()
+    assert np.all(np.abs(got - total) <= 2e-4 * total), (got, total)
+    assert np.max(np.abs(scores[:, :, :T] - mean_abs)) <= 2e-5 * np.max(mean_abs)
+    # the weights are the softmax of minus these scores (Eq. in App. A.3), from the oracle's scores
+    for kv, w_h in ((0, wk_h), (1, wv_h)):
+        z = -mean_abs[:, kv]
+        z = z - z.max(axis=0, keepdims=True)
+        ref_w = np.exp(z) / np.exp(z).sum(axis=0, keepdims=True)
+        assert np.max(np.abs(w_h[:, :T] - ref_w)) <= 2e-5
+
+    # ---- weighted apply on sampled slabs, with the oracle's own weights
+    for (l, h) in _sample_slabs(cfg, n=2):
+        for kv, which in ((0, "k"), (1, "v")):
+            z = -mean_abs[:, kv]
+            z = z - z.max(axis=0, keepdims=True)
+            ref_w = np.exp(z) / np.exp(z).sum(axis=0, keepdims=True)
+            ref, out = orc.apply_multi_slab(
+                _slab_bits(src, which, l, h), ref_w,
+                [getattr(a, "coeff_" + which)[l, h].cpu().numpy() for a in delta],
+                [getattr(a, "basis_" + which)[l, h].cpu().numpy() for a in delta],
+                [T] * 3, shift, f, which == "k")
+            gotb = _slab_bits(dst, which, l, h)
+            assert hp.tol_ratio(gotb, ref) <= 1.0
+            assert hp.ulp_mismatch_fraction(gotb, out) < 2e-2
