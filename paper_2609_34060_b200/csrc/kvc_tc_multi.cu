@@ -6,8 +6,9 @@
 // Differences from the single-state kernel (kvc_tc_apply.cu), whose skeleton this one shares
 // (persistent CTAs, TMA tiles, tcgen05 MMAs into TMEM, 16-warp team, store warp):
 //   * a tile has a variable number of ring entries, one per rank block that covers it; an entry
-//     holds the fp32 coefficient block of its anchor (converted to bf16 hi/lo in place, scaled by
-//     the anchor's token weights on the way), the block's basis operand and the tile's 128 weights;
+//     is the fp32 coefficient block of its anchor (converted to bf16 hi/lo in place, scaled by the
+//     anchor's token weights on the way) with the tile's 128 weights, in a deep ring (HBM latency),
+//     and the block's basis operand in a shallow ring of its own (L2 latency, separate producer);
 //   * the basis operands are too many to stay resident per slab, so a preparation kernel writes
 //     them once, transposed and split, into a workspace from where TMA drops them into the ring
 //     (L2 traffic, no work for the team);
@@ -38,10 +39,10 @@ constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a ba
 constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
 constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
 constexpr int kOperandBytes = 128 * 128;          // 128 channels x (32 hi + 32 lo) bf16
-constexpr int kEntryBytes = kCoeffBytes + kOperandBytes;
 constexpr int kWeightBytes = kTileTok * 4;
 constexpr int NSTAGE = 3;                         // base-tile slots
-constexpr int NE = 3;                             // ring entries (rank blocks in flight)
+constexpr int NC = 5;                             // coefficient blocks in flight (HBM latency)
+constexpr int NO = 2;                             // operand blocks in flight (served by L2)
 
 struct Block {                 // one rank block of one anchor
   const float* w_k;            // token weights of the anchor [T_pad] (nullptr: all ones)
@@ -67,7 +68,8 @@ struct MultiLaunch {
 
 struct Ctrl {
   uint64_t full[NSTAGE], ready[NSTAGE], empty[NSTAGE];      // base-tile ring
-  uint64_t efull[NE], econv[NE], eempty[NE];                // entry ring
+  uint64_t cfull[NC], conv[NC], cempty[NC];                 // coefficient ring (one entry per rank block of a tile)
+  uint64_t ofull[NO], oempty[NO];                           // operand ring (same sequence of entries)
   uint64_t mma_done[2], acc_empty[2];
   uint64_t drain;
   uint32_t tmem_base;
@@ -145,10 +147,12 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t stages = base;
-  constexpr int kEntryOff = NSTAGE * kBaseBytes;
-  constexpr int kWeightOff = kEntryOff + NE * kEntryBytes;
-  constexpr int kCtrlOff = kWeightOff + NE * kWeightBytes;
-  const uint32_t entries = base + kEntryOff;
+  constexpr int kCoeffOff = NSTAGE * kBaseBytes;
+  constexpr int kOperandOff = kCoeffOff + NC * kCoeffBytes;
+  constexpr int kWeightOff = kOperandOff + NO * kOperandBytes;
+  constexpr int kCtrlOff = kWeightOff + NC * kWeightBytes;
+  const uint32_t coeffs = base + kCoeffOff;
+  const uint32_t operands = base + kOperandOff;
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + kCtrlOff);
   volatile int* abort_flag = &ctrl->abort_flag;
 
@@ -163,10 +167,14 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
       mbar_init(smem_u32(&ctrl->ready[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
-    for (int c = 0; c < NE; ++c) {
-      mbar_init(smem_u32(&ctrl->efull[c]), 1);
-      mbar_init(smem_u32(&ctrl->econv[c]), kTeamThreads);
-      mbar_init(smem_u32(&ctrl->eempty[c]), 1);
+    for (int c = 0; c < NC; ++c) {
+      mbar_init(smem_u32(&ctrl->cfull[c]), 1);
+      mbar_init(smem_u32(&ctrl->conv[c]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->cempty[c]), 1);
+    }
+    for (int o = 0; o < NO; ++o) {
+      mbar_init(smem_u32(&ctrl->ofull[o]), 1);
+      mbar_init(smem_u32(&ctrl->oempty[o]), 1);
     }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
@@ -234,18 +242,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
       // the tile's rank blocks
       for (int e = 0; e < p.n_blocks; ++e) {
         if (!active(e, t0)) continue;
-        const int c = epos % NE;
+        const int c = epos % NC;
         if (lane == 0) {
-          ok = mbar_wait(smem_u32(&ctrl->eempty[c]), ((epos / NE) & 1u) ^ 1u, abort_flag) ? 1 : 0;
+          ok = mbar_wait(smem_u32(&ctrl->cempty[c]), ((epos / NC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
           if (ok) {
             const Block& b = p.blk[e];
             const float* wts = is_v ? b.w_v : b.w_k;
-            const uint32_t ebar = smem_u32(&ctrl->efull[c]);
-            mbar_expect_tx(ebar, (uint32_t)(kEntryBytes + (wts ? kWeightBytes : 0)));
+            const uint32_t ebar = smem_u32(&ctrl->cfull[c]);
+            mbar_expect_tx(ebar, (uint32_t)(kCoeffBytes + (wts ? kWeightBytes : 0)));
             const CUtensorMap* cmap = is_v ? &p.coeff_v[b.anchor] : &p.coeff_k[b.anchor];
-            tma_load_3d(entries + c * kEntryBytes, cmap, ebar, b.col0, t0, w.slab());
-            tma_load_2d(entries + c * kEntryBytes + kCoeffBytes, &p.operand, ebar, 0,
-                        ((e * 2 + is_v) * (p.L * p.H) + w.slab()) * 128);
+            tma_load_3d(coeffs + c * kCoeffBytes, cmap, ebar, b.col0, t0, w.slab());
             if (wts) bulk_load_1d(base + kWeightOff + c * kWeightBytes, wts + t0, kWeightBytes, ebar);
           }
         }
@@ -262,8 +268,8 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
     if (lane == 0) {
       for (uint32_t k = (i > NSTAGE ? i - NSTAGE : 0); k < i; ++k)
         mbar_wait_drain(smem_u32(&ctrl->full[k % NSTAGE]), (k / NSTAGE) & 1u);
-      for (uint32_t k = (epos > NE ? epos - NE : 0); k < epos; ++k)
-        mbar_wait_drain(smem_u32(&ctrl->efull[k % NE]), (k / NE) & 1u);
+      for (uint32_t k = (epos > NC ? epos - NC : 0); k < epos; ++k)
+        mbar_wait_drain(smem_u32(&ctrl->cfull[k % NC]), (k / NC) & 1u);
     }
   } else if (warp == 1) {
     // =============================================================== MMA issuer
@@ -281,14 +287,15 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
         uint32_t acc = 0;
         for (int e = 0; e < p.n_blocks; ++e) {
           if (!active(e, t0)) continue;
-          const int c = epos % NE;
-          if (!mbar_wait(smem_u32(&ctrl->econv[c]), (epos / NE) & 1u, abort_flag)) {
+          const int c = epos % NC, o = epos % NO;
+          if (!mbar_wait(smem_u32(&ctrl->conv[c]), (epos / NC) & 1u, abort_flag) ||
+              !mbar_wait(smem_u32(&ctrl->ofull[o]), (epos / NO) & 1u, abort_flag)) {
             alive = false;
             break;
           }
           tc_fence_after();
-          const uint64_t ad = umma_desc_sw128(entries + c * kEntryBytes);
-          const uint64_t bd = umma_desc_sw128(entries + c * kEntryBytes + kCoeffBytes);
+          const uint64_t ad = umma_desc_sw128(coeffs + c * kCoeffBytes);
+          const uint64_t bd = umma_desc_sw128(operands + o * kOperandBytes);
           // byte offsets inside the 128-byte row: c1 | c2 for A, B1 | B2 for B; 16 bf16 = 32 B per k-step
           const int aoff[6] = {0, 32, 64, 96, 0, 32};
           const int boff[6] = {0, 32, 0, 32, 64, 96};
@@ -297,7 +304,8 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
             umma_bf16(d_tmem, ad + (uint64_t)(aoff[k] >> 4), bd + (uint64_t)(boff[k] >> 4), kIdescBf16M128N128, acc);
             acc = 1;
           }
-          umma_commit(smem_u32(&ctrl->eempty[c]));        // the entry may be refilled
+          umma_commit(smem_u32(&ctrl->cempty[c]));        // both slots may be refilled
+          umma_commit(smem_u32(&ctrl->oempty[o]));
           ++epos;
         }
         if (!alive) break;
@@ -307,7 +315,32 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
       mbar_wait_drain(smem_u32(&ctrl->drain), 0);
     }
   } else if (warp == 2) {
-    // spare warp: keeps the team's warps aligned with the TMEM lane quadrants (warp id & 3)
+    // =============================================================== operand producer (one lane)
+    // the prepared basis operands come from L2: a shallow ring of their own, so that waiting for an
+    // operand slot never holds back the coefficient loads
+    if (lane == 0) {
+      Walker w;
+      w.init(p, tile_begin, tile_end);
+      uint32_t epos = 0;
+      bool alive = true;
+      for (; alive && !w.done(); w.next()) {
+        const int t0 = w.t0(), is_v = w.is_v();
+        for (int e = 0; e < p.n_blocks; ++e) {
+          if (!active(e, t0)) continue;
+          const int o = epos % NO;
+          if (!mbar_wait(smem_u32(&ctrl->oempty[o]), ((epos / NO) & 1u) ^ 1u, abort_flag)) {
+            alive = false;
+            break;
+          }
+          const uint32_t obar = smem_u32(&ctrl->ofull[o]);
+          mbar_expect_tx(obar, (uint32_t)kOperandBytes);
+          tma_load_2d(operands + o * kOperandBytes, &p.operand, obar, 0, ((e * 2 + is_v) * (p.L * p.H) + w.slab()) * 128);
+          ++epos;
+        }
+      }
+      for (uint32_t k = (epos > NO ? epos - NO : 0); k < epos; ++k)
+        mbar_wait_drain(smem_u32(&ctrl->ofull[k % NO]), (k / NO) & 1u);
+    }
   } else if (warp == 3) {
     // =============================================================== store warp
     Walker w;
@@ -400,13 +433,13 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
       const int t0 = cw.t0(), is_v = cw.is_v();
       for (int e = 0; e < p.n_blocks; ++e) {
         if (!active(e, t0)) continue;
-        const int c = epos % NE;
-        bool ok = mbar_wait(smem_u32(&ctrl->efull[c]), (epos / NE) & 1u, abort_flag);
+        const int c = epos % NC;
+        bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), (epos / NC) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) return false;
         const bool weighted = (is_v ? p.blk[e].w_v : p.blk[e].w_k) != nullptr;
         const float wt = weighted ? reinterpret_cast<const float*>(smem + kWeightOff + c * kWeightBytes)[crow] : 1.f;
-        uint8_t* row = smem + kEntryOff + c * kEntryBytes + crow * 128;
+        uint8_t* row = smem + kCoeffOff + c * kCoeffBytes + crow * 128;
         // this thread's 8 coefficients: fp32 chunks 2*cpart, 2*cpart+1 of the row
         float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
         float4 f1 = *reinterpret_cast<const float4*>(row + (((2 * cpart + 1) ^ csw) << 4));
@@ -419,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
         *reinterpret_cast<uint4*>(row + ((cpart ^ csw) << 4)) = hi;         // c1: chunks 0..3
         *reinterpret_cast<uint4*>(row + (((4 + cpart) ^ csw) << 4)) = lo;   // c2: chunks 4..7
         fence_proxy_async();
-        mbar_arrive(smem_u32(&ctrl->econv[c]));
+        mbar_arrive(smem_u32(&ctrl->conv[c]));
         ++epos;
       }
       return true;
@@ -638,7 +671,8 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(M.total_tiles < sms ? M.total_tiles : sms);
-  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NE * (kEntryBytes + kWeightBytes) + sizeof(Ctrl);
+  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
+                          (size_t)NO * kOperandBytes + sizeof(Ctrl);
   static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
   static bool set = false;
   if (!set) {
