@@ -257,6 +257,23 @@ int kvc_apply_multi(const kvc_cache *src, const kvc_state *deltas, int32_t n_anc
 size_t kvc_multi_workspace_bytes(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors);
 
 /*
+ * Positional re-alignment of a stored correction (App. A.2: a correction for a recurring prefix
+ * relation "is profiled once, stored in low-rank form, and positionally re-aligned when reused").
+ * A rotation is linear in the channels, Rot_s(c . B) = c . Rot_s(B), so re-aligning a stored key
+ * correction by `shift` positions is rotating every row of its key basis by `shift`:
+ *     basis_k_out[l,h,q,:] = Rot_shift(basis_k_in[l,h,q,:]) ,
+ * coefficients and value factors are not touched.  Uses: a state fitted at target position p and
+ * re-aligned by -p is the same correction in canonical coordinates; re-aligned by p' it applies at
+ * position p' through kvc_apply / kvc_apply_multi, whose own `shift` aligns the source cache.
+ *   L, H, d      geometry of the basis [L, H, st->r, d], d in {64, 128}
+ *   st           the state whose basis_k (device, basis_dtype) is read
+ *   basis_k_out  DEVICE, same shape and dtype; may be st->basis_k itself (in place)
+ * float32 rotation with the angles' cos / sin computed in float64 on the host, like kvc_apply.
+ */
+int kvc_state_realign(const kvc_state *st, int32_t L, int32_t H, int32_t d, int32_t shift, const kvc_rope *rope,
+                      void *basis_k_out, void *stream);
+
+/*
  * Token-wise interpolation weights (App. A.3 "Correction Weighting and Positional Alignment"):
  * for token t and anchor v the score is the mean over layers, heads and channels of
  *     | C_src[l,h,t,c] - coeff(v)[l,h,t,:] . basis(v)[l,h][:,c] | ,

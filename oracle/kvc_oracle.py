@@ -460,6 +460,15 @@ def stack_anchors(weights, coeffs, bases):
     return c, b
 
 
+def realign_basis(basis_k, s, inv_freq, pairing=ROPE_HALF):
+    """App. A.2 (PF-induced deltas): a stored key correction is "positionally re-aligned when reused".
+    A rotation acts on the channel axis and is linear, so Rot_s(c . B) = c . Rot_s(B): re-aligning a
+    stored correction by s positions is rotating every key-basis row by s; coefficients and value
+    factors are untouched.  basis_k [..., r, d] -> same shape, float64."""
+    b = np.asarray(basis_k, np.float64)
+    return rope_shift(b.reshape(-1, b.shape[-1]), s, inv_freq, pairing).reshape(b.shape)
+
+
 def token_weights(src_feat, anchor_feats, temperature=1.0):
     """App. A.3 "Correction Weighting": token-wise interpolation weights.  For token t and anchor v the
     score is the mean absolute difference between the source cache's features of t and the anchor's

@@ -32,6 +32,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
+    "kvc_state_realign",
 )
 
 
@@ -89,6 +90,7 @@ def load(path: Optional[str] = None):
     lib.kvc_apply_multi.argtypes = [PC, PS, i32, vp, vp, i32, PR, PC, vp, sz, vp]
     lib.kvc_multi_workspace_bytes.argtypes = [PC, PS, i32]
     lib.kvc_multi_workspace_bytes.restype = sz
+    lib.kvc_state_realign.argtypes = [PS, i32, i32, i32, i32, PR, vp, vp]
     lib.kvc_token_weights.argtypes = [PC, i32, PS, C.POINTER(i32), i32, PR, C.c_double, vp, vp, vp, sz, vp]
     lib.kvc_token_weights_workspace_bytes.argtypes = [PC, i32]
     lib.kvc_token_weights_workspace_bytes.restype = sz
@@ -343,6 +345,17 @@ def kvc_apply_multi(src: Cache, deltas: Sequence[State], w_k: Optional[torch.Ten
 
 
 KVC_MAX_ANCHORS = 16
+
+
+def kvc_state_realign(st: State, shift: int, rope: Rope, out: Optional[torch.Tensor] = None, stream=None) -> State:
+    """A state whose key correction is re-aligned by `shift` positions: basis_k rows rotated (into `out`,
+    a new tensor by default; pass st.basis_k for in place); coefficients and value factors are shared."""
+    L, H, r, d = (int(x) for x in st.basis_k.shape)
+    out = torch.empty_like(st.basis_k) if out is None else out
+    s, rp = st.struct(), rope.struct()
+    _check(load().kvc_state_realign(C.byref(s), L, H, d, int(shift), C.byref(rp), out.data_ptr(), _stream(stream)),
+           "kvc_state_realign")
+    return State(st.coeff_k, st.coeff_v, out, st.basis_v, n_cov=st.n_cov)
 
 
 def kvc_token_weights_workspace_bytes(src: Cache, n_anchors: int) -> int:

@@ -445,6 +445,28 @@ int kvc_apply_multi(const kvc_cache* src, const kvc_state* deltas, int32_t n_anc
   return rc;
 }
 
+int kvc_state_realign(const kvc_state* st, int32_t L, int32_t H, int32_t d, int32_t shift, const kvc_rope* rope,
+                      void* basis_k_out, void* stream) {
+  if (!st || L <= 0 || H <= 0 || st->r < 0) return KVC_E_INVALID_ARG;
+  if (d != 64 && d != 128) return KVC_E_UNSUPPORTED;
+  int rc;
+  if ((rc = check_rope(rope)) != KVC_OK) return rc;
+  if (st->basis_dtype != KVC_F32 && st->basis_dtype != KVC_BF16) return KVC_E_INVALID_ARG;
+  if (st->r == 0) return KVC_OK;
+  if (!st->basis_k || !basis_k_out) return KVC_E_INVALID_ARG;
+  RealignLaunch q;
+  memset(&q, 0, sizeof(q));
+  q.in = st->basis_k;
+  q.out = basis_k_out;
+  q.rows = (int64_t)L * H * st->r;
+  q.d = d;
+  q.bf16 = st->basis_dtype == KVC_BF16;
+  q.pairing = rope->pairing;
+  rope_tables(rope, d, shift, q.cs, q.sn);
+  if (launch_realign_basis(q, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return KVC_E_CUDA;
+  return KVC_OK;
+}
+
 size_t kvc_token_weights_workspace_bytes(const kvc_cache* src, int32_t n_anchors) {
   if (!src || n_anchors <= 0) return 0;
   return (size_t)n_anchors * 2 * (size_t)KVC_MULTI_TPAD(src->T) * sizeof(float);

@@ -90,6 +90,14 @@ struct TokenWeightsLaunch {    // softmax over anchors per token
   int32_t n_cov[16];
 };
 
+struct RealignLaunch {         // rotation of basis rows
+  const void* in;
+  void* out;                   // may be `in`
+  int64_t rows;                // L * H * r
+  int32_t d, bf16, pairing, pad;
+  float cs[kMaxHalfD], sn[kMaxHalfD];
+};
+
 // Address of row (l, h, t) of a cache; returns nullptr (and flags) on a bad page id.
 __device__ __forceinline__ __nv_bfloat16* row_ptr(const DevCache& c, __nv_bfloat16* base, int l, int h, int t,
                                                    uint32_t* status) {

@@ -113,4 +113,43 @@ cudaError_t launch_token_weights(const float* scores, const TokenWeightsLaunch& 
   return cudaGetLastError();
 }
 
+// Re-alignment of a stored key correction (App. A.2): every key-basis row rotated by a shift,
+// Rot_s(c . B) = c . Rot_s(B).  One thread per RoPE pair; float32 or bf16 rows of d values.
+__global__ void __launch_bounds__(256) realign_basis_kernel(const RealignLaunch q) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int half = q.d / 2;
+  if (i >= q.rows * half) return;
+  const int64_t row = i / half;
+  const int k = (int)(i - row * half);
+  const int c0 = q.pairing == 0 ? k : 2 * k, c1 = q.pairing == 0 ? k + half : 2 * k + 1;
+  const float cs = q.cs[k], sn = q.sn[k];
+  float u, v;
+  if (q.bf16) {
+    const __nv_bfloat16* in = reinterpret_cast<const __nv_bfloat16*>(q.in) + row * q.d;
+    u = __bfloat162float(in[c0]);
+    v = __bfloat162float(in[c1]);
+  } else {
+    const float* in = reinterpret_cast<const float*>(q.in) + row * q.d;
+    u = in[c0];
+    v = in[c1];
+  }
+  const float ru = u * cs - v * sn, rv = u * sn + v * cs;
+  if (q.bf16) {
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(q.out) + row * q.d;
+    out[c0] = __float2bfloat16_rn(ru);
+    out[c1] = __float2bfloat16_rn(rv);
+  } else {
+    float* out = reinterpret_cast<float*>(q.out) + row * q.d;
+    out[c0] = ru;
+    out[c1] = rv;
+  }
+}
+
+cudaError_t launch_realign_basis(const RealignLaunch& q, cudaStream_t s) {
+  const int64_t n = q.rows * (q.d / 2);
+  if (n <= 0) return cudaSuccess;
+  realign_basis_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(q);
+  return cudaGetLastError();
+}
+
 }  // namespace kvc

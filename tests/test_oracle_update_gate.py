@@ -287,3 +287,31 @@ def test_apply_multi_slab_pins():
     k = rng.standard_normal((T, d))
     moved = orc.rope_shift(k, 11, inv)
     assert np.allclose(orc.canonical_key_features([moved], 11, inv), k, atol=1e-12)
+
+
+def test_realign_basis_pins():
+    """Rot_s(c . B) = c . Rot_s(B); canonical storage: a correction fitted at target position p and
+    re-aligned by -p equals the correction fitted on inputs that were first moved to position 0."""
+    rng = np.random.default_rng(6)
+    T, d, r = 11, 8, 3
+    inv = orc.rope_inv_freq(d, 10000.0)
+    c = rng.standard_normal((T, r))
+    B = rng.standard_normal((r, d))
+    for s in (0, 7, -19):
+        lhs = orc.rope_shift(c @ B, s, inv)
+        assert np.allclose(lhs, c @ orc.realign_basis(B, s, inv), atol=1e-12)
+    assert np.array_equal(orc.realign_basis(B, 0, inv), B)
+    assert np.allclose(orc.realign_basis(orc.realign_basis(B, 5, inv), -5, inv), B, atol=1e-12)
+    # rows stay orthonormal (a rotation is orthogonal)
+    Q = np.linalg.qr(rng.standard_normal((d, r)))[0].T
+    Qr = orc.realign_basis(Q, 13, inv)
+    assert np.allclose(Qr @ Qr.T, np.eye(r), atol=1e-12)
+    # the deviation measured at target position p_t, moved back to position 0, is the deviation of the
+    # inputs moved back to their canonical coordinates: coefficients on the re-aligned basis agree
+    p_s, p_t = 40, 95
+    src = rng.standard_normal((T, d))
+    tgt = orc.rope_shift(src, p_t - p_s, inv) + c @ Q
+    delta_t = tgt - orc.rope_shift(src, p_t - p_s, inv)                       # Eq. 12, at the target's positions
+    delta_0 = orc.rope_shift(tgt, -p_t, inv) - orc.rope_shift(src, -p_s, inv)  # both sides canonical
+    assert np.allclose(orc.rope_shift(delta_t, -p_t, inv), delta_0, atol=1e-12)
+    assert np.allclose(delta_t @ Q.T, delta_0 @ orc.realign_basis(Q, -p_t, inv).T, atol=1e-12)
