@@ -372,7 +372,7 @@ def cpu_baseline(cfg: wl.Config, budget_s: float = 20.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="llama8b_8k", choices=sorted(wl.CONFIGS) + ["serve64"])
     ap.add_argument("--requests", type=int, default=64, help="serve64: number of concurrent requests")
@@ -467,10 +467,15 @@ def main():
     ev = {}
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin.record()
+    step_marks = []
     for _ in range(args.steps):
         run_step(W, kvc, ev)
+        m = torch.cuda.Event(enable_timing=True)
+        m.record()
+        step_marks.append(m)
     t_end.record()
     barrier()
+    per_step = [a.elapsed_time(b) for a, b in zip([t_begin] + step_marks[:-1], step_marks)]
     clocks = sampler.stop() if rank == 0 else None
     ms_total = t_begin.elapsed_time(t_end)
     chain_ms = sum(b.elapsed_time(e) for b, e in zip(ev.get("chain_begin", []), ev.get("chain_end", []))) / args.steps
@@ -535,6 +540,9 @@ def main():
            "roofline": roofline,
            "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
                          "us_per_agent_layer": hop_ms * 1e3 / cfg.L,
+                         "output_only_GBs": (sum(o.nbytes() for o in W.get("outs", [])) / max(len(W.get("outs", [])), 1))
+                         / (hop_ms * 1e-3) / 1e9 if W.get("outs") else None,
+                         "step_ms_median": sorted(per_step)[len(per_step) // 2], "step_ms_min": min(per_step),
                          "update_fit_GBs": upd_b / (upd_ms * 1e-3) / 1e9, "update_ms_per_step": upd_ms,
                          "chain_ms_per_step": chain_ms,
                          "kernel_family": {0: "auto", 1: "generic (CUDA cores)", 2: "tc (TMA + tcgen05)"}[last_path]}}
