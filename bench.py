@@ -113,7 +113,7 @@ def _dist():
 # --------------------------------------------------------------------------------------
 
 
-def build_workload(cfg: wl.Config, dev, kvc, only="all"):
+def build_workload(cfg: wl.Config, dev, kvc, only="all", grouped=False):
     """Everything one step reads, resident on the device.  Draws come from the seeded
     generator; the true target caches are derived with the library itself (aligned
     source + exact rank-r deviation, then N(0, sigma) noise, rounded to bf16)."""
@@ -137,6 +137,11 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all"):
         # the chain (or the gate) alone: the generator's states are used directly, no targets needed
         states = []
         for a in range(1, n):
+            if grouped:     # one state per layer over all KV heads (D = H d): coeff [L,T,r], basis [L,r,H d]
+                mkc = lambda tag: wl.coefficients(cfg.L, 1, cfg.T, cfg.r, cfg.seed, 4 * a + tag, dev)[:, 0].contiguous()
+                mkb = lambda tag: wl.orthonormal_basis(cfg.L, 1, cfg.r, cfg.H * cfg.d, cfg.seed, 4 * a + tag, dev)[:, 0].contiguous()
+                states.append(kvc.State(mkc(0), mkc(1), mkb(2), mkb(3), grouping=kvc.KVC_GROUP_LAYER))
+                continue
             s = wl.hop_state(cfg, a, dev)
             states.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
         if only == "gate":
@@ -383,6 +388,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
     ap.add_argument("--rank", type=int, default=0, help="override the rank r (experiments)")
+    ap.add_argument("--grouped", type=int, default=0, help="1: per-layer states (D = H d), with --only apply")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
     ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi", "weights"],
                     help="profiling aid: time only the chain or only the state updates")
@@ -446,7 +452,7 @@ def main():
     elif ring:
         W = build_ring(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
     else:
-        W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only)
+        W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only, grouped=bool(args.grouped) and args.only == "apply")
     if args.only != "all":
         args.no_e2e = True
     upd_b, app_b = step_bytes(W, kvc)
@@ -529,7 +535,7 @@ def main():
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "gate distance (one anchor, Eq. 9)" if args.only == "gate" else "multi-anchor apply (Eq. 8)" if args.only == "multi" else "token-weight scores (one anchor, App. A.3)" if args.only == "weights" else "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0 and args.only not in ("gate", "multi", "weights")) else None,
+                "traffic": APPLY_TRAFFIC_BYTES_LLAMA8B_8K if (args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0 and args.only not in ("gate", "multi", "weights") and not args.grouped) else None,
                 "algorithmic_bytes_per_launch": app_b // hops,
                 "us_per_launch": hop_ms * 1e3}
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -101,8 +101,23 @@ typedef struct kvc_state {
   int32_t r;
   int32_t n_cov;
   int32_t basis_dtype;        /* KVC_F32 | KVC_BF16                                */
-  int32_t reserved;
+  int32_t grouping;           /* KVC_GROUP_HEAD (0) | KVC_GROUP_LAYER              */
 } kvc_state;
+
+/*
+ * Feature grouping of a state (Sec. 3.1: B in R^{r x D} with "D the KV cache feature dimension").
+ *   KVC_GROUP_HEAD   one state per (layer, KV head), D = d:
+ *                    coeff [L, H, n_cov, r], basis [L, H, r, d]                    (the default)
+ *   KVC_GROUP_LAYER  one state per layer over all KV heads, D = H d: the coefficients of a token are
+ *                    shared by the heads of a layer,
+ *                    coeff [L, n_cov, r], basis [L, r, H d]  (head h uses columns h d .. (h+1) d - 1)
+ *                    K_dst[l,h,t,:] = bf16( Rot(K_src[l,h,t,:]) + coeff_k[l,t,:] . basis_k[l][:, h d : (h+1) d] )
+ * Grouping by layer is served by kvc_apply, kvc_chain, kvc_apply_batch and by kvc_state_update in
+ * KVC_PROJECT mode (the projection sums over the heads: coeff[l,t,:] = sum_h Delta[l,h,t,:] . basis[l][:, h]^T);
+ * KVC_FIT, the gate, token weights and kvc_apply_multi return KVC_E_UNSUPPORTED for it.
+ */
+#define KVC_GROUP_HEAD  0
+#define KVC_GROUP_LAYER 1
 
 /*
  * Rotary position embedding used for the key re-alignment that precedes every

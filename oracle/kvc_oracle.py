@@ -460,6 +460,29 @@ def stack_anchors(weights, coeffs, bases):
     return c, b
 
 
+def ungroup_state(coeff_k, coeff_v, basis_k, basis_v, H, n_cov=None):
+    """Sec. 3.1 with D = H d (one state per layer over all KV heads): coeff [L, n_cov, r] is shared by
+    the heads of a layer and basis [L, r, H d] holds head h's part in columns h d .. (h+1) d - 1.
+    Returns the same state in the per-(layer, head) form, coeff [L, H, n_cov, r] and basis
+    [L, H, r, d], which every other function of this module takes: the two forms define the same
+    low-rank product  Z[l] = coeff[l] @ basis[l]  with Z[l] = [Z[l,0] | ... | Z[l,H-1]]."""
+    ck, cv = np.asarray(coeff_k), np.asarray(coeff_v)
+    bk, bv = np.asarray(basis_k), np.asarray(basis_v)
+    L, r, HD = bk.shape
+    d = HD // H
+    split = lambda b: np.ascontiguousarray(b.reshape(L, r, H, d).transpose(0, 2, 1, 3))
+    rep = lambda c: np.ascontiguousarray(np.broadcast_to(c[:, None], (L, H) + c.shape[1:]))
+    return State(rep(ck), rep(cv), split(bk), split(bv), n_cov=n_cov)
+
+
+def project_grouped(delta_slabs, basis_l):
+    """Projection for one layer under D = H d: delta_slabs is the list over heads of [T, d]
+    deviations, basis_l [r, H d]; the coefficients are those of the concatenated deviation
+    [T, H d], i.e. the sum over heads of each head's projection on its own columns."""
+    cat = np.concatenate([np.asarray(x, np.float64) for x in delta_slabs], axis=1)
+    return cat @ np.asarray(basis_l, np.float64).T
+
+
 def realign_basis(basis_k, s, inv_freq, pairing=ROPE_HALF):
     """App. A.2 (PF-induced deltas): a stored key correction is "positionally re-aligned when reused".
     A rotation acts on the channel axis and is linear, so Rot_s(c . B) = c . Rot_s(B): re-aligning a

@@ -22,6 +22,7 @@ KVC_F32, KVC_BF16 = 0, 1
 KVC_ROPE_HALF, KVC_ROPE_INTERLEAVED = 0, 1
 KVC_PROJECT, KVC_FIT = 0, 1
 KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
+KVC_GROUP_HEAD, KVC_GROUP_LAYER = 0, 1
 KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4
 KVC_OK = 0
 (KVC_E_INVALID_ARG, KVC_E_SHAPE, KVC_E_UNSUPPORTED, KVC_E_ALIAS, KVC_E_CUDA, KVC_E_WORKSPACE, KVC_E_DEVICE_FLAG,
@@ -51,7 +52,7 @@ class kvc_cache(C.Structure):
 
 class kvc_state(C.Structure):
     _fields_ = [("coeff_k", C.c_void_p), ("coeff_v", C.c_void_p), ("basis_k", C.c_void_p), ("basis_v", C.c_void_p),
-                ("r", C.c_int32), ("n_cov", C.c_int32), ("basis_dtype", C.c_int32), ("reserved", C.c_int32)]
+                ("r", C.c_int32), ("n_cov", C.c_int32), ("basis_dtype", C.c_int32), ("grouping", C.c_int32)]
 
 
 class kvc_rope(C.Structure):
@@ -172,19 +173,22 @@ class Cache:
 
 
 class State:
-    """Rank-r state over torch tensors: coeff fp32 [L,H,n_cov,r], basis fp32|bf16 [L,H,r,d]."""
+    """Rank-r state over torch tensors.  Per (layer, head): coeff fp32 [L,H,n_cov,r], basis fp32|bf16
+    [L,H,r,d].  Per layer (``grouping=KVC_GROUP_LAYER``): coeff [L,n_cov,r], basis [L,r,H*d]."""
 
-    def __init__(self, coeff_k, coeff_v, basis_k, basis_v, n_cov: Optional[int] = None):
+    def __init__(self, coeff_k, coeff_v, basis_k, basis_v, n_cov: Optional[int] = None, grouping: int = KVC_GROUP_HEAD):
         self.coeff_k, self.coeff_v, self.basis_k, self.basis_v = coeff_k, coeff_v, basis_k, basis_v
-        self.r = 0 if basis_k is None else int(basis_k.shape[2])
-        self.n_cov = (0 if coeff_k is None else int(coeff_k.shape[2])) if n_cov is None else int(n_cov)
+        self.grouping = int(grouping)
+        g = self.grouping == KVC_GROUP_LAYER
+        self.r = 0 if basis_k is None else int(basis_k.shape[1 if g else 2])
+        self.n_cov = (0 if coeff_k is None else int(coeff_k.shape[1 if g else 2])) if n_cov is None else int(n_cov)
         if self.r > 0:
             assert basis_k.is_contiguous() and basis_v.is_contiguous() and basis_k.dtype == basis_v.dtype
             assert basis_k.dtype in (torch.float32, torch.bfloat16)
         if self.r > 0 and self.n_cov > 0:
             assert coeff_k.dtype == torch.float32 and coeff_v.dtype == torch.float32
             assert coeff_k.is_contiguous() and coeff_v.is_contiguous()
-            assert int(coeff_k.shape[2]) == self.n_cov and int(coeff_k.shape[3]) == self.r
+            assert int(coeff_k.shape[-2]) == self.n_cov and int(coeff_k.shape[-1]) == self.r
 
     @staticmethod
     def empty() -> "State":
@@ -206,6 +210,7 @@ class State:
         ptr = lambda t: 0 if t is None else t.data_ptr()
         s.coeff_k, s.coeff_v, s.basis_k, s.basis_v = ptr(self.coeff_k), ptr(self.coeff_v), ptr(self.basis_k), ptr(self.basis_v)
         s.r, s.n_cov = self.r, self.n_cov
+        s.grouping = getattr(self, "grouping", KVC_GROUP_HEAD)
         b = self.basis_k if self.basis_k is not None else self.basis_v
         s.basis_dtype = KVC_BF16 if (b is not None and b.dtype == torch.bfloat16) else KVC_F32
         return s
@@ -350,6 +355,8 @@ KVC_MAX_ANCHORS = 16
 def kvc_state_realign(st: State, shift: int, rope: Rope, out: Optional[torch.Tensor] = None, stream=None) -> State:
     """A state whose key correction is re-aligned by `shift` positions: basis_k rows rotated (into `out`,
     a new tensor by default; pass st.basis_k for in place); coefficients and value factors are shared."""
+    if getattr(st, "grouping", KVC_GROUP_HEAD) == KVC_GROUP_LAYER:
+        raise KvcError(KVC_E_UNSUPPORTED, "kvc_state_realign on a per-layer state: pass its geometry through the C call")
     L, H, r, d = (int(x) for x in st.basis_k.shape)
     out = torch.empty_like(st.basis_k) if out is None else out
     s, rp = st.struct(), rope.struct()

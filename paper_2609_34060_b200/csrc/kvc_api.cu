@@ -72,6 +72,7 @@ static int resolve_state(const kvc_state* st, int for_update, DevState* out) {
   if (st->r < 0 || st->n_cov < 0) return KVC_E_INVALID_ARG;
   if (st->r > 256) return KVC_E_UNSUPPORTED;
   if (st->basis_dtype != KVC_F32 && st->basis_dtype != KVC_BF16) return KVC_E_INVALID_ARG;
+  if (st->grouping != KVC_GROUP_HEAD && st->grouping != KVC_GROUP_LAYER) return KVC_E_INVALID_ARG;
   const bool live = st->r > 0 && st->n_cov > 0;
   if (live || (for_update && st->r > 0)) {
     if (!st->basis_k || !st->basis_v) return KVC_E_INVALID_ARG;
@@ -88,7 +89,7 @@ static int resolve_state(const kvc_state* st, int for_update, DevState* out) {
   d.r = st->r;
   d.n_cov = st->n_cov;
   d.basis_bf16 = st->basis_dtype == KVC_BF16;
-  d.pad = 0;
+  d.grouped = st->grouping == KVC_GROUP_LAYER;
   *out = d;
   return KVC_OK;
 }
@@ -268,6 +269,7 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   if (st->r == 0 || st->n_cov == 0) return KVC_OK;   // nothing to compute
   if (!st->coeff_k || !st->coeff_v) return KVC_E_INVALID_ARG;
   if (mode == KVC_FIT && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
+  if (mode == KVC_FIT && st->grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;   // needs a (H d) x (H d) eigensolver
   if (mode == KVC_FIT) {
     const size_t need = kvc_workspace_bytes(tgt, st, mode);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_E_WORKSPACE;
@@ -324,7 +326,13 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   U.L = tgt->L;
   U.H = tgt->H;
   U.status = status;
+  U.grouped = dst_state.grouped;
   rope_tables(rope, d, shift, U.cs, U.sn);
+  if (U.grouped) {      // every head adds its share: start from zero
+    const size_t nbytes = (size_t)tgt->L * st->n_cov * st->r * sizeof(float);
+    if (cudaMemsetAsync(st->coeff_k, 0, nbytes, s) != cudaSuccess || cudaMemsetAsync(st->coeff_v, 0, nbytes, s) != cudaSuccess)
+      return KVC_E_CUDA;
+  }
   if (tl_path_force != KVC_PATH_GENERIC) {
     const int trc = tc_project(U, d, s);
     if (trc == KVC_OK) {
@@ -431,6 +439,7 @@ int kvc_apply_multi(const kvc_cache* src, const kvc_state* deltas, int32_t n_anc
   int live = 0;
   for (int v = 0; v < n_anchors; ++v) {
     if ((rc = resolve_state(&deltas[v], 0, &st[v])) != KVC_OK) return rc;
+    if (st[v].grouped) return KVC_E_UNSUPPORTED;
     if (deltas[v].r > 0 && deltas[v].n_cov > src->T) return KVC_E_SHAPE;
     live += deltas[v].r > 0 && deltas[v].n_cov > 0;
   }
@@ -488,6 +497,7 @@ int kvc_token_weights(const kvc_cache* src, int32_t src_pos, const kvc_state* an
   DevState st[KVC_MAX_ANCHORS];
   for (int v = 0; v < n_anchors; ++v) {
     if ((rc = resolve_state(&anchors[v], 0, &st[v])) != KVC_OK) return rc;
+    if (st[v].grouped) return KVC_E_UNSUPPORTED;
     if (anchors[v].r <= 0 || anchors[v].n_cov < 0 || anchors[v].n_cov > src->T) return KVC_E_SHAPE;
   }
   uint32_t* status = status_ptr();
@@ -539,6 +549,7 @@ int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_
     if (a.n_cov < k) return KVC_E_SHAPE;            // not compatible at this comparison length
     if (k > 0 && (!a.coeff_v || !a.basis_v)) return KVC_E_INVALID_ARG;
     if (a.basis_dtype != KVC_F32 && a.basis_dtype != KVC_BF16) return KVC_E_INVALID_ARG;
+    if (a.grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(a.coeff_v) | reinterpret_cast<uintptr_t>(a.basis_v)) & 15) return KVC_E_UNSUPPORTED;
   }
   if (reinterpret_cast<uintptr_t>(dist_sq) & 7) return KVC_E_INVALID_ARG;
@@ -627,7 +638,8 @@ int64_t kvc_apply_bytes(const kvc_cache* src, const kvc_state* st) {
   const int64_t slabs = (int64_t)src->L * src->H * 2;
   const int64_t cache = slabs * src->T * src->d * 2;          // read once, written once
   const bool live = st->r > 0 && st->n_cov > 0;
-  const int64_t coeff = live ? slabs * st->n_cov * st->r * 4 : 0;
+  const int64_t cslabs = st->grouping == KVC_GROUP_LAYER ? (int64_t)src->L * 2 : slabs;   // coefficients shared by the heads
+  const int64_t coeff = live ? cslabs * st->n_cov * st->r * 4 : 0;
   const int64_t basis = live ? slabs * st->r * src->d * (st->basis_dtype == KVC_BF16 ? 2 : 4) : 0;
   return 2 * cache + coeff + basis;
 }
@@ -636,7 +648,8 @@ int64_t kvc_update_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode
   if (!tgt || !st) return 0;
   const int64_t slabs = (int64_t)tgt->L * tgt->H * 2;
   const int64_t rows = slabs * st->n_cov * tgt->d * 2 * (has_src ? 2 : 1);   // src + tgt rows
-  const int64_t coeff = slabs * st->n_cov * st->r * 4;
+  const int64_t cslabs = st->grouping == KVC_GROUP_LAYER ? (int64_t)tgt->L * 2 : slabs;
+  const int64_t coeff = cslabs * st->n_cov * st->r * 4;
   const int64_t basis = slabs * st->r * tgt->d * (st->basis_dtype == KVC_BF16 ? 2 : 4);
   int64_t b = rows + coeff + basis;                                          // projection pass
   if (mode == KVC_FIT) b += rows + 2 * slabs * tgt->d * tgt->d * 4;          // Gram pass + G write/read

@@ -23,8 +23,16 @@ struct DevState {
   const float* coeff_v;
   const void* basis_k;
   const void* basis_v;
-  int32_t r, n_cov, basis_bf16, pad;
+  int32_t r, n_cov, basis_bf16, grouped;   // grouped: one state per layer, coeff [L,n_cov,r], basis [L,r,H*d]
 };
+
+// Index of the coefficient slab and element offset of basis row q of (layer l, head h), in elements.
+__host__ __device__ __forceinline__ int64_t coeff_slab(const DevState& st, int l, int h, int H) {
+  return st.grouped ? (int64_t)l : (int64_t)l * H + h;
+}
+__host__ __device__ __forceinline__ int64_t basis_row_off(const DevState& st, int l, int h, int H, int q, int D) {
+  return st.grouped ? (((int64_t)l * st.r + q) * H + h) * D : (((int64_t)l * H + h) * st.r + q) * D;
+}
 
 // One hop over one request: what kvc_apply does for all (layer, head, token).
 // 16-byte aligned so that the cos / sin tables can be read as float4 wherever the
@@ -54,6 +62,7 @@ struct UpdateLaunch {
   int32_t r, n_cov, basis_bf16, pairing;
   int32_t shift, L, H, tiles_per_slab;
   uint32_t* status;
+  int32_t grouped, pad;        // grouped: one state per layer; the heads' projections are ADDED into coeff [L,n_cov,r]
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];
 };

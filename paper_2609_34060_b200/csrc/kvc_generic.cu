@@ -103,18 +103,17 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
     const void* basis = is_v ? it.st.basis_v : it.st.basis_k;
     for (int q0 = 0; q0 < r; q0 += RC) {
       const int rc = min(RC, r - q0);
-      const int64_t boff = ((int64_t)slab * r + q0) * D;
-      if (it.st.basis_bf16) {
-        const __nv_bfloat16* b = reinterpret_cast<const __nv_bfloat16*>(basis) + boff;
-        for (int i = tid; i < rc * D; i += 256) basis_s[i] = __bfloat162float(b[i]);
-      } else {
-        const float* b = reinterpret_cast<const float*>(basis) + boff;
-        for (int i = tid; i < rc * D; i += 256) basis_s[i] = b[i];
+      for (int i = tid; i < rc * D; i += 256) {
+        const int q = i / D, ch = i - q * D;
+        const int64_t off = basis_row_off(it.st, l, h, it.H, q0 + q, D) + ch;
+        basis_s[i] = it.st.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
+                                      : reinterpret_cast<const float*>(basis)[off];
       }
+      const int64_t cslab = coeff_slab(it.st, l, h, it.H);
       for (int i = tid; i < TILE * rc; i += 256) {
         const int tl = i / rc, q = i - tl * rc;
         const int t = t0 + tl;
-        coeff_s[tl * (RC + 1) + q] = (t < n_cov) ? coeff[((int64_t)slab * it.st.n_cov + t) * r + q0 + q] : 0.f;
+        coeff_s[tl * (RC + 1) + q] = (t < n_cov) ? coeff[(cslab * it.st.n_cov + t) * r + q0 + q] : 0.f;
       }
       __syncthreads();
       for (int q = 0; q < rc; ++q) {
@@ -252,7 +251,7 @@ __global__ void __launch_bounds__(256) project_generic_kernel(const __grid_const
       const int q = i / D, c = i % D;
       float b = 0.f;
       if (q0 + q < p.r) {
-        const int64_t off = ((int64_t)slab * p.r + q0 + q) * D + c;
+        const int64_t off = (p.grouped ? (((int64_t)l * p.r + q0 + q) * p.H + h) : ((int64_t)slab * p.r + q0 + q)) * D + c;
         b = p.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
                          : reinterpret_cast<const float*>(basis)[off];
       }
@@ -279,7 +278,10 @@ __global__ void __launch_bounds__(256) project_generic_kernel(const __grid_const
 #pragma unroll
       for (int a = 0; a < 8; ++a) {
         const int t = t0 + warp * 8 + a;
-        if (t < n_cov) coeff[((int64_t)slab * n_cov + t) * p.r + q0 + lane] = acc[a];
+        if (t < n_cov) {
+          if (p.grouped) atomicAdd(&coeff[((int64_t)l * n_cov + t) * p.r + q0 + lane], acc[a]);   // sum over the heads
+          else coeff[((int64_t)slab * n_cov + t) * p.r + q0 + lane] = acc[a];
+        }
       }
     }
   }

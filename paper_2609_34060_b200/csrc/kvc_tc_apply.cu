@@ -324,11 +324,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           ok = mbar_wait(smem_u32(&ctrl->cempty[bc]), ((bpos / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
           if (ok) {
             const uint32_t row_bytes = it.st.basis_bf16 ? 256u : 512u;
-            const uint8_t* src = reinterpret_cast<const uint8_t*>(t.is_v ? it.st.basis_v : it.st.basis_k) +
-                                 (size_t)t.slab * it.st.r * row_bytes;
+            const uint8_t* bbase = reinterpret_cast<const uint8_t*>(t.is_v ? it.st.basis_v : it.st.basis_k);
             const uint32_t bbar = smem_u32(&ctrl->cfull[bc]);
             mbar_expect_tx(bbar, it.st.r * row_bytes);
-            bulk_load_1d(coeffs + bc * kCoeffSlotBytes, src, it.st.r * row_bytes, bbar);
+            if (!it.st.grouped) {
+              bulk_load_1d(coeffs + bc * kCoeffSlotBytes, bbase + (size_t)t.slab * it.st.r * row_bytes, it.st.r * row_bytes, bbar);
+            } else {                                // one state per layer: this head's d columns of every basis row
+              for (int q = 0; q < it.st.r; ++q)
+                bulk_load_1d(coeffs + bc * kCoeffSlotBytes + q * row_bytes,
+                             bbase + (((size_t)t.l * it.st.r + q) * it.H + t.h) * row_bytes, row_bytes, bbar);
+            }
           }
         }
         if (ok) ok = mbar_wait(smem_u32(&ctrl->cempty[c]), ((cpos / NSC) & 1u) ^ 1u, abort_flag) ? 1 : 0;
@@ -339,7 +344,9 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             const CUtensorMap* cmap = t.is_v ? &t.mp->coeff_v : &t.mp->coeff_k;
 #pragma unroll
             for (int b = 0; b < RB; ++b)
-              if (b < t.nb) tma_load_3d(coeffs + c * kCoeffSlotBytes + b * kCoeffBlkBytes, cmap, cbar, 32 * b, t.t0, t.slab);
+              if (b < t.nb)
+                tma_load_3d(coeffs + c * kCoeffSlotBytes + b * kCoeffBlkBytes, cmap, cbar, 32 * b, t.t0,
+                            it.st.grouped ? t.l : t.slab);
           }
           ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
         }
@@ -792,8 +799,9 @@ static bool item_supported(const DevItem& it, int d) {
 static bool build_maps(const DevItem& it, ItemMaps* mp) {
   bool ok = encode_cache(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
             encode_cache(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
-  ok = ok && encode_coeff(&mp->coeff_k, it.st.coeff_k, it.st.r, it.st.n_cov, it.L * it.H) &&
-       encode_coeff(&mp->coeff_v, it.st.coeff_v, it.st.r, it.st.n_cov, it.L * it.H);
+  const int cslabs = it.st.grouped ? it.L : it.L * it.H;
+  ok = ok && encode_coeff(&mp->coeff_k, it.st.coeff_k, it.st.r, it.st.n_cov, cslabs) &&
+       encode_coeff(&mp->coeff_v, it.st.coeff_v, it.st.r, it.st.n_cov, cslabs);
   return ok;
 }
 

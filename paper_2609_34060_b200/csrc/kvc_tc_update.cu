@@ -52,6 +52,12 @@ struct ProjectTcLaunch {
   UpdMaps maps;
 };
 
+// element-wise float32 add of a shared-memory tile into global memory
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
@@ -268,7 +274,10 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
         const CUtensorMap* cmap = t.is_v ? &p.maps.coeff_v : &p.maps.coeff_k;
         const uint32_t st_base = stages + s * kStageBytes;
 #pragma unroll
-        for (int b = 0; b < RB; ++b) tma_store_3d(cmap, st_base + b * kHalfBytes, 32 * b, t.t0, t.slab);
+        for (int b = 0; b < RB; ++b) {
+          if (u.grouped) tma_reduce_add_3d(cmap, st_base + b * kHalfBytes, 32 * b, t.t0, t.l);   // sum over the heads of a layer
+          else tma_store_3d(cmap, st_base + b * kHalfBytes, 32 * b, t.t0, t.slab);
+        }
         tma_store_commit();
         tma_store_wait_read();
         mbar_arrive(smem_u32(&ctrl->empty[s]));
@@ -294,7 +303,7 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
 #pragma unroll
         for (int k = 0; k < 8; ++k) v[k] = w[k] = 0.f;
         if (row < u.r) {
-          const int64_t off = ((int64_t)t.slab * u.r + row) * 128;
+          const int64_t off = (u.grouped ? (((int64_t)t.l * u.r + row) * u.H + t.h) : ((int64_t)t.slab * u.r + row)) * 128;
           auto load8 = [&](int chunk, float* o) {
             if (u.basis_bf16) {
               unpack8(*reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(basis) + off + 8 * chunk), o);
@@ -773,8 +782,9 @@ int tc_project(const UpdateLaunch& U, int d, cudaStream_t s) {
   bool ok = tc::encode_cache(&L.maps.tgt_k, U.tgt, U.tgt.k, U.L, U.H) && tc::encode_cache(&L.maps.tgt_v, U.tgt, U.tgt.v, U.L, U.H);
   if (L.has_src)
     ok = ok && tc::encode_cache(&L.maps.src_k, U.src, U.src.k, U.L, U.H) && tc::encode_cache(&L.maps.src_v, U.src, U.src.v, U.L, U.H);
-  ok = ok && tc::encode_coeff(&L.maps.coeff_k, U.coeff_k, U.r, U.n_cov, U.L * U.H) &&
-       tc::encode_coeff(&L.maps.coeff_v, U.coeff_v, U.r, U.n_cov, U.L * U.H);
+  const int cslabs = U.grouped ? U.L : U.L * U.H;
+  ok = ok && tc::encode_coeff(&L.maps.coeff_k, U.coeff_k, U.r, U.n_cov, cslabs) &&
+       tc::encode_coeff(&L.maps.coeff_v, U.coeff_v, U.r, U.n_cov, cslabs);
   if (!ok) return KVC_E_CUDA;
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;

@@ -59,7 +59,8 @@ def to_dev(c_cpu: "kvc.Cache", dev) -> "kvc.Cache":
 
 def state_to_dev(s: "kvc.State", dev) -> "kvc.State":
     mv = lambda t: None if t is None else t.to(dev)
-    return kvc.State(mv(s.coeff_k), mv(s.coeff_v), mv(s.basis_k), mv(s.basis_v), n_cov=s.n_cov)
+    return kvc.State(mv(s.coeff_k), mv(s.coeff_v), mv(s.basis_k), mv(s.basis_v), n_cov=s.n_cov,
+                     grouping=getattr(s, "grouping", kvc.KVC_GROUP_HEAD))
 
 
 def make_cache(cfg: wl.Config, table_tag=0, extra_pages=3):

@@ -1,0 +1,162 @@
+"""GPU parity of the per-layer feature grouping (D = H d, Sec. 3.1): one state per layer whose
+coefficients are shared by the KV heads.  The oracle expands the grouped state into the
+per-(layer, head) form (the two define the same low-rank product) and applies / projects as usual."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_34060_b200 as kvc
+from paper_2609_34060_b200 import workloads as wl
+from oracle import kvc_oracle as orc
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+CFG_S = wl.CONFIGS["llama8b_8k"].scaled(name="8b_small", L=2, H=4, T=900)
+CFG_P = wl.CONFIGS["vlm_16k"].scaled(name="vlm_small", L=2, H=2, T=1301, image_spans=())
+CFG_R64 = wl.CONFIGS["llama70b_32k"].scaled(name="r64_small", L=1, H=3, T=515)
+CFG_T = wl.CONFIGS["tiny"]
+
+PATHS = [kvc.KVC_PATH_GENERIC, kvc.KVC_PATH_AUTO]
+PATH_IDS = ["generic", "auto"]
+
+
+@pytest.fixture(autouse=True)
+def _reset_path():
+    kvc.kvc_status_reset()
+    yield
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    assert kvc.kvc_status_poll() == 0
+
+
+def _grouped_state(cfg, hop, n_cov=None, basis_dtype=torch.float32):
+    """Seeded draws: coefficients [L, n_cov, r], orthonormal basis rows in R^{H d} as [L, r, H d]."""
+    n = cfg.T if n_cov is None else n_cov
+    one = cfg.scaled(H=1, d=cfg.H * cfg.d)              # the generator's per-"head" draw at D = H d
+    ck = wl.coefficients(cfg.L, 1, cfg.T, cfg.r, cfg.seed, 4 * hop + 0, "cpu")[:, 0, :n].contiguous()
+    cv = wl.coefficients(cfg.L, 1, cfg.T, cfg.r, cfg.seed, 4 * hop + 1, "cpu")[:, 0, :n].contiguous()
+    bk = wl.orthonormal_basis(cfg.L, 1, cfg.r, one.d, cfg.seed, 4 * hop + 2, "cpu")[:, 0].contiguous().to(basis_dtype)
+    bv = wl.orthonormal_basis(cfg.L, 1, cfg.r, one.d, cfg.seed, 4 * hop + 3, "cpu")[:, 0].contiguous().to(basis_dtype)
+    return kvc.State(ck, cv, bk, bv, n_cov=n, grouping=kvc.KVC_GROUP_LAYER)
+
+
+def _oracle_state(cfg, st):
+    f = lambda t: t.to(torch.float32).numpy()
+    return orc.ungroup_state(f(st.coeff_k), f(st.coeff_v), f(st.basis_k), f(st.basis_v), cfg.H, n_cov=st.n_cov)
+
+
+def _check(dst, odst, ref_k, ref_v):
+    gk, gv = hp.logical_bits(dst, "k"), hp.logical_bits(dst, "v")
+    assert hp.tol_ratio(gk, ref_k) <= 1.0 and hp.tol_ratio(gv, ref_v) <= 1.0
+    assert hp.ulp_mismatch_fraction(gk, hp.logical_bits(odst, "k")) < 1e-2
+    assert hp.ulp_mismatch_fraction(gv, hp.logical_bits(odst, "v")) < 1e-2
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("cfg", [CFG_S, CFG_P, CFG_R64, CFG_T], ids=lambda c: c.name)
+def test_grouped_apply(cfg, path):
+    kvc.kvc_set_path(path)
+    src_cpu = hp.make_cache(cfg)
+    for n_cov, shift in ((cfg.T, 77), (cfg.T // 2 + 3, 0)):
+        st = _grouped_state(cfg, 1, n_cov=n_cov)
+        src = hp.to_dev(src_cpu, DEV)
+        dst = hp.empty_dst(src_cpu, cfg, DEV, fill=3.0)
+        kvc.kvc_apply(src, hp.state_to_dev(st, DEV), shift, kvc.Rope(cfg.theta), dst)
+        torch.cuda.synchronize()
+        if path == kvc.KVC_PATH_AUTO and cfg.d == 128:
+            assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+        osrc = hp.oracle_cache(src_cpu)
+        odst = osrc.empty_like(page_table=None if dst.page_table is None else dst.page_table.cpu().numpy())
+        odst, rk, rv = orc.apply(osrc, _oracle_state(cfg, st), shift, hp.inv_freq(cfg), dst=odst, want_ref=True)
+        _check(dst, odst, rk, rv)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_grouped_chain_and_batch(path):
+    cfg = CFG_S.scaled(T=400)
+    kvc.kvc_set_path(path)
+    rope = kvc.Rope(cfg.theta)
+    pl = [100, 180, 140]
+    src_cpu = hp.make_cache(cfg)
+    src = hp.to_dev(src_cpu, DEV)
+    states = [_grouped_state(cfg, a) for a in (1, 2)]
+    dev_states = [hp.state_to_dev(s, DEV) for s in states]
+    outs = [hp.empty_dst(src_cpu, cfg, DEV) for _ in range(2)]
+    kvc.kvc_chain(src, pl, dev_states, rope, outs)
+    torch.cuda.synchronize()
+    ocur = hp.oracle_cache(src_cpu)
+    for a in (1, 2):
+        onext, rk, rv = orc.apply(ocur, _oracle_state(cfg, states[a - 1]), pl[a] - pl[a - 1], hp.inv_freq(cfg), want_ref=True)
+        if a == 1:
+            _check(outs[0], onext, rk, rv)
+        ocur = onext
+    # the chain equals its hops one by one, bit for bit; a ragged batch of the same hops too
+    one = hp.empty_dst(src_cpu, cfg, DEV)
+    kvc.kvc_apply(outs[0], dev_states[1], pl[2] - pl[1], rope, one)
+    torch.cuda.synchronize()
+    assert torch.equal(one.k, outs[1].k) and torch.equal(one.v, outs[1].v)
+    bd = [hp.empty_dst(src_cpu, cfg, DEV) for _ in range(2)]
+    items = [kvc.Item(src, bd[0], dev_states[0], pl[1] - pl[0]), kvc.Item(outs[0], bd[1], dev_states[1], pl[2] - pl[1])]
+    nb = kvc.kvc_batch_workspace_bytes(2)
+    ws = torch.empty(nb, dtype=torch.uint8, device=DEV)
+    stg = torch.empty(nb, dtype=torch.uint8).pin_memory()
+    kvc.kvc_apply_batch(items, rope, ws, stg)
+    torch.cuda.synchronize()
+    assert torch.equal(bd[0].k, outs[0].k) and torch.equal(bd[1].v, outs[1].v)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("cfg", [CFG_S, CFG_P, CFG_T], ids=lambda c: c.name)
+def test_grouped_project(cfg, path):
+    """coeff[l, t, :] = sum over heads of (tgt - Rot(src))[l, h, t, :] . basis[l][:, h d : (h+1) d]^T."""
+    kvc.kvc_set_path(path)
+    rope = kvc.Rope(cfg.theta)
+    inv = hp.inv_freq(cfg)
+    shift = 51
+    src_cpu = hp.make_cache(cfg)
+    tgt_cpu = hp.make_cache(cfg.scaled(seed=cfg.seed + 3))
+    if src_cpu.page_table is not None:       # same geometry, another table
+        tgt_cpu = hp.make_cache(cfg.scaled(seed=cfg.seed + 3), table_tag=9)
+    given = _grouped_state(cfg, 2)
+    n = cfg.T - 37
+    st = kvc.State(torch.full((cfg.L, n, cfg.r), 7.0, device=DEV), torch.full((cfg.L, n, cfg.r), 7.0, device=DEV),
+                   given.basis_k.to(DEV), given.basis_v.to(DEV), n_cov=n, grouping=kvc.KVC_GROUP_LAYER)
+    kvc.kvc_state_update(hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV), shift, rope, st, kvc.KVC_PROJECT)
+    torch.cuda.synchronize()
+    if path == kvc.KVC_PATH_AUTO and cfg.d == 128:
+        assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+    osrc, otgt = hp.oracle_cache(src_cpu), hp.oracle_cache(tgt_cpu)
+    for which, got, basis in (("k", st.coeff_k, given.basis_k), ("v", st.coeff_v, given.basis_v)):
+        g = got.cpu().numpy().astype(np.float64)
+        for l in range(cfg.L):
+            deltas = [orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, inv, which == "k")[:n]
+                      for h in range(cfg.H)]
+            ref = orc.project_grouped(deltas, basis[l].numpy())
+            # the per-head bound of the projection, summed over the heads
+            bn = np.linalg.norm(basis[l].numpy().astype(np.float64).reshape(cfg.r, cfg.H, cfg.d), axis=2)   # [r, H]
+            tol = 1e-6 * np.ones_like(ref)
+            for h in range(cfg.H):
+                xs = np.linalg.norm(orc.bf16_to_f64(osrc.get_bits(which, l, h))[:n], axis=1)
+                xt = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h))[:n], axis=1)
+                dn = np.linalg.norm(deltas[h], axis=1)
+                tol += (2.0 ** -12 * dn + 2.0 ** -18 * (xs + xt))[:, None] * bn[None, :, h]
+            assert np.all(np.abs(g[l] - ref) <= tol), (which, l, float(np.max(np.abs(g[l] - ref) / tol)))
+
+
+def test_grouped_is_rejected_where_it_is_not_served():
+    cfg = CFG_S.scaled(T=200)
+    st = hp.state_to_dev(_grouped_state(cfg, 1), DEV)
+    src = hp.to_dev(hp.make_cache(cfg), DEV)
+    d2 = torch.zeros(1, dtype=torch.float64, device=DEV)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_gate_distance(src, [st], cfg.T, d2)
+    assert e.value.code == kvc.KVC_E_UNSUPPORTED
+    ws = torch.empty(1 << 24, dtype=torch.uint8, device=DEV)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_state_update(None, src, 0, kvc.Rope(cfg.theta), st, kvc.KVC_FIT, workspace=ws)
+    assert e.value.code == kvc.KVC_E_UNSUPPORTED
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_apply_multi(src, [st], None, None, 0, kvc.Rope(cfg.theta), src, ws)
+    assert e.value.code == kvc.KVC_E_UNSUPPORTED

@@ -315,3 +315,28 @@ def test_realign_basis_pins():
     delta_0 = orc.rope_shift(tgt, -p_t, inv) - orc.rope_shift(src, -p_s, inv)  # both sides canonical
     assert np.allclose(orc.rope_shift(delta_t, -p_t, inv), delta_0, atol=1e-12)
     assert np.allclose(delta_t @ Q.T, delta_0 @ orc.realign_basis(Q, -p_t, inv).T, atol=1e-12)
+
+
+def test_grouped_state_pins():
+    """D = H d: the grouped state is the plain low-rank product on the concatenated feature axis."""
+    rng = np.random.default_rng(8)
+    L, H, T, d, r = 2, 3, 5, 4, 2
+    ck, cv = rng.standard_normal((L, T, r)), rng.standard_normal((L, T, r))
+    bk, bv = rng.standard_normal((L, r, H * d)), rng.standard_normal((L, r, H * d))
+    st = orc.ungroup_state(ck, cv, bk, bv, H)
+    assert st.coeff_k.shape == (L, H, T, r) and st.basis_k.shape == (L, H, r, d)
+    for l in range(L):
+        z = cv[l] @ bv[l]                                             # [T, H d]
+        per_head = np.concatenate([st.coeff_v[l, h] @ st.basis_v[l, h] for h in range(H)], axis=1)
+        assert np.allclose(z, per_head, atol=1e-12)
+    # the projection of a concatenated deviation is the sum of the heads' projections
+    delta = [rng.standard_normal((T, d)) for _ in range(H)]
+    c = orc.project_grouped(delta, bk[0])
+    by_head = sum(orc.project(delta[h], st.basis_k[0, h]) for h in range(H))
+    assert np.allclose(c, by_head, atol=1e-12)
+    # orthonormal rows in R^{H d}: projecting c @ B gives c back
+    Q = np.linalg.qr(rng.standard_normal((H * d, r)))[0].T
+    z = ck[0] @ Q
+    assert np.allclose(orc.project_grouped([z[:, h * d:(h + 1) * d] for h in range(H)], Q), ck[0], atol=1e-12)
+    # compactness (Sec. 3.1): float32 coefficients of a grouped state take r*4 / (H*d*2) of the bf16 cache
+    assert math.isclose((r * 4) / (H * d * 2), 8 / 24)
