@@ -272,6 +272,21 @@ int kvc_apply_multi(const kvc_cache *src, const kvc_state *deltas, int32_t n_anc
 size_t kvc_multi_workspace_bytes(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors);
 
 /*
+ * Effective rank (Sec. 3.1: "the minimum rank retaining 90% of the singular-value energy"), from the
+ * eigenvalues a KVC_FIT update leaves in its workspace (squared singular values of the factorised
+ * deviation or cache).  For every matrix m of n_matrices:
+ *     rank[m] = min { k : sum_{i<k} max(evals[m][i], 0) >= energy * sum_i max(evals[m][i], 0) }   (0 if the sum is 0)
+ *   evals   DEVICE float32 [n_matrices][d], each row descending (kvc_fit_eigenvalues(...) points at
+ *           them inside a FIT workspace: n_matrices = L*H*2, ordered (layer, head, K|V))
+ *   energy  in (0, 1], e.g. 0.9
+ *   rank    DEVICE int32 [n_matrices]
+ * Sums in float64.
+ */
+int kvc_effective_rank(const float *evals, int32_t n_matrices, int32_t d, double energy, int32_t *rank, void *stream);
+/* Address of the eigenvalues inside a KVC_FIT workspace of kvc_state_update for `tgt` (NULL on bad arguments). */
+const float *kvc_fit_eigenvalues(const kvc_cache *tgt, const void *workspace);
+
+/*
  * Positional re-alignment of a stored correction (App. A.2: a correction for a recurring prefix
  * relation "is profiled once, stored in low-rank form, and positionally re-aligned when reused").
  * A rotation is linear in the channels, Rot_s(c . B) = c . Rot_s(B), so re-aligning a stored key

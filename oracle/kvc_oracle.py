@@ -460,6 +460,19 @@ def stack_anchors(weights, coeffs, bases):
     return c, b
 
 
+def effective_rank(eigenvalues, energy=0.9):
+    """Sec. 3.1 (figure on effective rank): the minimum rank that retains `energy` (90 %) of the
+    singular-value energy, the energy of a matrix being the sum of its squared singular values =
+    the sum of the eigenvalues of its Gram matrix.  eigenvalues: 1-D, any order, negatives (rounding)
+    count as zero.  A zero matrix has effective rank 0."""
+    w = np.sort(np.clip(np.asarray(eigenvalues, np.float64), 0.0, None))[::-1]
+    total = float(np.sum(w))
+    if total <= 0.0:
+        return 0
+    acc = np.cumsum(w)
+    return int(np.searchsorted(acc, energy * total, side="left") + 1)
+
+
 def ungroup_state(coeff_k, coeff_v, basis_k, basis_v, H, n_cov=None):
     """Sec. 3.1 with D = H d (one state per layer over all KV heads): coeff [L, n_cov, r] is shared by
     the heads of a layer and basis [L, r, H d] holds head h's part in columns h d .. (h+1) d - 1.

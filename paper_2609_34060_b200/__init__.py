@@ -33,7 +33,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues",
 )
 
 
@@ -91,6 +91,9 @@ def load(path: Optional[str] = None):
     lib.kvc_apply_multi.argtypes = [PC, PS, i32, vp, vp, i32, PR, PC, vp, sz, vp]
     lib.kvc_multi_workspace_bytes.argtypes = [PC, PS, i32]
     lib.kvc_multi_workspace_bytes.restype = sz
+    lib.kvc_effective_rank.argtypes = [vp, i32, i32, C.c_double, vp, vp]
+    lib.kvc_fit_eigenvalues.argtypes = [PC, vp]
+    lib.kvc_fit_eigenvalues.restype = vp
     lib.kvc_state_realign.argtypes = [PS, i32, i32, i32, i32, PR, vp, vp]
     lib.kvc_token_weights.argtypes = [PC, i32, PS, C.POINTER(i32), i32, PR, C.c_double, vp, vp, vp, sz, vp]
     lib.kvc_token_weights_workspace_bytes.argtypes = [PC, i32]
@@ -350,6 +353,16 @@ def kvc_apply_multi(src: Cache, deltas: Sequence[State], w_k: Optional[torch.Ten
 
 
 KVC_MAX_ANCHORS = 16
+
+
+def kvc_effective_rank(tgt: Cache, workspace: torch.Tensor, energy: float = 0.9, stream=None) -> torch.Tensor:
+    """Effective ranks int32 [L, H, 2] (K, V) from the eigenvalues a FIT update left in `workspace`."""
+    c = tgt.struct()
+    ev = load().kvc_fit_eigenvalues(C.byref(c), workspace.data_ptr())
+    out = torch.empty(tgt.L, tgt.H, 2, dtype=torch.int32, device=workspace.device)
+    _check(load().kvc_effective_rank(ev, tgt.L * tgt.H * 2, tgt.d, float(energy), out.data_ptr(), _stream(stream)),
+           "kvc_effective_rank")
+    return out
 
 
 def kvc_state_realign(st: State, shift: int, rope: Rope, out: Optional[torch.Tensor] = None, stream=None) -> State:

@@ -454,6 +454,18 @@ int kvc_apply_multi(const kvc_cache* src, const kvc_state* deltas, int32_t n_anc
   return rc;
 }
 
+int kvc_effective_rank(const float* evals, int32_t n_matrices, int32_t d, double energy, int32_t* rank, void* stream) {
+  if (!evals || !rank || n_matrices < 0 || d <= 0 || !(energy > 0.0) || energy > 1.0) return KVC_E_INVALID_ARG;
+  if (launch_effective_rank(evals, n_matrices, d, (float)energy, rank, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return KVC_E_CUDA;
+  return KVC_OK;
+}
+
+const float* kvc_fit_eigenvalues(const kvc_cache* tgt, const void* workspace) {
+  if (!tgt || !workspace || tgt->L <= 0 || tgt->H <= 0 || tgt->d <= 0) return nullptr;
+  return reinterpret_cast<const float*>(workspace) + 2 * (size_t)tgt->L * tgt->H * 2 * tgt->d * tgt->d;
+}
+
 int kvc_state_realign(const kvc_state* st, int32_t L, int32_t H, int32_t d, int32_t shift, const kvc_rope* rope,
                       void* basis_k_out, void* stream) {
   if (!st || L <= 0 || H <= 0 || st->r < 0) return KVC_E_INVALID_ARG;

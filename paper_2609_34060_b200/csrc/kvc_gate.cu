@@ -113,6 +113,40 @@ cudaError_t launch_token_weights(const float* scores, const TokenWeightsLaunch& 
   return cudaGetLastError();
 }
 
+// Effective rank (Sec. 3.1): per matrix the minimum rank that keeps `energy` of the sum of its
+// eigenvalues.  One warp per matrix; eigenvalues descending (as the eigensolver leaves them).
+__global__ void __launch_bounds__(128) effective_rank_kernel(const float* evals, int n_mat, int d, float energy, int32_t* out) {
+  const int m = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (m >= n_mat) return;
+  const float* w = evals + (int64_t)m * d;
+  double total = 0.0;
+  for (int i = lane; i < d; i += 32) total += (double)fmaxf(w[i], 0.f);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+  int rank = 0;
+  if (total > 0.0) {
+    const double need = (double)energy * total;
+    double acc = 0.0;                              // running sum, lane 0 walks the (short) list
+    if (lane == 0) {
+      for (int i = 0; i < d; ++i) {
+        acc += (double)fmaxf(w[i], 0.f);
+        if (acc >= need) {
+          rank = i + 1;
+          break;
+        }
+      }
+      if (rank == 0) rank = d;
+    }
+  }
+  if (lane == 0) out[m] = rank;
+}
+
+cudaError_t launch_effective_rank(const float* evals, int n_mat, int d, float energy, int32_t* out, cudaStream_t s) {
+  if (n_mat <= 0) return cudaSuccess;
+  effective_rank_kernel<<<(unsigned)((n_mat + 3) / 4), 128, 0, s>>>(evals, n_mat, d, energy, out);
+  return cudaGetLastError();
+}
+
 // Re-alignment of a stored key correction (App. A.2): every key-basis row rotated by a shift,
 // Rot_s(c . B) = c . Rot_s(B).  One thread per RoPE pair; float32 or bf16 rows of d values.
 __global__ void __launch_bounds__(256) realign_basis_kernel(const RealignLaunch q) {

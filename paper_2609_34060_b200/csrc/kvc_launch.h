@@ -17,6 +17,7 @@ cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s);
 
 // reliability gate (kvc_gate.cu)
 cudaError_t launch_gate_generic(const GateLaunch& g, int d, cudaStream_t s);
+cudaError_t launch_effective_rank(const float* evals, int n_mat, int d, float energy, int32_t* out, cudaStream_t s);
 cudaError_t launch_realign_basis(const RealignLaunch& q, cudaStream_t s);
 cudaError_t launch_token_weights(const float* scores, const TokenWeightsLaunch& q, cudaStream_t s);
 cudaError_t launch_gate_weights(const double* dist_sq, int n, double temperature, double* gw, double* entropy, cudaStream_t s);

@@ -195,3 +195,39 @@ def test_fit_rank_limits(path):
     dl = orc.deviation(osrc.get_bits("k", 0, 0), otgt.get_bits("k", 0, 0), shift, hp.inv_freq(cfg), True)[:n_cov]
     c = st.coeff_k[0, 0].cpu().numpy().astype(np.float64)
     assert np.max(np.abs(c @ B[0, 0] - dl)) <= 1e-3 * np.max(np.abs(dl))
+
+
+def test_effective_rank_from_fit_eigenvalues():
+    """Sec. 3.1's diagnostic on the eigenvalues a FIT leaves behind: a deviation of exact rank 8 plus
+    bf16 rounding noise has effective rank <= 8 at 90 % energy and matches the oracle's count on the
+    oracle's eigenvalues; a flat Gaussian cache (base factorisation) needs most of its 128 directions."""
+    cfg = wl.CONFIGS["llama8b_8k"].scaled(name="er", L=1, H=2, T=512, r=8)
+    rope = kvc.Rope(cfg.theta)
+    src_cpu = hp.make_cache(cfg)
+    osrc = hp.oracle_cache(src_cpu)
+    true = hp.make_state(cfg, hop=1)
+    otgt = orc.apply(osrc, hp.oracle_state(true), 40, hp.inv_freq(cfg))
+    mk = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16)
+    src = hp.to_dev(src_cpu, DEV)
+    tgt = kvc.Cache(mk(otgt.k).to(DEV), mk(otgt.v).to(DEV))
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+    st = kvc.State(torch.empty(L, H, T, r, device=DEV), torch.empty(L, H, T, r, device=DEV),
+                   torch.empty(L, H, r, d, device=DEV), torch.empty(L, H, r, d, device=DEV))
+    ws = torch.empty(kvc.kvc_workspace_bytes(tgt, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(src, tgt, 40, rope, st, kvc.KVC_FIT, workspace=ws)
+    er = kvc.kvc_effective_rank(tgt, ws).cpu().numpy()
+    _, ev = orc.state_update(osrc, otgt, 40, hp.inv_freq(cfg), r=r, mode=orc.FIT)
+    for l in range(L):
+        for h in range(H):
+            for kv in range(2):
+                want = orc.effective_rank(ev[l, h, kv])
+                assert er[l, h, kv] == want and 1 <= want <= 8
+    # base factorisation of the Gaussian cache itself: no low-rank structure
+    kvc.kvc_state_update(None, src, 0, rope, st, kvc.KVC_FIT, workspace=ws)
+    er = kvc.kvc_effective_rank(src, ws).cpu().numpy()
+    for l in range(L):
+        for h in range(H):
+            v = orc.bf16_to_f64(osrc.get_bits("v", l, h))
+            want = orc.effective_rank(np.linalg.eigvalsh(v.T @ v))
+            assert abs(int(er[l, h, 1]) - want) <= 1 and want > 64      # a tie at the 90 % mark may fall either way
+    assert kvc.kvc_effective_rank(src, ws, energy=1.0).max().item() <= d

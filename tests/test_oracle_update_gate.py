@@ -317,6 +317,26 @@ def test_realign_basis_pins():
     assert np.allclose(delta_t @ Q.T, delta_0 @ orc.realign_basis(Q, -p_t, inv).T, atol=1e-12)
 
 
+def test_effective_rank_pins():
+    # one dominant direction: rank 1 keeps it all
+    assert orc.effective_rank([10.0, 0.0, 0.0]) == 1
+    # k equal eigenvalues: 90 % of the energy needs ceil(0.9 k) of them
+    for k in (1, 2, 5, 10, 32):
+        assert orc.effective_rank(np.ones(k)) == math.ceil(0.9 * k - 1e-12)
+    # hand case: energies 50, 30, 15, 5 -> cumulative 50, 80, 95: three directions reach 90 %
+    assert orc.effective_rank([5.0, 50.0, 15.0, 30.0]) == 3
+    assert orc.effective_rank([50.0, 30.0, 10.0, 10.0]) == 3          # exactly 90 % after three
+    assert orc.effective_rank([50.0, 30.0, 15.0, 5.0], energy=0.8) == 2
+    assert orc.effective_rank([0.0, 0.0]) == 0 and orc.effective_rank([-1e-9, 0.0]) == 0
+    # the singular values of a matrix: energy = squared singular values (library SVD)
+    rng = np.random.default_rng(9)
+    m = rng.standard_normal((40, 6)) @ np.diag([9.0, 5.0, 2.0, 1.0, 0.5, 0.1]) @ rng.standard_normal((6, 12))
+    sv = np.linalg.svd(m, compute_uv=False)
+    e = sv ** 2
+    k = orc.effective_rank(np.linalg.eigvalsh(m.T @ m))
+    assert e[:k].sum() >= 0.9 * e.sum() > e[:k - 1].sum()
+
+
 def test_grouped_state_pins():
     """D = H d: the grouped state is the plain low-rank product on the concatenated feature axis."""
     rng = np.random.default_rng(8)
