@@ -302,7 +302,10 @@ def run_step(W, kvc, ev=None):
             mark("update_end")
     if only != "update":
         mark("chain_begin")
-        kvc.kvc_chain(W["true"][0], pl, W["states"], rope, W["outs"])
+        if W.get("chain_ws") is not None:
+            kvc.kvc_chain_fused(W["true"][0], pl, W["states"], rope, W["outs"], W["chain_ws"])
+        else:
+            kvc.kvc_chain(W["true"][0], pl, W["states"], rope, W["outs"])
         mark("chain_end")
 
 
@@ -388,6 +391,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small profiling cases)")
     ap.add_argument("--rank", type=int, default=0, help="override the rank r (experiments)")
+    ap.add_argument("--chain", default="hops", choices=["hops", "fused"],
+                    help="hops: kvc_chain, one launch per hop; fused: kvc_chain_fused, one pass over agent 0's cache")
     ap.add_argument("--grouped", type=int, default=0, help="1: per-layer states (D = H d), with --only apply")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
     ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi", "weights"],
@@ -453,6 +458,9 @@ def main():
         W = build_ring(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
     else:
         W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only, grouped=bool(args.grouped) and args.only == "apply")
+    if args.chain == "fused" and W.get("kind") is None and W.get("outs") and args.only in ("all", "apply"):
+        W["chain_ws"] = torch.empty(max(kvc.kvc_chain_workspace_bytes(W["true"][0], cfg.n_agents), 128), dtype=torch.uint8,
+                                    device=dev)
     if args.only != "all":
         args.no_e2e = True
     upd_b, app_b = step_bytes(W, kvc)
@@ -526,6 +534,24 @@ def main():
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
         del host_in, host_out
 
+    # beside the headline: the same chain through kvc_chain_fused (one pass over agent 0's cache, same bits)
+    fused = None
+    if rank == 0 and W.get("kind") is None and args.only in ("all", "apply") and W.get("chain_ws") is None and cfg.n_agents >= 3:
+        cws = torch.empty(max(kvc.kvc_chain_workspace_bytes(W["true"][0], cfg.n_agents), 128), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            kvc.kvc_chain_fused(W["true"][0], W["pl"], W["states"], W["rope"], W["outs"], cws)
+        fb, fe = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fb.record()
+        for _ in range(5):
+            kvc.kvc_chain_fused(W["true"][0], W["pl"], W["states"], W["rope"], W["outs"], cws)
+        fe.record()
+        torch.cuda.synchronize()
+        f_ms = fb.elapsed_time(fe) / 5
+        c0 = W["true"][0]
+        f_bytes = c0.L * c0.H * c0.T * (4 * c0.d + sum(8 * st.r + 4 * c0.d for st in W["states"]))
+        fused = {"chain_ms": f_ms, "algorithmic_bytes": f_bytes, "GBs": f_bytes / (f_ms * 1e-3) / 1e9,
+                 "us_per_agent_layer": f_ms * 1e3 / (cfg.n_agents - 1) / cfg.L}
+        del cws
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -550,7 +576,7 @@ def main():
                          / (hop_ms * 1e-3) / 1e9 if W.get("outs") else None,
                          "step_ms_median": sorted(per_step)[len(per_step) // 2], "step_ms_min": min(per_step),
                          "update_fit_GBs": upd_b / (upd_ms * 1e-3) / 1e9, "update_ms_per_step": upd_ms,
-                         "chain_ms_per_step": chain_ms,
+                         "chain_ms_per_step": chain_ms, "chain_fused": fused,
                          "kernel_family": {0: "auto", 1: "generic (CUDA cores)", 2: "tc (TMA + tcgen05)"}[last_path]}}
     if not args.no_cpu_baseline:
         out["cpu_baseline"], _ = cpu_baseline(cfg, args.cpu_budget)

@@ -246,6 +246,23 @@ int kvc_apply_batch(const kvc_item *items, int32_t n_items, const kvc_rope *rope
 size_t kvc_batch_workspace_bytes(int32_t n_items);
 
 /*
+ * kvc_chain_fused -- kvc_chain in one pass over agent 0's cache (Sec. 3.2, Eq. 6): every tile of
+ * agent 0 is loaded once, carried through all hops in shared memory and stored after every hop, so
+ * no intermediate cache is read back.  Same arguments, same results bit for bit as kvc_chain (each
+ * hop rounds to bf16 before it feeds the next); per token, layer and head the chain moves
+ * 4d + (n_agents - 1)(8r + 4d) bytes instead of (n_agents - 1)(8d + 8r).
+ *   workspace  DEVICE, kvc_chain_workspace_bytes(agent0, n_agents) bytes, 128-byte aligned: the hops'
+ *              bases rewritten as tensor-core operands (rebuilt by every call)
+ * Served fused: head_dim 128, 3 <= n_agents <= KVC_CHAIN_MAX_HOPS + 1, every live state with r <= 64,
+ * r a multiple of 4, grouped by head.  Anything else runs hop by hop exactly like kvc_chain (with
+ * kvc_set_path(KVC_PATH_TC): KVC_E_UNSUPPORTED instead).
+ */
+#define KVC_CHAIN_MAX_HOPS 7
+int kvc_chain_fused(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_len, const kvc_state *states,
+                    const kvc_rope *rope, kvc_cache *outs, void *workspace, size_t workspace_bytes, void *stream);
+size_t kvc_chain_workspace_bytes(const kvc_cache *agent0, int32_t n_agents);
+
+/*
  * Multi-anchor apply (Eq. 8 with the token-wise weights of App. A.3 "Correction Weighting"):
  *     K_dst[l,h,t,:] = bf16( Rot_shift(K_src[l,h,t,:]) + sum_v w_k[v][t] * coeff_k(v)[l,h,t,:] . basis_k(v)[l,h] )
  *     V_dst[l,h,t,:] = bf16( V_src[l,h,t,:]            + sum_v w_v[v][t] * coeff_v(v)[l,h,t,:] . basis_v(v)[l,h] )

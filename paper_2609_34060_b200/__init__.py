@@ -33,7 +33,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_chain_fused", "kvc_chain_workspace_bytes",
 )
 
 
@@ -80,6 +80,9 @@ def load(path: Optional[str] = None):
     PC, PS, PR, PI = C.POINTER(kvc_cache), C.POINTER(kvc_state), C.POINTER(kvc_rope), C.POINTER(kvc_item)
     lib.kvc_apply.argtypes = [PC, PS, i32, PR, PC, vp]
     lib.kvc_chain.argtypes = [PC, i32, C.POINTER(i32), PS, PR, PC, vp]
+    lib.kvc_chain_fused.argtypes = [PC, i32, C.POINTER(i32), PS, PR, PC, vp, sz, vp]
+    lib.kvc_chain_workspace_bytes.argtypes = [PC, i32]
+    lib.kvc_chain_workspace_bytes.restype = sz
     lib.kvc_state_update.argtypes = [PC, PC, i32, PR, PS, i32, vp, sz, vp]
     lib.kvc_state_update_noalloc.argtypes = [PC, PC, i32, PR, PS, i32, vp]
     lib.kvc_state_update_noalloc.restype = C.c_int
@@ -258,6 +261,23 @@ def kvc_chain(agent0: Cache, prefix_len: Sequence[int], states: Sequence[State],
     sts = (kvc_state * max(n - 1, 1))(*[s.struct() for s in states])
     os_ = (kvc_cache * max(n - 1, 1))(*[o.struct() for o in outs])
     _check(load().kvc_chain(C.byref(a0), n, pl, sts, C.byref(r), os_, _stream(stream)), "kvc_chain")
+
+
+def kvc_chain_workspace_bytes(agent0: Cache, n_agents: int) -> int:
+    a0 = agent0.struct()
+    return int(load().kvc_chain_workspace_bytes(C.byref(a0), int(n_agents)))
+
+
+def kvc_chain_fused(agent0: Cache, prefix_len: Sequence[int], states: Sequence[State], rope: Rope, outs: Sequence[Cache],
+                    workspace: torch.Tensor, stream=None) -> None:
+    """kvc_chain in one pass over agent 0's cache (same results bit for bit)."""
+    n = len(prefix_len)
+    a0, r = agent0.struct(), rope.struct()
+    pl = (C.c_int32 * n)(*[int(x) for x in prefix_len])
+    sts = (kvc_state * max(n - 1, 1))(*[s.struct() for s in states])
+    os_ = (kvc_cache * max(n - 1, 1))(*[o.struct() for o in outs])
+    _check(load().kvc_chain_fused(C.byref(a0), n, pl, sts, C.byref(r), os_, workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_chain_fused")
 
 
 def kvc_workspace_bytes(tgt: Cache, st: State, mode: int) -> int:

@@ -245,6 +245,47 @@ int kvc_chain(const kvc_cache* agent0, int32_t n_agents, const int32_t* prefix_l
   return KVC_OK;
 }
 
+size_t kvc_chain_workspace_bytes(const kvc_cache* agent0, int32_t n_agents) {
+  if (!agent0 || n_agents < 2) return 0;
+  return tc_chain_workspace_bytes(n_agents - 1, agent0->L, agent0->H);
+}
+
+int kvc_chain_fused(const kvc_cache* agent0, int32_t n_agents, const int32_t* prefix_len, const kvc_state* states,
+                    const kvc_rope* rope, kvc_cache* outs, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!agent0 || n_agents < 1 || !prefix_len) return KVC_E_INVALID_ARG;
+  if (n_agents == 1) return KVC_OK;
+  if (!states || !outs) return KVC_E_INVALID_ARG;
+  const int n_hops = n_agents - 1;
+  if (n_hops >= 2 && n_hops <= KVC_CHAIN_MAX_HOPS && tl_path_force != KVC_PATH_GENERIC) {
+    // validate the whole chain exactly as kvc_chain does, keeping every resolved hop
+    DevItem items[KVC_CHAIN_MAX_HOPS];
+    int d = 0;
+    for (int a = 1; a < n_agents; ++a) {
+      ResolvedHop hop;
+      const kvc_cache* src = (a == 1) ? agent0 : &outs[a - 2];
+      const int rc = resolve_hop(src, &states[a - 1], prefix_len[a] - prefix_len[a - 1], rope, &outs[a - 1], &hop);
+      if (rc != KVC_OK) return rc;
+      if (outs[a - 1].k == agent0->k || outs[a - 1].v == agent0->v) return KVC_E_ALIAS;
+      for (int b = 1; b < a; ++b)
+        if (outs[b - 1].k == outs[a - 1].k && outs[b - 1].page_table == outs[a - 1].page_table) return KVC_E_ALIAS;
+      items[a - 1] = hop.item;
+      d = hop.d;
+    }
+    uint32_t* status = status_ptr();
+    if (!status) return KVC_E_CUDA;
+    const int trc = tc_chain_fused(items, n_hops, d, rope->pairing, status, workspace, workspace_bytes,
+                                   reinterpret_cast<cudaStream_t>(stream));
+    if (trc == KVC_OK) {
+      tl_last_path = KVC_PATH_TC;
+      return KVC_OK;
+    }
+    if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  } else if (tl_path_force == KVC_PATH_TC) {
+    return KVC_E_UNSUPPORTED;
+  }
+  return kvc_chain(agent0, n_agents, prefix_len, states, rope, outs, stream);
+}
+
 size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
   if (!tgt || !st || mode != KVC_FIT) return 0;
   const size_t m = (size_t)tgt->L * tgt->H * 2;

@@ -17,6 +17,9 @@ int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* s
 int tc_apply_batch(DevItem* tab_host, int64_t* prefix_host, int n_items, int d, int pairing, uint32_t* status,
                    void* workspace_dev, void* staging_host, size_t bytes, cudaStream_t s);
 size_t tc_batch_extra_bytes(int n_items);
+size_t tc_chain_workspace_bytes(int n_hops, int L, int H);
+int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_t* status, void* workspace, size_t ws_bytes,
+                   cudaStream_t s);
 size_t tc_multi_workspace_bytes(int n_blocks, int L, int H);
 int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d, const DevState* anchors, int n_anchors,
                    const float* w_k, const float* w_v, int64_t t_pad, int shift, const float* cs, const float* sn, int pairing,
