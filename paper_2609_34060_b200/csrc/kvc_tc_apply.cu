@@ -90,11 +90,17 @@ struct TileWalker {
   int item, slab2, n_slab2, tt, tps, l, h;
   bool first;
   const DevItem* it;
+  const ItemMaps* mp;
+  int H, nb, cov;              // of the current item, read once: heads, rank blocks, covered rows of a live state (else 0)
 
   __device__ void load_item() {
     it = p->items ? p->items + item : &p->one;
+    mp = p->maps ? p->maps + item : &p->one_maps;
     tps = it->tiles_per_slab;
-    n_slab2 = it->L * it->H * (VONLY ? 1 : 2);
+    H = it->H;
+    n_slab2 = it->L * H * (VONLY ? 1 : 2);
+    nb = (it->st.r + 31) >> 5;
+    cov = (it->st.r > 0 && it->st.n_cov > 0) ? it->st.n_cov : 0;
   }
   __device__ void init(const ApplyTcLaunch* pp, int64_t begin, int64_t end_) {
     p = pp;
@@ -121,14 +127,14 @@ struct TileWalker {
       tt = (int)(local % tps);
       slab2 = (int)(local / tps);
       const int slab = VONLY ? slab2 : slab2 >> 1;
-      l = slab / it->H;
-      h = slab - l * it->H;
+      l = slab / H;
+      h = slab - l * H;
     }
   }
   __device__ bool done() const { return remaining <= 0; }
   __device__ void get(Tile& t) const {
     t.it = it;
-    t.mp = p->maps ? p->maps + item : &p->one_maps;
+    t.mp = mp;
     t.item = item;
     t.first = first;
     t.is_v = VONLY ? 1 : slab2 & 1;
@@ -136,9 +142,9 @@ struct TileWalker {
     t.l = l;
     t.h = h;
     t.t0 = tt * kTileTok;
-    t.nb = (it->st.r + 31) >> 5;
-    t.uses_basis = it->st.r > 0 && it->st.n_cov > 0;
-    t.has_coeff = t.uses_basis && t.t0 < it->st.n_cov;
+    t.nb = nb;
+    t.uses_basis = cov > 0;
+    t.has_coeff = t.t0 < cov;
   }
   __device__ void next() {
     if (--remaining <= 0) return;
@@ -148,7 +154,7 @@ struct TileWalker {
     tt = 0;
     ++slab2;
     if (VONLY || (slab2 & 1) == 0) {              // K and V of one (layer, head) are adjacent
-      if (++h == it->H) {
+      if (++h == H) {
         h = 0;
         ++l;
       }
