@@ -75,13 +75,13 @@ struct PTile {
   int slab, is_v, t0, l, h;
 };
 
-// hi = bf16(x), lo2 = bf16(2 (x - hi)) for two values, packed as bf16x2 words
+// hi = bf16(x), lo2 = bf16(2 (x - hi)) for two values, packed as bf16x2 words (packed conversions)
 __device__ __forceinline__ void split2x(float x0, float x1, uint32_t& hi, uint32_t& lo2) {
-  const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
-  const __nv_bfloat16 l0 = __float2bfloat16_rn(2.f * (x0 - __bfloat162float(h0)));
-  const __nv_bfloat16 l1 = __float2bfloat16_rn(2.f * (x1 - __bfloat162float(h1)));
-  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-  lo2 = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xffff0000u);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(2.f * (x0 - h0), 2.f * (x1 - h1));
+  lo2 = *reinterpret_cast<const uint32_t*>(&l);
 }
 __device__ __forceinline__ PTile decode(const UpdateLaunch& u, int64_t tile) {
   PTile t;
