@@ -39,9 +39,9 @@ UNIT = "GB/s"
 HBM_FALLBACK_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one apply launch on the 8K workload, from the ncu
 # capture summarised in profiles/apply_tc_kernel_dram_traffic_L16.md: measured at L = 16
-# (811.99 MB read + 489.74 MB written per launch) and scaled by 2 to L = 32 (traffic is
+# (811.95 MB read + 493.36 MB written per launch) and scaled by 2 to L = 32 (traffic is
 # proportional to the token-slabs processed).  None for other workloads.
-APPLY_TRAFFIC_BYTES_LLAMA8B_8K = 2 * (811_990_000 + 489_740_000)
+APPLY_TRAFFIC_BYTES_LLAMA8B_8K = 2 * (811_950_000 + 493_360_000)
 
 
 def _peaks():
