@@ -123,3 +123,53 @@ def test_byte_accounting_and_strings(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(RuntimeError):
         kvc.load(str(tmp_path / "nope.so"))
+
+
+def test_multi_anchor_and_grouping_argument_errors(lib):
+    """The entry points added beside the core path reject bad arguments on the host, before any device work."""
+    src, dst, rope = _cache(), _cache(k=0x2000000, v=0x3000000), _rope()
+    # grouping: only the two declared values
+    bad = _state()
+    bad.grouping = 7
+    assert lib.kvc_apply(C.byref(src), C.byref(bad), 0, C.byref(rope), C.byref(dst), None) == -1
+    grouped = _state()
+    grouped.grouping = kvc.KVC_GROUP_LAYER
+    # per-layer states are not served by the fit, the gate and the multi-anchor apply
+    assert lib.kvc_state_update(None, C.byref(src), 0, C.byref(rope), C.byref(grouped), kvc.KVC_FIT, 0x7000100, 1 << 30, None) == -3
+    assert lib.kvc_gate_distance(C.byref(src), C.byref(grouped), 1, 8, 0x8000000, None) == -3
+    assert lib.kvc_apply_multi(C.byref(src), C.byref(grouped), 1, None, None, 0, C.byref(rope), C.byref(dst), 0x9000000, 1 << 30, None) == -3
+    # byte accounting of a grouped state: the coefficients are shared by the heads
+    big, st = _cache(L=32, H=8, T=8192, d=128), _state(r=32, n_cov=8192)
+    st.grouping = kvc.KVC_GROUP_LAYER
+    assert lib.kvc_apply_bytes(C.byref(big), C.byref(st)) == 32 * 8 * 8192 * 8 * 128 + 32 * 8192 * 8 * 32 + 32 * 8 * 2 * 32 * 128 * 4
+    # gate
+    st8 = _state()
+    assert lib.kvc_gate_distance(C.byref(src), C.byref(st8), 1, 65, 0x8000000, None) == -2      # k beyond T
+    assert lib.kvc_gate_distance(C.byref(src), C.byref(_state(n_cov=10)), 1, 20, 0x8000000, None) == -2   # anchor shorter than k
+    assert lib.kvc_gate_distance(C.byref(src), C.byref(st8), 1, 8, 0x8000004, None) == -1       # misaligned float64 output
+    assert lib.kvc_gate_distance(C.byref(src), None, 0, 8, None, None) == 0                       # no anchors: nothing to do
+    assert lib.kvc_gate_weights(0x8000000, 1, C.c_double(1.0), 0x8000100, 0x8000200, None) == -1  # fewer than two anchors
+    assert lib.kvc_gate_weights(0x8000000, 3, C.c_double(0.0), 0x8000100, 0x8000200, None) == -1  # temperature
+    # multi-anchor apply: limits and workspace
+    many = (kvc.kvc_state * 11)(*[_state() for _ in range(11)])
+    assert lib.kvc_apply_multi(C.byref(src), many, 11, None, None, 0, C.byref(rope), C.byref(dst), 0x9000000, 1 << 30, None) == -3
+    two = (kvc.kvc_state * 2)(_state(r=32), _state(r=64))
+    assert lib.kvc_multi_workspace_bytes(C.byref(src), two, 2) == 3 * 2 * 2 * 2 * 128 * 128      # three rank blocks
+    assert lib.kvc_apply_multi(C.byref(src), two, 2, 0x8000004, None, 0, C.byref(rope), C.byref(dst), 0x9000000, 1 << 30, None) == -1
+    # token weights
+    pos = (C.c_int32 * 2)(0, 0)
+    tw = lambda n, ws, nb, pr=rope: lib.kvc_token_weights(C.byref(src), 0, two, pos, n, C.byref(pr), C.c_double(1.0), 0xa000000, 0xb000000, ws, nb, None)
+    assert lib.kvc_token_weights_workspace_bytes(C.byref(src), 2) == 2 * 2 * 128 * 4              # T = 64 pads to 128
+    assert tw(2, None, 0) == -6
+    assert tw(17, 0xc000000, 1 << 20) == -3
+    inter = _rope()
+    inter.pairing = kvc.KVC_ROPE_INTERLEAVED
+    assert tw(2, 0xc000000, 1 << 20, inter) == -3
+    # chain workspace, effective rank, realign
+    assert lib.kvc_chain_workspace_bytes(C.byref(src), 4) == 3 * 2 * 2 * 2 * 2 * 128 * 128
+    assert lib.kvc_chain_workspace_bytes(C.byref(src), 1) == 0
+    assert lib.kvc_effective_rank(0x8000000, 4, 128, C.c_double(1.5), 0x8001000, None) == -1
+    assert lib.kvc_effective_rank(None, 4, 128, C.c_double(0.9), 0x8001000, None) == -1
+    assert lib.kvc_fit_eigenvalues(C.byref(src), None) is None
+    assert lib.kvc_state_realign(C.byref(st8), 2, 2, 96, 5, C.byref(rope), 0x8000000, None) == -3
+    assert lib.kvc_state_realign(C.byref(st8), 2, 2, 128, 5, C.byref(rope), None, None) == -1
