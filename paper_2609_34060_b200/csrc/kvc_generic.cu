@@ -376,6 +376,9 @@ __global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant
 #define KVC_EIG_THREADS 256
 #endif
 constexpr int kEigThreads = KVC_EIG_THREADS;
+#ifndef KVC_EIG_MINBLOCKS
+#define KVC_EIG_MINBLOCKS 2
+#endif
 constexpr int kEigMaxR = 64;
 
 __device__ __forceinline__ float warp_sum(float x) {
@@ -385,7 +388,7 @@ __device__ __forceinline__ float warp_sum(float x) {
 }
 
 template <int N>
-__global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs) {
+__global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs) {
   extern __shared__ __align__(16) float smem[];
   constexpr int n = N;
   constexpr int np = N + 4;           // row pitch of A = 4 (mod 32)
@@ -416,7 +419,11 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   // the back-transformation finds it later.  Two block barriers per step.
   constexpr int TPR = kEigThreads / N;          // threads per row: 4 (N = 128) or 8 (N = 64) at 512 threads
   constexpr int NCH = N / (4 * TPR);            // chunks per thread: 8 or 2
-  static_assert(TPR * N == kEigThreads && NCH * 4 * TPR == N && TPR <= 32, "thread layout");
+#ifndef KVC_EIG_GCH
+#define KVC_EIG_GCH 4
+#endif
+  constexpr int GCH = NCH < KVC_EIG_GCH ? NCH : KVC_EIG_GCH;   // chunks handled together: loads first, then arithmetic
+  static_assert(TPR * N == kEigThreads && NCH * 4 * TPR == N && TPR <= 32 && NCH % GCH == 0, "thread layout");
   const int trow = tid / TPR, tq = tid % TPR;
   float a[NCH][4];
   {
@@ -486,7 +493,7 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
         v0 = x0 - alpha;
         beta = 1.f / (s2 - x0 * alpha);           // 2 / |v|^2
       }
-      if (mine) {
+      if (lane < N / 4) {                         // the whole row: zeros up to column k
         if (c0 + 0 == k + 1) x.x = v0;
         if (c0 + 1 == k + 1) x.y = v0;
         if (c0 + 2 == k + 1) x.z = v0;
@@ -511,14 +518,19 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
         float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
         if (active) {
 #pragma unroll
-          for (int c = 0; c < NCH; ++c) {
-            const int col0 = 4 * (c * TPR + tq);
-            if (col0 + 3 > k) {
-              const float4 v4 = *reinterpret_cast<const float4*>(v + col0);
-              acc0 = fmaf(a[c][0], v4.x, acc0);
-              acc1 = fmaf(a[c][1], v4.y, acc1);
-              acc2 = fmaf(a[c][2], v4.z, acc2);
-              acc3 = fmaf(a[c][3], v4.w, acc3);
+          for (int g = 0; g < NCH / GCH; ++g) {
+            if (4 * ((GCH * g + GCH - 1) * TPR + TPR - 1) + 3 > k) {     // uniform over the block
+              float4 v4[GCH];
+#pragma unroll
+              for (int c = 0; c < GCH; ++c)
+                v4[c] = *reinterpret_cast<const float4*>(v + 4 * ((GCH * g + c) * TPR + tq));
+#pragma unroll
+              for (int c = 0; c < GCH; ++c) {
+                acc0 = fmaf(a[GCH * g + c][0], v4[c].x, acc0);
+                acc1 = fmaf(a[GCH * g + c][1], v4[c].y, acc1);
+                acc2 = fmaf(a[GCH * g + c][2], v4[c].z, acc2);
+                acc3 = fmaf(a[GCH * g + c][3], v4[c].w, acc3);
+              }
             }
           }
         }
@@ -543,15 +555,22 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
           const float K = 0.5f * beta * vdotp;
           const float vi = v[trow], ci = pp[trow] - 2.f * K * vi;
 #pragma unroll
-          for (int c = 0; c < NCH; ++c) {
-            const int col0 = 4 * (c * TPR + tq);
-            if (col0 + 3 > k) {
-              const float4 v4 = *reinterpret_cast<const float4*>(v + col0);
-              const float4 p4 = *reinterpret_cast<const float4*>(pp + col0);
-              a[c][0] -= fmaf(vi, p4.x, ci * v4.x);
-              a[c][1] -= fmaf(vi, p4.y, ci * v4.y);
-              a[c][2] -= fmaf(vi, p4.z, ci * v4.z);
-              a[c][3] -= fmaf(vi, p4.w, ci * v4.w);
+          for (int g = 0; g < NCH / GCH; ++g) {
+            if (4 * ((GCH * g + GCH - 1) * TPR + TPR - 1) + 3 > k) {
+              float4 v4[GCH], p4[GCH];
+#pragma unroll
+              for (int c = 0; c < GCH; ++c) {
+                const int col0 = 4 * ((GCH * g + c) * TPR + tq);
+                v4[c] = *reinterpret_cast<const float4*>(v + col0);
+                p4[c] = *reinterpret_cast<const float4*>(pp + col0);
+              }
+#pragma unroll
+              for (int c = 0; c < GCH; ++c) {
+                a[GCH * g + c][0] -= fmaf(vi, p4[c].x, ci * v4[c].x);
+                a[GCH * g + c][1] -= fmaf(vi, p4[c].y, ci * v4[c].y);
+                a[GCH * g + c][2] -= fmaf(vi, p4[c].z, ci * v4[c].z);
+                a[GCH * g + c][3] -= fmaf(vi, p4[c].w, ci * v4[c].w);
+              }
             }
           }
         }
@@ -596,8 +615,8 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   {
     // TPE threads per eigenvalue: each round tests TPE interior points, the interval shrinks (TPE + 1)x
     constexpr int TPE = kEigThreads / 128;         // 4 at 512 threads, 2 at 256
-    constexpr int kRounds = TPE == 4 ? 12 : 17;    // 5^12 = 2.4e8, 3^17 = 1.3e8: both beyond 2^26
-    static_assert(TPE == 4 || TPE == 2, "multisection layout");
+    constexpr int kRounds = TPE == 4 ? 12 : (TPE == 2 ? 17 : 27);   // 5^12, 3^17, 2^27: all beyond 2^26
+    static_assert(TPE == 4 || TPE == 2 || TPE == 1, "multisection layout");
     const int ev = tid / TPE, sub = tid % TPE;
     const int want = n - 1 - ev;                   // ascending index of this group's eigenvalue
     float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
@@ -712,7 +731,109 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
     // Re-orthonormalise all r_eff vectors at once: S = Z^T Z (close to the identity), S = L L^T,
     // Z <- Z L^-T.  Equivalent to Gram-Schmidt in eigenvalue order, without its r_eff sequential
     // rounds; S is well conditioned because inverse iteration already separates the vectors.
-    {
+    if (r_eff <= 32) {
+      // The common case in registers, padded to 32 vectors with unit vectors of their own (S = 1 on the
+      // padded diagonal).  S: every thread forms a 2 x 2 block.
+      {
+        const int i0 = 2 * (tid >> 4), j0 = 2 * (tid & 15);
+        const bool mi0 = i0 < r_eff, mi1 = i0 + 1 < r_eff, mj0 = j0 < r_eff, mj1 = j0 + 1 < r_eff;
+        float s00 = 0.f, s01 = 0.f, s10 = 0.f, s11 = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < n; ++c) {
+          const float* zr = Zt + c * zs;
+          const float a0 = mi0 ? zr[i0] : 0.f, a1 = mi1 ? zr[i0 + 1] : 0.f;
+          const float b0 = mj0 ? zr[j0] : 0.f, b1 = mj1 ? zr[j0 + 1] : 0.f;
+          s00 = fmaf(a0, b0, s00);
+          s01 = fmaf(a0, b1, s01);
+          s10 = fmaf(a1, b0, s10);
+          s11 = fmaf(a1, b1, s11);
+        }
+        if (i0 == j0) {
+          if (!mi0) s00 = 1.f;
+          if (!mi1) s11 = 1.f;
+        }
+        S[i0 * sp + j0] = s00;
+        S[i0 * sp + j0 + 1] = s01;
+        S[(i0 + 1) * sp + j0] = s10;
+        S[(i0 + 1) * sp + j0 + 1] = s11;
+      }
+      __syncthreads();
+      // Cholesky by one warp, lane i holding row i of S and then of L in registers.  At step j lane j
+      // publishes its finished row; the lanes below it form their entry of column j from it.  The
+      // factor is left transposed in place of S (Lt[j][i] = L[i][j], reciprocals on the diagonal).
+      if (warp == 0) {
+        float l[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) l[k] = S[lane * sp + k];
+        __syncwarp();                             // S is overwritten by the transposed factor from here on
+        float* rowbuf = cdot;                     // [32] the published row (cdot is free here)
+        float dacc = 0.f;                         // sum of squares of this lane's finished entries
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float piv = __shfl_sync(0xffffffffu, l[j] - dacc, j);
+          if (piv < 1e-6f) {                      // (nearly) dependent vectors: keep going, flag it
+            piv = 1e-6f;
+            if (lane == 0) atomicOr(p.status, 4u);
+          }
+          const float rl = rsqrtf(piv);
+          if (lane == j) {
+#pragma unroll
+            for (int k4 = 0; k4 < (j + 3) / 4; ++k4)
+              *reinterpret_cast<float4*>(rowbuf + 4 * k4) = make_float4(l[4 * k4], l[4 * k4 + 1], l[4 * k4 + 2], l[4 * k4 + 3]);
+          }
+          __syncwarp();
+          float acc0 = l[j], acc1 = 0.f;
+#pragma unroll
+          for (int k4 = 0; k4 < j / 4; ++k4) {
+            const float4 r4 = *reinterpret_cast<const float4*>(rowbuf + 4 * k4);
+            acc0 = fmaf(-l[4 * k4], r4.x, acc0);
+            acc1 = fmaf(-l[4 * k4 + 1], r4.y, acc1);
+            acc0 = fmaf(-l[4 * k4 + 2], r4.z, acc0);
+            acc1 = fmaf(-l[4 * k4 + 3], r4.w, acc1);
+          }
+#pragma unroll
+          for (int k = (j / 4) * 4; k < j; ++k) acc0 = fmaf(-l[k], rowbuf[k], acc0);
+          const float lij = (acc0 + acc1) * rl;
+          if (lane > j) {
+            l[j] = lij;
+            dacc = fmaf(lij, lij, dacc);
+          }
+          S[j * sp + lane] = (lane > j) ? lij : (lane == j ? rl : 0.f);
+          __syncwarp();                           // the row buffer is rewritten at the next step
+        }
+      }
+      __syncthreads();
+      if (tid < n) {                              // row tid of Z:  x L^T = z, column by column of L
+        float z[32];
+        float* zrow = Zt + tid * zs;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) z[j] = (j < r_eff) ? zrow[j] : 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float* lt = S + j * sp;           // column j of L: reciprocal diagonal at j, entries below it after
+          float zj = 0.f;
+#pragma unroll
+          for (int g = j / 4; g < 8; ++g) {
+            const float4 t4 = *reinterpret_cast<const float4*>(lt + 4 * g);
+            const float t[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int i = 4 * g + e;
+              if (i == j) {
+                zj = z[j] * t[e];
+                z[j] = zj;
+              } else if (i > j) {
+                z[i] = fmaf(-zj, t[e], z[i]);
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (j < r_eff) zrow[j] = z[j];
+      }
+      __syncthreads();
+    } else {
       for (int t2 = tid; t2 < r_eff * r_eff; t2 += kEigThreads) {
         const int i = t2 / r_eff, j = t2 - i * r_eff;
         if (j <= i) {
