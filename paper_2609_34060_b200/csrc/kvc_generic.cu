@@ -1,6 +1,7 @@
 // CUDA-core kernels: every supported shape (head_dim 64/128, any rank, both RoPE
 // pairings, contiguous or paged).  They are the correctness baseline and the
 // fallback for arguments the TMA + tcgen05 kernels do not take.
+#include <type_traits>
 #include "kvc_dev.cuh"
 #include "kvc_launch.h"
 
@@ -428,17 +429,28 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   float a[NCH][4];
   {
     // stage the fixed-order sum of the partial Grams (coalesced), then symmetrise into registers
-    for (int i = tid; i < n * n / 4; i += kEigThreads) {
-      const int rr = i / (n / 4), c4 = i % (n / 4);
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    constexpr int kStage = 4;                     // float4 columns in flight per thread
+    static_assert((N * N / 4) % (kStage * kEigThreads) == 0, "staging layout");
+    for (int i0 = tid; i0 < n * n / 4; i0 += kStage * kEigThreads) {
+      float4 acc[kStage];
+#pragma unroll
+      for (int u = 0; u < kStage; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int pt = 0; pt < p.n_parts; ++pt) {
-        const float4 g = *reinterpret_cast<const float4*>(G + pt * part_stride + (int64_t)rr * n + 4 * c4);
-        acc.x += g.x;
-        acc.y += g.y;
-        acc.z += g.z;
-        acc.w += g.w;
+#pragma unroll
+        for (int u = 0; u < kStage; ++u) {
+          const int i = i0 + u * kEigThreads;
+          const float4 g = *reinterpret_cast<const float4*>(G + pt * part_stride + 4 * (int64_t)i);
+          acc[u].x += g.x;
+          acc[u].y += g.y;
+          acc[u].z += g.z;
+          acc[u].w += g.w;
+        }
       }
-      *reinterpret_cast<float4*>(A + rr * np + 4 * c4) = acc;
+#pragma unroll
+      for (int u = 0; u < kStage; ++u) {
+        const int i = i0 + u * kEigThreads;
+        *reinterpret_cast<float4*>(A + (i / (n / 4)) * np + 4 * (i % (n / 4))) = acc[u];
+      }
     }
     __syncthreads();
 #pragma unroll
@@ -608,7 +620,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   if (tid < n) {
     ds[tid] = dd[tid] * tinv;
     const float es = ee[tid] * tinv;
-    es2[tid] = es * es;
+    es2[tid] = fmaxf(es * es, 1e-36f);
     e2[tid] = ee[tid] * ee[tid];
   }
   __syncthreads();
@@ -626,11 +638,13 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots
       int cnt = 0;
       if (ev < n) {
+        // a zero pivot needs no guard: its reciprocal is +inf, the next pivot -inf (counted), the one
+        // after that d - x again; the squared couplings are kept above zero so that 0 * inf cannot occur
         float qv = ds[0] - mid;
         cnt = qv < 0.f;
+#pragma unroll 8
         for (int i = 1; i < n; ++i) {
-          if (fabsf(qv) < 1e-30f) qv = -1e-30f;
-          qv = ds[i] - mid - __fdividef(es2[i - 1], qv);
+          qv = (ds[i] - mid) - __fdividef(es2[i - 1], qv);
           cnt += qv < 0.f;
         }
       }
@@ -681,26 +695,37 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       // U of the pivoted LU kept in local arrays: reciprocal pivot, first super-diagonal; the second
       // super-diagonal is e[i+1] where rows were swapped (one bit per row), else zero
       float R0[128], U1[128];
-      uint32_t swp[4] = {0u, 0u, 0u, 0u};
+      uint32_t swp[N / 32];
       float u = dd[0] - s, v = ee[0];
       float xp = Zt[j];                           // running right-hand side entry of the pivot row
-      for (int i = 1; i < n; ++i) {
-        const float sub = ee[i - 1], dg = dd[i] - s, sp = (i < n - 1) ? ee[i] : 0.f;
-        const float xi = Zt[i * zs + j];
-        // one elimination step, written without branches (the lanes of the warp pivot differently):
-        // swap rows i-1 and i when the sub-diagonal entry is the larger pivot
-        const bool swap = fabsf(sub) > fabsf(u);
-        float piv = swap ? sub : u;
-        if (piv == 0.f) piv = eps3;
-        const float rp = 1.f / piv;
-        const float mult = (swap ? u : sub) * rp;
-        R0[i - 1] = rp;
-        U1[i - 1] = swap ? dg : v;
-        if (swap) swp[(i - 1) >> 5] |= 1u << ((i - 1) & 31);
-        Zt[(i - 1) * zs + j] = swap ? xi : xp;
-        xp = swap ? (xp - mult * xi) : (xi - mult * xp);
-        u = swap ? (v - mult * dg) : (dg - mult * v);
-        v = swap ? (-mult * sp) : sp;
+      // rows m, m + 1 are combined at step m; the steps run in blocks of 32 so that the swap bits of a
+      // block stay in one register
+#pragma unroll
+      for (int w = 0; w < N / 32; ++w) {
+        uint32_t bits = 0u;
+#pragma unroll 4
+        for (int mm = 0; mm < 32; ++mm) {
+          const int i = 32 * w + mm + 1;
+          if (i < n) {
+            const float sub = ee[i - 1], dg = dd[i] - s, sp = (i < n - 1) ? ee[i] : 0.f;
+            const float xi = Zt[i * zs + j];
+            // one elimination step, written without branches (the lanes of the warp pivot differently):
+            // swap rows i-1 and i when the sub-diagonal entry is the larger pivot
+            const bool swap = fabsf(sub) > fabsf(u);
+            float piv = swap ? sub : u;
+            if (piv == 0.f) piv = eps3;
+            const float rp = __fdividef(1.f, piv);
+            const float mult = (swap ? u : sub) * rp;
+            R0[i - 1] = rp;
+            U1[i - 1] = swap ? dg : v;
+            bits |= (swap ? 1u : 0u) << mm;
+            Zt[(i - 1) * zs + j] = swap ? xi : xp;
+            xp = swap ? (xp - mult * xi) : (xi - mult * xp);
+            u = swap ? (v - mult * dg) : (dg - mult * v);
+            v = swap ? (-mult * sp) : sp;
+          }
+        }
+        swp[w] = bits;
       }
       if (fabsf(u) < eps3) u = (u < 0.f) ? -eps3 : eps3;
       float y2 = xp / u;
@@ -708,13 +733,21 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       float y1 = (Zt[(n - 2) * zs + j] - U1[n - 2] * y2) * R0[n - 2];
       Zt[(n - 2) * zs + j] = y1;
       float big = fmaxf(fabsf(y1), fabsf(y2));
-      for (int i = n - 3; i >= 0; --i) {
-        const float u2 = ((swp[i >> 5] >> (i & 31)) & 1u) ? ee[i + 1] : 0.f;
-        const float y0 = (Zt[i * zs + j] - U1[i] * y1 - u2 * y2) * R0[i];
-        Zt[i * zs + j] = y0;
-        big = fmaxf(big, fabsf(y0));
-        y2 = y1;
-        y1 = y0;
+#pragma unroll
+      for (int w = N / 32 - 1; w >= 0; --w) {
+        const uint32_t bits = swp[w];
+#pragma unroll 4
+        for (int mm = 31; mm >= 0; --mm) {
+          const int i = 32 * w + mm;
+          if (i <= n - 3) {
+            const float u2 = ((bits >> mm) & 1u) ? ee[i + 1] : 0.f;
+            const float y0 = (Zt[i * zs + j] - U1[i] * y1 - u2 * y2) * R0[i];
+            Zt[i * zs + j] = y0;
+            big = fmaxf(big, fabsf(y0));
+            y2 = y1;
+            y1 = y0;
+          }
+        }
       }
       // scale against overflow, then normalise
       const float sc = 1.f / fmaxf(big, 1e-30f);
@@ -879,33 +912,41 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
 
   // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, then output
   float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
-  // Sixteen threads (half a warp) carry one vector through all reflectors with its entries in
-  // registers: thread `part` holds rows RPT part .. RPT part + RPT-1.  Per reflector: v . z over the
-  // half-warp (four shuffles), then z -= beta (v . z) v.  No block barrier: vectors are independent.
-  {
-    constexpr int RPT = N / 16;                   // rows per thread: 8 (N = 128) or 4 (N = 64)
-    const int part = lane & 15;
-    for (int j0 = 0; j0 < r_eff; j0 += kEigThreads / 16) {
-      const int j = j0 + (tid >> 4);
-      const bool have = j < r_eff;                // uniform over the half-warp
-      float z[RPT];
+  // TPV neighbouring lanes carry one vector through all reflectors with its entries in registers
+  // (thread `part` holds rows RPT part .. RPT part + RPT-1).  Per reflector: v . z over the TPV lanes
+  // (shuffles), then z -= beta (v . z) v; the next reflector is fetched while the sum is formed.  No
+  // block barrier: vectors are independent.  TPV is picked so that one pass covers all vectors.
+  auto back_transform = [&](auto tpv_tag) {
+    constexpr int TPV = decltype(tpv_tag)::value;
+    constexpr int RPT = N / TPV;                  // rows per thread
+    const int part = lane & (TPV - 1);
+    auto fetch = [&](int k, float (&vr)[RPT]) {
+      const float* v = A + k * np + RPT * part;   // reflector entries are zero up to column k
+#pragma unroll
+      for (int e4 = 0; e4 < RPT / 4; ++e4) {
+        // a group of four columns that ends before column k - 2 may still hold what was there before
+        // the reflector was written: it counts as zero
+        float4 t4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (RPT * part + 4 * e4 + 3 > k) t4 = *reinterpret_cast<const float4*>(v + 4 * e4);
+        vr[4 * e4 + 0] = t4.x;
+        vr[4 * e4 + 1] = t4.y;
+        vr[4 * e4 + 2] = t4.z;
+        vr[4 * e4 + 3] = t4.w;
+      }
+    };
+    for (int j0 = 0; j0 < r_eff; j0 += kEigThreads / TPV) {
+      const int j = j0 + tid / TPV;
+      const bool have = j < r_eff;                // uniform over the TPV lanes
+      float z[RPT], vr[RPT], vn[RPT];
 #pragma unroll
       for (int e = 0; e < RPT; ++e) z[e] = have ? Zt[(RPT * part + e) * zs + j] : 0.f;
+      float beta = bet[n - 3];
+      fetch(n - 3, vr);
       for (int k = n - 3; k >= 0; --k) {
-        const float beta = bet[k];
-        if (beta == 0.f) continue;
-        const float* v = A + k * np + RPT * part;   // reflector entries are zero up to column k
-        float vr[RPT];
-#pragma unroll
-        for (int e4 = 0; e4 < RPT / 4; ++e4) {
-          // a group of four columns that ends at or before column k was never written as part of
-          // the reflector (the set-up rewrites only groups that reach beyond k): it counts as zero
-          float4 t4 = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (RPT * part + 4 * e4 + 3 > k) t4 = *reinterpret_cast<const float4*>(v + 4 * e4);
-          vr[4 * e4 + 0] = t4.x;
-          vr[4 * e4 + 1] = t4.y;
-          vr[4 * e4 + 2] = t4.z;
-          vr[4 * e4 + 3] = t4.w;
+        float beta_n = 0.f;
+        if (k > 0) {
+          beta_n = bet[k - 1];
+          fetch(k - 1, vn);
         }
         float d0 = 0.f, d1 = 0.f;
 #pragma unroll
@@ -915,17 +956,27 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
         }
         float dot = d0 + d1;
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        dot *= beta;
+        for (int o = TPV / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        dot *= beta;                              // beta = 0: the reflector is the identity
 #pragma unroll
-        for (int e = 0; e < RPT; ++e) z[e] = fmaf(-dot, vr[e], z[e]);
+        for (int e = 0; e < RPT; ++e) {
+          z[e] = fmaf(-dot, vr[e], z[e]);
+          vr[e] = vn[e];
+        }
+        beta = beta_n;
       }
       if (have) {
 #pragma unroll
         for (int e = 0; e < RPT; ++e) Zt[(RPT * part + e) * zs + j] = z[e];
       }
     }
-  }
+  };
+  if (r_eff <= kEigThreads / 16)
+    back_transform(std::integral_constant<int, 16>{});
+  else if (r_eff <= kEigThreads / 8)
+    back_transform(std::integral_constant<int, 8>{});
+  else
+    back_transform(std::integral_constant<int, 4>{});
   __syncthreads();
   for (int j = warp; j < p.r; j += NW) {
     const bool live = j < r_eff && lam[j] > 0.f;
