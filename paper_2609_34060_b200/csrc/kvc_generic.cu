@@ -913,7 +913,8 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, then output
   float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
   // TPV neighbouring lanes carry one vector through all reflectors with its entries in registers
-  // (thread `part` holds rows RPT part .. RPT part + RPT-1).  Per reflector: v . z over the TPV lanes
+  // (thread `part` holds the four-row groups part, part + TPV, ...: neighbouring lanes read
+  // neighbouring 16 bytes of a reflector, free of bank conflicts).  Per reflector: v . z over the TPV lanes
   // (shuffles), then z -= beta (v . z) v; the next reflector is fetched while the sum is formed.  No
   // block barrier: vectors are independent.  TPV is picked so that one pass covers all vectors.
   auto back_transform = [&](auto tpv_tag) {
@@ -921,13 +922,13 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
     constexpr int RPT = N / TPV;                  // rows per thread
     const int part = lane & (TPV - 1);
     auto fetch = [&](int k, float (&vr)[RPT]) {
-      const float* v = A + k * np + RPT * part;   // reflector entries are zero up to column k
+      const float* v = A + k * np + 4 * part;     // reflector entries are zero up to column k
 #pragma unroll
       for (int e4 = 0; e4 < RPT / 4; ++e4) {
         // a group of four columns that ends before column k - 2 may still hold what was there before
         // the reflector was written: it counts as zero
         float4 t4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (RPT * part + 4 * e4 + 3 > k) t4 = *reinterpret_cast<const float4*>(v + 4 * e4);
+        if (4 * (part + TPV * e4) + 3 > k) t4 = *reinterpret_cast<const float4*>(v + 4 * TPV * e4);
         vr[4 * e4 + 0] = t4.x;
         vr[4 * e4 + 1] = t4.y;
         vr[4 * e4 + 2] = t4.z;
@@ -939,7 +940,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       const bool have = j < r_eff;                // uniform over the TPV lanes
       float z[RPT], vr[RPT], vn[RPT];
 #pragma unroll
-      for (int e = 0; e < RPT; ++e) z[e] = have ? Zt[(RPT * part + e) * zs + j] : 0.f;
+      for (int e = 0; e < RPT; ++e) z[e] = have ? Zt[(4 * (part + TPV * (e / 4)) + (e & 3)) * zs + j] : 0.f;
       float beta = bet[n - 3];
       fetch(n - 3, vr);
       for (int k = n - 3; k >= 0; --k) {
@@ -967,7 +968,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       }
       if (have) {
 #pragma unroll
-        for (int e = 0; e < RPT; ++e) Zt[(RPT * part + e) * zs + j] = z[e];
+        for (int e = 0; e < RPT; ++e) Zt[(4 * (part + TPV * (e / 4)) + (e & 3)) * zs + j] = z[e];
       }
     }
   };
