@@ -546,14 +546,11 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
             }
           }
         }
-        float acc = row_sum((acc0 + acc1) + (acc2 + acc3));
-        float vp = 0.f;
-        if (active && tq == 0) {
-          acc *= beta;
-          pp[trow] = acc;
-          vp = acc * v[trow];
-        }
-        vp = warp_sum(vp);
+        // v . p needs no finished row sums: every thread adds v_i times its own part of row i
+        const float part = (acc0 + acc1) + (acc2 + acc3);
+        const float vp = beta * warp_sum(v[trow] * part);
+        const float acc = row_sum(part);
+        if (active && tq == 0) pp[trow] = beta * acc;
         if (lane == 0) redw[warp] = vp;
         __syncthreads();
         // A -= v w^T + w v^T with w = p - K v, written as  a_ij -= v_i p_j + (p_i - 2 K v_i) v_j
@@ -565,7 +562,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
             vdotp += (r4.x + r4.y) + (r4.z + r4.w);
           }
           const float K = 0.5f * beta * vdotp;
-          const float vi = v[trow], ci = pp[trow] - 2.f * K * vi;
+          const float vi = v[trow], nvi = -vi, nci = fmaf(2.f * K, vi, -pp[trow]);
 #pragma unroll
           for (int g = 0; g < NCH / GCH; ++g) {
             if (4 * ((GCH * g + GCH - 1) * TPR + TPR - 1) + 3 > k) {
@@ -578,10 +575,10 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
               }
 #pragma unroll
               for (int c = 0; c < GCH; ++c) {
-                a[GCH * g + c][0] -= fmaf(vi, p4[c].x, ci * v4[c].x);
-                a[GCH * g + c][1] -= fmaf(vi, p4[c].y, ci * v4[c].y);
-                a[GCH * g + c][2] -= fmaf(vi, p4[c].z, ci * v4[c].z);
-                a[GCH * g + c][3] -= fmaf(vi, p4[c].w, ci * v4[c].w);
+                a[GCH * g + c][0] = fmaf(nvi, p4[c].x, fmaf(nci, v4[c].x, a[GCH * g + c][0]));
+                a[GCH * g + c][1] = fmaf(nvi, p4[c].y, fmaf(nci, v4[c].y, a[GCH * g + c][1]));
+                a[GCH * g + c][2] = fmaf(nvi, p4[c].z, fmaf(nci, v4[c].z, a[GCH * g + c][2]));
+                a[GCH * g + c][3] = fmaf(nvi, p4[c].w, fmaf(nci, v4[c].w, a[GCH * g + c][3]));
               }
             }
           }
@@ -625,29 +622,50 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   }
   __syncthreads();
   {
-    // TPE threads per eigenvalue: each round tests TPE interior points, the interval shrinks (TPE + 1)x
+    // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots.
+    // A zero pivot needs no guard: its reciprocal is +inf, the next pivot -inf (counted), the one
+    // after that d - x again; the squared couplings are kept above zero so that 0 * inf cannot occur.
+    auto sturm = [&](float x) {
+      float qv = ds[0] - x;
+      int cnt = qv < 0.f;
+#pragma unroll 8
+      for (int i = 1; i < n; ++i) {
+        qv = (ds[i] - x) - __fdividef(es2[i - 1], qv);
+        cnt += qv < 0.f;
+      }
+      return cnt;
+    };
+    // TPE threads per eigenvalue.  First one grid of as many points as there are threads over the whole
+    // interval, shared by all eigenvalues; then each round tests TPE interior points of the eigenvalue's
+    // own interval, which shrinks (TPE + 1)x.
     constexpr int TPE = kEigThreads / 128;         // 4 at 512 threads, 2 at 256
-    constexpr int kRounds = TPE == 4 ? 12 : (TPE == 2 ? 17 : 27);   // 5^12, 3^17, 2^27: all beyond 2^26
+    // (threads + 1) * (TPE + 1)^rounds beyond 2^27:  513 * 5^8,  257 * 3^12,  129 * 2^20
+    constexpr int kRounds = TPE == 4 ? 8 : (TPE == 2 ? 12 : 20);
     static_assert(TPE == 4 || TPE == 2 || TPE == 1, "multisection layout");
     const int ev = tid / TPE, sub = tid % TPE;
     const int want = n - 1 - ev;                   // ascending index of this group's eigenvalue
     float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
+    {
+      int* gcnt = reinterpret_cast<int*>(Zt);      // free until step 3
+      const float gstep = (hi - lo) * (1.f / (float)(kEigThreads + 1));
+      gcnt[tid] = sturm(lo + gstep * (float)(tid + 1));
+      __syncthreads();
+      int a = 0, b = kEigThreads;                  // first grid point with more than `want` eigenvalues below it
+      while (a < b) {
+        const int m = (a + b) >> 1;
+        if (gcnt[m] <= want)
+          a = m + 1;
+        else
+          b = m;
+      }
+      const float nlo = lo + gstep * (float)a, nhi = (a < kEigThreads) ? lo + gstep * (float)(a + 1) : hi;
+      lo = nlo;
+      hi = nhi;                                    // (a block barrier separates these reads from step 3)
+    }
     for (int it = 0; it < kRounds; ++it) {
       const float step = (hi - lo) * (1.f / (float)(TPE + 1));
       const float mid = lo + step * (float)(sub + 1);
-      // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots
-      int cnt = 0;
-      if (ev < n) {
-        // a zero pivot needs no guard: its reciprocal is +inf, the next pivot -inf (counted), the one
-        // after that d - x again; the squared couplings are kept above zero so that 0 * inf cannot occur
-        float qv = ds[0] - mid;
-        cnt = qv < 0.f;
-#pragma unroll 8
-        for (int i = 1; i < n; ++i) {
-          qv = (ds[i] - mid) - __fdividef(es2[i - 1], qv);
-          cnt += qv < 0.f;
-        }
-      }
+      const int cnt = (ev < n) ? sturm(mid) : 0;
       const bool below = cnt <= want;              // the eigenvalue is at or above this point
       // the points are ordered: new lo = last point with `below`, new hi = first without
       const unsigned grp = __ballot_sync(0xffffffffu, below) >> (lane & ~(TPE - 1)) & ((1u << TPE) - 1u);
