@@ -706,7 +706,111 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   float* S = (2 * r_eff <= n) ? A + (n / 2) * np : cdot + kEigMaxR;
   const int sp = (2 * r_eff <= n) ? np : (r_eff | 1);
   for (int iter = 0; iter < 2; ++iter) {
-    if (tid < r_eff) {
+    if (r_eff <= 32) {
+      // Solve (T - s I) y = z in place, lane j of every warp working on vector j: elimination with
+      // partial pivoting runs down the rows, SPW rows per warp, each warp keeping its part of U
+      // (reciprocal pivot, first super-diagonal, one swap bit per row: the second super-diagonal is
+      // e[i+1] where rows were swapped) in registers and handing the running row to the next warp
+      // through shared memory; back-substitution runs up the same way.  The solution stays in
+      // registers until it is scaled to unit length.
+      constexpr int SPW = N / NW;
+      float R0r[SPW], U1r[SPW], yr[SPW];
+      uint32_t bits = 0u;
+      const int j = lane;
+      const bool have = lane < r_eff;
+      const float s = have ? shf[j] : 0.f;
+      float* st = vv;                             // [4][32] hand-over slots (vv and pp are free after step 2)
+      float u = 0.f, v = 0.f, xp = 0.f;
+      if (warp == 0) st[96 + lane] = 0.f;         // sum of squares per vector
+      for (int w = 0; w < NW; ++w) {
+        if (warp == w && have) {
+          if (w == 0) {
+            u = dd[0] - s;
+            v = ee[0];
+            xp = Zt[j];                           // running right-hand side entry of the pivot row
+          } else {
+            u = st[j];
+            v = st[32 + j];
+            xp = st[64 + j];
+          }
+#pragma unroll
+          for (int q = 0; q < SPW; ++q) {
+            const int i = SPW * w + q + 1;        // rows i-1 and i are combined at this step
+            if (i < n) {
+              const float sub = ee[i - 1], dg = dd[i] - s, sp = (i < n - 1) ? ee[i] : 0.f;
+              const float xi = Zt[i * zs + j];
+              // one elimination step, written without branches (the lanes of the warp pivot differently):
+              // swap rows i-1 and i when the sub-diagonal entry is the larger pivot
+              const bool swap = fabsf(sub) > fabsf(u);
+              float piv = swap ? sub : u;
+              if (piv == 0.f) piv = eps3;
+              const float rp = __fdividef(1.f, piv);
+              const float mult = (swap ? u : sub) * rp;
+              R0r[q] = rp;
+              U1r[q] = swap ? dg : v;
+              bits |= (swap ? 1u : 0u) << q;
+              Zt[(i - 1) * zs + j] = swap ? xi : xp;
+              xp = swap ? (xp - mult * xi) : (xi - mult * xp);
+              u = swap ? (v - mult * dg) : (dg - mult * v);
+              v = swap ? (-mult * sp) : sp;
+            }
+          }
+          st[j] = u;
+          st[32 + j] = v;
+          st[64 + j] = xp;
+        }
+        __syncthreads();
+      }
+      for (int w = NW - 1; w >= 0; --w) {
+        if (warp == w && have) {
+          float y1, y2, big;
+          if (w == NW - 1) {                      // the last row: u and xp are still in this warp's registers
+            if (fabsf(u) < eps3) u = (u < 0.f) ? -eps3 : eps3;
+            y1 = xp / u;
+            y2 = 0.f;
+            big = fabsf(y1);
+            yr[SPW - 1] = y1;
+          } else {
+            y1 = st[j];
+            y2 = st[32 + j];
+            big = st[64 + j];
+          }
+#pragma unroll
+          for (int q = SPW - 1; q >= 0; --q) {
+            const int i = SPW * w + q;
+            if (i <= n - 2) {
+              const float u2 = ((bits >> q) & 1u) ? ee[i + 1] : 0.f;
+              const float y0 = (Zt[i * zs + j] - U1r[q] * y1 - u2 * y2) * R0r[q];
+              yr[q] = y0;
+              big = fmaxf(big, fabsf(y0));
+              y2 = y1;
+              y1 = y0;
+            }
+          }
+          st[j] = y1;
+          st[32 + j] = y2;
+          st[64 + j] = big;
+        }
+        __syncthreads();
+      }
+      // scale against overflow, then normalise
+      const float sc = have ? 1.f / fmaxf(st[64 + j], 1e-30f) : 0.f;
+      if (have) {
+        float nn = 0.f;
+#pragma unroll
+        for (int q = 0; q < SPW; ++q) {
+          yr[q] *= sc;
+          nn = fmaf(yr[q], yr[q], nn);
+        }
+        atomicAdd(&st[96 + j], nn);
+      }
+      __syncthreads();
+      if (have) {
+        const float inv = rsqrtf(fmaxf(st[96 + j], 1e-30f));
+#pragma unroll
+        for (int q = 0; q < SPW; ++q) Zt[(SPW * warp + q) * zs + j] = yr[q] * inv;
+      }
+    } else if (tid < r_eff) {
       // solve (T - s I) y = z in place: elimination with partial pivoting, U kept in local arrays
       const int j = tid;
       const float s = shf[j];
