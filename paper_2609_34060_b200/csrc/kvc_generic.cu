@@ -625,52 +625,67 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
     // Sturm count: pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1}; eigenvalues below x = negative pivots.
     // A zero pivot needs no guard: its reciprocal is +inf, the next pivot -inf (counted), the one
     // after that d - x again; the squared couplings are kept above zero so that 0 * inf cannot occur.
-    auto sturm = [&](float x) {
-      float qv = ds[0] - x;
-      int cnt = qv < 0.f;
+    // Two points per thread: the two recurrences are independent and hide each other's latency.
+    auto rcp = [](float x) {
+      float y;
+      asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+      return y;
+    };
+    auto sturm2 = [&](float xa, float xb, int& ca, int& cb) {
+      float qa = ds[0] - xa, qb = ds[0] - xb;
+      ca = qa < 0.f;
+      cb = qb < 0.f;
 #pragma unroll 8
       for (int i = 1; i < n; ++i) {
-        qv = (ds[i] - x) - __fdividef(es2[i - 1], qv);
-        cnt += qv < 0.f;
+        const float d = ds[i], e = -es2[i - 1];
+        qa = fmaf(e, rcp(qa), d - xa);
+        qb = fmaf(e, rcp(qb), d - xb);
+        ca += qa < 0.f;
+        cb += qb < 0.f;
       }
-      return cnt;
     };
-    // TPE threads per eigenvalue.  First one grid of as many points as there are threads over the whole
-    // interval, shared by all eigenvalues; then each round tests TPE interior points of the eigenvalue's
-    // own interval, which shrinks (TPE + 1)x.
+    // TPE threads per eigenvalue, two points per thread.  First one grid of 2 x threads points over the
+    // whole interval, shared by all eigenvalues; then each round tests 2 TPE interior points of the
+    // eigenvalue's own interval, which shrinks (2 TPE + 1)x.
     constexpr int TPE = kEigThreads / 128;         // 4 at 512 threads, 2 at 256
-    // (threads + 1) * (TPE + 1)^rounds beyond 2^27:  513 * 5^8,  257 * 3^12,  129 * 2^20
-    constexpr int kRounds = TPE == 4 ? 8 : (TPE == 2 ? 12 : 20);
+    constexpr int kGrid = 2 * kEigThreads;
+    // (grid + 1) * (2 TPE + 1)^rounds beyond 2^27:  1025 * 9^6,  513 * 5^8,  257 * 3^12
+    constexpr int kRounds = TPE == 4 ? 6 : (TPE == 2 ? 8 : 12);
     static_assert(TPE == 4 || TPE == 2 || TPE == 1, "multisection layout");
     const int ev = tid / TPE, sub = tid % TPE;
     const int want = n - 1 - ev;                   // ascending index of this group's eigenvalue
     float lo = gl * tinv - 1e-6f, hi = gu * tinv + 1e-6f;
     {
-      int* gcnt = reinterpret_cast<int*>(Zt);      // free until step 3
-      const float gstep = (hi - lo) * (1.f / (float)(kEigThreads + 1));
-      gcnt[tid] = sturm(lo + gstep * (float)(tid + 1));
+      // counts (at most n, one byte each) go to rows n - 2 and n - 1 of A, which hold no reflector
+      static_assert(2 * np * sizeof(float) >= kGrid, "grid counts fit the two free rows");
+      uint8_t* gcnt = reinterpret_cast<uint8_t*>(A + (n - 2) * np);
+      const float gstep = (hi - lo) * (1.f / (float)(kGrid + 1));
+      int ca, cb;
+      sturm2(lo + gstep * (float)(2 * tid + 1), lo + gstep * (float)(2 * tid + 2), ca, cb);
+      gcnt[2 * tid] = (uint8_t)ca;
+      gcnt[2 * tid + 1] = (uint8_t)cb;
       __syncthreads();
-      int a = 0, b = kEigThreads;                  // first grid point with more than `want` eigenvalues below it
+      int a = 0, b = kGrid;                        // first grid point with more than `want` eigenvalues below it
       while (a < b) {
         const int m = (a + b) >> 1;
-        if (gcnt[m] <= want)
+        if ((int)gcnt[m] <= want)
           a = m + 1;
         else
           b = m;
       }
-      const float nlo = lo + gstep * (float)a, nhi = (a < kEigThreads) ? lo + gstep * (float)(a + 1) : hi;
+      const float nlo = lo + gstep * (float)a, nhi = (a < kGrid) ? lo + gstep * (float)(a + 1) : hi;
       lo = nlo;
-      hi = nhi;                                    // (a block barrier separates these reads from step 3)
+      hi = nhi;
     }
     for (int it = 0; it < kRounds; ++it) {
-      const float step = (hi - lo) * (1.f / (float)(TPE + 1));
-      const float mid = lo + step * (float)(sub + 1);
-      const int cnt = (ev < n) ? sturm(mid) : 0;
-      const bool below = cnt <= want;              // the eigenvalue is at or above this point
-      // the points are ordered: new lo = last point with `below`, new hi = first without
-      const unsigned grp = __ballot_sync(0xffffffffu, below) >> (lane & ~(TPE - 1)) & ((1u << TPE) - 1u);
-      const int nb = __popc(grp);                  // points 0 .. nb-1 are below (monotone up to rounding)
-      const float nlo = lo + step * (float)nb, nhi = (nb < TPE) ? lo + step * (float)(nb + 1) : hi;
+      const float step = (hi - lo) * (1.f / (float)(2 * TPE + 1));
+      int ca, cb;
+      sturm2(lo + step * (float)(2 * sub + 1), lo + step * (float)(2 * sub + 2), ca, cb);
+      // the points are ordered: the eigenvalue is at or above the first nb of them (monotone up to rounding)
+      int nb = (ca <= want) + (cb <= want);
+#pragma unroll
+      for (int o = 1; o < TPE; o <<= 1) nb += __shfl_xor_sync(0xffffffffu, nb, o);
+      const float nlo = lo + step * (float)nb, nhi = (nb < 2 * TPE) ? lo + step * (float)(nb + 1) : hi;
       lo = nlo;
       hi = nhi;
     }
