@@ -708,11 +708,20 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       prev = s;
     }
   }
+  // start vectors: pseudo-random in (-1, 1), no component zero, a well-mixed integer hash of
+  // (component, vector, draw) so that any set of them is as independent as random vectors are
+  auto start_value = [](int comp, int j, int draw) {
+    uint32_t h = (uint32_t)comp * 0x9E3779B1u + (uint32_t)j * 0x85EBCA77u + (uint32_t)draw * 0xC2B2AE3Du + 0x165667B1u;
+    h ^= h >> 16;
+    h *= 0x7FEB352Du;
+    h ^= h >> 15;
+    h *= 0x846CA68Bu;
+    h ^= h >> 16;
+    return ((float)(h >> 16) + 0.5f) * (1.f / 32768.f) - 1.f;
+  };
   for (int i = tid; i < n * zs; i += kEigThreads) {
     const int comp = i / zs, j = i - comp * zs;
-    // start vectors: different for every eigenvector, no component zero
-    const uint32_t hsh = (uint32_t)(comp * 2654435761u) ^ (uint32_t)(j * 40503u + 12345u);
-    Zt[i] = 1.f + 0.5f * (float)((hsh >> 8) & 1023) * (1.f / 1024.f);
+    Zt[i] = start_value(comp, j, 0);
   }
   __syncthreads();
 
@@ -720,7 +729,23 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   // free after the reduction (reflectors live right of the diagonal) when r_eff <= n / 2
   float* S = (2 * r_eff <= n) ? A + (n / 2) * np : cdot + kEigMaxR;
   const int sp = (2 * r_eff <= n) ? np : (r_eff | 1);
-  for (int iter = 0; iter < 2; ++iter) {
+  // Two rounds of (inverse iteration, re-orthonormalisation) settle well separated eigenvalues.  Where
+  // eigenvalues crowd together (closer than their own accuracy), vectors of neighbouring shifts come
+  // out nearly parallel and re-orthonormalising leaves mostly rounding noise in one of them: further
+  // rounds turn that vector towards the missing direction.  Rounds go on while the smallest Cholesky
+  // pivot (squared sine of the angle to the earlier vectors) stays below kPivOk, up to kMaxIter.
+  // A vector whose pivot falls below kPivBad is (numerically) a combination of the earlier ones: it is
+  // left out of the factor, so that it cannot blow the later columns up, and drawn afresh for the next
+  // round.  One that is still in that state after the last round gives a zero basis row, flagged.
+#ifndef KVC_EIG_MAXITER
+#define KVC_EIG_MAXITER 5
+#endif
+  constexpr int kMaxIter = KVC_EIG_MAXITER;
+  constexpr float kPivOk = 1e-2f, kPivBad = 1e-4f;
+  float min_piv = 1.f;
+  uint32_t bad0 = 0u, bad1 = 0u;                  // vectors 0-31 / 32-63 left out in the last round
+#pragma unroll 1
+  for (int iter = 0; iter < kMaxIter; ++iter) {   // one copy of the round: later rounds are rare
     if (r_eff <= 32) {
       // Solve (T - s I) y = z in place, lane j of every warp working on vector j: elimination with
       // partial pivoting runs down the rows, SPW rows per warp, each warp keeping its part of U
@@ -758,7 +783,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
               // swap rows i-1 and i when the sub-diagonal entry is the larger pivot
               const bool swap = fabsf(sub) > fabsf(u);
               float piv = swap ? sub : u;
-              if (piv == 0.f) piv = eps3;
+              if (fabsf(piv) < eps3) piv = (piv < 0.f) ? -eps3 : eps3;   // tiny pivots are perturbed, not only zeros
               const float rp = __fdividef(1.f, piv);
               const float mult = (swap ? u : sub) * rp;
               R0r[q] = rp;
@@ -850,7 +875,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
             // swap rows i-1 and i when the sub-diagonal entry is the larger pivot
             const bool swap = fabsf(sub) > fabsf(u);
             float piv = swap ? sub : u;
-            if (piv == 0.f) piv = eps3;
+            if (fabsf(piv) < eps3) piv = (piv < 0.f) ? -eps3 : eps3;   // tiny pivots are perturbed, not only zeros
             const float rp = __fdividef(1.f, piv);
             const float mult = (swap ? u : sub) * rp;
             R0[i - 1] = rp;
@@ -938,14 +963,15 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
         __syncwarp();                             // S is overwritten by the transposed factor from here on
         float* rowbuf = cdot;                     // [32] the published row (cdot is free here)
         float dacc = 0.f;                         // sum of squares of this lane's finished entries
+        float mp = 1.f;
+        uint32_t bad = 0u;
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          float piv = __shfl_sync(0xffffffffu, l[j] - dacc, j);
-          if (piv < 1e-6f) {                      // (nearly) dependent vectors: keep going, flag it
-            piv = 1e-6f;
-            if (lane == 0) atomicOr(p.status, 4u);
-          }
-          const float rl = rsqrtf(piv);
+          const float piv = __shfl_sync(0xffffffffu, l[j] - dacc, j);
+          mp = fminf(mp, piv);
+          const bool ok = piv >= kPivBad;         // uniform over the warp
+          if (!ok) bad |= 1u << j;
+          const float rl = ok ? rsqrtf(piv) : 0.f;   // a vector that is left out gets a zero column
           if (lane == j) {
 #pragma unroll
             for (int k4 = 0; k4 < (j + 3) / 4; ++k4)
@@ -968,8 +994,13 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
             l[j] = lij;
             dacc = fmaf(lij, lij, dacc);
           }
-          S[j * sp + lane] = (lane > j) ? lij : (lane == j ? rl : 0.f);
+          S[j * sp + lane] = (lane > j) ? lij : (lane == j ? (ok ? rl : 1.f) : 0.f);
           __syncwarp();                           // the row buffer is rewritten at the next step
+        }
+        if (lane == 0) {
+          red[0] = mp;
+          red[1] = __uint_as_float(bad);
+          red[2] = __uint_as_float(0u);
         }
       }
       __syncthreads();
@@ -1001,6 +1032,11 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
 #pragma unroll
         for (int j = 0; j < 32; ++j)
           if (j < r_eff) zrow[j] = z[j];
+        const uint32_t bad = __float_as_uint(red[1]);
+        if (bad != 0u) {                          // rare: vectors left out of the factor are drawn afresh
+          for (int j = 0; j < r_eff; ++j)
+            if ((bad >> j) & 1u) zrow[j] = start_value(tid, j, iter + 1);
+        }
       }
       __syncthreads();
     } else {
@@ -1014,24 +1050,30 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       }
       __syncthreads();
       if (warp == 0) {
+        float mp = 1.f;
+        uint32_t badw[2] = {0u, 0u};
         for (int j = 0; j < r_eff; ++j) {
           float dsum = 0.f;
           for (int k = lane; k < j; k += 32) dsum = fmaf(S[j * sp + k], S[j * sp + k], dsum);
           dsum = warp_sum(dsum);
-          float piv = S[j * sp + j] - dsum;
-          if (piv < 1e-6f) {                      // (nearly) dependent vectors: keep going, flag it
-            piv = 1e-6f;
-            if (lane == 0) atomicOr(p.status, 4u);
-          }
-          const float ljj = sqrtf(piv), rl = 1.f / ljj;
+          const float piv = S[j * sp + j] - dsum;
+          mp = fminf(mp, piv);
+          const bool ok = piv >= kPivBad;         // uniform over the warp
+          if (!ok) badw[j >> 5] |= 1u << (j & 31);
+          const float rl = ok ? rsqrtf(piv) : 0.f;   // a vector that is left out gets a zero column
           __syncwarp();
           for (int i = j + 1 + lane; i < r_eff; i += 32) {
             float acc = S[i * sp + j];
             for (int k = 0; k < j; ++k) acc = fmaf(-S[i * sp + k], S[j * sp + k], acc);
             S[i * sp + j] = acc * rl;
           }
-          if (lane == 0) S[j * sp + j] = rl;      // keep the reciprocal of the diagonal
+          if (lane == 0) S[j * sp + j] = ok ? rl : 1.f;   // keep the reciprocal of the diagonal
           __syncwarp();
+        }
+        if (lane == 0) {
+          red[0] = mp;
+          red[1] = __uint_as_float(badw[0]);
+          red[2] = __uint_as_float(badw[1]);
         }
       }
       __syncthreads();
@@ -1042,10 +1084,17 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
           for (int k = 0; k < j; ++k) acc = fmaf(-z[k], S[j * sp + k], acc);
           z[j] = acc * S[j * sp + j];
         }
+        for (int j = 0; j < r_eff; ++j)
+          if ((__float_as_uint(red[1 + (j >> 5)]) >> (j & 31)) & 1u) z[j] = start_value(tid, j, iter + 1);
       }
       __syncthreads();
     }
+    bad0 = __float_as_uint(red[1]);
+    bad1 = __float_as_uint(red[2]);
+    min_piv = red[0];                             // written before the last two barriers; next written after the next one
+    if (iter >= 1 && min_piv >= kPivOk) break;    // uniform over the block
   }
+  if (tid == 0 && (bad0 | bad1) != 0u) atomicOr(p.status, 4u);   // vectors still dependent after the last round: flagged
 
   // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, then output
   float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
@@ -1117,7 +1166,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
     back_transform(std::integral_constant<int, 4>{});
   __syncthreads();
   for (int j = warp; j < p.r; j += NW) {
-    const bool live = j < r_eff && lam[j] > 0.f;
+    const bool live = j < r_eff && lam[j] > 0.f && (((j < 32 ? bad0 : bad1) >> (j & 31)) & 1u) == 0u;
     if (live) {
       float nn = 0.f, best = -1.f;
       int besti = 0;

@@ -197,6 +197,40 @@ def test_fit_rank_limits(path):
     assert np.max(np.abs(c @ B[0, 0] - dl)) <= 1e-3 * np.max(np.abs(dl))
 
 
+@pytest.mark.parametrize("base", [CFG_TINY.scaled(L=1, H=1, T=300), CFG_8B_S.scaled(L=1, H=1, T=300, r=8)],
+                         ids=["d64", "d128"])
+def test_fit_rank_sweep(base):
+    """Fit ranks from 1 to 64 on a rank-8 deviation over a noise floor: ranks below, at and above the
+    signal rank, on both sides of 32 (where the eigensolver changes its vector path).  Whatever the
+    rank: orthonormal rows, the oracle's eigenvalues, no dependent-vector flag, and a residual at the
+    tail energy (Eckart-Young).  A float32 reduction to tridiagonal form moves every eigenvalue by up
+    to about d eps |T| (8e-6 |T| at d = 128), which is the size of the smallest eigenvalues kept at the
+    larger ranks: each kept vector may miss that much energy, hence the allowance per vector."""
+    src_cpu, tgt_cpu, osrc, otgt, true, shift = _edge(base)
+    f = hp.inv_freq(base)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    T, d = base.T, base.d
+    _, oev = orc.state_update(osrc, otgt, shift, f, r=8, mode=orc.FIT)
+    for r in (1, 2, 3, 7, 8, 9, 31, 32, 33, 48, 64):
+        st = kvc.State(torch.zeros(1, 1, T, r, device=DEV), torch.zeros(1, 1, T, r, device=DEV),
+                       torch.zeros(1, 1, r, d, device=DEV), torch.zeros(1, 1, r, d, device=DEV))
+        ws = torch.empty(kvc.kvc_workspace_bytes(tgt, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+        kvc.kvc_state_update(src, tgt, shift, kvc.Rope(base.theta), st, kvc.KVC_FIT, workspace=ws)
+        torch.cuda.synchronize()
+        ev = ws.view(torch.float32)[2 * 2 * d * d: 2 * 2 * d * d + 2 * d].cpu().numpy().astype(np.float64).reshape(2, d)
+        for i, (which, B_t, c_t) in enumerate((("k", st.basis_k, st.coeff_k), ("v", st.basis_v, st.coeff_v))):
+            dl = orc.deviation(osrc.get_bits(which, 0, 0), otgt.get_bits(which, 0, 0), shift, f, which == "k")
+            w = oev[0, 0, i]
+            assert np.max(np.abs(ev[i] - w)) <= 1e-4 * w[0], r
+            B = B_t[0, 0].cpu().numpy().astype(np.float64)
+            c = c_t[0, 0].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(B @ B.T - np.eye(r))) <= 1e-4, r
+            res = float(np.sum((dl - c @ B) ** 2))
+            tail = float(np.sum(w[r:]))
+            assert res <= tail + 8 * r * 1.2e-6 * w[0] + 1e-9 * float(np.sum(w)), (r, res, tail)
+    assert kvc.kvc_status_poll() == 0
+
+
 def test_effective_rank_from_fit_eigenvalues():
     """Sec. 3.1's diagnostic on the eigenvalues a FIT leaves behind: a deviation of exact rank 8 plus
     bf16 rounding noise has effective rank <= 8 at 90 % energy and matches the oracle's count on the
