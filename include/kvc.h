@@ -175,8 +175,13 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *   KVC_FIT    : G = Delta^T Delta (d x d), its top-r eigenvectors become the rows
  *                of st->basis_* (float32; right singular vectors of Delta, largest
  *                singular values first, each row's largest-magnitude entry made
- *                positive; rows beyond min(r, d, n_cov) are zero), then coeff as above
- *                (= U_r Sigma_r).  st->basis_dtype must be KVC_F32 and r <= 64 (else
+ *                positive; rows beyond min(r, d, n_cov) are zero, and so is a row whose
+ *                eigenvalue lies below what float32 resolves beside the largest one,
+ *                2.4e-7 of it: a deviation of rank < r gives that many zero rows), then
+ *                coeff as above (= U_r Sigma_r).  The eigenvalues and vectors come from a
+ *                float32 tridiagonal reduction: accurate to about d * 6e-8 of the largest
+ *                eigenvalue; where eigenvalues lie closer than that, the rows span their
+ *                common subspace.  st->basis_dtype must be KVC_F32 and r <= 64 (else
  *                KVC_E_UNSUPPORTED).
  *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
  *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte

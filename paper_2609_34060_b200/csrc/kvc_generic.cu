@@ -689,7 +689,8 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
       lo = nlo;
       hi = nhi;
     }
-    if (ev < n && sub == 0) lam[ev] = 0.5f * (lo + hi) * tscale;
+    // (an all-zero matrix has all-zero eigenvalues, not midpoints of the guard interval)
+    if (ev < n && sub == 0) lam[ev] = (tnorm > 0.f) ? 0.5f * (lo + hi) * tscale : 0.f;
   }
   __syncthreads();
   if (tid < n) p.evals[(int64_t)sk * n + tid] = lam[tid];
@@ -1166,7 +1167,8 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
     back_transform(std::integral_constant<int, 4>{});
   __syncthreads();
   for (int j = warp; j < p.r; j += NW) {
-    const bool live = j < r_eff && lam[j] > 0.f && (((j < 32 ? bad0 : bad1) >> (j & 31)) & 1u) == 0u;
+    // an eigenvalue below what float32 resolves next to the largest one counts as zero: no direction
+    const bool live = j < r_eff && lam[j] > 2.4e-7f * tnorm && (((j < 32 ? bad0 : bad1) >> (j & 31)) & 1u) == 0u;
     if (live) {
       float nn = 0.f, best = -1.f;
       int besti = 0;

@@ -231,6 +231,74 @@ def test_fit_rank_sweep(base):
     assert kvc.kvc_status_poll() == 0
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_fit_degenerate_spectra(d):
+    """Spectra with a closed form, factorising a hand-made cache by itself (src = NULL).
+    (a) All zeros: every eigenvalue 0, the basis rows and coefficients all zero, nothing flagged.
+    (b) Token t carries the value 1 in dimension t mod 8 only: the Gram matrix is diag(T/8 x 8, 0, ...),
+    an eight-fold eigenvalue.  At r = 8 the basis spans e_0..e_7 and reproduces the cache exactly; at
+    r = 4 any orthonormal four-dimensional part of that span is right and leaves exactly half the energy;
+    at r = 12 the four directions beyond the rank have eigenvalue zero: their rows are zero.
+    (c) Two equal pairs and a single: singular values (3, 3, 2, 2, 1) on orthogonal +-1 patterns."""
+    T = 256
+    rope = kvc.Rope(10000.0)
+
+    def fit(v_rows, r):
+        cache = kvc.Cache(v_rows.to(torch.bfloat16).reshape(1, 1, T, d).contiguous().to(DEV),
+                          v_rows.to(torch.bfloat16).reshape(1, 1, T, d).contiguous().to(DEV))
+        st = kvc.State(torch.ones(1, 1, T, r, device=DEV), torch.ones(1, 1, T, r, device=DEV),
+                       torch.ones(1, 1, r, d, device=DEV), torch.ones(1, 1, r, d, device=DEV))
+        ws = torch.empty(kvc.kvc_workspace_bytes(cache, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+        kvc.kvc_state_update(None, cache, 0, rope, st, kvc.KVC_FIT, workspace=ws)
+        torch.cuda.synchronize()
+        ev = ws.view(torch.float32)[2 * 2 * d * d: 2 * 2 * d * d + 2 * d].cpu().numpy().astype(np.float64).reshape(2, d)
+        return st, ev
+
+    # (a)
+    st, ev = fit(torch.zeros(T, d), 8)
+    assert np.all(ev == 0)
+    for t in (st.basis_k, st.basis_v, st.coeff_k, st.coeff_v):
+        assert torch.all(t == 0)
+    # (b)
+    x = torch.zeros(T, d)
+    x[torch.arange(T), torch.arange(T) % 8] = 1.0
+    xn = x.numpy().astype(np.float64)
+    for r in (4, 8, 12):
+        st, ev = fit(x, r)
+        for i, (B_t, c_t) in enumerate(((st.basis_k, st.coeff_k), (st.basis_v, st.coeff_v))):
+            assert np.max(np.abs(ev[i, :8] - T / 8)) <= 1e-4 * T / 8 and np.max(np.abs(ev[i, 8:])) <= 1e-5 * T / 8
+            B = B_t[0, 0].cpu().numpy().astype(np.float64)
+            c = c_t[0, 0].cpu().numpy().astype(np.float64)
+            k = min(r, 8)
+            assert np.max(np.abs(B[:k] @ B[:k].T - np.eye(k))) <= 1e-5
+            assert np.max(np.abs(B[:k, 8:])) <= 1e-5                     # inside span(e_0..e_7)
+            assert np.all(B[k:] == 0) and np.all(c[:, k:] == 0)            # nothing beyond the rank of the data
+            res = float(np.sum((xn - c @ B) ** 2))
+            assert abs(res - (8 - k) * T / 8) <= 1e-4 * T, (r, res)
+    # (c)
+    had = np.array([[1 if bin(i & j).count("1") % 2 == 0 else -1 for j in range(8)] for i in range(8)], dtype=np.float64)
+    u = np.repeat(had[:, :5], T // 8, axis=0) / np.sqrt(T)                 # orthonormal columns, entries +-1/16
+    vt = np.zeros((5, d))
+    for q in range(5):
+        vt[q, 8 * q: 8 * q + 4] = 0.5                                      # orthonormal rows
+    sv = np.array([3.0, 3.0, 2.0, 2.0, 1.0])
+    y = (u * (16.0 * sv)) @ vt                                             # entries are small dyadic numbers: exact in bf16
+    st, ev = fit(torch.from_numpy(y).float(), 5)
+    want = np.concatenate([(16.0 * sv) ** 2, np.zeros(d - 5)])
+    for i, (B_t, c_t) in enumerate(((st.basis_k, st.coeff_k), (st.basis_v, st.coeff_v))):
+        assert np.max(np.abs(ev[i] - want)) <= 1e-4 * want[0]
+        B = B_t[0, 0].cpu().numpy().astype(np.float64)
+        c = c_t[0, 0].cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(B @ B.T - np.eye(5))) <= 1e-5
+        assert np.max(np.abs(y - c @ B)) <= 1e-3
+        # the single value's direction is unique up to sign; the pairs are planes
+        assert abs(abs(B[4] @ vt[4]) - 1.0) <= 1e-4
+        for pair in ((0, 1), (2, 3)):
+            P = B[list(pair)]
+            assert np.max(np.abs(P @ vt[list(pair)].T @ vt[list(pair)] - P)) <= 1e-3
+    assert kvc.kvc_status_poll() == 0
+
+
 def test_effective_rank_from_fit_eigenvalues():
     """Sec. 3.1's diagnostic on the eigenvalues a FIT leaves behind: a deviation of exact rank 8 plus
     bf16 rounding noise has effective rank <= 8 at 90 % energy and matches the oracle's count on the
