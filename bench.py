@@ -511,22 +511,48 @@ def main():
         h2d = sum(k.numel() * 2 + v.numel() * 2 for k, v in host_in)
         d2h = sum(k.numel() * 2 + v.numel() * 2 for k, v in host_out)
 
+        # Three streams: every step copies all its inputs in, runs the path and copies all its results
+        # out; the copy-out of step i and the copy-in of step i + 1 share the link's two directions.
+        # A step's kernels wait for its inputs and for the previous results to have left the device;
+        # its copy-in waits for the previous step's kernels (they read the same buffers).
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        s_run = torch.cuda.current_stream()
+        state = {"run_done": None, "out_done": None}
+
         def e2e_step():
-            for c, (hk, hv) in zip(srcs, host_in):
-                c.k.copy_(hk, non_blocking=True)
-                c.v.copy_(hv, non_blocking=True)
+            with torch.cuda.stream(s_in):
+                if state["run_done"] is not None:
+                    s_in.wait_event(state["run_done"])
+                for c, (hk, hv) in zip(srcs, host_in):
+                    c.k.copy_(hk, non_blocking=True)
+                    c.v.copy_(hv, non_blocking=True)
+                in_done = torch.cuda.Event()
+                in_done.record(s_in)
+            s_run.wait_event(in_done)
+            if state["out_done"] is not None:
+                s_run.wait_event(state["out_done"])
             run_step(W, kvc)
-            for o, (hk, hv) in zip(W["outs"], host_out):
-                hk.copy_(o.k, non_blocking=True)
-                hv.copy_(o.v, non_blocking=True)
+            state["run_done"] = torch.cuda.Event()
+            state["run_done"].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(state["run_done"])
+                for o, (hk, hv) in zip(W["outs"], host_out):
+                    hk.copy_(o.k, non_blocking=True)
+                    hv.copy_(o.v, non_blocking=True)
+                state["out_done"] = torch.cuda.Event()
+                state["out_done"].record(s_out)
 
         e2e_step()
+        s_run.wait_event(state["out_done"])
         barrier()
-        n_e2e = max(1, min(args.steps, 3))
+        state["run_done"] = state["out_done"] = None
+        n_e2e = max(1, min(args.steps, 5))
         b, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         b.record()
+        s_in.wait_event(b)
         for _ in range(n_e2e):
             e2e_step()
+        s_run.wait_event(state["out_done"])
         e.record()
         barrier()
         te = dist_util.max_over_ranks(b.elapsed_time(e), dev)
