@@ -686,16 +686,27 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             float x[16];
             unpack8(*reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4)), x);
             unpack8(*reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4)), x + 8);
+            if (!t.is_v) {
+              // both tables, eight pairs each, as vector loads
+              const float4 ca = *reinterpret_cast<const float4*>(it.cs + 8 * j), cb = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
+              const float4 sa4 = *reinterpret_cast<const float4*>(it.sn + 8 * j), sb4 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
+              const float4 cc = *reinterpret_cast<const float4*>(p.cs2 + 8 * j), cd = *reinterpret_cast<const float4*>(p.cs2 + 8 * j + 4);
+              const float4 sc4 = *reinterpret_cast<const float4*>(p.sn2 + 8 * j), sd4 = *reinterpret_cast<const float4*>(p.sn2 + 8 * j + 4);
+              const float c1[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+              const float s1[8] = {sa4.x, sa4.y, sa4.z, sa4.w, sb4.x, sb4.y, sb4.z, sb4.w};
+              const float c2[8] = {cc.x, cc.y, cc.z, cc.w, cd.x, cd.y, cd.z, cd.w};
+              const float s2[8] = {sc4.x, sc4.y, sc4.z, sc4.w, sd4.x, sd4.y, sd4.z, sd4.w};
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              float u = x[k], v = x[8 + k], au = a0[8 * jj + k], av = a1[8 * jj + k];
-              if (!t.is_v) {
-                const float c1 = it.cs[8 * j + k], s1 = it.sn[8 * j + k], c2 = p.cs2[8 * j + k], s2 = p.sn2[8 * j + k];
-                const float ru = u * c1 - v * s1, rv = u * s1 + v * c1;
-                const float bu = au * c2 - av * s2, bv = au * s2 + av * c2;
-                u = ru, v = rv, au = bu, av = bv;
+              for (int k = 0; k < 8; ++k) {
+                const float u = x[k], v = x[8 + k], au = a0[8 * jj + k], av = a1[8 * jj + k];
+                // source rotated by the first table minus reconstruction rotated by the second
+                const float du = fmaf(u, c1[k], -v * s1[k]) - fmaf(au, c2[k], -av * s2[k]);
+                const float dv = fmaf(u, s1[k], v * c1[k]) - fmaf(au, s2[k], av * c2[k]);
+                sa += fabsf(du) + fabsf(dv);
               }
-              sa += fabsf(u - au) + fabsf(v - av);
+            } else {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) sa += fabsf(x[k] - a0[8 * jj + k]) + fabsf(x[8 + k] - a1[8 * jj + k]);
             }
           }
           atomicAdd(p.row_out + (int64_t)t.is_v * p.row_pad + tok, sa * p.row_scale);
@@ -764,8 +775,9 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
           }
         }
       }
-      // ---- 4. the tile is final in shared memory: hand it to the store warp
-      fence_proxy_async();
+      // ---- 4. the tile is final in shared memory: hand it to the store warp (the reducing modes
+      // wrote nothing that the async proxy will read)
+      if constexpr (!REDUCE) fence_proxy_async();
       mbar_arrive(smem_u32(&ctrl->ready[s]));
     }
     if constexpr (GATE) {
