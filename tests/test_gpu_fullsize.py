@@ -143,6 +143,21 @@ def test_state_update_full_size_sampled_slabs(name):
     wsf = ws.view(torch.float32)
     G_all = wsf[: L * H * 2 * d * d].view(L, H, 2, d, d)
     ev_all = wsf[2 * L * H * 2 * d * d: 2 * L * H * 2 * d * d + L * H * 2 * d].view(L, H, 2, d)
+    # properties of every one of the 2 L H decompositions (checked with library routines on the device):
+    # orthonormal rows, eigenvalues in descending order and equal to the trace of the Gram matrix in sum,
+    # and the Rayleigh quotients of the rows are the leading eigenvalues
+    eye = torch.eye(r, device=DEV, dtype=torch.float64)
+    for i, Bt in enumerate((fit.basis_k, fit.basis_v)):
+        B64 = Bt.to(torch.float64)
+        assert float((B64 @ B64.transpose(-1, -2) - eye).abs().max()) <= 1e-4
+        ev64 = ev_all[:, :, i].to(torch.float64)
+        top = ev64[..., :1]
+        assert bool(((ev64[..., 1:] - ev64[..., :-1]) <= 1e-6 * top).all())
+        G64 = G_all[:, :, i].to(torch.float64)
+        tr = torch.diagonal(G64, dim1=-2, dim2=-1).sum(-1)
+        assert float(((ev64.sum(-1) - tr).abs() / tr).max()) <= 1e-4
+        rq = torch.einsum("lhrd,lhde,lhre->lhr", B64, G64, B64)
+        assert float(((rq - ev64[..., :r]).abs() / top).max()) <= 1e-4
     for (l, h) in slabs:
         for i, (which, Bt, ct) in enumerate((("k", fit.basis_k, fit.coeff_k), ("v", fit.basis_v, fit.coeff_v))):
             dl = deltas[(l, h, which)]
