@@ -655,7 +655,11 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
         if (in_range) {
           const uint8_t* row0 = st_ptr + m * 128;
           const uint8_t* row1 = row0 + kHalfBytes;
-          float sq = 0.f;
+          if (!covered) {                           // no reconstruction for this row: distance to zero
+#pragma unroll
+            for (int k = 0; k < 16; ++k) a0[k] = a1[k] = 0.f;
+          }
+          float sq0 = 0.f, sq1 = 0.f;
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj) {
             const int j = 2 * cq + jj;
@@ -664,13 +668,13 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             unpack8(*reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4)), x + 8);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-              const float d0 = x[k] - (covered ? a0[8 * jj + k] : 0.f);
-              const float d1 = x[8 + k] - (covered ? a1[8 * jj + k] : 0.f);
-              sq = fmaf(d0, d0, sq);
-              sq = fmaf(d1, d1, sq);
+              const float d0 = x[k] - a0[8 * jj + k];
+              const float d1 = x[8 + k] - a1[8 * jj + k];
+              sq0 = fmaf(d0, d0, sq0);
+              sq1 = fmaf(d1, d1, sq1);
             }
           }
-          gate_acc += (double)sq;
+          gate_acc += (double)(sq0 + sq1);
         }
       } else if constexpr (MODE == 2) {
         // mean absolute distance between the source row and the anchor's reconstruction of it, this
