@@ -40,9 +40,9 @@ constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
 constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
 constexpr int kOperandBytes = 128 * 128;          // 128 channels x (32 hi + 32 lo) bf16
 constexpr int kWeightBytes = kTileTok * 4;
-constexpr int NSTAGE = 3;                         // base-tile slots
-constexpr int NC = 5;                             // coefficient blocks in flight (HBM latency)
-constexpr int NO = 2;                             // operand blocks in flight (served by L2)
+// Ring depths are template parameters of the kernel: NSTAGE base-tile slots, NC coefficient blocks in
+// flight (HBM latency), NO operand blocks in flight (served by L2).  Up to three rank blocks per tile
+// the base tiles are what the pipeline runs short of (4, 3, 3); beyond that the coefficient blocks (3, 5, 2).
 
 struct Block {                 // one rank block of one anchor
   const float* w_k;            // token weights of the anchor [T_pad] (nullptr: all ones)
@@ -66,6 +66,7 @@ struct MultiLaunch {
   CUtensorMap coeff_k[KVC_MULTI_MAX_BLOCKS], coeff_v[KVC_MULTI_MAX_BLOCKS];   // per anchor
 };
 
+template <int NSTAGE, int NC, int NO>
 struct Ctrl {
   uint64_t full[NSTAGE], ready[NSTAGE], empty[NSTAGE];      // base-tile ring
   uint64_t cfull[NC], conv[NC], cempty[NC];                 // coefficient ring (one entry per rank block of a tile)
@@ -141,7 +142,9 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   }
 }
 
+template <int NSTAGE, int NC, int NO>
 __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
+  using Ctrl = tcm::Ctrl<NSTAGE, NC, NO>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -591,6 +594,21 @@ static bool encode_operand(CUtensorMap* m, const __nv_bfloat16* ws, int64_t rows
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <int NSTAGE, int NC, int NO>
+static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s) {
+  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
+                          (size_t)NO * kOperandBytes + sizeof(Ctrl<NSTAGE, NC, NO>);
+  static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
+  static bool set = false;
+  if (!set) {
+    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    set = true;
+  }
+  apply_multi_tc_kernel<NSTAGE, NC, NO><<<grid, kThreads, smem, s>>>(M);
+  return cudaGetLastError();
+}
+
 }  // namespace tcm
 
 static_assert(offsetof(tcm::MultiLaunch, cs) % 16 == 0 && offsetof(tcm::MultiLaunch, sn) % 16 == 0, "rope tables: float4 reads");
@@ -671,17 +689,8 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(M.total_tiles < sms ? M.total_tiles : sms);
-  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
-                          (size_t)NO * kOperandBytes + sizeof(Ctrl);
-  static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
-  static bool set = false;
-  if (!set) {
-    if (cudaFuncSetAttribute(apply_multi_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return KVC_E_CUDA;
-    set = true;
-  }
-  apply_multi_tc_kernel<<<grid, kThreads, smem, s>>>(M);
-  return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+  const cudaError_t e = nb <= 3 ? tcm::launch_multi_t<4, 3, 3>(M, grid, s) : tcm::launch_multi_t<3, 5, 2>(M, grid, s);
+  return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
 }  // namespace kvc
