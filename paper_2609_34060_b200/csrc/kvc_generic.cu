@@ -363,23 +363,21 @@ __global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant
 // ---------------------------------------------------------------------------------
 // Symmetric eigensolver for the top-r eigenpairs of the d x d Gram matrices (Eq. 7: the basis
 // rows are the right singular vectors of Delta for its largest r singular values).
-// One block per matrix, everything in shared memory, float32:
-//   1. Householder reduction to tridiagonal form T = Q^T G Q (reflectors kept in place);
-//   2. all eigenvalues of T by bisection on Sturm counts (one thread per eigenvalue);
+// One block of 256 threads per matrix, float32, two blocks per SM:
+//   1. Householder reduction to tridiagonal form T = Q^T G Q, the matrix in registers (two threads
+//      per row), the reflectors in shared memory;
+//   2. all eigenvalues of T by multisection on Sturm counts (one grid of 512 points shared by all
+//      eigenvalues, then 5-section by two threads per eigenvalue);
 //   3. eigenvectors of T for the r largest by inverse iteration (tridiagonal LU with partial
-//      pivoting, one thread per vector), re-orthogonalised (Gram-Schmidt, twice) after each of
-//      two iterations so that equal or close eigenvalues still give an orthonormal set;
-//   4. back-transformation by the reflectors, sign convention, output.
+//      pivoting), re-orthonormalised through a Cholesky factor of their Gram matrix after every
+//      round; two rounds where the eigenvalues are separated, up to five where they crowd together,
+//      a vector that stays dependent on the earlier ones being drawn afresh;
+//   4. back-transformation by the reflectors, sign convention, output.  A row whose eigenvalue is
+//      below float32 resolution beside the largest one is zero.
 // The input is the sum of the partial Gram matrices, symmetrised; it is written back so that
 // the final Gram matrix stays readable in the workspace.
 // ---------------------------------------------------------------------------------
-#ifndef KVC_EIG_THREADS
-#define KVC_EIG_THREADS 256
-#endif
-constexpr int kEigThreads = KVC_EIG_THREADS;
-#ifndef KVC_EIG_MINBLOCKS
-#define KVC_EIG_MINBLOCKS 2
-#endif
+constexpr int kEigThreads = 256;                  // 128 and 512 were measured slower (per-matrix latency against resident matrices)
 constexpr int kEigMaxR = 64;
 
 __device__ __forceinline__ float warp_sum(float x) {
@@ -389,7 +387,7 @@ __device__ __forceinline__ float warp_sum(float x) {
 }
 
 template <int N>
-__global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs) {
+__global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs) {
   extern __shared__ __align__(16) float smem[];
   constexpr int n = N;
   constexpr int np = N + 4;           // row pitch of A = 4 (mod 32)
@@ -418,13 +416,11 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   // + 3), so the work of a row stays spread over its threads as the trailing block shrinks.
   // Reflector k is written to row k of the shared-memory copy (zeros left of the sub-diagonal), where
   // the back-transformation finds it later.  Two block barriers per step.
-  constexpr int TPR = kEigThreads / N;          // threads per row: 4 (N = 128) or 8 (N = 64) at 512 threads
-  constexpr int NCH = N / (4 * TPR);            // chunks per thread: 8 or 2
-#ifndef KVC_EIG_GCH
-#define KVC_EIG_GCH 4
-#endif
-  constexpr int GCH = NCH < KVC_EIG_GCH ? NCH : KVC_EIG_GCH;   // chunks handled together: loads first, then arithmetic
+  constexpr int TPR = kEigThreads / N;          // threads per row: 2 (N = 128) or 4 (N = 64)
+  constexpr int NCH = N / (4 * TPR);            // chunks per thread: 16 or 4
+  constexpr int GCH = NCH < 4 ? NCH : 4;        // chunks handled together: loads first, then arithmetic
   static_assert(TPR * N == kEigThreads && NCH * 4 * TPR == N && TPR <= 32 && NCH % GCH == 0, "thread layout");
+  static_assert(kEigThreads == 256, "the 2 x 2 blocks of the vectors' Gram matrix and the grid of Sturm counts assume 256 threads");
   const int trow = tid / TPR, tq = tid % TPR;
   float a[NCH][4];
   {
@@ -647,7 +643,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
     // TPE threads per eigenvalue, two points per thread.  First one grid of 2 x threads points over the
     // whole interval, shared by all eigenvalues; then each round tests 2 TPE interior points of the
     // eigenvalue's own interval, which shrinks (2 TPE + 1)x.
-    constexpr int TPE = kEigThreads / 128;         // 4 at 512 threads, 2 at 256
+    constexpr int TPE = kEigThreads / 128;         // 2
     constexpr int kGrid = 2 * kEigThreads;
     // (grid + 1) * (2 TPE + 1)^rounds beyond 2^27:  1025 * 9^6,  513 * 5^8,  257 * 3^12
     constexpr int kRounds = TPE == 4 ? 6 : (TPE == 2 ? 8 : 12);
@@ -738,10 +734,7 @@ __global__ void __launch_bounds__(kEigThreads, KVC_EIG_MINBLOCKS) eig_tridiag_ke
   // A vector whose pivot falls below kPivBad is (numerically) a combination of the earlier ones: it is
   // left out of the factor, so that it cannot blow the later columns up, and drawn afresh for the next
   // round.  One that is still in that state after the last round gives a zero basis row, flagged.
-#ifndef KVC_EIG_MAXITER
-#define KVC_EIG_MAXITER 5
-#endif
-  constexpr int kMaxIter = KVC_EIG_MAXITER;
+  constexpr int kMaxIter = 5;
   constexpr float kPivOk = 1e-2f, kPivBad = 1e-4f;
   float min_piv = 1.f;
   uint32_t bad0 = 0u, bad1 = 0u;                  // vectors 0-31 / 32-63 left out in the last round
