@@ -628,16 +628,18 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
       return y;
     };
     auto sturm2 = [&](float xa, float xb, int& ca, int& cb) {
+      // a pivot counts as negative by its sign bit, so that -0 (followed by +inf) and +0 (followed by
+      // -inf) both add one to the count
       float qa = ds[0] - xa, qb = ds[0] - xb;
-      ca = qa < 0.f;
-      cb = qb < 0.f;
+      ca = (int)(__float_as_uint(qa) >> 31);
+      cb = (int)(__float_as_uint(qb) >> 31);
 #pragma unroll 8
       for (int i = 1; i < n; ++i) {
         const float d = ds[i], e = -es2[i - 1];
         qa = fmaf(e, rcp(qa), d - xa);
         qb = fmaf(e, rcp(qb), d - xb);
-        ca += qa < 0.f;
-        cb += qb < 0.f;
+        ca += (int)(__float_as_uint(qa) >> 31);
+        cb += (int)(__float_as_uint(qb) >> 31);
       }
     };
     // TPE threads per eigenvalue, two points per thread.  First one grid of 2 x threads points over the
