@@ -740,9 +740,16 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   constexpr float kPivOk = 1e-2f, kPivBad = 1e-4f;
   float min_piv = 1.f;
   uint32_t bad0 = 0u, bad1 = 0u;                  // vectors 0-31 / 32-63 left out in the last round
+  // When the last round's factor was not close to the identity (pivot below kPivFine), the vectors
+  // it left are orthonormal only to about eps times the condition of their Gram matrix: one more
+  // pass, re-orthonormalisation alone, brings them to rounding level.
+  constexpr float kPivFine = 0.5f;
+  bool polish = false;                            // this pass: no solve
 #pragma unroll 1
-  for (int iter = 0; iter < kMaxIter; ++iter) {   // one copy of the round: later rounds are rare
-    if (r_eff <= 32) {
+  for (int iter = 0; iter <= kMaxIter; ++iter) {  // one copy of the round: later rounds are rare
+    if (polish) {
+      // nothing to solve
+    } else if (r_eff <= 32) {
       // Solve (T - s I) y = z in place, lane j of every warp working on vector j: elimination with
       // partial pivoting runs down the rows, SPW rows per warp, each warp keeping its part of U
       // (reciprocal pivot, first super-diagonal, one swap bit per row: the second super-diagonal is
@@ -1085,10 +1092,14 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
       }
       __syncthreads();
     }
+    if (polish) break;                            // (a vector that was left out keeps its mark)
     bad0 = __float_as_uint(red[1]);
     bad1 = __float_as_uint(red[2]);
     min_piv = red[0];                             // written before the last two barriers; next written after the next one
-    if (iter >= 1 && min_piv >= kPivOk) break;    // uniform over the block
+    if ((iter >= 1 && min_piv >= kPivOk) || iter == kMaxIter - 1) {   // uniform over the block
+      if (min_piv >= kPivFine) break;
+      polish = true;
+    }
   }
   if (tid == 0 && (bad0 | bad1) != 0u) atomicOr(p.status, 4u);   // vectors still dependent after the last round: flagged
 

@@ -192,6 +192,24 @@ class Request:
     prefix: tuple
 
 
+def clustered_rows(T: int, d: int, seed: int, tag: int):
+    """A [T, d] bf16 matrix whose singular values come in a few clusters of (nearly) equal values
+    over a low floor: orthonormal columns (QR of a Gaussian) times the drawn values times an
+    orthogonal matrix, rounded to bf16 (which spreads every cluster by about 2^-9).  Returns the
+    matrix and the singular values drawn.  A stress input for the truncated SVD of the update."""
+    g = _gen("cpu", seed, tag)
+    n_cl = int(torch.randint(1, 6, (1,), generator=g))
+    vals: List[float] = []
+    for _ in range(n_cl):
+        level = 10.0 ** float(torch.empty(1).uniform_(-2.0, 1.0, generator=g))
+        vals += [level] * int(torch.randint(1, 12, (1,), generator=g))
+    floor = 10.0 ** float(torch.empty(1).uniform_(-5.0, -3.0, generator=g))
+    sv = torch.tensor(sorted((vals + [floor] * d)[:d], reverse=True), dtype=torch.float64)
+    u, _ = torch.linalg.qr(torch.randn(T, d, generator=g, dtype=torch.float64))
+    v, _ = torch.linalg.qr(torch.randn(d, d, generator=g, dtype=torch.float64))
+    return ((u * sv) @ v.T * 16.0).to(torch.bfloat16), sv
+
+
 def serving_batch(n_requests: int = 64, seed: int = 0, median_T: int = 4096, sigma_ln: float = 0.6,
                   t_lo: int = 1024, t_hi: int = 32768, agents_lo: int = 3, agents_hi: int = 6,
                   ranks: Sequence[int] = (16, 32, 64), prefix_lo: int = 64, prefix_hi: int = 512) -> List[Request]:

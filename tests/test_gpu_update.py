@@ -299,6 +299,39 @@ def test_fit_degenerate_spectra(d):
     assert kvc.kvc_status_poll() == 0
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_fit_clustered_spectra(d):
+    """Twenty drawn spectra per head dimension with clusters of (nearly) equal singular values over a low
+    floor, each factorised at one rank up to 32 and one above (the two vector paths of the eigensolver).
+    Checked against a library eigensolver on the same bf16 data: eigenvalues, orthonormal rows at
+    rounding level, a residual at the tail energy (allowance as in the rank sweep), nothing flagged, and
+    as many live rows as there are eigenvalues the float32 solver can tell from zero."""
+    T = 512
+    for trial in range(20):
+        x, _ = wl.clustered_rows(T, d, seed=11, tag=100 * d + trial)
+        xn = x.to(torch.float64).numpy()
+        w = np.linalg.eigvalsh(xn.T @ xn)[::-1]
+        g = torch.Generator().manual_seed(1000 * d + trial)
+        for r in (int(torch.randint(1, 33, (1,), generator=g)), int(torch.randint(33, min(d, 64) + 1, (1,), generator=g))):
+            cache = kvc.Cache(x.reshape(1, 1, T, d).contiguous().to(DEV), x.reshape(1, 1, T, d).contiguous().to(DEV))
+            st = kvc.State(torch.zeros(1, 1, T, r, device=DEV), torch.zeros(1, 1, T, r, device=DEV),
+                           torch.zeros(1, 1, r, d, device=DEV), torch.zeros(1, 1, r, d, device=DEV))
+            ws = torch.empty(kvc.kvc_workspace_bytes(cache, st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+            kvc.kvc_state_update(None, cache, 0, kvc.Rope(10000.0), st, kvc.KVC_FIT, workspace=ws)
+            torch.cuda.synchronize()
+            assert kvc.kvc_status_poll() == 0, (trial, r)
+            ev = ws.view(torch.float32)[2 * 2 * d * d + d: 2 * 2 * d * d + 2 * d].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(ev - w)) <= 1e-4 * w[0], (trial, r)
+            B = st.basis_v[0, 0].cpu().numpy().astype(np.float64)
+            c = st.coeff_v[0, 0].cpu().numpy().astype(np.float64)
+            live = np.abs(B).sum(axis=1) > 0
+            k = int(live.sum())
+            assert np.all(live[:k]) and k >= min(r, int(np.sum(w > 1e-5 * w[0]))), (trial, r, k)
+            assert np.max(np.abs(B[:k] @ B[:k].T - np.eye(k))) <= 1e-5, (trial, r)
+            res = float(np.sum((xn - c @ B) ** 2))
+            assert res <= float(np.sum(w[k:])) + 8 * r * 1.2e-6 * w[0] + 1e-9 * float(np.sum(w)), (trial, r)
+
+
 def test_effective_rank_from_fit_eigenvalues():
     """Sec. 3.1's diagnostic on the eigenvalues a FIT leaves behind: a deviation of exact rank 8 plus
     bf16 rounding noise has effective rank <= 8 at 90 % energy and matches the oracle's count on the
