@@ -665,21 +665,27 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
               uint4* s1p = reinterpret_cast<uint4*>(sr + kHalfBytes + o);
               uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
               if (live) {
-                float x[16], y[16];
-                unpack8(*s0p, x);
-                unpack8(*s1p, x + 8);
-                unpack8(*t0p, y);
-                unpack8(*t1p, y + 8);
+                // packed float32 pairs throughout: word w of a 16-byte chunk holds channels 2w, 2w + 1
+                const uint4 sa = *s0p, sb = *s1p, ta = *t0p, tb = *t1p;
+                const uint32_t sw0[4] = {sa.x, sa.y, sa.z, sa.w}, sw1[4] = {sb.x, sb.y, sb.z, sb.w};
+                const uint32_t tw0[4] = {ta.x, ta.y, ta.z, ta.w}, tw1[4] = {tb.x, tb.y, tb.z, tb.w};
+                f32x2 xa[4], xb[4];
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  xa[z] = f2_from_bf16x2(sw0[z]);
+                  xb[z] = f2_from_bf16x2(sw1[z]);
+                }
                 if (rotate) {
                   const float4 c0 = *reinterpret_cast<const float4*>(f.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(f.cs + 8 * j + 4);
                   const float4 s0 = *reinterpret_cast<const float4*>(f.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(f.sn + 8 * j + 4);
-                  const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-                  const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                  const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
+                  const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
+                  const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
 #pragma unroll
-                  for (int z = 0; z < 8; ++z) {
-                    const float a = x[z], b = x[8 + z];
-                    x[z] = a * cs[z] - b * sn[z];
-                    x[8 + z] = a * sn[z] + b * cs[z];
+                  for (int z = 0; z < 4; ++z) {
+                    const f32x2 a = xa[z], b = xb[z];
+                    xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));       // a cos - b sin
+                    xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));        // a sin + b cos
                   }
                 }
                 uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
@@ -688,8 +694,13 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
                 uint32_t* lp1 = reinterpret_cast<uint32_t*>(&l1);
 #pragma unroll
                 for (int z = 0; z < 4; ++z) {
-                  split2x(y[2 * z] - x[2 * z], y[2 * z + 1] - x[2 * z + 1], hp0[z], lp0[z]);
-                  split2x(y[8 + 2 * z] - x[8 + 2 * z], y[9 + 2 * z] - x[9 + 2 * z], hp1[z], lp1[z]);
+                  // H = bf16(Delta); 2 L = bf16(Delta - H) with one added to both exponents (the doubling is
+                  // exact; a zero remainder becomes 2^-126, which no sum notices)
+                  const f32x2 da = f2_sub(f2_from_bf16x2(tw0[z]), xa[z]), db = f2_sub(f2_from_bf16x2(tw1[z]), xb[z]);
+                  hp0[z] = f2_to_bf16x2(da);
+                  hp1[z] = f2_to_bf16x2(db);
+                  lp0[z] = f2_to_bf16x2(f2_sub(da, f2_from_bf16x2(hp0[z]))) + 0x00800080u;
+                  lp1[z] = f2_to_bf16x2(f2_sub(db, f2_from_bf16x2(hp1[z]))) + 0x00800080u;
                 }
               }
               *t0p = h0;
