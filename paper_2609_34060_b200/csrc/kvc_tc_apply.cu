@@ -663,22 +663,25 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
 #pragma unroll
             for (int k = 0; k < 16; ++k) a0[k] = a1[k] = 0.f;
           }
-          float sq0 = 0.f, sq1 = 0.f;
+          f32x2 sq0 = f2_pack(0.f, 0.f), sq1 = sq0;    // packed float32 pairs
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj) {
             const int j = 2 * cq + jj;
-            float x[16];
-            unpack8(*reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4)), x);
-            unpack8(*reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4)), x + 8);
+            const uint4 ua = *reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4));
+            const uint4 ub = *reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4));
+            const uint32_t wa[4] = {ua.x, ua.y, ua.z, ua.w}, wb[4] = {ub.x, ub.y, ub.z, ub.w};
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              const float d0 = x[k] - a0[8 * jj + k];
-              const float d1 = x[8 + k] - a1[8 * jj + k];
-              sq0 = fmaf(d0, d0, sq0);
-              sq1 = fmaf(d1, d1, sq1);
+            for (int z = 0; z < 4; ++z) {
+              const f32x2 d0 = f2_sub(f2_from_bf16x2(wa[z]), f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
+              const f32x2 d1 = f2_sub(f2_from_bf16x2(wb[z]), f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]));
+              sq0 = f2_fma(d0, d0, sq0);
+              sq1 = f2_fma(d1, d1, sq1);
             }
           }
-          gate_acc += (double)(sq0 + sq1);
+          float s00, s01, s10, s11;
+          f2_unpack(sq0, s00, s01);
+          f2_unpack(sq1, s10, s11);
+          gate_acc += (double)((s00 + s01) + (s10 + s11));
         }
       } else if constexpr (MODE == 2) {
         // mean absolute distance between the source row and the anchor's reconstruction of it, this
@@ -705,12 +708,19 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
               const float c2[8] = {cc.x, cc.y, cc.z, cc.w, cd.x, cd.y, cd.z, cd.w};
               const float s2[8] = {sc4.x, sc4.y, sc4.z, sc4.w, sd4.x, sd4.y, sd4.z, sd4.w};
 #pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const float u = x[k], v = x[8 + k], au = a0[8 * jj + k], av = a1[8 * jj + k];
-                // source rotated by the first table minus reconstruction rotated by the second
-                const float du = fmaf(u, c1[k], -v * s1[k]) - fmaf(au, c2[k], -av * s2[k]);
-                const float dv = fmaf(u, s1[k], v * c1[k]) - fmaf(au, s2[k], av * c2[k]);
-                sa += fabsf(du) + fabsf(dv);
+              for (int z = 0; z < 4; ++z) {
+                // packed pairs: source rotated by the first table minus reconstruction rotated by the second
+                const f32x2 u = f2_pack(x[2 * z], x[2 * z + 1]), v = f2_pack(x[8 + 2 * z], x[9 + 2 * z]);
+                const f32x2 au = f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]), av = f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]);
+                const f32x2 pc1 = f2_pack(c1[2 * z], c1[2 * z + 1]), ps1 = f2_pack(s1[2 * z], s1[2 * z + 1]);
+                const f32x2 pc2 = f2_pack(c2[2 * z], c2[2 * z + 1]), ps2 = f2_pack(s2[2 * z], s2[2 * z + 1]);
+                const f32x2 nps1 = f2_pack(-s1[2 * z], -s1[2 * z + 1]), nps2 = f2_pack(-s2[2 * z], -s2[2 * z + 1]);
+                const f32x2 du = f2_sub(f2_fma(u, pc1, f2_mul(v, nps1)), f2_fma(au, pc2, f2_mul(av, nps2)));
+                const f32x2 dv = f2_sub(f2_fma(u, ps1, f2_mul(v, pc1)), f2_fma(au, ps2, f2_mul(av, pc2)));
+                float e0, e1, e2, e3;
+                f2_unpack(du, e0, e1);
+                f2_unpack(dv, e2, e3);
+                sa += (fabsf(e0) + fabsf(e1)) + (fabsf(e2) + fabsf(e3));
               }
             } else {
 #pragma unroll
