@@ -187,7 +187,7 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all", grouped=False):
     states = [kvc.State(torch.empty(L, H, T, r, device=dev), torch.empty(L, H, T, r, device=dev),
                         torch.empty(L, H, r, d, device=dev), torch.empty(L, H, r, d, device=dev)) for _ in range(n - 1)]
     outs = [mk(tables[n + a]) for a in range(1, n)]
-    ws = torch.empty(max(kvc.kvc_workspace_bytes(a0, states[0], kvc.KVC_FIT), 256), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(kvc.kvc_workspace_bytes(a0, states[0], kvc.KVC_FIT_FAST), 256), dtype=torch.uint8, device=dev)
     return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws, "only": only}
 
 
@@ -298,7 +298,7 @@ def run_step(W, kvc, ev=None):
         for a in range(1, n):
             mark("update_begin")
             kvc.kvc_state_update(W["true"][a - 1], W["true"][a], pl[a] - pl[a - 1], rope, W["states"][a - 1],
-                                 kvc.KVC_FIT, workspace=W["ws"])
+                                 W.get("fit_mode", kvc.KVC_FIT_FAST), workspace=W["ws"])
             mark("update_end")
     if only != "update":
         mark("chain_begin")
@@ -393,6 +393,8 @@ def main():
     ap.add_argument("--rank", type=int, default=0, help="override the rank r (experiments)")
     ap.add_argument("--chain", default="hops", choices=["hops", "fused"],
                     help="hops: kvc_chain, one launch per hop; fused: kvc_chain_fused, one pass over agent 0's cache")
+    ap.add_argument("--fit", default="fast", choices=["fast", "full"],
+                    help="fast: KVC_FIT_FAST (top-r subspace solver, full eigensolver where it declines); full: KVC_FIT")
     ap.add_argument("--grouped", type=int, default=0, help="1: per-layer states (D = H d), with --only apply")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
     ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi", "weights"],
@@ -415,7 +417,7 @@ def main():
              f"{cfg.name}: L={cfg.L} Hkv={cfg.H} d={cfg.d} T={cfg.T} agents={cfg.n_agents} r={cfg.r} "
              f"{'paged16' if cfg.paged else 'contiguous'} bf16, seed {cfg.seed}" + (" (two output buffers in turn)" if ring else ""))
     config = {"workload": wname,
-              "step": "per edge: kvc_state_update(FIT) ; then kvc_chain over all agents",
+              "step": f"per edge: kvc_state_update({'FIT_FAST' if args.fit == 'fast' else 'FIT'}) ; then kvc_chain over all agents",
               "l2": "inputs larger than L2 (126 MB): no flush between iterations", "parallelism": f"replicas x{world}",
               "only": args.only}
 
@@ -458,6 +460,7 @@ def main():
         W = build_ring(cfg.scaled(seed=cfg.seed + rank), dev, kvc)
     else:
         W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only, grouped=bool(args.grouped) and args.only == "apply")
+    W["fit_mode"] = kvc.KVC_FIT_FAST if args.fit == "fast" else kvc.KVC_FIT
     if args.chain == "fused" and W.get("kind") is None and W.get("outs") and args.only in ("all", "apply"):
         W["chain_ws"] = torch.empty(max(kvc.kvc_chain_workspace_bytes(W["true"][0], cfg.n_agents), 128), dtype=torch.uint8,
                                     device=dev)

@@ -53,6 +53,7 @@ extern "C" {
 
 #define KVC_PROJECT 0  /* bases given, compute coefficients                        */
 #define KVC_FIT     1  /* compute bases (truncated SVD), then coefficients         */
+#define KVC_FIT_FAST 2 /* as KVC_FIT, top-r subspace solver where the spectrum allows */
 
 #define KVC_PATH_AUTO    0  /* pick the fastest kernel that supports the arguments */
 #define KVC_PATH_GENERIC 1  /* CUDA-core kernels (any supported shape)             */
@@ -183,10 +184,24 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                eigenvalue; where eigenvalues lie closer than that, the rows span their
  *                common subspace.  st->basis_dtype must be KVC_F32 and r <= 64 (else
  *                KVC_E_UNSUPPORTED).
+ *   KVC_FIT_FAST: the same state (Eq. 7 asks for the r largest singular values only), but each
+ *                matrix is first tried with a block subspace iteration on its r leading
+ *                eigenvectors (r <= 32), which converges in a few steps when the spectrum has a
+ *                gap behind the r-th eigenvalue -- a deviation of rank r over a noise floor.  The
+ *                result is accepted only when, in float32, every row satisfies
+ *                |G b_j - lambda_j b_j| <= 1e-5 lambda_1 and the residual of the whole block is at most
+ *                2^-13 of the distance between lambda_r and a bound on every eigenvalue outside the
+ *                block (trace(G) minus the sum of the block's eigenvalues: G is positive
+ *                semi-definite); any other matrix is solved by KVC_FIT's full eigensolver in the same
+ *                call.  Bases, coefficients and the r leading eigenvalues meet KVC_FIT's accuracy.
+ *                Difference: for a matrix the subspace solver served, the d - r trailing eigenvalues in
+ *                the workspace all hold their MEAN (their exact sum divided by d - r), so the trace is
+ *                exact and kvc_effective_rank is exact whenever it does not exceed r.  Which solver
+ *                served which matrix is left in the workspace, see kvc_fit_solver.
  *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
  *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte
- *              aligned.  May be NULL when 0 is needed.  After a KVC_FIT call it holds, as
- *              float32: the Gram matrices [L, H, 2, d, d] (2 = K, V), then scratch of the
+ *              aligned.  May be NULL when 0 is needed.  After a KVC_FIT / KVC_FIT_FAST call it
+ *              holds, as float32: the Gram matrices [L, H, 2, d, d] (2 = K, V), then scratch of the
  *              same size, then the eigenvalues [L, H, 2, d] in descending order.
  * Errors as kvc_apply, plus KVC_E_WORKSPACE.
  */
@@ -195,6 +210,19 @@ int kvc_state_update(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, 
 
 /* Scratch kvc_state_update needs for this geometry and mode (0 for KVC_PROJECT). */
 size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mode);
+
+/*
+ * After a KVC_FIT_FAST update: DEVICE int32 [L, H, 2] inside its workspace, one entry per matrix
+ * (layer, head, K|V): KVC_SOLVER_SUBSPACE (0) when the subspace solver's result was accepted, otherwise
+ * the reason the full eigensolver ran instead.  NULL on bad arguments.
+ */
+#define KVC_SOLVER_SUBSPACE        0
+#define KVC_SOLVER_FULL_RANK     (-1)  /* min(r, d, n_cov) > 32: not tried                           */
+#define KVC_SOLVER_FULL_DEPENDENT  2   /* zero matrix, or block columns dependent at float32         */
+#define KVC_SOLVER_FULL_SLOW       3   /* block residual not at rounding level after five products   */
+#define KVC_SOLVER_FULL_NO_GAP     4   /* a-posteriori test failed: no gap behind the r-th eigenvalue */
+#define KVC_SOLVER_FULL_SWEEPS     5   /* Jacobi sweep limit                                         */
+const int32_t *kvc_fit_solver(const kvc_cache *tgt, const void *workspace);
 
 /*
  * kvc_state_update_noalloc -- kvc_state_update without a workspace argument.

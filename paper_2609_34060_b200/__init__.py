@@ -20,7 +20,9 @@ LIB_PATH = os.path.join(_HERE, "libkvc.so")
 KVC_CONTIG, KVC_PAGED = 0, 1
 KVC_F32, KVC_BF16 = 0, 1
 KVC_ROPE_HALF, KVC_ROPE_INTERLEAVED = 0, 1
-KVC_PROJECT, KVC_FIT = 0, 1
+KVC_PROJECT, KVC_FIT, KVC_FIT_FAST = 0, 1, 2
+(KVC_SOLVER_SUBSPACE, KVC_SOLVER_FULL_RANK, KVC_SOLVER_FULL_DEPENDENT, KVC_SOLVER_FULL_SLOW, KVC_SOLVER_FULL_NO_GAP,
+ KVC_SOLVER_FULL_SWEEPS) = (0, -1, 2, 3, 4, 5)
 KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
 KVC_GROUP_HEAD, KVC_GROUP_LAYER = 0, 1
 KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4
@@ -33,7 +35,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_chain_fused", "kvc_chain_workspace_bytes",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_chain_fused", "kvc_chain_workspace_bytes",
 )
 
 
@@ -97,6 +99,8 @@ def load(path: Optional[str] = None):
     lib.kvc_effective_rank.argtypes = [vp, i32, i32, C.c_double, vp, vp]
     lib.kvc_fit_eigenvalues.argtypes = [PC, vp]
     lib.kvc_fit_eigenvalues.restype = vp
+    lib.kvc_fit_solver.argtypes = [PC, vp]
+    lib.kvc_fit_solver.restype = vp
     lib.kvc_state_realign.argtypes = [PS, i32, i32, i32, i32, PR, vp, vp]
     lib.kvc_token_weights.argtypes = [PC, i32, PS, C.POINTER(i32), i32, PR, C.c_double, vp, vp, vp, sz, vp]
     lib.kvc_token_weights_workspace_bytes.argtypes = [PC, i32]
@@ -383,6 +387,18 @@ def kvc_effective_rank(tgt: Cache, workspace: torch.Tensor, energy: float = 0.9,
     _check(load().kvc_effective_rank(ev, tgt.L * tgt.H * 2, tgt.d, float(energy), out.data_ptr(), _stream(stream)),
            "kvc_effective_rank")
     return out
+
+
+def kvc_fit_solver(tgt: Cache, workspace: torch.Tensor) -> torch.Tensor:
+    """int32 [L, H, 2] view into the workspace of a KVC_FIT_FAST update: KVC_SOLVER_SUBSPACE (0) where
+    the subspace solver served the matrix, else the reason the full eigensolver ran."""
+    c = tgt.struct()
+    p = load().kvc_fit_solver(C.byref(c), workspace.data_ptr())
+    if not p:
+        raise KvcError(KVC_E_INVALID_ARG, "kvc_fit_solver")
+    off = p - workspace.data_ptr()
+    n = tgt.L * tgt.H * 2
+    return workspace.view(torch.uint8)[off: off + 4 * n].view(torch.int32).view(tgt.L, tgt.H, 2)
 
 
 def kvc_state_realign(st: State, shift: int, rope: Rope, out: Optional[torch.Tensor] = None, stream=None) -> State:

@@ -286,15 +286,24 @@ int kvc_chain_fused(const kvc_cache* agent0, int32_t n_agents, const int32_t* pr
   return kvc_chain(agent0, n_agents, prefix_len, states, rope, outs, stream);
 }
 
-size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
-  if (!tgt || !st || mode != KVC_FIT) return 0;
+// FIT workspace: two partial Grams, then the eigenvalues; KVC_FIT_FAST adds one int32 per matrix
+// (which solver served it) on the next 256-byte boundary.
+static size_t fit_evals_end(const kvc_cache* tgt) {
   const size_t m = (size_t)tgt->L * tgt->H * 2;
-  return 2 * m * tgt->d * tgt->d * sizeof(float) + m * tgt->d * sizeof(float);   // two partial Grams + eigenvalues
+  return 2 * m * tgt->d * tgt->d * sizeof(float) + m * tgt->d * sizeof(float);
+}
+static size_t fit_solver_offset(const kvc_cache* tgt) { return (fit_evals_end(tgt) + 255) & ~(size_t)255; }
+
+size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
+  if (!tgt || !st || (mode != KVC_FIT && mode != KVC_FIT_FAST)) return 0;
+  if (mode == KVC_FIT) return fit_evals_end(tgt);
+  return fit_solver_offset(tgt) + (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t);
 }
 
 int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
                      int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
-  if (mode != KVC_PROJECT && mode != KVC_FIT) return KVC_E_INVALID_ARG;
+  if (mode != KVC_PROJECT && mode != KVC_FIT && mode != KVC_FIT_FAST) return KVC_E_INVALID_ARG;
+  const bool fit = mode != KVC_PROJECT;
   int rc;
   if ((rc = check_rope(rope)) != KVC_OK) return rc;
   DevCache dt, ds;
@@ -309,9 +318,9 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   if (st->n_cov > tgt->T) return KVC_E_SHAPE;
   if (st->r == 0 || st->n_cov == 0) return KVC_OK;   // nothing to compute
   if (!st->coeff_k || !st->coeff_v) return KVC_E_INVALID_ARG;
-  if (mode == KVC_FIT && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
-  if (mode == KVC_FIT && st->grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;   // needs a (H d) x (H d) eigensolver
-  if (mode == KVC_FIT) {
+  if (fit && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
+  if (fit && st->grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;   // needs a (H d) x (H d) eigensolver
+  if (fit) {
     const size_t need = kvc_workspace_bytes(tgt, st, mode);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_E_WORKSPACE;
   }
@@ -320,7 +329,7 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const int d = tgt->d;
 
-  if (mode == KVC_FIT) {
+  if (fit) {
     FitLaunch F;
     memset(&F, 0, sizeof(F));
     F.src = ds;
@@ -348,7 +357,23 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
       else if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
     }
     if (!gram_done && launch_gram_generic(F, d, s) != cudaSuccess) return KVC_E_CUDA;
-    if (launch_eig(F, d, s) != cudaSuccess) return KVC_E_CUDA;
+    if (mode == KVC_FIT_FAST) {
+      // the subspace solver first (it also sums and symmetrises the partial Grams); the full solver
+      // then serves the matrices it declined
+      int32_t* solver = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(workspace) + fit_solver_offset(tgt));
+      int r_eff = st->r < d ? st->r : d;
+      r_eff = r_eff < st->n_cov ? r_eff : st->n_cov;
+      if (r_eff <= kSubspaceMaxRank) {
+        if (launch_eig_subspace(F, d, solver, s) != cudaSuccess) return KVC_E_CUDA;
+        F.n_parts = 1;
+        if (launch_eig(F, d, solver, s) != cudaSuccess) return KVC_E_CUDA;
+      } else {
+        if (cudaMemsetAsync(solver, 0xff, (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t), s) != cudaSuccess) return KVC_E_CUDA;
+        if (launch_eig(F, d, nullptr, s) != cudaSuccess) return KVC_E_CUDA;
+      }
+    } else if (launch_eig(F, d, nullptr, s) != cudaSuccess) {
+      return KVC_E_CUDA;
+    }
   }
 
   UpdateLaunch U;
@@ -505,6 +530,11 @@ int kvc_effective_rank(const float* evals, int32_t n_matrices, int32_t d, double
 const float* kvc_fit_eigenvalues(const kvc_cache* tgt, const void* workspace) {
   if (!tgt || !workspace || tgt->L <= 0 || tgt->H <= 0 || tgt->d <= 0) return nullptr;
   return reinterpret_cast<const float*>(workspace) + 2 * (size_t)tgt->L * tgt->H * 2 * tgt->d * tgt->d;
+}
+
+const int32_t* kvc_fit_solver(const kvc_cache* tgt, const void* workspace) {
+  if (!tgt || !workspace || tgt->L <= 0 || tgt->H <= 0 || tgt->d <= 0) return nullptr;
+  return reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(workspace) + fit_solver_offset(tgt));
 }
 
 int kvc_state_realign(const kvc_state* st, int32_t L, int32_t H, int32_t d, int32_t shift, const kvc_rope* rope,
@@ -705,7 +735,7 @@ int64_t kvc_update_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode
   const int64_t coeff = cslabs * st->n_cov * st->r * 4;
   const int64_t basis = slabs * st->r * tgt->d * (st->basis_dtype == KVC_BF16 ? 2 : 4);
   int64_t b = rows + coeff + basis;                                          // projection pass
-  if (mode == KVC_FIT) b += rows + 2 * slabs * tgt->d * tgt->d * 4;          // Gram pass + G write/read
+  if (mode == KVC_FIT || mode == KVC_FIT_FAST) b += rows + 2 * slabs * tgt->d * tgt->d * 4;          // Gram pass + G write/read
   return b;
 }
 

@@ -387,7 +387,10 @@ __device__ __forceinline__ float warp_sum(float x) {
 }
 
 template <int N>
-__global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs) {
+__global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs,
+                                                                      const int32_t* __restrict__ solver) {
+  // solver != nullptr: the subspace solver went first; a matrix it served (solver[m] == 0) is done
+  if (solver != nullptr && solver[blockIdx.x] == 0) return;
   extern __shared__ __align__(16) float smem[];
   constexpr int n = N;
   constexpr int np = N + 4;           // row pitch of A = 4 (mod 32)
@@ -1251,7 +1254,7 @@ cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
+cudaError_t launch_eig(const FitLaunch& F, int d, const int32_t* solver, cudaStream_t s) {
   const int blocks = F.L * F.H * 2;
   if (blocks <= 0) return cudaSuccess;
   int r_eff = F.r < d ? F.r : d;
@@ -1265,9 +1268,9 @@ cudaError_t launch_eig(const FitLaunch& F, int d, cudaStream_t s) {
                            : cudaFuncSetAttribute(eig_tridiag_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   if (d == 128)
-    eig_tridiag_kernel<128><<<blocks, kEigThreads, smem, s>>>(F, zs);
+    eig_tridiag_kernel<128><<<blocks, kEigThreads, smem, s>>>(F, zs, solver);
   else
-    eig_tridiag_kernel<64><<<blocks, kEigThreads, smem, s>>>(F, zs);
+    eig_tridiag_kernel<64><<<blocks, kEigThreads, smem, s>>>(F, zs, solver);
   return cudaGetLastError();
 }
 
