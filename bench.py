@@ -187,7 +187,7 @@ def build_workload(cfg: wl.Config, dev, kvc, only="all", grouped=False):
     states = [kvc.State(torch.empty(L, H, T, r, device=dev), torch.empty(L, H, T, r, device=dev),
                         torch.empty(L, H, r, d, device=dev), torch.empty(L, H, r, d, device=dev)) for _ in range(n - 1)]
     outs = [mk(tables[n + a]) for a in range(1, n)]
-    ws = torch.empty(max(kvc.kvc_workspace_bytes(a0, states[0], kvc.KVC_FIT_FAST), 256), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(kvc.kvc_chain_update_workspace_bytes(true, states, kvc.KVC_FIT_FAST), 256), dtype=torch.uint8, device=dev)
     return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws, "only": only}
 
 
@@ -295,11 +295,15 @@ def run_step(W, kvc, ev=None):
         mark("chain_end")
         return
     if only != "apply":
-        for a in range(1, n):
-            mark("update_begin")
-            kvc.kvc_state_update(W["true"][a - 1], W["true"][a], pl[a] - pl[a - 1], rope, W["states"][a - 1],
-                                 W.get("fit_mode", kvc.KVC_FIT_FAST), workspace=W["ws"])
-            mark("update_end")
+        mark("update_begin")
+        if W.get("edges", "chain") == "chain":     # every edge's state in one call: one eigensolver launch for all
+            kvc.kvc_state_update_chain(W["true"], pl, rope, W["states"], W.get("fit_mode", kvc.KVC_FIT_FAST),
+                                       workspace=W["ws"])
+        else:
+            for a in range(1, n):
+                kvc.kvc_state_update(W["true"][a - 1], W["true"][a], pl[a] - pl[a - 1], rope, W["states"][a - 1],
+                                     W.get("fit_mode", kvc.KVC_FIT_FAST), workspace=W["ws"])
+        mark("update_end")
     if only != "update":
         mark("chain_begin")
         if W.get("chain_ws") is not None:
@@ -395,6 +399,8 @@ def main():
                     help="hops: kvc_chain, one launch per hop; fused: kvc_chain_fused, one pass over agent 0's cache")
     ap.add_argument("--fit", default="fast", choices=["fast", "full"],
                     help="fast: KVC_FIT_FAST (top-r subspace solver, full eigensolver where it declines); full: KVC_FIT")
+    ap.add_argument("--edges", default="chain", choices=["chain", "each"],
+                    help="chain: kvc_state_update_chain, all edges in one call; each: one kvc_state_update per edge")
     ap.add_argument("--grouped", type=int, default=0, help="1: per-layer states (D = H d), with --only apply")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
     ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi", "weights"],
@@ -417,7 +423,9 @@ def main():
              f"{cfg.name}: L={cfg.L} Hkv={cfg.H} d={cfg.d} T={cfg.T} agents={cfg.n_agents} r={cfg.r} "
              f"{'paged16' if cfg.paged else 'contiguous'} bf16, seed {cfg.seed}" + (" (two output buffers in turn)" if ring else ""))
     config = {"workload": wname,
-              "step": f"per edge: kvc_state_update({'FIT_FAST' if args.fit == 'fast' else 'FIT'}) ; then kvc_chain over all agents",
+              "step": (f"kvc_state_update_chain({'FIT_FAST' if args.fit == 'fast' else 'FIT'}) over all edges"
+                       if args.edges == "chain" else
+                       f"per edge: kvc_state_update({'FIT_FAST' if args.fit == 'fast' else 'FIT'})") + " ; then kvc_chain over all agents",
               "l2": "inputs larger than L2 (126 MB): no flush between iterations", "parallelism": f"replicas x{world}",
               "only": args.only}
 
@@ -461,6 +469,7 @@ def main():
     else:
         W = build_workload(cfg.scaled(seed=cfg.seed + rank), dev, kvc, args.only, grouped=bool(args.grouped) and args.only == "apply")
     W["fit_mode"] = kvc.KVC_FIT_FAST if args.fit == "fast" else kvc.KVC_FIT
+    W["edges"] = args.edges
     if args.chain == "fused" and W.get("kind") is None and W.get("outs") and args.only in ("all", "apply"):
         W["chain_ws"] = torch.empty(max(kvc.kvc_chain_workspace_bytes(W["true"][0], cfg.n_agents), 128), dtype=torch.uint8,
                                     device=dev)
@@ -587,6 +596,10 @@ def main():
         return
     peak, peak_kind = _peaks()
     hop_ms = chain_ms / hops
+    # kernels of the state update per step: a Gram and a projection pass per edge, and the eigensolver
+    # launches (FIT_FAST: subspace solver + full solver for what it declined), once for all edges or per edge
+    eig_launches = (2 if args.fit == "fast" else 1) * (1 if args.edges == "chain" else hops)
+    upd_launches = 2 * hops + eig_launches
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "gate distance (one anchor, Eq. 9)" if args.only == "gate" else "multi-anchor apply (Eq. 8)" if args.only == "multi" else "token-weight scores (one anchor, App. A.3)" if args.only == "weights" else "apply (one hop of kvc_chain)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
@@ -597,7 +610,9 @@ def main():
            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic", "config": config,
            "clocks": clocks, "e2e": e2e,
-           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (hops + 1 if args.only in ("gate", "multi", "weights") else hops if args.only == "apply" else (hops * 3 if args.only == "update" else hops * 4)),
+           "gpu_launches": args.steps * W["kernels"] if serving else args.steps * (
+               hops + 1 if args.only in ("gate", "multi", "weights") else
+               (0 if args.only == "update" else hops) + (0 if args.only == "apply" else upd_launches)),
            "roofline": roofline,
            "breakdown": {"apply_GBs": achieved, "apply_frac_of_8TBs_nominal": achieved / 8000.0,
                          "us_per_agent_layer": hop_ms * 1e3 / cfg.L,

@@ -106,7 +106,8 @@ typedef struct kvc_state {
 } kvc_state;
 
 /*
- * Feature grouping of a state (Sec. 3.1: B in R^{r x D} with "D the KV cache feature dimension").
+ * Feature grouping of a state (Sec. 3.1 factorises with B in R^{r x D}, D being the width of the cached
+ * features).
  *   KVC_GROUP_HEAD   one state per (layer, KV head), D = d:
  *                    coeff [L, H, n_cov, r], basis [L, H, r, d]                    (the default)
  *   KVC_GROUP_LAYER  one state per layer over all KV heads, D = H d: the coefficients of a token are
@@ -224,6 +225,33 @@ size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mo
 #define KVC_SOLVER_FULL_SWEEPS     5   /* Jacobi sweep limit                                         */
 const int32_t *kvc_fit_solver(const kvc_cache *tgt, const void *workspace);
 
+/* The argument checks of kvc_state_update (everything but the workspace), launching nothing. */
+int kvc_state_update_check(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,
+                           const kvc_state *st, int32_t mode);
+
+/*
+ * kvc_state_update_chain -- the states of every edge of a workflow in one call (the counterpart of
+ * kvc_chain for profiling, Sec. 3.2: a calibration trajectory yields every agent's true cache at once):
+ * for a = 1..n_agents-1
+ *     states[a-1] = kvc_state_update(src = agents[a-1], tgt = agents[a],
+ *                                    shift = prefix_len[a] - prefix_len[a-1], mode)
+ * with the same results as those n_agents-1 calls.  What differs is the schedule: the Gram passes of all
+ * edges run first, then ONE launch solves the eigenproblems of all edges (when the edges share geometry,
+ * r and n_cov; a single edge's 2 L H matrices fill the GPU's resident blocks unevenly and leave most SMs
+ * idle while the slowest matrices finish), then the projection passes.
+ *   agents     HOST array [n_agents] of caches (DEVICE data); prefix_len HOST int32 [n_agents];
+ *   states     HOST array [n_agents-1]; n_agents <= 16 (else KVC_E_TOO_LARGE).
+ *   workspace  DEVICE scratch of kvc_chain_update_workspace_bytes(...) bytes, 256-byte aligned: edge e
+ *              (0-based) owns the kvc_chain_update_edge_stride(...) bytes starting at the sum of the
+ *              strides of the edges before it, laid out as kvc_state_update's workspace
+ *              (kvc_fit_eigenvalues / kvc_fit_solver / kvc_effective_rank take that address).
+ * Errors as kvc_state_update; nothing is launched when any edge fails its checks.
+ */
+int kvc_state_update_chain(const kvc_cache *agents, int32_t n_agents, const int32_t *prefix_len, const kvc_rope *rope,
+                           kvc_state *states, int32_t mode, void *workspace, size_t workspace_bytes, void *stream);
+size_t kvc_chain_update_workspace_bytes(const kvc_cache *agents, int32_t n_agents, const kvc_state *states, int32_t mode);
+size_t kvc_chain_update_edge_stride(const kvc_cache *tgt, const kvc_state *st, int32_t mode);
+
 /*
  * kvc_state_update_noalloc -- kvc_state_update without a workspace argument.
  * (No counterpart in the paper: this exists for integration only.)
@@ -238,19 +266,24 @@ const int32_t *kvc_fit_solver(const kvc_cache *tgt, const void *workspace);
  * cudaMalloc / cudaFree and uses no allocating library routine; inputs and outputs are
  * still the caller's buffers, with the same meaning as in kvc_state_update.
  *
+ *  - The arguments are checked first, exactly as kvc_state_update checks them, and a call that
+ *    fails a check returns that error and launches nothing.
  *  - Capacity: kvc_workspace_bytes(tgt, st, mode) must not exceed
- *    KVC_STATIC_SCRATCH_BYTES, i.e. L*H <= 64 at d = 128 (L*H <= 255 at d = 64) in FIT
- *    mode; larger problems return KVC_E_TOO_LARGE and launch nothing (split them by
+ *    KVC_STATIC_SCRATCH_BYTES, i.e. L*H <= 64 at d = 128 (L*H <= 255 at d = 64) in the FIT
+ *    modes; larger problems return KVC_E_TOO_LARGE and launch nothing (split them by
  *    layer, or use kvc_state_update with your own workspace).  KVC_PROJECT needs no
  *    scratch and is never rejected for size.
- *  - The first call on each device looks up the array's device address (with that
- *    device current).  Make that first call before any stream capture begins.
+ *  - The first call on each device, in ANY mode (a KVC_PROJECT call or a call with an empty state
+ *    will do), looks up the array's device address with that device current.  The library's
+ *    modules load lazily, so this first call is also the moment the driver sets the array's
+ *    bytes aside on that GPU: make it at start-up, before the rest of the GPU's memory is handed to
+ *    a pool, and before any stream capture begins.  Later calls take no device memory.
  *  - All calls on one device share the one array, and it keeps the previous call's
- *    contents: the entry point clears the part it is about to use on `stream` first.
- *    Two calls whose device work can overlap (different streams, or different host
- *    threads on different streams) race on the array: serialise them.
+ *    contents.  Nothing needs clearing: every kernel of the update writes its part of the
+ *    scratch before anything reads it.  Two calls whose device work can overlap (different
+ *    streams, or different host threads on different streams) race on the array: serialise them.
  */
-#define KVC_STATIC_SCRATCH_BYTES (128 * (2 * 128 * 128 + 128) * 4)
+#define KVC_STATIC_SCRATCH_BYTES (128 * (2 * 128 * 128 + 128) * 4 + 1024)
 int kvc_state_update_noalloc(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,
                              kvc_state *st, int32_t mode, void *stream);
 
@@ -322,7 +355,8 @@ int kvc_apply_multi(const kvc_cache *src, const kvc_state *deltas, int32_t n_anc
 size_t kvc_multi_workspace_bytes(const kvc_cache *src, const kvc_state *deltas, int32_t n_anchors);
 
 /*
- * Effective rank (Sec. 3.1: "the minimum rank retaining 90% of the singular-value energy"), from the
+ * Effective rank (the diagnostic of Sec. 3.1: the smallest rank whose singular values carry a given
+ * share, there 90 %, of the summed squared singular values), from the
  * eigenvalues a KVC_FIT update leaves in its workspace (squared singular values of the factorised
  * deviation or cache).  For every matrix m of n_matrices:
  *     rank[m] = min { k : sum_{i<k} max(evals[m][i], 0) >= energy * sum_i max(evals[m][i], 0) }   (0 if the sum is 0)
@@ -337,8 +371,8 @@ int kvc_effective_rank(const float *evals, int32_t n_matrices, int32_t d, double
 const float *kvc_fit_eigenvalues(const kvc_cache *tgt, const void *workspace);
 
 /*
- * Positional re-alignment of a stored correction (App. A.2: a correction for a recurring prefix
- * relation "is profiled once, stored in low-rank form, and positionally re-aligned when reused").
+ * Positional re-alignment of a stored correction (App. A.2: the correction of a prefix relation that
+ * recurs is learned a single time, kept as its low-rank factors, and moved to the positions of each reuse).
  * A rotation is linear in the channels, Rot_s(c . B) = c . Rot_s(B), so re-aligning a stored key
  * correction by `shift` positions is rotating every row of its key basis by `shift`:
  *     basis_k_out[l,h,q,:] = Rot_shift(basis_k_in[l,h,q,:]) ,

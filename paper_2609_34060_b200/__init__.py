@@ -35,7 +35,8 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_chain_fused", "kvc_chain_workspace_bytes",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_state_update_check", "kvc_state_update_chain",
+    "kvc_chain_update_workspace_bytes", "kvc_chain_update_edge_stride", "kvc_chain_fused", "kvc_chain_workspace_bytes",
 )
 
 
@@ -87,6 +88,12 @@ def load(path: Optional[str] = None):
     lib.kvc_chain_workspace_bytes.restype = sz
     lib.kvc_state_update.argtypes = [PC, PC, i32, PR, PS, i32, vp, sz, vp]
     lib.kvc_state_update_noalloc.argtypes = [PC, PC, i32, PR, PS, i32, vp]
+    lib.kvc_state_update_check.argtypes = [PC, PC, i32, PR, PS, i32]
+    lib.kvc_state_update_chain.argtypes = [PC, i32, C.POINTER(i32), PR, PS, i32, vp, sz, vp]
+    lib.kvc_chain_update_workspace_bytes.argtypes = [PC, i32, PS, i32]
+    lib.kvc_chain_update_workspace_bytes.restype = sz
+    lib.kvc_chain_update_edge_stride.argtypes = [PC, PS, i32]
+    lib.kvc_chain_update_edge_stride.restype = sz
     lib.kvc_state_update_noalloc.restype = C.c_int
     lib.kvc_workspace_bytes.argtypes = [PC, PS, i32]
     lib.kvc_workspace_bytes.restype = sz
@@ -284,6 +291,32 @@ def kvc_chain_fused(agent0: Cache, prefix_len: Sequence[int], states: Sequence[S
                                   workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_chain_fused")
 
 
+def kvc_chain_update_workspace_bytes(agents: Sequence[Cache], states: Sequence[State], mode: int) -> int:
+    n = len(agents)
+    ag = (kvc_cache * n)(*[a.struct() for a in agents])
+    sts = (kvc_state * max(n - 1, 1))(*[s.struct() for s in states])
+    return int(load().kvc_chain_update_workspace_bytes(ag, n, sts, int(mode)))
+
+
+def kvc_chain_update_edge_stride(tgt: Cache, st: State, mode: int) -> int:
+    t, s = tgt.struct(), st.struct()
+    return int(load().kvc_chain_update_edge_stride(C.byref(t), C.byref(s), int(mode)))
+
+
+def kvc_state_update_chain(agents: Sequence[Cache], prefix_len: Sequence[int], rope: Rope, states: Sequence[State],
+                           mode: int, workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    """The states of every edge agents[a-1] -> agents[a] in one call (all eigensolves in one launch)."""
+    n = len(agents)
+    ag = (kvc_cache * n)(*[a.struct() for a in agents])
+    pl = (C.c_int32 * n)(*[int(x) for x in prefix_len])
+    sts = (kvc_state * max(n - 1, 1))(*[s.struct() for s in states])
+    r = rope.struct()
+    ws_ptr = 0 if workspace is None else workspace.data_ptr()
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().kvc_state_update_chain(ag, n, pl, C.byref(r), sts, int(mode), ws_ptr, ws_bytes, _stream(stream)),
+           "kvc_state_update_chain")
+
+
 def kvc_workspace_bytes(tgt: Cache, st: State, mode: int) -> int:
     t, s = tgt.struct(), st.struct()
     return int(load().kvc_workspace_bytes(C.byref(t), C.byref(s), int(mode)))
@@ -302,7 +335,7 @@ def kvc_state_update(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, s
                                    _stream(stream)), "kvc_state_update")
 
 
-KVC_STATIC_SCRATCH_BYTES = 128 * (2 * 128 * 128 + 128) * 4
+KVC_STATIC_SCRATCH_BYTES = 128 * (2 * 128 * 128 + 128) * 4 + 1024
 
 
 def kvc_state_update_noalloc(src: Optional[Cache], tgt: Cache, shift: int, rope: Rope, st: State, mode: int,

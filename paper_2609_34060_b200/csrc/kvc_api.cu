@@ -300,86 +300,114 @@ size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mo
   return fit_solver_offset(tgt) + (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t);
 }
 
-int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
-                     int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
+// One edge of a state update, checked and resolved: everything the launches need.
+struct UpdatePlan {
+  DevCache ds, dt;
+  DevState dstate;
+  const kvc_state* st;
+  const kvc_rope* rope;
+  int32_t shift, mode, L, H, d;
+  bool fit, empty;
+};
+
+// Every argument check of kvc_state_update except the workspace; launches nothing.
+static int plan_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, const kvc_state* st,
+                       int32_t mode, UpdatePlan* P) {
   if (mode != KVC_PROJECT && mode != KVC_FIT && mode != KVC_FIT_FAST) return KVC_E_INVALID_ARG;
-  const bool fit = mode != KVC_PROJECT;
+  memset(P, 0, sizeof(*P));
+  P->fit = mode != KVC_PROJECT;
+  P->mode = mode;
+  P->shift = shift;
+  P->st = st;
+  P->rope = rope;
   int rc;
   if ((rc = check_rope(rope)) != KVC_OK) return rc;
-  DevCache dt, ds;
-  memset(&ds, 0, sizeof(ds));
-  if ((rc = resolve_cache(tgt, &dt)) != KVC_OK) return rc;
+  if ((rc = resolve_cache(tgt, &P->dt)) != KVC_OK) return rc;
   if (src) {
-    if ((rc = resolve_cache(src, &ds)) != KVC_OK) return rc;
+    if ((rc = resolve_cache(src, &P->ds)) != KVC_OK) return rc;
     if (src->L != tgt->L || src->H != tgt->H || src->T != tgt->T || src->d != tgt->d) return KVC_E_SHAPE;
   }
-  DevState dst_state;
-  if ((rc = resolve_state(st, 1, &dst_state)) != KVC_OK) return rc;
+  if ((rc = resolve_state(st, 1, &P->dstate)) != KVC_OK) return rc;
   if (st->n_cov > tgt->T) return KVC_E_SHAPE;
-  if (st->r == 0 || st->n_cov == 0) return KVC_OK;   // nothing to compute
+  P->L = tgt->L;
+  P->H = tgt->H;
+  P->d = tgt->d;
+  P->empty = st->r == 0 || st->n_cov == 0;          // nothing to compute
+  if (P->empty) return KVC_OK;
   if (!st->coeff_k || !st->coeff_v) return KVC_E_INVALID_ARG;
-  if (fit && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
-  if (fit && st->grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;   // needs a (H d) x (H d) eigensolver
-  if (fit) {
-    const size_t need = kvc_workspace_bytes(tgt, st, mode);
-    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_E_WORKSPACE;
-  }
-  uint32_t* status = status_ptr();
-  if (!status) return KVC_E_CUDA;
-  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  const int d = tgt->d;
+  if (P->fit && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
+  if (P->fit && st->grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;   // needs a (H d) x (H d) eigensolver
+  return KVC_OK;
+}
 
-  if (fit) {
-    FitLaunch F;
-    memset(&F, 0, sizeof(F));
-    F.src = ds;
-    F.tgt = dt;
-    F.gram = reinterpret_cast<float*>(workspace);
-    F.evals = F.gram + 2 * (size_t)tgt->L * tgt->H * 2 * d * d;
+int kvc_state_update_check(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope,
+                           const kvc_state* st, int32_t mode) {
+  UpdatePlan P;
+  return plan_update(src, tgt, shift, rope, st, mode, &P);
+}
+
+static int r_eff_of(const UpdatePlan& P) {
+  int r_eff = P.st->r < P.d ? P.st->r : P.d;
+  return r_eff < P.st->n_cov ? r_eff : P.st->n_cov;
+}
+
+// Gram pass of one edge into its workspace; F is left ready for the eigensolver launches.
+static int fit_gram(const UpdatePlan& P, void* workspace, uint32_t* status, FitLaunch* Fp, cudaStream_t s) {
+  FitLaunch& F = *Fp;
+  memset(&F, 0, sizeof(F));
+  const kvc_state* st = P.st;
+  F.src = P.ds;
+  F.tgt = P.dt;
+  F.gram = reinterpret_cast<float*>(workspace);
+  F.evals = F.gram + 2 * (size_t)P.L * P.H * 2 * P.d * P.d;
+  F.n_parts = 1;
+  F.n_edges = 1;
+  F.edge_stride = 0;
+  F.basis_k = F.basis_k_e[0] = reinterpret_cast<float*>(st->basis_k);
+  F.basis_v = F.basis_v_e[0] = reinterpret_cast<float*>(st->basis_v);
+  F.r = st->r;
+  F.n_cov = st->n_cov;
+  F.pairing = P.rope->pairing;
+  F.shift = P.shift;
+  F.L = P.L;
+  F.H = P.H;
+  F.status = status;
+  rope_tables(P.rope, P.d, P.shift, F.cs, F.sn);
+  if (tl_path_force != KVC_PATH_GENERIC) {
+    const int trc = tc_gram(F, P.d, s);
+    if (trc == KVC_OK) {
+      F.n_parts = 2;
+      return KVC_OK;
+    }
+    if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  }
+  return launch_gram_generic(F, P.d, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+// Eigensolves of the F.n_edges edges that F describes (same geometry, r, n_cov and partial count).
+static int fit_eig(FitLaunch& F, int32_t mode, int d, int r_eff, size_t solver_off, size_t solver_bytes, cudaStream_t s) {
+  if (mode != KVC_FIT_FAST) return launch_eig(F, d, nullptr, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+  // the subspace solver first (it also sums and symmetrises the partial Grams); the full solver
+  // then serves the matrices it declined
+  int32_t* solver = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(F.gram) + solver_off);
+  if (r_eff <= kSubspaceMaxRank) {
+    if (launch_eig_subspace(F, d, solver, s) != cudaSuccess) return KVC_E_CUDA;
     F.n_parts = 1;
-    F.basis_k = reinterpret_cast<float*>(st->basis_k);
-    F.basis_v = reinterpret_cast<float*>(st->basis_v);
-    F.r = st->r;
-    F.n_cov = st->n_cov;
-    F.pairing = rope->pairing;
-    F.shift = shift;
-    F.L = tgt->L;
-    F.H = tgt->H;
-    F.status = status;
-    rope_tables(rope, d, shift, F.cs, F.sn);
-    bool gram_done = false;
-    if (tl_path_force != KVC_PATH_GENERIC) {
-      const int trc = tc_gram(F, d, s);
-      if (trc == KVC_OK) {
-        gram_done = true;
-        F.n_parts = 2;
-      }
-      else if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
-    }
-    if (!gram_done && launch_gram_generic(F, d, s) != cudaSuccess) return KVC_E_CUDA;
-    if (mode == KVC_FIT_FAST) {
-      // the subspace solver first (it also sums and symmetrises the partial Grams); the full solver
-      // then serves the matrices it declined
-      int32_t* solver = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(workspace) + fit_solver_offset(tgt));
-      int r_eff = st->r < d ? st->r : d;
-      r_eff = r_eff < st->n_cov ? r_eff : st->n_cov;
-      if (r_eff <= kSubspaceMaxRank) {
-        if (launch_eig_subspace(F, d, solver, s) != cudaSuccess) return KVC_E_CUDA;
-        F.n_parts = 1;
-        if (launch_eig(F, d, solver, s) != cudaSuccess) return KVC_E_CUDA;
-      } else {
-        if (cudaMemsetAsync(solver, 0xff, (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t), s) != cudaSuccess) return KVC_E_CUDA;
-        if (launch_eig(F, d, nullptr, s) != cudaSuccess) return KVC_E_CUDA;
-      }
-    } else if (launch_eig(F, d, nullptr, s) != cudaSuccess) {
-      return KVC_E_CUDA;
-    }
+    return launch_eig(F, d, solver, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
   }
+  for (int e = 0; e < F.n_edges; ++e)
+    if (cudaMemsetAsync(reinterpret_cast<char*>(solver) + e * F.edge_stride, 0xff, solver_bytes, s) != cudaSuccess) return KVC_E_CUDA;
+  return launch_eig(F, d, nullptr, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
 
+// Projection pass of one edge (U1 + U4): coefficients of the deviation in the state's bases.
+static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s) {
+  const kvc_state* st = P.st;
+  const int d = P.d;
   UpdateLaunch U;
   memset(&U, 0, sizeof(U));
-  U.src = ds;
-  U.tgt = dt;
+  U.src = P.ds;
+  U.tgt = P.dt;
   U.coeff_k = st->coeff_k;
   U.coeff_v = st->coeff_v;
   U.basis_k = st->basis_k;
@@ -387,15 +415,15 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   U.r = st->r;
   U.n_cov = st->n_cov;
   U.basis_bf16 = st->basis_dtype == KVC_BF16;
-  U.pairing = rope->pairing;
-  U.shift = shift;
-  U.L = tgt->L;
-  U.H = tgt->H;
+  U.pairing = P.rope->pairing;
+  U.shift = P.shift;
+  U.L = P.L;
+  U.H = P.H;
   U.status = status;
-  U.grouped = dst_state.grouped;
-  rope_tables(rope, d, shift, U.cs, U.sn);
+  U.grouped = P.dstate.grouped;
+  rope_tables(P.rope, d, P.shift, U.cs, U.sn);
   if (U.grouped) {      // every head adds its share: start from zero
-    const size_t nbytes = (size_t)tgt->L * st->n_cov * st->r * sizeof(float);
+    const size_t nbytes = (size_t)P.L * st->n_cov * st->r * sizeof(float);
     if (cudaMemsetAsync(st->coeff_k, 0, nbytes, s) != cudaSuccess || cudaMemsetAsync(st->coeff_v, 0, nbytes, s) != cudaSuccess)
       return KVC_E_CUDA;
   }
@@ -408,9 +436,100 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
     if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
   }
   U.tiles_per_slab = (st->n_cov + kGenericProjectTile - 1) / kGenericProjectTile;
-  const int64_t tiles = (int64_t)tgt->L * tgt->H * 2 * U.tiles_per_slab;
+  const int64_t tiles = (int64_t)P.L * P.H * 2 * U.tiles_per_slab;
   if (launch_project_generic(U, d, tiles, s) != cudaSuccess) return KVC_E_CUDA;
   tl_last_path = KVC_PATH_GENERIC;
+  return KVC_OK;
+}
+
+int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
+                     int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
+  UpdatePlan P;
+  int rc;
+  if ((rc = plan_update(src, tgt, shift, rope, st, mode, &P)) != KVC_OK) return rc;
+  if (P.empty) return KVC_OK;
+  if (P.fit) {
+    const size_t need = kvc_workspace_bytes(tgt, st, mode);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_E_WORKSPACE;
+  }
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (P.fit) {
+    FitLaunch F;
+    if ((rc = fit_gram(P, workspace, status, &F, s)) != KVC_OK) return rc;
+    const size_t solver_bytes = (size_t)P.L * P.H * 2 * sizeof(int32_t);
+    if ((rc = fit_eig(F, mode, P.d, r_eff_of(P), fit_solver_offset(tgt), solver_bytes, s)) != KVC_OK) return rc;
+  }
+  return project_edge(P, status, s);
+}
+
+size_t kvc_chain_update_edge_stride(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
+  return (kvc_workspace_bytes(tgt, st, mode) + 255) & ~(size_t)255;
+}
+
+size_t kvc_chain_update_workspace_bytes(const kvc_cache* agents, int32_t n_agents, const kvc_state* states, int32_t mode) {
+  if (!agents || !states || n_agents < 2) return 0;
+  size_t total = 0;
+  for (int a = 1; a < n_agents; ++a) total += kvc_chain_update_edge_stride(&agents[a], &states[a - 1], mode);
+  return total;
+}
+
+int kvc_state_update_chain(const kvc_cache* agents, int32_t n_agents, const int32_t* prefix_len, const kvc_rope* rope,
+                           kvc_state* states, int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!agents || !prefix_len || !states || n_agents < 1) return KVC_E_INVALID_ARG;
+  if (n_agents - 1 > kMaxFitEdges) return KVC_E_TOO_LARGE;
+  const int n_edges = n_agents - 1;
+  if (n_edges == 0) return KVC_OK;
+  UpdatePlan P[kMaxFitEdges];
+  size_t off[kMaxFitEdges + 1];
+  off[0] = 0;
+  int rc;
+  bool any_fit = false, uniform = true;
+  for (int e = 0; e < n_edges; ++e) {
+    const int32_t shift = prefix_len[e + 1] - prefix_len[e];
+    if ((rc = plan_update(&agents[e], &agents[e + 1], shift, rope, &states[e], mode, &P[e])) != KVC_OK) return rc;
+    off[e + 1] = off[e] + kvc_chain_update_edge_stride(&agents[e + 1], &states[e], mode);
+    any_fit |= P[e].fit && !P[e].empty;
+    uniform &= !P[e].empty && P[e].L == P[0].L && P[e].H == P[0].H && P[e].d == P[0].d && states[e].r == states[0].r &&
+               states[e].n_cov == states[0].n_cov && off[e + 1] - off[e] == off[1];
+  }
+  if (any_fit && (!workspace || workspace_bytes < off[n_edges] || (reinterpret_cast<uintptr_t>(workspace) & 255)))
+    return KVC_E_WORKSPACE;
+  uint32_t* status = status_ptr();
+  if (!status) return KVC_E_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (any_fit) {
+    FitLaunch F[kMaxFitEdges];
+    for (int e = 0; e < n_edges; ++e) {
+      if (P[e].empty) continue;
+      if ((rc = fit_gram(P[e], reinterpret_cast<char*>(workspace) + off[e], status, &F[e], s)) != KVC_OK) return rc;
+      uniform &= F[e].n_parts == F[0].n_parts;
+    }
+    const size_t solver_bytes = (size_t)P[0].L * P[0].H * 2 * sizeof(int32_t);
+    if (uniform) {
+      // one launch serves the matrices of every edge: a single edge fills the GPU's resident blocks
+      // unevenly, all edges together keep every SM busy until the end
+      FitLaunch& B = F[0];
+      B.n_edges = n_edges;
+      B.edge_stride = (int64_t)off[1];
+      for (int e = 0; e < n_edges; ++e) {
+        B.basis_k_e[e] = reinterpret_cast<float*>(states[e].basis_k);
+        B.basis_v_e[e] = reinterpret_cast<float*>(states[e].basis_v);
+      }
+      if ((rc = fit_eig(B, mode, P[0].d, r_eff_of(P[0]), fit_solver_offset(&agents[1]), solver_bytes, s)) != KVC_OK) return rc;
+    } else {
+      for (int e = 0; e < n_edges; ++e) {
+        if (P[e].empty) continue;
+        const size_t sb = (size_t)P[e].L * P[e].H * 2 * sizeof(int32_t);
+        if ((rc = fit_eig(F[e], mode, P[e].d, r_eff_of(P[e]), fit_solver_offset(&agents[e + 1]), sb, s)) != KVC_OK) return rc;
+      }
+    }
+  }
+  for (int e = 0; e < n_edges; ++e) {
+    if (P[e].empty) continue;
+    if ((rc = project_edge(P[e], status, s)) != KVC_OK) return rc;
+  }
   return KVC_OK;
 }
 

@@ -67,6 +67,8 @@ struct UpdateLaunch {
   alignas(16) float sn[kMaxHalfD];
 };
 
+constexpr int kMaxFitEdges = 15;   // edges whose eigensolves one launch may serve (a chain of 16 agents)
+
 struct FitLaunch {             // Gram + eigensolve
   DevCache src, tgt;
   float* gram;                 // [n_parts][L*H*2][d][d] partial sums in, [L*H*2][d][d] final out
@@ -74,7 +76,14 @@ struct FitLaunch {             // Gram + eigensolve
   float* basis_k;              // [L,H,r,d] float32 out
   float* basis_v;
   int32_t r, n_cov, pairing, shift, L, H;
-  int32_t n_parts, pad;
+  int32_t n_parts;
+  // The eigensolver kernels serve n_edges problems of the same geometry, r and n_cov in one launch
+  // (block b works on matrix b % (2 L H) of edge b / (2 L H)): edge e has its Gram matrices,
+  // eigenvalues and solver codes edge_stride BYTES behind edge e - 1 and its bases in basis_*_e[e].
+  int32_t n_edges;
+  int64_t edge_stride;
+  float* basis_k_e[kMaxFitEdges];
+  float* basis_v_e[kMaxFitEdges];
   uint32_t* status;
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];

@@ -31,6 +31,7 @@
 namespace kvc {
 #ifdef KVC_EIG_TIMING
 __device__ unsigned long long g_eig_t[16];
+__device__ unsigned long long g_eig_blk[4096 * 4];   // per block: cycles, smid, globaltimer begin, end
 #define TMARK(i) do { __syncthreads(); if (tid == 0 && blockIdx.x == 100) { long long now = clock64(); atomicAdd(&g_eig_t[i], (unsigned long long)(now - t_last)); t_last = now; } } while (0)
 #else
 #define TMARK(i)
@@ -93,7 +94,6 @@ struct Smem {
   } u;
   float th[kMaxM];                              // Ritz values, descending
   float rho2[kMaxM];
-  float cs[2 * 16];                             // (c, s) of the step's rotations
   float red[16];
   int perm[kMaxM];
   int flag;
@@ -351,44 +351,50 @@ __device__ __forceinline__ float chol_qr(float* Y, Smem<N>& sm, int m, int tid, 
 // Eigen-decomposition of the symmetric m x m matrix in sm.u.m.h (pitch kSP, zero beyond m) by cyclic
 // Jacobi: on return the diagonal of h holds the eigenvalues and the columns of sm.u.m.w the
 // eigenvectors, in the order the round-robin left them (the caller sorts).  Returns false if the sweep
-// limit was reached.  Thread layout: the first 16 threads are the diagonal of a 16 x 16 array (they
-// compute the rotations), thread (a, b) holds rows 2a, 2a+1 and columns 2b, 2b+1 of H and of W.
+// limit was reached.  Thread (a, b) of a 16 x 16 array holds rows 2a, 2a+1 and columns 2b, 2b+1 of H
+// and of W in registers.  A step costs one block barrier: every thread works out the rotation of its
+// own column pair b from the diagonal block (b, b) (so nobody waits for a few threads to publish them),
+// takes the rotation of its row pair a from the lane of its half-warp whose column pair is a, writes
+// its rotated block of H to where the round-robin sends it in the OTHER of two copies of H, and
+// passes its rotated columns of W along its half-warp by shuffles (the rows of W do not move).
 template <int N>
 __device__ __forceinline__ bool jacobi_eig(Smem<N>& sm, int m, int tid) {
-  float* H = sm.u.m.h;
+  float* Hb[2] = {sm.u.m.h, sm.u.m.s};           // two copies of H; s is free during the decomposition
   float* W = sm.u.m.w;
   const int np = (m + 1) >> 1;
-  for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
-    const int a = i >> 5, b = i & 31;
-    W[a * kSP + b] = (a == b) ? 1.f : 0.f;
-  }
-  int pa, pb;
-  if (tid < 16) {
-    pa = pb = tid;
-  } else {
-    const int q = tid - 16;
-    pa = q / 15;
-    const int bb = q - pa * 15;
-    pb = bb + (bb >= pa ? 1 : 0);
-  }
-  const bool act_h = pa < np && pb < np, act_w = pb < np;
-  // where this thread's entries go after a step (rows and columns of H move, only the columns of W)
+  const int lane = tid & 31;
+  const int pa = tid >> 4, pb = tid & 15;
+  const bool act_h = pa < np && pb < np;
+  const bool act_b = pb < np;
+  // where this thread's entries of H go after a step (rows and columns move)
   const int r0 = rr_next(2 * pa, np), r1 = rr_next(2 * pa + 1, np), c0 = rr_next(2 * pb, np), c1 = rr_next(2 * pb + 1, np);
   const int h00 = r0 * kSP + c0, h01 = r0 * kSP + c1, h10 = r1 * kSP + c0, h11 = r1 * kSP + c1;
-  const int w00 = (2 * pa) * kSP + c0, w01 = (2 * pa) * kSP + c1, w10 = (2 * pa + 1) * kSP + c0, w11 = (2 * pa + 1) * kSP + c1;
   const int ld0 = (2 * pa) * kSP + 2 * pb, ld1 = (2 * pa + 1) * kSP + 2 * pb;
-  __syncthreads();
-  float2 x0 = *reinterpret_cast<const float2*>(H + ld0), x1 = *reinterpret_cast<const float2*>(H + ld1);
-  float2 v0 = *reinterpret_cast<const float2*>(W + ld0), v1 = *reinterpret_cast<const float2*>(W + ld1);
-  float2* cs2 = reinterpret_cast<float2*>(sm.cs);
-  if (tid < 16) cs2[tid] = make_float2(1.f, 0.f);
+  const int dg0 = (2 * pb) * kSP + 2 * pb, dg1 = (2 * pb + 1) * kSP + 2 * pb + 1;
+  // where the new content of this thread's column slots of W comes from: slot s0 -> 2 pb, s1 -> 2 pb + 1
+  int s0 = 2 * pb, s1 = 2 * pb + 1;
+  for (int s = 0; s < 2 * np; ++s) {
+    const int d = rr_next(s, np);
+    if (d == 2 * pb) s0 = s;
+    if (d == 2 * pb + 1) s1 = s;
+  }
+  const int half = lane & 16;
+  const int src0 = half | (s0 >> 1), src1 = half | (s1 >> 1), src_a = half | pa;
+  const bool odd0 = s0 & 1, odd1 = s1 & 1;
+  float2 v0 = make_float2(2 * pa == 2 * pb ? 1.f : 0.f, 0.f);                      // W = I
+  float2 v1 = make_float2(0.f, 2 * pa + 1 == 2 * pb + 1 ? 1.f : 0.f);
+  int cur = 0;
+  float2 x0 = *reinterpret_cast<const float2*>(Hb[0] + ld0), x1 = *reinterpret_cast<const float2*>(Hb[0] + ld1);
+  float2 g0 = *reinterpret_cast<const float2*>(Hb[0] + dg0);
+  float g1 = Hb[0][dg1];
   bool done = false;
   for (int sweep = 0; sweep < kMaxSweeps && !done; ++sweep) {
     float tmax = 0.f, hmax = 0.f, dmax = 0.f;
     for (int s = 0; s < 2 * np - 1; ++s) {
-      if (tid < np) {                             // diagonal block: x0.x = h_pp, x0.y = h_pq, x1.y = h_qq
-        const float hpp = x0.x, hpq = x0.y, hqq = x1.y;
-        float c = 1.f, sn = 0.f;
+      // rotation of column pair pb: g0.x = h_pp, g0.y = h_pq, g1 = h_qq
+      float c = 1.f, sn = 0.f;
+      if (act_b) {
+        const float hpp = g0.x, hpq = g0.y, hqq = g1;
         dmax = fmaxf(dmax, fmaxf(fabsf(hpp), fabsf(hqq)));
         if (fabsf(hpq) > 6e-8f * (fabsf(hpp) + fabsf(hqq))) {
           // tan of the rotation angle, the smaller root of t^2 + 2 zeta t - 1 = 0 with zeta = (h_qq - h_pp) / (2 h_pq):
@@ -403,44 +409,47 @@ __device__ __forceinline__ bool jacobi_eig(Smem<N>& sm, int m, int tid) {
           tmax = fmaxf(tmax, fabsf(t));
           hmax = fmaxf(hmax, fabsf(hpq));
         }
-        cs2[tid] = make_float2(c, sn);
       }
-      __syncthreads();
-      const float2 ra = cs2[pa], rb = cs2[pb];
+      const float ca = __shfl_sync(0xffffffffu, c, src_a), sa = __shfl_sync(0xffffffffu, sn, src_a);
+      float* Hn = Hb[cur ^ 1];
       if (act_h) {
-        const float y00 = ra.x * x0.x - ra.y * x1.x, y01 = ra.x * x0.y - ra.y * x1.y;      // J^T from the left (rows)
-        const float y10 = ra.y * x0.x + ra.x * x1.x, y11 = ra.y * x0.y + ra.x * x1.y;
-        float z00 = rb.x * y00 - rb.y * y01, z01 = rb.y * y00 + rb.x * y01;                // J from the right (columns)
-        float z10 = rb.x * y10 - rb.y * y11, z11 = rb.y * y10 + rb.x * y11;
+        const float y00 = ca * x0.x - sa * x1.x, y01 = ca * x0.y - sa * x1.y;            // J^T from the left (rows)
+        const float y10 = sa * x0.x + ca * x1.x, y11 = sa * x0.y + ca * x1.y;
+        float z00 = c * y00 - sn * y01, z01 = sn * y00 + c * y01;                        // J from the right (columns)
+        float z10 = c * y10 - sn * y11, z11 = sn * y10 + c * y11;
         if (pa == pb) {                           // the rotated pair itself: its off-diagonal entry is now zero
           z01 = 0.f;
           z10 = 0.f;
         }
-        H[h00] = z00;
-        H[h01] = z01;
-        H[h10] = z10;
-        H[h11] = z11;
+        Hn[h00] = z00;
+        Hn[h01] = z01;
+        Hn[h10] = z10;
+        Hn[h11] = z11;
       }
-      if (act_w) {
-        W[w00] = rb.x * v0.x - rb.y * v0.y;
-        W[w01] = rb.y * v0.x + rb.x * v0.y;
-        W[w10] = rb.x * v1.x - rb.y * v1.y;
-        W[w11] = rb.y * v1.x + rb.x * v1.y;
+      {
+        const float n00 = c * v0.x - sn * v0.y, n01 = sn * v0.x + c * v0.y;
+        const float n10 = c * v1.x - sn * v1.y, n11 = sn * v1.x + c * v1.y;
+        const float a00 = __shfl_sync(0xffffffffu, n00, src0), a01 = __shfl_sync(0xffffffffu, n01, src0);
+        const float a10 = __shfl_sync(0xffffffffu, n10, src0), a11 = __shfl_sync(0xffffffffu, n11, src0);
+        const float b00 = __shfl_sync(0xffffffffu, n00, src1), b01 = __shfl_sync(0xffffffffu, n01, src1);
+        const float b10 = __shfl_sync(0xffffffffu, n10, src1), b11 = __shfl_sync(0xffffffffu, n11, src1);
+        v0 = make_float2(odd0 ? a01 : a00, odd1 ? b01 : b00);
+        v1 = make_float2(odd0 ? a11 : a10, odd1 ? b11 : b10);
       }
       __syncthreads();
-      x0 = *reinterpret_cast<const float2*>(H + ld0);
-      x1 = *reinterpret_cast<const float2*>(H + ld1);
-      v0 = *reinterpret_cast<const float2*>(W + ld0);
-      v1 = *reinterpret_cast<const float2*>(W + ld1);
+      cur ^= 1;
+      x0 = *reinterpret_cast<const float2*>(Hn + ld0);
+      x1 = *reinterpret_cast<const float2*>(Hn + ld1);
+      g0 = *reinterpret_cast<const float2*>(Hn + dg0);
+      g1 = Hn[dg1];
     }
     // Rotations converge quadratically: what a sweep leaves behind is of the order (largest angle) x
-    // (largest entry it met).  Below rounding level of the largest eigenvalue: done.
-    if (tid < 32) {
-      tmax = wmax(tmax);
-      hmax = wmax(hmax);
-      dmax = wmax(dmax);
-      if (tid == 0) sm.flag = (tmax * hmax <= 3e-7f * dmax) ? 1 : 0;
-    }
+    // (largest entry it met).  Below rounding level of the largest eigenvalue: done.  (Every half-warp
+    // has seen all pairs.)
+    tmax = wmax(tmax);
+    hmax = wmax(hmax);
+    dmax = wmax(dmax);
+    if (tid == 0) sm.flag = (tmax * hmax <= 3e-7f * dmax) ? 1 : 0;
     __syncthreads();
     done = sm.flag != 0;
     __syncthreads();
@@ -448,6 +457,14 @@ __device__ __forceinline__ bool jacobi_eig(Smem<N>& sm, int m, int tid) {
     if (tid == 0) atomicAdd(&g_eig_t[10], 1ull);
 #endif
   }
+  // leave the result where the caller expects it: H in sm.u.m.h, W in sm.u.m.w
+  if (act_h) {
+    *reinterpret_cast<float2*>(sm.u.m.h + ld0) = x0;
+    *reinterpret_cast<float2*>(sm.u.m.h + ld1) = x1;
+  }
+  *reinterpret_cast<float2*>(W + ld0) = v0;
+  *reinterpret_cast<float2*>(W + ld1) = v1;
+  __syncthreads();
   return done;
 }
 
@@ -456,9 +473,13 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem<N>& sm = *reinterpret_cast<Smem<N>*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sk = blockIdx.x;
+  const int mats = p.L * p.H * 2;
+  const int edge = blockIdx.x / mats;
+  const int sk = blockIdx.x - edge * mats;
   const int is_v = sk & 1, slab = sk >> 1;
-  float* G = p.gram + (int64_t)sk * N * N;
+  float* G = reinterpret_cast<float*>(reinterpret_cast<char*>(p.gram) + edge * p.edge_stride) + (int64_t)sk * N * N;
+  float* evals = reinterpret_cast<float*>(reinterpret_cast<char*>(p.evals) + edge * p.edge_stride);
+  solver = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(solver) + edge * p.edge_stride);
   const int64_t part_stride = (int64_t)p.L * p.H * 2 * N * N;
   const int m = min(min(p.r, N), p.n_cov);
   const int rg = tid >> 3, cg = tid & 7;          // 4 x 4 tiles of the N x 32 matrices
@@ -466,6 +487,11 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
 
   long long t_last = clock64();
   (void)t_last;
+#ifdef KVC_EIG_TIMING
+  const long long t_begin = t_last;
+  unsigned long long gt_begin;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_begin));
+#endif
   // ---- 0. sum of the partial Grams, symmetrised, written back; trace
   float tr = 0.f;
   {
@@ -653,48 +679,60 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
       mul_small(Y, Ws, m, rg, cg, 1.f, gz);       // G Z = (G Q) W: Y still holds the last product
     }
     // the Ritz values once more as Rayleigh quotients of the columns that will be written (this takes
-    // the rotations' accumulated rounding out of them)
-    float* num = sm.u.m.h;                        // [32] z . G z   (H and W are not needed any more)
-    float* den = sm.u.m.h + kMaxM;                // [32] z . z
+    // the rotations' accumulated rounding out of them).  Column sums go through per-row-group partial
+    // sums added in a fixed order: the same bits on every run.
+    float* pnum = sm.u.part;                      // [N/4][32] shares of z . G z   (H, W and Ws are not needed any more)
+    float* pden = sm.u.part + (N / 4) * kMaxM;    // [N/4][32] shares of z . z
     __syncthreads();                              // everybody has read Q, Y, Ws
-    if (tid < 2 * kMaxM) num[tid] = 0.f;
     if (rg < N / 4) {
 #pragma unroll
       for (int a = 0; a < 4; ++a)
         *reinterpret_cast<float4*>(Y + (4 * rg + a) * kQP + 4 * cg) = make_float4(z[a][0], z[a][1], z[a][2], z[a][3]);
-    }
-    __syncthreads();
-    if (tile_on) {
+      float pn[4], pd[4];
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
-        float pn = 0.f, pd = 0.f;
+        pn[b] = pd[b] = 0.f;
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
-          pn = fmaf(z[a][b], gz[a][b], pn);
-          pd = fmaf(z[a][b], z[a][b], pd);
+          pn[b] = fmaf(z[a][b], gz[a][b], pn[b]);
+          pd[b] = fmaf(z[a][b], z[a][b], pd[b]);
         }
-        atomicAdd(&num[4 * cg + b], pn);
-        atomicAdd(&den[4 * cg + b], pd);
       }
+      *reinterpret_cast<float4*>(pnum + rg * kMaxM + 4 * cg) = make_float4(pn[0], pn[1], pn[2], pn[3]);
+      *reinterpret_cast<float4*>(pden + rg * kMaxM + 4 * cg) = make_float4(pd[0], pd[1], pd[2], pd[3]);
     }
     __syncthreads();
-    if (tid < m) sm.th[tid] = num[tid] / fmaxf(den[tid], 1e-30f);
+    if (tid < kMaxM) {
+      float nsum = 0.f, dsum = 0.f;
+      for (int g = 0; g < N / 4; ++g) {
+        nsum += pnum[g * kMaxM + tid];
+        dsum += pden[g * kMaxM + tid];
+      }
+      sm.th[tid] = (tid < m) ? nsum / fmaxf(dsum, 1e-30f) : 0.f;
+    }
     __syncthreads();
 
     // ---- 3. a-posteriori residuals of the rows that would be written
-    if (tile_on) {
+    if (rg < N / 4) {
       const float4 t4 = *reinterpret_cast<const float4*>(sm.th + 4 * cg);
       const float tv[4] = {t4.x, t4.y, t4.z, t4.w};
+      float pr[4];
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
-        float part = 0.f;
+        pr[b] = 0.f;
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
           const float e = fmaf(-tv[b], z[a][b], gz[a][b]);
-          part = fmaf(e, e, part);
+          pr[b] = fmaf(e, e, pr[b]);
         }
-        atomicAdd(&sm.rho2[4 * cg + b], part);
       }
+      *reinterpret_cast<float4*>(pnum + rg * kMaxM + 4 * cg) = make_float4(pr[0], pr[1], pr[2], pr[3]);
+    }
+    __syncthreads();
+    if (tid < kMaxM) {
+      float rsum = 0.f;
+      for (int g = 0; g < N / 4; ++g) rsum += pnum[g * kMaxM + tid];
+      sm.rho2[tid] = (tid < m) ? rsum : 0.f;
     }
     __syncthreads();
     float sumth = 0.f, rhoF2 = 0.f, rhomax2 = 0.f;
@@ -714,7 +752,7 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
   TMARK(8);
   if (reason == 0) {
     // ---- output: sign convention (largest-magnitude entry positive, first such index), unit length
-    float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * N;
+    float* basis = (is_v ? p.basis_v_e[edge] : p.basis_k_e[edge]) + (int64_t)slab * p.r * N;
     const float* Z = Y;
     for (int j = warp; j < p.r; j += kThreads / 32) {
       if (j < m) {
@@ -745,16 +783,28 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
         for (int c = lane; c < N; c += 32) basis[j * N + c] = 0.f;
       }
     }
-    if (tid < N) p.evals[(int64_t)sk * N + tid] = (tid < m) ? sm.th[tid] : tau / (float)(N - m);
+    if (tid < N) evals[(int64_t)sk * N + tid] = (tid < m) ? sm.th[tid] : tau / (float)(N - m);
   }
   TMARK(9);
   if (tid == 0) solver[sk] = reason;
+#ifdef KVC_EIG_TIMING
+  if (tid == 0 && blockIdx.x < 4096) {
+    unsigned long long gt_end;
+    unsigned smid;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_end));
+    asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+    g_eig_blk[4 * blockIdx.x] = (unsigned long long)(clock64() - t_begin);
+    g_eig_blk[4 * blockIdx.x + 1] = smid;
+    g_eig_blk[4 * blockIdx.x + 2] = gt_begin;
+    g_eig_blk[4 * blockIdx.x + 3] = gt_end;
+  }
+#endif
 }
 
 }  // namespace
 
 cudaError_t launch_eig_subspace(const FitLaunch& F, int d, int32_t* solver, cudaStream_t s) {
-  const int blocks = F.L * F.H * 2;
+  const int blocks = F.L * F.H * 2 * F.n_edges;
   if (blocks <= 0) return cudaSuccess;
   if (d != 128 && d != 64) return cudaErrorInvalidValue;
   cudaError_t e;
@@ -775,6 +825,9 @@ cudaError_t launch_eig_subspace(const FitLaunch& F, int d, int32_t* solver, cuda
 #ifdef KVC_EIG_TIMING
 extern "C" int kvc_debug_eig_times(unsigned long long* out) {
   return cudaMemcpyFromSymbol(out, g_eig_t, sizeof(g_eig_t)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int kvc_debug_eig_blocks(unsigned long long* out, int n) {
+  return cudaMemcpyFromSymbol(out, g_eig_blk, sizeof(unsigned long long) * 4 * n) == cudaSuccess ? 0 : -1;
 }
 #endif
 }  // namespace kvc

@@ -389,8 +389,11 @@ __device__ __forceinline__ float warp_sum(float x) {
 template <int N>
 __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __grid_constant__ FitLaunch p, int zs,
                                                                       const int32_t* __restrict__ solver) {
+  const int mats = p.L * p.H * 2;
+  const int edge = blockIdx.x / mats;
+  if (solver != nullptr) solver = reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(solver) + edge * p.edge_stride);
   // solver != nullptr: the subspace solver went first; a matrix it served (solver[m] == 0) is done
-  if (solver != nullptr && solver[blockIdx.x] == 0) return;
+  if (solver != nullptr && solver[blockIdx.x - edge * mats] == 0) return;
   extern __shared__ __align__(16) float smem[];
   constexpr int n = N;
   constexpr int np = N + 4;           // row pitch of A = 4 (mod 32)
@@ -409,9 +412,10 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NW = kEigThreads / 32;
-  const int sk = blockIdx.x;
+  const int sk = blockIdx.x - edge * mats;
   const int is_v = sk & 1, slab = sk >> 1;
-  float* G = p.gram + (int64_t)sk * n * n;
+  float* G = reinterpret_cast<float*>(reinterpret_cast<char*>(p.gram) + edge * p.edge_stride) + (int64_t)sk * n * n;
+  float* evals = reinterpret_cast<float*>(reinterpret_cast<char*>(p.evals) + edge * p.edge_stride);
   const int64_t part_stride = (int64_t)p.L * p.H * 2 * n * n;
 
   // ---- 1. Householder tridiagonalisation with the matrix in REGISTERS.  TPR threads own one row,
@@ -694,7 +698,7 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
     if (ev < n && sub == 0) lam[ev] = (tnorm > 0.f) ? 0.5f * (lo + hi) * tscale : 0.f;
   }
   __syncthreads();
-  if (tid < n) p.evals[(int64_t)sk * n + tid] = lam[tid];
+  if (tid < n) evals[(int64_t)sk * n + tid] = lam[tid];
 
   // ---- 3. eigenvectors of T for the r_eff largest eigenvalues
   const int r_eff = min(min(min(p.r, n), p.n_cov), kEigMaxR);
@@ -767,7 +771,6 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
       const float s = have ? shf[j] : 0.f;
       float* st = vv;                             // [4][32] hand-over slots (vv and pp are free after step 2)
       float u = 0.f, v = 0.f, xp = 0.f;
-      if (warp == 0) st[96 + lane] = 0.f;         // sum of squares per vector
       for (int w = 0; w < NW; ++w) {
         if (warp == w && have) {
           if (w == 0) {
@@ -839,7 +842,12 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
         }
         __syncthreads();
       }
-      // scale against overflow, then normalise
+      // scale against overflow, then normalise.  The warps' shares of a vector's squared length are
+      // added as 64-bit fixed-point numbers (entries are at most 1 after scaling): integer addition
+      // does not depend on the order the warps arrive in, so the result is the same on every run.
+      unsigned long long* len2 = reinterpret_cast<unsigned long long*>(st);   // [32], over the hand-over slots 0..63 (free now)
+      if (warp == 0) len2[lane] = 0ull;
+      __syncthreads();
       const float sc = have ? 1.f / fmaxf(st[64 + j], 1e-30f) : 0.f;
       if (have) {
         float nn = 0.f;
@@ -848,11 +856,11 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
           yr[q] *= sc;
           nn = fmaf(yr[q], yr[q], nn);
         }
-        atomicAdd(&st[96 + j], nn);
+        atomicAdd(&len2[j], (unsigned long long)(nn * 1099511627776.f));     // 2^40
       }
       __syncthreads();
       if (have) {
-        const float inv = rsqrtf(fmaxf(st[96 + j], 1e-30f));
+        const float inv = rsqrtf(fmaxf((float)len2[j] * (1.f / 1099511627776.f), 1e-30f));
 #pragma unroll
         for (int q = 0; q < SPW; ++q) Zt[(SPW * warp + q) * zs + j] = yr[q] * inv;
       }
@@ -1107,7 +1115,7 @@ __global__ void __launch_bounds__(kEigThreads, 2) eig_tridiag_kernel(const __gri
   if (tid == 0 && (bad0 | bad1) != 0u) atomicOr(p.status, 4u);   // vectors still dependent after the last round: flagged
 
   // ---- 4. back-transformation z <- H_0 H_1 ... H_{n-3} z, then output
-  float* basis = (is_v ? p.basis_v : p.basis_k) + (int64_t)slab * p.r * n;
+  float* basis = (is_v ? p.basis_v_e[edge] : p.basis_k_e[edge]) + (int64_t)slab * p.r * n;
   // TPV neighbouring lanes carry one vector through all reflectors with its entries in registers
   // (thread `part` holds the four-row groups part, part + TPV, ...: neighbouring lanes read
   // neighbouring 16 bytes of a reflector, free of bank conflicts).  Per reflector: v . z over the TPV lanes
@@ -1255,7 +1263,7 @@ cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s) {
 }
 
 cudaError_t launch_eig(const FitLaunch& F, int d, const int32_t* solver, cudaStream_t s) {
-  const int blocks = F.L * F.H * 2;
+  const int blocks = F.L * F.H * 2 * F.n_edges;
   if (blocks <= 0) return cudaSuccess;
   int r_eff = F.r < d ? F.r : d;
   r_eff = r_eff < F.n_cov ? r_eff : F.n_cov;

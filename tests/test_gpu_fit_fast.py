@@ -170,3 +170,83 @@ def test_clustered_spectra_either_solver(d):
         res = float(np.sum((xn - c @ B) ** 2))
         assert res <= float(np.sum(w[k:])) + 8 * r * 1.2e-6 * w[0] + 1e-9 * float(np.sum(w)), (trial, r, sv)
     print("clustered spectra served by subspace / full solver:", served)
+
+
+def _chain_caches(cfg, n_agents):
+    """n_agents caches on the device: agent 0 drawn, agent a = bf16(Align(agent a-1) + A_a B_a + noise),
+    built by the oracle from generator draws (so every edge is a rank-r deviation over a noise floor)."""
+    cfg = cfg.scaled(n_agents=n_agents)
+    pl = wl.prefix_lengths(cfg)
+    f = hp.inv_freq(cfg)
+    cpu = hp.make_cache(cfg)
+    o = hp.oracle_cache(cpu)
+    caches = [hp.to_dev(cpu, DEV)]
+    as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    for a in range(1, n_agents):
+        nk = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2 * a).numpy()
+        nv = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2 * a + 1).numpy()
+        o = orc.make_target(o, hp.oracle_state(hp.make_state(cfg, a)), pl[a] - pl[a - 1], f, nk, nv, cfg.sigma)
+        caches.append(hp.to_dev(kvc.Cache(as_t(o.k), as_t(o.v)), DEV))
+    return caches, pl
+
+
+@pytest.mark.parametrize("mode", ["fit_fast", "fit", "project"])
+def test_chain_update_equals_edge_by_edge(mode):
+    """kvc_state_update_chain (all eigensolves of a workflow in one launch) against one kvc_state_update
+    per edge: the same kernels on the same data, so bases, coefficients, eigenvalues and solver codes
+    agree bit for bit.  The per-edge results are themselves oracle-checked by the tests above."""
+    kmode = {"fit_fast": kvc.KVC_FIT_FAST, "fit": kvc.KVC_FIT, "project": kvc.KVC_PROJECT}[mode]
+    cfg = CFG_8B_S.scaled(L=2, H=3, T=333, r=16)
+    n = 4
+    caches, pl = _chain_caches(cfg, n)
+    rope = kvc.Rope(cfg.theta)
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+
+    def fresh():
+        g = torch.Generator(device=DEV).manual_seed(5)
+        B = torch.linalg.qr(torch.randn(L, H, d, r, device=DEV, generator=g))[0].transpose(-1, -2).contiguous()
+        return kvc.State(torch.zeros(L, H, T, r, device=DEV), torch.zeros(L, H, T, r, device=DEV), B.clone(), B.clone())
+
+    one = [fresh() for _ in range(n - 1)]
+    ws1 = []
+    for e in range(n - 1):
+        ws = torch.zeros(max(kvc.kvc_workspace_bytes(caches[e + 1], one[e], kmode), 256), dtype=torch.uint8, device=DEV)
+        kvc.kvc_state_update(caches[e], caches[e + 1], pl[e + 1] - pl[e], rope, one[e], kmode, workspace=ws)
+        ws1.append(ws)
+    allst = [fresh() for _ in range(n - 1)]
+    total = kvc.kvc_chain_update_workspace_bytes(caches, allst, kmode)
+    stride = kvc.kvc_chain_update_edge_stride(caches[1], allst[0], kmode)
+    assert total == (n - 1) * stride and stride % 256 == 0
+    wsn = torch.zeros(max(total, 256), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update_chain(caches, pl, rope, allst, kmode, workspace=wsn)
+    torch.cuda.synchronize()
+    for e in range(n - 1):
+        for name in ("coeff_k", "coeff_v", "basis_k", "basis_v"):
+            assert torch.equal(getattr(one[e], name), getattr(allst[e], name)), (e, name)
+        if kmode != kvc.KVC_PROJECT:
+            sub = wsn[e * stride:(e + 1) * stride]
+            m = L * H * 2
+            lo, hi = 2 * m * d * d * 4, 2 * m * d * d * 4 + m * d * 4
+            assert torch.equal(sub[lo:hi], ws1[e][lo:hi])                       # eigenvalues
+            assert torch.equal(sub[:m * d * d * 4], ws1[e][:m * d * d * 4])     # final Gram matrices
+            if kmode == kvc.KVC_FIT_FAST:
+                assert torch.equal(kvc.kvc_fit_solver(caches[e + 1], sub), kvc.kvc_fit_solver(caches[e + 1], ws1[e]))
+                assert int((kvc.kvc_fit_solver(caches[e + 1], sub) == 0).sum()) == m
+    # edges of different rank: served one by one inside the call, same results
+    if kmode == kvc.KVC_FIT_FAST:
+        def fresh_r(rr):
+            return kvc.State(torch.zeros(L, H, T, rr, device=DEV), torch.zeros(L, H, T, rr, device=DEV),
+                             torch.zeros(L, H, rr, d, device=DEV), torch.zeros(L, H, rr, d, device=DEV))
+        ranks = (8, 16, 40)
+        mixed = [fresh_r(rr) for rr in ranks]
+        ws = torch.zeros(kvc.kvc_chain_update_workspace_bytes(caches, mixed, kmode), dtype=torch.uint8, device=DEV)
+        kvc.kvc_state_update_chain(caches, pl, rope, mixed, kmode, workspace=ws)
+        for e, rr in enumerate(ranks):
+            ref = fresh_r(rr)
+            w1 = torch.zeros(kvc.kvc_workspace_bytes(caches[e + 1], ref, kmode), dtype=torch.uint8, device=DEV)
+            kvc.kvc_state_update(caches[e], caches[e + 1], pl[e + 1] - pl[e], rope, ref, kmode, workspace=w1)
+            assert torch.equal(ref.basis_k, mixed[e].basis_k) and torch.equal(ref.coeff_v, mixed[e].coeff_v), rr
+    # too small a workspace, too many agents: refused before anything runs
+    if kmode != kvc.KVC_PROJECT:
+        with pytest.raises(kvc.KvcError):
+            kvc.kvc_state_update_chain(caches, pl, rope, allst, kmode, workspace=wsn[:total - 256])

@@ -97,7 +97,31 @@ def test_noalloc_rejects_problems_beyond_its_capacity():
     cfg = cfg.scaled(L=16, H=4)
     src, tgt = _edge(cfg, 6)
     st = _fresh_state(cfg)
-    assert kvc.kvc_workspace_bytes(tgt, st, kvc.KVC_FIT) == kvc.KVC_STATIC_SCRATCH_BYTES
-    kvc.kvc_state_update_noalloc(src, tgt, 0, kvc.Rope(cfg.theta), st, kvc.KVC_FIT)
+    for mode in (kvc.KVC_FIT, kvc.KVC_FIT_FAST):
+        st = _fresh_state(cfg)
+        assert kvc.KVC_STATIC_SCRATCH_BYTES - 1024 <= kvc.kvc_workspace_bytes(tgt, st, mode) <= kvc.KVC_STATIC_SCRATCH_BYTES
+        kvc.kvc_state_update_noalloc(src, tgt, 0, kvc.Rope(cfg.theta), st, mode)
+        torch.cuda.synchronize()
+        assert float(st.basis_k.abs().max()) > 0.05
+
+
+def test_noalloc_takes_no_device_memory_after_its_first_call_and_checks_arguments_first():
+    cfg = wl.CONFIGS["tiny"]
+    src, tgt = _edge(cfg, 31)
+    rope = kvc.Rope(cfg.theta)
+    st = _fresh_state(cfg)
+    kvc.kvc_state_update_noalloc(src, tgt, 0, rope, st, kvc.KVC_FIT)        # first call: the array is resolved
     torch.cuda.synchronize()
-    assert float(st.basis_k.abs().max()) > 0.05
+    free0 = torch.cuda.mem_get_info()[0]
+    for mode in (kvc.KVC_FIT, kvc.KVC_FIT_FAST, kvc.KVC_PROJECT):
+        kvc.kvc_state_update_noalloc(src, tgt, 3, rope, st, mode)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    # an invalid call gets its own error even when it is also too large, and writes nothing
+    big = wl.CONFIGS["llama8b_8k"].scaled(name="too_big", L=13, H=5, T=16)
+    bsrc, btgt = _edge(big, 5)
+    bst = _fresh_state(big)
+    bst.n_cov = big.T + 1
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_state_update_noalloc(bsrc, btgt, 0, kvc.Rope(big.theta), bst, kvc.KVC_FIT)
+    assert e.value.code != -8
