@@ -455,6 +455,18 @@ int kvc_gate_weights(const double *dist_sq, int32_t n_anchors, double temperatur
 int kvc_status_poll(uint32_t *flags);
 int kvc_status_reset(void);
 
+/*
+ * kvc_selftest_wait_expiry -- run the give-up branch of the library's bounded waits once, safely.
+ * One CTA waits, through the same bounded wait the streaming kernels use but with a limit of
+ * limit_ms milliseconds (0 < limit_ms <= 100), on an mbarrier that nothing arrives on.  Every thread's
+ * wait must return "gave up", the CTA's abort flag must be raised and KVC_FLAG_WAIT_EXPIRED must
+ * appear in the status word; the context stays usable (nothing traps, faults or loops without bound).
+ *   result  HOST int32 [3]: threads whose wait claimed success (expected 0), the abort flag
+ *           (expected 1), SM cycles thread 0 spent waiting.
+ * Synchronises `stream`.  The caller clears the flag afterwards with kvc_status_reset.
+ */
+int kvc_selftest_wait_expiry(double limit_ms, int32_t *result, void *stream);
+
 /* Force a kernel family (testing / benchmarking); KVC_PATH_TC returns
  * KVC_E_UNSUPPORTED from later calls whose arguments it cannot serve. */
 int kvc_set_path(int32_t path);

@@ -35,7 +35,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_state_update_check", "kvc_state_update_chain",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_selftest_wait_expiry", "kvc_state_update_check", "kvc_state_update_chain",
     "kvc_chain_update_workspace_bytes", "kvc_chain_update_edge_stride", "kvc_chain_fused", "kvc_chain_workspace_bytes",
 )
 
@@ -88,6 +88,7 @@ def load(path: Optional[str] = None):
     lib.kvc_chain_workspace_bytes.restype = sz
     lib.kvc_state_update.argtypes = [PC, PC, i32, PR, PS, i32, vp, sz, vp]
     lib.kvc_state_update_noalloc.argtypes = [PC, PC, i32, PR, PS, i32, vp]
+    lib.kvc_selftest_wait_expiry.argtypes = [C.c_double, C.POINTER(i32), vp]
     lib.kvc_state_update_check.argtypes = [PC, PC, i32, PR, PS, i32]
     lib.kvc_state_update_chain.argtypes = [PC, i32, C.POINTER(i32), PR, PS, i32, vp, sz, vp]
     lib.kvc_chain_update_workspace_bytes.argtypes = [PC, i32, PS, i32]
@@ -289,6 +290,13 @@ def kvc_chain_fused(agent0: Cache, prefix_len: Sequence[int], states: Sequence[S
     os_ = (kvc_cache * max(n - 1, 1))(*[o.struct() for o in outs])
     _check(load().kvc_chain_fused(C.byref(a0), n, pl, sts, C.byref(r), os_, workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_chain_fused")
+
+
+def kvc_selftest_wait_expiry(limit_ms: float = 1.0, stream=None):
+    """(threads whose wait claimed success, abort flag, cycles waited) of a bounded wait made to run out."""
+    res = (C.c_int32 * 3)()
+    _check(load().kvc_selftest_wait_expiry(float(limit_ms), res, _stream(stream)), "kvc_selftest_wait_expiry")
+    return int(res[0]), int(res[1]), int(res[2])
 
 
 def kvc_chain_update_workspace_bytes(agents: Sequence[Cache], states: Sequence[State], mode: int) -> int:

@@ -17,11 +17,13 @@ __device__ uint32_t g_status_word;
 static thread_local int tl_path_force = KVC_PATH_AUTO;
 static thread_local int tl_last_path = KVC_PATH_AUTO;
 
-static uint32_t* status_ptr() {
+uint32_t* status_word_ptr() {
   uint32_t* p = nullptr;
   if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
   return p;
 }
+
+static uint32_t* status_ptr() { return status_word_ptr(); }
 
 static int ilog2_exact(int x) {
   if (x <= 0 || (x & (x - 1))) return -1;

@@ -1237,11 +1237,12 @@ int generic_apply_tile(int d) { return d == 128 ? 128 : 256; }
 template <int D>
 static cudaError_t launch_project_generic_t(const UpdateLaunch& U, int64_t tiles, cudaStream_t s) {
   const size_t smem = (64 * D + 32 * (D + 1)) * sizeof(float);
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     cudaError_t e = cudaFuncSetAttribute(project_generic_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    set = true;
+    once.mark(once_dev);
   }
   if (tiles <= 0) return cudaSuccess;
   project_generic_kernel<D><<<(unsigned)tiles, 256, smem, s>>>(U);

@@ -3,9 +3,50 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "kvc_dev.cuh"
 
 namespace kvc {
+
+// A kernel's attributes (the opt-in to more than 48 KB of dynamic shared memory) belong to the device
+// they were set on, and the device current at a call is the one that call uses: each launch site
+// keeps one of these and sets the attribute once per device, not once per process.
+class DeviceOnce {
+ public:
+  // true until mark() has been called for the current device; *dev is that device (-1 if unknown)
+  bool pending(int* dev) {
+    int d = -1;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= 64) {
+      *dev = -1;
+      return true;
+    }
+    *dev = d;
+    return !((mask_.load(std::memory_order_acquire) >> d) & 1ull);
+  }
+  void mark(int dev) {
+    if (dev >= 0) mask_.fetch_or(1ull << dev, std::memory_order_release);
+  }
+
+ private:
+  std::atomic<uint64_t> mask_{0};
+};
+
+// SM count of the current device (cached per device).
+inline int device_sm_count() {
+  static std::atomic<int> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  const bool cacheable = dev >= 0 && dev < 64;
+  int n = cacheable ? cache[dev].load(std::memory_order_relaxed) : 0;
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (cacheable) cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
+// device address of the current device's status word (kvc_api.cu); nullptr on failure
+uint32_t* status_word_ptr();
 
 // CUDA-core family (kvc_generic.cu)
 cudaError_t launch_apply_generic(const ApplyLaunch& L, int d, cudaStream_t s);

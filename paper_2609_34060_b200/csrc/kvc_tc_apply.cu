@@ -880,11 +880,12 @@ static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
                           sizeof(Ctrl<NSTAGE, NSC>);
   static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    set = true;
+    once.mark(once_dev);
   }
   apply_tc_kernel<RB, NSTAGE, NSC><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError();
@@ -908,11 +909,12 @@ template <int RB, int NSTAGE, int NSC, int MODE>
 static cudaError_t launch_reduce_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
                           sizeof(Ctrl<NSTAGE, NSC>);
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    set = true;
+    once.mark(once_dev);
   }
   apply_tc_kernel<RB, NSTAGE, NSC, MODE><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError();

@@ -24,19 +24,14 @@
 #include "kvc_tc.h"
 #include "kvc_tc_ptx.cuh"
 #include "kvc_tc_maps.h"
+#include "kvc_tc_stream.cuh"
 
 namespace kvc {
 namespace tcc {
 
 using namespace tc;
+using namespace tcs;    // tile geometry, Walker, operand layout
 
-constexpr int kTileTok = 128;
-constexpr int kThreads = 640;
-constexpr int kTeamThreads = 512;
-constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a cache tile (bf16)
-constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
-constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
-constexpr int kOperandBytes = 128 * 128;          // 128 channels x (32 hi + 32 lo) bf16
 constexpr int NB = 2;                             // input tiles of agent 0 in flight
 constexpr int NOUT = 2;                           // output slots (a hop's result: stored, and read by the next hop)
 constexpr int NC = 3;                             // coefficient blocks in flight
@@ -70,42 +65,6 @@ struct Ctrl {
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
-};
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-               : "memory");
-}
-
-// A contiguous range of tiles; tile = (slab2 = 2 (l H + h) + is_v, tt).  Stepping is incremental.
-struct Walker {
-  int64_t remaining;
-  int slab2, tt, tps, H, l, h;
-  __device__ void init(const ChainLaunch& p, int64_t begin, int64_t end_) {
-    remaining = end_ - begin;
-    tps = p.tps;
-    H = p.H;
-    tt = (int)(begin % tps);
-    slab2 = (int)(begin / tps);
-    const int slab = slab2 >> 1;
-    l = slab / H;
-    h = slab - l * H;
-  }
-  __device__ bool done() const { return remaining <= 0; }
-  __device__ void next() {
-    --remaining;
-    if (++tt < tps) return;
-    tt = 0;
-    ++slab2;
-    if ((slab2 & 1) == 0 && ++h == H) {
-      h = 0;
-      ++l;
-    }
-  }
-  __device__ int t0() const { return tt * kTileTok; }
-  __device__ int is_v() const { return slab2 & 1; }
-  __device__ int slab() const { return slab2 >> 1; }
 };
 
 __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
@@ -172,7 +131,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
   if (warp == 0) {
     // =============================================================== TMA producer (whole warp): agent 0's tiles, coefficient blocks
     Walker w;
-    w.init(p, tile_begin, tile_end);
+    w.init(p.tps, p.H, tile_begin, tile_end);
     uint32_t i = 0, epos = 0;
     bool alive = true;
     for (; alive && !w.done(); w.next(), ++i) {
@@ -242,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     // =============================================================== MMA issuer: one accumulator per (tile, hop)
     if (lane == 0) {
       Walker w;
-      w.init(p, tile_begin, tile_end);
+      w.init(p.tps, p.H, tile_begin, tile_end);
       uint32_t step = 0, epos = 0;
       bool alive = true;
       for (; alive && !w.done(); w.next()) {
@@ -289,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     // =============================================================== operand producer (one lane)
     if (lane == 0) {
       Walker w;
-      w.init(p, tile_begin, tile_end);
+      w.init(p.tps, p.H, tile_begin, tile_end);
       uint32_t epos = 0;
       bool alive = true;
       for (; alive && !w.done(); w.next()) {
@@ -317,7 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
   } else if (warp == 3) {
     // =============================================================== store warp: every hop's result to that hop's cache
     Walker w;
-    w.init(p, tile_begin, tile_end);
+    w.init(p.tps, p.H, tile_begin, tile_end);
     uint32_t step = 0;
     bool alive = true;
     for (; alive && !w.done(); w.next()) {
@@ -426,7 +385,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     };
 
     Walker w, wn;
-    w.init(p, tile_begin, tile_end);
+    w.init(p.tps, p.H, tile_begin, tile_end);
     wn = w;                                        // (tile, hop) one step ahead: its coefficients are converted first
     int an = 0;
     uint32_t i = 0, step = 0;
@@ -604,30 +563,7 @@ __global__ void __launch_bounds__(256) chain_prep_kernel(const PrepLaunch p) {
   if (col0 >= r) return;                          // the hop has no such block
   const void* basis = kv ? p.basis_v[a] : p.basis_k[a];
   __nv_bfloat16* out = p.out + ((((int64_t)a * 2 + b) * 2 + kv) * p.slabs + slab) * (128 * 64);
-  for (int i = threadIdx.x; i < 32 * 128; i += 256) {
-    const int q = i >> 7, ch = i & 127;
-    float x = 0.f;
-    if (col0 + q < r) {
-      const int64_t off = ((int64_t)slab * r + col0 + q) * 128 + ch;
-      x = p.bf16[a] ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
-                    : reinterpret_cast<const float*>(basis)[off];
-    }
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    out[ch * 64 + q] = hi;
-    out[ch * 64 + 32 + q] = __float2bfloat16_rn(x - __bfloat162float(hi));
-  }
-}
-
-static bool encode_operand(CUtensorMap* m, const __nv_bfloat16* ws, int64_t rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {64, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {128};
-  const cuuint32_t box[2] = {64, 128};
-  const cuuint32_t es[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(ws), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  write_operand_block(out, basis, p.bf16[a] != 0, slab, r, col0);
 }
 
 }  // namespace tcc
@@ -706,10 +642,11 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
   const int grid = (int)(C.total_tiles < sms ? C.total_tiles : sms);
   constexpr size_t smem = 1024 + (size_t)(NB + NOUT) * kBaseBytes + (size_t)NC * kCoeffBytes + (size_t)NO * kOperandBytes + sizeof(Ctrl);
   static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
-    set = true;
+    once.mark(once_dev);
   }
   chain_tc_kernel<<<grid, kThreads, smem, s>>>(C);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;

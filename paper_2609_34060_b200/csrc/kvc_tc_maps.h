@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include "kvc_dev.cuh"
+#include "kvc_launch.h"
 
 namespace kvc {
 namespace tc {
@@ -55,15 +56,7 @@ inline bool encode_coeff(CUtensorMap* m, const float* coeff, int r, int n_cov, i
 }
 
 
-inline int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-  }
-  return n;
-}
+inline int sm_count() { return device_sm_count(); }
 
 }  // namespace tc
 }  // namespace kvc

@@ -26,19 +26,14 @@
 #include "kvc_tc.h"
 #include "kvc_tc_ptx.cuh"
 #include "kvc_tc_maps.h"
+#include "kvc_tc_stream.cuh"
 
 namespace kvc {
 namespace tcm {
 
 using namespace tc;
+using namespace tcs;    // tile geometry, Walker, operand layout
 
-constexpr int kTileTok = 128;
-constexpr int kThreads = 640;
-constexpr int kTeamThreads = 512;
-constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a base tile (bf16)
-constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
-constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
-constexpr int kOperandBytes = 128 * 128;          // 128 channels x (32 hi + 32 lo) bf16
 constexpr int kWeightBytes = kTileTok * 4;
 // Ring depths are template parameters of the kernel: NSTAGE base-tile slots, NC coefficient blocks in
 // flight (HBM latency), NO operand blocks in flight (served by L2).  Up to three rank blocks per tile
@@ -77,42 +72,6 @@ struct Ctrl {
   int abort_flag;
 };
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-               : "memory");
-}
-
-// A contiguous range of tiles; tile = (slab2 = 2 (l H + h) + is_v, tt).  Stepping is incremental.
-struct Walker {
-  int64_t remaining;
-  int slab2, tt, tps, H, l, h;
-  __device__ void init(const MultiLaunch& p, int64_t begin, int64_t end_) {
-    remaining = end_ - begin;
-    tps = p.tps;
-    H = p.H;
-    tt = (int)(begin % tps);
-    slab2 = (int)(begin / tps);
-    const int slab = slab2 >> 1;
-    l = slab / H;
-    h = slab - l * H;
-  }
-  __device__ bool done() const { return remaining <= 0; }
-  __device__ void next() {
-    --remaining;
-    if (++tt < tps) return;
-    tt = 0;
-    ++slab2;
-    if ((slab2 & 1) == 0 && ++h == H) {
-      h = 0;
-      ++l;
-    }
-  }
-  __device__ int t0() const { return tt * kTileTok; }
-  __device__ int is_v() const { return slab2 & 1; }
-  __device__ int slab() const { return slab2 >> 1; }
-};
-
 // Writes the basis operands: for block e, K|V, slab: 128 rows (channel) of [32 hi | 32 lo] bf16,
 // ranks col0 .. col0+31 of the anchor's basis (zero beyond its rank).
 struct PrepLaunch {
@@ -128,18 +87,7 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   const void* basis = kv ? p.basis_v[e] : p.basis_k[e];
   const int r = p.r[e], col0 = p.col0[e];
   __nv_bfloat16* out = p.out + (((int64_t)e * 2 + kv) * p.slabs + slab) * (128 * 64);
-  for (int i = threadIdx.x; i < 32 * 128; i += 256) {
-    const int q = i >> 7, ch = i & 127;           // coalesced reads along the channel
-    float x = 0.f;
-    if (col0 + q < r) {
-      const int64_t off = ((int64_t)slab * r + col0 + q) * 128 + ch;
-      x = p.bf16[e] ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off])
-                    : reinterpret_cast<const float*>(basis)[off];
-    }
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    out[ch * 64 + q] = hi;
-    out[ch * 64 + 32 + q] = __float2bfloat16_rn(x - __bfloat162float(hi));
-  }
+  write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0);
 }
 
 template <int NSTAGE, int NC, int NO>
@@ -203,7 +151,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
   if (warp == 0) {
     // =============================================================== TMA producer (whole warp)
     Walker w;
-    w.init(p, tile_begin, tile_end);
+    w.init(p.tps, p.H, tile_begin, tile_end);
     uint32_t i = 0, epos = 0;
     bool alive = true;
     for (; alive && !w.done(); w.next(), ++i) {
@@ -278,7 +226,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
     // =============================================================== MMA issuer
     if (lane == 0) {
       Walker w;
-      w.init(p, tile_begin, tile_end);
+      w.init(p.tps, p.H, tile_begin, tile_end);
       uint32_t i = 0, epos = 0;
       bool alive = true;
       for (; alive && !w.done(); w.next(), ++i) {
@@ -323,7 +271,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
     // operand slot never holds back the coefficient loads
     if (lane == 0) {
       Walker w;
-      w.init(p, tile_begin, tile_end);
+      w.init(p.tps, p.H, tile_begin, tile_end);
       uint32_t epos = 0;
       bool alive = true;
       for (; alive && !w.done(); w.next()) {
@@ -347,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
   } else if (warp == 3) {
     // =============================================================== store warp
     Walker w;
-    w.init(p, tile_begin, tile_end);
+    w.init(p.tps, p.H, tile_begin, tile_end);
     uint32_t i = 0;
     for (; !w.done(); w.next(), ++i) {
       const int s = i % NSTAGE;
@@ -425,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
     const uint32_t csw = (uint32_t)(crow & 7);
 
     Walker w, wn;
-    w.init(p, tile_begin, tile_end);
+    w.init(p.tps, p.H, tile_begin, tile_end);
     wn = w;
     uint32_t i = 0, epos = 0;
     bool alive = true;
@@ -589,28 +537,17 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
   }
 }
 
-static bool encode_operand(CUtensorMap* m, const __nv_bfloat16* ws, int64_t rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {64, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {128};
-  const cuuint32_t box[2] = {64, 128};
-  const cuuint32_t es[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(ws), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int NSTAGE, int NC, int NO>
 static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
                           (size_t)NO * kOperandBytes + sizeof(Ctrl<NSTAGE, NC, NO>);
   static_assert(smem <= 232448, "exceeds the shared memory of one CTA");
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    set = true;
+    once.mark(once_dev);
   }
   apply_multi_tc_kernel<NSTAGE, NC, NO><<<grid, kThreads, smem, s>>>(M);
   return cudaGetLastError();

@@ -1,0 +1,85 @@
+// What the streaming kernels built on the apply skeleton (fused chain, multi-anchor apply) share:
+// tile geometry, the incremental walk over (layer, head, K|V, token tile), the split-bf16 basis
+// operand layout that the tensor-core contraction reads, and its tensor map.  One home for each.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvc_tc_maps.h"
+#include "kvc_tc_ptx.cuh"
+
+namespace kvc {
+namespace tcs {
+
+constexpr int kTileTok = 128;
+constexpr int kThreads = 640;                     // producer, MMA, two store warps ... and a team of 16 warps
+constexpr int kTeamThreads = 512;
+constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a cache tile (bf16)
+constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
+constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
+constexpr int kOperandBytes = 128 * 128;          // 128 channels x (32 hi + 32 lo) bf16
+
+// A contiguous range of tiles; tile = (slab2 = 2 (l H + h) + is_v, tt).  Stepping is incremental.
+struct Walker {
+  int64_t remaining;
+  int slab2, tt, tps, H, l, h;
+  __device__ void init(int tiles_per_slab, int heads, int64_t begin, int64_t end_) {
+    remaining = end_ - begin;
+    tps = tiles_per_slab;
+    H = heads;
+    tt = (int)(begin % tps);
+    slab2 = (int)(begin / tps);
+    const int slab = slab2 >> 1;
+    l = slab / H;
+    h = slab - l * H;
+  }
+  __device__ bool done() const { return remaining <= 0; }
+  __device__ void next() {
+    --remaining;
+    if (++tt < tps) return;
+    tt = 0;
+    ++slab2;
+    if ((slab2 & 1) == 0 && ++h == H) {
+      h = 0;
+      ++l;
+    }
+  }
+  __device__ int t0() const { return tt * kTileTok; }
+  __device__ int is_v() const { return slab2 & 1; }
+  __device__ int slab() const { return slab2 >> 1; }
+};
+
+// One basis operand block: 128 rows (channel) of [32 hi | 32 lo] bf16 for ranks col0 .. col0 + 31 of
+// the basis [slabs][r][128] (float32 or bf16; zero beyond rank r).  Called by a block of 256 threads.
+__device__ __forceinline__ void write_operand_block(__nv_bfloat16* out, const void* basis, bool basis_bf16, int slab, int r,
+                                                    int col0) {
+  for (int i = threadIdx.x; i < 32 * 128; i += 256) {
+    const int q = i >> 7, ch = i & 127;           // coalesced reads along the channel
+    float x = 0.f;
+    if (col0 + q < r) {
+      const int64_t off = ((int64_t)slab * r + col0 + q) * 128 + ch;
+      x = basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off]) : reinterpret_cast<const float*>(basis)[off];
+    }
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    out[ch * 64 + q] = hi;
+    out[ch * 64 + 32 + q] = __float2bfloat16_rn(x - __bfloat162float(hi));
+  }
+}
+
+// Tensor map over the operand blocks: rows of 64 bf16 (128 bytes, swizzled), boxes of 128 rows.
+inline bool encode_operand(CUtensorMap* m, const __nv_bfloat16* ws, int64_t rows) {
+  tc::EncodeTiledFn fn = tc::encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {64, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t es[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(ws), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace tcs
+}  // namespace kvc

@@ -418,11 +418,12 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
 template <int RB, int NS>
 static cudaError_t launch_project_t(const ProjectTcLaunch& L, int grid, cudaStream_t s) {
   const size_t smem = 1024 + (size_t)NS * kStageBytes + (size_t)8 * (32 * RB) * 128 + sizeof(Ctrl<NS>);
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     cudaError_t e = cudaFuncSetAttribute(project_tc_kernel<RB, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    set = true;
+    once.mark(once_dev);
   }
   project_tc_kernel<RB, NS><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError();
@@ -828,10 +829,11 @@ int tc_gram(const FitLaunch& F, int d, cudaStream_t s) {
   const int grid = (int)(L.total_units < sms ? L.total_units : sms);
   constexpr int NS = 3;
   const size_t smem = 1024 + (size_t)NS * kStageBytes + sizeof(GCtrl<NS>);
-  static bool set = false;
-  if (!set) {
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
     if (cudaFuncSetAttribute(gram_tc_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
-    set = true;
+    once.mark(once_dev);
   }
   gram_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;

@@ -53,3 +53,21 @@ def test_single_process_is_identity():
     assert dist_util.max_over_ranks(3.5) == 3.5
     assert dist_util.job_throughput(100.0, 50.0) == 2000.0
     assert dist_util.shard(list(range(10)), 1, 3) == [3, 4, 5]
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` outside a launcher starts two ranks itself; they rendezvous (gloo here),
+    combine their times by MAX and their units by SUM, and exactly one JSON line comes out."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--selftest-dist"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = lines[0]
+    assert rec["n_gpus"] == 2 and rec["asked_gpus"] == 2
+    assert rec["ms"] == 20.0 and abs(rec["value"] - 2000.0 / 20e-3) < 1e-6 * rec["value"]
