@@ -114,9 +114,11 @@ typedef struct kvc_state {
  *                    shared by the heads of a layer,
  *                    coeff [L, n_cov, r], basis [L, r, H d]  (head h uses columns h d .. (h+1) d - 1)
  *                    K_dst[l,h,t,:] = bf16( Rot(K_src[l,h,t,:]) + coeff_k[l,t,:] . basis_k[l][:, h d : (h+1) d] )
- * Grouping by layer is served by kvc_apply, kvc_chain, kvc_apply_batch and by kvc_state_update in
- * KVC_PROJECT mode (the projection sums over the heads: coeff[l,t,:] = sum_h Delta[l,h,t,:] . basis[l][:, h]^T);
- * KVC_FIT, the gate, token weights and kvc_apply_multi return KVC_E_UNSUPPORTED for it.
+ * Grouping by layer is served by kvc_apply, kvc_chain, kvc_apply_batch and by kvc_state_update: in
+ * KVC_PROJECT mode the projection sums over the heads (coeff[l,t,:] = sum_h Delta[l,h,t,:] . basis[l][:, h]^T);
+ * in the FIT modes (r <= 32) the basis rows are the r leading right singular vectors of the layer's
+ * concatenated deviation [n_cov, H d], see kvc_state_update.  The gate, token weights and
+ * kvc_apply_multi return KVC_E_UNSUPPORTED for it.
  */
 #define KVC_GROUP_HEAD  0
 #define KVC_GROUP_LAYER 1
@@ -199,6 +201,19 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                the workspace all hold their MEAN (their exact sum divided by d - r), so the trace is
  *                exact and kvc_effective_rank is exact whenever it does not exceed r.  Which solver
  *                served which matrix is left in the workspace, see kvc_fit_solver.
+ *   Layer-grouped states (KVC_GROUP_LAYER, D = H d), both FIT modes, r <= 32: the D x D Gram matrix is
+ *                never formed.  The r trial vectors live in the state's bases and are driven to the leading
+ *                eigenvectors of G = Delta^T Delta by three applications of G, each one the grouped
+ *                projection pass Z = Delta Q^T followed by a back-projection pass Y = Z^T Delta, with an
+ *                orthonormalisation of the r rows in between and a Rayleigh-Ritz step at the end
+ *                (a fixed schedule: 7 streaming passes over the two caches with the final projection).
+ *                Rows, coefficients and the r leading eigenvalues are as in KVC_FIT_FAST, the acceptance
+ *                test likewise with the rows' residual limit at 2e-4 lambda_1 (the passes contract in split
+ *                bf16 precision).  There is no second solver behind it: a matrix that fails the test (no
+ *                gap behind the r-th eigenvalue) still gets its Ritz rows, its code in kvc_group_fit_solver
+ *                says why, and KVC_FLAG_NOT_CONVERGED is raised.  Workspace layout: the eigenvalues
+ *                [L, 2, H d] first (kvc_group_fit_eigenvalues; the r leading ones, then the mean of the
+ *                rest), the codes [L, 2] (kvc_group_fit_solver), then scratch.
  *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
  *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte
  *              aligned.  May be NULL when 0 is needed.  After a KVC_FIT / KVC_FIT_FAST call it
@@ -224,6 +239,9 @@ size_t kvc_workspace_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mo
 #define KVC_SOLVER_FULL_NO_GAP     4   /* a-posteriori test failed: no gap behind the r-th eigenvalue */
 #define KVC_SOLVER_FULL_SWEEPS     5   /* Jacobi sweep limit                                         */
 const int32_t *kvc_fit_solver(const kvc_cache *tgt, const void *workspace);
+/* The same two accessors for the workspace of a layer-grouped FIT: float32 [L, 2, H d] and int32 [L, 2]. */
+const float *kvc_group_fit_eigenvalues(const kvc_cache *tgt, const void *workspace);
+const int32_t *kvc_group_fit_solver(const kvc_cache *tgt, const void *workspace);
 
 /* The argument checks of kvc_state_update (everything but the workspace), launching nothing. */
 int kvc_state_update_check(const kvc_cache *src, const kvc_cache *tgt, int32_t shift, const kvc_rope *rope,

@@ -496,6 +496,15 @@ def project_grouped(delta_slabs, basis_l):
     return cat @ np.asarray(basis_l, np.float64).T
 
 
+def fit_grouped(delta_slabs, r):
+    """Eq. 7 for one layer under D = H d (Sec. 3.1): the truncated SVD of the concatenated deviation
+    [T, H d] (the heads' deviations side by side on the feature axis).  delta_slabs: list over heads
+    of [T, d].  Returns (basis [r, H d], eigenvalues [H d] of its Gram matrix, descending), exactly
+    fit_basis on the concatenation."""
+    cat = np.concatenate([np.asarray(x, np.float64) for x in delta_slabs], axis=1)
+    return fit_basis(cat, r)
+
+
 def realign_basis(basis_k, s, inv_freq, pairing=ROPE_HALF):
     """App. A.2 (PF-induced deltas): a stored key correction is "positionally re-aligned when reused".
     A rotation acts on the channel axis and is linear, so Rot_s(c . B) = c . Rot_s(B): re-aligning a

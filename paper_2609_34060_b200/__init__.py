@@ -35,7 +35,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_selftest_wait_expiry", "kvc_state_update_check", "kvc_state_update_chain",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_group_fit_eigenvalues", "kvc_group_fit_solver", "kvc_selftest_wait_expiry", "kvc_state_update_check", "kvc_state_update_chain",
     "kvc_chain_update_workspace_bytes", "kvc_chain_update_edge_stride", "kvc_chain_fused", "kvc_chain_workspace_bytes",
 )
 
@@ -109,6 +109,10 @@ def load(path: Optional[str] = None):
     lib.kvc_fit_eigenvalues.restype = vp
     lib.kvc_fit_solver.argtypes = [PC, vp]
     lib.kvc_fit_solver.restype = vp
+    lib.kvc_group_fit_eigenvalues.argtypes = [PC, vp]
+    lib.kvc_group_fit_eigenvalues.restype = vp
+    lib.kvc_group_fit_solver.argtypes = [PC, vp]
+    lib.kvc_group_fit_solver.restype = vp
     lib.kvc_state_realign.argtypes = [PS, i32, i32, i32, i32, PR, vp, vp]
     lib.kvc_token_weights.argtypes = [PC, i32, PS, C.POINTER(i32), i32, PR, C.c_double, vp, vp, vp, sz, vp]
     lib.kvc_token_weights_workspace_bytes.argtypes = [PC, i32]
@@ -440,6 +444,28 @@ def kvc_fit_solver(tgt: Cache, workspace: torch.Tensor) -> torch.Tensor:
     off = p - workspace.data_ptr()
     n = tgt.L * tgt.H * 2
     return workspace.view(torch.uint8)[off: off + 4 * n].view(torch.int32).view(tgt.L, tgt.H, 2)
+
+
+def kvc_group_fit_eigenvalues(tgt: Cache, workspace: torch.Tensor) -> torch.Tensor:
+    """float32 [L, 2, H d] view into the workspace of a layer-grouped FIT update."""
+    c = tgt.struct()
+    p = load().kvc_group_fit_eigenvalues(C.byref(c), workspace.data_ptr())
+    if not p:
+        raise KvcError(KVC_E_INVALID_ARG, "kvc_group_fit_eigenvalues")
+    off = p - workspace.data_ptr()
+    n = tgt.L * 2 * tgt.H * tgt.d
+    return workspace.view(torch.uint8)[off: off + 4 * n].view(torch.float32).view(tgt.L, 2, tgt.H * tgt.d)
+
+
+def kvc_group_fit_solver(tgt: Cache, workspace: torch.Tensor) -> torch.Tensor:
+    """int32 [L, 2] view into the workspace of a layer-grouped FIT update: 0 where the result was accepted."""
+    c = tgt.struct()
+    p = load().kvc_group_fit_solver(C.byref(c), workspace.data_ptr())
+    if not p:
+        raise KvcError(KVC_E_INVALID_ARG, "kvc_group_fit_solver")
+    off = p - workspace.data_ptr()
+    n = tgt.L * 2
+    return workspace.view(torch.uint8)[off: off + 4 * n].view(torch.int32).view(tgt.L, 2)
 
 
 def kvc_state_realign(st: State, shift: int, rope: Rope, out: Optional[torch.Tensor] = None, stream=None) -> State:

@@ -296,8 +296,21 @@ static size_t fit_evals_end(const kvc_cache* tgt) {
 }
 static size_t fit_solver_offset(const kvc_cache* tgt) { return (fit_evals_end(tgt) + 255) & ~(size_t)255; }
 
+// FIT workspace of a layer-grouped state: eigenvalues [L*2][H d], solver codes [L*2] on the next 256-byte
+// boundary, then (again aligned) the partial back-projections and the partial traces.
+static size_t group_evals_bytes(const kvc_cache* tgt) { return (size_t)tgt->L * 2 * tgt->H * tgt->d * sizeof(float); }
+static size_t group_solver_offset(const kvc_cache* tgt) { return (group_evals_bytes(tgt) + 255) & ~(size_t)255; }
+static size_t group_ypart_offset(const kvc_cache* tgt) {
+  return (group_solver_offset(tgt) + (size_t)tgt->L * 2 * sizeof(int32_t) + 255) & ~(size_t)255;
+}
+static size_t group_trpart_offset(const kvc_cache* tgt, int r) {
+  return group_ypart_offset(tgt) + (size_t)kGroupFitParts * tgt->L * 2 * r * tgt->H * tgt->d * sizeof(float);
+}
+
 size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
   if (!tgt || !st || (mode != KVC_FIT && mode != KVC_FIT_FAST)) return 0;
+  if (st->grouping == KVC_GROUP_LAYER)
+    return group_trpart_offset(tgt, st->r) + (size_t)kGroupFitParts * tgt->L * 2 * tgt->H * sizeof(float);
   if (mode == KVC_FIT) return fit_evals_end(tgt);
   return fit_solver_offset(tgt) + (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t);
 }
@@ -338,7 +351,7 @@ static int plan_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift
   if (P->empty) return KVC_OK;
   if (!st->coeff_k || !st->coeff_v) return KVC_E_INVALID_ARG;
   if (P->fit && (st->basis_dtype != KVC_F32 || st->r > 64)) return KVC_E_UNSUPPORTED;
-  if (P->fit && st->grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;   // needs a (H d) x (H d) eigensolver
+  if (P->fit && st->grouping != KVC_GROUP_HEAD && st->r > kSubspaceMaxRank) return KVC_E_UNSUPPORTED;   // subspace solver only
   return KVC_OK;
 }
 
@@ -444,6 +457,48 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s) {
   return KVC_OK;
 }
 
+// FIT of a layer-grouped state (D = H d): block subspace iteration through the two streaming passes
+//   Z = Delta Q^T (the grouped projection)  and  Y = Z^T Delta (the back-projection),
+// three applications of G = Delta^T Delta in a fixed schedule, Rayleigh-Ritz, then the projection on the
+// final basis.  The state's own buffers hold the iterates: bases = trial rows, coefficients = Z.
+static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* workspace, uint32_t* status, cudaStream_t s) {
+  const kvc_state* st = P.st;
+  GroupFitLaunch G;
+  memset(&G, 0, sizeof(G));
+  G.src = P.ds;
+  G.tgt = P.dt;
+  G.coeff_k = st->coeff_k;
+  G.coeff_v = st->coeff_v;
+  G.basis_k = reinterpret_cast<float*>(st->basis_k);
+  G.basis_v = reinterpret_cast<float*>(st->basis_v);
+  char* ws = reinterpret_cast<char*>(workspace);
+  G.evals = reinterpret_cast<float*>(ws);
+  G.solver = reinterpret_cast<int32_t*>(ws + group_solver_offset(tgt));
+  G.ypart = reinterpret_cast<float*>(ws + group_ypart_offset(tgt));
+  G.trpart = reinterpret_cast<float*>(ws + group_trpart_offset(tgt, st->r));
+  G.r = st->r;
+  G.n_cov = st->n_cov;
+  G.pairing = P.rope->pairing;
+  G.shift = P.shift;
+  G.L = P.L;
+  G.H = P.H;
+  G.d = P.d;
+  G.parts = kGroupFitParts;
+  const int per = (st->n_cov + kGroupFitParts - 1) / kGroupFitParts;
+  G.tokens_per_part = (per + 31) / 32 * 32;
+  G.status = status;
+  rope_tables(P.rope, P.d, P.shift, G.cs, G.sn);
+  if (launch_group_small(G, KVC_GROUP_OP_START, s) != cudaSuccess) return KVC_E_CUDA;
+  static const int ops[3] = {KVC_GROUP_OP_ORTH_START, KVC_GROUP_OP_ORTH, KVC_GROUP_OP_RITZ};
+  for (int it = 0; it < 3; ++it) {
+    int rc = project_edge(P, status, s);
+    if (rc != KVC_OK) return rc;
+    if (launch_group_backproject(G, s) != cudaSuccess) return KVC_E_CUDA;
+    if (launch_group_small(G, ops[it], s) != cudaSuccess) return KVC_E_CUDA;
+  }
+  return KVC_OK;
+}
+
 int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
                      int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
   UpdatePlan P;
@@ -457,7 +512,9 @@ int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, 
   uint32_t* status = status_ptr();
   if (!status) return KVC_E_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  if (P.fit) {
+  if (P.fit && st->grouping == KVC_GROUP_LAYER) {
+    if ((rc = group_fit_edge(P, tgt, workspace, status, s)) != KVC_OK) return rc;
+  } else if (P.fit) {
     FitLaunch F;
     if ((rc = fit_gram(P, workspace, status, &F, s)) != KVC_OK) return rc;
     const size_t solver_bytes = (size_t)P.L * P.H * 2 * sizeof(int32_t);
@@ -487,17 +544,28 @@ int kvc_state_update_chain(const kvc_cache* agents, int32_t n_agents, const int3
   size_t off[kMaxFitEdges + 1];
   off[0] = 0;
   int rc;
-  bool any_fit = false, uniform = true;
+  bool any_fit = false, uniform = true, any_grouped_fit = false;
   for (int e = 0; e < n_edges; ++e) {
     const int32_t shift = prefix_len[e + 1] - prefix_len[e];
     if ((rc = plan_update(&agents[e], &agents[e + 1], shift, rope, &states[e], mode, &P[e])) != KVC_OK) return rc;
     off[e + 1] = off[e] + kvc_chain_update_edge_stride(&agents[e + 1], &states[e], mode);
     any_fit |= P[e].fit && !P[e].empty;
+    any_grouped_fit |= P[e].fit && !P[e].empty && states[e].grouping == KVC_GROUP_LAYER;
     uniform &= !P[e].empty && P[e].L == P[0].L && P[e].H == P[0].H && P[e].d == P[0].d && states[e].r == states[0].r &&
                states[e].n_cov == states[0].n_cov && off[e + 1] - off[e] == off[1];
   }
   if (any_fit && (!workspace || workspace_bytes < off[n_edges] || (reinterpret_cast<uintptr_t>(workspace) & 255)))
     return KVC_E_WORKSPACE;
+  if (any_grouped_fit) {
+    // layer-grouped states have no shared eigensolver launch: their edges run one after the other
+    for (int e = 0; e < n_edges; ++e) {
+      const int32_t shift = prefix_len[e + 1] - prefix_len[e];
+      rc = kvc_state_update(&agents[e], &agents[e + 1], shift, rope, &states[e], mode,
+                            reinterpret_cast<char*>(workspace) + off[e], off[e + 1] - off[e], stream);
+      if (rc != KVC_OK) return rc;
+    }
+    return KVC_OK;
+  }
   uint32_t* status = status_ptr();
   if (!status) return KVC_E_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -651,6 +719,16 @@ int kvc_effective_rank(const float* evals, int32_t n_matrices, int32_t d, double
 const float* kvc_fit_eigenvalues(const kvc_cache* tgt, const void* workspace) {
   if (!tgt || !workspace || tgt->L <= 0 || tgt->H <= 0 || tgt->d <= 0) return nullptr;
   return reinterpret_cast<const float*>(workspace) + 2 * (size_t)tgt->L * tgt->H * 2 * tgt->d * tgt->d;
+}
+
+const float* kvc_group_fit_eigenvalues(const kvc_cache* tgt, const void* workspace) {
+  if (!tgt || !workspace || tgt->L <= 0 || tgt->H <= 0 || tgt->d <= 0) return nullptr;
+  return reinterpret_cast<const float*>(workspace);
+}
+
+const int32_t* kvc_group_fit_solver(const kvc_cache* tgt, const void* workspace) {
+  if (!tgt || !workspace || tgt->L <= 0 || tgt->H <= 0 || tgt->d <= 0) return nullptr;
+  return reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(workspace) + group_solver_offset(tgt));
 }
 
 const int32_t* kvc_fit_solver(const kvc_cache* tgt, const void* workspace) {

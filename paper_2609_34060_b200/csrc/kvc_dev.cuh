@@ -89,6 +89,26 @@ struct FitLaunch {             // Gram + eigensolve
   alignas(16) float sn[kMaxHalfD];
 };
 
+struct GroupFitLaunch {        // FIT of states grouped by layer (D = H d): back-projection and small dense work
+  DevCache src, tgt;
+  const float* coeff_k;        // Z = Delta Q^T, [L][n_cov][r] (the state's coefficient buffers)
+  const float* coeff_v;
+  float* basis_k;              // the r trial vectors as rows, [L][r][H d] (the state's bases): in and out
+  float* basis_v;
+  float* ypart;                // [parts][L*2][r][H d] partial back-projections (part 0 doubles as their sum)
+  float* trpart;               // [parts][L*2][H] partial sums of Delta^2
+  float* evals;                // [L*2][H d]
+  int32_t* solver;             // [L*2] per-problem code
+  int32_t r, n_cov, pairing, shift, L, H, d, parts, tokens_per_part, pad;
+  uint32_t* status;
+  alignas(16) float cs[kMaxHalfD];
+  alignas(16) float sn[kMaxHalfD];
+};
+constexpr int KVC_GROUP_OP_START = 0;       // hashed start rows
+constexpr int KVC_GROUP_OP_ORTH_START = 1;  // rows <- orth(back-projection), conditioning unknown
+constexpr int KVC_GROUP_OP_ORTH = 2;        // rows <- orth(back-projection)
+constexpr int KVC_GROUP_OP_RITZ = 3;        // Rayleigh-Ritz, acceptance, output
+
 struct GateLaunch {            // Eq. 9 for one anchor, CUDA-core kernel
   DevCache src;                // values only
   const float* coeff;          // [L,H,n_cov,r] value coefficients of the anchor's base factorisation
@@ -192,6 +212,61 @@ __device__ __forceinline__ uint32_t f2_to_bf16x2(f32x2 v) {
   f2_unpack(v, a, b);
   const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// ---- helpers of the CUDA-core kernels: one lane handles 16 channels of a token (two 8-channel chunks)
+// HALF: x[i] pairs with x[8+i];  INTERLEAVED: (x[2m], x[2m+1]) inside each chunk.
+__device__ __forceinline__ void rope16(float* x, const float* cs, const float* sn, int pairing) {
+  if (pairing == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float a = x[i], b = x[8 + i];
+      x[i] = a * cs[i] - b * sn[i];
+      x[8 + i] = a * sn[i] + b * cs[i];
+    }
+  } else {
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const float a = x[2 * m], b = x[2 * m + 1];
+      x[2 * m] = a * cs[m] - b * sn[m];
+      x[2 * m + 1] = a * sn[m] + b * cs[m];
+    }
+  }
+}
+
+template <int D>
+__device__ __forceinline__ void lane_channels(int j, int pairing, int& chA, int& chB) {
+  if (pairing == 0) {
+    chA = 8 * j;
+    chB = D / 2 + 8 * j;
+  } else {
+    chA = 16 * j;
+    chB = 16 * j + 8;
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// deviation of one (token, lane) : 16 channels of  tgt - Rot(src)
+// ---------------------------------------------------------------------------------
+template <int D>
+__device__ __forceinline__ bool delta16(const DevCache& src, const DevCache& tgt, int is_v, int l, int h, int t,
+                                        int chA, int chB, const float* cs, const float* sn, bool rotate, int pairing,
+                                        uint32_t* status, float* out) {
+  const __nv_bfloat16* trow = row_ptr(tgt, is_v ? tgt.v : tgt.k, l, h, t, status);
+  if (!trow) return false;
+  unpack8(*reinterpret_cast<const uint4*>(trow + chA), out);
+  unpack8(*reinterpret_cast<const uint4*>(trow + chB), out + 8);
+  if (src.k) {
+    const __nv_bfloat16* srow = row_ptr(src, is_v ? src.v : src.k, l, h, t, status);
+    if (!srow) return false;
+    float x[16];
+    unpack8(*reinterpret_cast<const uint4*>(srow + chA), x);
+    unpack8(*reinterpret_cast<const uint4*>(srow + chB), x + 8);
+    if (rotate) rope16(x, cs, sn, pairing);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] -= x[i];
+  }
+  return true;
 }
 
 }  // namespace kvc

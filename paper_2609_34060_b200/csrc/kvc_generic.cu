@@ -27,36 +27,6 @@ __device__ __forceinline__ int find_item(const int64_t* prefix, int n_items, int
 }
 
 // Rotate the 16 channels one lane holds (two 8-channel chunks) by the item's shift.
-// HALF: x[i] pairs with x[8+i];  INTERLEAVED: (x[2m], x[2m+1]) inside each chunk.
-__device__ __forceinline__ void rope16(float* x, const float* cs, const float* sn, int pairing) {
-  if (pairing == 0) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float a = x[i], b = x[8 + i];
-      x[i] = a * cs[i] - b * sn[i];
-      x[8 + i] = a * sn[i] + b * cs[i];
-    }
-  } else {
-#pragma unroll
-    for (int m = 0; m < 8; ++m) {
-      const float a = x[2 * m], b = x[2 * m + 1];
-      x[2 * m] = a * cs[m] - b * sn[m];
-      x[2 * m + 1] = a * sn[m] + b * cs[m];
-    }
-  }
-}
-
-template <int D>
-__device__ __forceinline__ void lane_channels(int j, int pairing, int& chA, int& chB) {
-  if (pairing == 0) {
-    chA = 8 * j;
-    chB = D / 2 + 8 * j;
-  } else {
-    chA = 16 * j;
-    chB = 16 * j + 8;
-  }
-}
-
 // ---------------------------------------------------------------------------------
 // apply: dst = bf16(Rot(src) + coeff . basis)
 // ---------------------------------------------------------------------------------
@@ -167,30 +137,6 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
     *reinterpret_cast<uint4*>(drow + chA) = oa;
     *reinterpret_cast<uint4*>(drow + chB) = ob;
   }
-}
-
-// ---------------------------------------------------------------------------------
-// deviation of one (token, lane) : 16 channels of  tgt - Rot(src)
-// ---------------------------------------------------------------------------------
-template <int D>
-__device__ __forceinline__ bool delta16(const DevCache& src, const DevCache& tgt, int is_v, int l, int h, int t,
-                                        int chA, int chB, const float* cs, const float* sn, bool rotate, int pairing,
-                                        uint32_t* status, float* out) {
-  const __nv_bfloat16* trow = row_ptr(tgt, is_v ? tgt.v : tgt.k, l, h, t, status);
-  if (!trow) return false;
-  unpack8(*reinterpret_cast<const uint4*>(trow + chA), out);
-  unpack8(*reinterpret_cast<const uint4*>(trow + chB), out + 8);
-  if (src.k) {
-    const __nv_bfloat16* srow = row_ptr(src, is_v ? src.v : src.k, l, h, t, status);
-    if (!srow) return false;
-    float x[16];
-    unpack8(*reinterpret_cast<const uint4*>(srow + chA), x);
-    unpack8(*reinterpret_cast<const uint4*>(srow + chB), x + 8);
-    if (rotate) rope16(x, cs, sn, pairing);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) out[i] -= x[i];
-  }
-  return true;
 }
 
 // ---------------------------------------------------------------------------------

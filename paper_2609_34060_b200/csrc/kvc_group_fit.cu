@@ -1,0 +1,476 @@
+// FIT for states grouped by layer (Sec. 3.1 with D = H d, the width of a layer's cached features; Eq. 7):
+// the r leading right singular vectors of the deviation Delta [n_cov, D] of one layer (keys or values,
+// all KV heads side by side), without forming the D x D Gram matrix G = Delta^T Delta.
+//
+// Block subspace iteration on G through its factors: with the r trial vectors as the rows of the
+// state's basis [r, D],
+//     Z = Delta Q^T          the grouped projection pass (coefficients [n_cov, r]; it exists already)
+//     Y = Z^T Delta = Q G    the back-projection pass of this file, [r, D]
+// so one application of G costs two streaming passes over the caches and nothing of size D x D is
+// ever stored.  The schedule is fixed (nothing is read back to the host between launches):
+//     Q0 hashed;  Y = Q0 G, Q1 = orth(Y);  Y = Q1 G, Q2 = orth(Y);  Y = Q2 G;  Rayleigh-Ritz on (Q2, Y):
+// H = Q2 Y^T = W diag(theta) W^T, Ritz rows W^T Q2, their residuals from W^T Y, and the acceptance test
+// of the per-head subspace solver with trace(G) = |Delta|_F^2 accumulated by the back-projection pass.
+// The Ritz rows are written as the basis either way; when the test fails (no gap behind the r-th
+// eigenvalue: a subspace of G this schedule cannot resolve) the matrix's solver code says so and
+// KVC_FLAG_NOT_CONVERGED is raised.  The caller finishes with one projection pass on the final basis.
+//
+// The small dense work (orthonormalisation of r rows of length D by Cholesky QR, the r x r eigenproblem,
+// the Ritz rows) runs as one block of 256 threads per (layer, K|V) on rows that stay L2-resident.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kvc.h"
+#include "kvc_dev.cuh"
+#include "kvc_eig_small.cuh"
+#include "kvc_launch.h"
+
+namespace kvc {
+namespace {
+
+using namespace eigsmall;
+
+constexpr int kTT = 32;          // tokens per staged tile of the back-projection
+
+// ---------------------------------------------------------------------------------------------
+// Back-projection  Y[q, h d + c] = sum_t Z[t, q] Delta[l, h, t, c]  and  trace = sum Delta^2.
+// One block per (layer, head, K|V, token range); the ranges' partial sums are added later in a
+// fixed order.  Thread (cg, qg) accumulates channels 4 cg .. + 3 against RQ ranks.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) group_backproject_kernel(const __grid_constant__ GroupFitLaunch p) {
+  constexpr int LPT = D / 16;
+  constexpr int CG = D / 4;          // channel groups
+  constexpr int QG = 256 / CG;       // rank groups
+  constexpr int RQ = kMaxM / QG;     // ranks per thread: 4 (D = 128) or 2 (D = 64)
+  __shared__ __align__(16) float delta_s[kTT * D];
+  __shared__ __align__(16) float z_s[kTT * kMaxM];
+  __shared__ float red[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int b = blockIdx.x;
+  const int part = b % p.parts;
+  b /= p.parts;
+  const int is_v = b & 1, slab = b >> 1;
+  const int l = slab / p.H, h = slab % p.H;
+  const int t_begin = part * p.tokens_per_part, t_end = min(p.n_cov, t_begin + p.tokens_per_part);
+  const bool rotate = (!is_v) && (p.shift != 0);
+  const int cg = tid % CG, qg = tid / CG;
+  const float* coeff = (is_v ? p.coeff_v : p.coeff_k) + (int64_t)l * p.n_cov * p.r;
+  float acc[4][RQ];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int k = 0; k < RQ; ++k) acc[a][k] = 0.f;
+  float sq = 0.f;
+
+  for (int t0 = t_begin; t0 < t_end; t0 += kTT) {
+    __syncthreads();
+    for (int w = tid; w < kTT * LPT; w += 256) {
+      const int tl = w / LPT, j = w % LPT;
+      int chA, chB;
+      lane_channels<D>(j, p.pairing, chA, chB);
+      float dl[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) dl[i] = 0.f;
+      const int t = t0 + tl;
+      if (t < t_end) {
+        float cs[8], sn[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          cs[i] = p.cs[8 * j + i];
+          sn[i] = p.sn[8 * j + i];
+        }
+        if (!delta16<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, cs, sn, rotate, p.pairing, p.status, dl)) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) dl[i] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) sq = fmaf(dl[i], dl[i], sq);
+      float* row = delta_s + tl * D;
+      *reinterpret_cast<float4*>(row + chA) = *reinterpret_cast<float4*>(dl);
+      *reinterpret_cast<float4*>(row + chA + 4) = *reinterpret_cast<float4*>(dl + 4);
+      *reinterpret_cast<float4*>(row + chB) = *reinterpret_cast<float4*>(dl + 8);
+      *reinterpret_cast<float4*>(row + chB + 4) = *reinterpret_cast<float4*>(dl + 12);
+    }
+    for (int i = tid; i < kTT * kMaxM; i += 256) {
+      const int tl = i >> 5, q = i & 31;
+      const int t = t0 + tl;
+      z_s[i] = (t < t_end && q < p.r) ? coeff[(int64_t)t * p.r + q] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int tl = 0; tl < kTT; ++tl) {
+      const float4 dv = *reinterpret_cast<const float4*>(delta_s + tl * D + 4 * cg);
+      float zv[RQ];
+#pragma unroll
+      for (int k = 0; k < RQ; ++k) zv[k] = z_s[tl * kMaxM + RQ * qg + k];
+#pragma unroll
+      for (int k = 0; k < RQ; ++k) {
+        acc[0][k] = fmaf(dv.x, zv[k], acc[0][k]);
+        acc[1][k] = fmaf(dv.y, zv[k], acc[1][k]);
+        acc[2][k] = fmaf(dv.z, zv[k], acc[2][k]);
+        acc[3][k] = fmaf(dv.w, zv[k], acc[3][k]);
+      }
+    }
+  }
+  const int Dg = p.H * D;
+  float* y = p.ypart + ((int64_t)part * p.L * 2 + (l * 2 + is_v)) * p.r * Dg + h * D;
+#pragma unroll
+  for (int k = 0; k < RQ; ++k) {
+    const int q = RQ * qg + k;
+    if (q < p.r) *reinterpret_cast<float4*>(y + (int64_t)q * Dg + 4 * cg) = make_float4(acc[0][k], acc[1][k], acc[2][k], acc[3][k]);
+  }
+  sq = wsum(sq);
+  if (lane == 0) red[warp] = sq;
+  __syncthreads();
+  if (tid == 0) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += red[w];
+    p.trpart[((int64_t)part * p.L * 2 + (l * 2 + is_v)) * p.H + h] = s;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Small dense work on r rows of length Dg, one block per (layer, K|V).
+// ---------------------------------------------------------------------------------------------
+struct SmallMem {
+  float s[kMaxM * kSP];          // Gram matrix of the rows / Cholesky factor / scratch copy of H
+  float h[kMaxM * kSP];          // projected matrix
+  float w[kMaxM * kSP];          // its eigenvectors (sorted: ws)
+  float ta[kMaxM * 65];          // column tiles of the two row blocks of a product
+  float tb[kMaxM * 65];
+  float pn[8 * kMaxM], pd[8 * kMaxM], pr[8 * kMaxM];   // per-warp partial sums per row
+  float pbest[8 * kMaxM];
+  int pidx[8 * kMaxM];
+  float th[kMaxM], inv[kMaxM], rho2[kMaxM];
+  int perm[kMaxM];
+  float red[8];
+  int flag;
+};
+
+// S[i][j] = sum_c A[i][c] B[j][c]  for i, j < 32 (rows >= m count as zero); rows have stride Dg.
+__device__ __forceinline__ void gram_rows(const float* A, const float* B, float* S, SmallMem& sm, int m, int Dg, int tid) {
+  const int j = tid & 31, i0 = tid >> 5;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int c0 = 0; c0 < Dg; c0 += 64) {
+    __syncthreads();
+    for (int idx = tid; idx < kMaxM * 64; idx += kThreads) {
+      const int i = idx >> 6, cc = idx & 63;
+      const bool on = i < m && c0 + cc < Dg;
+      sm.ta[i * 65 + cc] = on ? A[(int64_t)i * Dg + c0 + cc] : 0.f;
+      sm.tb[i * 65 + cc] = on ? B[(int64_t)i * Dg + c0 + cc] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int cc = 0; cc < 64; ++cc) {
+      const float bv = sm.tb[j * 65 + cc];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[k] = fmaf(sm.ta[(i0 + 8 * k) * 65 + cc], bv, acc[k]);
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < 4; ++k) S[(i0 + 8 * k) * kSP + j] = acc[k];
+  __syncthreads();
+}
+
+// Cholesky factor of the m x m matrix S (in place, lower triangle, reciprocal pivots on the diagonal)
+// by warp 0.  shift_rel > 0 adds that fraction of the largest diagonal entry to the diagonal first.
+// Returns false when a pivot cancels (the rows are dependent at float32).
+__device__ __forceinline__ bool chol_small(float* S, SmallMem& sm, int m, int tid, float shift_rel) {
+  if (tid < 32) {
+    const int lane = tid;
+    float d0 = (lane < m) ? S[lane * kSP + lane] : 0.f;
+    const float dmax = wmax(d0);
+    if (lane < m && shift_rel > 0.f) {
+      d0 += shift_rel * dmax;
+      S[lane * kSP + lane] = d0;
+    }
+    __syncwarp();
+    bool ok = dmax > 0.f;
+    for (int j = 0; j < m && ok; ++j) {
+      const float piv = S[j * kSP + j];
+      const float dj = __shfl_sync(0xffffffffu, d0, j);
+      ok = piv > 1e-5f * dj;
+      const float rl = ok ? rsqrtf(piv) : 0.f;
+      float lij = 0.f;
+      if (lane > j && lane < m) {
+        lij = S[lane * kSP + j] * rl;
+        S[lane * kSP + j] = lij;
+      }
+      __syncwarp();
+      if (lane > j && lane < m) {
+        for (int k = j + 1; k <= lane; ++k) S[lane * kSP + k] = fmaf(-lij, S[k * kSP + j], S[lane * kSP + k]);
+      }
+      if (lane == j) S[j * kSP + j] = rl;
+      __syncwarp();
+    }
+    if (lane == 0) sm.flag = ok ? 1 : 0;
+  }
+  __syncthreads();
+  const bool ok = sm.flag != 0;
+  __syncthreads();
+  return ok;
+}
+
+// Rows of Dst = L^-1 (rows of A): every thread solves the triangular system for its own columns.
+__device__ __forceinline__ void solve_rows(const float* A, float* Dst, const float* S, int m, int Dg, int tid) {
+  for (int c = tid; c < Dg; c += kThreads) {
+    float x[kMaxM];
+#pragma unroll
+    for (int j = 0; j < kMaxM; ++j) x[j] = (j < m) ? A[(int64_t)j * Dg + c] : 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxM; ++j) {
+      if (j < m) {
+        float a = x[j];
+#pragma unroll
+        for (int k = 0; k < j; ++k) a = fmaf(-S[j * kSP + k], x[k], a);
+        x[j] = a * S[j * kSP + j];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kMaxM; ++j)
+      if (j < m) Dst[(int64_t)j * Dg + c] = x[j];
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_constant__ GroupFitLaunch p, int op) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SmallMem& sm = *reinterpret_cast<SmallMem*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int prob = blockIdx.x;                    // l * 2 + is_v
+  const int l = prob >> 1, is_v = prob & 1;
+  const int Dg = p.H * p.d;
+  const int m = min(min(p.r, Dg), p.n_cov);
+  float* Q = (is_v ? p.basis_v : p.basis_k) + (int64_t)l * p.r * Dg;          // [r][Dg]
+  float* Y = p.ypart + (int64_t)prob * p.r * Dg;                               // part 0 doubles as the sum
+  int32_t* code = p.solver + prob;
+
+  if (op == KVC_GROUP_OP_START) {
+    for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) {
+      const int q = (int)(i / Dg), c = (int)(i - (int64_t)q * Dg);
+      Q[i] = (q < m) ? start_value(c, q) : 0.f;
+    }
+    if (tid == 0) *code = 0;
+    return;
+  }
+
+  // the partial sums of the back-projection, added in a fixed order
+  for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) {
+    float a = Y[i];
+    for (int part = 1; part < p.parts; ++part) a += p.ypart[((int64_t)part * p.L * 2 + prob) * p.r * Dg + i];
+    Y[i] = a;
+  }
+  __syncthreads();
+  if (*code != 0 && op != KVC_GROUP_OP_RITZ) return;   // given up earlier: nothing to orthonormalise
+
+  if (op == KVC_GROUP_OP_ORTH || op == KVC_GROUP_OP_ORTH_START) {
+    // Cholesky QR on the rows of Y: a shifted pass first where the conditioning is unknown (the
+    // hashed start block after one product), then plain passes; the result becomes Q
+    const int passes = (op == KVC_GROUP_OP_ORTH_START) ? 3 : 2;
+    const float* src = Y;
+    for (int pass = 0; pass < passes; ++pass) {
+      gram_rows(src, src, sm.s, sm, m, Dg, tid);
+      const bool shifted = (pass == 0);
+      if (!chol_small(sm.s, sm, m, tid, shifted ? 1e-5f : 0.f)) {
+        if (tid == 0) *code = KVC_SOLVER_FULL_DEPENDENT;
+        return;
+      }
+      solve_rows(src, Q, sm.s, m, Dg, tid);
+      src = Q;
+    }
+    return;
+  }
+
+  // ---- KVC_GROUP_OP_RITZ: Rayleigh-Ritz on (Q, Y = Q G), acceptance, output
+  float tr = 0.f;
+  for (int part = 0; part < p.parts; ++part)
+    for (int h = 0; h < p.H; ++h) tr += p.trpart[((int64_t)part * p.L * 2 + prob) * p.H + h];
+  float* evals = p.evals + (int64_t)prob * Dg;
+  if (*code != 0 || !(tr > 0.f)) {
+    // a zero deviation (or rows that became dependent): no basis, all eigenvalues zero
+    for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) Q[i] = 0.f;
+    for (int i = tid; i < Dg; i += kThreads) evals[i] = 0.f;
+    if (tid == 0) {
+      *code = KVC_SOLVER_FULL_DEPENDENT;
+      if (tr > 0.f) atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
+    }
+    return;
+  }
+  gram_rows(Q, Y, sm.s, sm, m, Dg, tid);
+  for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
+    const int a = i >> 5, b = i & 31;
+    sm.h[a * kSP + b] = 0.5f * (sm.s[a * kSP + b] + sm.s[b * kSP + a]);
+  }
+  __syncthreads();
+  int reason = 0;
+  if (!jacobi_eig(sm.h, sm.s, sm.w, &sm.flag, m, tid)) reason = KVC_SOLVER_FULL_SWEEPS;
+  // Ritz values in descending order (the rotations leave them in an arbitrary one)
+  {
+    const int nj = 2 * ((m + 1) >> 1);
+    if (tid < kMaxM) {
+      // the padded slot of an odd m: the one whose eigenvector is still the unit vector e_m
+      const bool real = tid < nj && !(nj != m && sm.w[m * kSP + tid] != 0.f);
+      const float mine = real ? sm.h[tid * kSP + tid] : 0.f;
+      int rank = 0;
+      for (int i = 0; i < nj; ++i) {
+        const bool ireal = !(nj != m && sm.w[m * kSP + i] != 0.f);
+        const float o = sm.h[i * kSP + i];
+        if (ireal && real) rank += (o > mine || (o == mine && i < tid)) ? 1 : 0;
+      }
+      sm.perm[tid] = 0;
+      __syncwarp();
+      if (real) sm.perm[rank] = tid;
+    }
+    __syncthreads();
+    for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
+      const int a = i >> 5, b = i & 31;
+      sm.s[a * kSP + b] = (a < m && b < m) ? sm.w[a * kSP + sm.perm[b]] : 0.f;   // sorted eigenvectors, columns
+    }
+    for (int i = tid; i < 8 * kMaxM; i += kThreads) {
+      sm.pn[i] = sm.pd[i] = sm.pr[i] = 0.f;
+      sm.pbest[i] = -1.f;
+      sm.pidx[i] = 0;
+    }
+    __syncthreads();
+  }
+  const float* Ws = sm.s;
+  // pass 1: Ritz rows z_j = sum_k Ws[k][j] q_k over Q (in place) and G z_j over Y (in place), with the
+  // sums z.Gz, z.z and the largest-magnitude entry of every row
+  for (int c0 = 0; c0 < Dg; c0 += kThreads) {
+    const int c = c0 + tid;
+    const bool on = c < Dg;
+    float q[kMaxM], y[kMaxM];
+#pragma unroll
+    for (int k = 0; k < kMaxM; ++k) {
+      q[k] = (on && k < m) ? Q[(int64_t)k * Dg + c] : 0.f;
+      y[k] = (on && k < m) ? Y[(int64_t)k * Dg + c] : 0.f;
+    }
+    for (int j = 0; j < m; ++j) {
+      float zj = 0.f, gj = 0.f;
+#pragma unroll
+      for (int k = 0; k < kMaxM; ++k) {
+        const float wv = Ws[k * kSP + j];
+        zj = fmaf(wv, q[k], zj);
+        gj = fmaf(wv, y[k], gj);
+      }
+      if (on) {
+        Q[(int64_t)j * Dg + c] = zj;
+        Y[(int64_t)j * Dg + c] = gj;
+      }
+      const float n1 = wsum(zj * gj), d1 = wsum(zj * zj);
+      float best = fabsf(zj);
+      int bi = on ? c : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ob > best || (ob == best && oi < bi)) {
+          best = ob;
+          bi = oi;
+        }
+      }
+      if (lane == 0) {
+        sm.pn[warp * kMaxM + j] += n1;
+        sm.pd[warp * kMaxM + j] += d1;
+        if (best > sm.pbest[warp * kMaxM + j]) {      // later tiles have larger indices: strict '>' keeps the first
+          sm.pbest[warp * kMaxM + j] = best;
+          sm.pidx[warp * kMaxM + j] = bi;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (tid < kMaxM) {
+    float ns = 0.f, ds = 0.f, best = -1.f;
+    int bi = 0;
+    for (int w = 0; w < 8; ++w) {
+      ns += sm.pn[w * kMaxM + tid];
+      ds += sm.pd[w * kMaxM + tid];
+      const float ob = sm.pbest[w * kMaxM + tid];
+      const int oi = sm.pidx[w * kMaxM + tid];
+      if (ob > best || (ob == best && oi < bi)) {
+        best = ob;
+        bi = oi;
+      }
+    }
+    const bool live = tid < m;
+    sm.th[tid] = live ? ns / fmaxf(ds, 1e-30f) : 0.f;
+    const float sgn = (live && Q[(int64_t)tid * Dg + bi] < 0.f) ? -1.f : 1.f;
+    sm.inv[tid] = live ? sgn * rsqrtf(fmaxf(ds, 1e-30f)) : 0.f;
+  }
+  __syncthreads();
+  // pass 2: residuals |G z_j - theta_j z_j|^2 of the unit-length rows, and the rows written out
+  for (int c0 = 0; c0 < Dg; c0 += kThreads) {
+    const int c = c0 + tid;
+    const bool on = c < Dg;
+    for (int j = 0; j < m; ++j) {
+      const float zj = on ? Q[(int64_t)j * Dg + c] : 0.f, gj = on ? Y[(int64_t)j * Dg + c] : 0.f;
+      const float iv = sm.inv[j];
+      const float e = (gj - sm.th[j] * zj) * iv;
+      if (on) Q[(int64_t)j * Dg + c] = zj * iv;
+      const float r1 = wsum(e * e);
+      if (lane == 0) sm.pr[warp * kMaxM + j] += r1;
+    }
+  }
+  for (int64_t i = (int64_t)m * Dg + tid; i < (int64_t)p.r * Dg; i += kThreads) Q[i] = 0.f;
+  __syncthreads();
+  if (tid < kMaxM) {
+    float rs = 0.f;
+    for (int w = 0; w < 8; ++w) rs += sm.pr[w * kMaxM + tid];
+    sm.rho2[tid] = (tid < m) ? rs : 0.f;
+  }
+  __syncthreads();
+  float sumth = 0.f, rhoF2 = 0.f, rhomax2 = 0.f;
+  for (int j = 0; j < m; ++j) {
+    sumth += sm.th[j];
+    rhoF2 += sm.rho2[j];
+    rhomax2 = fmaxf(rhomax2, sm.rho2[j]);
+  }
+  const float th1 = sm.th[0], thm = sm.th[m - 1];
+  const float tau = fmaxf(tr - sumth, 0.f);
+  const float rhoF = sqrtf(rhoF2);
+  const float gap = thm - tau - rhoF;
+  // The products run through the split-precision projection pass (about 2e-5 of a row's length), so the
+  // rows' residuals are held to 2e-4 of the largest eigenvalue; the gap test is the per-head solver's.
+  const bool accept = rhomax2 <= (2e-4f * th1) * (2e-4f * th1) && gap > 0.f && rhoF <= (1.f / 1024.f) * gap;
+  if (reason == 0 && !accept) reason = (gap > 0.f) ? KVC_SOLVER_FULL_SLOW : KVC_SOLVER_FULL_NO_GAP;
+  for (int i = tid; i < Dg; i += kThreads) evals[i] = (i < m) ? sm.th[i] : (Dg > m ? tau / (float)(Dg - m) : 0.f);
+  if (tid == 0) {
+    *code = reason;
+    if (reason != 0) atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_group_backproject(const GroupFitLaunch& G, cudaStream_t s) {
+  const int blocks = G.L * G.H * 2 * G.parts;
+  if (blocks <= 0) return cudaSuccess;
+  if (G.d == 128)
+    group_backproject_kernel<128><<<blocks, 256, 0, s>>>(G);
+  else if (G.d == 64)
+    group_backproject_kernel<64><<<blocks, 256, 0, s>>>(G);
+  else
+    return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_group_small(const GroupFitLaunch& G, int op, cudaStream_t s) {
+  const int blocks = G.L * 2;
+  if (blocks <= 0) return cudaSuccess;
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
+    cudaError_t e = cudaFuncSetAttribute(group_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmallMem));
+    if (e != cudaSuccess) return e;
+    once.mark(once_dev);
+  }
+  group_small_kernel<<<blocks, kThreads, sizeof(SmallMem), s>>>(G, op);
+  return cudaGetLastError();
+}
+
+}  // namespace kvc

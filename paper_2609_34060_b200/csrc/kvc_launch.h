@@ -61,6 +61,11 @@ cudaError_t launch_eig(const FitLaunch& F, int d, const int32_t* solver, cudaStr
 constexpr int kSubspaceMaxRank = 32;
 cudaError_t launch_eig_subspace(const FitLaunch& F, int d, int32_t* solver, cudaStream_t s);
 
+// FIT of layer-grouped states (kvc_group_fit.cu)
+constexpr int kGroupFitParts = 4;   // token ranges whose back-projections are summed in a fixed order
+cudaError_t launch_group_backproject(const GroupFitLaunch& G, cudaStream_t s);
+cudaError_t launch_group_small(const GroupFitLaunch& G, int op, cudaStream_t s);
+
 // reliability gate (kvc_gate.cu)
 cudaError_t launch_gate_generic(const GateLaunch& g, int d, cudaStream_t s);
 cudaError_t launch_effective_rank(const float* evals, int n_mat, int d, float energy, int32_t* out, cudaStream_t s);

@@ -234,7 +234,15 @@ def step_bytes(W):
             + sum(8 * s.r * c.d * c.L * c.H for s in W["states"])
     upd = 0 if only == "apply" else sum(kvc.kvc_update_bytes(W["true"][0], W["states"][a - 1], kvc.KVC_FIT, True)
                                          for a in range(1, n))
-    app = 0 if only == "update" else sum(kvc.kvc_apply_bytes(W["true"][0], W["states"][a - 1]) for a in range(1, n))
+    if only == "update":
+        app = 0
+    elif W.get("chain_ws") is not None:
+        # the fused chain reads agent 0's cache once (4d B per token-slab), every hop's coefficients (8r) and bases,
+        # and writes every hop's cache (4d)
+        c = W["true"][0]
+        app = c.L * c.H * (c.T * (4 * c.d + sum(8 * s.r + 4 * c.d for s in W["states"])) + sum(8 * s.r * c.d for s in W["states"]))
+    else:
+        app = sum(kvc.kvc_apply_bytes(W["true"][0], W["states"][a - 1]) for a in range(1, n))
     return upd, app
 
 

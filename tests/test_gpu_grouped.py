@@ -145,6 +145,127 @@ def test_grouped_project(cfg, path):
             assert np.all(np.abs(g[l] - ref) <= tol), (which, l, float(np.max(np.abs(g[l] - ref) / tol)))
 
 
+def _grouped_edge(cfg, sigma, hop=1):
+    """Source and target of one edge whose deviation has rank r on the concatenated feature axis
+    (D = H d): target = bf16(Align(src) + c B + sigma noise) with B [r, H d] orthonormal rows, built by
+    the oracle from generator draws.  Also the oracle's unrounded Align(src) + c B."""
+    src_cpu = hp.make_cache(cfg)
+    true = _grouped_state(cfg, hop)
+    pl = wl.prefix_lengths(cfg)
+    shift = pl[hop] - pl[hop - 1]
+    nk = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2 * hop).numpy()
+    nv = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2 * hop + 1).numpy()
+    osrc = hp.oracle_cache(src_cpu)
+    ost = _oracle_state(cfg, true)
+    otgt = orc.make_target(osrc, ost, shift, hp.inv_freq(cfg), nk, nv, sigma)
+    as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    if cfg.paged:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v), T=cfg.T, page_table=src_cpu.page_table)
+    else:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v))
+    return src_cpu, tgt_cpu, osrc, otgt, ost, shift
+
+
+def _fit_grouped(src, tgt, shift, cfg, r, mode):
+    L, H, T, d = cfg.L, cfg.H, cfg.T, cfg.d
+    st = kvc.State(torch.zeros(L, T, r, device=DEV), torch.zeros(L, T, r, device=DEV),
+                   torch.full((L, r, H * d), 3.0, device=DEV), torch.full((L, r, H * d), 3.0, device=DEV),
+                   grouping=kvc.KVC_GROUP_LAYER)
+    ws = torch.zeros(kvc.kvc_workspace_bytes(tgt, st, mode), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(src, tgt, shift, kvc.Rope(cfg.theta), st, mode, workspace=ws)
+    torch.cuda.synchronize()
+    return st, ws
+
+
+CFG_G2 = wl.CONFIGS["llama8b_8k"].scaled(name="8b_H2", L=2, H=2, T=700, r=16)
+CFG_G8 = wl.CONFIGS["llama8b_8k"].scaled(name="8b_H8", L=1, H=8, T=1100)           # D = 1024, r = 32
+CFG_GP = wl.CONFIGS["vlm_16k"].scaled(name="vlm_H4", L=1, H=4, T=901, image_spans=())  # paged, D = 512
+
+
+@pytest.mark.parametrize("cfg", [CFG_G2, CFG_G8, CFG_GP], ids=lambda c: c.name)
+@pytest.mark.parametrize("mode", ["fit", "fit_fast"])
+def test_grouped_fit(cfg, mode):
+    """FIT under D = H d (Sec. 3.1, Eq. 7): the r leading right singular vectors of a layer's concatenated
+    deviation.  Against the oracle's concatenated deviation: eigenvalues from a library routine on its
+    Gram matrix, the leading subspace's projector, orthonormal rows with the sign rule, the Eckart-Young
+    residual of coeff . basis, coefficient columns orthogonal with the eigenvalues as energies."""
+    kmode = kvc.KVC_FIT if mode == "fit" else kvc.KVC_FIT_FAST
+    src_cpu, tgt_cpu, osrc, otgt, ost, shift = _grouped_edge(cfg, cfg.sigma)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    r, D = cfg.r, cfg.H * cfg.d
+    st, ws = _fit_grouped(src, tgt, shift, cfg, r, kmode)
+    assert kvc.kvc_status_poll() == 0
+    assert bool((kvc.kvc_group_fit_solver(tgt, ws) == kvc.KVC_SOLVER_SUBSPACE).all())
+    ev = kvc.kvc_group_fit_eigenvalues(tgt, ws).cpu().numpy().astype(np.float64)
+    f = hp.inv_freq(cfg)
+    for l in range(cfg.L):
+        for i, (which, B_t, c_t) in enumerate((("k", st.basis_k, st.coeff_k), ("v", st.basis_v, st.coeff_v))):
+            cat = np.concatenate([orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, f, which == "k")
+                                  for h in range(cfg.H)], axis=1)                       # [T, H d]
+            G = orc.gram(cat)
+            w, V = np.linalg.eigh(G)
+            w, V = w[::-1], V[:, ::-1]
+            e = ev[l, i]
+            assert np.max(np.abs(e[:r] - w[:r])) <= 2e-4 * w[0]
+            assert np.allclose(e[r:], e[r]) and e[r] <= e[r - 1]
+            assert abs(np.sum(e) - np.sum(w)) <= 2e-4 * np.sum(w)                       # the trace
+            B = B_t[l].cpu().numpy().astype(np.float64)
+            c = c_t[l].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(B @ B.T - np.eye(r))) <= 2e-5
+            assert np.all(B[np.arange(r), np.argmax(np.abs(B), axis=1)] > 0)
+            assert np.linalg.norm(B.T @ B - V[:, :r] @ V[:, :r].T) <= 1e-2
+            tail = float(np.sum(w[r:]))
+            res = float(np.sum((cat - c @ B) ** 2))
+            assert res <= 1.001 * tail + 1e-6 * float(np.sum(w)), (res, tail)
+            Gc = c.T @ c
+            assert np.max(np.abs(Gc - np.diag(np.diag(Gc)))) <= 2e-3 * w[0]
+            assert np.max(np.abs(np.diag(Gc) - w[:r])) <= 1e-3 * w[0]
+            # every row is an eigenvector of the oracle's Gram matrix to the solver's stated level
+            assert np.max(np.linalg.norm(G @ B.T - B.T * np.diag(B @ G @ B.T)[None, :], axis=0)) <= 4e-4 * w[0]
+
+
+@pytest.mark.parametrize("cfg", [CFG_G2, CFG_G8], ids=lambda c: c.name)
+def test_grouped_update_then_apply_round_trip(cfg):
+    """A rank-r deviation across the heads, fitted under grouping and applied again, gives back the
+    target up to the noise floor and the bf16 roundings (the bound of the per-head round trip: the
+    target's own rounding error, large in the outlier channels, is part of the fitted deviation and
+    comes back through the coefficients)."""
+    src_cpu, tgt_cpu, osrc, otgt, ost, shift = _grouped_edge(cfg, cfg.sigma)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    st, ws = _fit_grouped(src, tgt, shift, cfg, cfg.r, kvc.KVC_FIT)
+    assert kvc.kvc_status_poll() == 0
+    dst = hp.empty_dst(src_cpu, cfg, DEV)
+    kvc.kvc_apply(src, st, shift, kvc.Rope(cfg.theta), dst)
+    torch.cuda.synchronize()
+    for which in ("k", "v"):
+        got = orc.bf16_to_f64(hp.logical_bits(dst, which))
+        want = orc.bf16_to_f64(hp.logical_bits(otgt, which))
+        err = np.abs(got - want)
+        assert np.mean(err > 2.0 ** -6 * np.abs(want) + 0.02) < 1e-3
+        assert np.max(err) <= 2.0 ** -4 * np.max(np.abs(want))
+
+
+def test_grouped_fit_without_a_gap_is_flagged_and_zero_is_zero():
+    """A flat spectrum (a Gaussian cache factorised by itself) has no gap behind the r-th eigenvalue: the
+    rows come back orthonormal, the matrix's code names the reason and KVC_FLAG_NOT_CONVERGED is raised
+    (there is no second solver at D = H d).  An all-zero deviation gives a zero state without a flag."""
+    cfg = CFG_G2.scaled(T=400, r=8)
+    src = hp.to_dev(hp.make_cache(cfg), DEV)
+    st, ws = _fit_grouped(None, src, 0, cfg, 8, kvc.KVC_FIT_FAST)
+    codes = kvc.kvc_group_fit_solver(src, ws).cpu().numpy()
+    assert np.all(codes[:, 1] > 0), codes                 # values: no structure at all
+    assert kvc.kvc_status_poll() & kvc.KVC_FLAG_NOT_CONVERGED
+    kvc.kvc_status_reset()
+    B = st.basis_v[0].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(B @ B.T - np.eye(8))) <= 1e-4
+    z = kvc.Cache(torch.zeros_like(src.k), torch.zeros_like(src.v))
+    st, ws = _fit_grouped(None, z, 0, cfg, 8, kvc.KVC_FIT)
+    assert kvc.kvc_status_poll() == 0
+    assert np.all(kvc.kvc_group_fit_solver(z, ws).cpu().numpy() == kvc.KVC_SOLVER_FULL_DEPENDENT)
+    assert torch.all(st.basis_k == 0) and torch.all(st.coeff_v == 0)
+    assert float(kvc.kvc_group_fit_eigenvalues(z, ws).abs().max()) == 0.0
+
+
 def test_grouped_is_rejected_where_it_is_not_served():
     cfg = CFG_S.scaled(T=200)
     st = hp.state_to_dev(_grouped_state(cfg, 1), DEV)
@@ -153,9 +274,10 @@ def test_grouped_is_rejected_where_it_is_not_served():
     with pytest.raises(kvc.KvcError) as e:
         kvc.kvc_gate_distance(src, [st], cfg.T, d2)
     assert e.value.code == kvc.KVC_E_UNSUPPORTED
-    ws = torch.empty(1 << 24, dtype=torch.uint8, device=DEV)
+    ws = torch.empty(1 << 26, dtype=torch.uint8, device=DEV)
+    big = _grouped_state(cfg.scaled(r=64), 1)            # the grouped fit serves r <= 32
     with pytest.raises(kvc.KvcError) as e:
-        kvc.kvc_state_update(None, src, 0, kvc.Rope(cfg.theta), st, kvc.KVC_FIT, workspace=ws)
+        kvc.kvc_state_update(None, src, 0, kvc.Rope(cfg.theta), hp.state_to_dev(big, DEV), kvc.KVC_FIT, workspace=ws)
     assert e.value.code == kvc.KVC_E_UNSUPPORTED
     with pytest.raises(kvc.KvcError) as e:
         kvc.kvc_apply_multi(src, [st], None, None, 0, kvc.Rope(cfg.theta), src, ws)

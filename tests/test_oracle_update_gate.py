@@ -360,3 +360,33 @@ def test_grouped_state_pins():
     assert np.allclose(orc.project_grouped([z[:, h * d:(h + 1) * d] for h in range(H)], Q), ck[0], atol=1e-12)
     # compactness (Sec. 3.1): float32 coefficients of a grouped state take r*4 / (H*d*2) of the bf16 cache
     assert math.isclose((r * 4) / (H * d * 2), 8 / 24)
+
+
+def test_grouped_fit_matches_library_svd():
+    """D = H d fit (Sec. 3.1, Eq. 7): the oracle's grouped basis spans the library SVD's leading right
+    singular subspace of the concatenated deviation, its eigenvalues are the squared singular values,
+    and a deviation built exactly rank r across the heads is reconstructed to rounding.  A per-head
+    fit of the same data does NOT reproduce it (the heads share coefficients only under grouping)."""
+    rng = np.random.default_rng(21)
+    H, T, d, r = 3, 40, 6, 4
+    c = rng.standard_normal((T, r))
+    Q = np.linalg.qr(rng.standard_normal((H * d, r)))[0].T                 # orthonormal rows in R^{H d}
+    cat = c @ Q + 1e-4 * rng.standard_normal((T, H * d))
+    slabs = [cat[:, h * d:(h + 1) * d] for h in range(H)]
+    B, w = orc.fit_grouped(slabs, r)
+    sv = np.linalg.svd(cat, compute_uv=False)
+    assert np.allclose(w[:H * d], sv[:H * d] ** 2 if sv.size >= H * d else np.concatenate([sv ** 2, np.zeros(H * d - sv.size)]),
+                       rtol=1e-9, atol=1e-12)
+    Vt = np.linalg.svd(cat, full_matrices=False)[2][:r]
+    assert np.linalg.norm(B.T @ B - Vt.T @ Vt) <= 1e-8
+    assert np.allclose(B @ B.T, np.eye(r), atol=1e-12)
+    # exactly rank r: reconstructed to rounding, with coefficients shared by the heads
+    exact = c @ Q
+    Be, _ = orc.fit_grouped([exact[:, h * d:(h + 1) * d] for h in range(H)], r)
+    ce = orc.project_grouped([exact[:, h * d:(h + 1) * d] for h in range(H)], Be)
+    assert np.max(np.abs(ce @ Be - exact)) <= 1e-12
+    # per-head rank-r fits of the same data need H sets of coefficients to do the same
+    per_head = [orc.fit_basis(exact[:, h * d:(h + 1) * d], r)[0] for h in range(H)]
+    assert all(np.max(np.abs(orc.project(exact[:, h * d:(h + 1) * d], per_head[h]) @ per_head[h]
+                             - exact[:, h * d:(h + 1) * d])) <= 1e-12 for h in range(H))
+    assert not np.allclose(orc.project(exact[:, :d], per_head[0]), ce)
