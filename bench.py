@@ -208,7 +208,8 @@ def main():
                     help="fast: KVC_FIT_FAST (top-r subspace solver, full eigensolver where it declines); full: KVC_FIT")
     ap.add_argument("--edges", default="chain", choices=["chain", "each"],
                     help="chain: kvc_state_update_chain, all edges in one call; each: one kvc_state_update per edge")
-    ap.add_argument("--grouped", type=int, default=0, help="1: per-layer states (D = H d), with --only apply")
+    ap.add_argument("--grouped", type=int, default=0,
+                    help="1: per-layer states (D = H d): grouped FIT (Gram-free subspace iteration) and grouped chain")
     ap.add_argument("--paged", type=int, default=-1, help="override the layout: 1 paged, 0 contiguous (experiments)")
     ap.add_argument("--only", default="all", choices=["all", "apply", "update", "gate", "multi", "weights"],
                     help="profiling aid: time only the chain or only the state updates")
@@ -243,6 +244,9 @@ def main():
                        f"per edge: kvc_state_update({'FIT_FAST' if args.fit == 'fast' else 'FIT'})") + " ; then kvc_chain over all agents",
               "l2": "inputs larger than L2 (126 MB): no flush between iterations", "parallelism": f"replicas x{world}",
               "only": args.only}
+    if args.grouped:
+        config["grouping"] = ("per layer, D = H d: coefficients [L, T, r] shared by the heads; FIT = 3 applications of "
+                              "Delta^T Delta as projection + back-projection passes, 7 passes over the caches per edge")
 
     if args.impl == "reference":
         if rank != 0:
@@ -282,7 +286,7 @@ def main():
     elif ring:
         W = sc.build_ring(cfg.scaled(seed=cfg.seed + rank), dev)
     else:
-        W = sc.build_workload(cfg.scaled(seed=cfg.seed + rank), dev, args.only, grouped=bool(args.grouped) and args.only == "apply")
+        W = sc.build_workload(cfg.scaled(seed=cfg.seed + rank), dev, args.only, grouped=bool(args.grouped) and args.only in ("apply", "all", "update"))
     W["fit_mode"] = kvc.KVC_FIT_FAST if args.fit == "fast" else kvc.KVC_FIT
     W["edges"] = args.edges
     if args.chain == "fused" and W.get("kind") is None and W.get("outs") and args.only in ("all", "apply"):
@@ -436,6 +440,8 @@ def main():
     # launches (FIT_FAST: subspace solver + full solver for what it declined), once for all edges or per edge
     eig_launches = (2 if args.fit == "fast" else 1) * (1 if args.edges == "chain" else hops)
     upd_launches = 2 * hops + eig_launches
+    if args.grouped:    # per edge: start rows, 3 x (projection, back-projection, small dense step), final projection
+        upd_launches = hops * 20          # + 2 refinement rounds of 4 launches each (they return at once when not needed) + 1
     achieved = (app_b / hops) / (hop_ms * 1e-3) / 1e9
     has_traffic = (not fused_chain and args.workload == "llama8b_8k" and args.layers == 0 and args.rank == 0 and args.paged < 0
                    and args.only not in ("gate", "multi", "weights") and not args.grouped)

@@ -206,14 +206,18 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                eigenvectors of G = Delta^T Delta by three applications of G, each one the grouped
  *                projection pass Z = Delta Q^T followed by a back-projection pass Y = Z^T Delta, with an
  *                orthonormalisation of the r rows in between and a Rayleigh-Ritz step at the end
- *                (a fixed schedule: 7 streaming passes over the two caches with the final projection).
- *                Rows, coefficients and the r leading eigenvalues are as in KVC_FIT_FAST, the acceptance
- *                test likewise with the rows' residual limit at 2e-4 lambda_1 (the passes contract in split
- *                bf16 precision).  There is no second solver behind it: a matrix that fails the test (no
- *                gap behind the r-th eigenvalue) still gets its Ritz rows, its code in kvc_group_fit_solver
- *                says why, and KVC_FLAG_NOT_CONVERGED is raised.  Workspace layout: the eigenvalues
- *                [L, 2, H d] first (kvc_group_fit_eigenvalues; the r leading ones, then the mean of the
- *                rest), the codes [L, 2] (kvc_group_fit_solver), then scratch.
+ *                (7 streaming passes over the two caches with the final projection).  A block that the
+ *                step finds merely slow (its hashed start was unlucky) gets up to two further rounds of
+ *                orthonormalisation, application and Rayleigh-Ritz; their kernels are always launched and
+ *                return at once when the round is not needed (nothing is read back to the host).
+ *                Rows, coefficients and the r leading eigenvalues are as in KVC_FIT_FAST; the acceptance
+ *                test likewise, with the rows' residual limit at 5e-5 lambda_1 and the block's at 1/4096 of
+ *                the gap (the projection pass contracts in split bf16 precision, which bounds what can be
+ *                measured).  There is no second solver behind it: a matrix that still fails the test (no
+ *                gap behind the r-th eigenvalue) gets its Ritz rows all the same, its code in
+ *                kvc_group_fit_solver says why, and KVC_FLAG_NOT_CONVERGED is raised.  Workspace layout: the
+ *                eigenvalues [L, 2, H d] first (kvc_group_fit_eigenvalues; the r leading ones, then the
+ *                mean of the rest), the codes [L, 2] (kvc_group_fit_solver), then scratch.
  *   src == NULL factorises tgt itself (the anchor's base representation, Sec. 3.3).
  *   workspace  DEVICE scratch of at least kvc_workspace_bytes(...) bytes, 256-byte
  *              aligned.  May be NULL when 0 is needed.  After a KVC_FIT / KVC_FIT_FAST call it
@@ -492,7 +496,9 @@ int kvc_set_path(int32_t path);
 int kvc_last_path(void);
 
 /* Algorithmic HBM bytes one hop moves (reads + writes of caches, coefficients and
- * bases), the figure the roofline is reported against. */
+ * bases), the figure the roofline is reported against.  For the FIT modes: two passes over
+ * the source and target rows (one for the Gram matrix, one for the projection), however many
+ * the implementation makes (the layer-grouped fit makes seven). */
 int64_t kvc_apply_bytes(const kvc_cache *src, const kvc_state *st);
 int64_t kvc_update_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mode, int32_t has_src);
 

@@ -306,11 +306,14 @@ static size_t group_ypart_offset(const kvc_cache* tgt) {
 static size_t group_trpart_offset(const kvc_cache* tgt, int r) {
   return group_ypart_offset(tgt) + (size_t)kGroupFitParts * tgt->L * 2 * r * tgt->H * tgt->d * sizeof(float);
 }
+static size_t group_flags_offset(const kvc_cache* tgt, int r) {
+  return (group_trpart_offset(tgt, r) + (size_t)kGroupFitParts * tgt->L * 2 * tgt->H * sizeof(float) + 255) & ~(size_t)255;
+}
 
 size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
   if (!tgt || !st || (mode != KVC_FIT && mode != KVC_FIT_FAST)) return 0;
   if (st->grouping == KVC_GROUP_LAYER)
-    return group_trpart_offset(tgt, st->r) + (size_t)kGroupFitParts * tgt->L * 2 * tgt->H * sizeof(float);
+    return group_flags_offset(tgt, st->r) + 256;
   if (mode == KVC_FIT) return fit_evals_end(tgt);
   return fit_solver_offset(tgt) + (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t);
 }
@@ -416,7 +419,7 @@ static int fit_eig(FitLaunch& F, int32_t mode, int d, int r_eff, size_t solver_o
 }
 
 // Projection pass of one edge (U1 + U4): coefficients of the deviation in the state's bases.
-static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s) {
+static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, const int32_t* run_if = nullptr) {
   const kvc_state* st = P.st;
   const int d = P.d;
   UpdateLaunch U;
@@ -436,6 +439,7 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s) {
   U.H = P.H;
   U.status = status;
   U.grouped = P.dstate.grouped;
+  U.run_if = run_if;
   rope_tables(P.rope, d, P.shift, U.cs, U.sn);
   if (U.grouped) {      // every head adds its share: start from zero
     const size_t nbytes = (size_t)P.L * st->n_cov * st->r * sizeof(float);
@@ -476,6 +480,7 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   G.solver = reinterpret_cast<int32_t*>(ws + group_solver_offset(tgt));
   G.ypart = reinterpret_cast<float*>(ws + group_ypart_offset(tgt));
   G.trpart = reinterpret_cast<float*>(ws + group_trpart_offset(tgt, st->r));
+  G.need_more = reinterpret_cast<int32_t*>(ws + group_flags_offset(tgt, st->r));
   G.r = st->r;
   G.n_cov = st->n_cov;
   G.pairing = P.rope->pairing;
@@ -488,6 +493,8 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   G.tokens_per_part = (per + 31) / 32 * 32;
   G.status = status;
   rope_tables(P.rope, P.d, P.shift, G.cs, G.sn);
+  G.round = 0;
+  G.last_round = kGroupFitRounds;
   if (launch_group_small(G, KVC_GROUP_OP_START, s) != cudaSuccess) return KVC_E_CUDA;
   static const int ops[3] = {KVC_GROUP_OP_ORTH_START, KVC_GROUP_OP_ORTH, KVC_GROUP_OP_RITZ};
   for (int it = 0; it < 3; ++it) {
@@ -495,6 +502,19 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
     if (rc != KVC_OK) return rc;
     if (launch_group_backproject(G, s) != cudaSuccess) return KVC_E_CUDA;
     if (launch_group_small(G, ops[it], s) != cudaSuccess) return KVC_E_CUDA;
+  }
+  // Refinement rounds, for the case that a block was merely slow (the hashed start had a small component
+  // along one leading direction): the rows become orth(G x Ritz rows) - that product is what the
+  // Rayleigh-Ritz step left behind - then one more application of G and a Rayleigh-Ritz step.  Nothing is
+  // read back: a round's kernels are launched regardless and return at once unless the previous
+  // Rayleigh-Ritz step asked for the round.
+  for (int round = 1; round <= kGroupFitRounds; ++round) {
+    G.round = round;
+    if (launch_group_small(G, KVC_GROUP_OP_ORTH_KEEP, s) != cudaSuccess) return KVC_E_CUDA;
+    int rc = project_edge(P, status, s, G.need_more + round);
+    if (rc != KVC_OK) return rc;
+    if (launch_group_backproject(G, s) != cudaSuccess) return KVC_E_CUDA;
+    if (launch_group_small(G, KVC_GROUP_OP_RITZ, s) != cudaSuccess) return KVC_E_CUDA;
   }
   return KVC_OK;
 }
@@ -934,7 +954,10 @@ int64_t kvc_update_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode
   const int64_t coeff = cslabs * st->n_cov * st->r * 4;
   const int64_t basis = slabs * st->r * tgt->d * (st->basis_dtype == KVC_BF16 ? 2 : 4);
   int64_t b = rows + coeff + basis;                                          // projection pass
-  if (mode == KVC_FIT || mode == KVC_FIT_FAST) b += rows + 2 * slabs * tgt->d * tgt->d * 4;          // Gram pass + G write/read
+  if (mode == KVC_FIT || mode == KVC_FIT_FAST) {
+    b += rows;                                                                // a second pass over the rows (Gram)
+    if (st->grouping != KVC_GROUP_LAYER) b += 2 * slabs * tgt->d * tgt->d * 4;  // G written and read (no G under grouping)
+  }
   return b;
 }
 

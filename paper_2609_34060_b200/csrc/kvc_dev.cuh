@@ -63,6 +63,8 @@ struct UpdateLaunch {
   int32_t shift, L, H, tiles_per_slab;
   uint32_t* status;
   int32_t grouped, pad;        // grouped: one state per layer; the heads' projections are ADDED into coeff [L,n_cov,r]
+  const int32_t* run_if;       // DEVICE flag or nullptr: when given and zero, the kernel returns at once (a pass
+                               // of the grouped fit's refinement rounds that turned out not to be needed)
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];
 };
@@ -99,15 +101,19 @@ struct GroupFitLaunch {        // FIT of states grouped by layer (D = H d): back
   float* trpart;               // [parts][L*2][H] partial sums of Delta^2
   float* evals;                // [L*2][H d]
   int32_t* solver;             // [L*2] per-problem code
-  int32_t r, n_cov, pairing, shift, L, H, d, parts, tokens_per_part, pad;
+  int32_t* need_more;          // [kGroupFitRounds + 1]: round k runs only when need_more[k] != 0 (round 0 always)
+  int32_t r, n_cov, pairing, shift, L, H, d, parts, tokens_per_part;
+  int32_t round, last_round, pad;
   uint32_t* status;
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];
 };
+constexpr int kGroupFitRounds = 2;          // refinement rounds (one more application of G each) after the fixed schedule
 constexpr int KVC_GROUP_OP_START = 0;       // hashed start rows
 constexpr int KVC_GROUP_OP_ORTH_START = 1;  // rows <- orth(back-projection), conditioning unknown
 constexpr int KVC_GROUP_OP_ORTH = 2;        // rows <- orth(back-projection)
 constexpr int KVC_GROUP_OP_RITZ = 3;        // Rayleigh-Ritz, acceptance, output
+constexpr int KVC_GROUP_OP_ORTH_KEEP = 4;   // rows <- orth(G x Ritz rows), which the Rayleigh-Ritz step left in place
 
 struct GateLaunch {            // Eq. 9 for one anchor, CUDA-core kernel
   DevCache src;                // values only

@@ -144,6 +144,7 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
 // ---------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256) project_generic_kernel(const __grid_constant__ UpdateLaunch p) {
+  if (p.run_if != nullptr && *p.run_if == 0) return;
   constexpr int LPT = D / 16;
   constexpr int TILE = 64;
   constexpr int QC = 32;

@@ -46,6 +46,7 @@ __global__ void __launch_bounds__(256) group_backproject_kernel(const __grid_con
   __shared__ __align__(16) float delta_s[kTT * D];
   __shared__ __align__(16) float z_s[kTT * kMaxM];
   __shared__ float red[8];
+  if (p.round > 0 && p.need_more[p.round] == 0) return;       // a refinement round nobody asked for
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   int b = blockIdx.x;
   const int part = b % p.parts;
@@ -240,6 +241,7 @@ __device__ __forceinline__ void solve_rows(const float* A, float* Dst, const flo
 __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_constant__ GroupFitLaunch p, int op) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SmallMem& sm = *reinterpret_cast<SmallMem*>(smem_raw);
+  if (p.round > 0 && p.need_more[p.round] == 0) return;       // a refinement round nobody asked for
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int prob = blockIdx.x;                    // l * 2 + is_v
   const int l = prob >> 1, is_v = prob & 1;
@@ -254,20 +256,25 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
       const int q = (int)(i / Dg), c = (int)(i - (int64_t)q * Dg);
       Q[i] = (q < m) ? start_value(c, q) : 0.f;
     }
-    if (tid == 0) *code = 0;
+    if (tid == 0) {
+      *code = 0;
+      if (prob == 0)
+        for (int k = 0; k <= kGroupFitRounds; ++k) p.need_more[k] = 0;
+    }
     return;
   }
 
   // the partial sums of the back-projection, added in a fixed order
+  if (op != KVC_GROUP_OP_ORTH_KEEP)
   for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) {
     float a = Y[i];
     for (int part = 1; part < p.parts; ++part) a += p.ypart[((int64_t)part * p.L * 2 + prob) * p.r * Dg + i];
     Y[i] = a;
   }
   __syncthreads();
-  if (*code != 0 && op != KVC_GROUP_OP_RITZ) return;   // given up earlier: nothing to orthonormalise
+  if (*code == KVC_SOLVER_FULL_DEPENDENT && op != KVC_GROUP_OP_RITZ) return;   // given up earlier: nothing to orthonormalise
 
-  if (op == KVC_GROUP_OP_ORTH || op == KVC_GROUP_OP_ORTH_START) {
+  if (op == KVC_GROUP_OP_ORTH || op == KVC_GROUP_OP_ORTH_START || op == KVC_GROUP_OP_ORTH_KEEP) {
     // Cholesky QR on the rows of Y: a shifted pass first where the conditioning is unknown (the
     // hashed start block after one product), then plain passes; the result becomes Q
     const int passes = (op == KVC_GROUP_OP_ORTH_START) ? 3 : 2;
@@ -290,7 +297,7 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
   for (int part = 0; part < p.parts; ++part)
     for (int h = 0; h < p.H; ++h) tr += p.trpart[((int64_t)part * p.L * 2 + prob) * p.H + h];
   float* evals = p.evals + (int64_t)prob * Dg;
-  if (*code != 0 || !(tr > 0.f)) {
+  if (*code == KVC_SOLVER_FULL_DEPENDENT || !(tr > 0.f)) {
     // a zero deviation (or rows that became dependent): no basis, all eigenvalues zero
     for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) Q[i] = 0.f;
     for (int i = tid; i < Dg; i += kThreads) evals[i] = 0.f;
@@ -434,14 +441,19 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
   const float tau = fmaxf(tr - sumth, 0.f);
   const float rhoF = sqrtf(rhoF2);
   const float gap = thm - tau - rhoF;
-  // The products run through the split-precision projection pass (about 2e-5 of a row's length), so the
-  // rows' residuals are held to 2e-4 of the largest eigenvalue; the gap test is the per-head solver's.
-  const bool accept = rhomax2 <= (2e-4f * th1) * (2e-4f * th1) && gap > 0.f && rhoF <= (1.f / 1024.f) * gap;
+  // The projection pass contracts in split bf16 precision (a few 1e-5 of a coefficient's size), which
+  // bounds what a residual can be measured to: converged blocks show about 4e-6 lambda_1 per row on keys
+  // with outlier channels.  Rows are held to 5e-5 lambda_1, the block to 1/4096 of the gap.
+  const bool accept = rhomax2 <= (5e-5f * th1) * (5e-5f * th1) && gap > 0.f && rhoF <= (1.f / 4096.f) * gap;
   if (reason == 0 && !accept) reason = (gap > 0.f) ? KVC_SOLVER_FULL_SLOW : KVC_SOLVER_FULL_NO_GAP;
   for (int i = tid; i < Dg; i += kThreads) evals[i] = (i < m) ? sm.th[i] : (Dg > m ? tau / (float)(Dg - m) : 0.f);
   if (tid == 0) {
     *code = reason;
-    if (reason != 0) atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
+    // a block that is only slow (there is a gap) gets another application of G while rounds are left
+    if (reason == KVC_SOLVER_FULL_SLOW && p.round < p.last_round)
+      p.need_more[p.round + 1] = 1;
+    else if (reason != 0)
+      atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
   }
 }
 

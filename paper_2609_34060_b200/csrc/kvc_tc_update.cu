@@ -140,6 +140,7 @@ __device__ __forceinline__ void tile_issue(const DevCache& c, const CUtensorMap*
 // RB = rank blocks of 32 (accumulator columns = 32 RB), NS = stages
 template <int RB, int NS>
 __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_constant__ ProjectTcLaunch p) {
+  if (p.u.run_if != nullptr && *p.u.run_if == 0) return;      // uniform over the grid: nothing has been set up yet
   constexpr int RN = 32 * RB;
   constexpr int kBlk = RN * 128;                 // RN basis rows x 64 channels, bf16
   constexpr int kSlotBytes = 8 * kBlk;           // {B, Bs} x {hi, lo} x {channels 0-63, 64-127}

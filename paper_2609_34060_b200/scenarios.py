@@ -33,17 +33,18 @@ def build_workload(cfg: wl.Config, dev, only="all", grouped=False):
         tables = [None] * (2 * n)
         a0 = kvc.Cache(k0, v0)
     true = [a0]
+
+    def drawn_state(a):
+        if grouped:     # one state per layer over all KV heads (D = H d): coeff [L,T,r], basis [L,r,H d]
+            mkc = lambda tag: wl.coefficients(cfg.L, 1, cfg.T, cfg.r, cfg.seed, 4 * a + tag, dev)[:, 0].contiguous()
+            mkb = lambda tag: wl.orthonormal_basis(cfg.L, 1, cfg.r, cfg.H * cfg.d, cfg.seed, 4 * a + tag, dev)[:, 0].contiguous()
+            return kvc.State(mkc(0), mkc(1), mkb(2), mkb(3), grouping=kvc.KVC_GROUP_LAYER)
+        s = wl.hop_state(cfg, a, dev)
+        return kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"])
+
     if only in ("apply", "gate", "multi", "weights"):
         # the chain (or the gate) alone: the generator's states are used directly, no targets needed
-        states = []
-        for a in range(1, n):
-            if grouped:     # one state per layer over all KV heads (D = H d): coeff [L,T,r], basis [L,r,H d]
-                mkc = lambda tag: wl.coefficients(cfg.L, 1, cfg.T, cfg.r, cfg.seed, 4 * a + tag, dev)[:, 0].contiguous()
-                mkb = lambda tag: wl.orthonormal_basis(cfg.L, 1, cfg.r, cfg.H * cfg.d, cfg.seed, 4 * a + tag, dev)[:, 0].contiguous()
-                states.append(kvc.State(mkc(0), mkc(1), mkb(2), mkb(3), grouping=kvc.KVC_GROUP_LAYER))
-                continue
-            s = wl.hop_state(cfg, a, dev)
-            states.append(kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"]))
+        states = [drawn_state(a) for a in range(1, n)]
         if only == "gate":
             # the reliability gate over a pool whose anchors are the hop states' value factors
             f64 = lambda m: torch.empty(m, dtype=torch.float64, device=dev)
@@ -68,8 +69,7 @@ def build_workload(cfg: wl.Config, dev, only="all", grouped=False):
         outs = [mk(tables[n + a]) for a in range(1, n)]
         return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": None, "only": only}
     for a in range(1, n):
-        s = wl.hop_state(cfg, a, dev)
-        st = kvc.State(s["coeff_k"], s["coeff_v"], s["basis_k"], s["basis_v"])
+        st = drawn_state(a)
         tgt = mk(tables[a])
         kvc.kvc_apply(true[-1], st, pl[a] - pl[a - 1], rope, tgt)
         for t, tag in ((tgt.k, 0), (tgt.v, 1)):      # noise below one bf16 step mostly dithers the rounding
@@ -81,11 +81,16 @@ def build_workload(cfg: wl.Config, dev, only="all", grouped=False):
                 seg = flat[o:o + chunk]
                 seg.copy_((seg.float() + cfg.sigma * torch.randn(seg.numel(), device=dev, generator=g)).to(torch.bfloat16))
         true.append(tgt)
-        del s, st
+        del st
     torch.cuda.synchronize()
     L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
-    states = [kvc.State(torch.empty(L, H, T, r, device=dev), torch.empty(L, H, T, r, device=dev),
-                        torch.empty(L, H, r, d, device=dev), torch.empty(L, H, r, d, device=dev)) for _ in range(n - 1)]
+    if grouped:
+        states = [kvc.State(torch.empty(L, T, r, device=dev), torch.empty(L, T, r, device=dev),
+                            torch.empty(L, r, H * d, device=dev), torch.empty(L, r, H * d, device=dev),
+                            grouping=kvc.KVC_GROUP_LAYER) for _ in range(n - 1)]
+    else:
+        states = [kvc.State(torch.empty(L, H, T, r, device=dev), torch.empty(L, H, T, r, device=dev),
+                            torch.empty(L, H, r, d, device=dev), torch.empty(L, H, r, d, device=dev)) for _ in range(n - 1)]
     outs = [mk(tables[n + a]) for a in range(1, n)]
     ws = torch.empty(max(kvc.kvc_chain_update_workspace_bytes(true, states, kvc.KVC_FIT_FAST), 256), dtype=torch.uint8, device=dev)
     return {"rope": rope, "pl": pl, "true": true, "states": states, "outs": outs, "ws": ws, "only": only}

@@ -134,8 +134,14 @@ def test_multi_anchor_and_grouping_argument_errors(lib):
     assert lib.kvc_apply(C.byref(src), C.byref(bad), 0, C.byref(rope), C.byref(dst), None) == -1
     grouped = _state()
     grouped.grouping = kvc.KVC_GROUP_LAYER
-    # per-layer states are not served by the fit, the gate and the multi-anchor apply
-    assert lib.kvc_state_update(None, C.byref(src), 0, C.byref(rope), C.byref(grouped), kvc.KVC_FIT, 0x7000100, 1 << 30, None) == -3
+    # per-layer states: the fit serves ranks up to 32 (and wants its own, larger workspace); the gate and
+    # the multi-anchor apply do not serve them
+    wide = _state(r=40)
+    wide.grouping = kvc.KVC_GROUP_LAYER
+    assert lib.kvc_state_update(None, C.byref(src), 0, C.byref(rope), C.byref(wide), kvc.KVC_FIT, 0x7000100, 1 << 30, None) == -3
+    need = lib.kvc_workspace_bytes(C.byref(src), C.byref(grouped), kvc.KVC_FIT)
+    assert need >= 4 * src.L * 2 * (src.H * src.d) * (1 + 4 * grouped.r)       # eigenvalues + four partial back-projections
+    assert lib.kvc_state_update(None, C.byref(src), 0, C.byref(rope), C.byref(grouped), kvc.KVC_FIT, 0x7000100, need - 1, None) == kvc.KVC_E_WORKSPACE
     assert lib.kvc_gate_distance(C.byref(src), C.byref(grouped), 1, 8, 0x8000000, None) == -3
     assert lib.kvc_apply_multi(C.byref(src), C.byref(grouped), 1, None, None, 0, C.byref(rope), C.byref(dst), 0x9000000, 1 << 30, None) == -3
     # byte accounting of a grouped state: the coefficients are shared by the heads
