@@ -275,6 +275,45 @@ size_t kvc_chain_update_workspace_bytes(const kvc_cache *agents, int32_t n_agent
 size_t kvc_chain_update_edge_stride(const kvc_cache *tgt, const kvc_state *st, int32_t mode);
 
 /*
+ * Multi-segment contexts (Eq. 1; App. A.2).  A trajectory interleaves agent-specific pieces with the
+ * shared ones, so between two agents the shared tokens are displaced by an amount that is constant
+ * inside a segment and changes from one segment to the next.  A segment list gives every token range
+ * its own shift; one call then serves the whole context (no splitting into one call, and for paged
+ * caches one page-aligned table slice, per segment).  Segment boundaries need not fall on pages or tiles.
+ *   n        1 .. KVC_MAX_SEGMENTS
+ *   t_begin  HOST int32 [n], ascending, t_begin[0] == 0: segment j covers tokens t_begin[j] .. t_begin[j+1]-1,
+ *            the last one runs to T
+ *   shift    HOST int32 [n]
+ *   coords   where the low-rank correction lives:
+ *            KVC_COORDS_TARGET  at the target's positions, as Eq. 12 measures it:
+ *                               K_dst = Rot_s(K_src) + c . B ,   Delta = K_tgt - Rot_s(K_src)
+ *            KVC_COORDS_SOURCE  at the source's positions (the canonical-coordinate form of App. A.2: the
+ *                               correction is stored once and moves with the token it corrects):
+ *                               K_dst = Rot_s(K_src + c . B) ,   Delta = Rot_{-s}(K_tgt) - K_src
+ *            With one shift for all tokens, SOURCE coordinates equal TARGET coordinates with the key basis
+ *            rotated by kvc_state_realign; with several shifts only SOURCE coordinates keep one basis.
+ *            Values are never rotated: the two agree for them.
+ * The lists are host arrays on purpose: the cos / sin tables of every segment are formed in float64 on the
+ * host, exactly like the single shift's, and travel in the launch parameters (a device position array would
+ * need sincos per token and frequency inside the kernels).  These entry points are served by the CUDA-core
+ * kernel family (KVC_PATH_TC forced: KVC_E_UNSUPPORTED); everything else is as in kvc_apply / kvc_state_update,
+ * including layer-grouped states and the FIT modes.
+ */
+#define KVC_MAX_SEGMENTS   16
+#define KVC_COORDS_TARGET  0
+#define KVC_COORDS_SOURCE  1
+typedef struct kvc_segments {
+  int32_t n;
+  const int32_t *t_begin;
+  const int32_t *shift;
+  int32_t coords;
+} kvc_segments;
+int kvc_apply_segmented(const kvc_cache *src, const kvc_state *st, const kvc_segments *segs, const kvc_rope *rope,
+                        kvc_cache *dst, void *stream);
+int kvc_state_update_segmented(const kvc_cache *src, const kvc_cache *tgt, const kvc_segments *segs, const kvc_rope *rope,
+                               kvc_state *st, int32_t mode, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * kvc_state_update_noalloc -- kvc_state_update without a workspace argument.
  * (No counterpart in the paper: this exists for integration only.)
  *

@@ -505,6 +505,86 @@ def fit_grouped(delta_slabs, r):
     return fit_basis(cat, r)
 
 
+# --------------------------------------------------------------------------
+# Multi-segment contexts (Eq. 1): a trajectory interleaves agent-specific pieces with the shared ones,
+# so the shared tokens of two agents differ by a shift that is constant inside a segment and changes
+# from segment to segment.
+# --------------------------------------------------------------------------
+COORDS_TARGET = 0   # the correction lives at the target's positions: C_hat = Rot_s(src) + c . B      (Eq. 12)
+COORDS_SOURCE = 1   # the correction lives at the source's positions: C_hat = Rot_s(src + c . B)      (App. A.2)
+
+
+def segment_shifts(T, t_begin, shift):
+    """Per-token shift vector [T] of a piecewise-constant shift: segment j covers tokens
+    t_begin[j] .. t_begin[j+1] - 1 (the last one runs to T) and is shifted by shift[j]."""
+    t_begin, shift = list(t_begin), list(shift)
+    assert len(t_begin) == len(shift) and (not t_begin or t_begin[0] == 0)
+    out = np.zeros(T, dtype=np.int64)
+    for j, t0 in enumerate(t_begin):
+        t1 = t_begin[j + 1] if j + 1 < len(t_begin) else T
+        assert t0 <= t1
+        out[t0:t1] = shift[j]
+    return out
+
+
+def rope_shift_tokens(x, s_tok, inv_freq, pairing=ROPE_HALF):
+    """rope_shift with one shift per token: row t of x [T, d] is rotated by s_tok[t] * f_k.
+    Rows whose shift is 0 are returned untouched."""
+    x = np.asarray(x, dtype=np.float64)
+    s_tok = np.asarray(s_tok, dtype=np.int64)
+    T, d = x.shape
+    a = s_tok.astype(np.float64)[:, None] * np.asarray(inv_freq, dtype=np.float64)[None, :]   # [T, d/2]
+    c, sn = np.cos(a), np.sin(a)
+    y = np.empty_like(x)
+    if pairing == ROPE_HALF:
+        x1, x2 = x[:, : d // 2], x[:, d // 2:]
+        y[:, : d // 2] = x1 * c - x2 * sn
+        y[:, d // 2:] = x1 * sn + x2 * c
+    else:
+        x1, x2 = x[:, 0::2], x[:, 1::2]
+        y[:, 0::2] = x1 * c - x2 * sn
+        y[:, 1::2] = x1 * sn + x2 * c
+    still = s_tok == 0
+    y[still] = x[still]
+    return y
+
+
+def apply_slab_tokens(src_bits, coeff, basis, s_tok, inv_freq, n_cov, is_key, pairing=ROPE_HALF, coords=COORDS_TARGET):
+    """apply_slab with a per-token shift vector and the choice of the correction's coordinates.
+    TARGET: ref = Rot_s(src) + c . B;  SOURCE: ref = Rot_s(src + c . B).  Values are never rotated, so
+    for them the two agree.  Rows that are neither covered nor shifted keep their bits."""
+    x = bf16_to_f64(src_bits)
+    T = x.shape[0]
+    s_tok = np.asarray(s_tok, dtype=np.int64) if is_key else np.zeros(T, dtype=np.int64)
+    r = 0 if basis is None else int(np.asarray(basis).shape[0])
+    n = min(int(n_cov), T) if r > 0 else 0
+    corr = np.zeros_like(x)
+    if n > 0:
+        corr[:n] = np.asarray(coeff[:n], dtype=np.float64) @ np.asarray(basis, dtype=np.float64)
+    if coords == COORDS_SOURCE:
+        ref = rope_shift_tokens(x + corr, s_tok, inv_freq, pairing)
+    else:
+        ref = rope_shift_tokens(x, s_tok, inv_freq, pairing) + corr
+    out = f64_to_bf16_bits(ref)
+    keep = (s_tok == 0) & (np.arange(T) >= n)
+    out[keep] = src_bits[keep]
+    return ref, out
+
+
+def deviation_tokens(src_bits, tgt_bits, s_tok, inv_freq, is_key, pairing=ROPE_HALF, coords=COORDS_TARGET):
+    """The deviation a state is fitted to, with per-token shifts.  TARGET: tgt - Rot_s(src) (Eq. 12);
+    SOURCE: Rot_{-s}(tgt) - src, the same deviation carried back to the source's positions."""
+    tgt = bf16_to_f64(tgt_bits)
+    if src_bits is None:
+        return tgt
+    src = bf16_to_f64(src_bits)
+    T = src.shape[0]
+    s_tok = np.asarray(s_tok, dtype=np.int64) if is_key else np.zeros(T, dtype=np.int64)
+    if coords == COORDS_SOURCE:
+        return rope_shift_tokens(tgt, -s_tok, inv_freq, pairing) - src
+    return tgt - rope_shift_tokens(src, s_tok, inv_freq, pairing)
+
+
 def realign_basis(basis_k, s, inv_freq, pairing=ROPE_HALF):
     """App. A.2 (PF-induced deltas): a stored key correction is "positionally re-aligned when reused".
     A rotation acts on the channel axis and is linear, so Rot_s(c . B) = c . Rot_s(B): re-aligning a

@@ -24,6 +24,7 @@ KVC_PROJECT, KVC_FIT, KVC_FIT_FAST = 0, 1, 2
 (KVC_SOLVER_SUBSPACE, KVC_SOLVER_FULL_RANK, KVC_SOLVER_FULL_DEPENDENT, KVC_SOLVER_FULL_SLOW, KVC_SOLVER_FULL_NO_GAP,
  KVC_SOLVER_FULL_SWEEPS) = (0, -1, 2, 3, 4, 5)
 KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
+KVC_MAX_SEGMENTS, KVC_COORDS_TARGET, KVC_COORDS_SOURCE = 16, 0, 1
 KVC_GROUP_HEAD, KVC_GROUP_LAYER = 0, 1
 KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4
 KVC_OK = 0
@@ -35,7 +36,7 @@ EXPORTS = (
     "kvc_batch_workspace_bytes", "kvc_status_poll", "kvc_status_reset", "kvc_set_path", "kvc_last_path",
     "kvc_apply_bytes", "kvc_update_bytes", "kvc_strerror", "kvc_version", "kvc_gate_distance", "kvc_gate_weights",
     "kvc_apply_multi", "kvc_multi_workspace_bytes", "kvc_token_weights", "kvc_token_weights_workspace_bytes",
-    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_group_fit_eigenvalues", "kvc_group_fit_solver", "kvc_selftest_wait_expiry", "kvc_state_update_check", "kvc_state_update_chain",
+    "kvc_state_realign", "kvc_effective_rank", "kvc_fit_eigenvalues", "kvc_fit_solver", "kvc_group_fit_eigenvalues", "kvc_group_fit_solver", "kvc_selftest_wait_expiry", "kvc_apply_segmented", "kvc_state_update_segmented", "kvc_state_update_check", "kvc_state_update_chain",
     "kvc_chain_update_workspace_bytes", "kvc_chain_update_edge_stride", "kvc_chain_fused", "kvc_chain_workspace_bytes",
 )
 
@@ -60,6 +61,10 @@ class kvc_state(C.Structure):
 
 class kvc_rope(C.Structure):
     _fields_ = [("theta", C.c_double), ("pairing", C.c_int32), ("reserved", C.c_int32), ("inv_freq", C.c_void_p)]
+
+
+class kvc_segments(C.Structure):
+    _fields_ = [("n", C.c_int32), ("t_begin", C.POINTER(C.c_int32)), ("shift", C.POINTER(C.c_int32)), ("coords", C.c_int32)]
 
 
 class kvc_item(C.Structure):
@@ -89,6 +94,9 @@ def load(path: Optional[str] = None):
     lib.kvc_state_update.argtypes = [PC, PC, i32, PR, PS, i32, vp, sz, vp]
     lib.kvc_state_update_noalloc.argtypes = [PC, PC, i32, PR, PS, i32, vp]
     lib.kvc_selftest_wait_expiry.argtypes = [C.c_double, C.POINTER(i32), vp]
+    PSeg = C.POINTER(kvc_segments)
+    lib.kvc_apply_segmented.argtypes = [PC, PS, PSeg, PR, PC, vp]
+    lib.kvc_state_update_segmented.argtypes = [PC, PC, PSeg, PR, PS, i32, vp, sz, vp]
     lib.kvc_state_update_check.argtypes = [PC, PC, i32, PR, PS, i32]
     lib.kvc_state_update_chain.argtypes = [PC, i32, C.POINTER(i32), PR, PS, i32, vp, sz, vp]
     lib.kvc_chain_update_workspace_bytes.argtypes = [PC, i32, PS, i32]
@@ -294,6 +302,40 @@ def kvc_chain_fused(agent0: Cache, prefix_len: Sequence[int], states: Sequence[S
     os_ = (kvc_cache * max(n - 1, 1))(*[o.struct() for o in outs])
     _check(load().kvc_chain_fused(C.byref(a0), n, pl, sts, C.byref(r), os_, workspace.data_ptr(),
                                   workspace.numel() * workspace.element_size(), _stream(stream)), "kvc_chain_fused")
+
+
+class Segments:
+    """Piecewise-constant shifts over the token axis: segment j covers t_begin[j] .. t_begin[j+1]-1."""
+
+    def __init__(self, t_begin: Sequence[int], shift: Sequence[int], coords: int = KVC_COORDS_TARGET):
+        assert len(t_begin) == len(shift)
+        self.t_begin, self.shift, self.coords = [int(x) for x in t_begin], [int(x) for x in shift], int(coords)
+        self._tb = (C.c_int32 * len(self.t_begin))(*self.t_begin)
+        self._sh = (C.c_int32 * len(self.shift))(*self.shift)
+
+    def struct(self) -> kvc_segments:
+        s = kvc_segments()
+        s.n, s.t_begin, s.shift, s.coords = len(self.t_begin), self._tb, self._sh, self.coords
+        return s
+
+
+def kvc_apply_segmented(src: Cache, st: State, segs: Segments, rope: Rope, dst: Cache, stream=None) -> None:
+    s, d, t, r, g = src.struct(), dst.struct(), st.struct(), rope.struct(), segs.struct()
+    _check(load().kvc_apply_segmented(C.byref(s), C.byref(t), C.byref(g), C.byref(r), C.byref(d), _stream(stream)),
+           "kvc_apply_segmented")
+
+
+def kvc_state_update_segmented(src: Optional[Cache], tgt: Cache, segs: Segments, rope: Rope, st: State, mode: int,
+                               workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    t, s, r, g = tgt.struct(), st.struct(), rope.struct(), segs.struct()
+    sp = None
+    if src is not None:
+        ss = src.struct()
+        sp = C.byref(ss)
+    ws_ptr = 0 if workspace is None else workspace.data_ptr()
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().kvc_state_update_segmented(sp, C.byref(t), C.byref(g), C.byref(r), C.byref(s), int(mode), ws_ptr, ws_bytes,
+                                             _stream(stream)), "kvc_state_update_segmented")
 
 
 def kvc_selftest_wait_expiry(limit_ms: float = 1.0, stream=None):

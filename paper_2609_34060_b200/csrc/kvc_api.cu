@@ -153,6 +153,26 @@ static int alias_check(const kvc_cache* src, const DevCache& ds, const kvc_cache
   return KVC_OK;
 }
 
+// Validate a segment list and resolve it into the kernels' table (cos / sin per segment from float64).
+static int resolve_segments(const kvc_segments* segs, const kvc_rope* rope, int d, int T, SegTable* out) {
+  memset(out, 0, sizeof(*out));
+  if (!segs || segs->n < 1 || segs->n > KVC_MAX_SEGMENTS || !segs->t_begin || !segs->shift) return KVC_E_INVALID_ARG;
+  if (segs->coords != KVC_COORDS_TARGET && segs->coords != KVC_COORDS_SOURCE) return KVC_E_INVALID_ARG;
+  if (segs->t_begin[0] != 0) return KVC_E_INVALID_ARG;
+  for (int j = 1; j < segs->n; ++j)
+    if (segs->t_begin[j] < segs->t_begin[j - 1] || segs->t_begin[j] > T) return KVC_E_INVALID_ARG;
+  int rc = check_rope(rope);
+  if (rc != KVC_OK) return rc;
+  out->n = segs->n;
+  out->coords = segs->coords;
+  for (int j = 0; j < segs->n; ++j) {
+    out->t_begin[j] = segs->t_begin[j];
+    out->shifted[j] = segs->shift[j] != 0;
+    rope_tables(rope, d, segs->shift[j], out->cs[j], out->sn[j]);
+  }
+  return KVC_OK;
+}
+
 struct ResolvedHop {
   DevItem item;
   int d;
@@ -177,12 +197,13 @@ static int resolve_hop(const kvc_cache* src, const kvc_state* st, int32_t shift,
   return KVC_OK;
 }
 
-static int apply_resolved(ResolvedHop& hop, int pairing, cudaStream_t s) {
+static int apply_resolved(ResolvedHop& hop, int pairing, cudaStream_t s, const SegTable* seg = nullptr) {
   uint32_t* status = status_ptr();
   if (!status) return KVC_E_CUDA;
   const int T = hop.item.src.T;
   if (T == 0) return KVC_OK;
-  const bool want_tc = tl_path_force != KVC_PATH_GENERIC;
+  if (seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;   // segment tables: CUDA-core kernels only
+  const bool want_tc = tl_path_force != KVC_PATH_GENERIC && !seg;
   if (want_tc) {
     const int trc = tc_apply_single(hop.item, hop.d, pairing, status, s);
     if (trc == KVC_OK) {
@@ -202,6 +223,7 @@ static int apply_resolved(ResolvedHop& hop, int pairing, cudaStream_t s) {
   L.total_tiles = (int64_t)hop.item.L * hop.item.H * 2 * hop.item.tiles_per_slab;
   L.status = status;
   L.one = hop.item;
+  if (seg) L.seg = *seg;
   if (launch_apply_generic(L, hop.d, s) != cudaSuccess) return KVC_E_CUDA;
   tl_last_path = KVC_PATH_GENERIC;
   return KVC_OK;
@@ -219,6 +241,18 @@ int kvc_apply(const kvc_cache* src, const kvc_state* st, int32_t shift, const kv
   const int rc = resolve_hop(src, st, shift, rope, dst, &hop);
   if (rc != KVC_OK) return rc;
   return apply_resolved(hop, rope->pairing, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int kvc_apply_segmented(const kvc_cache* src, const kvc_state* st, const kvc_segments* segs, const kvc_rope* rope,
+                        kvc_cache* dst, void* stream) {
+  if (!src || !segs) return KVC_E_INVALID_ARG;
+  SegTable seg;
+  int rc = resolve_segments(segs, rope, src->d, src->T, &seg);
+  if (rc != KVC_OK) return rc;
+  ResolvedHop hop;
+  if ((rc = resolve_hop(src, st, segs->shift[0], rope, dst, &hop)) != KVC_OK) return rc;
+  if (st && st->grouping == KVC_GROUP_LAYER && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
+  return apply_resolved(hop, rope->pairing, reinterpret_cast<cudaStream_t>(stream), &seg);
 }
 
 int kvc_chain(const kvc_cache* agent0, int32_t n_agents, const int32_t* prefix_len, const kvc_state* states,
@@ -326,6 +360,7 @@ struct UpdatePlan {
   const kvc_rope* rope;
   int32_t shift, mode, L, H, d;
   bool fit, empty;
+  const SegTable* seg;         // per-segment shifts / source coordinates, or nullptr: the CUDA-core kernels serve them
 };
 
 // Every argument check of kvc_state_update except the workspace; launches nothing.
@@ -391,7 +426,7 @@ static int fit_gram(const UpdatePlan& P, void* workspace, uint32_t* status, FitL
   F.H = P.H;
   F.status = status;
   rope_tables(P.rope, P.d, P.shift, F.cs, F.sn);
-  if (tl_path_force != KVC_PATH_GENERIC) {
+  if (tl_path_force != KVC_PATH_GENERIC && !P.seg) {
     const int trc = tc_gram(F, P.d, s);
     if (trc == KVC_OK) {
       F.n_parts = 2;
@@ -399,7 +434,8 @@ static int fit_gram(const UpdatePlan& P, void* workspace, uint32_t* status, FitL
     }
     if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
   }
-  return launch_gram_generic(F, P.d, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+  if (P.seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
+  return launch_gram_generic(F, P.seg, P.d, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
 // Eigensolves of the F.n_edges edges that F describes (same geometry, r, n_cov and partial count).
@@ -446,7 +482,8 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, c
     if (cudaMemsetAsync(st->coeff_k, 0, nbytes, s) != cudaSuccess || cudaMemsetAsync(st->coeff_v, 0, nbytes, s) != cudaSuccess)
       return KVC_E_CUDA;
   }
-  if (tl_path_force != KVC_PATH_GENERIC) {
+  if (P.seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
+  if (tl_path_force != KVC_PATH_GENERIC && !P.seg) {
     const int trc = tc_project(U, d, s);
     if (trc == KVC_OK) {
       tl_last_path = KVC_PATH_TC;
@@ -456,7 +493,7 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, c
   }
   U.tiles_per_slab = (st->n_cov + kGenericProjectTile - 1) / kGenericProjectTile;
   const int64_t tiles = (int64_t)P.L * P.H * 2 * U.tiles_per_slab;
-  if (launch_project_generic(U, d, tiles, s) != cudaSuccess) return KVC_E_CUDA;
+  if (launch_project_generic(U, P.seg, d, tiles, s) != cudaSuccess) return KVC_E_CUDA;
   tl_last_path = KVC_PATH_GENERIC;
   return KVC_OK;
 }
@@ -500,7 +537,7 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   for (int it = 0; it < 3; ++it) {
     int rc = project_edge(P, status, s);
     if (rc != KVC_OK) return rc;
-    if (launch_group_backproject(G, s) != cudaSuccess) return KVC_E_CUDA;
+    if (launch_group_backproject(G, P.seg, s) != cudaSuccess) return KVC_E_CUDA;
     if (launch_group_small(G, ops[it], s) != cudaSuccess) return KVC_E_CUDA;
   }
   // Refinement rounds, for the case that a block was merely slow (the hashed start had a small component
@@ -513,17 +550,38 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
     if (launch_group_small(G, KVC_GROUP_OP_ORTH_KEEP, s) != cudaSuccess) return KVC_E_CUDA;
     int rc = project_edge(P, status, s, G.need_more + round);
     if (rc != KVC_OK) return rc;
-    if (launch_group_backproject(G, s) != cudaSuccess) return KVC_E_CUDA;
+    if (launch_group_backproject(G, P.seg, s) != cudaSuccess) return KVC_E_CUDA;
     if (launch_group_small(G, KVC_GROUP_OP_RITZ, s) != cudaSuccess) return KVC_E_CUDA;
   }
   return KVC_OK;
 }
+
+static int update_planned(UpdatePlan& P, const kvc_cache* tgt, kvc_state* st, int32_t mode, void* workspace,
+                          size_t workspace_bytes, void* stream);
 
 int kvc_state_update(const kvc_cache* src, const kvc_cache* tgt, int32_t shift, const kvc_rope* rope, kvc_state* st,
                      int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
   UpdatePlan P;
   int rc;
   if ((rc = plan_update(src, tgt, shift, rope, st, mode, &P)) != KVC_OK) return rc;
+  return update_planned(P, tgt, st, mode, workspace, workspace_bytes, stream);
+}
+
+int kvc_state_update_segmented(const kvc_cache* src, const kvc_cache* tgt, const kvc_segments* segs, const kvc_rope* rope,
+                               kvc_state* st, int32_t mode, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!tgt || !segs) return KVC_E_INVALID_ARG;
+  SegTable seg;
+  int rc = resolve_segments(segs, rope, tgt->d, tgt->T, &seg);
+  if (rc != KVC_OK) return rc;
+  UpdatePlan P;
+  if ((rc = plan_update(src, tgt, segs->shift[0], rope, st, mode, &P)) != KVC_OK) return rc;
+  P.seg = &seg;
+  return update_planned(P, tgt, st, mode, workspace, workspace_bytes, stream);
+}
+
+static int update_planned(UpdatePlan& P, const kvc_cache* tgt, kvc_state* st, int32_t mode, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  int rc;
   if (P.empty) return KVC_OK;
   if (P.fit) {
     const size_t need = kvc_workspace_bytes(tgt, st, mode);

@@ -44,6 +44,26 @@ struct alignas(16) DevItem {
   float cs[kMaxHalfD], sn[kMaxHalfD];    // cos / sin of shift * f_k, rounded from float64
 };
 
+// Piecewise-constant shifts over the token axis (Eq. 1: the shared pieces of a context sit at offsets
+// that differ from agent to agent, by an amount that is constant inside a segment).  n == 0: one shift
+// for all tokens, the launch's own tables.  Carried by value in the launch structs of the CUDA-core
+// kernels (the tables come from float64 on the host, as the single-shift ones do).
+constexpr int kMaxSegments = 16;
+struct SegTable {
+  int32_t n;                                   // segments; segment j covers tokens t_begin[j] .. t_begin[j+1]-1
+  int32_t coords;                              // 0: the correction lives at the target's positions (Eq. 12);
+                                               // 1: at the source's positions (App. A.2): Rot(src + c B), Rot^-1(tgt) - src
+  int32_t t_begin[kMaxSegments];
+  int32_t shifted[kMaxSegments];               // shift != 0
+  alignas(16) float cs[kMaxSegments][kMaxHalfD];
+  alignas(16) float sn[kMaxSegments][kMaxHalfD];
+};
+__device__ __forceinline__ int seg_index(const SegTable& s, int t) {
+  int k = 0;
+  for (int i = 1; i < s.n; ++i) k += (t >= s.t_begin[i]) ? 1 : 0;
+  return k;
+}
+
 struct ApplyLaunch {
   const DevItem* items;        // device table, or nullptr => `one`
   const int64_t* tile_prefix;  // device [n_items + 1] exclusive prefix of tile counts
@@ -51,6 +71,7 @@ struct ApplyLaunch {
   int64_t total_tiles;
   uint32_t* status;
   DevItem one;
+  SegTable seg;                // single-item launches only
 };
 
 struct UpdateLaunch {
@@ -257,11 +278,28 @@ __device__ __forceinline__ void lane_channels(int j, int pairing, int& chA, int&
 template <int D>
 __device__ __forceinline__ bool delta16(const DevCache& src, const DevCache& tgt, int is_v, int l, int h, int t,
                                         int chA, int chB, const float* cs, const float* sn, bool rotate, int pairing,
-                                        uint32_t* status, float* out) {
+                                        uint32_t* status, float* out, int coords = 0) {
   const __nv_bfloat16* trow = row_ptr(tgt, is_v ? tgt.v : tgt.k, l, h, t, status);
   if (!trow) return false;
   unpack8(*reinterpret_cast<const uint4*>(trow + chA), out);
   unpack8(*reinterpret_cast<const uint4*>(trow + chB), out + 8);
+  if (src.k && coords == 1) {
+    // the deviation at the source's positions: Rot_{-s}(tgt) - src
+    const __nv_bfloat16* srow = row_ptr(src, is_v ? src.v : src.k, l, h, t, status);
+    if (!srow) return false;
+    if (rotate) {
+      float nsn[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) nsn[i] = -sn[i];
+      rope16(out, cs, nsn, pairing);
+    }
+    float x[16];
+    unpack8(*reinterpret_cast<const uint4*>(srow + chA), x);
+    unpack8(*reinterpret_cast<const uint4*>(srow + chB), x + 8);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] -= x[i];
+    return true;
+  }
   if (src.k) {
     const __nv_bfloat16* srow = row_ptr(src, is_v ? src.v : src.k, l, h, t, status);
     if (!srow) return false;
@@ -273,6 +311,30 @@ __device__ __forceinline__ bool delta16(const DevCache& src, const DevCache& tgt
     for (int i = 0; i < 16; ++i) out[i] -= x[i];
   }
   return true;
+}
+
+// delta16 for a launch that may carry a segment table: lane j's cos / sin come from the token's segment.
+template <int D>
+__device__ __forceinline__ bool delta16_seg(const DevCache& src, const DevCache& tgt, int is_v, int l, int h, int t,
+                                            int chA, int chB, int j, const float* cs1, const float* sn1, bool rotate1,
+                                            const SegTable& seg, int pairing, uint32_t* status, float* out) {
+  if (seg.n == 0) {
+    float cs[8], sn[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      cs[i] = cs1[8 * j + i];
+      sn[i] = sn1[8 * j + i];
+    }
+    return delta16<D>(src, tgt, is_v, l, h, t, chA, chB, cs, sn, rotate1, pairing, status, out, seg.coords);
+  }
+  const int k = seg_index(seg, t);
+  float cs[8], sn[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    cs[i] = seg.cs[k][8 * j + i];
+    sn[i] = seg.sn[k][8 * j + i];
+  }
+  return delta16<D>(src, tgt, is_v, l, h, t, chA, chB, cs, sn, (!is_v) && seg.shifted[k] != 0, pairing, status, out, seg.coords);
 }
 
 }  // namespace kvc

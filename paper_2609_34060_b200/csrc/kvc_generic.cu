@@ -104,7 +104,9 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
     }
   }
 
-  const bool rotate = (!is_v) && (it.shift != 0);
+  bool rotate = (!is_v) && (it.shift != 0);
+  const bool segmented = (p.items == nullptr) && p.seg.n > 0;
+  const bool at_source = (p.items == nullptr) && p.seg.coords == 1;     // correction added before the rotation
   float cs[8], sn[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -115,6 +117,15 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
   for (int a = 0; a < TOK; ++a) {
     const int t = t0 + a * GROUPS + g;
     if (t >= T) continue;
+    if (segmented) {                              // this token's segment: its own shift and tables
+      const int k = seg_index(p.seg, t);
+      rotate = (!is_v) && p.seg.shifted[k] != 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        cs[i] = p.seg.cs[k][8 * j + i];
+        sn[i] = p.seg.sn[k][8 * j + i];
+      }
+    }
     const __nv_bfloat16* srow = row_ptr(it.src, is_v ? it.src.v : it.src.k, l, h, t, p.status);
     __nv_bfloat16* drow = row_ptr(it.dst, is_v ? it.dst.v : it.dst.k, l, h, t, p.status);
     if (!srow || !drow) continue;
@@ -126,8 +137,12 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
       float x[16];
       unpack8(ua, x);
       unpack8(ub, x + 8);
+      if (covered && at_source) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] += acc[a][i];
+      }
       if (rotate) rope16(x, cs, sn, p.pairing);
-      if (covered) {
+      if (covered && !at_source) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) x[i] += acc[a][i];
       }
@@ -143,7 +158,7 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
 // project: coeff[t, q] = sum_c Delta[t, c] * basis[q, c]
 // ---------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(256) project_generic_kernel(const __grid_constant__ UpdateLaunch p) {
+__global__ void __launch_bounds__(256) project_generic_kernel(const __grid_constant__ UpdateLaunch p, const __grid_constant__ SegTable seg) {
   if (p.run_if != nullptr && *p.run_if == 0) return;
   constexpr int LPT = D / 16;
   constexpr int TILE = 64;
@@ -172,13 +187,7 @@ __global__ void __launch_bounds__(256) project_generic_kernel(const __grid_const
     for (int i = 0; i < 16; ++i) dl[i] = 0.f;
     const int t = t0 + tl;
     if (t < n_cov) {
-      float cs[8], sn[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        cs[i] = p.cs[8 * j + i];
-        sn[i] = p.sn[8 * j + i];
-      }
-      if (!delta16<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, cs, sn, rotate, p.pairing, p.status, dl)) {
+      if (!delta16_seg<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, j, p.cs, p.sn, rotate, seg, p.pairing, p.status, dl)) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) dl[i] = 0.f;
       }
@@ -239,7 +248,7 @@ __global__ void __launch_bounds__(256) project_generic_kernel(const __grid_const
 // Gram: G = Delta^T Delta, one block per (layer, head, K|V), fixed summation order
 // ---------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant__ FitLaunch p) {
+__global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant__ FitLaunch p, const __grid_constant__ SegTable seg) {
   constexpr int LPT = D / 16;
   constexpr int TS = D / 16;     // each thread owns a TS x TS block of G
   constexpr int TT = 32;         // tokens per smem tile
@@ -268,13 +277,7 @@ __global__ void __launch_bounds__(256) gram_generic_kernel(const __grid_constant
       for (int i = 0; i < 16; ++i) dl[i] = 0.f;
       const int t = t0 + tl;
       if (t < p.n_cov) {
-        float cs[8], sn[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          cs[i] = p.cs[8 * j + i];
-          sn[i] = p.sn[8 * j + i];
-        }
-        if (!delta16<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, cs, sn, rotate, p.pairing, p.status, dl)) {
+        if (!delta16_seg<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, j, p.cs, p.sn, rotate, seg, p.pairing, p.status, dl)) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) dl[i] = 0.f;
         }
@@ -1181,8 +1184,10 @@ cudaError_t launch_apply_generic(const ApplyLaunch& L, int d, cudaStream_t s) {
 
 int generic_apply_tile(int d) { return d == 128 ? 128 : 256; }
 
+static const SegTable kNoSegments = {};
+
 template <int D>
-static cudaError_t launch_project_generic_t(const UpdateLaunch& U, int64_t tiles, cudaStream_t s) {
+static cudaError_t launch_project_generic_t(const UpdateLaunch& U, const SegTable& seg, int64_t tiles, cudaStream_t s) {
   const size_t smem = (64 * D + 32 * (D + 1)) * sizeof(float);
   static DeviceOnce once;
   int once_dev;
@@ -1192,21 +1197,23 @@ static cudaError_t launch_project_generic_t(const UpdateLaunch& U, int64_t tiles
     once.mark(once_dev);
   }
   if (tiles <= 0) return cudaSuccess;
-  project_generic_kernel<D><<<(unsigned)tiles, 256, smem, s>>>(U);
+  project_generic_kernel<D><<<(unsigned)tiles, 256, smem, s>>>(U, seg);
   return cudaGetLastError();
 }
 
-cudaError_t launch_project_generic(const UpdateLaunch& U, int d, int64_t tiles, cudaStream_t s) {
-  return d == 128 ? launch_project_generic_t<128>(U, tiles, s) : launch_project_generic_t<64>(U, tiles, s);
+cudaError_t launch_project_generic(const UpdateLaunch& U, const SegTable* seg, int d, int64_t tiles, cudaStream_t s) {
+  const SegTable& sg = seg ? *seg : kNoSegments;
+  return d == 128 ? launch_project_generic_t<128>(U, sg, tiles, s) : launch_project_generic_t<64>(U, sg, tiles, s);
 }
 
-cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s) {
+cudaError_t launch_gram_generic(const FitLaunch& F, const SegTable* seg, int d, cudaStream_t s) {
   const int blocks = F.L * F.H * 2;
   if (blocks <= 0) return cudaSuccess;
+  const SegTable& sg = seg ? *seg : kNoSegments;
   if (d == 128)
-    gram_generic_kernel<128><<<blocks, 256, 0, s>>>(F);
+    gram_generic_kernel<128><<<blocks, 256, 0, s>>>(F, sg);
   else
-    gram_generic_kernel<64><<<blocks, 256, 0, s>>>(F);
+    gram_generic_kernel<64><<<blocks, 256, 0, s>>>(F, sg);
   return cudaGetLastError();
 }
 

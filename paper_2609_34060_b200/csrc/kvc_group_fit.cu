@@ -38,7 +38,7 @@ constexpr int kTT = 32;          // tokens per staged tile of the back-projectio
 // fixed order.  Thread (cg, qg) accumulates channels 4 cg .. + 3 against RQ ranks.
 // ---------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(256) group_backproject_kernel(const __grid_constant__ GroupFitLaunch p) {
+__global__ void __launch_bounds__(256) group_backproject_kernel(const __grid_constant__ GroupFitLaunch p, const __grid_constant__ SegTable seg) {
   constexpr int LPT = D / 16;
   constexpr int CG = D / 4;          // channel groups
   constexpr int QG = 256 / CG;       // rank groups
@@ -75,13 +75,7 @@ __global__ void __launch_bounds__(256) group_backproject_kernel(const __grid_con
       for (int i = 0; i < 16; ++i) dl[i] = 0.f;
       const int t = t0 + tl;
       if (t < t_end) {
-        float cs[8], sn[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          cs[i] = p.cs[8 * j + i];
-          sn[i] = p.sn[8 * j + i];
-        }
-        if (!delta16<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, cs, sn, rotate, p.pairing, p.status, dl)) {
+        if (!delta16_seg<D>(p.src, p.tgt, is_v, l, h, t, chA, chB, j, p.cs, p.sn, rotate, seg, p.pairing, p.status, dl)) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) dl[i] = 0.f;
         }
@@ -459,13 +453,15 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
 
 }  // namespace
 
-cudaError_t launch_group_backproject(const GroupFitLaunch& G, cudaStream_t s) {
+cudaError_t launch_group_backproject(const GroupFitLaunch& G, const SegTable* seg, cudaStream_t s) {
   const int blocks = G.L * G.H * 2 * G.parts;
   if (blocks <= 0) return cudaSuccess;
+  static const SegTable kNoSegments = {};
+  const SegTable& sg = seg ? *seg : kNoSegments;
   if (G.d == 128)
-    group_backproject_kernel<128><<<blocks, 256, 0, s>>>(G);
+    group_backproject_kernel<128><<<blocks, 256, 0, s>>>(G, sg);
   else if (G.d == 64)
-    group_backproject_kernel<64><<<blocks, 256, 0, s>>>(G);
+    group_backproject_kernel<64><<<blocks, 256, 0, s>>>(G, sg);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

@@ -52,8 +52,8 @@ uint32_t* status_word_ptr();
 cudaError_t launch_apply_generic(const ApplyLaunch& L, int d, cudaStream_t s);
 int generic_apply_tile(int d);                     // tokens per tile of the generic apply kernel
 constexpr int kGenericProjectTile = 64;
-cudaError_t launch_project_generic(const UpdateLaunch& U, int d, int64_t tiles, cudaStream_t s);
-cudaError_t launch_gram_generic(const FitLaunch& F, int d, cudaStream_t s);
+cudaError_t launch_project_generic(const UpdateLaunch& U, const SegTable* seg, int d, int64_t tiles, cudaStream_t s);
+cudaError_t launch_gram_generic(const FitLaunch& F, const SegTable* seg, int d, cudaStream_t s);
 // full eigensolver; solver != nullptr: matrices with solver[m] == 0 are skipped (already served)
 cudaError_t launch_eig(const FitLaunch& F, int d, const int32_t* solver, cudaStream_t s);
 // top-r subspace solver (kvc_eig_subspace.cu): sums and symmetrises the partial Grams, serves the
@@ -63,7 +63,7 @@ cudaError_t launch_eig_subspace(const FitLaunch& F, int d, int32_t* solver, cuda
 
 // FIT of layer-grouped states (kvc_group_fit.cu)
 constexpr int kGroupFitParts = 4;   // token ranges whose back-projections are summed in a fixed order
-cudaError_t launch_group_backproject(const GroupFitLaunch& G, cudaStream_t s);
+cudaError_t launch_group_backproject(const GroupFitLaunch& G, const SegTable* seg, cudaStream_t s);
 cudaError_t launch_group_small(const GroupFitLaunch& G, int op, cudaStream_t s);
 
 // reliability gate (kvc_gate.cu)

@@ -116,3 +116,56 @@ def test_rope_preserves_dot_products_at_equal_shift():
     q, k = rng.standard_normal((5, d)), rng.standard_normal((5, d))
     s = 211
     assert np.allclose(np.sum(orc.rope_shift(q, s, f) * orc.rope_shift(k, s, f), -1), np.sum(q * k, -1), atol=1e-11)
+
+
+def test_per_token_shifts_equal_constant_shifts_segment_by_segment():
+    """Multi-segment contexts (Eq. 1): rotating with a per-token shift vector is rotating every segment
+    by its own constant shift; the segmented apply is the plain apply segment by segment; and the two
+    coordinate conventions differ exactly by the rotation of the correction."""
+    rng = np.random.default_rng(31)
+    T, d, r = 37, 16, 3
+    f = orc.rope_inv_freq(d, 10000.0)
+    t_begin, shift = [0, 9, 20], [5, 0, -13]
+    s_tok = orc.segment_shifts(T, t_begin, shift)
+    assert s_tok.tolist() == [5] * 9 + [0] * 11 + [-13] * 17
+    x = rng.standard_normal((T, d))
+    for pairing in (orc.ROPE_HALF, orc.ROPE_INTERLEAVED):
+        y = orc.rope_shift_tokens(x, s_tok, f, pairing)
+        for j, t0 in enumerate(t_begin):
+            t1 = t_begin[j + 1] if j + 1 < len(t_begin) else T
+            assert np.array_equal(y[t0:t1], np.asarray(orc.rope_shift(x[t0:t1], shift[j], f, pairing)))
+        # a scalar re-derivation of one element: pair (k, k + d/2) or (2k, 2k+1) turned by s f_k
+        t, k = 30, 2
+        i, j2 = (k, k + d // 2) if pairing == orc.ROPE_HALF else (2 * k, 2 * k + 1)
+        ang = -13 * f[k]
+        assert math.isclose(y[t, i], x[t, i] * math.cos(ang) - x[t, j2] * math.sin(ang), rel_tol=1e-12, abs_tol=1e-15)
+        assert math.isclose(y[t, j2], x[t, i] * math.sin(ang) + x[t, j2] * math.cos(ang), rel_tol=1e-12, abs_tol=1e-15)
+    # apply: segment by segment with the plain apply_slab (TARGET coordinates)
+    bits = orc.f64_to_bf16_bits(x)
+    c, B = rng.standard_normal((T, r)), rng.standard_normal((r, d))
+    n_cov = 29
+    ref, out = orc.apply_slab_tokens(bits, c, B, s_tok, f, n_cov, True)
+    for j, t0 in enumerate(t_begin):
+        t1 = t_begin[j + 1] if j + 1 < len(t_begin) else T
+        n_seg = max(0, min(n_cov, t1) - t0)
+        ref_j, out_j = orc.apply_slab(bits[t0:t1], c[t0:t1], B, shift[j], f, n_seg, True)
+        assert np.array_equal(ref[t0:t1], ref_j) and np.array_equal(out[t0:t1], out_j)
+    # values ignore the shifts; uncovered unshifted key rows keep their bits
+    ref_v, out_v = orc.apply_slab_tokens(bits, c, B, s_tok, f, n_cov, False)
+    ref_v0, out_v0 = orc.apply_slab(bits, c, B, 0, f, n_cov, False)
+    assert np.array_equal(ref_v, ref_v0) and np.array_equal(out_v, out_v0)
+    # SOURCE coordinates: the correction is rotated with the token; equal to TARGET with the rotated correction
+    ref_s, _ = orc.apply_slab_tokens(bits, c, B, s_tok, f, T, True, coords=orc.COORDS_SOURCE)
+    rotated_corr = orc.rope_shift_tokens(c @ B, s_tok, f)
+    assert np.allclose(ref_s, orc.rope_shift_tokens(orc.bf16_to_f64(bits), s_tok, f) + rotated_corr, atol=1e-12)
+    # with one shift for all tokens this is the re-aligned basis of App. A.2
+    one = orc.segment_shifts(T, [0], [7])
+    ref_1, _ = orc.apply_slab_tokens(bits, c, B, one, f, T, True, coords=orc.COORDS_SOURCE)
+    ref_2, _ = orc.apply_slab(bits, c, orc.realign_basis(B, 7, f), 7, f, T, True)
+    assert np.allclose(ref_1, ref_2, atol=1e-12)
+    # deviations: SOURCE is TARGET carried back by the inverse rotation; fitting either reproduces the target
+    tgt_bits = orc.f64_to_bf16_bits(rng.standard_normal((T, d)))
+    d_t = orc.deviation_tokens(bits, tgt_bits, s_tok, f, True)
+    d_s = orc.deviation_tokens(bits, tgt_bits, s_tok, f, True, coords=orc.COORDS_SOURCE)
+    assert np.allclose(orc.rope_shift_tokens(d_s, s_tok, f), d_t, atol=1e-12)
+    assert np.allclose(orc.rope_shift_tokens(orc.bf16_to_f64(bits) + d_s, s_tok, f), orc.bf16_to_f64(tgt_bits), atol=1e-12)
