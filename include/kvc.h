@@ -117,8 +117,8 @@ typedef struct kvc_state {
  * Grouping by layer is served by kvc_apply, kvc_chain, kvc_apply_batch and by kvc_state_update: in
  * KVC_PROJECT mode the projection sums over the heads (coeff[l,t,:] = sum_h Delta[l,h,t,:] . basis[l][:, h]^T);
  * in the FIT modes (r <= 32) the basis rows are the r leading right singular vectors of the layer's
- * concatenated deviation [n_cov, H d], see kvc_state_update.  The gate, token weights and
- * kvc_apply_multi return KVC_E_UNSUPPORTED for it.
+ * concatenated deviation [n_cov, H d], see kvc_state_update.  The gate, the token weights and
+ * kvc_apply_multi take grouped states as well (per anchor: pools may mix the two groupings).
  */
 #define KVC_GROUP_HEAD  0
 #define KVC_GROUP_LAYER 1

@@ -772,7 +772,6 @@ int kvc_apply_multi(const kvc_cache* src, const kvc_state* deltas, int32_t n_anc
   int live = 0;
   for (int v = 0; v < n_anchors; ++v) {
     if ((rc = resolve_state(&deltas[v], 0, &st[v])) != KVC_OK) return rc;
-    if (st[v].grouped) return KVC_E_UNSUPPORTED;
     if (deltas[v].r > 0 && deltas[v].n_cov > src->T) return KVC_E_SHAPE;
     live += deltas[v].r > 0 && deltas[v].n_cov > 0;
   }
@@ -857,7 +856,6 @@ int kvc_token_weights(const kvc_cache* src, int32_t src_pos, const kvc_state* an
   DevState st[KVC_MAX_ANCHORS];
   for (int v = 0; v < n_anchors; ++v) {
     if ((rc = resolve_state(&anchors[v], 0, &st[v])) != KVC_OK) return rc;
-    if (st[v].grouped) return KVC_E_UNSUPPORTED;
     if (anchors[v].r <= 0 || anchors[v].n_cov < 0 || anchors[v].n_cov > src->T) return KVC_E_SHAPE;
   }
   uint32_t* status = status_ptr();
@@ -909,7 +907,7 @@ int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_
     if (a.n_cov < k) return KVC_E_SHAPE;            // not compatible at this comparison length
     if (k > 0 && (!a.coeff_v || !a.basis_v)) return KVC_E_INVALID_ARG;
     if (a.basis_dtype != KVC_F32 && a.basis_dtype != KVC_BF16) return KVC_E_INVALID_ARG;
-    if (a.grouping != KVC_GROUP_HEAD) return KVC_E_UNSUPPORTED;
+    if (a.grouping != KVC_GROUP_HEAD && a.grouping != KVC_GROUP_LAYER) return KVC_E_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a.coeff_v) | reinterpret_cast<uintptr_t>(a.basis_v)) & 15) return KVC_E_UNSUPPORTED;
   }
   if (reinterpret_cast<uintptr_t>(dist_sq) & 7) return KVC_E_INVALID_ARG;
@@ -933,6 +931,7 @@ int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_
       it.st.r = a.r;
       it.st.n_cov = a.n_cov;
       it.st.basis_bf16 = a.basis_dtype == KVC_BF16;
+      it.st.grouped = a.grouping == KVC_GROUP_LAYER;
       it.L = src->L;
       it.H = src->H;
       for (int c = 0; c < kMaxHalfD; ++c) it.cs[c] = 1.f;
@@ -953,6 +952,7 @@ int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_
       g.r = a.r;
       g.n_cov = a.n_cov;
       g.basis_bf16 = a.basis_dtype == KVC_BF16;
+      g.grouped = a.grouping == KVC_GROUP_LAYER;
       g.k = k;
       g.L = src->L;
       g.H = src->H;

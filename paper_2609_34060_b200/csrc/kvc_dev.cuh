@@ -142,6 +142,7 @@ struct GateLaunch {            // Eq. 9 for one anchor, CUDA-core kernel
   const void* basis;           // [L,H,r,d]
   int32_t r, n_cov, basis_bf16, k;
   int32_t L, H;
+  int32_t grouped, pad;        // the anchor's state is grouped by layer: coeff [L,n_cov,r], basis [L,r,H*d]
   double* out;                 // the squared distance is added here
   uint32_t* status;
 };

@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(256) gate_generic_kernel(const GateLaunch g) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int slab = blockIdx.y;
   const int l = slab / g.H, h = slab - l * g.H;
-  const float* coeff = g.coeff + (int64_t)slab * g.n_cov * g.r;
+  const float* coeff = g.coeff + (int64_t)(g.grouped ? l : slab) * g.n_cov * g.r;
   double acc = 0.0;
   for (int t = blockIdx.x * 8 + warp; t < g.k; t += gridDim.x * 8) {
     const __nv_bfloat16* row = row_ptr(g.src, g.src.v, l, h, t, g.status);
@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(256) gate_generic_kernel(const GateLaunch g) {
     const float* ct = coeff + (int64_t)t * g.r;
     for (int q = 0; q < g.r; ++q) {
       const float cq = ct[q];
-      const int64_t boff = ((int64_t)slab * g.r + q) * D + lane;
+      const int64_t boff = (g.grouped ? ((int64_t)l * g.r + q) * g.H + h : (int64_t)slab * g.r + q) * D + lane;
 #pragma unroll
       for (int c = 0; c < CPL; ++c) {
         const float b = g.basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(g.basis)[boff + 32 * c])

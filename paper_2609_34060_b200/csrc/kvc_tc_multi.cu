@@ -45,7 +45,7 @@ struct Block {                 // one rank block of one anchor
   int32_t col0;                // first rank of the block inside the anchor's state
   int32_t n_cov;               // rows the anchor covers
   int32_t anchor;              // index of the anchor's coefficient maps
-  int32_t pad;
+  int32_t grouped;             // the anchor's state is grouped by layer: coefficient slab = layer
 };
 
 struct MultiLaunch {
@@ -77,8 +77,8 @@ struct Ctrl {
 struct PrepLaunch {
   const void* basis_k[KVC_MULTI_MAX_BLOCKS];
   const void* basis_v[KVC_MULTI_MAX_BLOCKS];
-  int32_t r[KVC_MULTI_MAX_BLOCKS], col0[KVC_MULTI_MAX_BLOCKS], bf16[KVC_MULTI_MAX_BLOCKS];
-  int32_t n_blocks, slabs;
+  int32_t r[KVC_MULTI_MAX_BLOCKS], col0[KVC_MULTI_MAX_BLOCKS], bf16[KVC_MULTI_MAX_BLOCKS], grouped[KVC_MULTI_MAX_BLOCKS];
+  int32_t n_blocks, slabs, H, pad;
   __nv_bfloat16* out;
 };
 
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   const void* basis = kv ? p.basis_v[e] : p.basis_k[e];
   const int r = p.r[e], col0 = p.col0[e];
   __nv_bfloat16* out = p.out + (((int64_t)e * 2 + kv) * p.slabs + slab) * (128 * 64);
-  write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0);
+  write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0, p.grouped[e] != 0, p.H);
 }
 
 template <int NSTAGE, int NC, int NO>
@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
             const uint32_t ebar = smem_u32(&ctrl->cfull[c]);
             mbar_expect_tx(ebar, (uint32_t)(kCoeffBytes + (wts ? kWeightBytes : 0)));
             const CUtensorMap* cmap = is_v ? &p.coeff_v[b.anchor] : &p.coeff_k[b.anchor];
-            tma_load_3d(coeffs + c * kCoeffBytes, cmap, ebar, b.col0, t0, w.slab());
+            tma_load_3d(coeffs + c * kCoeffBytes, cmap, ebar, b.col0, t0, b.grouped ? w.l : w.slab());
             if (wts) bulk_load_1d(base + kWeightOff + c * kWeightBytes, wts + t0, kWeightBytes, ebar);
           }
         }
@@ -583,8 +583,9 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
     const DevState& a = anchors[v];
     if (a.r <= 0 || a.n_cov <= 0) continue;                     // an empty anchor contributes nothing
     if (a.r > 64 || (a.r & 3)) return KVC_E_UNSUPPORTED;
-    if (!encode_coeff(&M.coeff_k[v], a.coeff_k, a.r, a.n_cov, L * H) ||
-        !encode_coeff(&M.coeff_v[v], a.coeff_v, a.r, a.n_cov, L * H))
+    const int cslabs = a.grouped ? L : L * H;
+    if (!encode_coeff(&M.coeff_k[v], a.coeff_k, a.r, a.n_cov, cslabs) ||
+        !encode_coeff(&M.coeff_v[v], a.coeff_v, a.r, a.n_cov, cslabs))
       return KVC_E_CUDA;
     for (int col0 = 0; col0 < a.r; col0 += 32) {
       if (nb == KVC_MULTI_MAX_BLOCKS) return KVC_E_UNSUPPORTED;
@@ -594,6 +595,8 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
       b.col0 = col0;
       b.n_cov = a.n_cov;
       b.anchor = v;
+      b.grouped = a.grouped;
+      P.grouped[nb] = a.grouped;
       P.basis_k[nb] = a.basis_k;
       P.basis_v[nb] = a.basis_v;
       P.r[nb] = a.r;
@@ -627,6 +630,7 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
     return KVC_E_CUDA;
   P.n_blocks = nb;
   P.slabs = L * H;
+  P.H = H;
   P.out = ops;
   multi_prep_kernel<<<dim3((unsigned)(L * H), 2, (unsigned)nb), 256, 0, s>>>(P);
   if (cudaGetLastError() != cudaSuccess) return KVC_E_CUDA;

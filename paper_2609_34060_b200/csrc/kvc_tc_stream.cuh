@@ -53,13 +53,15 @@ struct Walker {
 
 // One basis operand block: 128 rows (channel) of [32 hi | 32 lo] bf16 for ranks col0 .. col0 + 31 of
 // the basis [slabs][r][128] (float32 or bf16; zero beyond rank r).  Called by a block of 256 threads.
+// A state grouped by layer keeps [layers][r][H * 128]: head h of layer l reads columns h * 128 .. of row q.
 __device__ __forceinline__ void write_operand_block(__nv_bfloat16* out, const void* basis, bool basis_bf16, int slab, int r,
-                                                    int col0) {
+                                                    int col0, bool grouped = false, int H = 1) {
+  const int l = slab / H, h = slab - l * H;
   for (int i = threadIdx.x; i < 32 * 128; i += 256) {
     const int q = i >> 7, ch = i & 127;           // coalesced reads along the channel
     float x = 0.f;
     if (col0 + q < r) {
-      const int64_t off = ((int64_t)slab * r + col0 + q) * 128 + ch;
+      const int64_t off = grouped ? (((int64_t)l * r + col0 + q) * H + h) * 128 + ch : ((int64_t)slab * r + col0 + q) * 128 + ch;
       x = basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off]) : reinterpret_cast<const float*>(basis)[off];
     }
     const __nv_bfloat16 hi = __float2bfloat16_rn(x);

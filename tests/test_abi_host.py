@@ -142,8 +142,10 @@ def test_multi_anchor_and_grouping_argument_errors(lib):
     need = lib.kvc_workspace_bytes(C.byref(src), C.byref(grouped), kvc.KVC_FIT)
     assert need >= 4 * src.L * 2 * (src.H * src.d) * (1 + 4 * grouped.r)       # eigenvalues + four partial back-projections
     assert lib.kvc_state_update(None, C.byref(src), 0, C.byref(rope), C.byref(grouped), kvc.KVC_FIT, 0x7000100, need - 1, None) == kvc.KVC_E_WORKSPACE
-    assert lib.kvc_gate_distance(C.byref(src), C.byref(grouped), 1, 8, 0x8000000, None) == -3
-    assert lib.kvc_apply_multi(C.byref(src), C.byref(grouped), 1, None, None, 0, C.byref(rope), C.byref(dst), 0x9000000, 1 << 30, None) == -3
+    bad_group = _state()
+    bad_group.grouping = 9
+    assert lib.kvc_gate_distance(C.byref(src), C.byref(bad_group), 1, 8, 0x8000000, None) == -1
+    assert lib.kvc_apply_multi(C.byref(src), C.byref(bad_group), 1, None, None, 0, C.byref(rope), C.byref(dst), 0x9000000, 1 << 30, None) == -1
     # byte accounting of a grouped state: the coefficients are shared by the heads
     big, st = _cache(L=32, H=8, T=8192, d=128), _state(r=32, n_cov=8192)
     st.grouping = kvc.KVC_GROUP_LAYER

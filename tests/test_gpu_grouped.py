@@ -266,19 +266,79 @@ def test_grouped_fit_without_a_gap_is_flagged_and_zero_is_zero():
     assert float(kvc.kvc_group_fit_eigenvalues(z, ws).abs().max()) == 0.0
 
 
-def test_grouped_is_rejected_where_it_is_not_served():
+def _expand(cfg, g):
+    """The per-(layer, head) state that defines the same low-rank product as the grouped state g."""
+    L, H, d, r = cfg.L, cfg.H, cfg.d, g.r
+    ex = lambda c: c[:, None].expand(L, H, c.shape[1], r).contiguous()
+    sp = lambda b: b.to(torch.float32).view(L, r, H, d).permute(0, 2, 1, 3).contiguous()
+    return kvc.State(ex(g.coeff_k), ex(g.coeff_v), sp(g.basis_k), sp(g.basis_v), n_cov=g.n_cov)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_grouped_anchors_in_gate_token_weights_and_multi_apply(path):
+    """Anchor pools whose states are grouped by layer (one of the three per head, to show that pools may
+    mix): gate distances (Eq. 9), token-wise weights (App. A.3) and the weighted multi-anchor apply (Eq. 8),
+    each against the oracle run on the expanded per-head form of the same states."""
+    from test_gpu_gate import _oracle_dist
+    from test_gpu_multi import _oracle, _oracle_token_weights, _weights, _check as _check_multi
+    cfg = CFG_S.scaled(T=777)
+    L, H, T, d = cfg.L, cfg.H, cfg.T, cfg.d
+    grouped = [_grouped_state(cfg, 1), _grouped_state(cfg, 2, n_cov=T - 130), hp.make_state(cfg, 3)]
+    per_head = [_expand(cfg, grouped[0]), _expand(cfg, grouped[1]), grouped[2]]
+    anchor_pos, src_pos = [100, 37, 412], 250
+    # the source cache: close to anchor 0's reconstruction (keys moved to the source's positions), oracle arithmetic
+    src_cpu = hp.make_cache(cfg)
+    osrc = hp.oracle_cache(src_cpu)
+    inv = hp.inv_freq(cfg)
+    eps = wl.noise((2, L, H, T, d), cfg.seed, 91, "cpu").numpy().astype(np.float64)
+    for l in range(L):
+        for h in range(H):
+            for wi, which in enumerate(("k", "v")):
+                c = getattr(per_head[0], "coeff_" + which)[l, h].numpy().astype(np.float64)
+                b = getattr(per_head[0], "basis_" + which)[l, h].numpy().astype(np.float64)
+                x = c @ b
+                if which == "k":
+                    x = orc.rope_shift(x, src_pos - anchor_pos[0], inv)
+                osrc.put_bits(which, l, h, orc.f64_to_bf16_bits(x + 0.2 * eps[wi, l, h]))
+    mk = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16)
+    src_cpu = kvc.Cache(mk(osrc.k), mk(osrc.v))
+    src = hp.to_dev(src_cpu, DEV)
+    dev = [hp.state_to_dev(a, DEV) for a in grouped]
+    kvc.kvc_set_path(path)
+    # ---- gate distance at a length every anchor covers
+    k = T - 200
+    d2 = torch.full((3,), -1.0, dtype=torch.float64, device=DEV)
+    kvc.kvc_gate_distance(src, dev, k, d2)
+    torch.cuda.synchronize()
+    ref = _oracle_dist(cfg, osrc, per_head, k)
+    assert np.all(np.abs(np.sqrt(d2.cpu().numpy()) - ref) <= 1e-4 * ref + 1e-6), (d2, ref)
+    if path != kvc.KVC_PATH_AUTO:
+        return                                   # token weights and the multi-anchor apply are tensor-core kernels
+    # ---- token weights
+    tp = kvc.kvc_multi_tpad(T)
+    wk, wv = torch.full((3, tp), -1.0, device=DEV), torch.full((3, tp), -1.0, device=DEV)
+    ws = torch.empty(kvc.kvc_token_weights_workspace_bytes(src, 3), dtype=torch.uint8, device=DEV)
+    kvc.kvc_token_weights(src, src_pos, dev, anchor_pos, kvc.Rope(cfg.theta), wk, wv, ws)
+    torch.cuda.synchronize()
+    rk, rv = _oracle_token_weights(cfg, osrc, src_pos, per_head, anchor_pos)
+    gk, gv = wk.cpu().numpy().astype(np.float64), wv.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(gk[:, :T] - rk)) <= 2e-5 and np.max(np.abs(gv[:, :T] - rv)) <= 2e-5
+    # ---- weighted multi-anchor apply with seeded weights
+    w_k, w_v = _weights(3, T, cfg.seed, 1), _weights(3, T, cfg.seed, 2)
+    shift = -41
+    dst = hp.empty_dst(src_cpu, cfg, DEV, fill=-7.0)
+    ws2 = torch.empty(max(kvc.kvc_multi_workspace_bytes(src, dev), 128), dtype=torch.uint8, device=DEV)
+    kvc.kvc_apply_multi(src, dev, w_k.to(DEV), w_v.to(DEV), shift, kvc.Rope(cfg.theta), dst, ws2)
+    torch.cuda.synchronize()
+    odst, ref_k, ref_v = _oracle(cfg, src_cpu, per_head, w_k, w_v, shift)
+    _check_multi(dst, odst, ref_k, ref_v)
+
+
+def test_grouped_fit_beyond_rank_32_is_rejected():
     cfg = CFG_S.scaled(T=200)
-    st = hp.state_to_dev(_grouped_state(cfg, 1), DEV)
     src = hp.to_dev(hp.make_cache(cfg), DEV)
-    d2 = torch.zeros(1, dtype=torch.float64, device=DEV)
-    with pytest.raises(kvc.KvcError) as e:
-        kvc.kvc_gate_distance(src, [st], cfg.T, d2)
-    assert e.value.code == kvc.KVC_E_UNSUPPORTED
     ws = torch.empty(1 << 26, dtype=torch.uint8, device=DEV)
     big = _grouped_state(cfg.scaled(r=64), 1)            # the grouped fit serves r <= 32
     with pytest.raises(kvc.KvcError) as e:
         kvc.kvc_state_update(None, src, 0, kvc.Rope(cfg.theta), hp.state_to_dev(big, DEV), kvc.KVC_FIT, workspace=ws)
-    assert e.value.code == kvc.KVC_E_UNSUPPORTED
-    with pytest.raises(kvc.KvcError) as e:
-        kvc.kvc_apply_multi(src, [st], None, None, 0, kvc.Rope(cfg.theta), src, ws)
     assert e.value.code == kvc.KVC_E_UNSUPPORTED
