@@ -341,7 +341,7 @@ static size_t group_trpart_offset(const kvc_cache* tgt, int r) {
   return group_ypart_offset(tgt) + (size_t)kGroupFitParts * tgt->L * 2 * r * tgt->H * tgt->d * sizeof(float);
 }
 static size_t group_flags_offset(const kvc_cache* tgt, int r) {
-  return (group_trpart_offset(tgt, r) + (size_t)kGroupFitParts * tgt->L * 2 * tgt->H * sizeof(float) + 255) & ~(size_t)255;
+  return (group_trpart_offset(tgt, r) + (size_t)kGroupFitTraceParts * tgt->L * 2 * tgt->H * sizeof(float) + 255) & ~(size_t)255;
 }
 
 size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
@@ -525,7 +525,12 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   G.L = P.L;
   G.H = P.H;
   G.d = P.d;
-  G.parts = kGroupFitParts;
+  // the back-projection runs on the tensor cores where they take the geometry (two partial sums), else on CUDA cores
+  const bool use_tc = tl_path_force != KVC_PATH_GENERIC && !P.seg && P.d == 128 && (st->r & 3) == 0 &&
+                      !(P.dt.page_table && P.dt.page_mask + 1 > 128) && !(P.ds.page_table && P.ds.page_mask + 1 > 128);
+  if (!use_tc && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
+  G.parts = use_tc ? 2 : kGroupFitParts;
+  G.tr_parts = use_tc ? kGroupFitTraceParts : kGroupFitParts;
   const int per = (st->n_cov + kGroupFitParts - 1) / kGroupFitParts;
   G.tokens_per_part = (per + 31) / 32 * 32;
   G.status = status;
@@ -537,7 +542,11 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   for (int it = 0; it < 3; ++it) {
     int rc = project_edge(P, status, s);
     if (rc != KVC_OK) return rc;
-    if (launch_group_backproject(G, P.seg, s) != cudaSuccess) return KVC_E_CUDA;
+    if (use_tc) {
+      if ((rc = tc_backproject(G, s)) != KVC_OK) return rc;
+    } else if (launch_group_backproject(G, P.seg, s) != cudaSuccess) {
+      return KVC_E_CUDA;
+    }
     if (launch_group_small(G, ops[it], s) != cudaSuccess) return KVC_E_CUDA;
   }
   // Refinement rounds, for the case that a block was merely slow (the hashed start had a small component
@@ -550,7 +559,11 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
     if (launch_group_small(G, KVC_GROUP_OP_ORTH_KEEP, s) != cudaSuccess) return KVC_E_CUDA;
     int rc = project_edge(P, status, s, G.need_more + round);
     if (rc != KVC_OK) return rc;
-    if (launch_group_backproject(G, P.seg, s) != cudaSuccess) return KVC_E_CUDA;
+    if (use_tc) {
+      if ((rc = tc_backproject(G, s)) != KVC_OK) return rc;
+    } else if (launch_group_backproject(G, P.seg, s) != cudaSuccess) {
+      return KVC_E_CUDA;
+    }
     if (launch_group_small(G, KVC_GROUP_OP_RITZ, s) != cudaSuccess) return KVC_E_CUDA;
   }
   return KVC_OK;

@@ -124,7 +124,8 @@ struct GroupFitLaunch {        // FIT of states grouped by layer (D = H d): back
   int32_t* solver;             // [L*2] per-problem code
   int32_t* need_more;          // [kGroupFitRounds + 1]: round k runs only when need_more[k] != 0 (round 0 always)
   int32_t r, n_cov, pairing, shift, L, H, d, parts, tokens_per_part;
-  int32_t round, last_round, pad;
+  int32_t round, last_round;
+  int32_t tr_parts;            // partial sums of the trace: parts (CUDA-core pass) or 32 (tensor-core pass: half x team warp)
   uint32_t* status;
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];

@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
 
   // ---- KVC_GROUP_OP_RITZ: Rayleigh-Ritz on (Q, Y = Q G), acceptance, output
   float tr = 0.f;
-  for (int part = 0; part < p.parts; ++part)
+  for (int part = 0; part < p.tr_parts; ++part)
     for (int h = 0; h < p.H; ++h) tr += p.trpart[((int64_t)part * p.L * 2 + prob) * p.H + h];
   float* evals = p.evals + (int64_t)prob * Dg;
   if (*code == KVC_SOLVER_FULL_DEPENDENT || !(tr > 0.f)) {

@@ -62,7 +62,8 @@ constexpr int kSubspaceMaxRank = 32;
 cudaError_t launch_eig_subspace(const FitLaunch& F, int d, int32_t* solver, cudaStream_t s);
 
 // FIT of layer-grouped states (kvc_group_fit.cu)
-constexpr int kGroupFitParts = 4;   // token ranges whose back-projections are summed in a fixed order
+constexpr int kGroupFitParts = 4;   // token ranges whose back-projections are summed in a fixed order (CUDA-core pass; the tensor-core pass uses 2)
+constexpr int kGroupFitTraceParts = 32;   // room for the partial sums of the trace (tensor-core pass: half x team warp)
 cudaError_t launch_group_backproject(const GroupFitLaunch& G, const SegTable* seg, cudaStream_t s);
 cudaError_t launch_group_small(const GroupFitLaunch& G, int op, cudaStream_t s);
 

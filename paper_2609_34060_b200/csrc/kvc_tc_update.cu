@@ -772,6 +772,410 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Back-projection of the layer-grouped fit:  Y[q, h d + c] = sum_t Z[t, q] Delta[l, h, t, c]  (Z = the
+// grouped coefficients [L, n_cov, r], r <= 32), and trace = sum Delta^2.  The Gram kernel's pipeline with
+// a second operand: the team forms H and 2 L of Delta as there and converts the tile's float32
+// coefficients to [Z hi | Z lo] bf16 (64 columns); the tensor cores accumulate
+//     P1 = H^T [Zh | Zl]   and   P2 = (2 L)^T [Zh | Zl]        (two 128 x 64 accumulators)
+// and the flush forms  Y = P1[:, :32] + P1[:, 32:] + P2[:, :32] / 2 = H^T Zh + H^T Zl + L^T Zh.
+// Work unit = half of a slab's tokens; the two halves' sums are added by the consumer in a fixed order.
+// ---------------------------------------------------------------------------------------------
+constexpr int kZBytes = kTileTok * 128;        // 128 tokens x 32 float32, and as large again as [hi | lo] bf16
+
+struct BackprojTcLaunch {
+  FitLaunch f;                 // caches, n_cov, pairing, shift, L, H, status, rope tables
+  float* ypart;                // [2][L*2][r][H*128]
+  float* trpart;               // [2 * 16][L*2][H]: one entry per (half, team warp)
+  const int32_t* run_if;
+  int64_t total_units;
+  int32_t tiles_per_slab, tiles_per_unit, has_src, r;
+  UpdMaps maps;
+};
+__device__ __forceinline__ GUnit gdecode(const BackprojTcLaunch& p, int64_t unit) {
+  GUnit g;
+  g.part = (int)(unit & 1);
+  const int64_t sk = unit >> 1;
+  g.is_v = (int)(sk & 1);
+  g.slab = (int)(sk >> 1);
+  g.l = g.slab / p.f.H;
+  g.h = g.slab % p.f.H;
+  g.tile0 = g.part * p.tiles_per_unit;
+  g.n_tiles = max(0, min(p.tiles_per_unit, p.tiles_per_slab - g.tile0));
+  return g;
+}
+// hi = bf16(x), lo = bf16(x - hi) for two values, packed as bf16x2 words
+__device__ __forceinline__ void split2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xffff0000u);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - h0, x1 - h1);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __grid_constant__ BackprojTcLaunch p) {
+  if (p.run_if != nullptr && *p.run_if == 0) return;      // uniform over the grid: nothing has been set up yet
+  // kind::f16, bf16 x bf16 -> f32, both operands MN-major, M = 128 (channels), N = 64 ([Z hi | Z lo])
+  constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+  constexpr int kStage = kStageBytes + 2 * kZBytes;       // target tile, source tile, Z (float32), Z operand (bf16 hi | lo)
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t stages = base;
+  GCtrl<NS>* ctrl = reinterpret_cast<GCtrl<NS>*>(smem + NS * kStage);
+  volatile int* abort_flag = &ctrl->abort_flag;
+  const FitLaunch& f = p.f;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t nu = p.total_units;
+  const int64_t unit_begin = nu * blockIdx.x / gridDim.x;
+  const int64_t unit_end = nu * (blockIdx.x + 1) / gridDim.x;
+
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->conv[s]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&ctrl->acc_full[g]), 1);
+      mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
+    }
+    mbar_init(smem_u32(&ctrl->drain), 1);
+    ctrl->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctrl->tmem_base), 256);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+
+  if (warp == 0) {
+    // =============================================================== TMA producer
+    uint32_t i = 0;
+    bool dead = false;
+    for (int64_t un = unit_begin; un < unit_end && !dead; ++un) {
+      const GUnit g = gdecode(p, un);
+      for (int k = 0; k < g.n_tiles; ++k, ++i) {
+        PTile t;
+        t.slab = g.slab;
+        t.is_v = g.is_v;
+        t.l = g.l;
+        t.h = g.h;
+        t.t0 = (g.tile0 + k) * kTileTok;
+        const int s = i % NS;
+        const uint32_t use = i / NS;
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) {
+          dead = true;
+          break;
+        }
+        const uint32_t st_base = stages + s * kStage;
+        const uint32_t bar = smem_u32(&ctrl->full[s]);
+        int id_t, id_s = 0;
+        bool ok_t, ok_s = false;
+        uint32_t bytes = tile_bytes(f.tgt, t.t0, lane, id_t, ok_t, f.status);
+        if (p.has_src) bytes += tile_bytes(f.src, t.t0, lane, id_s, ok_s, f.status);
+        bytes += kZBytes;                                     // the coefficient tile always arrives whole (zero-filled past n_cov)
+        if (lane == 0) mbar_expect_tx(bar, bytes);
+        __syncwarp();
+        tile_issue(f.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
+        if (p.has_src) tile_issue(f.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
+        if (lane == 0) tma_load_3d(st_base + kStageBytes, t.is_v ? &p.maps.coeff_v : &p.maps.coeff_k, bar, 0, t.t0, t.l);
+        __syncwarp();
+      }
+    }
+    if (lane == 0) {
+      for (uint32_t k = (i > NS ? i - NS : 0); k < i; ++k) mbar_wait_drain(smem_u32(&ctrl->full[k % NS]), (k / NS) & 1u);
+    }
+  } else if (warp == 1) {
+    // =============================================================== MMA issuer
+    if (lane == 0) {
+      uint32_t i = 0, ui = 0;
+      bool dead = false;
+      for (int64_t un = unit_begin; un < unit_end && !dead; ++un, ++ui) {
+        const GUnit g = gdecode(p, un);
+        const int a = ui & 1;
+        if (!mbar_wait(smem_u32(&ctrl->acc_empty[a]), ((ui >> 1) & 1u) ^ 1u, abort_flag)) break;
+        const uint32_t d_tmem = tmem_base + a * 128;
+        uint32_t acc = 0;
+        for (int k = 0; k < g.n_tiles; ++k, ++i) {
+          const int s = i % NS;
+          const uint32_t use = i / NS;
+          if (!mbar_wait(smem_u32(&ctrl->conv[s]), use & 1u, abort_flag)) {
+            dead = true;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t hb = stages + s * kStage;          // H over the target tile
+          const uint32_t lb = hb + kTileBytes;                    // 2 L over the source tile
+          const uint32_t zb = hb + kStageBytes + kZBytes;         // [Z hi | Z lo], 128 tokens x 64
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {                        // 16 tokens = two 1 KB atoms per step
+            const uint64_t zd = umma_desc_mn_sw128(zb + ks * 2048);
+            umma_bf16(d_tmem, umma_desc_mn_sw128(hb + ks * 2048), zd, kIdesc, acc);              // H^T [Zh | Zl]
+            if (p.has_src) umma_bf16(d_tmem + 64, umma_desc_mn_sw128(lb + ks * 2048), zd, kIdesc, acc);   // (2 L)^T [Zh | Zl]
+            acc = 1;
+          }
+          umma_commit(smem_u32(&ctrl->empty[s]));                  // operands consumed => stage free
+        }
+        if (dead) break;
+        umma_commit(smem_u32(&ctrl->acc_full[a]));
+      }
+      umma_commit(smem_u32(&ctrl->drain));
+      mbar_wait_drain(smem_u32(&ctrl->drain), 0);
+    }
+  } else if (warp >= 4) {
+    // =============================================================== the team (16 warps)
+    const int e = warp - 4;
+    const int q = e & 3;
+    const int cq = e >> 2;
+    const int m = q * 32 + lane;                   // token row (conversion) / Gram row (flush)
+    const uint32_t sw = (uint32_t)(m & 7);
+    const bool rot_any = f.shift != 0;
+
+    float sq_cur = 0.f, sq_prev = 0.f;               // this thread's share of sum Delta^2: the unit being converted, the one being flushed
+    f32x2 sq2 = f2_pack(0.f, 0.f);
+    auto flush = [&](const GUnit& g, uint32_t ui) {
+      const int a = ui & 1;
+      bool ok = mbar_wait(smem_u32(&ctrl->acc_full[a]), (ui >> 1) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return false;
+      tc_fence_after();
+      const int64_t prob = (int64_t)g.l * 2 + g.is_v;
+      if (cq == 0) {
+        // Y[q, channel m] = (H^T Zh + H^T Zl + L^T Zh)[m, q]: columns q, 32 + q and half of 64 + q
+        const uint32_t t_acc = tmem_base + a * 128 + ((uint32_t)(q * 32) << 16);
+        float y[32], c0[16], c1[16];
+        tmem_ld16(t_acc, c0);
+        tmem_ld16(t_acc + 16, c1);
+        tmem_ld_wait();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          y[k] = c0[k];
+          y[16 + k] = c1[k];
+        }
+        tmem_ld16(t_acc + 32, c0);
+        tmem_ld16(t_acc + 48, c1);
+        tmem_ld_wait();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          y[k] += c0[k];
+          y[16 + k] += c1[k];
+        }
+        if (p.has_src) {
+          tmem_ld16(t_acc + 64, c0);
+          tmem_ld16(t_acc + 80, c1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            y[k] = fmaf(0.5f, c0[k], y[k]);
+            y[16 + k] = fmaf(0.5f, c1[k], y[16 + k]);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctrl->acc_empty[a]));
+        const int64_t Dg = (int64_t)f.H * 128;
+        float* yp = p.ypart + (((int64_t)g.part * f.L * 2 + prob) * p.r) * Dg + (int64_t)g.h * 128 + m;
+#pragma unroll
+        for (int k = 0; k < 32; ++k)
+          if (k < p.r) yp[(int64_t)k * Dg] = (g.n_tiles == 0) ? 0.f : y[k];
+      } else {
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctrl->acc_empty[a]));
+      }
+      // the unit's share of the trace, one entry per team warp (added in a fixed order by the consumer)
+      float sq = sq_prev;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if (lane == 0) p.trpart[(((int64_t)g.part * 16 + e) * f.L * 2 + prob) * f.H + g.h] = sq;
+      return true;
+    };
+
+    uint32_t i = 0, ui = 0;
+    bool alive = true, have_prev = false;
+    GUnit prev;
+    for (int64_t un = unit_begin; un < unit_end && alive; ++un, ++ui) {
+      const GUnit g = gdecode(p, un);
+      for (int k = 0; k < g.n_tiles && alive; ++k, ++i) {
+        const int s = i % NS;
+        const uint32_t use = i / NS;
+        bool ok = mbar_wait(smem_u32(&ctrl->full[s]), use & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+          alive = false;
+          break;
+        }
+        uint8_t* tg = smem + s * kStage;
+        uint8_t* sr = tg + kTileBytes;
+        const int tok = (g.tile0 + k) * kTileTok + m;
+        const bool live = tok < f.n_cov;
+        const bool rotate = rot_any && !g.is_v;
+        if (p.has_src || !live) {
+          if (f.pairing == 0) {
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+              const int j = 2 * cq + jj;
+              const uint32_t o = (uint32_t)(m * 128 + ((j ^ sw) << 4));
+              uint4* t0p = reinterpret_cast<uint4*>(tg + o);
+              uint4* t1p = reinterpret_cast<uint4*>(tg + kHalfBytes + o);
+              uint4* s0p = reinterpret_cast<uint4*>(sr + o);
+              uint4* s1p = reinterpret_cast<uint4*>(sr + kHalfBytes + o);
+              uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
+              if (live) {
+                // packed float32 pairs throughout: word w of a 16-byte chunk holds channels 2w, 2w + 1
+                const uint4 sa = *s0p, sb = *s1p, ta = *t0p, tb = *t1p;
+                const uint32_t sw0[4] = {sa.x, sa.y, sa.z, sa.w}, sw1[4] = {sb.x, sb.y, sb.z, sb.w};
+                const uint32_t tw0[4] = {ta.x, ta.y, ta.z, ta.w}, tw1[4] = {tb.x, tb.y, tb.z, tb.w};
+                f32x2 xa[4], xb[4];
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  xa[z] = f2_from_bf16x2(sw0[z]);
+                  xb[z] = f2_from_bf16x2(sw1[z]);
+                }
+                if (rotate) {
+                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(f.cs + 8 * j + 4);
+                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(f.sn + 8 * j + 4);
+                  const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
+                  const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
+                  const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
+#pragma unroll
+                  for (int z = 0; z < 4; ++z) {
+                    const f32x2 a = xa[z], b = xb[z];
+                    xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));       // a cos - b sin
+                    xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));        // a sin + b cos
+                  }
+                }
+                uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
+                uint32_t* hp1 = reinterpret_cast<uint32_t*>(&h1);
+                uint32_t* lp0 = reinterpret_cast<uint32_t*>(&l0);
+                uint32_t* lp1 = reinterpret_cast<uint32_t*>(&l1);
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  // H = bf16(Delta); 2 L = bf16(Delta - H) with one added to both exponents (the doubling is
+                  // exact; a zero remainder becomes 2^-126, which no sum notices)
+                  const f32x2 da = f2_sub(f2_from_bf16x2(tw0[z]), xa[z]), db = f2_sub(f2_from_bf16x2(tw1[z]), xb[z]);
+                  sq2 = f2_fma(da, da, f2_fma(db, db, sq2));
+                  hp0[z] = f2_to_bf16x2(da);
+                  hp1[z] = f2_to_bf16x2(db);
+                  lp0[z] = f2_to_bf16x2(f2_sub(da, f2_from_bf16x2(hp0[z]))) + 0x00800080u;
+                  lp1[z] = f2_to_bf16x2(f2_sub(db, f2_from_bf16x2(hp1[z]))) + 0x00800080u;
+                }
+              }
+              *t0p = h0;
+              *t1p = h1;
+              if (p.has_src) {
+                *s0p = l0;
+                *s1p = l1;
+              }
+            }
+          } else {
+            const uint32_t hb = (uint32_t)((cq >> 1) * kHalfBytes);
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+              const int j = 4 * (cq & 1) + jj;
+              const uint32_t o = hb + (uint32_t)(m * 128 + ((j ^ sw) << 4));
+              uint4* tp = reinterpret_cast<uint4*>(tg + o);
+              uint4* sp = reinterpret_cast<uint4*>(sr + o);
+              uint4 h = make_uint4(0, 0, 0, 0), l = h;
+              if (live) {
+                float x[8], y[8];
+                unpack8(*sp, x);
+                unpack8(*tp, y);
+                if (rotate) {
+                  const int f0 = 16 * cq + 4 * jj;
+                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + f0);
+                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + f0);
+                  const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
+                  const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
+#pragma unroll
+                  for (int z = 0; z < 4; ++z) {
+                    const float a = x[2 * z], b = x[2 * z + 1];
+                    x[2 * z] = a * cs[z] - b * sn[z];
+                    x[2 * z + 1] = a * sn[z] + b * cs[z];
+                  }
+                }
+                uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
+                uint32_t* lp = reinterpret_cast<uint32_t*>(&l);
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  const float e0 = y[2 * z] - x[2 * z], e1 = y[2 * z + 1] - x[2 * z + 1];
+                  sq_cur = fmaf(e0, e0, fmaf(e1, e1, sq_cur));
+                  split2x(e0, e1, hp[z], lp[z]);
+                }
+              }
+              *tp = h;
+              if (p.has_src) *sp = l;
+            }
+          }
+          fence_proxy_async();
+        } else {
+          // no source and a live row: the target tile is H as it stands; only its squares are needed
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj) {
+            const int j = 2 * cq + jj;
+            const uint32_t o = (uint32_t)(m * 128 + ((j ^ sw) << 4));
+            float y0[8], y1[8];
+            unpack8(*reinterpret_cast<const uint4*>(tg + o), y0);
+            unpack8(*reinterpret_cast<const uint4*>(tg + kHalfBytes + o), y1);
+#pragma unroll
+            for (int z = 0; z < 8; ++z) sq_cur = fmaf(y0[z], y0[z], fmaf(y1[z], y1[z], sq_cur));
+          }
+        }
+        {
+          // the coefficient tile: float32 [128 tokens][32] -> per token [hi (32) | lo (32)] bf16, the B operand
+          const uint8_t* zf = tg + kStageBytes;
+          uint8_t* zo = tg + kStageBytes + kZBytes;
+          const float4 z0 = *reinterpret_cast<const float4*>(zf + m * 128 + (((2 * cq) ^ sw) << 4));
+          const float4 z1 = *reinterpret_cast<const float4*>(zf + m * 128 + (((2 * cq + 1) ^ sw) << 4));
+          uint4 hi, lo;
+          split2(z0.x, z0.y, hi.x, lo.x);
+          split2(z0.z, z0.w, hi.y, lo.y);
+          split2(z1.x, z1.y, hi.z, lo.z);
+          split2(z1.z, z1.w, hi.w, lo.w);
+          *reinterpret_cast<uint4*>(zo + m * 128 + ((cq ^ sw) << 4)) = hi;
+          *reinterpret_cast<uint4*>(zo + m * 128 + (((4 + cq) ^ sw) << 4)) = lo;
+          fence_proxy_async();
+        }
+        mbar_arrive(smem_u32(&ctrl->conv[s]));
+        // the previous unit's accumulator is complete by now (its MMAs were issued a tile ago)
+        if (k == 0 && have_prev) {
+          alive = flush(prev, ui - 1);
+          have_prev = false;
+        }
+      }
+      if (have_prev && alive) alive = flush(prev, ui - 1);   // the unit before this one had no successor tile yet
+      prev = g;
+      have_prev = true;
+      {
+        float s0, s1;
+        f2_unpack(sq2, s0, s1);
+        sq_prev = sq_cur + s0 + s1;
+        sq_cur = 0.f;
+        sq2 = f2_pack(0.f, 0.f);
+      }
+    }
+    if (have_prev && alive) flush(prev, ui - 1);
+  }
+
+  __syncthreads();
+  if (tid == 0 && *abort_flag) atomicOr(f.status, KVC_FLAG_WAIT_EXPIRED);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
 static bool cache_ok(const DevCache& c) {
   if (c.page_table && (c.page_mask + 1) > 128) return false;
   return c.T < (1 << 30);
@@ -837,6 +1241,54 @@ int tc_gram(const FitLaunch& F, int d, cudaStream_t s) {
     once.mark(once_dev);
   }
   gram_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
+  return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
+}
+
+// The back-projection pass of the layer-grouped fit on the tensor cores (two partial sums: G.parts must be 2,
+// the trace comes in 32 partial sums).  KVC_E_UNSUPPORTED for what it does not take.
+int tc_backproject(const GroupFitLaunch& G, cudaStream_t s) {
+  using namespace tcu;
+  if (G.d != 128 || G.r <= 0 || G.r > 32 || (G.r & 3) || G.n_cov <= 0 || G.parts != 2) return KVC_E_UNSUPPORTED;
+  if (!cache_ok(G.tgt) || (G.src.k && !cache_ok(G.src)) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
+  BackprojTcLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.f.src = G.src;
+  L.f.tgt = G.tgt;
+  L.f.r = G.r;
+  L.f.n_cov = G.n_cov;
+  L.f.pairing = G.pairing;
+  L.f.shift = G.shift;
+  L.f.L = G.L;
+  L.f.H = G.H;
+  L.f.status = G.status;
+  memcpy(L.f.cs, G.cs, sizeof(L.f.cs));
+  memcpy(L.f.sn, G.sn, sizeof(L.f.sn));
+  L.ypart = G.ypart;
+  L.trpart = G.trpart;
+  L.run_if = (G.round > 0) ? G.need_more + G.round : nullptr;
+  L.r = G.r;
+  L.tiles_per_slab = (G.n_cov + kTileTok - 1) / kTileTok;
+  L.tiles_per_unit = (L.tiles_per_slab + 1) / 2;
+  L.total_units = (int64_t)G.L * G.H * 2 * 2;
+  L.has_src = G.src.k != nullptr;
+  bool ok = tc::encode_cache(&L.maps.tgt_k, G.tgt, G.tgt.k, G.L, G.H) && tc::encode_cache(&L.maps.tgt_v, G.tgt, G.tgt.v, G.L, G.H);
+  if (L.has_src)
+    ok = ok && tc::encode_cache(&L.maps.src_k, G.src, G.src.k, G.L, G.H) && tc::encode_cache(&L.maps.src_v, G.src, G.src.v, G.L, G.H);
+  ok = ok && tc::encode_coeff(&L.maps.coeff_k, const_cast<float*>(G.coeff_k), G.r, G.n_cov, G.L) &&
+       tc::encode_coeff(&L.maps.coeff_v, const_cast<float*>(G.coeff_v), G.r, G.n_cov, G.L);
+  if (!ok) return KVC_E_CUDA;
+  const int sms = tc::sm_count();
+  if (sms <= 0) return KVC_E_CUDA;
+  const int grid = (int)(L.total_units < sms ? L.total_units : sms);
+  constexpr int NS = 2;
+  const size_t smem = 1024 + (size_t)NS * (kStageBytes + 2 * kZBytes) + sizeof(GCtrl<NS>);
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
+    if (cudaFuncSetAttribute(backproject_tc_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+    once.mark(once_dev);
+  }
+  backproject_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
