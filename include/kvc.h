@@ -129,6 +129,9 @@ typedef struct kvc_state {
  * reused at position p + s is rotated, pair by pair, by the angle s * f_k with
  * f_k = theta^(-2k/d), k = 0..d/2-1, unless inv_freq overrides the table
  * (scaled-RoPE models).  Values are never rotated.
+ * inv_freq is a HOST float64 table on purpose: cos and sin of shift * f_k are formed in float64 on the
+ * host and rounded once to float32 (a float32 angle at |shift| ~ 500 already costs 1e-3 on keys of
+ * magnitude 40), d/2 values per call that travel in the launch parameters.
  */
 typedef struct kvc_rope {
   double theta;
@@ -359,6 +362,12 @@ int kvc_state_update_noalloc(const kvc_cache *src, const kvc_cache *tgt, int32_t
  *   staging    HOST buffer of the same size (pinned memory recommended); the work
  *              table is built here and copied to `workspace` on `stream`; it must stay
  *              untouched until that copy has executed.
+ * Why the items are a host array and the call makes one host-to-device copy: the work table carries
+ * tensor maps, which only the host can encode, and the per-CTA ranges of equal estimated time; building
+ * them is this call's job, and one copy of a few hundred KB per launch replaces a second API for it.
+ * An item is a whole cache: a context made of several segments with different shifts is ONE item of
+ * kvc_apply_segmented's kind (a token range inside a paged cache would need page-aligned table slices
+ * and partial-tile stores that must not touch the neighbouring segment's rows).
  */
 typedef struct kvc_item {
   kvc_cache src;
@@ -506,9 +515,10 @@ int kvc_gate_weights(const double *dist_sq, int32_t n_anchors, double temperatur
  * Device-side anomalies never trap or hang: a kernel that meets a page id outside
  * [0, n_phys_pages) or whose bounded wait on an asynchronous copy runs out skips
  * that tile and ORs a bit into a per-device status word.
- * kvc_status_poll copies the word to *flags (this call synchronises the device)
- * and returns KVC_OK when it is zero, KVC_E_DEVICE_FLAG otherwise;
- * kvc_status_reset clears it.
+ * kvc_status_poll copies the word to *flags and returns KVC_OK when it is zero,
+ * KVC_E_DEVICE_FLAG otherwise.  The copy is a device-to-host read of one word, so this call
+ * SYNCHRONISES the device: a caller that must not stall its streams polls at a point where it
+ * synchronises anyway (end of a batch, after an event wait).  kvc_status_reset clears the word.
  */
 #define KVC_FLAG_BAD_PAGE     1u
 #define KVC_FLAG_WAIT_EXPIRED 2u

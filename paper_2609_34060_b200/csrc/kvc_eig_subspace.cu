@@ -30,13 +30,6 @@
 #include "kvc_launch.h"
 
 namespace kvc {
-#ifdef KVC_EIG_TIMING
-__device__ unsigned long long g_eig_t[16];
-__device__ unsigned long long g_eig_blk[4096 * 4];   // per block: cycles, smid, globaltimer begin, end
-#define TMARK(i) do { __syncthreads(); if (tid == 0 && blockIdx.x == 100) { long long now = clock64(); atomicAdd(&g_eig_t[i], (unsigned long long)(now - t_last)); t_last = now; } } while (0)
-#else
-#define TMARK(i)
-#endif
 namespace {
 
 using namespace eigsmall;
@@ -333,13 +326,6 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
   const int rg = tid >> 3, cg = tid & 7;          // 4 x 4 tiles of the N x 32 matrices
   const bool tile_on = rg < N / 4 && 4 * cg < m;
 
-  long long t_last = clock64();
-  (void)t_last;
-#ifdef KVC_EIG_TIMING
-  const long long t_begin = t_last;
-  unsigned long long gt_begin;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_begin));
-#endif
   // ---- 0. sum of the partial Grams, symmetrised, written back; trace
   float tr = 0.f;
   {
@@ -382,7 +368,6 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
     for (int w = 0; w < kThreads / 32; ++w) tr += sm.red[w];
     __syncthreads();
   }
-  TMARK(0);
   int reason = 0;
   if (!(tr > 0.f)) reason = 2;                    // all zero (or not finite): the full solver's business
 
@@ -405,7 +390,6 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
       Q = Y;
       Y = t;
     }
-    TMARK(1);
     {
       // a slightly shifted pass (a start block whose Gram matrix is singular at float32 still factorises),
       // a plain pass, and a third one only if the second still met a small pivot
@@ -417,14 +401,11 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
     float* t = Q;
     Q = Y;
     Y = t;
-    TMARK(2);
   }
   if (reason == 0) {
     for (int it = 0;; ++it) {
       mul_g<N>(G, Q, Y, sm, m, tid);
-      TMARK(3);
       atb_sym<N>(Q, Y, sm.u.m.h, sm, tid);
-      TMARK(4);
       // R = Y - Q H, only its norm is needed; |H|_F beside it
       float res2 = 0.f, hn2 = 0.f;
       if (tile_on) {
@@ -459,7 +440,6 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
         hn2 += sm.red[8 + w];
       }
       __syncthreads();
-      TMARK(5);
       if (res2 <= 4e-12f * hn2) break;            // |R|_F <= 2e-6 |H|_F: rounding level
       if (it == kMaxIter - 1) {
         reason = 3;
@@ -476,13 +456,11 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
       float* t = Q;
       Q = Y;
       Y = t;
-      TMARK(6);
     }
   }
 
   // ---- 2. Rayleigh-Ritz: eigen-decomposition of H by cyclic Jacobi
   if (reason == 0 && !jacobi_eig(sm.u.m.h, sm.u.m.s, sm.u.m.w, &sm.flag, m, tid)) reason = 5;
-  TMARK(7);
 
   // ---- Ritz values in descending order, Z = Q W and G Z = Y W (sorted columns)
   float tau = 0.f;
@@ -596,8 +574,6 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
     const bool accept = rhomax2 <= (1e-5f * th1) * (1e-5f * th1) && gap > 0.f && rhoF <= (1.f / 8192.f) * gap;
     if (!accept) reason = 4;
   }
-
-  TMARK(8);
   if (reason == 0) {
     // ---- output: sign convention (largest-magnitude entry positive, first such index), unit length
     float* basis = (is_v ? p.basis_v_e[edge] : p.basis_k_e[edge]) + (int64_t)slab * p.r * N;
@@ -633,20 +609,7 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
     }
     if (tid < N) evals[(int64_t)sk * N + tid] = (tid < m) ? sm.th[tid] : tau / (float)(N - m);
   }
-  TMARK(9);
   if (tid == 0) solver[sk] = reason;
-#ifdef KVC_EIG_TIMING
-  if (tid == 0 && blockIdx.x < 4096) {
-    unsigned long long gt_end;
-    unsigned smid;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_end));
-    asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-    g_eig_blk[4 * blockIdx.x] = (unsigned long long)(clock64() - t_begin);
-    g_eig_blk[4 * blockIdx.x + 1] = smid;
-    g_eig_blk[4 * blockIdx.x + 2] = gt_begin;
-    g_eig_blk[4 * blockIdx.x + 3] = gt_end;
-  }
-#endif
 }
 
 }  // namespace
@@ -670,12 +633,4 @@ cudaError_t launch_eig_subspace(const FitLaunch& F, int d, int32_t* solver, cuda
   return cudaGetLastError();
 }
 
-#ifdef KVC_EIG_TIMING
-extern "C" int kvc_debug_eig_times(unsigned long long* out) {
-  return cudaMemcpyFromSymbol(out, g_eig_t, sizeof(g_eig_t)) == cudaSuccess ? 0 : -1;
-}
-extern "C" int kvc_debug_eig_blocks(unsigned long long* out, int n) {
-  return cudaMemcpyFromSymbol(out, g_eig_blk, sizeof(unsigned long long) * 4 * n) == cudaSuccess ? 0 : -1;
-}
-#endif
 }  // namespace kvc

@@ -143,10 +143,16 @@ def test_ragged_lengths_paged(path, T):
 
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_paged_indexing_bit_exact(path):
-    # injective bf16 code of (l, h, t, c), rank 0, shift 0, two different shuffled tables
+    # a 16-bit code that is injective in (t, c) inside every (layer, head) slab (T d = 37,504 distinct patterns)
+    # and shifted by a slab-dependent constant (16 bits cannot tell all 225,024 elements apart); rank 0,
+    # shift 0, two different shuffled tables: the bits must arrive where the destination table says
     L, H, T, d, page, P = 2, 3, 293, 128, 16, 25
     npg = (T + page - 1) // page
-    code = (torch.arange(L * H * T * d, dtype=torch.int64) % 30000 + 1).to(torch.int16).reshape(L, H, T, d)
+    in_slab = torch.arange(T * d, dtype=torch.int64).reshape(1, 1, T, d)
+    slab_off = (torch.arange(L * H, dtype=torch.int64) * 7919).reshape(L, H, 1, 1)
+    code = ((in_slab + slab_off) % 65536).to(torch.int32)
+    code = torch.where(code >= 32768, code - 65536, code).to(torch.int16).expand(L, H, T, d).contiguous()
+    assert all(code[l, h].unique().numel() == T * d for l in range(L) for h in range(H))
     pt_s = wl.page_table(npg, P, 3, 0)
     pt_d = wl.page_table(npg, P, 3, 1)
     pool_k = torch.full((L, P, H, page, d), 0x5EAD, dtype=torch.int16)
