@@ -195,7 +195,7 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                eigenvectors (r <= 32), which converges in a few steps when the spectrum has a
  *                gap behind the r-th eigenvalue -- a deviation of rank r over a noise floor.  The
  *                result is accepted only when, in float32, every row satisfies
- *                |G b_j - lambda_j b_j| <= 1e-5 lambda_1 and the residual of the whole block is at most
+ *                |G b_j - lambda_j b_j| <= 3e-5 lambda_1 and the residual of the whole block is at most
  *                2^-13 of the distance between lambda_r and a bound on every eigenvalue outside the
  *                block (trace(G) minus the sum of the block's eigenvalues: G is positive
  *                semi-definite); any other matrix is solved by KVC_FIT's full eigensolver in the same
@@ -209,7 +209,8 @@ int kvc_chain(const kvc_cache *agent0, int32_t n_agents, const int32_t *prefix_l
  *                eigenvectors of G = Delta^T Delta by three applications of G, each one the grouped
  *                projection pass Z = Delta Q^T followed by a back-projection pass Y = Z^T Delta, with an
  *                orthonormalisation of the r rows in between and a Rayleigh-Ritz step at the end
- *                (7 streaming passes over the two caches with the final projection).  A block that the
+ *                (6 streaming passes over the two caches; the final coefficients are the last projection's
+ *                times the Rayleigh-Ritz rotation, a pass over the coefficients only).  A block that the
  *                step finds merely slow (its hashed start was unlucky) gets up to two further rounds of
  *                orthonormalisation, application and Rayleigh-Ritz; their kernels are always launched and
  *                return at once when the round is not needed (nothing is read back to the host).
@@ -547,7 +548,7 @@ int kvc_last_path(void);
 /* Algorithmic HBM bytes one hop moves (reads + writes of caches, coefficients and
  * bases), the figure the roofline is reported against.  For the FIT modes: two passes over
  * the source and target rows (one for the Gram matrix, one for the projection), however many
- * the implementation makes (the layer-grouped fit makes seven). */
+ * the implementation makes (the layer-grouped fit makes six). */
 int64_t kvc_apply_bytes(const kvc_cache *src, const kvc_state *st);
 int64_t kvc_update_bytes(const kvc_cache *tgt, const kvc_state *st, int32_t mode, int32_t has_src);
 

@@ -340,14 +340,17 @@ static size_t group_ypart_offset(const kvc_cache* tgt) {
 static size_t group_trpart_offset(const kvc_cache* tgt, int r) {
   return group_ypart_offset(tgt) + (size_t)kGroupFitParts * tgt->L * 2 * r * tgt->H * tgt->d * sizeof(float);
 }
+static size_t group_mtx_offset(const kvc_cache* tgt, int r);
 static size_t group_flags_offset(const kvc_cache* tgt, int r) {
   return (group_trpart_offset(tgt, r) + (size_t)kGroupFitTraceParts * tgt->L * 2 * tgt->H * sizeof(float) + 255) & ~(size_t)255;
 }
 
+static size_t group_mtx_offset(const kvc_cache* tgt, int r) { return group_flags_offset(tgt, r) + 256; }
+
 size_t kvc_workspace_bytes(const kvc_cache* tgt, const kvc_state* st, int32_t mode) {
   if (!tgt || !st || (mode != KVC_FIT && mode != KVC_FIT_FAST)) return 0;
   if (st->grouping == KVC_GROUP_LAYER)
-    return group_flags_offset(tgt, st->r) + 256;
+    return group_mtx_offset(tgt, st->r) + (size_t)tgt->L * 2 * 32 * 32 * sizeof(float);
   if (mode == KVC_FIT) return fit_evals_end(tgt);
   return fit_solver_offset(tgt) + (size_t)tgt->L * tgt->H * 2 * sizeof(int32_t);
 }
@@ -479,8 +482,13 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, c
   rope_tables(P.rope, d, P.shift, U.cs, U.sn);
   if (U.grouped) {      // every head adds its share: start from zero
     const size_t nbytes = (size_t)P.L * st->n_cov * st->r * sizeof(float);
-    if (cudaMemsetAsync(st->coeff_k, 0, nbytes, s) != cudaSuccess || cudaMemsetAsync(st->coeff_v, 0, nbytes, s) != cudaSuccess)
+    if (run_if) {       // a pass that may turn out not to be needed must then leave the coefficients alone
+      const int64_t n = (int64_t)P.L * st->n_cov * st->r;
+      if (launch_zero_if(st->coeff_k, n, run_if, s) != cudaSuccess || launch_zero_if(st->coeff_v, n, run_if, s) != cudaSuccess)
+        return KVC_E_CUDA;
+    } else if (cudaMemsetAsync(st->coeff_k, 0, nbytes, s) != cudaSuccess || cudaMemsetAsync(st->coeff_v, 0, nbytes, s) != cudaSuccess) {
       return KVC_E_CUDA;
+    }
   }
   if (P.seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
   if (tl_path_force != KVC_PATH_GENERIC && !P.seg) {
@@ -518,6 +526,9 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   G.ypart = reinterpret_cast<float*>(ws + group_ypart_offset(tgt));
   G.trpart = reinterpret_cast<float*>(ws + group_trpart_offset(tgt, st->r));
   G.need_more = reinterpret_cast<int32_t*>(ws + group_flags_offset(tgt, st->r));
+  G.mtx = reinterpret_cast<float*>(ws + group_mtx_offset(tgt, st->r));
+  G.coeff_k_rw = st->coeff_k;
+  G.coeff_v_rw = st->coeff_v;
   G.r = st->r;
   G.n_cov = st->n_cov;
   G.pairing = P.rope->pairing;
@@ -566,7 +577,9 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
     }
     if (launch_group_small(G, KVC_GROUP_OP_RITZ, s) != cudaSuccess) return KVC_E_CUDA;
   }
-  return KVC_OK;
+  // the coefficients of the final rows: those of the rows the last Rayleigh-Ritz step started from, times its
+  // rotation (a pass over the coefficients only, instead of one more projection pass over the caches)
+  return launch_group_coeff_transform(G, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
 static int update_planned(UpdatePlan& P, const kvc_cache* tgt, kvc_state* st, int32_t mode, void* workspace,
@@ -603,9 +616,8 @@ static int update_planned(UpdatePlan& P, const kvc_cache* tgt, kvc_state* st, in
   uint32_t* status = status_ptr();
   if (!status) return KVC_E_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  if (P.fit && st->grouping == KVC_GROUP_LAYER) {
-    if ((rc = group_fit_edge(P, tgt, workspace, status, s)) != KVC_OK) return rc;
-  } else if (P.fit) {
+  if (P.fit && st->grouping == KVC_GROUP_LAYER) return group_fit_edge(P, tgt, workspace, status, s);
+  if (P.fit) {
     FitLaunch F;
     if ((rc = fit_gram(P, workspace, status, &F, s)) != KVC_OK) return rc;
     const size_t solver_bytes = (size_t)P.L * P.H * 2 * sizeof(int32_t);

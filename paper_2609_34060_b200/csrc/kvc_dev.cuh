@@ -123,6 +123,9 @@ struct GroupFitLaunch {        // FIT of states grouped by layer (D = H d): back
   float* evals;                // [L*2][H d]
   int32_t* solver;             // [L*2] per-problem code
   int32_t* need_more;          // [kGroupFitRounds + 1]: round k runs only when need_more[k] != 0 (round 0 always)
+  float* mtx;                  // [L*2][32][32]: coefficients of the final rows = (last Z) . mtx, written by the Rayleigh-Ritz step
+  float* coeff_k_rw;           // the state's coefficient buffers once more, writable (the final transform runs in place)
+  float* coeff_v_rw;
   int32_t r, n_cov, pairing, shift, L, H, d, parts, tokens_per_part;
   int32_t round, last_round;
   int32_t tr_parts;            // partial sums of the trace: parts (CUDA-core pass) or 32 (tensor-core pass: half x team warp)

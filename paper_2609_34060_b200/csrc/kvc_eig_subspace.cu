@@ -14,8 +14,8 @@
 //      at once: a 16 x 16 array of threads, each holding one 2 x 2 block of H and of W in registers,
 //      the rows and columns moving one place along the round-robin cycle after every step;
 //      Z = Q W with the columns sorted by theta, theta_j refreshed as the Rayleigh quotient of z_j;
-//   3. a-posteriori test on the rows that would be written:  rho_j = |G z_j - theta_j z_j| at rounding
-//      level for every j, and  |rho|_F <= 2^-13 (theta_r - tau - |rho|_F)  with tau = trace(G) - sum theta
+//   3. a-posteriori test on the rows that would be written:  rho_j = |G z_j - theta_j z_j| <= 3e-5 theta_1
+//      for every j, and  |rho|_F <= 2^-13 (theta_r - tau - |rho|_F)  with tau = trace(G) - sum theta
 //      (G is positive semi-definite, so no eigenvalue outside the block exceeds tau + |rho|_F: the block
 //      holds the r largest and its subspace is off by at most that ratio).
 // A matrix that passes gets its basis rows, its r largest eigenvalues and, for the other d - r, their
@@ -440,7 +440,7 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
         hn2 += sm.red[8 + w];
       }
       __syncthreads();
-      if (res2 <= 4e-12f * hn2) break;            // |R|_F <= 2e-6 |H|_F: rounding level
+      if (res2 <= 36e-12f * hn2) break;           // |R|_F <= 6e-6 |H|_F: every row then passes the acceptance test below
       if (it == kMaxIter - 1) {
         reason = 3;
         break;
@@ -571,7 +571,7 @@ __global__ void __launch_bounds__(kThreads, 4) eig_subspace_kernel(const __grid_
     tau = fmaxf(tr - sumth, 0.f);
     const float rhoF = sqrtf(rhoF2);
     const float gap = thm - tau - rhoF;
-    const bool accept = rhomax2 <= (1e-5f * th1) * (1e-5f * th1) && gap > 0.f && rhoF <= (1.f / 8192.f) * gap;
+    const bool accept = rhomax2 <= (3e-5f * th1) * (3e-5f * th1) && gap > 0.f && rhoF <= (1.f / 8192.f) * gap;
     if (!accept) reason = 4;
   }
   if (reason == 0) {

@@ -295,6 +295,7 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
     // a zero deviation (or rows that became dependent): no basis, all eigenvalues zero
     for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) Q[i] = 0.f;
     for (int i = tid; i < Dg; i += kThreads) evals[i] = 0.f;
+    for (int i = tid; i < kMaxM * kMaxM; i += kThreads) p.mtx[(int64_t)prob * kMaxM * kMaxM + i] = 0.f;
     if (tid == 0) {
       *code = KVC_SOLVER_FULL_DEPENDENT;
       if (tr > 0.f) atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
@@ -404,6 +405,12 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
     sm.inv[tid] = live ? sgn * rsqrtf(fmaxf(ds, 1e-30f)) : 0.f;
   }
   __syncthreads();
+  // the coefficients of the final rows follow from those of the rows they were formed from:
+  // row_j = inv_j sum_k Ws[k][j] q_k   =>   c'_j = inv_j sum_k Ws[k][j] c_k
+  for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
+    const int k = i >> 5, j = i & 31;
+    p.mtx[(int64_t)prob * kMaxM * kMaxM + i] = (k < m && j < m) ? Ws[k * kSP + j] * sm.inv[j] : 0.f;
+  }
   // pass 2: residuals |G z_j - theta_j z_j|^2 of the unit-length rows, and the rows written out
   for (int c0 = 0; c0 < Dg; c0 += kThreads) {
     const int c = c0 + tid;
@@ -451,7 +458,51 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
   }
 }
 
+// coeff[l][t][:] <- coeff[l][t][:] . M  for every covered token: the coefficients of the final rows from those of
+// the rows the last Rayleigh-Ritz step started from.  One thread per token, M in shared memory.
+__global__ void __launch_bounds__(kThreads) group_coeff_transform_kernel(const __grid_constant__ GroupFitLaunch p) {
+  __shared__ float M[kMaxM * kMaxM];
+  const int prob = blockIdx.y, l = prob >> 1, is_v = prob & 1;
+  for (int i = threadIdx.x; i < kMaxM * kMaxM; i += kThreads) M[i] = p.mtx[(int64_t)prob * kMaxM * kMaxM + i];
+  __syncthreads();
+  const int t = blockIdx.x * kThreads + threadIdx.x;
+  if (t >= p.n_cov) return;
+  float* row = (is_v ? p.coeff_v_rw : p.coeff_k_rw) + ((int64_t)l * p.n_cov + t) * p.r;
+  float c[kMaxM], o[kMaxM];
+#pragma unroll
+  for (int k = 0; k < kMaxM; ++k) c[k] = (k < p.r) ? row[k] : 0.f;
+#pragma unroll
+  for (int j = 0; j < kMaxM; ++j) o[j] = 0.f;
+#pragma unroll
+  for (int k = 0; k < kMaxM; ++k)
+#pragma unroll
+    for (int j = 0; j < kMaxM; ++j) o[j] = fmaf(c[k], M[k * kMaxM + j], o[j]);
+#pragma unroll
+  for (int j = 0; j < kMaxM; ++j)
+    if (j < p.r) row[j] = o[j];
+}
+
+// ptr[0 .. n) <- 0 unless a run flag is given and zero (the start of a projection pass that adds into its output)
+__global__ void zero_if_kernel(float* ptr, int64_t n, const int32_t* run_if) {
+  if (run_if != nullptr && *run_if == 0) return;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) ptr[i] = 0.f;
+}
+
 }  // namespace
+
+cudaError_t launch_zero_if(float* ptr, int64_t n, const int32_t* run_if, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  const int blocks = (int)((n + 256 * 8 - 1) / (256 * 8) < 1184 ? (n + 256 * 8 - 1) / (256 * 8) : 1184);
+  zero_if_kernel<<<blocks, 256, 0, s>>>(ptr, n, run_if);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_group_coeff_transform(const GroupFitLaunch& G, cudaStream_t s) {
+  if (G.n_cov <= 0 || G.L <= 0) return cudaSuccess;
+  dim3 grid((unsigned)((G.n_cov + kThreads - 1) / kThreads), (unsigned)(G.L * 2));
+  group_coeff_transform_kernel<<<grid, kThreads, 0, s>>>(G);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_group_backproject(const GroupFitLaunch& G, const SegTable* seg, cudaStream_t s) {
   const int blocks = G.L * G.H * 2 * G.parts;

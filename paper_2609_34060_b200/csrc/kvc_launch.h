@@ -66,6 +66,8 @@ constexpr int kGroupFitParts = 4;   // token ranges whose back-projections are s
 constexpr int kGroupFitTraceParts = 32;   // room for the partial sums of the trace (tensor-core pass: half x team warp)
 cudaError_t launch_group_backproject(const GroupFitLaunch& G, const SegTable* seg, cudaStream_t s);
 cudaError_t launch_group_small(const GroupFitLaunch& G, int op, cudaStream_t s);
+cudaError_t launch_group_coeff_transform(const GroupFitLaunch& G, cudaStream_t s);
+cudaError_t launch_zero_if(float* ptr, int64_t n, const int32_t* run_if, cudaStream_t s);
 
 // reliability gate (kvc_gate.cu)
 cudaError_t launch_gate_generic(const GateLaunch& g, int d, cudaStream_t s);
