@@ -175,6 +175,97 @@ def test_state_update_full_size_sampled_slabs(name):
             assert res <= 1.001 * float(np.sum(w[r:])) + 1e-6 * float(np.sum(w)), (res, float(np.sum(w[r:])))
 
 
+def test_chain_update_full_size_as_benchmarked():
+    """The state update exactly as bench.py times it: kvc_state_update_chain(KVC_FIT_FAST) over the three
+    edges of the 8K config (one eigensolver launch for 1536 matrices).  Properties of every decomposition on
+    the device with library routines, and sampled slabs of every edge against the oracle."""
+    from paper_2609_34060_b200 import scenarios as sc
+    cfg = wl.CONFIGS["llama8b_8k"]
+    kvc.kvc_status_reset()
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    W = sc.build_workload(cfg, DEV, "update")
+    pl, rope, true, states = W["pl"], W["rope"], W["true"], W["states"]
+    f = hp.inv_freq(cfg)
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+    W["ws"].zero_()
+    kvc.kvc_state_update_chain(true, pl, rope, states, kvc.KVC_FIT_FAST, workspace=W["ws"])
+    torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == kvc.KVC_PATH_TC and kvc.kvc_status_poll() == 0
+    stride = kvc.kvc_chain_update_edge_stride(true[1], states[0], kvc.KVC_FIT_FAST)
+    eye = torch.eye(r, device=DEV, dtype=torch.float64)
+    m = L * H * 2
+    for e in range(cfg.n_agents - 1):
+        ws = W["ws"][e * stride:(e + 1) * stride]
+        solver = kvc.kvc_fit_solver(true[e + 1], ws)
+        assert int((solver == kvc.KVC_SOLVER_SUBSPACE).sum()) == m          # rank-32 deviations over a noise floor
+        wsf = ws.view(torch.float32)
+        G_all = wsf[: m * d * d].view(L, H, 2, d, d)
+        ev_all = wsf[2 * m * d * d: 2 * m * d * d + m * d].view(L, H, 2, d)
+        for i, Bt in enumerate((states[e].basis_k, states[e].basis_v)):
+            B64 = Bt.to(torch.float64)
+            assert float((B64 @ B64.transpose(-1, -2) - eye).abs().max()) <= 1e-4
+            ev64 = ev_all[:, :, i].to(torch.float64)
+            top = ev64[..., :1]
+            assert bool(((ev64[..., 1:] - ev64[..., :-1]) <= 1e-6 * top).all())
+            G64 = G_all[:, :, i].to(torch.float64)
+            tr = torch.diagonal(G64, dim1=-2, dim2=-1).sum(-1)
+            assert float(((ev64.sum(-1) - tr).abs() / tr).max()) <= 1e-4
+            rq = torch.einsum("lhrd,lhde,lhre->lhr", B64, G64, B64)
+            assert float(((rq - ev64[..., :r]).abs() / top).max()) <= 1e-4
+            # every row is an eigenvector of the Gram matrix the call left behind, to the solver's stated level
+            res = torch.einsum("lhrd,lhde->lhre", B64, G64) - rq[..., None] * B64
+            assert float((res.norm(dim=-1) / top).max()) <= 1e-4
+        for (l, h) in _sample_slabs(cfg, n=1):
+            for i, (which, Bt, ct) in enumerate((("k", states[e].basis_k, states[e].coeff_k), ("v", states[e].basis_v, states[e].coeff_v))):
+                dl = orc.deviation(_slab_bits(true[e], which, l, h), _slab_bits(true[e + 1], which, l, h), pl[e + 1] - pl[e], f, which == "k")
+                Gref = orc.gram(dl)
+                dg = np.sqrt(np.diag(Gref))
+                G = G_all[l, h, i].cpu().numpy().astype(np.float64)
+                assert np.max(np.abs(G - Gref) / (2.0 ** -12 * np.outer(dg, dg) + 1e-6)) <= 1.0
+                w = np.linalg.eigvalsh(Gref)[::-1]
+                ev = ev_all[l, h, i].cpu().numpy().astype(np.float64)
+                assert np.max(np.abs(ev[:r] - w[:r])) <= 1e-4 * w[0]
+                B = Bt[l, h].cpu().numpy().astype(np.float64)
+                c = ct[l, h].cpu().numpy().astype(np.float64)
+                res = float(np.sum((dl - c @ B) ** 2))
+                assert res <= 1.001 * float(np.sum(w[r:])) + 1e-6 * float(np.sum(w)), (e, l, h, which)
+
+
+def test_grouped_fit_full_size_sampled_layers():
+    """FIT under D = H d = 1024 at the 8K config's size (one edge): every matrix accepted, orthonormal rows
+    everywhere, and two sampled layers against a library eigensolver on the oracle's 1024 x 1024 Gram matrix."""
+    from paper_2609_34060_b200 import scenarios as sc
+    cfg = wl.CONFIGS["llama8b_8k"].scaled(n_agents=2)
+    kvc.kvc_status_reset()
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    W = sc.build_workload(cfg, DEV, "update", grouped=True)
+    pl, rope, true, st = W["pl"], W["rope"], W["true"], W["states"][0]
+    f = hp.inv_freq(cfg)
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+    ws = torch.zeros(kvc.kvc_workspace_bytes(true[1], st, kvc.KVC_FIT), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(true[0], true[1], pl[1] - pl[0], rope, st, kvc.KVC_FIT, workspace=ws)
+    torch.cuda.synchronize()
+    assert kvc.kvc_status_poll() == 0
+    assert bool((kvc.kvc_group_fit_solver(true[1], ws) == 0).all())
+    eye = torch.eye(r, device=DEV, dtype=torch.float64)
+    for Bt in (st.basis_k, st.basis_v):
+        B64 = Bt.to(torch.float64)
+        assert float((B64 @ B64.transpose(-1, -2) - eye).abs().max()) <= 2e-5
+    ev = kvc.kvc_group_fit_eigenvalues(true[1], ws).cpu().numpy().astype(np.float64)
+    for l in (0, L - 1):
+        for i, (which, Bt, ct) in enumerate((("k", st.basis_k, st.coeff_k), ("v", st.basis_v, st.coeff_v))):
+            cat = np.concatenate([orc.deviation(_slab_bits(true[0], which, l, h), _slab_bits(true[1], which, l, h), pl[1] - pl[0], f, which == "k")
+                                  for h in range(H)], axis=1)
+            w, V = np.linalg.eigh(orc.gram(cat))
+            w, V = w[::-1], V[:, ::-1]
+            assert np.max(np.abs(ev[l, i, :r] - w[:r])) <= 2e-4 * w[0]
+            B = Bt[l].cpu().numpy().astype(np.float64)
+            c = ct[l].cpu().numpy().astype(np.float64)
+            assert np.linalg.norm(B.T @ B - V[:, :r] @ V[:, :r].T) <= 1e-2
+            res = float(np.sum((cat - c @ B) ** 2))
+            assert res <= 1.001 * float(np.sum(w[r:])) + 1e-6 * float(np.sum(w)), (l, which)
+
+
 def _free_gb():
     import gc
     gc.collect()
