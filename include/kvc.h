@@ -299,9 +299,11 @@ size_t kvc_chain_update_edge_stride(const kvc_cache *tgt, const kvc_state *st, i
  *            Values are never rotated: the two agree for them.
  * The lists are host arrays on purpose: the cos / sin tables of every segment are formed in float64 on the
  * host, exactly like the single shift's, and travel in the launch parameters (a device position array would
- * need sincos per token and frequency inside the kernels).  These entry points are served by the CUDA-core
- * kernel family (KVC_PATH_TC forced: KVC_E_UNSUPPORTED); everything else is as in kvc_apply / kvc_state_update,
- * including layer-grouped states and the FIT modes.
+ * need sincos per token and frequency inside the kernels).  kvc_apply_segmented runs on the tensor-core
+ * kernel where kvc_apply does (every row picks its segment's table in the epilogue); the passes of
+ * kvc_state_update_segmented over the caches are served by the CUDA-core kernel family (KVC_PATH_TC forced:
+ * KVC_E_UNSUPPORTED).  Everything else is as in kvc_apply / kvc_state_update, including layer-grouped states
+ * and the FIT modes.
  */
 #define KVC_MAX_SEGMENTS   16
 #define KVC_COORDS_TARGET  0

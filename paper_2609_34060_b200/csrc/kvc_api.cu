@@ -202,10 +202,9 @@ static int apply_resolved(ResolvedHop& hop, int pairing, cudaStream_t s, const S
   if (!status) return KVC_E_CUDA;
   const int T = hop.item.src.T;
   if (T == 0) return KVC_OK;
-  if (seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;   // segment tables: CUDA-core kernels only
-  const bool want_tc = tl_path_force != KVC_PATH_GENERIC && !seg;
+  const bool want_tc = tl_path_force != KVC_PATH_GENERIC;
   if (want_tc) {
-    const int trc = tc_apply_single(hop.item, hop.d, pairing, status, s);
+    const int trc = tc_apply_single(hop.item, hop.d, pairing, status, s, seg);
     if (trc == KVC_OK) {
       tl_last_path = KVC_PATH_TC;
       return KVC_OK;
@@ -251,7 +250,6 @@ int kvc_apply_segmented(const kvc_cache* src, const kvc_state* st, const kvc_seg
   if (rc != KVC_OK) return rc;
   ResolvedHop hop;
   if ((rc = resolve_hop(src, st, segs->shift[0], rope, dst, &hop)) != KVC_OK) return rc;
-  if (st && st->grouping == KVC_GROUP_LAYER && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
   return apply_resolved(hop, rope->pairing, reinterpret_cast<cudaStream_t>(stream), &seg);
 }
 

@@ -10,7 +10,7 @@
 
 namespace kvc {
 
-int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s);
+int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s, const SegTable* seg = nullptr);
 int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, cudaStream_t s);
 int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* sn2, uint32_t* status, float* row_out,
                     int64_t t_pad, cudaStream_t s);

@@ -241,14 +241,18 @@ __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_
 // MODE 2, row distance (token weights of App. A.3): key and value slabs; per token the mean of
 //         |src - c.B| over layers, heads and channels is accumulated in row_out, keys after both
 //         sides were rotated into canonical positional coordinates.
-template <int RB, int NSTAGE, int NSC, int MODE = 0>
-__global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
+// MODE 0: apply; 1: gate distance; 2: row distances; 3: apply with a segment table (per-row shift and
+// tables, correction before or after the rotation) - the table is a second launch parameter of its own
+// kernel, so the other launches do not carry it.
+template <int RB, int NSTAGE, int NSC, int MODE>
+__device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegTable* segp) {
   constexpr bool GATE = MODE == 1;                // walks value slabs only
+  constexpr bool SEG = MODE == 3;
   // The epilogue works on packed float32 pairs except in the configuration of a contiguous source with
   // r <= 32, which runs at the HBM roof either way and measured 0.7 % slower with them (the paged and
   // r = 64 configurations, bound by the team's instruction stream, gain 3 %).
   constexpr bool kPackedEpilogue = !(RB == 1 && NSTAGE == 5 && NSC == 2);
-  constexpr bool REDUCE = MODE != 0;              // no stores
+  constexpr bool REDUCE = MODE == 1 || MODE == 2;   // no stores
   constexpr int kStageBytes = kBaseBytes;
   constexpr int kCoeffSlotBytes = RB * kCoeffBlkBytes;
   constexpr int kBasisSlotBytes = RB * kBasisBlkBytes;
@@ -637,7 +641,17 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
       const int tok = t.t0 + m;
       const bool in_range = tok < it.src.T;
       const bool covered = t.has_coeff && tok < it.st.n_cov;
-      const bool rotate = !t.is_v && it.shift != 0;
+      bool rotate = !t.is_v && it.shift != 0;
+      const float* csp = it.cs;
+      const float* snp = it.sn;
+      bool at_source = false;
+      if constexpr (SEG) {                          // this row's segment: its own shift and tables
+        const int k = seg_index(*segp, tok);
+        csp = segp->cs[k];
+        snp = segp->sn[k];
+        rotate = !t.is_v && segp->shifted[k] != 0;
+        at_source = segp->coords == 1;
+      }
       const bool work = in_range && (covered || rotate);
       const uint32_t t_acc = tmem_base + g * 128 + ((uint32_t)(q * 32) << 16);
       float a0[16], a1[16];
@@ -748,9 +762,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
                 xa[z] = f2_from_bf16x2(wa[z]);
                 xb[z] = f2_from_bf16x2(wb[z]);
               }
+              if (SEG && covered && at_source) {       // the correction lives at the source's positions: add, then rotate
+  #pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  xa[z] = f2_add(xa[z], f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
+                  xb[z] = f2_add(xb[z], f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]));
+                }
+              }
               if (rotate) {
-                const float4 c0 = *reinterpret_cast<const float4*>(it.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
-                const float4 s0 = *reinterpret_cast<const float4*>(it.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
+                const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
+                const float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
                 const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
                 const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
                 const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
@@ -761,7 +782,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
                   xb[z] = f2_fma(u, sn[z], f2_mul(v, cs[z]));            // u sin + v cos
                 }
               }
-              if (covered) {
+              if (covered && !(SEG && at_source)) {
   #pragma unroll
                 for (int z = 0; z < 4; ++z) {
                   xa[z] = f2_add(xa[z], f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
@@ -774,9 +795,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
               float x[16];
               unpack8(*p0, x);
               unpack8(*p1, x + 8);
+              if (SEG && covered && at_source) {
+  #pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                  x[k] += a0[8 * jj + k];
+                  x[8 + k] += a1[8 * jj + k];
+                }
+              }
               if (rotate) {
-                const float4 c0 = *reinterpret_cast<const float4*>(it.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
-                const float4 s0 = *reinterpret_cast<const float4*>(it.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
+                const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
+                const float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
                 const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
                 const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
   #pragma unroll
@@ -786,7 +814,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
                   x[8 + k] = u * sn[k] + v * cs[k];
                 }
               }
-              if (covered) {
+              if (covered && !(SEG && at_source)) {
   #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                   x[k] += a0[8 * jj + k];
@@ -806,10 +834,14 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
             uint4* pp = reinterpret_cast<uint4*>(rowp + ((j ^ sw) << 4));
             float x[8];
             unpack8(*pp, x);
+            if (SEG && covered && at_source) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) x[k] += (jj < 2) ? a0[8 * jj + k] : a1[8 * (jj - 2) + k];
+            }
             if (rotate) {
               const int f0 = 16 * cq + 4 * jj;         // pair index of the chunk's first pair
-              const float4 c0 = *reinterpret_cast<const float4*>(it.cs + f0);
-              const float4 s0 = *reinterpret_cast<const float4*>(it.sn + f0);
+              const float4 c0 = *reinterpret_cast<const float4*>(csp + f0);
+              const float4 s0 = *reinterpret_cast<const float4*>(snp + f0);
               const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
               const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
 #pragma unroll
@@ -819,7 +851,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
                 x[2 * k + 1] = u * sn[k] + v * cs[k];
               }
             }
-            if (covered) {
+            if (covered && !(SEG && at_source)) {
 #pragma unroll
               for (int k = 0; k < 8; ++k) x[k] += (jj < 2) ? a0[8 * jj + k] : a1[8 * (jj - 2) + k];
             }
@@ -847,6 +879,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_cons
     tc_fence_after();
     tmem_dealloc(tmem_base, 256);
   }
+}
+
+template <int RB, int NSTAGE, int NSC, int MODE = 0>
+__global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
+  apply_tc_body<RB, NSTAGE, NSC, MODE>(p, nullptr);
+}
+template <int RB, int NSTAGE, int NSC>
+__global__ void __launch_bounds__(kThreads, 1) apply_tc_seg_kernel(const __grid_constant__ ApplyTcLaunch p,
+                                                                   const __grid_constant__ SegTable seg) {
+  apply_tc_body<RB, NSTAGE, NSC, 3>(p, &seg);
 }
 
 // ------------------------------------------------------------------ host side
@@ -891,14 +933,33 @@ static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+template <int RB, int NSTAGE, int NSC>
+static cudaError_t launch_seg_t(const ApplyTcLaunch& L, const SegTable& seg, int grid, cudaStream_t s) {
+  constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
+                          sizeof(Ctrl<NSTAGE, NSC>);
+  static DeviceOnce once;
+  int once_dev;
+  if (once.pending(&once_dev)) {
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_seg_kernel<RB, NSTAGE, NSC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    once.mark(once_dev);
+  }
+  apply_tc_seg_kernel<RB, NSTAGE, NSC><<<grid, kThreads, smem, s>>>(L, seg);
+  return cudaGetLastError();
+}
+
 // Ring depths by measurement: with one rank block, a contiguous source streams best with two
 // coefficient slots (0.98 of the copy bandwidth against 0.84 with three), a paged one with three
 // (0.925 against 0.906); two rank blocks leave room for four base and two coefficient slots.
-static int launch(const ApplyTcLaunch& L, int max_r, bool paged, cudaStream_t s, int grid = 0) {
+static int launch(const ApplyTcLaunch& L, int max_r, bool paged, cudaStream_t s, int grid = 0, const SegTable* seg = nullptr) {
   if (grid <= 0) {
     const int sms = sm_count();
     if (sms <= 0) return KVC_E_CUDA;
     grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
+  }
+  if (seg) {      // per-row tables: the paged ring depths (three coefficient slots) for one rank block
+    cudaError_t es = (max_r > 32) ? launch_seg_t<2, 4, 2>(L, *seg, grid, s) : launch_seg_t<1, 5, 3>(L, *seg, grid, s);
+    return es == cudaSuccess ? KVC_OK : KVC_E_CUDA;
   }
   cudaError_t e = (max_r > 32) ? launch_t<2, 4, 2>(L, grid, s)
                                : (paged ? launch_t<1, 5, 3>(L, grid, s) : launch_t<1, 5, 2>(L, grid, s));
@@ -927,7 +988,7 @@ static_assert(alignof(DevItem) >= 16 && sizeof(DevItem) % 16 == 0, "items in a t
 static_assert(offsetof(tc::ApplyTcLaunch, one) % 16 == 0, "the by-value item must keep the alignment");
 static_assert(offsetof(tc::ApplyTcLaunch, one_maps) % 64 == 0, "tensor maps need 64-byte alignment");
 
-int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s) {
+int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, cudaStream_t s, const SegTable* seg) {
   if (!tc::item_supported(item, d) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
   tc::ApplyTcLaunch L;
   memset(&L, 0, sizeof(L));
@@ -939,7 +1000,7 @@ int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, c
   L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
   L.status = status;
   if (L.total_tiles == 0) return KVC_OK;
-  return tc::launch(L, item.st.r, item.src.page_table != nullptr, s);
+  return tc::launch(L, item.st.r, item.src.page_table != nullptr, s, 0, seg);
 }
 
 namespace tc {

@@ -32,9 +32,11 @@ def _clean_status():
     assert kvc.kvc_status_poll() == 0
 
 
+@pytest.mark.parametrize("path", [kvc.KVC_PATH_GENERIC, kvc.KVC_PATH_AUTO], ids=["generic", "auto"])
 @pytest.mark.parametrize("coords", COORDS, ids=["target", "source"])
 @pytest.mark.parametrize("cfg", [CFG_C, CFG_P, CFG_T], ids=lambda c: c.name)
-def test_apply_segmented(cfg, coords):
+def test_apply_segmented(cfg, coords, path):
+    kvc.kvc_set_path(path)
     t_begin, shift = SEGS[cfg.name]
     s_tok = orc.segment_shifts(cfg.T, t_begin, shift)
     f = hp.inv_freq(cfg)
@@ -45,6 +47,7 @@ def test_apply_segmented(cfg, coords):
     kvc.kvc_apply_segmented(hp.to_dev(src_cpu, DEV), hp.state_to_dev(st_cpu, DEV), kvc.Segments(t_begin, shift, coords),
                             kvc.Rope(cfg.theta), dst)
     torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == (kvc.KVC_PATH_TC if (path == kvc.KVC_PATH_AUTO and cfg.d == 128) else kvc.KVC_PATH_GENERIC)
     osrc, ost = hp.oracle_cache(src_cpu), hp.oracle_state(st_cpu)
     for which in ("k", "v"):
         got = hp.logical_bits(dst, which)
@@ -169,9 +172,10 @@ def test_segment_argument_errors():
         with pytest.raises(kvc.KvcError) as e:
             kvc.kvc_apply_segmented(src, st, bad, rope, dst)
         assert e.value.code == kvc.KVC_E_INVALID_ARG
+    # the update passes with segment tables are CUDA-core kernels: forcing the tensor-core family is refused
     kvc.kvc_set_path(kvc.KVC_PATH_TC)
     with pytest.raises(kvc.KvcError) as e:
-        kvc.kvc_apply_segmented(src, st, kvc.Segments([0, 9], [1, 2]), rope, dst)
+        kvc.kvc_state_update_segmented(src, src, kvc.Segments([0, 9], [1, 2]), rope, st, kvc.KVC_PROJECT)
     assert e.value.code == kvc.KVC_E_UNSUPPORTED
 
 
