@@ -220,6 +220,22 @@ def test_memory_example_from_the_paper():
     lr = orc.lowrank_state_bytes(V, N, tok, L, Hkv, hd, r=32)
     per_matrix = 32 * (tok + hd) * 4
     assert lr == V * (1 + N) * 2 * L * Hkv * per_matrix
+    # counted, not computed: allocate a tiny pool's factors (a base factorisation and N corrections per
+    # anchor, keys and values, one state per (layer, KV head)) and add up what the arrays occupy
+    v, n, t, l, h, d, r = 3, 2, 7, 2, 3, 8, 4
+    arrays = []
+    for _anchor in range(v):
+        for _state in range(1 + n):
+            for _kv in range(2):
+                arrays.append(np.zeros((l, h, t, r), np.float32))       # coefficients
+                arrays.append(np.zeros((l, h, r, d), np.float32))       # basis
+    assert orc.lowrank_state_bytes(v, n, t, l, h, d, r) == sum(a.nbytes for a in arrays)
+    full = [np.zeros((l, h, t, d), np.float16) for _ in range(v * (1 + n) * 2)]   # 2-byte elements, like bf16
+    assert orc.full_state_bytes(v, n, t, l, h, d, 2) == sum(a.nbytes for a in full)
+    # the scaling the paper states: for long segments the ratio full / low-rank tends to D b_full / (r b_coeff)
+    big = 1 << 22
+    ratio = orc.full_state_bytes(1, 1, big, 1, 1, 128, 2) / orc.lowrank_state_bytes(1, 1, big, 1, 1, 128, 32)
+    assert abs(ratio - 128 * 2 / (32 * 4)) < 1e-3
 
 
 def test_token_weights_pins():
@@ -390,3 +406,42 @@ def test_grouped_fit_matches_library_svd():
     assert all(np.max(np.abs(orc.project(exact[:, h * d:(h + 1) * d], per_head[h]) @ per_head[h]
                              - exact[:, h * d:(h + 1) * d])) <= 1e-12 for h in range(H))
     assert not np.allclose(orc.project(exact[:, :d], per_head[0]), ce)
+
+
+def test_state_update_fit_wrapper_against_library_svd():
+    """state_update(FIT) as a whole (the covered prefix, the float32 storage of the basis that then
+    projects, keys against the aligned source, values unshifted) against a library SVD of deviations
+    re-derived here with scalar rotations: the coefficient Gram matrix carries the squared singular
+    values, coeff . basis is the best rank-r approximation of the covered rows, rows beyond n_cov do not
+    influence anything."""
+    rng = np.random.default_rng(77)
+    L, H, T, d, r, n_cov, s = 1, 2, 19, 8, 3, 13, 5
+    f = orc.rope_inv_freq(d, 10000.0)
+    sk, sv = _bits(rng.standard_normal((L, H, T, d))), _bits(rng.standard_normal((L, H, T, d)))
+    tk, tv = _bits(rng.standard_normal((L, H, T, d))), _bits(rng.standard_normal((L, H, T, d)))
+    src, tgt = orc.Cache(sk, sv), orc.Cache(tk, tv)
+    st, ev = orc.state_update(src, tgt, s, f, r=r, mode=orc.FIT, n_cov=n_cov)
+    assert st.coeff_k.shape == (L, H, n_cov, r) and st.coeff_k.dtype == np.float32 and st.basis_k.dtype == np.float32
+    # changing the uncovered rows changes nothing
+    tk2 = tk.copy()
+    tk2[:, :, n_cov:] = _bits(rng.standard_normal((L, H, T - n_cov, d)))
+    st2, ev2 = orc.state_update(src, orc.Cache(tk2, tv), s, f, r=r, mode=orc.FIT, n_cov=n_cov)
+    assert np.array_equal(st2.basis_k, st.basis_k) and np.array_equal(st2.coeff_k, st.coeff_k) and np.array_equal(ev2, ev)
+    for h in range(H):
+        # keys: tgt - Rot_s(src), the rotation written out per pair with math functions
+        x, y = _val(sk[0, h]), _val(tk[0, h])
+        dk = np.zeros((n_cov, d))
+        for t in range(n_cov):
+            for k in range(d // 2):
+                c, sn = math.cos(s * f[k]), math.sin(s * f[k])
+                dk[t, k] = y[t, k] - (x[t, k] * c - x[t, k + d // 2] * sn)
+                dk[t, k + d // 2] = y[t, k + d // 2] - (x[t, k] * sn + x[t, k + d // 2] * c)
+        dv = (_val(tv[0, h]) - _val(sv[0, h]))[:n_cov]
+        for dl, B, c, w in ((dk, st.basis_k[0, h], st.coeff_k[0, h], ev[0, h, 0]), (dv, st.basis_v[0, h], st.coeff_v[0, h], ev[0, h, 1])):
+            U, S, Vt = np.linalg.svd(dl, full_matrices=False)
+            assert np.allclose(w[:len(S)], S ** 2, rtol=1e-9, atol=1e-12)
+            B64, c64 = B.astype(np.float64), c.astype(np.float64)
+            best = (U[:, :r] * S[:r]) @ Vt[:r]
+            assert np.max(np.abs(c64 @ B64 - best)) <= 1e-5             # float32 storage of both factors
+            assert np.max(np.abs(c64.T @ c64 - np.diag(S[:r] ** 2))) <= 1e-4 * S[0] ** 2
+            assert np.allclose(c64, dl @ B64.T, atol=1e-6)               # the STORED (float32) basis is what projects
