@@ -41,6 +41,8 @@ namespace tc {
 constexpr int kTileTok = 128;
 constexpr int kThreads = 640;
 constexpr int kTeamThreads = 512;
+constexpr int kConvThreads = 128;                 // CV kernels: four more warps that do nothing but convert operands
+constexpr int kThreadsCv = kThreads + kConvThreads;
 constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a base tile (bf16)
 constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
 constexpr int kCoeffBlkBytes = kTileTok * 128;    // 128 tokens x 32 fp32 (one rank block)
@@ -190,24 +192,36 @@ struct Ctrl {
 // channels each, then per channel one 16-byte chunk of hi parts and one of lo parts.  Consecutive
 // callers take the 4 k8 groups of 8 channel groups, which spreads both the loads and the swizzled
 // stores over all banks.
+// rcs / rsn (optional, half-split pairing): the basis rows are rotated by that table on the way, so that
+// the contraction yields the rotated reconstruction,  Rot(c . B) = c . Rot(B)  row by row.
+__device__ __forceinline__ float4 raw_basis4(const uint8_t* raw, int q, int chg, int r, int bf16) {
+  if (q >= r) return make_float4(0.f, 0.f, 0.f, 0.f);
+  if (bf16) {
+    const uint2 u = *reinterpret_cast<const uint2*>(raw + q * 256 + chg * 8);
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xffff0000u));
+  }
+  return *reinterpret_cast<const float4*>(raw + q * 512 + chg * 16);
+}
 template <int RB>
-__device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_ptr, int r, int bf16, int first, int stride) {
+__device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_ptr, int r, int bf16, int first, int stride,
+                                              const float* rcs = nullptr, const float* rsn = nullptr) {
   const int nb = (r + 31) >> 5;
   const int n_task = (nb < RB ? nb : RB) * 128;
   for (int task = first; task < n_task; task += stride) {
     const int k8 = (task >> 3) & 3, chg = ((task >> 5) & 3) * 8 + (task & 7), b = task >> 7;
     float4 v[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int q = 32 * b + 8 * k8 + e;
-      if (q >= r) {
-        v[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-      } else if (bf16) {
-        const uint2 u = *reinterpret_cast<const uint2*>(raw + q * 256 + chg * 8);
-        v[e] = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-                           __uint_as_float(u.y & 0xffff0000u));
-      } else {
-        v[e] = *reinterpret_cast<const float4*>(raw + q * 512 + chg * 16);
+    for (int e = 0; e < 8; ++e) v[e] = raw_basis4(raw, 32 * b + 8 * k8 + e, chg, r, bf16);
+    if (rcs) {
+      // channels 4 chg .. + 3 and their partners 64 away (pair index = channel mod 64)
+      const float4 c4 = *reinterpret_cast<const float4*>(rcs + 4 * (chg & 15)), s4 = *reinterpret_cast<const float4*>(rsn + 4 * (chg & 15));
+      const float sg = chg < 16 ? -1.f : 1.f;       // u' = u cos - v sin;  v' = v cos + u sin
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float4 o = raw_basis4(raw, 32 * b + 8 * k8 + e, chg ^ 16, r, bf16);
+        v[e] = make_float4(fmaf(v[e].x, c4.x, sg * o.x * s4.x), fmaf(v[e].y, c4.y, sg * o.y * s4.y),
+                           fmaf(v[e].z, c4.z, sg * o.z * s4.z), fmaf(v[e].w, c4.w, sg * o.w * s4.w));
       }
     }
 #pragma unroll
@@ -244,8 +258,10 @@ __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_
 // MODE 0: apply; 1: gate distance; 2: row distances; 3: apply with a segment table (per-row shift and
 // tables, correction before or after the rotation) - the table is a second launch parameter of its own
 // kernel, so the other launches do not carry it.
-template <int RB, int NSTAGE, int NSC, int MODE>
+template <int RB, int NSTAGE, int NSC, int MODE, bool CV>
 __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegTable* segp) {
+  constexpr int kConvArrivals = CV ? kConvThreads : kTeamThreads;   // who converts: the converter warps or the team
+  static_assert(MODE != 2 || CV, "the row-distance mode relies on the converter warps (rotated key basis)");
   constexpr bool GATE = MODE == 1;                // walks value slabs only
   constexpr bool SEG = MODE == 3;
   // The epilogue works on packed float32 pairs except in the configuration of a contiguous source with
@@ -280,14 +296,14 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
     }
     for (int c = 0; c < NSC; ++c) {
       mbar_init(smem_u32(&ctrl->cfull[c]), 1);
-      mbar_init(smem_u32(&ctrl->conv[c]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->conv[c]), kConvArrivals);
       mbar_init(smem_u32(&ctrl->cempty[c]), 1);
     }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&ctrl->mma_done[g]), 1);
       mbar_init(smem_u32(&ctrl->acc_empty[g]), kTeamThreads);
     }
-    mbar_init(smem_u32(&ctrl->basis_full), kTeamThreads);
+    mbar_init(smem_u32(&ctrl->basis_full), kConvArrivals);
     mbar_init(smem_u32(&ctrl->drain), 1);
     ctrl->abort_flag = 0;
     fence_barrier_init();
@@ -528,6 +544,67 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[s]));
     }
+  } else if (CV && warp >= 4 + kTeamThreads / 32) {
+    // =============================================================== converter warps (CV kernels)
+    // Thread ct owns coefficient row ct of every tile: fp32 -> bf16 head and tail in place, and the
+    // slab's operand from its raw basis.  They run ahead of the team by as many tiles as the
+    // coefficient ring has free slots, so neither the conversion nor the MMA's latency sits on the
+    // team's path from one tile to the next.
+    const int ct = tid - (128 + kTeamThreads);
+    const uint32_t csw = (uint32_t)(ct & 7);
+    TileWalker<GATE> w;
+    w.init(&p, tile_begin, tile_end);
+    uint32_t i = 0, cpos = 0;
+    for (; !w.done(); w.next(), ++i) {
+      Tile t;
+      w.get(t);
+      if (t.first && t.uses_basis) {
+        const uint32_t pos = cpos++;
+        const int bc = pos % NSC;
+        bool ok = mbar_wait(smem_u32(&ctrl->cfull[bc]), (pos / NSC) & 1u, abort_flag);
+        // the operand slot is rebuilt: the MMAs of the previous tile (the last of its slab) must be complete
+        if (ok && i > 0) ok = mbar_wait(smem_u32(&ctrl->mma_done[(i - 1) & 1]), ((i - 1) >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        // row distances: the key basis is rotated into canonical coordinates here, once per slab, so that
+        // the team meets the reconstruction already rotated
+        const bool rot_basis = MODE == 2 && !t.is_v;
+        convert_basis<RB>(smem + NSTAGE * kStageBytes + bc * kCoeffSlotBytes, smem + kOperandOff, t.it->st.r,
+                          t.it->st.basis_bf16, ct, kConvThreads, rot_basis ? p.cs2 : nullptr, rot_basis ? p.sn2 : nullptr);
+        fence_proxy_async();
+        mbar_arrive(smem_u32(&ctrl->basis_full));
+        mbar_arrive(smem_u32(&ctrl->conv[bc]));       // the issuer hands the ring slot back
+      }
+      const uint32_t pos = cpos++;
+      const int c = pos % NSC;
+      bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), (pos / NSC) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (t.has_coeff) {
+        uint8_t* c_ptr = smem + NSTAGE * kStageBytes + c * kCoeffSlotBytes;
+#pragma unroll
+        for (int b = 0; b < RB; ++b) {
+          if (b >= t.nb) break;                       // uniform over the CTA
+          uint8_t* row = c_ptr + b * kCoeffBlkBytes + ct * 128;
+          float4 f[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) f[k] = *reinterpret_cast<const float4*>(row + (((uint32_t)k ^ csw) << 4));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {               // ranks 8 j .. 8 j + 7: heads to chunk j, tails to chunk 4 + j
+            uint4 hi, lo;
+            split2(f[2 * j].x, f[2 * j].y, hi.x, lo.x);
+            split2(f[2 * j].z, f[2 * j].w, hi.y, lo.y);
+            split2(f[2 * j + 1].x, f[2 * j + 1].y, hi.z, lo.z);
+            split2(f[2 * j + 1].z, f[2 * j + 1].w, hi.w, lo.w);
+            *reinterpret_cast<uint4*>(row + (((uint32_t)j ^ csw) << 4)) = hi;
+            *reinterpret_cast<uint4*>(row + (((uint32_t)(4 + j) ^ csw) << 4)) = lo;
+          }
+        }
+        fence_proxy_async();
+      }
+      mbar_arrive(smem_u32(&ctrl->conv[c]));
+    }
   } else {
     // =============================================================== the team (16 warps)
     const int e = warp - 4;
@@ -596,23 +673,27 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
     };
     uint32_t pending_basis = 0;                     // ring position of a raw basis not yet consumed
     bool have_pending = false;
-    if (!w.done()) {
-      Tile t0;
-      w.get(t0);
-      if (t0.uses_basis) alive = take_basis(t0, cpos++);
-      if (alive) alive = convert(wn, cpos++);
+    if constexpr (!CV) {
+      if (!w.done()) {
+        Tile t0;
+        w.get(t0);
+        if (t0.uses_basis) alive = take_basis(t0, cpos++);
+        if (alive) alive = convert(wn, cpos++);
+      }
     }
     for (; alive && !w.done(); w.next(), ++i) {
-      // ---- 1. get the next tile's coefficients converted and its MMA going
-      wn.next();
-      if (!wn.done()) {
-        Tile tn;
-        wn.get(tn);
-        have_pending = tn.uses_basis && tn.first;
-        if (have_pending) pending_basis = cpos++;
-        if (!convert(wn, cpos++)) break;
-      } else {
-        have_pending = false;
+      // ---- 1. get the next tile's coefficients converted and its MMA going (unless the converter warps do that)
+      if constexpr (!CV) {
+        wn.next();
+        if (!wn.done()) {
+          Tile tn;
+          wn.get(tn);
+          have_pending = tn.uses_basis && tn.first;
+          if (have_pending) pending_basis = cpos++;
+          if (!convert(wn, cpos++)) break;
+        } else {
+          have_pending = false;
+        }
       }
       Tile t;
       w.get(t);
@@ -712,25 +793,20 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
             unpack8(*reinterpret_cast<const uint4*>(row0 + ((j ^ sw) << 4)), x);
             unpack8(*reinterpret_cast<const uint4*>(row1 + ((j ^ sw) << 4)), x + 8);
             if (!t.is_v) {
-              // both tables, eight pairs each, as vector loads
+              // the source rotated by the item's table, eight pairs; the reconstruction arrives rotated
+              // (the converter warps rotated the basis rows by the second table)
               const float4 ca = *reinterpret_cast<const float4*>(it.cs + 8 * j), cb = *reinterpret_cast<const float4*>(it.cs + 8 * j + 4);
               const float4 sa4 = *reinterpret_cast<const float4*>(it.sn + 8 * j), sb4 = *reinterpret_cast<const float4*>(it.sn + 8 * j + 4);
-              const float4 cc = *reinterpret_cast<const float4*>(p.cs2 + 8 * j), cd = *reinterpret_cast<const float4*>(p.cs2 + 8 * j + 4);
-              const float4 sc4 = *reinterpret_cast<const float4*>(p.sn2 + 8 * j), sd4 = *reinterpret_cast<const float4*>(p.sn2 + 8 * j + 4);
               const float c1[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
               const float s1[8] = {sa4.x, sa4.y, sa4.z, sa4.w, sb4.x, sb4.y, sb4.z, sb4.w};
-              const float c2[8] = {cc.x, cc.y, cc.z, cc.w, cd.x, cd.y, cd.z, cd.w};
-              const float s2[8] = {sc4.x, sc4.y, sc4.z, sc4.w, sd4.x, sd4.y, sd4.z, sd4.w};
 #pragma unroll
               for (int z = 0; z < 4; ++z) {
-                // packed pairs: source rotated by the first table minus reconstruction rotated by the second
                 const f32x2 u = f2_pack(x[2 * z], x[2 * z + 1]), v = f2_pack(x[8 + 2 * z], x[9 + 2 * z]);
                 const f32x2 au = f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]), av = f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]);
                 const f32x2 pc1 = f2_pack(c1[2 * z], c1[2 * z + 1]), ps1 = f2_pack(s1[2 * z], s1[2 * z + 1]);
-                const f32x2 pc2 = f2_pack(c2[2 * z], c2[2 * z + 1]), ps2 = f2_pack(s2[2 * z], s2[2 * z + 1]);
-                const f32x2 nps1 = f2_pack(-s1[2 * z], -s1[2 * z + 1]), nps2 = f2_pack(-s2[2 * z], -s2[2 * z + 1]);
-                const f32x2 du = f2_sub(f2_fma(u, pc1, f2_mul(v, nps1)), f2_fma(au, pc2, f2_mul(av, nps2)));
-                const f32x2 dv = f2_sub(f2_fma(u, ps1, f2_mul(v, pc1)), f2_fma(au, ps2, f2_mul(av, pc2)));
+                const f32x2 nps1 = f2_pack(-s1[2 * z], -s1[2 * z + 1]);
+                const f32x2 du = f2_sub(f2_fma(u, pc1, f2_mul(v, nps1)), au);
+                const f32x2 dv = f2_sub(f2_fma(u, ps1, f2_mul(v, pc1)), av);
                 float e0, e1, e2, e3;
                 f2_unpack(du, e0, e1);
                 f2_unpack(dv, e2, e3);
@@ -881,14 +957,14 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
   }
 }
 
-template <int RB, int NSTAGE, int NSC, int MODE = 0>
-__global__ void __launch_bounds__(kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
-  apply_tc_body<RB, NSTAGE, NSC, MODE>(p, nullptr);
+template <int RB, int NSTAGE, int NSC, int MODE = 0, bool CV = false>
+__global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_tc_kernel(const __grid_constant__ ApplyTcLaunch p) {
+  apply_tc_body<RB, NSTAGE, NSC, MODE, CV>(p, nullptr);
 }
-template <int RB, int NSTAGE, int NSC>
-__global__ void __launch_bounds__(kThreads, 1) apply_tc_seg_kernel(const __grid_constant__ ApplyTcLaunch p,
-                                                                   const __grid_constant__ SegTable seg) {
-  apply_tc_body<RB, NSTAGE, NSC, 3>(p, &seg);
+template <int RB, int NSTAGE, int NSC, bool CV = false>
+__global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_tc_seg_kernel(const __grid_constant__ ApplyTcLaunch p,
+                                                                                    const __grid_constant__ SegTable seg) {
+  apply_tc_body<RB, NSTAGE, NSC, 3, CV>(p, &seg);
 }
 
 // ------------------------------------------------------------------ host side
@@ -917,7 +993,7 @@ static bool build_maps(const DevItem& it, ItemMaps* mp) {
   return ok;
 }
 
-template <int RB, int NSTAGE, int NSC>
+template <int RB, int NSTAGE, int NSC, bool CV = false>
 static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
                           sizeof(Ctrl<NSTAGE, NSC>);
@@ -925,26 +1001,26 @@ static cudaError_t launch_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, 0, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     once.mark(once_dev);
   }
-  apply_tc_kernel<RB, NSTAGE, NSC><<<grid, kThreads, smem, s>>>(L);
+  apply_tc_kernel<RB, NSTAGE, NSC, 0, CV><<<grid, CV ? kThreadsCv : kThreads, smem, s>>>(L);
   return cudaGetLastError();
 }
 
-template <int RB, int NSTAGE, int NSC>
+template <int RB, int NSTAGE, int NSC, bool CV = false>
 static cudaError_t launch_seg_t(const ApplyTcLaunch& L, const SegTable& seg, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
                           sizeof(Ctrl<NSTAGE, NSC>);
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    cudaError_t e = cudaFuncSetAttribute(apply_tc_seg_kernel<RB, NSTAGE, NSC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_seg_kernel<RB, NSTAGE, NSC, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     once.mark(once_dev);
   }
-  apply_tc_seg_kernel<RB, NSTAGE, NSC><<<grid, kThreads, smem, s>>>(L, seg);
+  apply_tc_seg_kernel<RB, NSTAGE, NSC, CV><<<grid, CV ? kThreadsCv : kThreads, smem, s>>>(L, seg);
   return cudaGetLastError();
 }
 
@@ -961,23 +1037,26 @@ static int launch(const ApplyTcLaunch& L, int max_r, bool paged, cudaStream_t s,
     cudaError_t es = (max_r > 32) ? launch_seg_t<2, 4, 2>(L, *seg, grid, s) : launch_seg_t<1, 5, 3>(L, *seg, grid, s);
     return es == cudaSuccess ? KVC_OK : KVC_E_CUDA;
   }
-  cudaError_t e = (max_r > 32) ? launch_t<2, 4, 2>(L, grid, s)
-                               : (paged ? launch_t<1, 5, 3>(L, grid, s) : launch_t<1, 5, 2>(L, grid, s));
+  // converter warps (CV) where the team's instruction stream, not HBM, set the pace: paged sources and
+  // two rank blocks; a contiguous source with one rank block streams at the copy bandwidth without them
+  // and measured 4 % slower with them
+  cudaError_t e = (max_r > 32) ? launch_t<2, 4, 2, true>(L, grid, s)
+                               : (paged ? launch_t<1, 5, 3, true>(L, grid, s) : launch_t<1, 5, 2>(L, grid, s));
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
-template <int RB, int NSTAGE, int NSC, int MODE>
+template <int RB, int NSTAGE, int NSC, int MODE, bool CV = false>
 static cudaError_t launch_reduce_t(const ApplyTcLaunch& L, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NSC * RB * kCoeffBlkBytes + (size_t)RB * kBasisBlkBytes +
                           sizeof(Ctrl<NSTAGE, NSC>);
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(apply_tc_kernel<RB, NSTAGE, NSC, MODE, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     once.mark(once_dev);
   }
-  apply_tc_kernel<RB, NSTAGE, NSC, MODE><<<grid, kThreads, smem, s>>>(L);
+  apply_tc_kernel<RB, NSTAGE, NSC, MODE, CV><<<grid, CV ? kThreadsCv : kThreads, smem, s>>>(L);
   return cudaGetLastError();
 }
 
@@ -1029,7 +1108,7 @@ int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, 
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
-  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 5, 3, 1>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 1>(L, grid, s);
+  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 5, 3, 1, true>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 1, true>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
@@ -1057,8 +1136,7 @@ int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* s
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
-  // three base slots and six coefficient slots: measured 3 % faster here than the apply kernel's five and three
-  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 3, 6, 2>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 2>(L, grid, s);
+  cudaError_t e = (item.st.r <= 32) ? tc::launch_reduce_t<1, 5, 3, 2, true>(L, grid, s) : tc::launch_reduce_t<2, 4, 2, 2, true>(L, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

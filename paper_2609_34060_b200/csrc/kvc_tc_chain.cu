@@ -67,7 +67,9 @@ struct Ctrl {
   int abort_flag;
 };
 
-__global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
+template <bool CV>
+__global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
+  constexpr int kConvArrivals = CV ? kConvThreads : kTeamThreads;   // who converts: the converter warps or the team
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -100,7 +102,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     }
     for (int c = 0; c < NC; ++c) {
       mbar_init(smem_u32(&ctrl->cfull[c]), 1);
-      mbar_init(smem_u32(&ctrl->conv[c]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->conv[c]), kConvArrivals);
       mbar_init(smem_u32(&ctrl->cempty[c]), 1);
     }
     for (int o = 0; o < NO; ++o) {
@@ -347,6 +349,48 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->ostored[s]));
       }
     }
+  } else if (CV && warp >= 4 + kTeamThreads / 32) {
+    // =============================================================== converter warps (CV kernel)
+    // thread ct owns coefficient row ct of every ring entry (fp32 -> bf16 [c1 | c2] in place), in the
+    // order the steps consume them, ahead of the team by as many entries as the ring has free slots
+    const int ct = tid - (128 + kTeamThreads);
+    const uint32_t csw = (uint32_t)(ct & 7);
+    Walker w;
+    w.init(p.tps, p.H, tile_begin, tile_end);
+    uint32_t epos = 0;
+    bool alive = true;
+    for (; alive && !w.done(); w.next()) {
+      const int t0 = w.t0();
+      for (int a = 0; alive && a < NH; ++a) {
+        const int nb = blocks_of(a, t0);
+        for (int b = 0; b < nb; ++b) {
+          const int c = epos % NC;
+          bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), (epos / NC) & 1u, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) {
+            alive = false;
+            break;
+          }
+          uint8_t* row = smem + kCoeffOff + c * kCoeffBytes + ct * 128;
+          float4 f[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) f[k] = *reinterpret_cast<const float4*>(row + (((uint32_t)k ^ csw) << 4));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {               // ranks 8 j .. 8 j + 7: heads to chunk j, tails to chunk 4 + j
+            uint4 hi, lo;
+            split2(f[2 * j].x, f[2 * j].y, hi.x, lo.x);
+            split2(f[2 * j].z, f[2 * j].w, hi.y, lo.y);
+            split2(f[2 * j + 1].x, f[2 * j + 1].y, hi.z, lo.z);
+            split2(f[2 * j + 1].z, f[2 * j + 1].w, hi.w, lo.w);
+            *reinterpret_cast<uint4*>(row + (((uint32_t)j ^ csw) << 4)) = hi;
+            *reinterpret_cast<uint4*>(row + (((uint32_t)(4 + j) ^ csw) << 4)) = lo;
+          }
+          fence_proxy_async();
+          mbar_arrive(smem_u32(&ctrl->conv[c]));
+          ++epos;
+        }
+      }
+    }
   } else {
     // =============================================================== the team (16 warps)
     const int e16 = warp - 4;
@@ -396,7 +440,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         wn.next();
       }
     };
-    if (!w.done()) {
+    if (!CV && !w.done()) {
       alive = convert_hop(0, wn.t0());
       advance_next();
     }
@@ -406,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
       const uint8_t* in_ptr = smem + sb * kBaseBytes;   // hop 0 reads agent 0's tile
       for (int a = 0; a < NH; ++a, ++step) {
         // ---- 1. the next step's coefficients, so that its MMAs run under this step's epilogue
-        if (!wn.done()) {
+        if (!CV && !wn.done()) {
           if (!convert_hop(an, wn.t0())) {
             alive = false;
             break;
@@ -645,10 +689,10 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+    if (cudaFuncSetAttribute(chain_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
     once.mark(once_dev);
   }
-  chain_tc_kernel<<<grid, kThreads, smem, s>>>(C);
+  chain_tc_kernel<true><<<grid, kThreadsCv, smem, s>>>(C);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

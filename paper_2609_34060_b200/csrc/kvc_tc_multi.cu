@@ -90,9 +90,10 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0, p.grouped[e] != 0, p.H);
 }
 
-template <int NSTAGE, int NC, int NO>
-__global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
+template <int NSTAGE, int NC, int NO, bool CV>
+__global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
   using Ctrl = tcm::Ctrl<NSTAGE, NC, NO>;
+  constexpr int kConvArrivals = CV ? kConvThreads : kTeamThreads;   // who converts: the converter warps or the team
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -120,7 +121,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
     }
     for (int c = 0; c < NC; ++c) {
       mbar_init(smem_u32(&ctrl->cfull[c]), 1);
-      mbar_init(smem_u32(&ctrl->conv[c]), kTeamThreads);
+      mbar_init(smem_u32(&ctrl->conv[c]), kConvArrivals);
       mbar_init(smem_u32(&ctrl->cempty[c]), 1);
     }
     for (int o = 0; o < NO; ++o) {
@@ -361,6 +362,48 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[s]));
     }
+  } else if (CV && warp >= 4 + kTeamThreads / 32) {
+    // =============================================================== converter warps (CV kernels)
+    // thread ct owns coefficient row ct of every ring entry: fp32 coefficients x token weight ->
+    // bf16 [c1 | c2] in place, ahead of the team by as many entries as the ring has free slots
+    const int ct = tid - (128 + kTeamThreads);
+    const uint32_t csw = (uint32_t)(ct & 7);
+    Walker w;
+    w.init(p.tps, p.H, tile_begin, tile_end);
+    uint32_t epos = 0;
+    bool alive = true;
+    for (; alive && !w.done(); w.next()) {
+      const int t0 = w.t0(), is_v = w.is_v();
+      for (int e = 0; e < p.n_blocks; ++e) {
+        if (!active(e, t0)) continue;
+        const int c = epos % NC;
+        bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), (epos / NC) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+          alive = false;
+          break;
+        }
+        const bool weighted = (is_v ? p.blk[e].w_v : p.blk[e].w_k) != nullptr;
+        const float wt = weighted ? reinterpret_cast<const float*>(smem + kWeightOff + c * kWeightBytes)[ct] : 1.f;
+        uint8_t* row = smem + kCoeffOff + c * kCoeffBytes + ct * 128;
+        float4 f[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) f[k] = *reinterpret_cast<const float4*>(row + (((uint32_t)k ^ csw) << 4));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {                 // ranks 8 j .. 8 j + 7: heads to chunk j, tails to chunk 4 + j
+          uint4 hi, lo;
+          split2(f[2 * j].x * wt, f[2 * j].y * wt, hi.x, lo.x);
+          split2(f[2 * j].z * wt, f[2 * j].w * wt, hi.y, lo.y);
+          split2(f[2 * j + 1].x * wt, f[2 * j + 1].y * wt, hi.z, lo.z);
+          split2(f[2 * j + 1].z * wt, f[2 * j + 1].w * wt, hi.w, lo.w);
+          *reinterpret_cast<uint4*>(row + (((uint32_t)j ^ csw) << 4)) = hi;
+          *reinterpret_cast<uint4*>(row + (((uint32_t)(4 + j) ^ csw) << 4)) = lo;
+        }
+        fence_proxy_async();
+        mbar_arrive(smem_u32(&ctrl->conv[c]));
+        ++epos;
+      }
+    }
   } else {
     // =============================================================== the team (16 warps)
     const int e16 = warp - 4;
@@ -409,12 +452,16 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
       return true;
     };
 
-    if (!w.done()) alive = convert_tile(wn);
+    if constexpr (!CV) {
+      if (!w.done()) alive = convert_tile(wn);
+    }
     for (; alive && !w.done(); w.next(), ++i) {
-      // ---- 1. get the next tile's rank blocks converted and their MMAs going
-      wn.next();
-      if (!wn.done()) {
-        if (!convert_tile(wn)) break;
+      // ---- 1. get the next tile's rank blocks converted and their MMAs going (unless the converter warps do that)
+      if constexpr (!CV) {
+        wn.next();
+        if (!wn.done()) {
+          if (!convert_tile(wn)) break;
+        }
       }
       const int s = i % NSTAGE, g = i & 1;
       const int t0 = w.t0(), is_v = w.is_v();
@@ -537,7 +584,7 @@ __global__ void __launch_bounds__(kThreads, 1) apply_multi_tc_kernel(const __gri
   }
 }
 
-template <int NSTAGE, int NC, int NO>
+template <int NSTAGE, int NC, int NO, bool CV = false>
 static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
                           (size_t)NO * kOperandBytes + sizeof(Ctrl<NSTAGE, NC, NO>);
@@ -545,11 +592,11 @@ static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     once.mark(once_dev);
   }
-  apply_multi_tc_kernel<NSTAGE, NC, NO><<<grid, kThreads, smem, s>>>(M);
+  apply_multi_tc_kernel<NSTAGE, NC, NO, CV><<<grid, CV ? kThreadsCv : kThreads, smem, s>>>(M);
   return cudaGetLastError();
 }
 
@@ -637,7 +684,7 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(M.total_tiles < sms ? M.total_tiles : sms);
-  const cudaError_t e = nb <= 3 ? tcm::launch_multi_t<4, 3, 3>(M, grid, s) : tcm::launch_multi_t<3, 5, 2>(M, grid, s);
+  const cudaError_t e = tcm::launch_multi_t<3, 5, 2, true>(M, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

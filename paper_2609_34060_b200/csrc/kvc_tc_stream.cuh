@@ -16,6 +16,8 @@ namespace tcs {
 constexpr int kTileTok = 128;
 constexpr int kThreads = 640;                     // producer, MMA, two store warps ... and a team of 16 warps
 constexpr int kTeamThreads = 512;
+constexpr int kConvThreads = 128;                 // kernels with converter warps: four more warps after the team
+constexpr int kThreadsCv = kThreads + kConvThreads;
 constexpr int kHalfBytes = kTileTok * 128;        // one 64-channel half of a cache tile (bf16)
 constexpr int kBaseBytes = 2 * kHalfBytes;        // 32 KB
 constexpr int kCoeffBytes = kTileTok * 128;       // 128 tokens x 32 fp32 (one rank block)
