@@ -56,20 +56,39 @@ struct Walker {
 // One basis operand block: 128 rows (channel) of [32 hi | 32 lo] bf16 for ranks col0 .. col0 + 31 of
 // the basis [slabs][r][128] (float32 or bf16; zero beyond rank r).  Called by a block of 256 threads.
 // A state grouped by layer keeps [layers][r][H * 128]: head h of layer l reads columns h * 128 .. of row q.
+// The 32 x 128 values are read along the channel (coalesced), turned through shared memory, and written
+// as whole 64-byte halves of the operand rows (a warp writes 2 KB of consecutive bytes).
 __device__ __forceinline__ void write_operand_block(__nv_bfloat16* out, const void* basis, bool basis_bf16, int slab, int r,
                                                     int col0, bool grouped = false, int H = 1) {
+  constexpr int P = 129;                          // pitch of the staged rows (floats): a thread per channel reads without bank conflicts
+  __shared__ float stage[32 * P];
   const int l = slab / H, h = slab - l * H;
   for (int i = threadIdx.x; i < 32 * 128; i += 256) {
-    const int q = i >> 7, ch = i & 127;           // coalesced reads along the channel
+    const int q = i >> 7, ch = i & 127;
     float x = 0.f;
     if (col0 + q < r) {
       const int64_t off = grouped ? (((int64_t)l * r + col0 + q) * H + h) * 128 + ch : ((int64_t)slab * r + col0 + q) * 128 + ch;
       x = basis_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(basis)[off]) : reinterpret_cast<const float*>(basis)[off];
     }
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    out[ch * 64 + q] = hi;
-    out[ch * 64 + 32 + q] = __float2bfloat16_rn(x - __bfloat162float(hi));
+    stage[q * P + ch] = x;
   }
+  __syncthreads();
+  const int ch = threadIdx.x >> 1, lo_half = threadIdx.x & 1;       // thread: one 64-byte half of row ch
+  uint32_t w[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    float x0 = stage[(2 * k) * P + ch], x1 = stage[(2 * k + 1) * P + ch];
+    if (lo_half) {
+      x0 -= __bfloat162float(__float2bfloat16_rn(x0));
+      x1 -= __bfloat162float(__float2bfloat16_rn(x1));
+    }
+    const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
+    w[k] = *reinterpret_cast<const uint32_t*>(&pr);
+  }
+  uint4* dst = reinterpret_cast<uint4*>(out + ch * 64 + lo_half * 32);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) dst[k] = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+  __syncthreads();                                // the stage may be refilled by the caller's next block
 }
 
 // Tensor map over the operand blocks: rows of 64 bf16 (128 bytes, swizzled), boxes of 128 rows.
