@@ -15,9 +15,13 @@
 //   warp 1      MMA issuer (one lane) and TMEM owner (two accumulators of 128 columns)
 //   warp 2      spare
 //   warp 3      store warp: TMA stores of finished tiles, releases the base slot
-//   warps 4-19  the team: converts the next tile's coefficient rows to bf16 hi/lo in place, rebuilds
-//               the operand slot when a slab starts, and for the current tile reads the accumulator
-//               row from TMEM, rotates, adds, rounds and writes the row back in place.
+//   warps 4-19  the team: for the current tile reads the accumulator row from TMEM, rotates, adds,
+//               rounds and writes the row back in place (or reduces, in the distance modes)
+//   warps 20-23 converter warps (CV kernels only): a thread per coefficient row turns the fp32 tile into
+//               bf16 hi/lo in place and the group rebuilds the operand slot when a slab starts, as far
+//               ahead of the team as the coefficient ring has slots.  Without them (CV = false: a
+//               contiguous source with one rank block, which streams at the copy bandwidth anyway)
+//               the team does both before its own tile, one tile ahead.
 // Precision: c = c1 + c2 and B = B1 + B2 with bf16 terms; c.B ~= c1.B1 + c2.B1 + c1.B2
 // (relative error about 2^-16 per product), accumulated in fp32.
 // Every wait is bounded; on expiry the CTA records KVC_FLAG_WAIT_EXPIRED, drains and returns.
@@ -243,7 +247,7 @@ __device__ __forceinline__ void convert_basis(const uint8_t* raw, uint8_t* slot_
 }
 
 // ------------------------------------------------------------------ the kernel
-// Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 spare, 3 store warp, 4..19 the team.
+// Warps: 0 producer, 1 MMA issuer + TMEM owner, 2 spare, 3 store warp, 4..19 the team, 20..23 converters (CV).
 // Team warp e (0..15): TMEM lane quadrant e & 3 (rows 32q..32q+31), channel quarter e >> 2.
 //
 // Two rings of shared-memory slots: NSTAGE base tiles (alive from the load until the TMA store has

@@ -10,7 +10,8 @@
 // arithmetic of the single-hop kernel, so the results are bit-identical to hop-by-hop kvc_apply) and
 // its own output slot, which the store warp sends to that hop's destination cache while the next
 // hop reads it as its input.  A thread reads and writes the same elements in every hop, so the
-// hops of a tile need no synchronisation inside the team.
+// hops of a tile need no synchronisation inside the team.  Four converter warps turn the fp32
+// coefficient blocks into bf16 hi/lo operands ahead of the team.
 // Every wait is bounded; on expiry the CTA records KVC_FLAG_WAIT_EXPIRED, drains and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -67,9 +68,7 @@ struct Ctrl {
   int abort_flag;
 };
 
-template <bool CV>
-__global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
-  constexpr int kConvArrivals = CV ? kConvThreads : kTeamThreads;   // who converts: the converter warps or the team
+__global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -102,7 +101,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel
     }
     for (int c = 0; c < NC; ++c) {
       mbar_init(smem_u32(&ctrl->cfull[c]), 1);
-      mbar_init(smem_u32(&ctrl->conv[c]), kConvArrivals);
+      mbar_init(smem_u32(&ctrl->conv[c]), kConvThreads);
       mbar_init(smem_u32(&ctrl->cempty[c]), 1);
     }
     for (int o = 0; o < NO; ++o) {
@@ -349,8 +348,8 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->ostored[s]));
       }
     }
-  } else if (CV && warp >= 4 + kTeamThreads / 32) {
-    // =============================================================== converter warps (CV kernel)
+  } else if (warp >= 4 + kTeamThreads / 32) {
+    // =============================================================== converter warps
     // thread ct owns coefficient row ct of every ring entry (fp32 -> bf16 [c1 | c2] in place), in the
     // order the steps consume them, ahead of the team by as many entries as the ring has free slots
     const int ct = tid - (128 + kTeamThreads);
@@ -398,70 +397,20 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel
     const int cq = e16 >> 2;                       // channel quarter
     const int m = q * 32 + lane;                   // epilogue row = token of the tile
     const uint32_t sw = (uint32_t)(m & 7);
-    const int crow = e16 * 8 + (lane >> 2), cpart = lane & 3;   // conversion: four threads per coefficient row
-    const uint32_t csw = (uint32_t)(crow & 7);
-
-    uint32_t epos = 0;                             // ring position of the next entry to convert
-    // converts the rank blocks of one (tile, hop): fp32 coefficients -> bf16 [c1 | c2] in place
-    auto convert_hop = [&](int a, int t0) {
-      const int nb = blocks_of(a, t0);
-      for (int b = 0; b < nb; ++b) {
-        const int c = epos % NC;
-        bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), (epos / NC) & 1u, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) return false;
-        uint8_t* row = smem + kCoeffOff + c * kCoeffBytes + crow * 128;
-        const float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
-        const float4 f1 = *reinterpret_cast<const float4*>(row + (((2 * cpart + 1) ^ csw) << 4));
-        uint4 hi, lo;
-        split2(f0.x, f0.y, hi.x, lo.x);
-        split2(f0.z, f0.w, hi.y, lo.y);
-        split2(f1.x, f1.y, hi.z, lo.z);
-        split2(f1.z, f1.w, hi.w, lo.w);
-        __syncwarp();                               // all four threads of the row have read
-        *reinterpret_cast<uint4*>(row + ((cpart ^ csw) << 4)) = hi;
-        *reinterpret_cast<uint4*>(row + (((4 + cpart) ^ csw) << 4)) = lo;
-        fence_proxy_async();
-        mbar_arrive(smem_u32(&ctrl->conv[c]));
-        ++epos;
-      }
-      return true;
-    };
-
-    Walker w, wn;
+    Walker w;
     w.init(p.tps, p.H, tile_begin, tile_end);
-    wn = w;                                        // (tile, hop) one step ahead: its coefficients are converted first
-    int an = 0;
     uint32_t i = 0, step = 0;
     bool alive = true;
-    auto advance_next = [&]() {
-      if (++an == NH) {
-        an = 0;
-        wn.next();
-      }
-    };
-    if (!CV && !w.done()) {
-      alive = convert_hop(0, wn.t0());
-      advance_next();
-    }
     for (; alive && !w.done(); w.next(), ++i) {
       const int sb = i % NB;
       const int t0 = w.t0(), is_v = w.is_v();
       const uint8_t* in_ptr = smem + sb * kBaseBytes;   // hop 0 reads agent 0's tile
       for (int a = 0; a < NH; ++a, ++step) {
-        // ---- 1. the next step's coefficients, so that its MMAs run under this step's epilogue
-        if (!CV && !wn.done()) {
-          if (!convert_hop(an, wn.t0())) {
-            alive = false;
-            break;
-          }
-          advance_next();
-        }
         const Hop& hp = p.hop[a];
         const int g = step & 1, so = step % NOUT;
         uint8_t* out_ptr = smem + kOutOff + so * kBaseBytes;
         const bool has_coeff = blocks_of(a, t0) > 0;
-        // ---- 2. accumulator ready, input present, output slot free
+        // ---- 1. accumulator ready, input present, output slot free
         bool ok = mbar_wait(smem_u32(&ctrl->mma_done[g]), (step >> 1) & 1u, abort_flag);
         if (ok && a == 0) ok = mbar_wait(smem_u32(&ctrl->bfull[sb]), (i / NB) & 1u, abort_flag);
         if (ok) ok = mbar_wait(smem_u32(&ctrl->ostored[so]), ((step / NOUT) & 1u) ^ 1u, abort_flag);
@@ -490,7 +439,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel
         }
         tc_fence_before();
         mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
-        // ---- 3. rotate, add, round: row m, this warp's channel quarter, from the input slot to the output slot
+        // ---- 2. rotate, add, round: row m, this warp's channel quarter, from the input slot to the output slot
         if (p.pairing == 0) {
           const uint8_t* irow0 = in_ptr + m * 128;
           const uint8_t* irow1 = irow0 + kHalfBytes;
@@ -569,7 +518,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) chain_tc_kernel
             *reinterpret_cast<uint4*>(orow + ((j ^ sw) << 4)) = u0;
           }
         }
-        // ---- 4. the hop's result is final in shared memory: to the store warp; agent 0's tile is done after hop 0
+        // ---- 3. the hop's result is final in shared memory: to the store warp; agent 0's tile is done after hop 0
         fence_proxy_async();
         mbar_arrive(smem_u32(&ctrl->oready[so]));
         if (a == 0) mbar_arrive(smem_u32(&ctrl->bempty[sb]));
@@ -689,10 +638,10 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    if (cudaFuncSetAttribute(chain_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+    if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
     once.mark(once_dev);
   }
-  chain_tc_kernel<true><<<grid, kThreadsCv, smem, s>>>(C);
+  chain_tc_kernel<<<grid, kThreadsCv, smem, s>>>(C);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

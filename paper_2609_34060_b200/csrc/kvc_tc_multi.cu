@@ -4,10 +4,10 @@
 // effective rank of 320 - without materialising a stacked state.
 //
 // Differences from the single-state kernel (kvc_tc_apply.cu), whose skeleton this one shares
-// (persistent CTAs, TMA tiles, tcgen05 MMAs into TMEM, 16-warp team, store warp):
+// (persistent CTAs, TMA tiles, tcgen05 MMAs into TMEM, 16-warp team, store warp, four converter warps):
 //   * a tile has a variable number of ring entries, one per rank block that covers it; an entry
-//     is the fp32 coefficient block of its anchor (converted to bf16 hi/lo in place, scaled by the
-//     anchor's token weights on the way) with the tile's 128 weights, in a deep ring (HBM latency),
+//     is the fp32 coefficient block of its anchor (converted to bf16 hi/lo in place by the converter
+//     warps, scaled by the anchor's token weights on the way) with the tile's 128 weights, in a deep ring (HBM latency),
 //     and the block's basis operand in a shallow ring of its own (L2 latency, separate producer);
 //   * the basis operands are too many to stay resident per slab, so a preparation kernel writes
 //     them once, transposed and split, into a workspace from where TMA drops them into the ring
@@ -90,10 +90,9 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0, p.grouped[e] != 0, p.H);
 }
 
-template <int NSTAGE, int NC, int NO, bool CV>
-__global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
+template <int NSTAGE, int NC, int NO>
+__global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
   using Ctrl = tcm::Ctrl<NSTAGE, NC, NO>;
-  constexpr int kConvArrivals = CV ? kConvThreads : kTeamThreads;   // who converts: the converter warps or the team
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -121,7 +120,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_
     }
     for (int c = 0; c < NC; ++c) {
       mbar_init(smem_u32(&ctrl->cfull[c]), 1);
-      mbar_init(smem_u32(&ctrl->conv[c]), kConvArrivals);
+      mbar_init(smem_u32(&ctrl->conv[c]), kConvThreads);
       mbar_init(smem_u32(&ctrl->cempty[c]), 1);
     }
     for (int o = 0; o < NO; ++o) {
@@ -362,8 +361,8 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[s]));
     }
-  } else if (CV && warp >= 4 + kTeamThreads / 32) {
-    // =============================================================== converter warps (CV kernels)
+  } else if (warp >= 4 + kTeamThreads / 32) {
+    // =============================================================== converter warps
     // thread ct owns coefficient row ct of every ring entry: fp32 coefficients x token weight ->
     // bf16 [c1 | c2] in place, ahead of the team by as many entries as the ring has free slots
     const int ct = tid - (128 + kTeamThreads);
@@ -411,64 +410,16 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_
     const int cq = e16 >> 2;                       // channel quarter
     const int m = q * 32 + lane;                   // epilogue row = token of the tile
     const uint32_t sw = (uint32_t)(m & 7);
-    // conversion mapping: the four threads of a coefficient row sit in one warp
-    const int crow = e16 * 8 + (lane >> 2), cpart = lane & 3;
-    const uint32_t csw = (uint32_t)(crow & 7);
-
-    Walker w, wn;
+    Walker w;
     w.init(p.tps, p.H, tile_begin, tile_end);
-    wn = w;
-    uint32_t i = 0, epos = 0;
-    bool alive = true;
-
-    // converts all entries of the tile the walker points at: fp32 coefficients x token weight ->
-    // bf16 [c1 | c2] in place
-    auto convert_tile = [&](const Walker& cw) {
-      const int t0 = cw.t0(), is_v = cw.is_v();
-      for (int e = 0; e < p.n_blocks; ++e) {
-        if (!active(e, t0)) continue;
-        const int c = epos % NC;
-        bool ok = mbar_wait(smem_u32(&ctrl->cfull[c]), (epos / NC) & 1u, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) return false;
-        const bool weighted = (is_v ? p.blk[e].w_v : p.blk[e].w_k) != nullptr;
-        const float wt = weighted ? reinterpret_cast<const float*>(smem + kWeightOff + c * kWeightBytes)[crow] : 1.f;
-        uint8_t* row = smem + kCoeffOff + c * kCoeffBytes + crow * 128;
-        // this thread's 8 coefficients: fp32 chunks 2*cpart, 2*cpart+1 of the row
-        float4 f0 = *reinterpret_cast<const float4*>(row + (((2 * cpart) ^ csw) << 4));
-        float4 f1 = *reinterpret_cast<const float4*>(row + (((2 * cpart + 1) ^ csw) << 4));
-        uint4 hi, lo;
-        split2(f0.x * wt, f0.y * wt, hi.x, lo.x);
-        split2(f0.z * wt, f0.w * wt, hi.y, lo.y);
-        split2(f1.x * wt, f1.y * wt, hi.z, lo.z);
-        split2(f1.z * wt, f1.w * wt, hi.w, lo.w);
-        __syncwarp();                               // all four threads of the row have read
-        *reinterpret_cast<uint4*>(row + ((cpart ^ csw) << 4)) = hi;         // c1: chunks 0..3
-        *reinterpret_cast<uint4*>(row + (((4 + cpart) ^ csw) << 4)) = lo;   // c2: chunks 4..7
-        fence_proxy_async();
-        mbar_arrive(smem_u32(&ctrl->conv[c]));
-        ++epos;
-      }
-      return true;
-    };
-
-    if constexpr (!CV) {
-      if (!w.done()) alive = convert_tile(wn);
-    }
-    for (; alive && !w.done(); w.next(), ++i) {
-      // ---- 1. get the next tile's rank blocks converted and their MMAs going (unless the converter warps do that)
-      if constexpr (!CV) {
-        wn.next();
-        if (!wn.done()) {
-          if (!convert_tile(wn)) break;
-        }
-      }
+    uint32_t i = 0;
+    for (; !w.done(); w.next(), ++i) {
       const int s = i % NSTAGE, g = i & 1;
       const int t0 = w.t0(), is_v = w.is_v();
       uint8_t* st_ptr = smem + s * kBaseBytes;
       const bool has_coeff = t0 < p.cov_max;
 
-      // ---- 2. accumulator of this tile ready, base tile landed
+      // ---- 1. accumulator of this tile ready, base tile landed
       bool ok = mbar_wait(smem_u32(&ctrl->mma_done[g]), (i >> 1) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -477,7 +428,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
 
-      // ---- 3. rotate, add, round: row m, this warp's channel quarter, in place
+      // ---- 2. rotate, add, round: row m, this warp's channel quarter, in place
       const int tok = t0 + m;
       const bool in_range = tok < p.src.T;
       const bool covered = has_coeff && tok < p.cov_max;
@@ -568,7 +519,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_
           }
         }
       }
-      // ---- 4. the tile is final in shared memory: hand it to the store warp
+      // ---- 3. the tile is final in shared memory: hand it to the store warp
       fence_proxy_async();
       mbar_arrive(smem_u32(&ctrl->ready[s]));
     }
@@ -584,7 +535,7 @@ __global__ void __launch_bounds__(CV ? kThreadsCv : kThreads, 1) apply_multi_tc_
   }
 }
 
-template <int NSTAGE, int NC, int NO, bool CV = false>
+template <int NSTAGE, int NC, int NO>
 static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
                           (size_t)NO * kOperandBytes + sizeof(Ctrl<NSTAGE, NC, NO>);
@@ -592,11 +543,11 @@ static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     once.mark(once_dev);
   }
-  apply_multi_tc_kernel<NSTAGE, NC, NO, CV><<<grid, CV ? kThreadsCv : kThreads, smem, s>>>(M);
+  apply_multi_tc_kernel<NSTAGE, NC, NO><<<grid, kThreadsCv, smem, s>>>(M);
   return cudaGetLastError();
 }
 
@@ -684,7 +635,7 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
   const int grid = (int)(M.total_tiles < sms ? M.total_tiles : sms);
-  const cudaError_t e = tcm::launch_multi_t<3, 5, 2, true>(M, grid, s);
+  const cudaError_t e = tcm::launch_multi_t<3, 5, 2>(M, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
