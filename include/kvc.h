@@ -368,15 +368,20 @@ int kvc_state_update_noalloc(const kvc_cache *src, const kvc_cache *tgt, int32_t
  * Why the items are a host array and the call makes one host-to-device copy: the work table carries
  * tensor maps, which only the host can encode, and the per-CTA ranges of equal estimated time; building
  * them is this call's job, and one copy of a few hundred KB per launch replaces a second API for it.
- * An item is a whole cache: a context made of several segments with different shifts is ONE item of
- * kvc_apply_segmented's kind (a token range inside a paged cache would need page-aligned table slices
- * and partial-tile stores that must not touch the neighbouring segment's rows).
+ * An item works on the token range [t_begin, t_end) of its caches (0, 0: all rows), so a context made of
+ * several shared pieces at different offsets (Eq. 1) is one item per piece over the same caches, each with
+ * its own shift: rows outside the range stay untouched in dst, row t of the state's coefficients corrects
+ * token t (absolute), covered are the rows t < st.n_cov.  Errors: KVC_E_INVALID_ARG unless
+ * 0 <= t_begin < t_end <= T of both caches; KVC_E_UNSUPPORTED when a paged cache's range does not start
+ * on a page boundary (kvc_apply_segmented takes boundaries anywhere, for one request at a time).
+ * Ranges of two items of one launch must not overlap in dst.
  */
 typedef struct kvc_item {
   kvc_cache src;
   kvc_cache dst;
   kvc_state st;
   int32_t shift;
+  int32_t t_begin, t_end;   /* token range of the item; both 0: the whole cache */
   int32_t reserved;
 } kvc_item;
 

@@ -69,7 +69,7 @@ class kvc_segments(C.Structure):
 
 class kvc_item(C.Structure):
     _fields_ = [("src", kvc_cache), ("dst", kvc_cache), ("st", kvc_state), ("shift", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("t_begin", C.c_int32), ("t_end", C.c_int32), ("reserved", C.c_int32)]
 
 
 _lib = None
@@ -410,8 +410,11 @@ def kvc_state_update_noalloc(src: Optional[Cache], tgt: Cache, shift: int, rope:
 
 
 class Item:
-    def __init__(self, src: Cache, dst: Cache, st: State, shift: int):
+    """One work item of kvc_apply_batch; (t_begin, t_end) = (0, 0) means all rows of the caches."""
+
+    def __init__(self, src: Cache, dst: Cache, st: State, shift: int, t_begin: int = 0, t_end: int = 0):
         self.src, self.dst, self.st, self.shift = src, dst, st, int(shift)
+        self.t_begin, self.t_end = int(t_begin), int(t_end)
 
 
 def kvc_batch_workspace_bytes(n_items: int) -> int:
@@ -424,6 +427,7 @@ def kvc_apply_batch(items: Sequence[Item], rope: Rope, workspace: torch.Tensor, 
     arr = (kvc_item * max(n, 1))()
     for i, it in enumerate(items):
         arr[i].src, arr[i].dst, arr[i].st, arr[i].shift = it.src.struct(), it.dst.struct(), it.st.struct(), it.shift
+        arr[i].t_begin, arr[i].t_end = getattr(it, "t_begin", 0), getattr(it, "t_end", 0)
     r = rope.struct()
     assert staging.device.type == "cpu" and staging.numel() * staging.element_size() >= kvc_batch_workspace_bytes(n)
     _check(load().kvc_apply_batch(arr, n, C.byref(r), workspace.data_ptr(),

@@ -92,6 +92,8 @@ static int resolve_state(const kvc_state* st, int for_update, DevState* out) {
   d.n_cov = st->n_cov;
   d.basis_bf16 = st->basis_dtype == KVC_BF16;
   d.grouped = st->grouping == KVC_GROUP_LAYER;
+  d.coeff_rows = st->n_cov;
+  d.pad_[0] = d.pad_[1] = d.pad_[2] = 0;
   *out = d;
   return KVC_OK;
 }
@@ -712,6 +714,31 @@ size_t kvc_batch_workspace_bytes(int32_t n_items) {
   return batch_prefix_bytes(n_items) + (size_t)n_items * sizeof(DevItem) + tc_batch_extra_bytes(n_items);
 }
 
+// Narrows a resolved hop to the token range [t_begin, t_end) of its caches: the caches start at row
+// t_begin and are t_end - t_begin rows long, the coefficient rows start at row t_begin of every slab
+// (whose spacing stays that of the whole state), n_cov counts the covered rows inside the window.
+static int window_item(DevItem* it, int32_t t_begin, int32_t t_end) {
+  if (t_begin < 0 || t_end <= t_begin || t_end > it->src.T || t_end > it->dst.T) return KVC_E_INVALID_ARG;
+  for (DevCache* c : {&it->src, &it->dst}) {
+    if (c->page_table) {
+      if (t_begin & c->page_mask) return KVC_E_UNSUPPORTED;   // a paged window starts on a page boundary
+      c->page_table += t_begin >> c->page_shift;
+    } else {
+      c->k += (int64_t)t_begin * c->s_tok;
+      c->v += (int64_t)t_begin * c->s_tok;
+    }
+    c->T = t_end - t_begin;
+  }
+  DevState& st = it->st;
+  if (st.r > 0 && st.n_cov > 0) {
+    const int32_t cov = st.n_cov - t_begin;
+    st.coeff_k += (int64_t)t_begin * st.r;
+    st.coeff_v += (int64_t)t_begin * st.r;
+    st.n_cov = cov < 0 ? 0 : (cov > t_end - t_begin ? t_end - t_begin : cov);
+  }
+  return KVC_OK;
+}
+
 int kvc_apply_batch(const kvc_item* items, int32_t n_items, const kvc_rope* rope, void* workspace,
                     size_t workspace_bytes, void* staging, void* stream) {
   if (n_items < 0 || (n_items > 0 && !items)) return KVC_E_INVALID_ARG;
@@ -733,6 +760,9 @@ int kvc_apply_batch(const kvc_item* items, int32_t n_items, const kvc_rope* rope
     if ((rc = resolve_hop(&items[i].src, &items[i].st, items[i].shift, rope, &items[i].dst, &hop)) != KVC_OK) return rc;
     if (hop.d != d) return KVC_E_SHAPE;
     tab[i] = hop.item;
+    if (items[i].t_begin != 0 || items[i].t_end != 0) {
+      if ((rc = window_item(&tab[i], items[i].t_begin, items[i].t_end)) != KVC_OK) return rc;
+    }
   }
   if (tl_path_force != KVC_PATH_GENERIC) {
     const int trc = tc_apply_batch(tab, prefix, n_items, d, rope->pairing, status, workspace, staging, need, s);
@@ -953,6 +983,7 @@ int kvc_gate_distance(const kvc_cache* src, const kvc_state* anchors, int32_t n_
       it.st.basis_k = it.st.basis_v = a.basis_v;
       it.st.r = a.r;
       it.st.n_cov = a.n_cov;
+      it.st.coeff_rows = a.n_cov;
       it.st.basis_bf16 = a.basis_dtype == KVC_BF16;
       it.st.grouped = a.grouping == KVC_GROUP_LAYER;
       it.L = src->L;

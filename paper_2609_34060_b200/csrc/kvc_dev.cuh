@@ -24,6 +24,8 @@ struct DevState {
   const void* basis_k;
   const void* basis_v;
   int32_t r, n_cov, basis_bf16, grouped;   // grouped: one state per layer, coeff [L,n_cov,r], basis [L,r,H*d]
+  int32_t coeff_rows;                      // rows between two coefficient slabs (= n_cov, unless the item is a token
+  int32_t pad_[3];                         // window of a longer state: then n_cov counts the window's covered rows)
 };
 
 // Index of the coefficient slab and element offset of basis row q of (layer l, head h), in elements.

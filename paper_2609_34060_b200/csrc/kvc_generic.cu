@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(256) apply_generic_kernel(const __grid_constan
       for (int i = tid; i < TILE * rc; i += 256) {
         const int tl = i / rc, q = i - tl * rc;
         const int t = t0 + tl;
-        coeff_s[tl * (RC + 1) + q] = (t < n_cov) ? coeff[(cslab * it.st.n_cov + t) * r + q0 + q] : 0.f;
+        coeff_s[tl * (RC + 1) + q] = (t < n_cov) ? coeff[(cslab * (it.st.coeff_rows > 0 ? it.st.coeff_rows : it.st.n_cov) + t) * r + q0 + q] : 0.f;
       }
       __syncthreads();
       for (int q = 0; q < rc; ++q) {

@@ -992,8 +992,8 @@ static bool build_maps(const DevItem& it, ItemMaps* mp) {
   bool ok = encode_cache(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
             encode_cache(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
   const int cslabs = it.st.grouped ? it.L : it.L * it.H;
-  ok = ok && encode_coeff(&mp->coeff_k, it.st.coeff_k, it.st.r, it.st.n_cov, cslabs) &&
-       encode_coeff(&mp->coeff_v, it.st.coeff_v, it.st.r, it.st.n_cov, cslabs);
+  ok = ok && encode_coeff(&mp->coeff_k, it.st.coeff_k, it.st.r, it.st.n_cov, cslabs, it.st.coeff_rows) &&
+       encode_coeff(&mp->coeff_v, it.st.coeff_v, it.st.r, it.st.n_cov, cslabs, it.st.coeff_rows);
   return ok;
 }
 

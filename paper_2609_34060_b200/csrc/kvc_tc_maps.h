@@ -43,11 +43,13 @@ inline bool encode_cache(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-inline bool encode_coeff(CUtensorMap* m, const float* coeff, int r, int n_cov, int slabs) {
+// slab_rows: rows between two slabs (0: n_cov, the dense layout)
+inline bool encode_coeff(CUtensorMap* m, const float* coeff, int r, int n_cov, int slabs, int slab_rows = 0) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
+  if (slab_rows <= 0) slab_rows = n_cov;
   const cuuint64_t dims[3] = {(cuuint64_t)r, (cuuint64_t)n_cov, (cuuint64_t)slabs};
-  const cuuint64_t strides[2] = {(cuuint64_t)r * 4, (cuuint64_t)r * 4 * (cuuint64_t)n_cov};
+  const cuuint64_t strides[2] = {(cuuint64_t)r * 4, (cuuint64_t)r * 4 * (cuuint64_t)slab_rows};
   const cuuint32_t box[3] = {32, 128, 1};
   const cuuint32_t es[3] = {1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(coeff), dims, strides, box, es,

@@ -221,3 +221,64 @@ def test_grouped_state_with_segments():
         Btrue = Bo[0].numpy().astype(np.float64)
         assert np.max(np.abs(B @ B.T - np.eye(r))) <= 1e-4
         assert np.linalg.norm(B.T @ B - Btrue.T @ Btrue) <= 2e-2          # the rows span the true basis' space
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The same multi-segment context as ONE launch of kvc_apply_batch: an item per segment over the same
+# caches, each with its token range and its own shift.
+# ---------------------------------------------------------------------------------------------------------
+ITEM_SEGS = {"8b_small": ([0, 133, 390], [37, 0, -211]),      # contiguous: boundaries anywhere
+             "vlm_small": ([0, 32, 528], [-5, 512, 64])}      # paged: boundaries on 16-token pages
+
+
+@pytest.mark.parametrize("path", [kvc.KVC_PATH_GENERIC, kvc.KVC_PATH_AUTO], ids=["generic", "auto"])
+@pytest.mark.parametrize("cfg", [CFG_C, CFG_P], ids=lambda c: c.name)
+def test_batch_items_with_token_ranges(cfg, path):
+    kvc.kvc_set_path(path)
+    t_begin, shift = ITEM_SEGS[cfg.name]
+    T = cfg.T
+    t_stop = T - 29                                 # the last rows belong to no item: they keep the fill
+    s_tok = orc.segment_shifts(T, t_begin, shift)
+    f = hp.inv_freq(cfg)
+    src_cpu = hp.make_cache(cfg)
+    n_cov = t_begin[2] + 77                         # the coverage ends inside the last segment
+    st_cpu = hp.make_state(cfg, 1, n_cov=n_cov)
+    src, st = hp.to_dev(src_cpu, DEV), hp.state_to_dev(st_cpu, DEV)
+    dst = hp.empty_dst(src_cpu, cfg, DEV, fill=1.0)
+    ends = t_begin[1:] + [t_stop]
+    items = [kvc.Item(src, dst, st, sh, tb, te) for tb, te, sh in zip(t_begin, ends, shift)]
+    nb = kvc.kvc_batch_workspace_bytes(len(items))
+    ws = torch.empty(nb, dtype=torch.uint8, device=DEV)
+    staging = torch.empty(nb, dtype=torch.uint8).pin_memory()
+    kvc.kvc_apply_batch(items, kvc.Rope(cfg.theta), ws, staging)
+    torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == (kvc.KVC_PATH_TC if path == kvc.KVC_PATH_AUTO else kvc.KVC_PATH_GENERIC)
+    osrc, ost = hp.oracle_cache(src_cpu), hp.oracle_state(st_cpu)
+    one = orc.f64_to_bf16_bits(np.ones(1))[0]
+    for which in ("k", "v"):
+        got = hp.logical_bits(dst, which)
+        for l in range(cfg.L):
+            for h in range(cfg.H):
+                c = (ost.coeff_k if which == "k" else ost.coeff_v)[l, h]
+                b = (ost.basis_k if which == "k" else ost.basis_v)[l, h]
+                ref, exp = orc.apply_slab_tokens(osrc.get_bits(which, l, h), c, b, s_tok, f, n_cov, which == "k")
+                assert hp.tol_ratio(got[l, h][:t_stop], ref[:t_stop]) <= 1.0, (which, l, h)
+                assert hp.ulp_mismatch_fraction(got[l, h][:t_stop], exp[:t_stop]) < 1e-2
+                assert np.all(got[l, h][t_stop:] == one), "rows outside every item's range were written"
+
+
+def test_batch_item_range_errors():
+    cfg = CFG_P
+    src_cpu = hp.make_cache(cfg)
+    st = hp.state_to_dev(hp.make_state(cfg, 1), DEV)
+    src = hp.to_dev(src_cpu, DEV)
+    dst = hp.empty_dst(src_cpu, cfg, DEV)
+    nb = kvc.kvc_batch_workspace_bytes(1)
+    ws = torch.empty(nb, dtype=torch.uint8, device=DEV)
+    staging = torch.empty(nb, dtype=torch.uint8).pin_memory()
+    rope = kvc.Rope(cfg.theta)
+    for tb, te, code in ((10, 5, kvc.KVC_E_INVALID_ARG), (0, cfg.T + 1, kvc.KVC_E_INVALID_ARG), (-16, 32, kvc.KVC_E_INVALID_ARG),
+                         (8, 64, kvc.KVC_E_UNSUPPORTED)):        # a paged range must start on a page boundary
+        with pytest.raises(kvc.KvcError) as e:
+            kvc.kvc_apply_batch([kvc.Item(src, dst, st, 3, tb, te)], rope, ws, staging)
+        assert e.value.code == code, (tb, te, str(e.value))
