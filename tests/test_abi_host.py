@@ -38,7 +38,7 @@ def test_struct_sizes_match_the_header(lib):
     assert C.sizeof(kvc.kvc_cache) == 8 + 8 + 7 * 4 + 4 + 8 + 32
     assert C.sizeof(kvc.kvc_state) == 4 * 8 + 4 * 4
     assert C.sizeof(kvc.kvc_rope) == 8 + 4 + 4 + 8
-    assert C.sizeof(kvc.kvc_item) == 2 * C.sizeof(kvc.kvc_cache) + C.sizeof(kvc.kvc_state) + 8
+    assert C.sizeof(kvc.kvc_item) == 2 * C.sizeof(kvc.kvc_cache) + C.sizeof(kvc.kvc_state) + 16   # shift, t_begin, t_end, reserved
 
 
 def _cache(k=0x1000, v=0x100000, L=2, H=2, T=64, d=128, layout=kvc.KVC_CONTIG, **kw):
