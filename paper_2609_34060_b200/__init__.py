@@ -235,6 +235,64 @@ class State:
         assert basis_v.dtype in (torch.float32, torch.bfloat16) and int(coeff_v.shape[3]) == s.r
         return s
 
+    # ---- a state as one self-describing blob (header, coefficients, bases): checkpoint / resume of a profiled
+    # correction, and the way to keep a failing case.  Host-side plumbing only.
+    _BLOB_MAGIC = b"KVCSTATE"
+
+    def dump(self) -> bytes:
+        import struct as _st
+        parts, meta = [], []
+        for t in (self.coeff_k, self.coeff_v, self.basis_k, self.basis_v):
+            if t is None:
+                meta.append((0, 0, ()))
+                continue
+            c = t.detach().cpu().contiguous()
+            raw = c.view(torch.int16).numpy().tobytes() if c.dtype == torch.bfloat16 else c.numpy().tobytes()
+            meta.append((1, 2 if c.dtype == torch.bfloat16 else 4, tuple(int(x) for x in c.shape)))
+            parts.append(raw)
+        head = self._BLOB_MAGIC + _st.pack("<5i", 1, self.r, self.n_cov, getattr(self, "grouping", KVC_GROUP_HEAD), len(meta))
+        for present, esize, shape in meta:
+            head += _st.pack("<3i", present, esize, len(shape)) + _st.pack("<%dq" % len(shape), *shape)
+        return head + b"".join(parts)
+
+    @staticmethod
+    def load(blob: bytes, device="cpu") -> "State":
+        import struct as _st
+        import numpy as _np
+        if blob[:8] != State._BLOB_MAGIC:
+            raise ValueError("not a state blob")
+        ver, r, n_cov, grouping, n = _st.unpack_from("<5i", blob, 8)
+        if ver != 1 or n != 4:
+            raise ValueError("unknown state blob version")
+        off, meta = 8 + 20, []
+        for _ in range(n):
+            present, esize, nd = _st.unpack_from("<3i", blob, off)
+            off += 12
+            shape = _st.unpack_from("<%dq" % nd, blob, off)
+            off += 8 * nd
+            meta.append((present, esize, shape))
+        ts = []
+        for present, esize, shape in meta:
+            if not present:
+                ts.append(None)
+                continue
+            cnt = 1
+            for x in shape:
+                cnt *= x
+            if esize == 2:
+                a = _np.frombuffer(blob, dtype=_np.int16, count=cnt, offset=off).copy()
+                t = torch.from_numpy(a).view(torch.bfloat16)
+            else:
+                a = _np.frombuffer(blob, dtype=_np.float32, count=cnt, offset=off).copy()
+                t = torch.from_numpy(a)
+            off += cnt * esize
+            ts.append(t.reshape(shape).to(device))
+        if off != len(blob):
+            raise ValueError("state blob has trailing or missing bytes")
+        if ts[0] is None and ts[2] is None and ts[3] is not None:
+            return State.values_only(ts[1], ts[3])
+        return State(ts[0], ts[1], ts[2], ts[3], n_cov=n_cov, grouping=grouping)
+
     def struct(self) -> kvc_state:
         s = kvc_state()
         ptr = lambda t: 0 if t is None else t.data_ptr()

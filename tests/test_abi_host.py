@@ -5,6 +5,7 @@ import os
 import re
 
 import pytest
+import torch
 
 import paper_2609_34060_b200 as kvc
 from paper_2609_34060_b200 import build as kbuild
@@ -181,3 +182,31 @@ def test_multi_anchor_and_grouping_argument_errors(lib):
     assert lib.kvc_fit_eigenvalues(C.byref(src), None) is None
     assert lib.kvc_state_realign(C.byref(st8), 2, 2, 96, 5, C.byref(rope), 0x8000000, None) == -3
     assert lib.kvc_state_realign(C.byref(st8), 2, 2, 128, 5, C.byref(rope), None, None) == -1
+
+
+def test_state_blob_round_trip():
+    """A state goes to one self-describing blob and back bit for bit (per-head, grouped, bf16 bases, value factors
+    only, empty), and a damaged blob is refused."""
+    g = torch.Generator().manual_seed(3)
+    L, H, T, r, d = 2, 3, 17, 4, 8
+    per_head = kvc.State(torch.randn(L, H, T, r, generator=g), torch.randn(L, H, T, r, generator=g),
+                         torch.randn(L, H, r, d, generator=g), torch.randn(L, H, r, d, generator=g), n_cov=T)
+    grouped = kvc.State(torch.randn(L, T, r, generator=g), torch.randn(L, T, r, generator=g),
+                        torch.randn(L, r, H * d, generator=g).bfloat16(), torch.randn(L, r, H * d, generator=g).bfloat16(),
+                        grouping=kvc.KVC_GROUP_LAYER)
+    values = kvc.State.values_only(torch.randn(L, H, T, r, generator=g), torch.randn(L, H, r, d, generator=g))
+    for st in (per_head, grouped, values, kvc.State.empty()):
+        back = kvc.State.load(st.dump())
+        assert (back.r, back.n_cov, getattr(back, "grouping", 0)) == (st.r, st.n_cov, getattr(st, "grouping", 0))
+        for name in ("coeff_k", "coeff_v", "basis_k", "basis_v"):
+            a, b = getattr(st, name), getattr(back, name)
+            assert (a is None) == (b is None)
+            if a is not None:
+                assert a.dtype == b.dtype and a.shape == b.shape
+                assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                                   b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+    blob = per_head.dump()
+    with pytest.raises(ValueError):
+        kvc.State.load(b"XXXXXXXX" + blob[8:])
+    with pytest.raises(ValueError):
+        kvc.State.load(blob[:-4])
