@@ -590,20 +590,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
 #pragma unroll
         for (int b = 0; b < RB; ++b) {
           if (b >= t.nb) break;                       // uniform over the CTA
-          uint8_t* row = c_ptr + b * kCoeffBlkBytes + ct * 128;
-          float4 f[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) f[k] = *reinterpret_cast<const float4*>(row + (((uint32_t)k ^ csw) << 4));
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {               // ranks 8 j .. 8 j + 7: heads to chunk j, tails to chunk 4 + j
-            uint4 hi, lo;
-            split2(f[2 * j].x, f[2 * j].y, hi.x, lo.x);
-            split2(f[2 * j].z, f[2 * j].w, hi.y, lo.y);
-            split2(f[2 * j + 1].x, f[2 * j + 1].y, hi.z, lo.z);
-            split2(f[2 * j + 1].z, f[2 * j + 1].w, hi.w, lo.w);
-            *reinterpret_cast<uint4*>(row + (((uint32_t)j ^ csw) << 4)) = hi;
-            *reinterpret_cast<uint4*>(row + (((uint32_t)(4 + j) ^ csw) << 4)) = lo;
-          }
+          convert_coeff_row(c_ptr + b * kCoeffBlkBytes + ct * 128, csw);
         }
         fence_proxy_async();
       }

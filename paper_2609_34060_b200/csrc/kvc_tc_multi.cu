@@ -384,20 +384,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
         }
         const bool weighted = (is_v ? p.blk[e].w_v : p.blk[e].w_k) != nullptr;
         const float wt = weighted ? reinterpret_cast<const float*>(smem + kWeightOff + c * kWeightBytes)[ct] : 1.f;
-        uint8_t* row = smem + kCoeffOff + c * kCoeffBytes + ct * 128;
-        float4 f[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) f[k] = *reinterpret_cast<const float4*>(row + (((uint32_t)k ^ csw) << 4));
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {                 // ranks 8 j .. 8 j + 7: heads to chunk j, tails to chunk 4 + j
-          uint4 hi, lo;
-          split2(f[2 * j].x * wt, f[2 * j].y * wt, hi.x, lo.x);
-          split2(f[2 * j].z * wt, f[2 * j].w * wt, hi.y, lo.y);
-          split2(f[2 * j + 1].x * wt, f[2 * j + 1].y * wt, hi.z, lo.z);
-          split2(f[2 * j + 1].z * wt, f[2 * j + 1].w * wt, hi.w, lo.w);
-          *reinterpret_cast<uint4*>(row + (((uint32_t)j ^ csw) << 4)) = hi;
-          *reinterpret_cast<uint4*>(row + (((uint32_t)(4 + j) ^ csw) << 4)) = lo;
-        }
+        convert_coeff_row(smem + kCoeffOff + c * kCoeffBytes + ct * 128, csw, wt);
         fence_proxy_async();
         mbar_arrive(smem_u32(&ctrl->conv[c]));
         ++epos;

@@ -170,6 +170,25 @@ __device__ __forceinline__ void split2(float x0, float x1, uint32_t& hi, uint32_
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
+// One row of a coefficient tile in shared memory (32 float32 = 128 bytes, its 16-byte chunks XOR-swizzled by
+// csw = row & 7) turned into the MMA's operand in place: chunk j (j < 4) gets the bf16 heads of ranks
+// 8 j .. 8 j + 7, chunk 4 + j their tails.  The whole row is read before anything is written.
+__device__ __forceinline__ void convert_coeff_row(uint8_t* row, uint32_t csw, float scale = 1.f) {
+  float4 f[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) f[k] = *reinterpret_cast<const float4*>(row + (((uint32_t)k ^ csw) << 4));
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint4 hi, lo;
+    split2(f[2 * j].x * scale, f[2 * j].y * scale, hi.x, lo.x);
+    split2(f[2 * j].z * scale, f[2 * j].w * scale, hi.y, lo.y);
+    split2(f[2 * j + 1].x * scale, f[2 * j + 1].y * scale, hi.z, lo.z);
+    split2(f[2 * j + 1].z * scale, f[2 * j + 1].w * scale, hi.w, lo.w);
+    *reinterpret_cast<uint4*>(row + (((uint32_t)j ^ csw) << 4)) = hi;
+    *reinterpret_cast<uint4*>(row + (((uint32_t)(4 + j) ^ csw) << 4)) = lo;
+  }
+}
+
 // 16 consecutive fp32 columns of this thread's TMEM lane
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
