@@ -16,7 +16,9 @@
 // KVC_FLAG_NOT_CONVERGED is raised.  The caller finishes with one projection pass on the final basis.
 //
 // The small dense work (orthonormalisation of r rows of length D by Cholesky QR, the r x r eigenproblem,
-// the Ritz rows) runs as one block of 256 threads per (layer, K|V) on rows that stay L2-resident.
+// the Ritz rows) runs as a cluster of four blocks of 256 threads per (layer, K|V), each on its slice of
+// the columns of rows that stay L2-resident.
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -128,16 +130,24 @@ __global__ void __launch_bounds__(256) group_backproject_kernel(const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------
-// Small dense work on r rows of length Dg, one block per (layer, K|V).
+// Small dense work on r rows of length Dg: a CLUSTER of kCl blocks per (layer, K|V).  Every block owns
+// a slice of the columns; sums over the columns (the r x r Gram matrices, per-row norms and residuals)
+// are formed per block and added over the cluster in rank order through distributed shared memory, so
+// that every block holds the same bits and the r x r steps (Cholesky factor, eigen-decomposition,
+// acceptance) are simply done by all of them.  One block per problem left 64 blocks on 148 SMs with
+// every global-memory round trip exposed.
 // ---------------------------------------------------------------------------------------------
+constexpr int kCl = 4;           // blocks per problem: 64 problems x 4 = 256 blocks, one wave at two blocks per SM (eight took two waves)
+
 struct SmallMem {
   float s[kMaxM * kSP];          // Gram matrix of the rows / Cholesky factor / scratch copy of H
   float h[kMaxM * kSP];          // projected matrix
   float w[kMaxM * kSP];          // its eigenvectors (sorted: ws)
+  float part[kMaxM * kSP];       // this block's share of a sum over the columns (read by the whole cluster)
   float ta[kMaxM * 65];          // column tiles of the two row blocks of a product
   float tb[kMaxM * 65];
   float pn[8 * kMaxM], pd[8 * kMaxM], pr[8 * kMaxM];   // per-warp partial sums per row
-  float pbest[8 * kMaxM];
+  float pbest[8 * kMaxM], pval[8 * kMaxM];
   int pidx[8 * kMaxM];
   float th[kMaxM], inv[kMaxM], rho2[kMaxM];
   int perm[kMaxM];
@@ -145,15 +155,32 @@ struct SmallMem {
   int flag;
 };
 
-// S[i][j] = sum_c A[i][c] B[j][c]  for i, j < 32 (rows >= m count as zero); rows have stride Dg.
-__device__ __forceinline__ void gram_rows(const float* A, const float* B, float* S, SmallMem& sm, int m, int Dg, int tid) {
+namespace cgx = cooperative_groups;
+
+// out[i] = sum over the cluster's blocks (rank order) of their part[i], i < n; every block gets the same bits.
+// part must be complete in every block's shared memory on entry (the first cluster barrier orders that).
+__device__ __forceinline__ void cluster_sum(cgx::cluster_group& cl, float* part, float* out, int n, int tid) {
+  cl.sync();
+  for (int i = tid; i < n; i += kThreads) {
+    float a = 0.f;
+#pragma unroll
+    for (int r = 0; r < kCl; ++r) a += cl.map_shared_rank(part, r)[i];
+    out[i] = a;
+  }
+  cl.sync();                                       // nobody overwrites its part while others still read it
+}
+
+// S[i][j] = sum_c A[i][c] B[j][c]  over ALL columns, for i, j < 32 (rows >= m count as zero); rows have
+// stride Dg; this block adds up the columns [c_lo, c_hi).
+__device__ __forceinline__ void gram_rows(cgx::cluster_group& cl, const float* A, const float* B, float* S, SmallMem& sm, int m,
+                                          int Dg, int c_lo, int c_hi, int tid) {
   const int j = tid & 31, i0 = tid >> 5;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int c0 = 0; c0 < Dg; c0 += 64) {
+  for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
     __syncthreads();
     for (int idx = tid; idx < kMaxM * 64; idx += kThreads) {
       const int i = idx >> 6, cc = idx & 63;
-      const bool on = i < m && c0 + cc < Dg;
+      const bool on = i < m && c0 + cc < c_hi;
       sm.ta[i * 65 + cc] = on ? A[(int64_t)i * Dg + c0 + cc] : 0.f;
       sm.tb[i * 65 + cc] = on ? B[(int64_t)i * Dg + c0 + cc] : 0.f;
     }
@@ -165,43 +192,64 @@ __device__ __forceinline__ void gram_rows(const float* A, const float* B, float*
       for (int k = 0; k < 4; ++k) acc[k] = fmaf(sm.ta[(i0 + 8 * k) * 65 + cc], bv, acc[k]);
     }
   }
-  __syncthreads();
 #pragma unroll
-  for (int k = 0; k < 4; ++k) S[(i0 + 8 * k) * kSP + j] = acc[k];
+  for (int k = 0; k < 4; ++k) sm.part[(i0 + 8 * k) * kSP + j] = acc[k];
+  cluster_sum(cl, sm.part, S, kMaxM * kSP, tid);
   __syncthreads();
 }
 
 // Cholesky factor of the m x m matrix S (in place, lower triangle, reciprocal pivots on the diagonal)
-// by warp 0.  shift_rel > 0 adds that fraction of the largest diagonal entry to the diagonal first.
+// by warp 0, left-looking with row `lane` of the factor in that lane's registers: at step j lane j
+// publishes its finished row and every lane below subtracts its part of column j.
+// shift_rel > 0 adds that fraction of the largest diagonal entry to the diagonal first.
 // Returns false when a pivot cancels (the rows are dependent at float32).
 __device__ __forceinline__ bool chol_small(float* S, SmallMem& sm, int m, int tid, float shift_rel) {
   if (tid < 32) {
     const int lane = tid;
+    float l[kMaxM];
+#pragma unroll
+    for (int k = 0; k < kMaxM; ++k) l[k] = (lane < m && k < m) ? S[k * kSP + lane] : 0.f;   // S is symmetric: column reads meet no bank conflict
     float d0 = (lane < m) ? S[lane * kSP + lane] : 0.f;
     const float dmax = wmax(d0);
-    if (lane < m && shift_rel > 0.f) {
-      d0 += shift_rel * dmax;
-      S[lane * kSP + lane] = d0;
-    }
+    if (lane < m && shift_rel > 0.f) d0 += shift_rel * dmax;
+#pragma unroll
+    for (int k = 0; k < kMaxM; ++k)
+      if (k == lane) l[k] = d0;
     __syncwarp();
+    float* rowbuf = sm.pn;                          // [32] the published row (free during the factorisation)
     bool ok = dmax > 0.f;
-    for (int j = 0; j < m && ok; ++j) {
-      const float piv = S[j * kSP + j];
-      const float dj = __shfl_sync(0xffffffffu, d0, j);
-      ok = piv > 1e-5f * dj;
-      const float rl = ok ? rsqrtf(piv) : 0.f;
-      float lij = 0.f;
-      if (lane > j && lane < m) {
-        lij = S[lane * kSP + j] * rl;
-        S[lane * kSP + j] = lij;
+    float dacc = 0.f;                               // sum of the squares of this lane's finished entries
+#pragma unroll
+    for (int j = 0; j < kMaxM; ++j) {
+      if (j < m) {                                  // uniform over the warp
+        const float piv = __shfl_sync(0xffffffffu, l[j] - dacc, j);
+        const float dj = __shfl_sync(0xffffffffu, d0, j);
+        const bool good = piv > 1e-5f * dj;
+        ok = ok && good;
+        const float rl = good ? rsqrtf(piv) : 0.f;
+        if (lane == j) {
+#pragma unroll
+          for (int k = 0; k < kMaxM; ++k)
+            if (k < j) rowbuf[k] = l[k];
+        }
+        __syncwarp();
+        float acc = l[j];
+#pragma unroll
+        for (int k = 0; k < kMaxM; ++k)
+          if (k < j) acc = fmaf(-l[k], rowbuf[k], acc);
+        const float lij = acc * rl;
+        if (lane > j && lane < m) {
+          l[j] = lij;
+          dacc = fmaf(lij, lij, dacc);
+        }
+        if (lane == j) l[j] = rl;                   // reciprocal pivot on the diagonal
+        __syncwarp();
       }
-      __syncwarp();
-      if (lane > j && lane < m) {
-        for (int k = j + 1; k <= lane; ++k) S[lane * kSP + k] = fmaf(-lij, S[k * kSP + j], S[lane * kSP + k]);
-      }
-      if (lane == j) S[j * kSP + j] = rl;
-      __syncwarp();
     }
+    // the factor back to shared memory: row lane, columns 0 .. lane
+#pragma unroll
+    for (int k = 0; k < kMaxM; ++k)
+      if (lane < m && k <= lane) S[lane * kSP + k] = l[k];
     if (lane == 0) sm.flag = ok ? 1 : 0;
   }
   __syncthreads();
@@ -210,9 +258,10 @@ __device__ __forceinline__ bool chol_small(float* S, SmallMem& sm, int m, int ti
   return ok;
 }
 
-// Rows of Dst = L^-1 (rows of A): every thread solves the triangular system for its own columns.
-__device__ __forceinline__ void solve_rows(const float* A, float* Dst, const float* S, int m, int Dg, int tid) {
-  for (int c = tid; c < Dg; c += kThreads) {
+// Rows of Dst = L^-1 (rows of A) on the columns [c_lo, c_hi): every thread solves the triangular system
+// for its own columns.
+__device__ __forceinline__ void solve_rows(const float* A, float* Dst, const float* S, int m, int Dg, int c_lo, int c_hi, int tid) {
+  for (int c = c_lo + tid; c < c_hi; c += kThreads) {
     float x[kMaxM];
 #pragma unroll
     for (int j = 0; j < kMaxM; ++j) x[j] = (j < m) ? A[(int64_t)j * Dg + c] : 0.f;
@@ -232,25 +281,26 @@ __device__ __forceinline__ void solve_rows(const float* A, float* Dst, const flo
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_constant__ GroupFitLaunch p, int op) {
+__global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kThreads) group_small_kernel(const __grid_constant__ GroupFitLaunch p, int op) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SmallMem& sm = *reinterpret_cast<SmallMem*>(smem_raw);
-  if (p.round > 0 && p.need_more[p.round] == 0) return;       // a refinement round nobody asked for
+  if (p.round > 0 && p.need_more[p.round] == 0) return;       // a refinement round nobody asked for (the whole grid returns)
+  cgx::cluster_group cl = cgx::this_cluster();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int prob = blockIdx.x;                    // l * 2 + is_v
+  const int prob = blockIdx.x / kCl;              // l * 2 + is_v
+  const int rank = (int)cl.block_rank();
   const int l = prob >> 1, is_v = prob & 1;
   const int Dg = p.H * p.d;
+  const int c_lo = (int)((int64_t)rank * Dg / kCl), c_hi = (int)((int64_t)(rank + 1) * Dg / kCl);   // this block's columns
   const int m = min(min(p.r, Dg), p.n_cov);
   float* Q = (is_v ? p.basis_v : p.basis_k) + (int64_t)l * p.r * Dg;          // [r][Dg]
   float* Y = p.ypart + (int64_t)prob * p.r * Dg;                               // part 0 doubles as the sum
   int32_t* code = p.solver + prob;
 
   if (op == KVC_GROUP_OP_START) {
-    for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) {
-      const int q = (int)(i / Dg), c = (int)(i - (int64_t)q * Dg);
-      Q[i] = (q < m) ? start_value(c, q) : 0.f;
-    }
-    if (tid == 0) {
+    for (int q = 0; q < p.r; ++q)
+      for (int c = c_lo + tid; c < c_hi; c += kThreads) Q[(int64_t)q * Dg + c] = (q < m) ? start_value(c, q) : 0.f;
+    if (tid == 0 && rank == 0) {
       *code = 0;
       if (prob == 0)
         for (int k = 0; k <= kGroupFitRounds; ++k) p.need_more[k] = 0;
@@ -258,15 +308,21 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
     return;
   }
 
-  // the partial sums of the back-projection, added in a fixed order
-  if (op != KVC_GROUP_OP_ORTH_KEEP)
-  for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) {
-    float a = Y[i];
-    for (int part = 1; part < p.parts; ++part) a += p.ypart[((int64_t)part * p.L * 2 + prob) * p.r * Dg + i];
-    Y[i] = a;
+  // the partial sums of the back-projection, added in a fixed order (this block's columns)
+  if (op != KVC_GROUP_OP_ORTH_KEEP) {
+    for (int q = 0; q < p.r; ++q)
+      for (int c = c_lo + tid; c < c_hi; c += kThreads) {
+        const int64_t i = (int64_t)q * Dg + c;
+        float a = Y[i];
+        for (int part = 1; part < p.parts; ++part) a += p.ypart[((int64_t)part * p.L * 2 + prob) * p.r * Dg + i];
+        Y[i] = a;
+      }
   }
   __syncthreads();
-  if (*code == KVC_SOLVER_FULL_DEPENDENT && op != KVC_GROUP_OP_RITZ) return;   // given up earlier: nothing to orthonormalise
+  // (every block of the cluster reads the code here, before any of them can have written it below: the cluster
+  // barriers of the first product lie in between)
+  const int code_in = *code;
+  if (code_in == KVC_SOLVER_FULL_DEPENDENT && op != KVC_GROUP_OP_RITZ) return;   // given up earlier: nothing to orthonormalise
 
   if (op == KVC_GROUP_OP_ORTH || op == KVC_GROUP_OP_ORTH_START || op == KVC_GROUP_OP_ORTH_KEEP) {
     // Cholesky QR on the rows of Y: a shifted pass first where the conditioning is unknown (the
@@ -274,42 +330,63 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
     const int passes = (op == KVC_GROUP_OP_ORTH_START) ? 3 : 2;
     const float* src = Y;
     for (int pass = 0; pass < passes; ++pass) {
-      gram_rows(src, src, sm.s, sm, m, Dg, tid);
+      gram_rows(cl, src, src, sm.s, sm, m, Dg, c_lo, c_hi, tid);
       const bool shifted = (pass == 0);
-      if (!chol_small(sm.s, sm, m, tid, shifted ? 1e-5f : 0.f)) {
-        if (tid == 0) *code = KVC_SOLVER_FULL_DEPENDENT;
+      if (!chol_small(sm.s, sm, m, tid, shifted ? 1e-5f : 0.f)) {       // the same matrix in every block: the same answer
+        if (tid == 0 && rank == 0) *code = KVC_SOLVER_FULL_DEPENDENT;
         return;
       }
-      solve_rows(src, Q, sm.s, m, Dg, tid);
+      solve_rows(src, Q, sm.s, m, Dg, c_lo, c_hi, tid);
       src = Q;
     }
     return;
   }
 
   // ---- KVC_GROUP_OP_RITZ: Rayleigh-Ritz on (Q, Y = Q G), acceptance, output
+  // trace(G) = |Delta|_F^2 from the back-projection's partial sums: loaded in parallel, added in a fixed order
   float tr = 0.f;
-  for (int part = 0; part < p.tr_parts; ++part)
-    for (int h = 0; h < p.H; ++h) tr += p.trpart[((int64_t)part * p.L * 2 + prob) * p.H + h];
+  {
+    const int n_tr = p.tr_parts * p.H;
+    float mine = 0.f;
+    for (int i = tid; i < n_tr; i += kThreads) {   // (thread t takes entries t, t + 256, ...: more than 256 entries only with many heads)
+      const int part = i / p.H, h = i - part * p.H;
+      mine += p.trpart[((int64_t)part * p.L * 2 + prob) * p.H + h];
+    }
+    sm.ta[tid] = mine;
+    __syncthreads();
+    if (tid < 32) {
+      float a = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) a += sm.ta[8 * tid + k];
+      sm.tb[tid] = a;
+    }
+    __syncthreads();
+    for (int k = 0; k < 32; ++k) tr += sm.tb[k];
+    __syncthreads();
+  }
   float* evals = p.evals + (int64_t)prob * Dg;
-  if (*code == KVC_SOLVER_FULL_DEPENDENT || !(tr > 0.f)) {
+  if (code_in == KVC_SOLVER_FULL_DEPENDENT || !(tr > 0.f)) {
     // a zero deviation (or rows that became dependent): no basis, all eigenvalues zero
-    for (int64_t i = tid; i < (int64_t)p.r * Dg; i += kThreads) Q[i] = 0.f;
-    for (int i = tid; i < Dg; i += kThreads) evals[i] = 0.f;
-    for (int i = tid; i < kMaxM * kMaxM; i += kThreads) p.mtx[(int64_t)prob * kMaxM * kMaxM + i] = 0.f;
-    if (tid == 0) {
-      *code = KVC_SOLVER_FULL_DEPENDENT;
-      if (tr > 0.f) atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
+    for (int q = 0; q < p.r; ++q)
+      for (int c = c_lo + tid; c < c_hi; c += kThreads) Q[(int64_t)q * Dg + c] = 0.f;
+    for (int i = c_lo + tid; i < c_hi; i += kThreads) evals[i] = 0.f;
+    if (rank == 0) {
+      for (int i = tid; i < kMaxM * kMaxM; i += kThreads) p.mtx[(int64_t)prob * kMaxM * kMaxM + i] = 0.f;
+      if (tid == 0) {
+        *code = KVC_SOLVER_FULL_DEPENDENT;
+        if (tr > 0.f) atomicOr(p.status, KVC_FLAG_NOT_CONVERGED);
+      }
     }
     return;
   }
-  gram_rows(Q, Y, sm.s, sm, m, Dg, tid);
+  gram_rows(cl, Q, Y, sm.s, sm, m, Dg, c_lo, c_hi, tid);
   for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
     const int a = i >> 5, b = i & 31;
     sm.h[a * kSP + b] = 0.5f * (sm.s[a * kSP + b] + sm.s[b * kSP + a]);
   }
   __syncthreads();
   int reason = 0;
-  if (!jacobi_eig(sm.h, sm.s, sm.w, &sm.flag, m, tid)) reason = KVC_SOLVER_FULL_SWEEPS;
+  if (!jacobi_eig(sm.h, sm.s, sm.w, &sm.flag, m, tid)) reason = KVC_SOLVER_FULL_SWEEPS;     // every block, on the same bits
   // Ritz values in descending order (the rotations leave them in an arbitrary one)
   {
     const int nj = 2 * ((m + 1) >> 1);
@@ -317,15 +394,15 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
       // the padded slot of an odd m: the one whose eigenvector is still the unit vector e_m
       const bool real = tid < nj && !(nj != m && sm.w[m * kSP + tid] != 0.f);
       const float mine = real ? sm.h[tid * kSP + tid] : 0.f;
-      int rank = 0;
+      int rk = 0;
       for (int i = 0; i < nj; ++i) {
         const bool ireal = !(nj != m && sm.w[m * kSP + i] != 0.f);
         const float o = sm.h[i * kSP + i];
-        if (ireal && real) rank += (o > mine || (o == mine && i < tid)) ? 1 : 0;
+        if (ireal && real) rk += (o > mine || (o == mine && i < tid)) ? 1 : 0;
       }
       sm.perm[tid] = 0;
       __syncwarp();
-      if (real) sm.perm[rank] = tid;
+      if (real) sm.perm[rk] = tid;
     }
     __syncthreads();
     for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
@@ -335,16 +412,17 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
     for (int i = tid; i < 8 * kMaxM; i += kThreads) {
       sm.pn[i] = sm.pd[i] = sm.pr[i] = 0.f;
       sm.pbest[i] = -1.f;
+      sm.pval[i] = 0.f;
       sm.pidx[i] = 0;
     }
     __syncthreads();
   }
   const float* Ws = sm.s;
   // pass 1: Ritz rows z_j = sum_k Ws[k][j] q_k over Q (in place) and G z_j over Y (in place), with the
-  // sums z.Gz, z.z and the largest-magnitude entry of every row
-  for (int c0 = 0; c0 < Dg; c0 += kThreads) {
+  // sums z.Gz, z.z and the largest-magnitude entry of every row (its value travels with it: the sign rule)
+  for (int c0 = c_lo; c0 < c_hi; c0 += kThreads) {
     const int c = c0 + tid;
-    const bool on = c < Dg;
+    const bool on = c < c_hi;
     float q[kMaxM], y[kMaxM];
 #pragma unroll
     for (int k = 0; k < kMaxM; ++k) {
@@ -364,31 +442,37 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
         Y[(int64_t)j * Dg + c] = gj;
       }
       const float n1 = wsum(zj * gj), d1 = wsum(zj * zj);
-      float best = fabsf(zj);
+      float best = on ? fabsf(zj) : -1.f, bval = zj;
       int bi = on ? c : 0x7fffffff;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const float ov = __shfl_xor_sync(0xffffffffu, bval, o);
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
         if (ob > best || (ob == best && oi < bi)) {
           best = ob;
+          bval = ov;
           bi = oi;
         }
       }
       if (lane == 0) {
         sm.pn[warp * kMaxM + j] += n1;
         sm.pd[warp * kMaxM + j] += d1;
-        if (best > sm.pbest[warp * kMaxM + j]) {      // later tiles have larger indices: strict '>' keeps the first
+        const float cb = sm.pbest[warp * kMaxM + j];
+        if (best > cb || (best == cb && bi < sm.pidx[warp * kMaxM + j])) {
           sm.pbest[warp * kMaxM + j] = best;
+          sm.pval[warp * kMaxM + j] = bval;
           sm.pidx[warp * kMaxM + j] = bi;
         }
       }
     }
   }
   __syncthreads();
+  // this block's sums per row -> part[0..31] = z.Gz, [32..63] = z.z, [64..95] = largest |entry|, [96..127] = its value,
+  // [128..159] = its column (as float bits)
   if (tid < kMaxM) {
-    float ns = 0.f, ds = 0.f, best = -1.f;
-    int bi = 0;
+    float ns = 0.f, ds = 0.f, best = -1.f, bval = 0.f;
+    int bi = 0x7fffffff;
     for (int w = 0; w < 8; ++w) {
       ns += sm.pn[w * kMaxM + tid];
       ds += sm.pd[w * kMaxM + tid];
@@ -396,25 +480,50 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
       const int oi = sm.pidx[w * kMaxM + tid];
       if (ob > best || (ob == best && oi < bi)) {
         best = ob;
+        bval = sm.pval[w * kMaxM + tid];
+        bi = oi;
+      }
+    }
+    sm.part[tid] = ns;
+    sm.part[32 + tid] = ds;
+    sm.part[64 + tid] = best;
+    sm.part[96 + tid] = bval;
+    sm.part[128 + tid] = __int_as_float(bi);
+  }
+  cl.sync();
+  if (tid < kMaxM) {
+    float ns = 0.f, ds = 0.f, best = -1.f, bval = 0.f;
+    int bi = 0x7fffffff;
+    for (int r = 0; r < kCl; ++r) {
+      const float* rp = cl.map_shared_rank(sm.part, r);
+      ns += rp[tid];
+      ds += rp[32 + tid];
+      const float ob = rp[64 + tid];
+      const int oi = __float_as_int(rp[128 + tid]);
+      if (ob > best || (ob == best && oi < bi)) {
+        best = ob;
+        bval = rp[96 + tid];
         bi = oi;
       }
     }
     const bool live = tid < m;
     sm.th[tid] = live ? ns / fmaxf(ds, 1e-30f) : 0.f;
-    const float sgn = (live && Q[(int64_t)tid * Dg + bi] < 0.f) ? -1.f : 1.f;
+    const float sgn = (live && bval < 0.f) ? -1.f : 1.f;
     sm.inv[tid] = live ? sgn * rsqrtf(fmaxf(ds, 1e-30f)) : 0.f;
   }
-  __syncthreads();
+  cl.sync();
   // the coefficients of the final rows follow from those of the rows they were formed from:
   // row_j = inv_j sum_k Ws[k][j] q_k   =>   c'_j = inv_j sum_k Ws[k][j] c_k
-  for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
-    const int k = i >> 5, j = i & 31;
-    p.mtx[(int64_t)prob * kMaxM * kMaxM + i] = (k < m && j < m) ? Ws[k * kSP + j] * sm.inv[j] : 0.f;
+  if (rank == 0) {
+    for (int i = tid; i < kMaxM * kMaxM; i += kThreads) {
+      const int k = i >> 5, j = i & 31;
+      p.mtx[(int64_t)prob * kMaxM * kMaxM + i] = (k < m && j < m) ? Ws[k * kSP + j] * sm.inv[j] : 0.f;
+    }
   }
   // pass 2: residuals |G z_j - theta_j z_j|^2 of the unit-length rows, and the rows written out
-  for (int c0 = 0; c0 < Dg; c0 += kThreads) {
+  for (int c0 = c_lo; c0 < c_hi; c0 += kThreads) {
     const int c = c0 + tid;
-    const bool on = c < Dg;
+    const bool on = c < c_hi;
     for (int j = 0; j < m; ++j) {
       const float zj = on ? Q[(int64_t)j * Dg + c] : 0.f, gj = on ? Y[(int64_t)j * Dg + c] : 0.f;
       const float iv = sm.inv[j];
@@ -424,13 +533,15 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
       if (lane == 0) sm.pr[warp * kMaxM + j] += r1;
     }
   }
-  for (int64_t i = (int64_t)m * Dg + tid; i < (int64_t)p.r * Dg; i += kThreads) Q[i] = 0.f;
+  for (int q = m; q < p.r; ++q)
+    for (int c = c_lo + tid; c < c_hi; c += kThreads) Q[(int64_t)q * Dg + c] = 0.f;
   __syncthreads();
   if (tid < kMaxM) {
     float rs = 0.f;
     for (int w = 0; w < 8; ++w) rs += sm.pr[w * kMaxM + tid];
-    sm.rho2[tid] = (tid < m) ? rs : 0.f;
+    sm.part[tid] = (tid < m) ? rs : 0.f;
   }
+  cluster_sum(cl, sm.part, sm.rho2, kMaxM, tid);
   __syncthreads();
   float sumth = 0.f, rhoF2 = 0.f, rhomax2 = 0.f;
   for (int j = 0; j < m; ++j) {
@@ -447,8 +558,8 @@ __global__ void __launch_bounds__(kThreads) group_small_kernel(const __grid_cons
   // with outlier channels.  Rows are held to 5e-5 lambda_1, the block to 1/4096 of the gap.
   const bool accept = rhomax2 <= (5e-5f * th1) * (5e-5f * th1) && gap > 0.f && rhoF <= (1.f / 4096.f) * gap;
   if (reason == 0 && !accept) reason = (gap > 0.f) ? KVC_SOLVER_FULL_SLOW : KVC_SOLVER_FULL_NO_GAP;
-  for (int i = tid; i < Dg; i += kThreads) evals[i] = (i < m) ? sm.th[i] : (Dg > m ? tau / (float)(Dg - m) : 0.f);
-  if (tid == 0) {
+  for (int i = c_lo + tid; i < c_hi; i += kThreads) evals[i] = (i < m) ? sm.th[i] : (Dg > m ? tau / (float)(Dg - m) : 0.f);
+  if (tid == 0 && rank == 0) {
     *code = reason;
     // a block that is only slow (there is a gap) gets another application of G while rounds are left
     if (reason == KVC_SOLVER_FULL_SLOW && p.round < p.last_round)
@@ -519,7 +630,7 @@ cudaError_t launch_group_backproject(const GroupFitLaunch& G, const SegTable* se
 }
 
 cudaError_t launch_group_small(const GroupFitLaunch& G, int op, cudaStream_t s) {
-  const int blocks = G.L * 2;
+  const int blocks = G.L * 2 * kCl;               // a cluster of kCl blocks per (layer, K|V): the kernel carries __cluster_dims__
   if (blocks <= 0) return cudaSuccess;
   static DeviceOnce once;
   int once_dev;
