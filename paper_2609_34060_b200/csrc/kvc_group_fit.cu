@@ -570,27 +570,50 @@ __global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kThreads) group_sm
 }
 
 // coeff[l][t][:] <- coeff[l][t][:] . M  for every covered token: the coefficients of the final rows from those of
-// the rows the last Rayleigh-Ritz step started from.  One thread per token, M in shared memory.
+// the rows the last Rayleigh-Ritz step started from.  A block takes 256 consecutive tokens: their rows go through
+// shared memory (coalesced both ways, pitch 33), one thread per token multiplies its row by M (read as float4).
 __global__ void __launch_bounds__(kThreads) group_coeff_transform_kernel(const __grid_constant__ GroupFitLaunch p) {
-  __shared__ float M[kMaxM * kMaxM];
+  __shared__ __align__(16) float M[kMaxM * kMaxM];
+  __shared__ float rows[kThreads * 33];
   const int prob = blockIdx.y, l = prob >> 1, is_v = prob & 1;
-  for (int i = threadIdx.x; i < kMaxM * kMaxM; i += kThreads) M[i] = p.mtx[(int64_t)prob * kMaxM * kMaxM + i];
+  const int tid = threadIdx.x;
+  for (int i = tid; i < kMaxM * kMaxM; i += kThreads) M[i] = p.mtx[(int64_t)prob * kMaxM * kMaxM + i];
+  const int t0 = blockIdx.x * kThreads;
+  const int nt = min(kThreads, p.n_cov - t0);
+  if (nt <= 0) return;
+  float* base = (is_v ? p.coeff_v_rw : p.coeff_k_rw) + ((int64_t)l * p.n_cov + t0) * p.r;
+  const int r = p.r;
+  for (int i = tid; i < nt * r; i += kThreads) {
+    const int t = i / r, k = i - t * r;
+    rows[t * 33 + k] = base[i];
+  }
   __syncthreads();
-  const int t = blockIdx.x * kThreads + threadIdx.x;
-  if (t >= p.n_cov) return;
-  float* row = (is_v ? p.coeff_v_rw : p.coeff_k_rw) + ((int64_t)l * p.n_cov + t) * p.r;
-  float c[kMaxM], o[kMaxM];
+  if (tid < nt) {
+    float c[kMaxM], o[kMaxM];
 #pragma unroll
-  for (int k = 0; k < kMaxM; ++k) c[k] = (k < p.r) ? row[k] : 0.f;
+    for (int k = 0; k < kMaxM; ++k) c[k] = (k < r) ? rows[tid * 33 + k] : 0.f;
 #pragma unroll
-  for (int j = 0; j < kMaxM; ++j) o[j] = 0.f;
+    for (int j = 0; j < kMaxM; ++j) o[j] = 0.f;
 #pragma unroll
-  for (int k = 0; k < kMaxM; ++k)
+    for (int k = 0; k < kMaxM; ++k) {
 #pragma unroll
-    for (int j = 0; j < kMaxM; ++j) o[j] = fmaf(c[k], M[k * kMaxM + j], o[j]);
+      for (int j4 = 0; j4 < kMaxM / 4; ++j4) {
+        const float4 m4 = *reinterpret_cast<const float4*>(M + k * kMaxM + 4 * j4);
+        o[4 * j4] = fmaf(c[k], m4.x, o[4 * j4]);
+        o[4 * j4 + 1] = fmaf(c[k], m4.y, o[4 * j4 + 1]);
+        o[4 * j4 + 2] = fmaf(c[k], m4.z, o[4 * j4 + 2]);
+        o[4 * j4 + 3] = fmaf(c[k], m4.w, o[4 * j4 + 3]);
+      }
+    }
 #pragma unroll
-  for (int j = 0; j < kMaxM; ++j)
-    if (j < p.r) row[j] = o[j];
+    for (int j = 0; j < kMaxM; ++j)
+      if (j < r) rows[tid * 33 + j] = o[j];
+  }
+  __syncthreads();
+  for (int i = tid; i < nt * r; i += kThreads) {
+    const int t = i / r, k = i - t * r;
+    base[i] = rows[t * 33 + k];
+  }
 }
 
 // ptr[0 .. n) <- 0 unless a run flag is given and zero (the start of a projection pass that adds into its output)
