@@ -428,7 +428,10 @@ def main():
         c0 = W["true"][0]
         f_bytes = c0.L * c0.H * c0.T * (4 * c0.d + sum(8 * st.r + 4 * c0.d for st in W["states"]))
         fused = {"chain_ms": f_ms, "algorithmic_bytes": f_bytes, "GBs": f_bytes / (f_ms * 1e-3) / 1e9,
-                 "us_per_agent_layer": f_ms * 1e3 / (cfg.n_agents - 1) / cfg.L}
+                 "us_per_agent_layer": f_ms * 1e3 / (cfg.n_agents - 1) / cfg.L,
+                 # the same step with the chain run fused: fewer algorithmic bytes in less time (a short side
+                 # measurement at whatever clock it met, not the sustained figure of the headline)
+                 "step_ms_with_fused_chain": (upd_ms + f_ms) if args.only == "all" else None}
         del cws
     if rank != 0:
         if world > 1:
