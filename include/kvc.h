@@ -300,10 +300,13 @@ size_t kvc_chain_update_edge_stride(const kvc_cache *tgt, const kvc_state *st, i
  * The lists are host arrays on purpose: the cos / sin tables of every segment are formed in float64 on the
  * host, exactly like the single shift's, and travel in the launch parameters (a device position array would
  * need sincos per token and frequency inside the kernels).  kvc_apply_segmented runs on the tensor-core
- * kernel where kvc_apply does (every row picks its segment's table in the epilogue); the passes of
- * kvc_state_update_segmented over the caches are served by the CUDA-core kernel family (KVC_PATH_TC forced:
- * KVC_E_UNSUPPORTED).  Everything else is as in kvc_apply / kvc_state_update, including layer-grouped states
- * and the FIT modes.
+ * kernel where kvc_apply does (every row picks its segment's table in the epilogue), and so do the passes
+ * of kvc_state_update_segmented over the caches where kvc_state_update's do: the Gram pass picks every
+ * row's table while it forms the deviation, the projection runs as one launch per segment over that
+ * segment's token window (it rotates the basis, not the tokens).  A paged cache whose segment boundaries
+ * do not fall on page boundaries has its projection served by the CUDA-core kernel (KVC_PATH_TC forced:
+ * KVC_E_UNSUPPORTED), as has the fit of a layer-grouped state.  Everything else is as in kvc_apply /
+ * kvc_state_update, including layer-grouped states and the FIT modes.
  */
 #define KVC_MAX_SEGMENTS   16
 #define KVC_COORDS_TARGET  0

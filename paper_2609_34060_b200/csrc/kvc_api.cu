@@ -429,15 +429,14 @@ static int fit_gram(const UpdatePlan& P, void* workspace, uint32_t* status, FitL
   F.H = P.H;
   F.status = status;
   rope_tables(P.rope, P.d, P.shift, F.cs, F.sn);
-  if (tl_path_force != KVC_PATH_GENERIC && !P.seg) {
-    const int trc = tc_gram(F, P.d, s);
+  if (tl_path_force != KVC_PATH_GENERIC) {
+    const int trc = tc_gram(F, P.d, s, P.seg);            // per-row tables when the context has segments
     if (trc == KVC_OK) {
       F.n_parts = 2;
       return KVC_OK;
     }
     if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
   }
-  if (P.seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
   return launch_gram_generic(F, P.seg, P.d, s) == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
@@ -490,7 +489,6 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, c
       return KVC_E_CUDA;
     }
   }
-  if (P.seg && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
   if (tl_path_force != KVC_PATH_GENERIC && !P.seg) {
     const int trc = tc_project(U, d, s);
     if (trc == KVC_OK) {
@@ -498,6 +496,50 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, c
       return KVC_OK;
     }
     if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  }
+  if (tl_path_force != KVC_PATH_GENERIC && P.seg) {
+    // A context of several segments: the projection is independent token by token, so every segment is a
+    // launch of its own over its token window, with its own shift (the basis is rotated, not the tokens).
+    // Windows of a paged cache must start on a page boundary; otherwise the CUDA-core kernel serves the call.
+    const SegTable& sg = *P.seg;
+    bool windows_ok = true;
+    for (int j = 1; j < sg.n; ++j)
+      for (const DevCache* c : {&U.src, &U.tgt})
+        if (c->k && c->page_table && (sg.t_begin[j] & c->page_mask)) windows_ok = false;
+    int trc = windows_ok ? KVC_OK : KVC_E_UNSUPPORTED;
+    bool launched = false;
+    for (int j = 0; j < sg.n && trc == KVC_OK; ++j) {
+      const int tb = sg.t_begin[j];
+      const int nxt = j + 1 < sg.n ? sg.t_begin[j + 1] : st->n_cov;
+      const int te = nxt < st->n_cov ? nxt : st->n_cov;      // the segment's covered rows
+      if (te <= tb) continue;
+      UpdateLaunch W = U;
+      for (DevCache* c : {&W.src, &W.tgt}) {
+        if (!c->k) continue;
+        if (c->page_table) {
+          c->page_table += tb >> c->page_shift;
+        } else {
+          c->k += (int64_t)tb * c->s_tok;
+          c->v += (int64_t)tb * c->s_tok;
+        }
+        c->T -= tb;
+      }
+      W.coeff_k += (int64_t)tb * st->r;
+      W.coeff_v += (int64_t)tb * st->r;
+      W.coeff_rows = st->n_cov;
+      W.n_cov = te - tb;
+      W.shift = sg.shifted[j];
+      W.coords = sg.coords;
+      memcpy(W.cs, sg.cs[j], sizeof(W.cs));
+      memcpy(W.sn, sg.sn[j], sizeof(W.sn));
+      trc = tc_project(W, d, s);
+      launched = launched || trc == KVC_OK;
+    }
+    if (trc == KVC_OK) {
+      tl_last_path = KVC_PATH_TC;
+      return KVC_OK;
+    }
+    if (trc != KVC_E_UNSUPPORTED || launched || tl_path_force == KVC_PATH_TC) return trc;
   }
   U.tiles_per_slab = (st->n_cov + kGenericProjectTile - 1) / kGenericProjectTile;
   const int64_t tiles = (int64_t)P.L * P.H * 2 * U.tiles_per_slab;

@@ -85,9 +85,11 @@ struct UpdateLaunch {
   int32_t r, n_cov, basis_bf16, pairing;
   int32_t shift, L, H, tiles_per_slab;
   uint32_t* status;
-  int32_t grouped, pad;        // grouped: one state per layer; the heads' projections are ADDED into coeff [L,n_cov,r]
+  int32_t grouped, coords;     // grouped: one state per layer; the heads' projections are ADDED into coeff [L,n_cov,r]
+                               // coords (tensor-core kernel): 0 = Delta = tgt - Rot_s(src), 1 = Rot_-s(tgt) - src
   const int32_t* run_if;       // DEVICE flag or nullptr: when given and zero, the kernel returns at once (a pass
                                // of the grouped fit's refinement rounds that turned out not to be needed)
+  int32_t coeff_rows, pad2;    // rows between two coefficient slabs (0: n_cov); larger when the launch is a token window
   alignas(16) float cs[kMaxHalfD];
   alignas(16) float sn[kMaxHalfD];
 };

@@ -294,7 +294,9 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
     const int tt = tid - 128;                      // 0..511
     const uint32_t sw = (uint32_t)(m & 7);
 
-    // B and Bs = -Rot_{-shift}(B) of one slab as swizzled K-major bf16 hi/lo operands
+    // The operands of one slab as swizzled K-major bf16 hi/lo blocks: B for the target tile and
+    // Bs = -Rot_{-shift}(B) for the source tile (Delta = tgt - Rot_s(src): coeff = tgt.B^T + src.Bs^T); with the
+    // deviation taken at the source's positions (Delta = Rot_{-s}(tgt) - src) Rot_s(B) for the target and -B for the source.
     auto stage_basis = [&](const PTile& t) {
       const void* basis = t.is_v ? u.basis_v : u.basis_k;
       const bool rotate = u.shift != 0 && !t.is_v;
@@ -335,6 +337,33 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
             const float c = u.cs[4 * jj + k], sn = u.sn[4 * jj + k];
             sneg[2 * k] = -(v[2 * k] * c + v[2 * k + 1] * sn);
             sneg[2 * k + 1] = -(v[2 * k + 1] * c - v[2 * k] * sn);
+          }
+        }
+        if (u.coords == 1) {
+          // target operand Rot_{+shift}(b), source operand -b
+          float rot[8];
+          if (!rotate) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) rot[k] = v[k];
+          } else if (u.pairing == 0) {
+            const int f0 = 8 * (jj & 7);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const float c = u.cs[f0 + k], sn = u.sn[f0 + k];
+              rot[k] = (jj < 8) ? (v[k] * c - w[k] * sn) : (v[k] * c + w[k] * sn);
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float c = u.cs[4 * jj + k], sn = u.sn[4 * jj + k];
+              rot[2 * k] = v[2 * k] * c - v[2 * k + 1] * sn;
+              rot[2 * k + 1] = v[2 * k + 1] * c + v[2 * k] * sn;
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            sneg[k] = -v[k];
+            v[k] = rot[k];
           }
         }
         uint4 bh, bl, sh, sl;
@@ -484,8 +513,10 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr) {
   return d;
 }
 
-template <int NS>
-__global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcLaunch p) {
+// SEG: per-row shifts and tables from a segment table (Eq. 1), and the choice of coordinates (App. A.2):
+// Delta = tgt - Rot_s(src) at the target's positions, Rot_{-s}(tgt) - src at the source's.
+template <int NS, bool SEG>
+__device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTable* segp) {
   // kind::f16, bf16 x bf16 -> f32, both operands MN-major, M = 128, N = 128
   constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
   extern __shared__ uint8_t smem_raw[];
@@ -654,7 +685,17 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
         uint8_t* sr = tg + kTileBytes;
         const int tok = (g.tile0 + k) * kTileTok + m;
         const bool live = tok < f.n_cov;
-        const bool rotate = rot_any && !g.is_v;
+        bool rotate = rot_any && !g.is_v;
+        const float* csp = f.cs;
+        const float* snp = f.sn;
+        bool at_source = false;
+        if constexpr (SEG) {                        // this row's segment
+          const int sk = seg_index(*segp, tok);
+          csp = segp->cs[sk];
+          snp = segp->sn[sk];
+          rotate = !g.is_v && segp->shifted[sk] != 0;
+          at_source = segp->coords == 1;
+        }
         if (p.has_src || !live) {
           if (f.pairing == 0) {
 #pragma unroll
@@ -677,17 +718,36 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
                   xa[z] = f2_from_bf16x2(sw0[z]);
                   xb[z] = f2_from_bf16x2(sw1[z]);
                 }
+                f32x2 ya[4], yb[4];
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  ya[z] = f2_from_bf16x2(tw0[z]);
+                  yb[z] = f2_from_bf16x2(tw1[z]);
+                }
                 if (rotate) {
-                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(f.cs + 8 * j + 4);
-                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(f.sn + 8 * j + 4);
+                  const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
+                  float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
+                  if (SEG && at_source) {                    // the target goes back by the shift: the same rotation with the sines negated
+                    s0 = make_float4(-s0.x, -s0.y, -s0.z, -s0.w);
+                    s1 = make_float4(-s1.x, -s1.y, -s1.z, -s1.w);
+                  }
                   const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
                   const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
                   const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
+                  if (SEG && at_source) {
 #pragma unroll
-                  for (int z = 0; z < 4; ++z) {
-                    const f32x2 a = xa[z], b = xb[z];
-                    xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));       // a cos - b sin
-                    xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));        // a sin + b cos
+                    for (int z = 0; z < 4; ++z) {
+                      const f32x2 a = ya[z], b = yb[z];
+                      ya[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));
+                      yb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));
+                    }
+                  } else {
+#pragma unroll
+                    for (int z = 0; z < 4; ++z) {
+                      const f32x2 a = xa[z], b = xb[z];
+                      xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));     // a cos - b sin
+                      xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));      // a sin + b cos
+                    }
                   }
                 }
                 uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
@@ -698,7 +758,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
                 for (int z = 0; z < 4; ++z) {
                   // H = bf16(Delta); 2 L = bf16(Delta - H) with one added to both exponents (the doubling is
                   // exact; a zero remainder becomes 2^-126, which no sum notices)
-                  const f32x2 da = f2_sub(f2_from_bf16x2(tw0[z]), xa[z]), db = f2_sub(f2_from_bf16x2(tw1[z]), xb[z]);
+                  const f32x2 da = f2_sub(ya[z], xa[z]), db = f2_sub(yb[z], xb[z]);
                   hp0[z] = f2_to_bf16x2(da);
                   hp1[z] = f2_to_bf16x2(db);
                   lp0[z] = f2_to_bf16x2(f2_sub(da, f2_from_bf16x2(hp0[z]))) + 0x00800080u;
@@ -727,15 +787,17 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
                 unpack8(*tp, y);
                 if (rotate) {
                   const int f0 = 16 * cq + 4 * jj;
-                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + f0);
-                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + f0);
+                  const float4 c0 = *reinterpret_cast<const float4*>(csp + f0);
+                  const float4 s0 = *reinterpret_cast<const float4*>(snp + f0);
                   const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
-                  const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
+                  const float sgn = (SEG && at_source) ? -1.f : 1.f;
+                  const float sn[4] = {sgn * s0.x, sgn * s0.y, sgn * s0.z, sgn * s0.w};
+                  float* rv = (SEG && at_source) ? y : x;     // source coordinates: the target goes back by the shift
 #pragma unroll
                   for (int z = 0; z < 4; ++z) {
-                    const float a = x[2 * z], b = x[2 * z + 1];
-                    x[2 * z] = a * cs[z] - b * sn[z];
-                    x[2 * z + 1] = a * sn[z] + b * cs[z];
+                    const float a = rv[2 * z], b = rv[2 * z + 1];
+                    rv[2 * z] = a * cs[z] - b * sn[z];
+                    rv[2 * z + 1] = a * sn[z] + b * cs[z];
                   }
                 }
                 uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
@@ -770,6 +832,16 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
     tc_fence_after();
     tmem_dealloc(tmem_base, 256);
   }
+}
+
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcLaunch p) {
+  gram_tc_body<NS, false>(p, nullptr);
+}
+// the segment table travels as a launch parameter of its own, so the plain launch does not carry it
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1) gram_tc_seg_kernel(const __grid_constant__ GramTcLaunch p, const __grid_constant__ SegTable seg) {
+  gram_tc_body<NS, true>(p, &seg);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1200,8 +1272,8 @@ int tc_project(const UpdateLaunch& U, int d, cudaStream_t s) {
   if (L.has_src)
     ok = ok && tc::encode_cache(&L.maps.src_k, U.src, U.src.k, U.L, U.H) && tc::encode_cache(&L.maps.src_v, U.src, U.src.v, U.L, U.H);
   const int cslabs = U.grouped ? U.L : U.L * U.H;
-  ok = ok && tc::encode_coeff(&L.maps.coeff_k, U.coeff_k, U.r, U.n_cov, cslabs) &&
-       tc::encode_coeff(&L.maps.coeff_v, U.coeff_v, U.r, U.n_cov, cslabs);
+  ok = ok && tc::encode_coeff(&L.maps.coeff_k, U.coeff_k, U.r, U.n_cov, cslabs, U.coeff_rows) &&
+       tc::encode_coeff(&L.maps.coeff_v, U.coeff_v, U.r, U.n_cov, cslabs, U.coeff_rows);
   if (!ok) return KVC_E_CUDA;
   const int sms = tc::sm_count();
   if (sms <= 0) return KVC_E_CUDA;
@@ -1214,7 +1286,7 @@ static_assert(offsetof(FitLaunch, cs) % 16 == 0 && offsetof(FitLaunch, sn) % 16 
 static_assert(offsetof(tcu::GramTcLaunch, maps) % 64 == 0, "tensor maps need 64-byte alignment");
 
 // Writes two partial Gram matrices per (layer, head, K|V): part p at F.gram + p * (L*H*2) * d * d.
-int tc_gram(const FitLaunch& F, int d, cudaStream_t s) {
+int tc_gram(const FitLaunch& F, int d, cudaStream_t s, const SegTable* seg) {
   using namespace tcu;
   if (d != 128 || F.n_cov <= 0) return KVC_E_UNSUPPORTED;
   if (!cache_ok(F.tgt) || (F.src.k && !cache_ok(F.src)) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
@@ -1240,7 +1312,16 @@ int tc_gram(const FitLaunch& F, int d, cudaStream_t s) {
     if (cudaFuncSetAttribute(gram_tc_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
     once.mark(once_dev);
   }
-  gram_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
+  if (seg) {
+    static DeviceOnce once_seg;
+    if (once_seg.pending(&once_dev)) {
+      if (cudaFuncSetAttribute(gram_tc_seg_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+      once_seg.mark(once_dev);
+    }
+    gram_tc_seg_kernel<NS><<<grid, kThreads, smem, s>>>(L, *seg);
+  } else {
+    gram_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
+  }
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

@@ -64,12 +64,15 @@ def test_apply_segmented(cfg, coords, path):
 
 
 @pytest.mark.parametrize("coords", COORDS, ids=["target", "source"])
-@pytest.mark.parametrize("cfg", [CFG_C, CFG_P], ids=lambda c: c.name)
-def test_project_and_fit_segmented(cfg, coords):
+@pytest.mark.parametrize("cfg,on_pages", [(CFG_C, False), (CFG_P, False), (CFG_P, True)],
+                         ids=["8b_small", "vlm_small", "vlm_small-page-aligned"])
+def test_project_and_fit_segmented(cfg, on_pages, coords):
     """PROJECT: coefficients of the per-token-shift deviation in a given basis.  FIT: the deviation is built
     exactly rank r in the chosen coordinates, so the fitted state reproduces the oracle's subspace and the
     update -> apply round trip gives back the target."""
     t_begin, shift = SEGS[cfg.name]
+    if on_pages:                                   # boundaries on the 16-token page grid: tensor-core windows on a paged source
+        t_begin = [0, 32, 528]
     s_tok = orc.segment_shifts(cfg.T, t_begin, shift)
     f = hp.inv_freq(cfg)
     segs = kvc.Segments(t_begin, shift, coords)
@@ -97,7 +100,9 @@ def test_project_and_fit_segmented(cfg, coords):
                    given.basis_k.to(DEV), given.basis_v.to(DEV))
     kvc.kvc_state_update_segmented(src, tgt, segs, rope, st, kvc.KVC_PROJECT)
     torch.cuda.synchronize()
-    assert kvc.kvc_last_path() == kvc.KVC_PATH_GENERIC
+    # contiguous caches: a tensor-core launch per segment window; the paged case has boundaries off the page grid
+    # and is served by the CUDA-core kernel
+    assert kvc.kvc_last_path() == (kvc.KVC_PATH_GENERIC if (cfg.paged and not on_pages) else kvc.KVC_PATH_TC)
     deltas = {}
     for which, cf, bs in (("k", st.coeff_k, given.basis_k), ("v", st.coeff_v, given.basis_v)):
         for l in range(L):
