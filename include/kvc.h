@@ -305,8 +305,8 @@ size_t kvc_chain_update_edge_stride(const kvc_cache *tgt, const kvc_state *st, i
  * row's table while it forms the deviation, the projection runs as one launch per segment over that
  * segment's token window (it rotates the basis, not the tokens).  A paged cache whose segment boundaries
  * do not fall on page boundaries has its projection served by the CUDA-core kernel (KVC_PATH_TC forced:
- * KVC_E_UNSUPPORTED), as has the fit of a layer-grouped state.  Everything else is as in kvc_apply /
- * kvc_state_update, including layer-grouped states and the FIT modes.
+ * KVC_E_UNSUPPORTED).  Everything else is as in kvc_apply / kvc_state_update, including layer-grouped
+ * states (whose back-projection pass picks the rows' tables like the Gram pass) and the FIT modes.
  */
 #define KVC_MAX_SEGMENTS   16
 #define KVC_COORDS_TARGET  0

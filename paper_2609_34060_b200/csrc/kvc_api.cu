@@ -579,7 +579,7 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
   G.H = P.H;
   G.d = P.d;
   // the back-projection runs on the tensor cores where they take the geometry (two partial sums), else on CUDA cores
-  const bool use_tc = tl_path_force != KVC_PATH_GENERIC && !P.seg && P.d == 128 && (st->r & 3) == 0 &&
+  const bool use_tc = tl_path_force != KVC_PATH_GENERIC && P.d == 128 && (st->r & 3) == 0 &&
                       !(P.dt.page_table && P.dt.page_mask + 1 > 128) && !(P.ds.page_table && P.ds.page_mask + 1 > 128);
   if (!use_tc && tl_path_force == KVC_PATH_TC) return KVC_E_UNSUPPORTED;
   G.parts = use_tc ? 2 : kGroupFitParts;
@@ -596,7 +596,7 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
     int rc = project_edge(P, status, s);
     if (rc != KVC_OK) return rc;
     if (use_tc) {
-      if ((rc = tc_backproject(G, s)) != KVC_OK) return rc;
+      if ((rc = tc_backproject(G, s, P.seg)) != KVC_OK) return rc;
     } else if (launch_group_backproject(G, P.seg, s) != cudaSuccess) {
       return KVC_E_CUDA;
     }
@@ -613,7 +613,7 @@ static int group_fit_edge(const UpdatePlan& P, const kvc_cache* tgt, void* works
     int rc = project_edge(P, status, s, G.need_more + round);
     if (rc != KVC_OK) return rc;
     if (use_tc) {
-      if ((rc = tc_backproject(G, s)) != KVC_OK) return rc;
+      if ((rc = tc_backproject(G, s, P.seg)) != KVC_OK) return rc;
     } else if (launch_group_backproject(G, P.seg, s) != cudaSuccess) {
       return KVC_E_CUDA;
     }

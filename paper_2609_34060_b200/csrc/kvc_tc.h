@@ -26,6 +26,6 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
                    uint32_t* status, void* workspace, size_t ws_bytes, cudaStream_t s);
 int tc_project(const UpdateLaunch& U, int d, cudaStream_t s);
 int tc_gram(const FitLaunch& F, int d, cudaStream_t s, const SegTable* seg = nullptr);
-int tc_backproject(const GroupFitLaunch& G, cudaStream_t s);
+int tc_backproject(const GroupFitLaunch& G, cudaStream_t s, const SegTable* seg = nullptr);
 
 }  // namespace kvc

@@ -885,8 +885,9 @@ __device__ __forceinline__ void split2(float x0, float x1, uint32_t& hi, uint32_
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-template <int NS>
-__global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __grid_constant__ BackprojTcLaunch p) {
+// SEG: per-row shifts and tables from a segment table and the choice of coordinates, as in the Gram kernel.
+template <int NS, bool SEG>
+__device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, const SegTable* segp) {
   if (p.run_if != nullptr && *p.run_if == 0) return;      // uniform over the grid: nothing has been set up yet
   // kind::f16, bf16 x bf16 -> f32, both operands MN-major, M = 128 (channels), N = 64 ([Z hi | Z lo])
   constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
@@ -1091,7 +1092,17 @@ __global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __gri
         uint8_t* sr = tg + kTileBytes;
         const int tok = (g.tile0 + k) * kTileTok + m;
         const bool live = tok < f.n_cov;
-        const bool rotate = rot_any && !g.is_v;
+        bool rotate = rot_any && !g.is_v;
+        const float* csp = f.cs;
+        const float* snp = f.sn;
+        bool at_source = false;
+        if constexpr (SEG) {                        // this row's segment
+          const int sk = seg_index(*segp, tok);
+          csp = segp->cs[sk];
+          snp = segp->sn[sk];
+          rotate = !g.is_v && segp->shifted[sk] != 0;
+          at_source = segp->coords == 1;
+        }
         if (p.has_src || !live) {
           if (f.pairing == 0) {
 #pragma unroll
@@ -1114,17 +1125,36 @@ __global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __gri
                   xa[z] = f2_from_bf16x2(sw0[z]);
                   xb[z] = f2_from_bf16x2(sw1[z]);
                 }
+                f32x2 ya[4], yb[4];
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                  ya[z] = f2_from_bf16x2(tw0[z]);
+                  yb[z] = f2_from_bf16x2(tw1[z]);
+                }
                 if (rotate) {
-                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + 8 * j), c1 = *reinterpret_cast<const float4*>(f.cs + 8 * j + 4);
-                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + 8 * j), s1 = *reinterpret_cast<const float4*>(f.sn + 8 * j + 4);
+                  const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
+                  float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
+                  if (SEG && at_source) {                    // the target goes back by the shift: the same rotation with the sines negated
+                    s0 = make_float4(-s0.x, -s0.y, -s0.z, -s0.w);
+                    s1 = make_float4(-s1.x, -s1.y, -s1.z, -s1.w);
+                  }
                   const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
                   const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
                   const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
+                  if (SEG && at_source) {
 #pragma unroll
-                  for (int z = 0; z < 4; ++z) {
-                    const f32x2 a = xa[z], b = xb[z];
-                    xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));       // a cos - b sin
-                    xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));        // a sin + b cos
+                    for (int z = 0; z < 4; ++z) {
+                      const f32x2 a = ya[z], b = yb[z];
+                      ya[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));
+                      yb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));
+                    }
+                  } else {
+#pragma unroll
+                    for (int z = 0; z < 4; ++z) {
+                      const f32x2 a = xa[z], b = xb[z];
+                      xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));     // a cos - b sin
+                      xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));      // a sin + b cos
+                    }
                   }
                 }
                 uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
@@ -1135,7 +1165,7 @@ __global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __gri
                 for (int z = 0; z < 4; ++z) {
                   // H = bf16(Delta); 2 L = bf16(Delta - H) with one added to both exponents (the doubling is
                   // exact; a zero remainder becomes 2^-126, which no sum notices)
-                  const f32x2 da = f2_sub(f2_from_bf16x2(tw0[z]), xa[z]), db = f2_sub(f2_from_bf16x2(tw1[z]), xb[z]);
+                  const f32x2 da = f2_sub(ya[z], xa[z]), db = f2_sub(yb[z], xb[z]);
                   sq2 = f2_fma(da, da, f2_fma(db, db, sq2));
                   hp0[z] = f2_to_bf16x2(da);
                   hp1[z] = f2_to_bf16x2(db);
@@ -1165,15 +1195,17 @@ __global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __gri
                 unpack8(*tp, y);
                 if (rotate) {
                   const int f0 = 16 * cq + 4 * jj;
-                  const float4 c0 = *reinterpret_cast<const float4*>(f.cs + f0);
-                  const float4 s0 = *reinterpret_cast<const float4*>(f.sn + f0);
+                  const float4 c0 = *reinterpret_cast<const float4*>(csp + f0);
+                  const float4 s0 = *reinterpret_cast<const float4*>(snp + f0);
                   const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
-                  const float sn[4] = {s0.x, s0.y, s0.z, s0.w};
+                  const float sgn = (SEG && at_source) ? -1.f : 1.f;
+                  const float sn[4] = {sgn * s0.x, sgn * s0.y, sgn * s0.z, sgn * s0.w};
+                  float* rv = (SEG && at_source) ? y : x;     // source coordinates: the target goes back by the shift
 #pragma unroll
                   for (int z = 0; z < 4; ++z) {
-                    const float a = x[2 * z], b = x[2 * z + 1];
-                    x[2 * z] = a * cs[z] - b * sn[z];
-                    x[2 * z + 1] = a * sn[z] + b * cs[z];
+                    const float a = rv[2 * z], b = rv[2 * z + 1];
+                    rv[2 * z] = a * cs[z] - b * sn[z];
+                    rv[2 * z + 1] = a * sn[z] + b * cs[z];
                   }
                 }
                 uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
@@ -1246,6 +1278,16 @@ __global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __gri
     tc_fence_after();
     tmem_dealloc(tmem_base, 256);
   }
+}
+
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1) backproject_tc_kernel(const __grid_constant__ BackprojTcLaunch p) {
+  backproject_tc_body<NS, false>(p, nullptr);
+}
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1) backproject_tc_seg_kernel(const __grid_constant__ BackprojTcLaunch p,
+                                                                        const __grid_constant__ SegTable seg) {
+  backproject_tc_body<NS, true>(p, &seg);
 }
 
 static bool cache_ok(const DevCache& c) {
@@ -1327,7 +1369,7 @@ int tc_gram(const FitLaunch& F, int d, cudaStream_t s, const SegTable* seg) {
 
 // The back-projection pass of the layer-grouped fit on the tensor cores (two partial sums: G.parts must be 2,
 // the trace comes in 32 partial sums).  KVC_E_UNSUPPORTED for what it does not take.
-int tc_backproject(const GroupFitLaunch& G, cudaStream_t s) {
+int tc_backproject(const GroupFitLaunch& G, cudaStream_t s, const SegTable* seg) {
   using namespace tcu;
   if (G.d != 128 || G.r <= 0 || G.r > 32 || (G.r & 3) || G.n_cov <= 0 || G.parts != 2) return KVC_E_UNSUPPORTED;
   if (!cache_ok(G.tgt) || (G.src.k && !cache_ok(G.src)) || !tc::encode_fn()) return KVC_E_UNSUPPORTED;
@@ -1368,6 +1410,15 @@ int tc_backproject(const GroupFitLaunch& G, cudaStream_t s) {
   if (once.pending(&once_dev)) {
     if (cudaFuncSetAttribute(backproject_tc_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
     once.mark(once_dev);
+  }
+  if (seg) {
+    static DeviceOnce once_seg;
+    if (once_seg.pending(&once_dev)) {
+      if (cudaFuncSetAttribute(backproject_tc_seg_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+      once_seg.mark(once_dev);
+    }
+    backproject_tc_seg_kernel<NS><<<grid, kThreads, smem, s>>>(L, *seg);
+    return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
   }
   backproject_tc_kernel<NS><<<grid, kThreads, smem, s>>>(L);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
