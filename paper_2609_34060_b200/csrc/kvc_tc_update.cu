@@ -460,6 +460,100 @@ static cudaError_t launch_project_t(const ProjectTcLaunch& L, int grid, cudaStre
 }
 
 // ---------------------------------------------------------------------------------------------
+// The deviation of one token row, 16 channels at a time, as the tensor-core operands of the Gram and
+// back-projection passes: H = bf16(Delta) and 2 L = bf16(Delta - H) with one added to both exponents (the
+// doubling is exact; a zero remainder becomes 2^-126, which no sum notices).  Delta = tgt - Rot_s(src), or
+// Rot_{-s}(tgt) - src when the correction lives at the source's positions (at_source).  One home for both
+// kernels; SQ adds the squares of Delta (the back-projection's trace).
+// ---------------------------------------------------------------------------------------------
+// Half-split pairing: chunk j of the two 64-channel halves (pairs (c, c + 64)).  csp / snp: this row's tables.
+template <bool SQ>
+__device__ __forceinline__ void delta_operands_half(const uint4& ta, const uint4& tb, const uint4& sa, const uint4& sb, const float* csp,
+                                                    const float* snp, int j, bool rotate, bool at_source, uint4& h0, uint4& h1,
+                                                    uint4& l0, uint4& l1, f32x2& sq2) {
+  // packed float32 pairs throughout: word w of a 16-byte chunk holds channels 2w, 2w + 1
+  const uint32_t sw0[4] = {sa.x, sa.y, sa.z, sa.w}, sw1[4] = {sb.x, sb.y, sb.z, sb.w};
+  const uint32_t tw0[4] = {ta.x, ta.y, ta.z, ta.w}, tw1[4] = {tb.x, tb.y, tb.z, tb.w};
+  f32x2 xa[4], xb[4], ya[4], yb[4];
+#pragma unroll
+  for (int z = 0; z < 4; ++z) {
+    xa[z] = f2_from_bf16x2(sw0[z]);
+    xb[z] = f2_from_bf16x2(sw1[z]);
+    ya[z] = f2_from_bf16x2(tw0[z]);
+    yb[z] = f2_from_bf16x2(tw1[z]);
+  }
+  if (rotate) {
+    const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
+    float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
+    if (at_source) {                                // the target goes back by the shift: the same rotation with the sines negated
+      s0 = make_float4(-s0.x, -s0.y, -s0.z, -s0.w);
+      s1 = make_float4(-s1.x, -s1.y, -s1.z, -s1.w);
+    }
+    const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
+    const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
+    const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
+    if (at_source) {
+#pragma unroll
+      for (int z = 0; z < 4; ++z) {
+        const f32x2 a = ya[z], b = yb[z];
+        ya[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));
+        yb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));
+      }
+    } else {
+#pragma unroll
+      for (int z = 0; z < 4; ++z) {
+        const f32x2 a = xa[z], b = xb[z];
+        xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));   // a cos - b sin
+        xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));    // a sin + b cos
+      }
+    }
+  }
+  uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
+  uint32_t* hp1 = reinterpret_cast<uint32_t*>(&h1);
+  uint32_t* lp0 = reinterpret_cast<uint32_t*>(&l0);
+  uint32_t* lp1 = reinterpret_cast<uint32_t*>(&l1);
+#pragma unroll
+  for (int z = 0; z < 4; ++z) {
+    const f32x2 da = f2_sub(ya[z], xa[z]), db = f2_sub(yb[z], xb[z]);
+    if (SQ) sq2 = f2_fma(da, da, f2_fma(db, db, sq2));
+    hp0[z] = f2_to_bf16x2(da);
+    hp1[z] = f2_to_bf16x2(db);
+    lp0[z] = f2_to_bf16x2(f2_sub(da, f2_from_bf16x2(hp0[z]))) + 0x00800080u;
+    lp1[z] = f2_to_bf16x2(f2_sub(db, f2_from_bf16x2(hp1[z]))) + 0x00800080u;
+  }
+}
+// Interleaved pairing: one chunk of 8 consecutive channels (pairs (2k, 2k + 1)); f0 = index of its first pair.
+template <bool SQ>
+__device__ __forceinline__ void delta_operands_interleaved(const uint4& t, const uint4& sr, const float* csp, const float* snp, int f0,
+                                                           bool rotate, bool at_source, uint4& h, uint4& l, float& sq) {
+  float x[8], y[8];
+  unpack8(sr, x);
+  unpack8(t, y);
+  if (rotate) {
+    const float4 c0 = *reinterpret_cast<const float4*>(csp + f0);
+    const float4 s0 = *reinterpret_cast<const float4*>(snp + f0);
+    const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
+    const float sgn = at_source ? -1.f : 1.f;
+    const float sn[4] = {sgn * s0.x, sgn * s0.y, sgn * s0.z, sgn * s0.w};
+    float* rv = at_source ? y : x;                  // source coordinates: the target goes back by the shift
+#pragma unroll
+    for (int z = 0; z < 4; ++z) {
+      const float a = rv[2 * z], b = rv[2 * z + 1];
+      rv[2 * z] = a * cs[z] - b * sn[z];
+      rv[2 * z + 1] = a * sn[z] + b * cs[z];
+    }
+  }
+  uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
+  uint32_t* lp = reinterpret_cast<uint32_t*>(&l);
+#pragma unroll
+  for (int z = 0; z < 4; ++z) {
+    const float e0 = y[2 * z] - x[2 * z], e1 = y[2 * z + 1] - x[2 * z + 1];
+    if (SQ) sq = fmaf(e0, e0, fmaf(e1, e1, sq));
+    split2x(e0, e1, hp[z], lp[z]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Gram:  G = Delta^T Delta  per (layer, head, K|V)   (Eq. 7: the d x d matrix whose top-r eigenvectors
 // are the basis).  Delta has to be explicit here (its Gram is quadratically small against the
 // inputs'), so the team forms Delta = tgt - Rot(src) in fp32, and writes H = bf16(Delta) over the
@@ -708,62 +802,8 @@ __device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTab
               uint4* s1p = reinterpret_cast<uint4*>(sr + kHalfBytes + o);
               uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
               if (live) {
-                // packed float32 pairs throughout: word w of a 16-byte chunk holds channels 2w, 2w + 1
-                const uint4 sa = *s0p, sb = *s1p, ta = *t0p, tb = *t1p;
-                const uint32_t sw0[4] = {sa.x, sa.y, sa.z, sa.w}, sw1[4] = {sb.x, sb.y, sb.z, sb.w};
-                const uint32_t tw0[4] = {ta.x, ta.y, ta.z, ta.w}, tw1[4] = {tb.x, tb.y, tb.z, tb.w};
-                f32x2 xa[4], xb[4];
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  xa[z] = f2_from_bf16x2(sw0[z]);
-                  xb[z] = f2_from_bf16x2(sw1[z]);
-                }
-                f32x2 ya[4], yb[4];
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  ya[z] = f2_from_bf16x2(tw0[z]);
-                  yb[z] = f2_from_bf16x2(tw1[z]);
-                }
-                if (rotate) {
-                  const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
-                  float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
-                  if (SEG && at_source) {                    // the target goes back by the shift: the same rotation with the sines negated
-                    s0 = make_float4(-s0.x, -s0.y, -s0.z, -s0.w);
-                    s1 = make_float4(-s1.x, -s1.y, -s1.z, -s1.w);
-                  }
-                  const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
-                  const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
-                  const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
-                  if (SEG && at_source) {
-#pragma unroll
-                    for (int z = 0; z < 4; ++z) {
-                      const f32x2 a = ya[z], b = yb[z];
-                      ya[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));
-                      yb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));
-                    }
-                  } else {
-#pragma unroll
-                    for (int z = 0; z < 4; ++z) {
-                      const f32x2 a = xa[z], b = xb[z];
-                      xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));     // a cos - b sin
-                      xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));      // a sin + b cos
-                    }
-                  }
-                }
-                uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
-                uint32_t* hp1 = reinterpret_cast<uint32_t*>(&h1);
-                uint32_t* lp0 = reinterpret_cast<uint32_t*>(&l0);
-                uint32_t* lp1 = reinterpret_cast<uint32_t*>(&l1);
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  // H = bf16(Delta); 2 L = bf16(Delta - H) with one added to both exponents (the doubling is
-                  // exact; a zero remainder becomes 2^-126, which no sum notices)
-                  const f32x2 da = f2_sub(ya[z], xa[z]), db = f2_sub(yb[z], xb[z]);
-                  hp0[z] = f2_to_bf16x2(da);
-                  hp1[z] = f2_to_bf16x2(db);
-                  lp0[z] = f2_to_bf16x2(f2_sub(da, f2_from_bf16x2(hp0[z]))) + 0x00800080u;
-                  lp1[z] = f2_to_bf16x2(f2_sub(db, f2_from_bf16x2(hp1[z]))) + 0x00800080u;
-                }
+                f32x2 unused = 0;
+                delta_operands_half<false>(*t0p, *t1p, *s0p, *s1p, csp, snp, j, rotate, SEG && at_source, h0, h1, l0, l1, unused);
               }
               *t0p = h0;
               *t1p = h1;
@@ -782,28 +822,8 @@ __device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTab
               uint4* sp = reinterpret_cast<uint4*>(sr + o);
               uint4 h = make_uint4(0, 0, 0, 0), l = h;
               if (live) {
-                float x[8], y[8];
-                unpack8(*sp, x);
-                unpack8(*tp, y);
-                if (rotate) {
-                  const int f0 = 16 * cq + 4 * jj;
-                  const float4 c0 = *reinterpret_cast<const float4*>(csp + f0);
-                  const float4 s0 = *reinterpret_cast<const float4*>(snp + f0);
-                  const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
-                  const float sgn = (SEG && at_source) ? -1.f : 1.f;
-                  const float sn[4] = {sgn * s0.x, sgn * s0.y, sgn * s0.z, sgn * s0.w};
-                  float* rv = (SEG && at_source) ? y : x;     // source coordinates: the target goes back by the shift
-#pragma unroll
-                  for (int z = 0; z < 4; ++z) {
-                    const float a = rv[2 * z], b = rv[2 * z + 1];
-                    rv[2 * z] = a * cs[z] - b * sn[z];
-                    rv[2 * z + 1] = a * sn[z] + b * cs[z];
-                  }
-                }
-                uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
-                uint32_t* lp = reinterpret_cast<uint32_t*>(&l);
-#pragma unroll
-                for (int z = 0; z < 4; ++z) split2x(y[2 * z] - x[2 * z], y[2 * z + 1] - x[2 * z + 1], hp[z], lp[z]);
+                float unused = 0.f;
+                delta_operands_interleaved<false>(*tp, *sp, csp, snp, 16 * cq + 4 * jj, rotate, SEG && at_source, h, l, unused);
               }
               *tp = h;
               if (p.has_src) *sp = l;
@@ -1114,65 +1134,7 @@ __device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, c
               uint4* s0p = reinterpret_cast<uint4*>(sr + o);
               uint4* s1p = reinterpret_cast<uint4*>(sr + kHalfBytes + o);
               uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0, l0 = h0, l1 = h0;
-              if (live) {
-                // packed float32 pairs throughout: word w of a 16-byte chunk holds channels 2w, 2w + 1
-                const uint4 sa = *s0p, sb = *s1p, ta = *t0p, tb = *t1p;
-                const uint32_t sw0[4] = {sa.x, sa.y, sa.z, sa.w}, sw1[4] = {sb.x, sb.y, sb.z, sb.w};
-                const uint32_t tw0[4] = {ta.x, ta.y, ta.z, ta.w}, tw1[4] = {tb.x, tb.y, tb.z, tb.w};
-                f32x2 xa[4], xb[4];
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  xa[z] = f2_from_bf16x2(sw0[z]);
-                  xb[z] = f2_from_bf16x2(sw1[z]);
-                }
-                f32x2 ya[4], yb[4];
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  ya[z] = f2_from_bf16x2(tw0[z]);
-                  yb[z] = f2_from_bf16x2(tw1[z]);
-                }
-                if (rotate) {
-                  const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
-                  float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
-                  if (SEG && at_source) {                    // the target goes back by the shift: the same rotation with the sines negated
-                    s0 = make_float4(-s0.x, -s0.y, -s0.z, -s0.w);
-                    s1 = make_float4(-s1.x, -s1.y, -s1.z, -s1.w);
-                  }
-                  const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
-                  const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
-                  const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
-                  if (SEG && at_source) {
-#pragma unroll
-                    for (int z = 0; z < 4; ++z) {
-                      const f32x2 a = ya[z], b = yb[z];
-                      ya[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));
-                      yb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));
-                    }
-                  } else {
-#pragma unroll
-                    for (int z = 0; z < 4; ++z) {
-                      const f32x2 a = xa[z], b = xb[z];
-                      xa[z] = f2_fma(a, cs[z], f2_mul(b, nsn[z]));     // a cos - b sin
-                      xb[z] = f2_fma(a, sn[z], f2_mul(b, cs[z]));      // a sin + b cos
-                    }
-                  }
-                }
-                uint32_t* hp0 = reinterpret_cast<uint32_t*>(&h0);
-                uint32_t* hp1 = reinterpret_cast<uint32_t*>(&h1);
-                uint32_t* lp0 = reinterpret_cast<uint32_t*>(&l0);
-                uint32_t* lp1 = reinterpret_cast<uint32_t*>(&l1);
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  // H = bf16(Delta); 2 L = bf16(Delta - H) with one added to both exponents (the doubling is
-                  // exact; a zero remainder becomes 2^-126, which no sum notices)
-                  const f32x2 da = f2_sub(ya[z], xa[z]), db = f2_sub(yb[z], xb[z]);
-                  sq2 = f2_fma(da, da, f2_fma(db, db, sq2));
-                  hp0[z] = f2_to_bf16x2(da);
-                  hp1[z] = f2_to_bf16x2(db);
-                  lp0[z] = f2_to_bf16x2(f2_sub(da, f2_from_bf16x2(hp0[z]))) + 0x00800080u;
-                  lp1[z] = f2_to_bf16x2(f2_sub(db, f2_from_bf16x2(hp1[z]))) + 0x00800080u;
-                }
-              }
+              if (live) delta_operands_half<true>(*t0p, *t1p, *s0p, *s1p, csp, snp, j, rotate, SEG && at_source, h0, h1, l0, l1, sq2);
               *t0p = h0;
               *t1p = h1;
               if (p.has_src) {
@@ -1189,34 +1151,7 @@ __device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, c
               uint4* tp = reinterpret_cast<uint4*>(tg + o);
               uint4* sp = reinterpret_cast<uint4*>(sr + o);
               uint4 h = make_uint4(0, 0, 0, 0), l = h;
-              if (live) {
-                float x[8], y[8];
-                unpack8(*sp, x);
-                unpack8(*tp, y);
-                if (rotate) {
-                  const int f0 = 16 * cq + 4 * jj;
-                  const float4 c0 = *reinterpret_cast<const float4*>(csp + f0);
-                  const float4 s0 = *reinterpret_cast<const float4*>(snp + f0);
-                  const float cs[4] = {c0.x, c0.y, c0.z, c0.w};
-                  const float sgn = (SEG && at_source) ? -1.f : 1.f;
-                  const float sn[4] = {sgn * s0.x, sgn * s0.y, sgn * s0.z, sgn * s0.w};
-                  float* rv = (SEG && at_source) ? y : x;     // source coordinates: the target goes back by the shift
-#pragma unroll
-                  for (int z = 0; z < 4; ++z) {
-                    const float a = rv[2 * z], b = rv[2 * z + 1];
-                    rv[2 * z] = a * cs[z] - b * sn[z];
-                    rv[2 * z + 1] = a * sn[z] + b * cs[z];
-                  }
-                }
-                uint32_t* hp = reinterpret_cast<uint32_t*>(&h);
-                uint32_t* lp = reinterpret_cast<uint32_t*>(&l);
-#pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  const float e0 = y[2 * z] - x[2 * z], e1 = y[2 * z + 1] - x[2 * z + 1];
-                  sq_cur = fmaf(e0, e0, fmaf(e1, e1, sq_cur));
-                  split2x(e0, e1, hp[z], lp[z]);
-                }
-              }
+              if (live) delta_operands_interleaved<true>(*tp, *sp, csp, snp, 16 * cq + 4 * jj, rotate, SEG && at_source, h, l, sq_cur);
               *tp = h;
               if (p.has_src) *sp = l;
             }
