@@ -38,6 +38,7 @@
 #include "kvc_tc.h"
 #include "kvc_tc_ptx.cuh"
 #include "kvc_tc_maps.h"
+#include "kvc_tc_store.cuh"
 
 namespace kvc {
 namespace tc {
@@ -485,24 +486,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
       const DevItem& it = *t.it;
       // paged destination: one lane per page; ids (and the validity of the matching source pages)
       // are fetched before waiting for the tile
-      const bool dpaged = it.dst.page_table != nullptr;
-      const int dpage = it.dst.page_mask + 1;
-      int id = -1, n_pages = 0, first = 0;
-      bool src_ok = true;
-      if (dpaged) {
-        const int per_tile = kTileTok >> it.dst.page_shift;
-        first = t.t0 >> it.dst.page_shift;
-        n_pages = min(per_tile, ((it.dst.T + dpage - 1) >> it.dst.page_shift) - first);
-        if (lane < n_pages) {
-          id = it.dst.page_table[first + lane];
-          if (it.src.page_table) {
-            const int tk0 = t.t0 + lane * dpage;
-            const int tk1 = min(tk0 + dpage, it.src.T);
-            for (int sp = tk0 >> it.src.page_shift; (sp << it.src.page_shift) < tk1; ++sp)
-              if ((unsigned)it.src.page_table[sp] >= (unsigned)it.src.n_phys) src_ok = false;
-          }
-        }
-      }
+      const StorePages pg = store_pages(it.dst, it.src, t.t0, lane);
       int ok = 1;
       if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), use & 1u, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -512,36 +496,8 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
       uint8_t* st_ptr = smem + s * kStageBytes;
       if constexpr (REDUCE) {
         // nothing to store: the slot goes straight back to the producer
-      } else if (!dpaged) {
-        if (lane == 0) {          // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
-          tma_store_5d(dmap, st_base, 0, t.t0, t.h, 0, t.l);
-          tma_store_5d(dmap, st_base + kHalfBytes, 64, t.t0, t.h, 0, t.l);
-        }
       } else {
-        // the last, partial page goes out row by row so that rows >= T stay untouched; pages whose
-        // source could not be loaded are skipped
-        const int last_pg = (it.dst.T - 1) >> it.dst.page_shift;
-        const bool last_partial = (it.dst.T & it.dst.page_mask) != 0;
-        const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.dst.n_phys;
-        if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
-        const bool partial = last_partial && (first + lane) == last_pg;
-        if (valid && src_ok && !partial) {
-          tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, t.h, id, t.l);
-          tma_store_5d(dmap, st_base + kHalfBytes + lane * dpage * 128, 64, 0, t.h, id, t.l);
-        }
-        const unsigned pm = __ballot_sync(0xffffffffu, valid && src_ok && partial);
-        if (pm) {
-          const int u = __ffs(pm) - 1;
-          const int rows = it.dst.T & it.dst.page_mask;
-          __nv_bfloat16* dbase = t.is_v ? it.dst.v : it.dst.k;
-          for (int c = lane; c < rows * 16; c += 32) {
-            const int row = u * dpage + (c >> 4), half = (c >> 3) & 1, j = c & 7;
-            __nv_bfloat16* drow = row_ptr(it.dst, dbase, t.l, t.h, t.t0 + row, p.status);
-            if (drow)
-              *reinterpret_cast<uint4*>(drow + half * 64 + j * 8) =
-                  *reinterpret_cast<const uint4*>(st_ptr + half * kHalfBytes + row * 128 + ((j ^ (row & 7)) << 4));
-          }
-        }
+        store_tile(it.dst, dmap, st_base, st_ptr, t.t0, t.l, t.h, t.is_v != 0, lane, pg, p.status);
       }
       tma_store_commit();
       tma_store_wait_read();

@@ -25,6 +25,7 @@
 #include "kvc_tc.h"
 #include "kvc_tc_ptx.cuh"
 #include "kvc_tc_maps.h"
+#include "kvc_tc_store.cuh"
 #include "kvc_tc_stream.cuh"
 
 namespace kvc {
@@ -285,24 +286,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
       for (int a = 0; a < NH; ++a, ++step) {
         const int s = step % NOUT;
         const DevCache& dc = p.hop[a].dst;
-        const bool dpaged = dc.page_table != nullptr;
-        const int dpage = dc.page_mask + 1;
-        int id = -1, n_pages = 0, first = 0;
-        bool src_ok = true;
-        if (dpaged) {
-          const int per_tile = kTileTok >> dc.page_shift;
-          first = t0 >> dc.page_shift;
-          n_pages = min(per_tile, ((dc.T + dpage - 1) >> dc.page_shift) - first);
-          if (lane < n_pages) {
-            id = dc.page_table[first + lane];
-            if (p.src.page_table) {
-              const int tk0 = t0 + lane * dpage;
-              const int tk1 = min(tk0 + dpage, p.src.T);
-              for (int sp = tk0 >> p.src.page_shift; (sp << p.src.page_shift) < tk1; ++sp)
-                if ((unsigned)p.src.page_table[sp] >= (unsigned)p.src.n_phys) src_ok = false;
-            }
-          }
-        }
+        const StorePages pg = store_pages(dc, p.src, t0, lane);   // page ids fetched before the wait
         int ok = 1;
         if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->oready[s]), (step / NOUT) & 1u, abort_flag) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -313,35 +297,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
         const CUtensorMap* dmap = is_v ? &p.dst_v[a] : &p.dst_k[a];
         const uint32_t st_base = outs + s * kBaseBytes;
         uint8_t* st_ptr = smem + kOutOff + s * kBaseBytes;
-        if (!dpaged) {
-          if (lane == 0) {        // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
-            tma_store_5d(dmap, st_base, 0, t0, h, 0, l);
-            tma_store_5d(dmap, st_base + kHalfBytes, 64, t0, h, 0, l);
-          }
-        } else {
-          const int last_pg = (dc.T - 1) >> dc.page_shift;
-          const bool last_partial = (dc.T & dc.page_mask) != 0;
-          const bool valid = lane < n_pages && (unsigned)id < (unsigned)dc.n_phys;
-          if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
-          const bool partial = last_partial && (first + lane) == last_pg;
-          if (valid && src_ok && !partial) {
-            tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, h, id, l);
-            tma_store_5d(dmap, st_base + kHalfBytes + lane * dpage * 128, 64, 0, h, id, l);
-          }
-          const unsigned pm = __ballot_sync(0xffffffffu, valid && src_ok && partial);
-          if (pm) {
-            const int u = __ffs(pm) - 1;
-            const int rows = dc.T & dc.page_mask;
-            __nv_bfloat16* dbase = is_v ? dc.v : dc.k;
-            for (int c = lane; c < rows * 16; c += 32) {
-              const int row = u * dpage + (c >> 4), half = (c >> 3) & 1, j = c & 7;
-              __nv_bfloat16* drow = row_ptr(dc, dbase, l, h, t0 + row, p.status);
-              if (drow)
-                *reinterpret_cast<uint4*>(drow + half * 64 + j * 8) =
-                    *reinterpret_cast<const uint4*>(st_ptr + half * kHalfBytes + row * 128 + ((j ^ (row & 7)) << 4));
-            }
-          }
-        }
+        store_tile(dc, dmap, st_base, st_ptr, t0, l, h, is_v != 0, lane, pg, p.status);
         tma_store_commit();
         tma_store_wait_read();
         __syncwarp();

@@ -26,6 +26,7 @@
 #include "kvc_tc.h"
 #include "kvc_tc_ptx.cuh"
 #include "kvc_tc_maps.h"
+#include "kvc_tc_store.cuh"
 #include "kvc_tc_stream.cuh"
 
 namespace kvc {
@@ -300,24 +301,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
     for (; !w.done(); w.next(), ++i) {
       const int s = i % NSTAGE;
       const int t0 = w.t0(), is_v = w.is_v(), l = w.l, h = w.h;
-      const bool dpaged = p.dst.page_table != nullptr;
-      const int dpage = p.dst.page_mask + 1;
-      int id = -1, n_pages = 0, first = 0;
-      bool src_ok = true;
-      if (dpaged) {
-        const int per_tile = kTileTok >> p.dst.page_shift;
-        first = t0 >> p.dst.page_shift;
-        n_pages = min(per_tile, ((p.dst.T + dpage - 1) >> p.dst.page_shift) - first);
-        if (lane < n_pages) {
-          id = p.dst.page_table[first + lane];
-          if (p.src.page_table) {
-            const int tk0 = t0 + lane * dpage;
-            const int tk1 = min(tk0 + dpage, p.src.T);
-            for (int sp = tk0 >> p.src.page_shift; (sp << p.src.page_shift) < tk1; ++sp)
-              if ((unsigned)p.src.page_table[sp] >= (unsigned)p.src.n_phys) src_ok = false;
-          }
-        }
-      }
+      const StorePages pg = store_pages(p.dst, p.src, t0, lane);     // page ids fetched before the wait
       int ok = 1;
       if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->ready[s]), (i / NSTAGE) & 1u, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -325,37 +309,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
       const CUtensorMap* dmap = is_v ? &p.dst_v : &p.dst_k;
       const uint32_t st_base = stages + s * kBaseBytes;
       uint8_t* st_ptr = smem + s * kBaseBytes;
-      if (!dpaged) {
-        if (lane == 0) {          // a contiguous tile is stored whole; rows >= T are clipped by the tensor map
-          tma_store_5d(dmap, st_base, 0, t0, h, 0, l);
-          tma_store_5d(dmap, st_base + kHalfBytes, 64, t0, h, 0, l);
-        }
-      } else {
-        // the last, partial page goes out row by row so that rows >= T stay untouched; pages whose
-        // source could not be loaded are skipped
-        const int last_pg = (p.dst.T - 1) >> p.dst.page_shift;
-        const bool last_partial = (p.dst.T & p.dst.page_mask) != 0;
-        const bool valid = lane < n_pages && (unsigned)id < (unsigned)p.dst.n_phys;
-        if (lane < n_pages && !valid) atomicOr(p.status, KVC_FLAG_BAD_PAGE);
-        const bool partial = last_partial && (first + lane) == last_pg;
-        if (valid && src_ok && !partial) {
-          tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, h, id, l);
-          tma_store_5d(dmap, st_base + kHalfBytes + lane * dpage * 128, 64, 0, h, id, l);
-        }
-        const unsigned pm = __ballot_sync(0xffffffffu, valid && src_ok && partial);
-        if (pm) {
-          const int u = __ffs(pm) - 1;
-          const int rows = p.dst.T & p.dst.page_mask;
-          __nv_bfloat16* dbase = is_v ? p.dst.v : p.dst.k;
-          for (int c = lane; c < rows * 16; c += 32) {
-            const int row = u * dpage + (c >> 4), half = (c >> 3) & 1, j = c & 7;
-            __nv_bfloat16* drow = row_ptr(p.dst, dbase, l, h, t0 + row, p.status);
-            if (drow)
-              *reinterpret_cast<uint4*>(drow + half * 64 + j * 8) =
-                  *reinterpret_cast<const uint4*>(st_ptr + half * kHalfBytes + row * 128 + ((j ^ (row & 7)) << 4));
-          }
-        }
-      }
+      store_tile(p.dst, dmap, st_base, st_ptr, t0, l, h, is_v != 0, lane, pg, p.status);
       tma_store_commit();
       tma_store_wait_read();
       __syncwarp();
