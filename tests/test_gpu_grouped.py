@@ -180,9 +180,11 @@ def _fit_grouped(src, tgt, shift, cfg, r, mode):
 CFG_G2 = wl.CONFIGS["llama8b_8k"].scaled(name="8b_H2", L=2, H=2, T=700, r=16)
 CFG_G8 = wl.CONFIGS["llama8b_8k"].scaled(name="8b_H8", L=1, H=8, T=1100)           # D = 1024, r = 32
 CFG_GP = wl.CONFIGS["vlm_16k"].scaled(name="vlm_H4", L=1, H=4, T=901, image_spans=())  # paged, D = 512
+CFG_G64 = wl.CONFIGS["tiny"].scaled(name="tiny_d64", L=2, H=3, T=333)                  # head_dim 64: D = 192, the CUDA-core
+                                                                                        # passes; 48 columns per block of a cluster
 
 
-@pytest.mark.parametrize("cfg", [CFG_G2, CFG_G8, CFG_GP], ids=lambda c: c.name)
+@pytest.mark.parametrize("cfg", [CFG_G2, CFG_G8, CFG_GP, CFG_G64], ids=lambda c: c.name)
 @pytest.mark.parametrize("mode", ["fit", "fit_fast"])
 def test_grouped_fit(cfg, mode):
     """FIT under D = H d (Sec. 3.1, Eq. 7): the r leading right singular vectors of a layer's concatenated
