@@ -105,6 +105,14 @@ def test_grouped_chain_and_batch(path):
     kvc.kvc_apply_batch(items, rope, ws, stg)
     torch.cuda.synchronize()
     assert torch.equal(bd[0].k, outs[0].k) and torch.equal(bd[1].v, outs[1].v)
+    # the first hop once more as two items with token ranges over the same caches (the grouped coefficient rows are
+    # addressed by absolute token): the same bits as the whole-cache item
+    cut = 256
+    tw = hp.empty_dst(src_cpu, cfg, DEV)
+    parts = [kvc.Item(src, tw, dev_states[0], pl[1] - pl[0], 0, cut), kvc.Item(src, tw, dev_states[0], pl[1] - pl[0], cut, cfg.T)]
+    kvc.kvc_apply_batch(parts, rope, ws, stg)
+    torch.cuda.synchronize()
+    assert torch.equal(tw.k, outs[0].k) and torch.equal(tw.v, outs[0].v)
 
 
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
