@@ -1,0 +1,251 @@
+"""Seeded sweep over random shapes: kvc_apply and kvc_state_update (project) against the fp64 oracle.
+
+The other GPU tests pick their shapes by hand around known tile and page boundaries; this one
+draws them (head_dim, rank, layers, heads, length, coverage, page size, shift, RoPE pairing,
+basis dtype), so that combinations nobody thought of are compared element by element too.
+Whatever kernel family the library chooses for a shape is the one that is checked.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_34060_b200 as kvc
+from paper_2609_34060_b200 import workloads as wl
+from oracle import kvc_oracle as orc
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+BASE = wl.CONFIGS["llama8b_8k"]
+
+
+@pytest.fixture(autouse=True)
+def _clean_status():
+    kvc.kvc_status_reset()
+    kvc.kvc_set_path(kvc.KVC_PATH_AUTO)
+    yield
+    assert kvc.kvc_status_poll() == 0
+
+
+def _draw(seed):
+    g = np.random.default_rng(77000 + seed)
+    d = int(g.choice([64, 128, 128, 128]))
+    r = int(g.choice([1, 3, 4, 8, 12, 16, 17, 24, 32, 33, 40, 48, 64]))
+    T = int(g.choice([g.integers(1, 140), g.integers(140, 900)]))
+    paged = bool(g.integers(0, 2))
+    cfg = BASE.scaled(name=f"rand{seed}", L=int(g.integers(1, 4)), H=int(g.integers(1, 4)), d=d, T=T, r=r,
+                      n_agents=4, paged=paged, page=int(g.choice([8, 16, 32, 64])), outliers=int(g.integers(0, 3)),
+                      theta=float(g.choice([10000.0, 500000.0])), seed=seed)
+    n_cov = int(g.choice([T, T, g.integers(0, T + 1)]))
+    shift = int(g.choice([0, g.integers(-600, 600)]))
+    pairing = int(g.choice([kvc.KVC_ROPE_HALF, kvc.KVC_ROPE_HALF, kvc.KVC_ROPE_INTERLEAVED]))
+    bdt = torch.bfloat16 if g.integers(0, 4) == 0 else torch.float32
+    return cfg, n_cov, shift, pairing, bdt
+
+
+def _opair(pairing):
+    return orc.ROPE_HALF if pairing == kvc.KVC_ROPE_HALF else orc.ROPE_INTERLEAVED
+
+
+@pytest.mark.parametrize("seed", range(28))
+def test_apply_random_shape(seed):
+    cfg, n_cov, shift, pairing, bdt = _draw(seed)
+    src_cpu = hp.make_cache(cfg)
+    if n_cov:
+        st_cpu = hp.make_state(cfg, 1 + seed % 3, n_cov=n_cov, basis_dtype=bdt)
+    else:
+        full = hp.make_state(cfg, 1, basis_dtype=bdt)
+        st_cpu = kvc.State(None, None, full.basis_k, full.basis_v, n_cov=0)
+    src = hp.to_dev(src_cpu, DEV)
+    dst = hp.empty_dst(src_cpu, cfg, DEV, fill=-3.0)
+    kvc.kvc_apply(src, hp.state_to_dev(st_cpu, DEV), shift, kvc.Rope(cfg.theta, pairing), dst)
+    torch.cuda.synchronize()
+    osrc = hp.oracle_cache(src_cpu)
+    odst = osrc.empty_like(page_table=None if dst.page_table is None else dst.page_table.cpu().numpy())
+    odst, ref_k, ref_v = orc.apply(osrc, hp.oracle_state(st_cpu), shift, hp.inv_freq(cfg), dst=odst,
+                                   pairing=_opair(pairing), want_ref=True)
+    gk, gv = hp.logical_bits(dst, "k"), hp.logical_bits(dst, "v")
+    rk, rv = hp.tol_ratio(gk, ref_k), hp.tol_ratio(gv, ref_v)
+    assert rk <= 1.0 and rv <= 1.0, (cfg, n_cov, shift, pairing, rk, rv)
+    assert hp.ulp_mismatch_fraction(gk, hp.logical_bits(odst, "k")) < 1e-2
+    assert hp.ulp_mismatch_fraction(gv, hp.logical_bits(odst, "v")) < 1e-2
+    # rows behind the covered prefix: values pass through bit for bit
+    assert np.array_equal(gv[:, :, n_cov:], hp.logical_bits(src_cpu, "v")[:, :, n_cov:])
+    assert torch.equal(src.k.cpu(), src_cpu.k) and torch.equal(src.v.cpu(), src_cpu.v)
+    if dst.page_table is not None:
+        fill = torch.tensor(-3.0, dtype=torch.bfloat16)
+        mapped = set(int(p) for p in dst.page_table.cpu())
+        for p in range(dst.P):
+            if p not in mapped:
+                assert torch.all(dst.k[:, p].cpu() == fill) and torch.all(dst.v[:, p].cpu() == fill)
+        tail = cfg.T % cfg.page
+        if tail:
+            last = int(dst.page_table[-1])
+            assert torch.all(dst.k[:, last, :, tail:].cpu() == fill) and torch.all(dst.v[:, last, :, tail:].cpu() == fill)
+
+
+@pytest.mark.parametrize("seed", range(100, 116))
+def test_project_random_shape(seed):
+    cfg, n_cov, shift, pairing, bdt = _draw(seed)
+    n_cov = max(n_cov, 1)
+    f = hp.inv_freq(cfg)
+    src_cpu = hp.make_cache(cfg)
+    true = hp.make_state(cfg, 1)
+    nk = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2).numpy()
+    nv = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 3).numpy()
+    osrc = hp.oracle_cache(src_cpu)
+    otgt = orc.make_target(osrc, hp.oracle_state(true), shift, f, nk, nv, cfg.sigma, pairing=_opair(pairing))
+    as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    if cfg.paged:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v), T=cfg.T, page_table=src_cpu.page_table)
+    else:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v))
+    other = hp.make_state(cfg, 3, basis_dtype=bdt)
+    bk, bv = other.basis_k.float().numpy(), other.basis_v.float().numpy()
+    ost, _ = orc.state_update(osrc, otgt, shift, f, mode=orc.PROJECT, n_cov=n_cov, basis_k=bk, basis_v=bv,
+                              pairing=_opair(pairing))
+    st = kvc.State(torch.full((cfg.L, cfg.H, n_cov, cfg.r), 7.0, device=DEV),
+                   torch.full((cfg.L, cfg.H, n_cov, cfg.r), 7.0, device=DEV),
+                   other.basis_k.to(DEV), other.basis_v.to(DEV), n_cov=n_cov)
+    kvc.kvc_state_update(hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV), shift, kvc.Rope(cfg.theta, pairing), st,
+                         kvc.KVC_PROJECT)
+    torch.cuda.synchronize()
+    worst = 0.0
+    for l in range(cfg.L):
+        for h in range(cfg.H):
+            for which, got, ref, bs in (("k", st.coeff_k, ost.coeff_k, bk), ("v", st.coeff_v, ost.coeff_v, bv)):
+                dl = orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, f, which == "k",
+                                   pairing=_opair(pairing))[:n_cov]
+                bn = np.linalg.norm(bs[l, h].astype(np.float64), axis=1)[None, :]
+                dn = np.linalg.norm(dl, axis=1)[:, None]
+                sn = np.linalg.norm(orc.bf16_to_f64(osrc.get_bits(which, l, h)), axis=1)[:n_cov, None]
+                tn = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h)), axis=1)[:n_cov, None]
+                # product rounding of the split-precision contraction; float32 rotation and
+                # cancellation in tgt - Rot(src), relative to the inputs' size
+                tol = 2.0 ** -12 * dn * bn + 2.0 ** -18 * (sn + tn) * bn + 1e-6
+                err = np.abs(got[l, h].cpu().numpy().astype(np.float64) - ref[l, h].astype(np.float64))
+                worst = max(worst, float(np.max(err / tol)))
+    assert worst <= 1.0, (cfg, n_cov, shift, pairing, worst)
+
+
+@pytest.mark.parametrize("seed", range(200, 212))
+def test_chain_random_shape(seed):
+    """kvc_chain against the oracle's chain at every hop; kvc_chain_fused equal to kvc_chain bit for bit
+    (whether the fused kernel serves the shape or the call runs hop by hop)."""
+    cfg, _, _, pairing, _ = _draw(seed)
+    g = np.random.default_rng(88000 + seed)
+    n = int(g.integers(2, 6))
+    cfg = cfg.scaled(n_agents=n)
+    pl = [int(x) for x in g.integers(0, 700, size=n)]
+    states_cpu = []
+    for a in range(1, n):
+        kind = int(g.integers(0, 6))
+        if kind == 0:
+            states_cpu.append(kvc.State.empty())
+            continue
+        r = int(g.choice([4, 8, 16, 32, 48, 64, cfg.r]))
+        n_cov = cfg.T if kind < 4 else int(g.integers(1, cfg.T + 1))
+        bdt = torch.bfloat16 if kind == 3 else torch.float32
+        states_cpu.append(hp.make_state(cfg, a, n_cov=n_cov, r=r, basis_dtype=bdt))
+    rope = kvc.Rope(cfg.theta, pairing)
+    src_cpu = hp.make_cache(cfg)
+    src = hp.to_dev(src_cpu, DEV)
+    states = [hp.state_to_dev(s, DEV) for s in states_cpu]
+    ref = [hp.empty_dst(src_cpu, cfg, DEV, table_tag=60 + a, fill=2.0) for a in range(1, n)]
+    got = [kvc.Cache(torch.full_like(o.k, 2.0), torch.full_like(o.v, 2.0), T=o.T if o.page_table is not None else None,
+                     page_table=o.page_table) for o in ref]
+    kvc.kvc_chain(src, pl, states, rope, ref)
+    ws = torch.empty(max(kvc.kvc_chain_workspace_bytes(src, n), 128), dtype=torch.uint8, device=DEV)
+    kvc.kvc_chain_fused(src, pl, states, rope, got, ws)
+    torch.cuda.synchronize()
+    for a, (x, y) in enumerate(zip(got, ref)):
+        assert torch.equal(x.k, y.k) and torch.equal(x.v, y.v), (cfg, pl, a + 1)
+    tables = [None if o.page_table is None else o.page_table.cpu().numpy() for o in ref]
+    out, refs = orc.chain(hp.oracle_cache(src_cpu), pl, [hp.oracle_state(s) for s in states_cpu], hp.inv_freq(cfg),
+                          dst_tables=tables, pairing=_opair(pairing), want_ref=True)
+    for a in range(1, n):
+        # strict parity of every hop from oracle-identical inputs: hop 1 reads agent 0, a later hop is run
+        # once more from the ORACLE's materialised cache of the agent before (oracle -> library only)
+        rk, rv = refs[a - 1]
+        if a == 1:
+            dst = ref[0]
+        else:
+            o_src = out[a - 2]
+            as_t = lambda x: torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).to(DEV)
+            hop_src = kvc.Cache(as_t(o_src.k), as_t(o_src.v), T=cfg.T if cfg.paged else None,
+                                page_table=None if not cfg.paged else torch.from_numpy(o_src.page_table).to(DEV))
+            dst = hp.empty_dst(src_cpu, cfg, DEV, table_tag=60 + a, fill=2.0)
+            kvc.kvc_apply(hop_src, states[a - 1], pl[a] - pl[a - 1], rope, dst)
+            torch.cuda.synchronize()
+        assert hp.tol_ratio(hp.logical_bits(dst, "k"), rk) <= 1.0, (cfg, pl, a)
+        assert hp.tol_ratio(hp.logical_bits(dst, "v"), rv) <= 1.0, (cfg, pl, a)
+        # end to end the two chains stay together: a rare one-ulp difference at a hop moves the next
+        # hop's input by one bf16 step, so this bar is statistical
+        for which, r_ in (("k", rk), ("v", rv)):
+            got_f = orc.bf16_to_f64(hp.logical_bits(ref[a - 1], which))
+            bad = np.abs(got_f - r_) > hp.BF16_REL * np.abs(r_) + hp.BF16_ABS
+            assert bad.mean() < 2e-3, (cfg, pl, a, which)
+
+
+@pytest.mark.parametrize("mode", ["fit", "fit_fast"])
+@pytest.mark.parametrize("seed", range(300, 310))
+def test_fit_random_shape(seed, mode):
+    """Both fit modes on drawn shapes (lengths below and above the rank and the head dimension, partial
+    coverage, pages, shifts): the oracle's eigenvalues, orthonormal rows where the eigenvalue is not zero,
+    zero rows beyond the number of covered tokens, a residual at the tail energy (Eckart-Young), and
+    coefficients that are the projection of the deviation onto the library's own basis."""
+    cfg, n_cov, shift, pairing, _ = _draw(seed)
+    g = np.random.default_rng(99000 + seed)
+    r_fit = int(g.choice([1, 4, 8, 16, 32])) if mode == "fit_fast" else int(g.choice([1, 4, 8, 16, 32, 33, 64]))
+    r_fit = min(r_fit, cfg.d)
+    n_cov = max(n_cov, 1)
+    kmode = kvc.KVC_FIT if mode == "fit" else kvc.KVC_FIT_FAST
+    f = hp.inv_freq(cfg)
+    src_cpu = hp.make_cache(cfg)
+    true = hp.make_state(cfg, 1, r=min(cfg.r, 8))
+    nk = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 2).numpy()
+    nv = wl.noise((cfg.L, cfg.H, cfg.T, cfg.d), cfg.seed, 3).numpy()
+    osrc = hp.oracle_cache(src_cpu)
+    otgt = orc.make_target(osrc, hp.oracle_state(true), shift, f, nk, nv, cfg.sigma, pairing=_opair(pairing))
+    as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    if cfg.paged:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v), T=cfg.T, page_table=src_cpu.page_table)
+    else:
+        tgt_cpu = kvc.Cache(as_t(otgt.k), as_t(otgt.v))
+    L, H, d = cfg.L, cfg.H, cfg.d
+    tgt = hp.to_dev(tgt_cpu, DEV)
+    st = kvc.State(torch.full((L, H, n_cov, r_fit), 5.0, device=DEV), torch.full((L, H, n_cov, r_fit), 5.0, device=DEV),
+                   torch.full((L, H, r_fit, d), 3.0, device=DEV), torch.full((L, H, r_fit, d), 3.0, device=DEV), n_cov=n_cov)
+    ws = torch.zeros(kvc.kvc_workspace_bytes(tgt, st, kmode), dtype=torch.uint8, device=DEV)
+    kvc.kvc_state_update(hp.to_dev(src_cpu, DEV), tgt, shift, kvc.Rope(cfg.theta, pairing), st, kmode, workspace=ws)
+    torch.cuda.synchronize()
+    m = L * H * 2
+    ev = ws.view(torch.float32)[2 * m * d * d: 2 * m * d * d + m * d].cpu().numpy().astype(np.float64).reshape(L, H, 2, d)
+    for l in range(L):
+        for h in range(H):
+            for i, (which, B_t, c_t) in enumerate((("k", st.basis_k, st.coeff_k), ("v", st.basis_v, st.coeff_v))):
+                dl = orc.deviation(osrc.get_bits(which, l, h), otgt.get_bits(which, l, h), shift, f, which == "k",
+                                   pairing=_opair(pairing))[:n_cov]
+                w = np.sort(np.linalg.eigvalsh(orc.gram(dl)))[::-1]
+                w = np.maximum(w, 0.0)
+                B = B_t[l, h].cpu().numpy().astype(np.float64)
+                c = c_t[l, h].cpu().numpy().astype(np.float64)
+                what = (cfg, n_cov, shift, r_fit, l, h, which)
+                if mode == "fit":
+                    assert np.max(np.abs(ev[l, h, i] - w)) <= 1e-4 * w[0] + 1e-12, what
+                live = min(r_fit, n_cov, d)
+                assert np.all(B[live:] == 0), what                       # more rank asked for than rows exist
+                Gb = B[:live] @ B[:live].T
+                nz = np.diag(Gb) > 0.5                                   # rows of eigenvalue zero may be zero
+                assert np.max(np.abs(Gb[np.ix_(nz, nz)] - np.eye(int(nz.sum())))) <= 1e-4, what
+                assert np.all(w[:live][~nz] <= 1e-5 * w[0] + 1e-12), what
+                res = float(np.sum((dl - c @ B) ** 2))
+                tail = float(np.sum(w[r_fit:]))
+                assert res <= 1.001 * tail + 8 * r_fit * 1.2e-6 * w[0] + 1e-9 * float(np.sum(w)) + 1e-9, what + (res, tail)
+                bn = np.linalg.norm(B, axis=1)[None, :]
+                dn = np.linalg.norm(dl, axis=1)[:, None]
+                sn = np.linalg.norm(orc.bf16_to_f64(osrc.get_bits(which, l, h)), axis=1)[:n_cov, None]
+                tn = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h)), axis=1)[:n_cov, None]
+                tol = 2.0 ** -12 * dn * bn + 2.0 ** -18 * (sn + tn) * bn + 1e-6
+                assert np.max(np.abs(c - dl @ B.T) / tol) <= 1.0, what
