@@ -249,3 +249,83 @@ def test_fit_random_shape(seed, mode):
                 tn = np.linalg.norm(orc.bf16_to_f64(otgt.get_bits(which, l, h)), axis=1)[:n_cov, None]
                 tol = 2.0 ** -12 * dn * bn + 2.0 ** -18 * (sn + tn) * bn + 1e-6
                 assert np.max(np.abs(c - dl @ B.T) / tol) <= 1.0, what
+
+
+@pytest.mark.parametrize("seed", range(400, 414))
+def test_apply_segmented_random_shape(seed):
+    """kvc_apply_segmented on drawn shapes with one to five drawn segments (boundaries anywhere, shifts of
+    either sign or zero, both coordinate conventions) against the oracle's per-token-shift apply."""
+    cfg, n_cov, _, _, bdt = _draw(seed)
+    g = np.random.default_rng(55000 + seed)
+    n_seg = int(g.integers(1, min(5, cfg.T) + 1))
+    t_begin = [0] + sorted(int(x) for x in g.choice(np.arange(1, max(cfg.T, 2)), size=n_seg - 1, replace=False)) if cfg.T > 1 else [0]
+    shift = [int(g.choice([0, g.integers(-600, 600)])) for _ in t_begin]
+    coords = int(g.choice([kvc.KVC_COORDS_TARGET, kvc.KVC_COORDS_SOURCE]))
+    n_cov = max(n_cov, 1)
+    s_tok = orc.segment_shifts(cfg.T, t_begin, shift)
+    f = hp.inv_freq(cfg)
+    src_cpu = hp.make_cache(cfg)
+    st_cpu = hp.make_state(cfg, 1, n_cov=n_cov, basis_dtype=bdt)
+    dst = hp.empty_dst(src_cpu, cfg, DEV, fill=-3.0)
+    kvc.kvc_apply_segmented(hp.to_dev(src_cpu, DEV), hp.state_to_dev(st_cpu, DEV), kvc.Segments(t_begin, shift, coords),
+                            kvc.Rope(cfg.theta), dst)
+    torch.cuda.synchronize()
+    osrc, ost = hp.oracle_cache(src_cpu), hp.oracle_state(st_cpu)
+    for which in ("k", "v"):
+        got = hp.logical_bits(dst, which)
+        for l in range(cfg.L):
+            for h in range(cfg.H):
+                c = (ost.coeff_k if which == "k" else ost.coeff_v)[l, h]
+                b = (ost.basis_k if which == "k" else ost.basis_v)[l, h]
+                ref, exp = orc.apply_slab_tokens(osrc.get_bits(which, l, h), c, b, s_tok, f, n_cov, which == "k", coords=coords)
+                what = (cfg, n_cov, t_begin, shift, coords, which, l, h)
+                assert hp.tol_ratio(got[l, h], ref) <= 1.0, what
+                assert hp.ulp_mismatch_fraction(got[l, h], exp) < 1e-2, what
+                keep = (s_tok == 0) & (np.arange(cfg.T) >= n_cov) if which == "k" else (np.arange(cfg.T) >= n_cov)
+                assert np.array_equal(got[l, h][keep], osrc.get_bits(which, l, h)[keep]), what
+
+
+@pytest.mark.parametrize("seed", range(500, 512))
+def test_apply_multi_random_shape(seed):
+    """kvc_apply_multi (Eq. 8, token-wise weights) on drawn shapes: one to five anchors of drawn ranks
+    (multiples of 4 up to 64) and coverages, weighted or with unit weights, against the oracle."""
+    cfg, _, shift, _, _ = _draw(seed)
+    cfg = cfg.scaled(d=128)
+    g = np.random.default_rng(66000 + seed)
+    V = int(g.integers(1, 6))
+    ranks = [int(g.choice([4, 8, 16, 20, 32, 48, 64])) for _ in range(V)]
+    n_covs = [cfg.T if g.integers(0, 2) else int(g.integers(1, cfg.T + 1)) for _ in range(V)]
+    anchors = [hp.make_state(cfg, hop=v + 1, r=r, n_cov=n) for v, (r, n) in enumerate(zip(ranks, n_covs))]
+    src_cpu = hp.make_cache(cfg)
+    wk = wv = None
+    if g.integers(0, 3) > 0:
+        tp = kvc.kvc_multi_tpad(cfg.T)
+
+        def weights(tag):
+            w = wl.noise((V, cfg.T), cfg.seed, 300 + tag, "cpu").abs() + 0.05
+            w = w / w.sum(dim=0, keepdim=True)
+            out = torch.zeros(V, tp, dtype=torch.float32)
+            out[:, :cfg.T] = w
+            return out
+        wk, wv = weights(0), weights(1)
+    src = hp.to_dev(src_cpu, DEV)
+    dst = hp.empty_dst(src_cpu, cfg, DEV, fill=-7.0)
+    dev_anchors = [hp.state_to_dev(a, DEV) for a in anchors]
+    ws = torch.empty(max(kvc.kvc_multi_workspace_bytes(src, dev_anchors), 128), dtype=torch.uint8, device=DEV)
+    mv = lambda t: None if t is None else t.to(DEV)
+    kvc.kvc_apply_multi(src, dev_anchors, mv(wk), mv(wv), shift, kvc.Rope(cfg.theta), dst, ws)
+    torch.cuda.synchronize()
+    osrc = hp.oracle_cache(src_cpu)
+    inv = hp.inv_freq(cfg)
+    for which, w in (("k", wk), ("v", wv)):
+        got = hp.logical_bits(dst, which)
+        for l in range(cfg.L):
+            for h in range(cfg.H):
+                ref, out = orc.apply_multi_slab(
+                    osrc.get_bits(which, l, h), None if w is None else w.numpy()[:, :cfg.T],
+                    [getattr(a, "coeff_" + which)[l, h].numpy() for a in anchors],
+                    [getattr(a, "basis_" + which)[l, h].to(torch.float32).numpy() for a in anchors],
+                    n_covs, shift, inv, which == "k", orc.ROPE_HALF)
+                what = (cfg, ranks, n_covs, shift, which, l, h)
+                assert hp.tol_ratio(got[l, h], ref) <= 1.0, what
+                assert hp.ulp_mismatch_fraction(got[l, h], out) < 2e-2, what
