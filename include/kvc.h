@@ -58,6 +58,7 @@ extern "C" {
 #define KVC_PATH_AUTO    0  /* pick the fastest kernel that supports the arguments */
 #define KVC_PATH_GENERIC 1  /* CUDA-core kernels (any supported shape)             */
 #define KVC_PATH_TC      2  /* TMA + tcgen05 kernels (d = 128, r <= 64 ...)        */
+#define KVC_PATH_MIXED   3  /* kvc_last_path only: a batch split between the two   */
 
 /*
  * One agent's cache of the shared context (the paper's C_{i,seg}, Sec. 2.1 /
@@ -362,6 +363,10 @@ int kvc_state_update_noalloc(const kvc_cache *src, const kvc_cache *tgt, int32_t
  * item is one request's next hop, with its own length, rank, shift and tables).
  * The computation per item is exactly kvc_apply's.
  *   items      HOST array [n_items]; every item's caches must share d.
+ *              Items the tensor-core kernels serve (head_dim 128, 0 < r <= 64 a multiple of 4, ...) run
+ *              there, the others (empty states, odd ranks) on the CUDA-core kernel in a launch of
+ *              their own: one such request does not slow the rest of the batch down
+ *              (kvc_last_path: KVC_PATH_MIXED).
  *   workspace  DEVICE scratch >= kvc_batch_workspace_bytes(n_items), 256-byte aligned;
  *              receives the launch's work table and must stay untouched until the
  *              launch has finished.

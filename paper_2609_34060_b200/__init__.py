@@ -23,7 +23,7 @@ KVC_ROPE_HALF, KVC_ROPE_INTERLEAVED = 0, 1
 KVC_PROJECT, KVC_FIT, KVC_FIT_FAST = 0, 1, 2
 (KVC_SOLVER_SUBSPACE, KVC_SOLVER_FULL_RANK, KVC_SOLVER_FULL_DEPENDENT, KVC_SOLVER_FULL_SLOW, KVC_SOLVER_FULL_NO_GAP,
  KVC_SOLVER_FULL_SWEEPS) = (0, -1, 2, 3, 4, 5)
-KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC = 0, 1, 2
+KVC_PATH_AUTO, KVC_PATH_GENERIC, KVC_PATH_TC, KVC_PATH_MIXED = 0, 1, 2, 3
 KVC_MAX_SEGMENTS, KVC_COORDS_TARGET, KVC_COORDS_SOURCE = 16, 0, 1
 KVC_GROUP_HEAD, KVC_GROUP_LAYER = 0, 1
 KVC_FLAG_BAD_PAGE, KVC_FLAG_WAIT_EXPIRED, KVC_FLAG_NOT_CONVERGED = 1, 2, 4

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 
 #include "../../include/kvc.h"
@@ -753,7 +754,9 @@ static size_t batch_prefix_bytes(int32_t n) { return (((size_t)(n + 1) * sizeof(
 
 size_t kvc_batch_workspace_bytes(int32_t n_items) {
   if (n_items <= 0) return 0;
-  return batch_prefix_bytes(n_items) + (size_t)n_items * sizeof(DevItem) + tc_batch_extra_bytes(n_items);
+  // the last batch_prefix_bytes: the tile prefix of the items a mixed launch leaves to the CUDA-core kernel
+  return batch_prefix_bytes(n_items) + (size_t)n_items * sizeof(DevItem) + tc_batch_extra_bytes(n_items) +
+         256 + batch_prefix_bytes(n_items);
 }
 
 // Narrows a resolved hop to the token range [t_begin, t_end) of its caches: the caches start at row
@@ -806,36 +809,53 @@ int kvc_apply_batch(const kvc_item* items, int32_t n_items, const kvc_rope* rope
       if ((rc = window_item(&tab[i], items[i].t_begin, items[i].t_end)) != KVC_OK) return rc;
     }
   }
-  if (tl_path_force != KVC_PATH_GENERIC) {
-    const int trc = tc_apply_batch(tab, prefix, n_items, d, rope->pairing, status, workspace, staging, need, s);
-    if (trc == KVC_OK) {
-      tl_last_path = KVC_PATH_TC;
-      return KVC_OK;
-    }
-    if (trc != KVC_E_UNSUPPORTED || tl_path_force == KVC_PATH_TC) return trc;
+  // Items the tensor-core kernels serve go first in the table (items are independent: the order is free) and
+  // run there; the others (empty states, odd ranks, ...) run on the CUDA-core kernel in a launch of their own,
+  // so that one such request does not take the whole batch with it.
+  int n_tc = 0;
+  if (tl_path_force == KVC_PATH_TC) {
+    n_tc = n_items;                                   // all of them or KVC_E_UNSUPPORTED
+  } else if (tl_path_force != KVC_PATH_GENERIC) {
+    n_tc = (int)(std::stable_partition(tab, tab + n_items, [d](const DevItem& it) { return tc_batch_item_supported(it, d); }) - tab);
   }
+  const int n_rest = n_items - n_tc;
   const int tile = generic_apply_tile(d);
+  const size_t rest_off = need - batch_prefix_bytes(n_items);           // 8-byte aligned, behind everything else
+  int64_t* rest_prefix = reinterpret_cast<int64_t*>(reinterpret_cast<char*>(staging) + rest_off);
   int64_t total = 0;
-  for (int i = 0; i < n_items; ++i) {
-    prefix[i] = total;
-    tab[i].tiles_per_slab = (tab[i].src.T + tile - 1) / tile;
-    total += (int64_t)tab[i].L * tab[i].H * 2 * tab[i].tiles_per_slab;
+  for (int i = 0; i < n_rest; ++i) {
+    DevItem& it = tab[n_tc + i];
+    rest_prefix[i] = total;
+    it.tiles_per_slab = (it.src.T + tile - 1) / tile;
+    total += (int64_t)it.L * it.H * 2 * it.tiles_per_slab;
   }
-  prefix[n_items] = total;
-  if (total == 0) return KVC_OK;
+  rest_prefix[n_rest] = total;
   if (total > 0x7fffffffLL) return KVC_E_UNSUPPORTED;
-  const size_t bytes = batch_prefix_bytes(n_items) + (size_t)n_items * sizeof(DevItem);
-  if (cudaMemcpyAsync(workspace, staging, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return KVC_E_CUDA;
+  const size_t tab_off = batch_prefix_bytes(n_items);
+  if (n_tc > 0) {
+    // one copy of the whole table (the rest's items included) and up to two launches
+    const int trc = tc_apply_batch(tab, prefix, n_tc, n_items, d, rope->pairing, status, workspace, staging, need, s);
+    if (trc != KVC_OK) return trc;
+    tl_last_path = n_rest > 0 && total > 0 ? KVC_PATH_MIXED : KVC_PATH_TC;
+  } else if (total > 0) {
+    if (cudaMemcpyAsync(reinterpret_cast<char*>(workspace) + tab_off, tab, (size_t)n_items * sizeof(DevItem), cudaMemcpyHostToDevice, s) !=
+        cudaSuccess)
+      return KVC_E_CUDA;
+    tl_last_path = KVC_PATH_GENERIC;
+  }
+  if (total == 0) return KVC_OK;
+  if (cudaMemcpyAsync(reinterpret_cast<char*>(workspace) + rest_off, rest_prefix, (size_t)(n_rest + 1) * sizeof(int64_t),
+                      cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return KVC_E_CUDA;
   ApplyLaunch L;
   memset(&L, 0, sizeof(L));
-  L.tile_prefix = reinterpret_cast<const int64_t*>(workspace);
-  L.items = reinterpret_cast<const DevItem*>(reinterpret_cast<char*>(workspace) + batch_prefix_bytes(n_items));
-  L.n_items = n_items;
+  L.tile_prefix = reinterpret_cast<const int64_t*>(reinterpret_cast<char*>(workspace) + rest_off);
+  L.items = reinterpret_cast<const DevItem*>(reinterpret_cast<char*>(workspace) + tab_off) + n_tc;
+  L.n_items = n_rest;
   L.pairing = rope->pairing;
   L.total_tiles = total;
   L.status = status;
   if (launch_apply_generic(L, d, s) != cudaSuccess) return KVC_E_CUDA;
-  tl_last_path = KVC_PATH_GENERIC;
   return KVC_OK;
 }
 

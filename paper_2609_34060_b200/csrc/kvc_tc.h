@@ -14,9 +14,10 @@ int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, c
 int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, cudaStream_t s);
 int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* sn2, uint32_t* status, float* row_out,
                     int64_t t_pad, cudaStream_t s);
-int tc_apply_batch(DevItem* tab_host, int64_t* prefix_host, int n_items, int d, int pairing, uint32_t* status,
+int tc_apply_batch(DevItem* tab_host, int64_t* prefix_host, int n_items, int n_table, int d, int pairing, uint32_t* status,
                    void* workspace_dev, void* staging_host, size_t bytes, cudaStream_t s);
 size_t tc_batch_extra_bytes(int n_items);
+bool tc_batch_item_supported(const DevItem& item, int d);
 size_t tc_chain_workspace_bytes(int n_hops, int L, int H);
 int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_t* status, void* workspace, size_t ws_bytes,
                    cudaStream_t s);

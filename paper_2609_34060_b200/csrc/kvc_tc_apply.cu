@@ -1091,11 +1091,15 @@ size_t tc_batch_extra_bytes(int n_items) {
   return 256 + (size_t)n_items * sizeof(tc::ItemMaps) + 2 * 8 * (size_t)(tc::kMaxGrid + 1) + 8 * (size_t)(n_items + 1);
 }
 
+bool tc_batch_item_supported(const DevItem& item, int d) { return tc::encode_fn() && tc::item_supported(item, d); }
+
 // A ragged batch runs as up to two launches, one per rank class (r <= 32: one rank block, five base
 // slots; r > 32: two rank blocks, four base slots), so that small-rank requests do not run in the
 // configuration the large-rank ones need.  Items are independent, so the table may be reordered.
-int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int d, int pairing, uint32_t* status, void* workspace,
-                   void* staging, size_t bytes, cudaStream_t s) {
+// The table may hold more items than this call launches (n_table >= n_items: the caller runs the rest on
+// the CUDA-core kernel); the layout leaves room for all of them and the one copy carries them along.
+int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int n_table, int d, int pairing, uint32_t* status,
+                   void* workspace, void* staging, size_t bytes, cudaStream_t s) {
   if (!tc::encode_fn()) return KVC_E_UNSUPPORTED;
   for (int i = 0; i < n_items; ++i)
     if (!tc::item_supported(tab[i], d)) return KVC_E_UNSUPPORTED;
@@ -1107,7 +1111,7 @@ int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int d, int pairin
   // layout, identical in staging and workspace
   char* stg = reinterpret_cast<char*>(staging);
   const size_t tab_off = reinterpret_cast<char*>(tab) - stg;
-  const size_t maps_off = (tab_off + (size_t)n_items * sizeof(DevItem) + 255) & ~(size_t)255;
+  const size_t maps_off = (tab_off + (size_t)n_table * sizeof(DevItem) + 255) & ~(size_t)255;
   const size_t bounds_off = maps_off + (size_t)n_items * sizeof(tc::ItemMaps);
   const size_t prefix2_off = bounds_off + 2 * 8 * (size_t)(tc::kMaxGrid + 1);
   const size_t copy = prefix2_off + 8 * (size_t)(n_items + 1);

@@ -329,3 +329,50 @@ def test_apply_multi_random_shape(seed):
                 what = (cfg, ranks, n_covs, shift, which, l, h)
                 assert hp.tol_ratio(got[l, h], ref) <= 1.0, what
                 assert hp.ulp_mismatch_fraction(got[l, h], out) < 2e-2, what
+
+
+@pytest.mark.parametrize("seed", range(600, 608))
+def test_apply_batch_random_items(seed):
+    """kvc_apply_batch over three to nine items whose shapes are drawn independently (rank,
+    layers, heads, length, layout, coverage, shift differ from item to item; some states are empty): every
+    item equals its own kvc_apply bit for bit and meets the oracle."""
+    g = np.random.default_rng(44000 + seed)
+    n = int(g.integers(3, 10))
+    rope_theta = float(g.choice([10000.0, 500000.0]))
+    rope = kvc.Rope(rope_theta)
+    d_batch = int(g.choice([64, 128, 128]))
+    items, singles, oracles = [], [], []
+    for i in range(n):
+        cfg, n_cov, shift, _, bdt = _draw(1000 * seed + i)
+        cfg = cfg.scaled(theta=rope_theta, d=d_batch)         # the items of a launch share head_dim
+        src_cpu = hp.make_cache(cfg)
+        kind = int(g.integers(0, 5))
+        if kind == 0 or n_cov == 0:
+            st_cpu = kvc.State.empty()
+        else:
+            st_cpu = hp.make_state(cfg, 1 + i % 3, n_cov=n_cov, basis_dtype=bdt)
+        src, st = hp.to_dev(src_cpu, DEV), hp.state_to_dev(st_cpu, DEV)
+        dst = hp.empty_dst(src_cpu, cfg, DEV, fill=1.0)
+        one = hp.empty_dst(src_cpu, cfg, DEV, fill=1.0)
+        items.append(kvc.Item(src, dst, st, shift))
+        singles.append((src, st, shift, one))
+        oracles.append((cfg, src_cpu, st_cpu, shift))
+    nb = kvc.kvc_batch_workspace_bytes(len(items))
+    ws = torch.empty(nb, dtype=torch.uint8, device=DEV)
+    staging = torch.empty(nb, dtype=torch.uint8).pin_memory()
+    kvc.kvc_apply_batch(items, rope, ws, staging)
+    batch_path = kvc.kvc_last_path()
+    single_path = []
+    for (src, st, shift, one) in singles:
+        kvc.kvc_apply(src, st, shift, rope, one)
+        single_path.append(kvc.kvc_last_path())
+    torch.cuda.synchronize()
+    # every item runs on the kernel family it would get alone (a launch splits between the two), so the bits agree
+    assert batch_path == (kvc.KVC_PATH_MIXED if len(set(single_path)) == 2 else single_path[0])
+    for i, (it, (_, _, _, one), (cfg, src_cpu, st_cpu, shift)) in enumerate(zip(items, singles, oracles)):
+        assert torch.equal(it.dst.k, one.k) and torch.equal(it.dst.v, one.v), (cfg, shift)
+        osrc = hp.oracle_cache(src_cpu)
+        odst = osrc.empty_like(page_table=None if it.dst.page_table is None else it.dst.page_table.cpu().numpy())
+        odst, ref_k, ref_v = orc.apply(osrc, hp.oracle_state(st_cpu), shift, hp.inv_freq(cfg), dst=odst, want_ref=True)
+        assert hp.tol_ratio(hp.logical_bits(it.dst, "k"), ref_k) <= 1.0, (cfg, shift)
+        assert hp.tol_ratio(hp.logical_bits(it.dst, "v"), ref_v) <= 1.0, (cfg, shift)
