@@ -376,3 +376,49 @@ def test_apply_batch_random_items(seed):
         odst, ref_k, ref_v = orc.apply(osrc, hp.oracle_state(st_cpu), shift, hp.inv_freq(cfg), dst=odst, want_ref=True)
         assert hp.tol_ratio(hp.logical_bits(it.dst, "k"), ref_k) <= 1.0, (cfg, shift)
         assert hp.tol_ratio(hp.logical_bits(it.dst, "v"), ref_v) <= 1.0, (cfg, shift)
+
+
+@pytest.mark.parametrize("seed", range(700, 712))
+def test_grouped_apply_and_gate_random_shape(seed):
+    """Per-layer states (D = H d, Sec. 3.1) on drawn shapes through kvc_apply, and the gate distance (Eq. 9)
+    of the same source against drawn per-head anchors at a drawn comparison length."""
+    cfg, n_cov, shift, pairing, bdt = _draw(seed)
+    g = np.random.default_rng(33000 + seed)
+    n_cov = max(n_cov, 1)
+    one = cfg.scaled(H=1, d=cfg.H * cfg.d)
+    r = min(cfg.r, 64)
+    ck = wl.coefficients(cfg.L, 1, cfg.T, r, cfg.seed, 4, "cpu")[:, 0, :n_cov].contiguous()
+    cv = wl.coefficients(cfg.L, 1, cfg.T, r, cfg.seed, 5, "cpu")[:, 0, :n_cov].contiguous()
+    bk = wl.orthonormal_basis(cfg.L, 1, r, one.d, cfg.seed, 6, "cpu")[:, 0].contiguous().to(bdt)
+    bv = wl.orthonormal_basis(cfg.L, 1, r, one.d, cfg.seed, 7, "cpu")[:, 0].contiguous().to(bdt)
+    st = kvc.State(ck, cv, bk, bv, n_cov=n_cov, grouping=kvc.KVC_GROUP_LAYER)
+    src_cpu = hp.make_cache(cfg)
+    src = hp.to_dev(src_cpu, DEV)
+    dst = hp.empty_dst(src_cpu, cfg, DEV, fill=3.0)
+    kvc.kvc_apply(src, hp.state_to_dev(st, DEV), shift, kvc.Rope(cfg.theta, pairing), dst)
+    torch.cuda.synchronize()
+    f32 = lambda t: t.to(torch.float32).numpy()
+    ost = orc.ungroup_state(f32(ck), f32(cv), f32(bk), f32(bv), cfg.H, n_cov=n_cov)
+    osrc = hp.oracle_cache(src_cpu)
+    odst = osrc.empty_like(page_table=None if dst.page_table is None else dst.page_table.cpu().numpy())
+    odst, rk, rv = orc.apply(osrc, ost, shift, hp.inv_freq(cfg), dst=odst, pairing=_opair(pairing), want_ref=True)
+    gk, gv = hp.logical_bits(dst, "k"), hp.logical_bits(dst, "v")
+    assert hp.tol_ratio(gk, rk) <= 1.0 and hp.tol_ratio(gv, rv) <= 1.0, (cfg, n_cov, shift, pairing)
+    assert hp.ulp_mismatch_fraction(gk, hp.logical_bits(odst, "k")) < 1e-2
+    assert hp.ulp_mismatch_fraction(gv, hp.logical_bits(odst, "v")) < 1e-2
+    # ---- gate distance against two per-head anchors
+    anchors = [hp.make_state(cfg, hop=v + 1, basis_dtype=bdt if v else torch.float32) for v in range(2)]
+    k = int(g.integers(1, cfg.T + 1))
+    d2 = torch.full((2,), -1.0, dtype=torch.float64, device=DEV)
+    kvc.kvc_gate_distance(src, [hp.state_to_dev(a, DEV) for a in anchors], k, d2)
+    torch.cuda.synchronize()
+    ref = []
+    for a in anchors:
+        c = a.coeff_v.numpy().astype(np.float64)
+        b = a.basis_v.to(torch.float32).numpy().astype(np.float64)
+        v_src = [np.concatenate([orc.bf16_to_f64(osrc.get_bits("v", l, h)) for h in range(cfg.H)], axis=1) for l in range(cfg.L)]
+        v_anc = [np.concatenate([c[l, h] @ b[l, h] for h in range(cfg.H)], axis=1) for l in range(cfg.L)]
+        ref.append(orc.gate_distance(v_src, v_anc, k))
+    ref = np.array(ref)
+    got = np.sqrt(d2.cpu().numpy())
+    assert np.all(np.abs(got - ref) <= 1e-4 * ref + 1e-6), (cfg, k, got, ref)
