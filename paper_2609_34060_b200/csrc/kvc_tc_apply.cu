@@ -55,6 +55,8 @@ constexpr int kBasisBlkBytes = 128 * 128;         // 128 channels x (32 hi + 32 
 
 struct alignas(64) ItemMaps {
   CUtensorMap src_k, src_v, dst_k, dst_v, coeff_k, coeff_v;
+  int32_t lay_shift;   // 7: base tiles are [half][128 rows][64 ch]; a page shift < 7: page boxes (see encode_cache_page_box)
+  int32_t pad_[15];
 };
 
 struct ApplyTcLaunch {
@@ -82,6 +84,7 @@ struct Tile {
   const ItemMaps* mp;
   int item, slab, is_v, t0, l, h;
   int nb;            // rank blocks of 32 the item's state really has
+  int lay;           // layout of the base tile in shared memory (ItemMaps::lay_shift)
   bool first;        // first tile of its slab within this walk (the slab's operands must be staged)
   bool has_coeff;    // the tile holds covered rows of a live state
   bool uses_basis;   // its slab has a live state (basis staged for the slab)
@@ -98,7 +101,7 @@ struct TileWalker {
   bool first;
   const DevItem* it;
   const ItemMaps* mp;
-  int H, nb, cov;              // of the current item, read once: heads, rank blocks, covered rows of a live state (else 0)
+  int H, nb, cov, lay;         // of the current item, read once: heads, rank blocks, covered rows of a live state (else 0), tile layout
 
   __device__ void load_item() {
     it = p->items ? p->items + item : &p->one;
@@ -108,6 +111,7 @@ struct TileWalker {
     n_slab2 = it->L * H * (VONLY ? 1 : 2);
     nb = (it->st.r + 31) >> 5;
     cov = (it->st.r > 0 && it->st.n_cov > 0) ? it->st.n_cov : 0;
+    lay = mp->lay_shift;
   }
   __device__ void init(const ApplyTcLaunch* pp, int64_t begin, int64_t end_) {
     p = pp;
@@ -150,6 +154,7 @@ struct TileWalker {
     t.h = h;
     t.t0 = tt * kTileTok;
     t.nb = nb;
+    t.lay = lay;
     t.uses_basis = cov > 0;
     t.has_coeff = t.t0 < cov;
   }
@@ -274,6 +279,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
   // r = 64 configurations, bound by the team's instruction stream, gain 3 %).
   constexpr bool kPackedEpilogue = !(RB == 1 && NSTAGE == 5 && NSC == 2);
   constexpr bool REDUCE = MODE == 1 || MODE == 2;   // no stores
+  constexpr bool kPageBoxes = CV && MODE != 2;      // the host encodes page-box maps only for these kernels (uses_cv_kernel)
   constexpr int kStageBytes = kBaseBytes;
   constexpr int kCoeffSlotBytes = RB * kCoeffBlkBytes;
   constexpr int kBasisSlotBytes = RB * kBasisBlkBytes;
@@ -405,8 +411,12 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_ok * page * 256));
         __syncwarp();
         if (valid) {
-          tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, t.h, id, t.l);
-          tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, t.h, id, t.l);
+          if (kPageBoxes && t.lay < 7) {              // one box per page: both halves of this head's rows
+            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, t.h * page, 0, id, t.l);
+          } else {
+            tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, t.h, id, t.l);
+            tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, t.h, id, t.l);
+          }
         }
       }
       __syncwarp();
@@ -497,7 +507,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
       if constexpr (REDUCE) {
         // nothing to store: the slot goes straight back to the producer
       } else {
-        store_tile(it.dst, dmap, st_base, st_ptr, t.t0, t.l, t.h, t.is_v != 0, lane, pg, p.status);
+        store_tile(it.dst, dmap, st_base, st_ptr, t.t0, t.l, t.h, t.is_v != 0, lane, pg, p.status, kPageBoxes ? t.lay : 7);
       }
       tma_store_commit();
       tma_store_wait_read();
@@ -666,6 +676,12 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
       ok = mbar_wait(smem_u32(&ctrl->full[s]), (i / NSTAGE) & 1u, abort_flag);   // the base tile has landed
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      // row m of the tile in shared memory: offset of its first half, distance to its second
+      // (page boxes only in the converter-warp kernels, which serve the paged sources, and not in the row-distance
+      // mode, whose epilogue has no registers to spare: elsewhere the layout is a compile-time constant)
+      const int lay = kPageBoxes ? t.lay : 7;
+      const int row_off = ((m >> lay) << (lay + 8)) + ((m & ((1 << lay) - 1)) << 7);
+      const int half_stride = 128 << lay;
       const int tok = t.t0 + m;
       const bool in_range = tok < it.src.T;
       const bool covered = t.has_coeff && tok < it.st.n_cov;
@@ -699,8 +715,8 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
         // squared distance between the stored values and the anchor's reconstruction, this row and
         // this warp's 32 channels; fp32 within the tile, float64 across tiles
         if (in_range) {
-          const uint8_t* row0 = st_ptr + m * 128;
-          const uint8_t* row1 = row0 + kHalfBytes;
+          const uint8_t* row0 = st_ptr + row_off;
+          const uint8_t* row1 = row0 + half_stride;
           if (!covered) {                           // no reconstruction for this row: distance to zero
 #pragma unroll
             for (int k = 0; k < 16; ++k) a0[k] = a1[k] = 0.f;
@@ -730,8 +746,8 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
         // warp's 32 channels (pairs (c, c + 64) sit in one thread): keys are compared after rotating
         // the source by the item's table and the reconstruction by the second table
         if (in_range && covered) {
-          const uint8_t* row0 = st_ptr + m * 128;
-          const uint8_t* row1 = row0 + kHalfBytes;
+          const uint8_t* row0 = st_ptr + row_off;
+          const uint8_t* row1 = row0 + half_stride;
           float sa = 0.f;
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj) {
@@ -768,8 +784,8 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
         }
       } else if (work) {
         if (p.pairing == 0) {
-          uint8_t* row0 = st_ptr + m * 128;
-          uint8_t* row1 = row0 + kHalfBytes;
+          uint8_t* row0 = st_ptr + row_off;
+          uint8_t* row1 = row0 + half_stride;
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj) {
             const int j = 2 * cq + jj;                 // chunk of 8 channels inside each half
@@ -850,7 +866,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
           }
         } else {
           // interleaved pairs (2k, 2k+1): 32 consecutive channels 32cq .. 32cq+31
-          uint8_t* rowp = st_ptr + (cq >> 1) * kHalfBytes + m * 128;
+          uint8_t* rowp = st_ptr + (cq >> 1) * half_stride + row_off;
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
             const int j = 4 * (cq & 1) + jj;           // chunk inside the half
@@ -931,9 +947,21 @@ static bool item_supported(const DevItem& it, int d) {
   return true;
 }
 
-static bool build_maps(const DevItem& it, ItemMaps* mp) {
-  bool ok = encode_cache(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
-            encode_cache(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
+// Does a launch with these properties run on a converter-warp kernel (see launch())?  Only those read page boxes.
+static bool uses_cv_kernel(int max_r, bool paged, bool seg) { return !seg && (max_r > 32 || paged); }
+
+static bool build_maps(const DevItem& it, ItemMaps* mp, bool page_boxes) {
+  // packed paged pools on both sides with one page size: a box per page instead of one per page and half
+  mp->lay_shift = 7;
+  bool ok = false;
+  if (page_boxes && page_box_ok(it.src) && page_box_ok(it.dst) && it.src.page_shift == it.dst.page_shift) {
+    ok = encode_cache_page_box(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache_page_box(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
+         encode_cache_page_box(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache_page_box(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
+    if (ok) mp->lay_shift = it.src.page_shift;
+  }
+  if (!ok)
+    ok = encode_cache(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
+         encode_cache(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
   const int cslabs = it.st.grouped ? it.L : it.L * it.H;
   ok = ok && encode_coeff(&mp->coeff_k, it.st.coeff_k, it.st.r, it.st.n_cov, cslabs, it.st.coeff_rows) &&
        encode_coeff(&mp->coeff_v, it.st.coeff_v, it.st.r, it.st.n_cov, cslabs, it.st.coeff_rows);
@@ -1020,7 +1048,7 @@ int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, c
   memset(&L, 0, sizeof(L));
   L.one = item;
   L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
-  if (!tc::build_maps(L.one, &L.one_maps)) return KVC_E_CUDA;
+  if (!tc::build_maps(L.one, &L.one_maps, tc::uses_cv_kernel(item.st.r, item.src.page_table != nullptr, seg != nullptr))) return KVC_E_CUDA;
   L.n_items = 1;
   L.pairing = pairing;
   L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
@@ -1046,7 +1074,7 @@ int tc_gate_distance(const DevItem& item, int d, uint32_t* status, double* out, 
   memset(&L, 0, sizeof(L));
   L.one = item;
   L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
-  if (!tc::build_maps(L.one, &L.one_maps)) return KVC_E_CUDA;
+  if (!tc::build_maps(L.one, &L.one_maps, true)) return KVC_E_CUDA;
   L.n_items = 1;
   L.total_tiles = (int64_t)item.L * item.H * L.one.tiles_per_slab;      // value slabs only
   L.status = status;
@@ -1070,7 +1098,7 @@ int tc_row_distance(const DevItem& item, int d, const float* cs2, const float* s
   memset(&L, 0, sizeof(L));
   L.one = item;
   L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
-  if (!tc::build_maps(L.one, &L.one_maps)) return KVC_E_CUDA;
+  if (!tc::build_maps(L.one, &L.one_maps, false)) return KVC_E_CUDA;
   L.n_items = 1;
   L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
   L.status = status;
@@ -1117,9 +1145,11 @@ int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int n_table, int 
   const size_t copy = prefix2_off + 8 * (size_t)(n_items + 1);
   if (copy > bytes) return KVC_E_WORKSPACE;
   tc::ItemMaps* maps = reinterpret_cast<tc::ItemMaps*>(stg + maps_off);
+  // the class of r <= 32 runs on a converter-warp kernel (which reads page boxes) if its first item is paged
+  const bool class_cv[2] = {n_class[0] > 0 && tc::uses_cv_kernel(32, tab[0].src.page_table != nullptr, false), true};
   for (int i = 0; i < n_items; ++i) {
     tab[i].tiles_per_slab = (tab[i].src.T + tc::kTileTok - 1) / tc::kTileTok;
-    if (!tc::build_maps(tab[i], &maps[i])) return KVC_E_CUDA;
+    if (!tc::build_maps(tab[i], &maps[i], class_cv[i < n_class[0] ? 0 : 1])) return KVC_E_CUDA;
   }
 
   struct Plan {

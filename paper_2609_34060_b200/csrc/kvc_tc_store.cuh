@@ -45,8 +45,11 @@ __device__ __forceinline__ StorePages store_pages(const DevCache& dst, const Dev
 }
 
 // Whole warp.  st_base / st_ptr: the tile in shared memory (address for the TMA, pointer for plain reads).
+// lay: 7 = the tile is [half][128 rows][64 channels]; a page shift below 7 = the page-box layout, pages one
+// after the other, each [half][page rows][64 channels], stored with one instruction per page.
 __device__ __forceinline__ void store_tile(const DevCache& dst, const CUtensorMap* dmap, uint32_t st_base, const uint8_t* st_ptr,
-                                           int t0, int l, int h, bool is_v, int lane, const StorePages& g, uint32_t* status) {
+                                           int t0, int l, int h, bool is_v, int lane, const StorePages& g, uint32_t* status,
+                                           int lay = 7) {
   constexpr int kHalf = 128 * 128;                // bytes of one 64-channel half
   if (dst.page_table == nullptr) {
     if (lane == 0) {
@@ -62,20 +65,26 @@ __device__ __forceinline__ void store_tile(const DevCache& dst, const CUtensorMa
   if (lane < g.n_pages && !valid) atomicOr(status, KVC_FLAG_BAD_PAGE);
   const bool partial = last_partial && (g.first + lane) == last_pg;
   if (valid && g.src_ok && !partial) {
-    tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, h, g.id, l);
-    tma_store_5d(dmap, st_base + kHalf + lane * dpage * 128, 64, 0, h, g.id, l);
+    if (lay < 7) {
+      tma_store_5d(dmap, st_base + lane * dpage * 256, 0, h * dpage, 0, g.id, l);
+    } else {
+      tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, h, g.id, l);
+      tma_store_5d(dmap, st_base + kHalf + lane * dpage * 128, 64, 0, h, g.id, l);
+    }
   }
   const unsigned pm = __ballot_sync(0xffffffffu, valid && g.src_ok && partial);
   if (pm) {
+    // all rows lie in the one page whose (checked) id lane u holds: no table look-up per row
     const int u = __ffs(pm) - 1;
+    const int pid = __shfl_sync(0xffffffffu, g.id, u);
     const int rows = dst.T & dst.page_mask;
-    __nv_bfloat16* dbase = is_v ? dst.v : dst.k;
+    __nv_bfloat16* pbase = (is_v ? dst.v : dst.k) + (int64_t)l * dst.s_layer + (int64_t)pid * dst.s_page + (int64_t)h * dst.s_head;
+    const int half_stride = lay < 7 ? dpage * 128 : kHalf;
+    const uint8_t* pg_ptr = st_ptr + (lay < 7 ? u * dpage * 256 : u * dpage * 128);
     for (int c = lane; c < rows * 16; c += 32) {
-      const int row = u * dpage + (c >> 4), half = (c >> 3) & 1, j = c & 7;
-      __nv_bfloat16* drow = row_ptr(dst, dbase, l, h, t0 + row, status);
-      if (drow)
-        *reinterpret_cast<uint4*>(drow + half * 64 + j * 8) =
-            *reinterpret_cast<const uint4*>(st_ptr + half * kHalf + row * 128 + ((j ^ (row & 7)) << 4));
+      const int rp = c >> 4, half = (c >> 3) & 1, j = c & 7;      // pages hold a multiple of 8 rows: rp & 7 is the swizzle row
+      *reinterpret_cast<uint4*>(pbase + (int64_t)rp * dst.s_tok + half * 64 + j * 8) =
+          *reinterpret_cast<const uint4*>(pg_ptr + half * half_stride + rp * 128 + ((j ^ (rp & 7)) << 4));
     }
   }
 }
