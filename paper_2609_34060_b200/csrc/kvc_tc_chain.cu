@@ -50,7 +50,7 @@ struct Hop {
 struct ChainLaunch {
   DevCache src;
   int32_t L, H, tps, pairing;
-  int32_t n_hops, pad;
+  int32_t n_hops, lay;   // lay: 7, or the page shift when all caches are read and written as page boxes (PB kernel)
   int64_t total_tiles;
   uint32_t* status;
   alignas(16) Hop hop[kMaxHops];
@@ -69,6 +69,9 @@ struct Ctrl {
   int abort_flag;
 };
 
+// PB: agent 0's cache and every hop's destination are packed paged pools of one page size, moved with one TMA
+// box per page (encode_cache_page_box); the tiles then sit page by page in shared memory.
+template <bool PB>
 __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -168,8 +171,12 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_ok * page * 256));
         __syncwarp();
         if (valid) {
-          tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
-          tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
+          if (PB) {
+            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, h * page, 0, id, l);
+          } else {
+            tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
+            tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
+          }
         }
       }
       for (int a = 0; a < NH && alive; ++a) {
@@ -297,7 +304,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
         const CUtensorMap* dmap = is_v ? &p.dst_v[a] : &p.dst_k[a];
         const uint32_t st_base = outs + s * kBaseBytes;
         uint8_t* st_ptr = smem + kOutOff + s * kBaseBytes;
-        store_tile(dc, dmap, st_base, st_ptr, t0, l, h, is_v != 0, lane, pg, p.status);
+        store_tile(dc, dmap, st_base, st_ptr, t0, l, h, is_v != 0, lane, pg, p.status, PB ? p.lay : 7);
         tma_store_commit();
         tma_store_wait_read();
         __syncwarp();
@@ -340,6 +347,10 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
     const int cq = e16 >> 2;                       // channel quarter
     const int m = q * 32 + lane;                   // epilogue row = token of the tile
     const uint32_t sw = (uint32_t)(m & 7);
+    // row m of a tile in shared memory: offset of its first half, distance to its second
+    const int lay = PB ? p.lay : 7;
+    const int row_off = ((m >> lay) << (lay + 8)) + ((m & ((1 << lay) - 1)) << 7);
+    const int half_stride = 128 << lay;
     Walker w;
     w.init(p.tps, p.H, tile_begin, tile_end);
     uint32_t i = 0, step = 0;
@@ -384,10 +395,10 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
         mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
         // ---- 2. rotate, add, round: row m, this warp's channel quarter, from the input slot to the output slot
         if (p.pairing == 0) {
-          const uint8_t* irow0 = in_ptr + m * 128;
-          const uint8_t* irow1 = irow0 + kHalfBytes;
-          uint8_t* orow0 = out_ptr + m * 128;
-          uint8_t* orow1 = orow0 + kHalfBytes;
+          const uint8_t* irow0 = in_ptr + row_off;
+          const uint8_t* irow1 = irow0 + half_stride;
+          uint8_t* orow0 = out_ptr + row_off;
+          uint8_t* orow1 = orow0 + half_stride;
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj) {
             const int j = 2 * cq + jj;                 // chunk of 8 channels inside each half
@@ -430,8 +441,8 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
           }
         } else {
           // interleaved pairs (2k, 2k+1): 32 consecutive channels 32cq .. 32cq+31
-          const uint8_t* irow = in_ptr + (cq >> 1) * kHalfBytes + m * 128;
-          uint8_t* orow = out_ptr + (cq >> 1) * kHalfBytes + m * 128;
+          const uint8_t* irow = in_ptr + (cq >> 1) * half_stride + row_off;
+          uint8_t* orow = out_ptr + (cq >> 1) * half_stride + row_off;
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
             const int j = 4 * (cq & 1) + jj;           // chunk inside the half
@@ -552,7 +563,6 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
     P.basis_v[a] = it.st.basis_v;
     P.r[a] = hp.r;
     P.bf16[a] = it.st.basis_bf16;
-    if (!encode_cache(&C.dst_k[a], it.dst, it.dst.k, L, H) || !encode_cache(&C.dst_v[a], it.dst, it.dst.v, L, H)) return KVC_E_CUDA;
   }
   const size_t need = tc_chain_workspace_bytes(n_hops, L, H);
   if (!workspace || ws_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 127)) return KVC_E_WORKSPACE;
@@ -566,9 +576,23 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
   C.status = status;
   if (C.total_tiles == 0) return KVC_OK;
   __nv_bfloat16* ops = reinterpret_cast<__nv_bfloat16*>(workspace);
-  if (!encode_cache(&C.src_k, first.src, first.src.k, L, H) || !encode_cache(&C.src_v, first.src, first.src.v, L, H) ||
-      !encode_operand(&C.operand, ops, (int64_t)n_hops * 2 * 2 * L * H * 128))
-    return KVC_E_CUDA;
+  // page boxes when agent 0's cache and every destination are packed pools of one page size
+  bool pb = page_box_ok(first.src);
+  for (int a = 0; a < n_hops && pb; ++a) pb = page_box_ok(items[a].dst) && items[a].dst.page_shift == first.src.page_shift;
+  if (pb) {
+    pb = encode_cache_page_box(&C.src_k, first.src, first.src.k, L, H) && encode_cache_page_box(&C.src_v, first.src, first.src.v, L, H);
+    for (int a = 0; a < n_hops && pb; ++a)
+      pb = encode_cache_page_box(&C.dst_k[a], items[a].dst, items[a].dst.k, L, H) &&
+           encode_cache_page_box(&C.dst_v[a], items[a].dst, items[a].dst.v, L, H);
+  }
+  if (!pb) {
+    if (!encode_cache(&C.src_k, first.src, first.src.k, L, H) || !encode_cache(&C.src_v, first.src, first.src.v, L, H)) return KVC_E_CUDA;
+    for (int a = 0; a < n_hops; ++a)
+      if (!encode_cache(&C.dst_k[a], items[a].dst, items[a].dst.k, L, H) || !encode_cache(&C.dst_v[a], items[a].dst, items[a].dst.v, L, H))
+        return KVC_E_CUDA;
+  }
+  C.lay = pb ? first.src.page_shift : 7;
+  if (!encode_operand(&C.operand, ops, (int64_t)n_hops * 2 * 2 * L * H * 128)) return KVC_E_CUDA;
   P.slabs = L * H;
   P.out = ops;
   chain_prep_kernel<<<dim3((unsigned)(L * H), 4, (unsigned)n_hops), 256, 0, s>>>(P);
@@ -581,10 +605,15 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVC_E_CUDA;
+    if (cudaFuncSetAttribute(chain_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(chain_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return KVC_E_CUDA;
     once.mark(once_dev);
   }
-  chain_tc_kernel<<<grid, kThreadsCv, smem, s>>>(C);
+  if (pb)
+    chain_tc_kernel<true><<<grid, kThreadsCv, smem, s>>>(C);
+  else
+    chain_tc_kernel<false><<<grid, kThreadsCv, smem, s>>>(C);
   return cudaGetLastError() == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 

@@ -52,7 +52,7 @@ struct Block {                 // one rank block of one anchor
 struct MultiLaunch {
   DevCache src, dst;
   int32_t shift, L, H, tps;    // tps = tiles per slab
-  int32_t pairing, n_blocks, cov_max, pad;
+  int32_t pairing, n_blocks, cov_max, lay;   // lay: 7, or the page shift when both caches move as page boxes (PB kernel)
   int64_t total_tiles;
   uint32_t* status;
   alignas(16) float cs[kMaxHalfD];
@@ -91,7 +91,9 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0, p.grouped[e] != 0, p.H);
 }
 
-template <int NSTAGE, int NC, int NO>
+// PB: source and destination are packed paged pools of one page size, moved with one TMA box per page
+// (encode_cache_page_box); the tile then sits page by page in shared memory.
+template <int NSTAGE, int NC, int NO, bool PB>
 __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
   using Ctrl = tcm::Ctrl<NSTAGE, NC, NO>;
   extern __shared__ uint8_t smem_raw[];
@@ -187,8 +189,12 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_ok * page * 256));
         __syncwarp();
         if (valid) {
-          tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
-          tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
+          if (PB) {
+            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, h * page, 0, id, l);
+          } else {
+            tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
+            tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
+          }
         }
       }
       // the tile's rank blocks
@@ -309,7 +315,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
       const CUtensorMap* dmap = is_v ? &p.dst_v : &p.dst_k;
       const uint32_t st_base = stages + s * kBaseBytes;
       uint8_t* st_ptr = smem + s * kBaseBytes;
-      store_tile(p.dst, dmap, st_base, st_ptr, t0, l, h, is_v != 0, lane, pg, p.status);
+      store_tile(p.dst, dmap, st_base, st_ptr, t0, l, h, is_v != 0, lane, pg, p.status, PB ? p.lay : 7);
       tma_store_commit();
       tma_store_wait_read();
       __syncwarp();
@@ -370,6 +376,9 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
       if (!ok) break;
 
       // ---- 2. rotate, add, round: row m, this warp's channel quarter, in place
+      const int lay = PB ? p.lay : 7;                // row m in shared memory: offset of its first half, distance to its second
+      const int row_off = ((m >> lay) << (lay + 8)) + ((m & ((1 << lay) - 1)) << 7);
+      const int half_stride = 128 << lay;
       const int tok = t0 + m;
       const bool in_range = tok < p.src.T;
       const bool covered = has_coeff && tok < p.cov_max;
@@ -391,8 +400,8 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
       mbar_arrive(smem_u32(&ctrl->acc_empty[g]));
       if (work) {
         if (p.pairing == 0) {
-          uint8_t* row0 = st_ptr + m * 128;
-          uint8_t* row1 = row0 + kHalfBytes;
+          uint8_t* row0 = st_ptr + row_off;
+          uint8_t* row1 = row0 + half_stride;
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj) {
             const int j = 2 * cq + jj;                 // chunk of 8 channels inside each half
@@ -432,7 +441,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
           }
         } else {
           // interleaved pairs (2k, 2k+1): 32 consecutive channels 32cq .. 32cq+31
-          uint8_t* rowp = st_ptr + (cq >> 1) * kHalfBytes + m * 128;
+          uint8_t* rowp = st_ptr + (cq >> 1) * half_stride + row_off;
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
             const int j = 4 * (cq & 1) + jj;           // chunk inside the half
@@ -476,7 +485,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
   }
 }
 
-template <int NSTAGE, int NC, int NO>
+template <int NSTAGE, int NC, int NO, bool PB>
 static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s) {
   constexpr size_t smem = 1024 + (size_t)NSTAGE * kBaseBytes + (size_t)NC * (kCoeffBytes + kWeightBytes) +
                           (size_t)NO * kOperandBytes + sizeof(Ctrl<NSTAGE, NC, NO>);
@@ -484,11 +493,11 @@ static cudaError_t launch_multi_t(const MultiLaunch& M, int grid, cudaStream_t s
   static DeviceOnce once;
   int once_dev;
   if (once.pending(&once_dev)) {
-    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(apply_multi_tc_kernel<NSTAGE, NC, NO, PB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     once.mark(once_dev);
   }
-  apply_multi_tc_kernel<NSTAGE, NC, NO><<<grid, kThreadsCv, smem, s>>>(M);
+  apply_multi_tc_kernel<NSTAGE, NC, NO, PB><<<grid, kThreadsCv, smem, s>>>(M);
   return cudaGetLastError();
 }
 
@@ -563,10 +572,14 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   memcpy(M.sn, sn, sizeof(M.sn));
   if (M.total_tiles == 0) return KVC_OK;
   __nv_bfloat16* ops = reinterpret_cast<__nv_bfloat16*>(workspace);
-  if (!encode_cache(&M.src_k, src, src.k, L, H) || !encode_cache(&M.src_v, src, src.v, L, H) ||
-      !encode_cache(&M.dst_k, dst, dst.k, L, H) || !encode_cache(&M.dst_v, dst, dst.v, L, H) ||
-      !encode_operand(&M.operand, ops, (int64_t)nb * 2 * L * H * 128))
+  bool pb = page_box_ok(src) && page_box_ok(dst) && src.page_shift == dst.page_shift &&
+            encode_cache_page_box(&M.src_k, src, src.k, L, H) && encode_cache_page_box(&M.src_v, src, src.v, L, H) &&
+            encode_cache_page_box(&M.dst_k, dst, dst.k, L, H) && encode_cache_page_box(&M.dst_v, dst, dst.v, L, H);
+  if (!pb && (!encode_cache(&M.src_k, src, src.k, L, H) || !encode_cache(&M.src_v, src, src.v, L, H) ||
+              !encode_cache(&M.dst_k, dst, dst.k, L, H) || !encode_cache(&M.dst_v, dst, dst.v, L, H)))
     return KVC_E_CUDA;
+  M.lay = pb ? src.page_shift : 7;
+  if (!encode_operand(&M.operand, ops, (int64_t)nb * 2 * L * H * 128)) return KVC_E_CUDA;
   P.n_blocks = nb;
   P.slabs = L * H;
   P.H = H;
@@ -578,7 +591,7 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   const int grid = (int)(M.total_tiles < sms ? M.total_tiles : sms);
   // three base, four coefficient and three operand slots: of the depths tried with the converter warps this is the
   // fastest at three rank blocks per tile (622 us against 642 at 3/5/2 and 654 at 4/3/3) and level with 3/5/2 at six
-  const cudaError_t e = tcm::launch_multi_t<3, 4, 3>(M, grid, s);
+  const cudaError_t e = pb ? tcm::launch_multi_t<3, 4, 3, true>(M, grid, s) : tcm::launch_multi_t<3, 4, 3, false>(M, grid, s);
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
