@@ -163,9 +163,12 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
   const int64_t tile_end = n * (blockIdx.x + 1) / gridDim.x;
   const uint32_t n_my = (uint32_t)(tile_end - tile_begin);
 
+  // Paged caches are a TMA instruction per page and half: sixteen per cache and tile, more than one warp issues in
+  // the time HBM needs for the tile.  The source's pages then come from a second producer (the spare warp).
+  const bool split = p.has_src && (u.tgt.page_table != nullptr || u.src.page_table != nullptr);
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->full[s]), split ? 2 : 1);
       mbar_init(smem_u32(&ctrl->ready[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
@@ -188,27 +191,30 @@ __global__ void __launch_bounds__(kThreads, 1) project_tc_kernel(const __grid_co
   tc_fence_after();
   const uint32_t tmem_base = ctrl->tmem_base;
 
-  if (warp == 0) {
-    // =============================================================== TMA producer
+  if (warp == 0 || (warp == 2 && split)) {
+    // =============================================================== TMA producer(s)
+    const bool do_tgt = warp == 0, do_src = p.has_src && (split ? warp == 2 : true);
     uint32_t i = 0;
     for (; i < n_my; ++i) {
       const PTile t = decode(u, tile_begin + i);
       const int s = i % NS;
       const uint32_t use = i / NS;
+      // page ids before the wait: their latency hides behind it
+      int id_t = 0, id_s = 0;
+      bool ok_t = false, ok_s = false;
+      uint32_t bytes = 0;
+      if (do_tgt) bytes += tile_bytes(u.tgt, t.t0, lane, id_t, ok_t, u.status);
+      if (do_src) bytes += tile_bytes(u.src, t.t0, lane, id_s, ok_s, u.status);
       int ok = 1;
       if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       const uint32_t st_base = stages + s * kStageBytes;
       const uint32_t bar = smem_u32(&ctrl->full[s]);
-      int id_t, id_s = 0;
-      bool ok_t, ok_s = false;
-      uint32_t bytes = tile_bytes(u.tgt, t.t0, lane, id_t, ok_t, u.status);
-      if (p.has_src) bytes += tile_bytes(u.src, t.t0, lane, id_s, ok_s, u.status);
       if (lane == 0) mbar_expect_tx(bar, bytes);
       __syncwarp();
-      tile_issue(u.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
-      if (p.has_src) tile_issue(u.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
+      if (do_tgt) tile_issue(u.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
+      if (do_src) tile_issue(u.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
       __syncwarp();
     }
     if (lane == 0) {
@@ -627,9 +633,11 @@ __device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTab
   const int64_t unit_begin = nu * blockIdx.x / gridDim.x;
   const int64_t unit_end = nu * (blockIdx.x + 1) / gridDim.x;
 
+  // paged caches: the source's pages come from a second producer (the spare warp), as in the projection kernel
+  const bool split = p.has_src && (f.tgt.page_table != nullptr || f.src.page_table != nullptr);
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->full[s]), split ? 2 : 1);
       mbar_init(smem_u32(&ctrl->conv[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
@@ -651,8 +659,9 @@ __device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTab
   tc_fence_after();
   const uint32_t tmem_base = ctrl->tmem_base;
 
-  if (warp == 0) {
-    // =============================================================== TMA producer
+  if (warp == 0 || (warp == 2 && split)) {
+    // =============================================================== TMA producer(s)
+    const bool do_tgt = warp == 0, do_src = p.has_src && (split ? warp == 2 : true);
     uint32_t i = 0;
     bool dead = false;
     for (int64_t un = unit_begin; un < unit_end && !dead; ++un) {
@@ -666,6 +675,11 @@ __device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTab
         t.t0 = (g.tile0 + k) * kTileTok;
         const int s = i % NS;
         const uint32_t use = i / NS;
+        int id_t = 0, id_s = 0;                            // page ids before the wait
+        bool ok_t = false, ok_s = false;
+        uint32_t bytes = 0;
+        if (do_tgt) bytes += tile_bytes(f.tgt, t.t0, lane, id_t, ok_t, f.status);
+        if (do_src) bytes += tile_bytes(f.src, t.t0, lane, id_s, ok_s, f.status);
         int ok = 1;
         if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -675,14 +689,10 @@ __device__ __forceinline__ void gram_tc_body(const GramTcLaunch& p, const SegTab
         }
         const uint32_t st_base = stages + s * kStageBytes;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
-        int id_t, id_s = 0;
-        bool ok_t, ok_s = false;
-        uint32_t bytes = tile_bytes(f.tgt, t.t0, lane, id_t, ok_t, f.status);
-        if (p.has_src) bytes += tile_bytes(f.src, t.t0, lane, id_s, ok_s, f.status);
         if (lane == 0) mbar_expect_tx(bar, bytes);
         __syncwarp();
-        tile_issue(f.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
-        if (p.has_src) tile_issue(f.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
+        if (do_tgt) tile_issue(f.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
+        if (do_src) tile_issue(f.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
         __syncwarp();
       }
     }
@@ -926,9 +936,11 @@ __device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, c
   const int64_t unit_begin = nu * blockIdx.x / gridDim.x;
   const int64_t unit_end = nu * (blockIdx.x + 1) / gridDim.x;
 
+  // paged caches: the source's pages come from a second producer (the spare warp), as in the projection kernel
+  const bool split = p.has_src && (f.tgt.page_table != nullptr || f.src.page_table != nullptr);
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->full[s]), split ? 2 : 1);
       mbar_init(smem_u32(&ctrl->conv[s]), kTeamThreads);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
@@ -950,8 +962,9 @@ __device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, c
   tc_fence_after();
   const uint32_t tmem_base = ctrl->tmem_base;
 
-  if (warp == 0) {
-    // =============================================================== TMA producer
+  if (warp == 0 || (warp == 2 && split)) {
+    // =============================================================== TMA producer(s)
+    const bool do_tgt = warp == 0, do_src = p.has_src && (split ? warp == 2 : true);
     uint32_t i = 0;
     bool dead = false;
     for (int64_t un = unit_begin; un < unit_end && !dead; ++un) {
@@ -965,6 +978,11 @@ __device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, c
         t.t0 = (g.tile0 + k) * kTileTok;
         const int s = i % NS;
         const uint32_t use = i / NS;
+        int id_t = 0, id_s = 0;                            // page ids before the wait
+        bool ok_t = false, ok_s = false;
+        uint32_t bytes = 0;
+        if (do_tgt) bytes += tile_bytes(f.tgt, t.t0, lane, id_t, ok_t, f.status) + kZBytes;   // the coefficient tile always arrives whole (zero-filled past n_cov)
+        if (do_src) bytes += tile_bytes(f.src, t.t0, lane, id_s, ok_s, f.status);
         int ok = 1;
         if (lane == 0) ok = mbar_wait(smem_u32(&ctrl->empty[s]), (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -974,16 +992,11 @@ __device__ __forceinline__ void backproject_tc_body(const BackprojTcLaunch& p, c
         }
         const uint32_t st_base = stages + s * kStage;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
-        int id_t, id_s = 0;
-        bool ok_t, ok_s = false;
-        uint32_t bytes = tile_bytes(f.tgt, t.t0, lane, id_t, ok_t, f.status);
-        if (p.has_src) bytes += tile_bytes(f.src, t.t0, lane, id_s, ok_s, f.status);
-        bytes += kZBytes;                                     // the coefficient tile always arrives whole (zero-filled past n_cov)
         if (lane == 0) mbar_expect_tx(bar, bytes);
         __syncwarp();
-        tile_issue(f.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
-        if (p.has_src) tile_issue(f.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
-        if (lane == 0) tma_load_3d(st_base + kStageBytes, t.is_v ? &p.maps.coeff_v : &p.maps.coeff_k, bar, 0, t.t0, t.l);
+        if (do_tgt) tile_issue(f.tgt, t.is_v ? &p.maps.tgt_v : &p.maps.tgt_k, st_base, bar, t, lane, id_t, ok_t);
+        if (do_src) tile_issue(f.src, t.is_v ? &p.maps.src_v : &p.maps.src_k, st_base + kTileBytes, bar, t, lane, id_s, ok_s);
+        if (do_tgt && lane == 0) tma_load_3d(st_base + kStageBytes, t.is_v ? &p.maps.coeff_v : &p.maps.coeff_k, bar, 0, t.t0, t.l);
         __syncwarp();
       }
     }
