@@ -163,20 +163,27 @@ class Cache:
 
     contiguous: ``k``, ``v`` bf16 [L, H, T, d].
     paged:      ``k``, ``v`` bf16 pools [L, P, H, page, d], ``page_table`` int32
-                [ceil(T/page)], ``T`` the logical length.
+                [ceil(T/page)], ``T`` the logical length.  ``token_major=True``: the pools
+                are [L, P, page, H, d] (a page holds its tokens one after the other, each
+                with all heads), described to the library through the strides.
     """
 
     def __init__(self, k: torch.Tensor, v: torch.Tensor, T: Optional[int] = None,
-                 page_table: Optional[torch.Tensor] = None):
+                 page_table: Optional[torch.Tensor] = None, token_major: bool = False):
         assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16
         assert k.is_contiguous() and v.is_contiguous() and k.shape == v.shape
         self.k, self.v, self.page_table = k, v, page_table
+        self.token_major = bool(token_major)
         if page_table is None:
+            assert not token_major
             self.L, self.H, self.T, self.d = (int(x) for x in k.shape)
             self.page, self.P = 0, 0
         else:
             assert page_table.dtype == torch.int32 and page_table.is_contiguous() and T is not None
-            self.L, self.P, self.H, self.page, self.d = (int(x) for x in k.shape)
+            if token_major:
+                self.L, self.P, self.page, self.H, self.d = (int(x) for x in k.shape)
+            else:
+                self.L, self.P, self.H, self.page, self.d = (int(x) for x in k.shape)
             self.T = int(T)
 
     def struct(self) -> kvc_cache:
@@ -189,6 +196,10 @@ class Cache:
             s.layout = KVC_PAGED
             s.page_size, s.n_phys_pages = self.page, self.P
             s.page_table = self.page_table.data_ptr()
+            if self.token_major:
+                s.s_tok, s.s_head = self.H * self.d, self.d
+                s.s_page = self.page * self.H * self.d
+                s.s_layer = self.P * s.s_page
         return s
 
     def empty_like(self, page_table: Optional[torch.Tensor] = None, fill: Optional[float] = None) -> "Cache":
@@ -196,7 +207,7 @@ class Cache:
         if self.page_table is None:
             return Cache(mk(self.k), mk(self.v))
         return Cache(mk(self.k), mk(self.v), T=self.T,
-                     page_table=self.page_table if page_table is None else page_table)
+                     page_table=self.page_table if page_table is None else page_table, token_major=self.token_major)
 
     def nbytes(self) -> int:
         return self.k.numel() * 2 + self.v.numel() * 2

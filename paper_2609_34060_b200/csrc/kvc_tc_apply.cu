@@ -412,7 +412,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
         __syncwarp();
         if (valid) {
           if (kPageBoxes && t.lay < 7) {              // one box per page: both halves of this head's rows
-            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, t.h * page, 0, id, t.l);
+            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, 0, 0, t.h, id + t.l * it.src.n_phys);
           } else {
             tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, t.h, id, t.l);
             tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, t.h, id, t.l);
@@ -951,10 +951,11 @@ static bool item_supported(const DevItem& it, int d) {
 static bool uses_cv_kernel(int max_r, bool paged, bool seg) { return !seg && (max_r > 32 || paged); }
 
 static bool build_maps(const DevItem& it, ItemMaps* mp, bool page_boxes) {
-  // packed paged pools on both sides with one page size: a box per page instead of one per page and half
+  // paged pools on both sides with one page size (and all layers in one allocation): a box per page instead of one
+  // per page and half
   mp->lay_shift = 7;
   bool ok = false;
-  if (page_boxes && page_box_ok(it.src) && page_box_ok(it.dst) && it.src.page_shift == it.dst.page_shift) {
+  if (page_boxes && page_box_ok(it.src, it.L) && page_box_ok(it.dst, it.L) && it.src.page_shift == it.dst.page_shift) {
     ok = encode_cache_page_box(&mp->src_k, it.src, it.src.k, it.L, it.H) && encode_cache_page_box(&mp->src_v, it.src, it.src.v, it.L, it.H) &&
          encode_cache_page_box(&mp->dst_k, it.dst, it.dst.k, it.L, it.H) && encode_cache_page_box(&mp->dst_v, it.dst, it.dst.v, it.L, it.H);
     if (ok) mp->lay_shift = it.src.page_shift;

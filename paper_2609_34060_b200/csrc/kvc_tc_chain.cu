@@ -69,7 +69,7 @@ struct Ctrl {
   int abort_flag;
 };
 
-// PB: agent 0's cache and every hop's destination are packed paged pools of one page size, moved with one TMA
+// PB: agent 0's cache and every hop's destination are paged pools of one page size with all layers in one allocation, moved with one TMA
 // box per page (encode_cache_page_box); the tiles then sit page by page in shared memory.
 template <bool PB>
 __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_constant__ ChainLaunch p) {
@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
         __syncwarp();
         if (valid) {
           if (PB) {
-            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, h * page, 0, id, l);
+            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, 0, 0, h, id + l * p.src.n_phys);
           } else {
             tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
             tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
@@ -576,9 +576,9 @@ int tc_chain_fused(const DevItem* items, int n_hops, int d, int pairing, uint32_
   C.status = status;
   if (C.total_tiles == 0) return KVC_OK;
   __nv_bfloat16* ops = reinterpret_cast<__nv_bfloat16*>(workspace);
-  // page boxes when agent 0's cache and every destination are packed pools of one page size
-  bool pb = page_box_ok(first.src);
-  for (int a = 0; a < n_hops && pb; ++a) pb = page_box_ok(items[a].dst) && items[a].dst.page_shift == first.src.page_shift;
+  // page boxes when agent 0's cache and every destination are such pools of one page size
+  bool pb = page_box_ok(first.src, L);
+  for (int a = 0; a < n_hops && pb; ++a) pb = page_box_ok(items[a].dst, L) && items[a].dst.page_shift == first.src.page_shift;
   if (pb) {
     pb = encode_cache_page_box(&C.src_k, first.src, first.src.k, L, H) && encode_cache_page_box(&C.src_v, first.src, first.src.v, L, H);
     for (int a = 0; a < n_hops && pb; ++a)

@@ -43,21 +43,22 @@ inline bool encode_cache(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// A paged cache whose heads follow each other inside a page (s_head = page * s_tok, the packed pool layout) has a
-// second view in which ONE box holds a whole page of one head, both 64-channel halves: (channel-in-half, row of
-// the page's H * page rows, half, page, layer), box 64 x page x 2.  In shared memory the box lands as
-// [half][row][64 channels], 128B-swizzled: half the number of TMA instructions per tile of the per-half view.
-inline bool page_box_ok(const DevCache& c) {
+// A paged cache whose layers follow each other at a distance of n_phys pages (one pool allocation for all layers; or
+// a single layer) has a second view in which ONE box holds a whole page of one head, both 64-channel halves:
+// (channel-in-half, row of the page, half, head, page + layer * n_phys), box 64 x page x 2.  In shared memory the
+// box lands as [half][row][64 channels], 128B-swizzled: half the number of TMA instructions per tile of the per-half
+// view.  Whatever the order of heads and rows inside a page (head-major [H, page, d] or token-major [page, H, d]).
+inline bool page_box_ok(const DevCache& c, int L) {
   if (!c.page_table) return false;
   const int page = c.page_mask + 1;
-  return page < 128 && c.s_head == (int64_t)page * c.s_tok;
+  return page < 128 && (L == 1 || c.s_layer == (int64_t)c.n_phys * c.s_page);
 }
 inline bool encode_cache_page_box(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base, int L, int H) {
   EncodeTiledFn fn = encode_fn();
-  if (!fn || !page_box_ok(c)) return false;
+  if (!fn || !page_box_ok(c, L)) return false;
   const cuuint32_t page = (cuuint32_t)(c.page_mask + 1);
-  const cuuint64_t dims[5] = {64, (cuuint64_t)H * page, 2, (cuuint64_t)c.n_phys, (cuuint64_t)L};
-  const cuuint64_t strides[4] = {(cuuint64_t)c.s_tok * 2, 128, (cuuint64_t)c.s_page * 2, (cuuint64_t)c.s_layer * 2};
+  const cuuint64_t dims[5] = {64, page, 2, (cuuint64_t)H, (cuuint64_t)c.n_phys * (cuuint64_t)L};
+  const cuuint64_t strides[4] = {(cuuint64_t)c.s_tok * 2, 128, (cuuint64_t)c.s_head * 2, (cuuint64_t)c.s_page * 2};
   const cuuint32_t box[5] = {64, page, 2, 1, 1};
   const cuuint32_t es[5] = {1, 1, 1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,

@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256) multi_prep_kernel(const PrepLaunch p) {
   write_operand_block(out, basis, p.bf16[e] != 0, slab, r, col0, p.grouped[e] != 0, p.H);
 }
 
-// PB: source and destination are packed paged pools of one page size, moved with one TMA box per page
+// PB: source and destination are paged pools of one page size with all layers in one allocation, moved with one TMA box per page
 // (encode_cache_page_box); the tile then sits page by page in shared memory.
 template <int NSTAGE, int NC, int NO, bool PB>
 __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __grid_constant__ MultiLaunch p) {
@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) apply_multi_tc_kernel(const __g
         __syncwarp();
         if (valid) {
           if (PB) {
-            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, h * page, 0, id, l);
+            tma_load_5d(st_base + lane * page * 256, smap, bar, 0, 0, 0, h, id + l * p.src.n_phys);
           } else {
             tma_load_5d(st_base + lane * page * 128, smap, bar, 0, 0, h, id, l);
             tma_load_5d(st_base + kHalfBytes + lane * page * 128, smap, bar, 64, 0, h, id, l);
@@ -572,7 +572,7 @@ int tc_apply_multi(const DevCache& src, const DevCache& dst, int L, int H, int d
   memcpy(M.sn, sn, sizeof(M.sn));
   if (M.total_tiles == 0) return KVC_OK;
   __nv_bfloat16* ops = reinterpret_cast<__nv_bfloat16*>(workspace);
-  bool pb = page_box_ok(src) && page_box_ok(dst) && src.page_shift == dst.page_shift &&
+  bool pb = page_box_ok(src, L) && page_box_ok(dst, L) && src.page_shift == dst.page_shift &&
             encode_cache_page_box(&M.src_k, src, src.k, L, H) && encode_cache_page_box(&M.src_v, src, src.v, L, H) &&
             encode_cache_page_box(&M.dst_k, dst, dst.k, L, H) && encode_cache_page_box(&M.dst_v, dst, dst.v, L, H);
   if (!pb && (!encode_cache(&M.src_k, src, src.k, L, H) || !encode_cache(&M.src_v, src, src.v, L, H) ||

@@ -66,7 +66,7 @@ __device__ __forceinline__ void store_tile(const DevCache& dst, const CUtensorMa
   const bool partial = last_partial && (g.first + lane) == last_pg;
   if (valid && g.src_ok && !partial) {
     if (lay < 7) {
-      tma_store_5d(dmap, st_base + lane * dpage * 256, 0, h * dpage, 0, g.id, l);
+      tma_store_5d(dmap, st_base + lane * dpage * 256, 0, 0, 0, h, g.id + l * dst.n_phys);
     } else {
       tma_store_5d(dmap, st_base + lane * dpage * 128, 0, 0, h, g.id, l);
       tma_store_5d(dmap, st_base + kHalf + lane * dpage * 128, 64, 0, h, g.id, l);

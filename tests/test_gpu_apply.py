@@ -314,3 +314,48 @@ def test_apply_batch_ragged(path):
         odst, ref_k, ref_v = _oracle_hop(cfg, src_cpu, st_cpu, shift,
                                          None if dst.page_table is None else dst.page_table.cpu().numpy())
         _assert_parity(it.dst, ref_k, ref_v, odst)
+
+
+@pytest.mark.parametrize("cfg", [CFG_VLM_S, CFG_R64_S, CFG_VLM_S.scaled(name="vlm_page32", page=32, T=1999)], ids=lambda c: c.name)
+def test_token_major_pages_give_the_same_bits(cfg):
+    """A pool whose pages are [page, H, d] (each token with all its heads, the layout of the common paged
+    attention kernels) instead of [H, page, d]: the same call, described through the strides, gives the same bits
+    in the same logical places - one hop, the fused chain and the multi-anchor apply."""
+    rope = kvc.Rope(cfg.theta)
+    src_cpu = hp.make_cache(cfg)
+    tm = lambda t: t.permute(0, 1, 3, 2, 4).contiguous()
+    hm = lambda t: t.permute(0, 1, 3, 2, 4).contiguous()           # its own inverse: swaps the two middle axes back
+    src = hp.to_dev(src_cpu, DEV)
+    src_t = kvc.Cache(tm(src.k), tm(src.v), T=cfg.T, page_table=src.page_table, token_major=True)
+    pl = wl.prefix_lengths(cfg)[:3]
+    states = [hp.state_to_dev(hp.make_state(cfg, a), DEV) for a in (1, 2)]
+    def dsts(token_major, n):
+        out = []
+        for a in range(n):
+            d = hp.empty_dst(src_cpu, cfg, DEV, table_tag=70 + a, fill=4.0)
+            out.append(kvc.Cache(tm(d.k), tm(d.v), T=cfg.T, page_table=d.page_table, token_major=True) if token_major else d)
+        return out
+    # one hop
+    a, b = dsts(False, 1)[0], dsts(True, 1)[0]
+    kvc.kvc_apply(src, states[0], pl[1] - pl[0], rope, a)
+    kvc.kvc_apply(src_t, states[0], pl[1] - pl[0], rope, b)
+    torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+    assert torch.equal(hm(b.k), a.k) and torch.equal(hm(b.v), a.v)
+    # fused chain (two hops)
+    ca, cb = dsts(False, 2), dsts(True, 2)
+    ws = torch.empty(max(kvc.kvc_chain_workspace_bytes(src, 3), 128), dtype=torch.uint8, device=DEV)
+    kvc.kvc_chain_fused(src, pl, states, rope, ca, ws)
+    kvc.kvc_chain_fused(src_t, pl, states, rope, cb, ws)
+    torch.cuda.synchronize()
+    for x, y in zip(ca, cb):
+        assert torch.equal(hm(y.k), x.k) and torch.equal(hm(y.v), x.v)
+    assert torch.equal(ca[0].k, a.k)                          # and the chain's first hop is the single hop
+    # multi-anchor apply, unit weights
+    if cfg.r <= 64:
+        ma, mb = dsts(False, 1)[0], dsts(True, 1)[0]
+        wsm = torch.empty(max(kvc.kvc_multi_workspace_bytes(src, states), 128), dtype=torch.uint8, device=DEV)
+        kvc.kvc_apply_multi(src, states, None, None, 11, rope, ma, wsm)
+        kvc.kvc_apply_multi(src_t, states, None, None, 11, rope, mb, wsm)
+        torch.cuda.synchronize()
+        assert torch.equal(hm(mb.k), ma.k) and torch.equal(hm(mb.v), ma.v)
