@@ -366,3 +366,30 @@ def test_effective_rank_from_fit_eigenvalues():
             want = orc.effective_rank(np.linalg.eigvalsh(v.T @ v))
             assert abs(int(er[l, h, 1]) - want) <= 1 and want > 64      # a tie at the 90 % mark may fall either way
     assert kvc.kvc_effective_rank(src, ws, energy=1.0).max().item() <= d
+
+
+def test_token_major_pages_update_gives_the_same_bits():
+    """Pools whose pages are [page, H, d] instead of [H, page, d], described through the strides: projection and
+    FIT_FAST give the same coefficients, bases and eigenvalues bit for bit."""
+    cfg = CFG_VLM_S
+    src_cpu, tgt_cpu, osrc, otgt, true, shift = _edge(cfg)
+    src, tgt = hp.to_dev(src_cpu, DEV), hp.to_dev(tgt_cpu, DEV)
+    tm = lambda t: t.permute(0, 1, 3, 2, 4).contiguous()
+    as_tm = lambda c: kvc.Cache(tm(c.k), tm(c.v), T=cfg.T, page_table=c.page_table, token_major=True)
+    src_t, tgt_t = as_tm(src), as_tm(tgt)
+    L, H, T, d, r = cfg.L, cfg.H, cfg.T, cfg.d, cfg.r
+    given = hp.make_state(cfg, 3)
+    rope = kvc.Rope(cfg.theta)
+    for mode in (kvc.KVC_PROJECT, kvc.KVC_FIT_FAST):
+        outs = []
+        for s_, t_ in ((src, tgt), (src_t, tgt_t)):
+            st = kvc.State(torch.zeros(L, H, T, r, device=DEV), torch.zeros(L, H, T, r, device=DEV),
+                           given.basis_k.to(DEV).clone(), given.basis_v.to(DEV).clone())
+            ws = torch.zeros(max(kvc.kvc_workspace_bytes(t_, st, mode), 256), dtype=torch.uint8, device=DEV)
+            kvc.kvc_state_update(s_, t_, shift, rope, st, mode, workspace=ws)
+            torch.cuda.synchronize()
+            assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+            outs.append(st)
+        a, b = outs
+        assert torch.equal(a.coeff_k, b.coeff_k) and torch.equal(a.coeff_v, b.coeff_v)
+        assert torch.equal(a.basis_k, b.basis_k) and torch.equal(a.basis_v, b.basis_v)
