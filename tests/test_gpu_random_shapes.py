@@ -4,7 +4,11 @@ The other GPU tests pick their shapes by hand around known tile and page boundar
 draws them (head_dim, rank, layers, heads, length, coverage, page size, shift, RoPE pairing,
 basis dtype), so that combinations nobody thought of are compared element by element too.
 Whatever kernel family the library chooses for a shape is the one that is checked.
+The environment variable KVC_SWEEP_OFFSET (an integer, default 0) moves every draw to another part of
+the seed space: the committed sweep is one sample, a campaign runs it at several offsets.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -18,6 +22,7 @@ import helpers as hp
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 BASE = wl.CONFIGS["llama8b_8k"]
+SWEEP_OFFSET = int(os.environ.get("KVC_SWEEP_OFFSET", "0"))
 
 
 @pytest.fixture(autouse=True)
@@ -29,7 +34,7 @@ def _clean_status():
 
 
 def _draw(seed):
-    g = np.random.default_rng(77000 + seed)
+    g = np.random.default_rng(77000 + seed + 100000 * SWEEP_OFFSET)
     d = int(g.choice([64, 128, 128, 128]))
     r = int(g.choice([1, 3, 4, 8, 12, 16, 17, 24, 32, 33, 40, 48, 64]))
     T = int(g.choice([g.integers(1, 140), g.integers(140, 900)]))
