@@ -324,14 +324,16 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ev = {}
+    evs = []                                # per block: the phase events of its steps
     blocks, per_step = [], []
     for rep in range(repeats):
         t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev = {}
+        evs.append(ev)
         t_begin.record()
         step_marks = []
         for _ in range(args.steps):
-            sc.run_step(W, ev if rep == 0 else None)
+            sc.run_step(W, ev)
             m = torch.cuda.Event(enable_timing=True)
             m.record()
             step_marks.append(m)
@@ -343,7 +345,9 @@ def main():
         block_ms.append(dist_util.max_over_ranks(t_begin.elapsed_time(t_end), dev))
         per_step += [a.elapsed_time(b) for a, b in zip([t_begin] + step_marks[:-1], step_marks)]
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = sorted(block_ms)[len(block_ms) // 2]
+    med = sorted(range(len(block_ms)), key=lambda b: block_ms[b])[len(block_ms) // 2]
+    ms_total = block_ms[med]
+    ev = evs[med]                           # the kernel times reported are those of the same, median, block
     chain_ms = sum(b.elapsed_time(e) for b, e in zip(ev.get("chain_begin", []), ev.get("chain_end", []))) / args.steps
     upd_ms = sum(b.elapsed_time(e) for b, e in zip(ev.get("update_begin", []), ev.get("update_end", []))) / args.steps
     chain_ms, upd_ms = max(chain_ms, 1e-9), max(upd_ms, 1e-9)
