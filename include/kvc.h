@@ -304,9 +304,10 @@ size_t kvc_chain_update_edge_stride(const kvc_cache *tgt, const kvc_state *st, i
  * kernel where kvc_apply does (every row picks its segment's table in the epilogue), and so do the passes
  * of kvc_state_update_segmented over the caches where kvc_state_update's do: the Gram pass picks every
  * row's table while it forms the deviation, the projection runs as one launch per segment over that
- * segment's token window (it rotates the basis, not the tokens).  A paged cache whose segment boundaries
- * do not fall on page boundaries has its projection served by the CUDA-core kernel (KVC_PATH_TC forced:
- * KVC_E_UNSUPPORTED).  Everything else is as in kvc_apply / kvc_state_update, including layer-grouped
+ * segment's token window (it rotates the basis, not the tokens; on a paged cache a window starts with its
+ * page, and the segments run from the last to the first so that every row is last written by its own).
+ * Only a layer-grouped state on a paged cache whose segment boundaries are off the page grid has its
+ * projection served by the CUDA-core kernel (KVC_PATH_TC forced: KVC_E_UNSUPPORTED).  Everything else is as in kvc_apply / kvc_state_update, including layer-grouped
  * states (whose back-projection pass picks the rows' tables like the Gram pass) and the FIT modes.
  */
 #define KVC_MAX_SEGMENTS   16

@@ -501,19 +501,27 @@ static int project_edge(const UpdatePlan& P, uint32_t* status, cudaStream_t s, c
   if (tl_path_force != KVC_PATH_GENERIC && P.seg) {
     // A context of several segments: the projection is independent token by token, so every segment is a
     // launch of its own over its token window, with its own shift (the basis is rotated, not the tokens).
-    // Windows of a paged cache must start on a page boundary; otherwise the CUDA-core kernel serves the call.
+    // A window of a paged cache starts on a page boundary: where a segment does not, its window starts at the
+    // page's first row and the launch also writes the rows in front of the segment, with the wrong shift.  The
+    // segments are therefore launched from the last to the first, each window ending exactly with its segment:
+    // the rows in front of a segment are written again, correctly, by the launches of the segments they belong
+    // to.  (A layer-grouped state ADDS every head's share to its rows, so rows written twice would be wrong:
+    // there the CUDA-core kernel serves boundaries off the page grid.)
     const SegTable& sg = *P.seg;
+    int align = 1;
+    for (const DevCache* c : {&U.src, &U.tgt})
+      if (c->k && c->page_table && c->page_mask + 1 > align) align = c->page_mask + 1;
     bool windows_ok = true;
-    for (int j = 1; j < sg.n; ++j)
-      for (const DevCache* c : {&U.src, &U.tgt})
-        if (c->k && c->page_table && (sg.t_begin[j] & c->page_mask)) windows_ok = false;
+    if (U.grouped)
+      for (int j = 1; j < sg.n; ++j)
+        if (sg.t_begin[j] & (align - 1)) windows_ok = false;
     int trc = windows_ok ? KVC_OK : KVC_E_UNSUPPORTED;
     bool launched = false;
-    for (int j = 0; j < sg.n && trc == KVC_OK; ++j) {
-      const int tb = sg.t_begin[j];
+    for (int j = sg.n - 1; j >= 0 && trc == KVC_OK; --j) {
+      const int tb = sg.t_begin[j] & ~(align - 1);             // window start: the segment's, or its page's
       const int nxt = j + 1 < sg.n ? sg.t_begin[j + 1] : st->n_cov;
       const int te = nxt < st->n_cov ? nxt : st->n_cov;      // the segment's covered rows
-      if (te <= tb) continue;
+      if (te <= sg.t_begin[j]) continue;
       UpdateLaunch W = U;
       for (DevCache* c : {&W.src, &W.tgt}) {
         if (!c->k) continue;

@@ -20,7 +20,10 @@ DEV = "cuda:0"
 CFG_C = wl.CONFIGS["llama8b_8k"].scaled(name="8b_small", L=2, H=2, T=700)
 CFG_P = wl.CONFIGS["vlm_16k"].scaled(name="vlm_small", L=1, H=2, T=1003, image_spans=())
 CFG_T = wl.CONFIGS["tiny"]
-SEGS = {"8b_small": ([0, 133, 390], [37, 0, -211]), "vlm_small": ([0, 21, 530], [-5, 512, 64]), "tiny": ([0, 7, 100], [3, -2, 0])}
+SEGS = {"8b_small": ([0, 133, 390], [37, 0, -211]), "vlm_small": ([0, 21, 530], [-5, 512, 64]), "tiny": ([0, 7, 100], [3, -2, 0]),
+        # several segments inside one 16-token page, and one that ends inside the page the next begins in
+        "vlm_short_segments": ([0, 5, 9, 40, 300], [3, -7, 0, 25, -100])}
+CFG_PS = CFG_P.scaled(name="vlm_short_segments", T=403)
 COORDS = [kvc.KVC_COORDS_TARGET, kvc.KVC_COORDS_SOURCE]
 
 
@@ -64,8 +67,8 @@ def test_apply_segmented(cfg, coords, path):
 
 
 @pytest.mark.parametrize("coords", COORDS, ids=["target", "source"])
-@pytest.mark.parametrize("cfg,on_pages", [(CFG_C, False), (CFG_P, False), (CFG_P, True)],
-                         ids=["8b_small", "vlm_small", "vlm_small-page-aligned"])
+@pytest.mark.parametrize("cfg,on_pages", [(CFG_C, False), (CFG_P, False), (CFG_P, True), (CFG_PS, False)],
+                         ids=["8b_small", "vlm_small", "vlm_small-page-aligned", "vlm_short_segments"])
 def test_project_and_fit_segmented(cfg, on_pages, coords):
     """PROJECT: coefficients of the per-token-shift deviation in a given basis.  FIT: the deviation is built
     exactly rank r in the chosen coordinates, so the fitted state reproduces the oracle's subspace and the
@@ -100,9 +103,9 @@ def test_project_and_fit_segmented(cfg, on_pages, coords):
                    given.basis_k.to(DEV), given.basis_v.to(DEV))
     kvc.kvc_state_update_segmented(src, tgt, segs, rope, st, kvc.KVC_PROJECT)
     torch.cuda.synchronize()
-    # contiguous caches: a tensor-core launch per segment window; the paged case has boundaries off the page grid
-    # and is served by the CUDA-core kernel
-    assert kvc.kvc_last_path() == (kvc.KVC_PATH_GENERIC if (cfg.paged and not on_pages) else kvc.KVC_PATH_TC)
+    # a tensor-core launch per segment window, also where the boundaries of a paged cache are off the page grid
+    # (the windows then start at the page's first row and the segments are launched from the last to the first)
+    assert kvc.kvc_last_path() == (kvc.KVC_PATH_TC if cfg.d == 128 else kvc.KVC_PATH_GENERIC)
     deltas = {}
     for which, cf, bs in (("k", st.coeff_k, given.basis_k), ("v", st.coeff_v, given.basis_v)):
         for l in range(L):
