@@ -947,8 +947,9 @@ static bool item_supported(const DevItem& it, int d) {
   return true;
 }
 
-// Does a launch with these properties run on a converter-warp kernel (see launch())?  Only those read page boxes.
-static bool uses_cv_kernel(int max_r, bool paged, bool seg) { return !seg && (max_r > 32 || paged); }
+// Does a launch run on a converter-warp kernel (see launch())?  Only those read page boxes: all but the kernels
+// with a segment table.
+static bool uses_cv_kernel(bool seg) { return !seg; }
 
 static bool build_maps(const DevItem& it, ItemMaps* mp, bool page_boxes) {
   // paged pools on both sides with one page size (and all layers in one allocation): a box per page instead of one
@@ -1013,11 +1014,12 @@ static int launch(const ApplyTcLaunch& L, int max_r, bool paged, cudaStream_t s,
     cudaError_t es = (max_r > 32) ? launch_seg_t<2, 4, 2>(L, *seg, grid, s) : launch_seg_t<1, 5, 3>(L, *seg, grid, s);
     return es == cudaSuccess ? KVC_OK : KVC_E_CUDA;
   }
-  // converter warps (CV) where the team's instruction stream, not HBM, set the pace: paged sources and
-  // two rank blocks; a contiguous source with one rank block streams at the copy bandwidth without them
-  // and measured 4 % slower with them
+  // converter warps (CV) everywhere: with the SM clock where the power cap holds it in a long run (1.7-1.8 GHz)
+  // the team's instruction stream sets the pace, for a contiguous source with one rank block too (0.975 against
+  // 0.94 of the copy bandwidth; only in a short run at 1.96 GHz is the kernel without them ahead, 0.99 against
+  // 0.94).  A contiguous source keeps two coefficient slots (three: 0.85).
   cudaError_t e = (max_r > 32) ? launch_t<2, 4, 2, true>(L, grid, s)
-                               : (paged ? launch_t<1, 5, 3, true>(L, grid, s) : launch_t<1, 5, 2>(L, grid, s));
+                               : (paged ? launch_t<1, 5, 3, true>(L, grid, s) : launch_t<1, 5, 2, true>(L, grid, s));
   return e == cudaSuccess ? KVC_OK : KVC_E_CUDA;
 }
 
@@ -1049,7 +1051,7 @@ int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, c
   memset(&L, 0, sizeof(L));
   L.one = item;
   L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
-  if (!tc::build_maps(L.one, &L.one_maps, tc::uses_cv_kernel(item.st.r, item.src.page_table != nullptr, seg != nullptr))) return KVC_E_CUDA;
+  if (!tc::build_maps(L.one, &L.one_maps, tc::uses_cv_kernel(seg != nullptr))) return KVC_E_CUDA;
   L.n_items = 1;
   L.pairing = pairing;
   L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
@@ -1146,11 +1148,9 @@ int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int n_table, int 
   const size_t copy = prefix2_off + 8 * (size_t)(n_items + 1);
   if (copy > bytes) return KVC_E_WORKSPACE;
   tc::ItemMaps* maps = reinterpret_cast<tc::ItemMaps*>(stg + maps_off);
-  // the class of r <= 32 runs on a converter-warp kernel (which reads page boxes) if its first item is paged
-  const bool class_cv[2] = {n_class[0] > 0 && tc::uses_cv_kernel(32, tab[0].src.page_table != nullptr, false), true};
   for (int i = 0; i < n_items; ++i) {
     tab[i].tiles_per_slab = (tab[i].src.T + tc::kTileTok - 1) / tc::kTileTok;
-    if (!tc::build_maps(tab[i], &maps[i], class_cv[i < n_class[0] ? 0 : 1])) return KVC_E_CUDA;
+    if (!tc::build_maps(tab[i], &maps[i], tc::uses_cv_kernel(false))) return KVC_E_CUDA;
   }
 
   struct Plan {
