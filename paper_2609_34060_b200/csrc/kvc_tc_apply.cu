@@ -274,10 +274,6 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
   static_assert(MODE != 2 || CV, "the row-distance mode relies on the converter warps (rotated key basis)");
   constexpr bool GATE = MODE == 1;                // walks value slabs only
   constexpr bool SEG = MODE == 3;
-  // The epilogue works on packed float32 pairs except in the configuration of a contiguous source with
-  // r <= 32, which runs at the HBM roof either way and measured 0.7 % slower with them (the paged and
-  // r = 64 configurations, bound by the team's instruction stream, gain 3 %).
-  constexpr bool kPackedEpilogue = !(RB == 1 && NSTAGE == 5 && NSC == 2);
   constexpr bool REDUCE = MODE == 1 || MODE == 2;   // no stores
   constexpr bool kPageBoxes = CV && MODE != 2;      // the host encodes page-box maps only for these kernels (uses_cv_kernel)
   constexpr int kStageBytes = kBaseBytes;
@@ -791,78 +787,44 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
             const int j = 2 * cq + jj;                 // chunk of 8 channels inside each half
             uint4* p0 = reinterpret_cast<uint4*>(row0 + ((j ^ sw) << 4));
             uint4* p1 = reinterpret_cast<uint4*>(row1 + ((j ^ sw) << 4));
-            if constexpr (kPackedEpilogue) {
-              // packed float32 pairs: word w of a 16-byte chunk holds channels 2w, 2w + 1
-              const uint4 ua = *p0, ub = *p1;
-              const uint32_t wa[4] = {ua.x, ua.y, ua.z, ua.w}, wb[4] = {ub.x, ub.y, ub.z, ub.w};
-              f32x2 xa[4], xb[4];
-  #pragma unroll
-              for (int z = 0; z < 4; ++z) {
-                xa[z] = f2_from_bf16x2(wa[z]);
-                xb[z] = f2_from_bf16x2(wb[z]);
-              }
-              if (SEG && covered && at_source) {       // the correction lives at the source's positions: add, then rotate
-  #pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  xa[z] = f2_add(xa[z], f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
-                  xb[z] = f2_add(xb[z], f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]));
-                }
-              }
-              if (rotate) {
-                const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
-                const float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
-                const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
-                const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
-                const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
-  #pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  const f32x2 u = xa[z], v = xb[z];
-                  xa[z] = f2_fma(u, cs[z], f2_mul(v, nsn[z]));           // u cos - v sin
-                  xb[z] = f2_fma(u, sn[z], f2_mul(v, cs[z]));            // u sin + v cos
-                }
-              }
-              if (covered && !(SEG && at_source)) {
-  #pragma unroll
-                for (int z = 0; z < 4; ++z) {
-                  xa[z] = f2_add(xa[z], f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
-                  xb[z] = f2_add(xb[z], f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]));
-                }
-              }
-              *p0 = make_uint4(f2_to_bf16x2(xa[0]), f2_to_bf16x2(xa[1]), f2_to_bf16x2(xa[2]), f2_to_bf16x2(xa[3]));
-              *p1 = make_uint4(f2_to_bf16x2(xb[0]), f2_to_bf16x2(xb[1]), f2_to_bf16x2(xb[2]), f2_to_bf16x2(xb[3]));
-            } else {
-              float x[16];
-              unpack8(*p0, x);
-              unpack8(*p1, x + 8);
-              if (SEG && covered && at_source) {
-  #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  x[k] += a0[8 * jj + k];
-                  x[8 + k] += a1[8 * jj + k];
-                }
-              }
-              if (rotate) {
-                const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
-                const float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
-                const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-                const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-  #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  const float u = x[k], v = x[8 + k];
-                  x[k] = u * cs[k] - v * sn[k];
-                  x[8 + k] = u * sn[k] + v * cs[k];
-                }
-              }
-              if (covered && !(SEG && at_source)) {
-  #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  x[k] += a0[8 * jj + k];
-                  x[8 + k] += a1[8 * jj + k];
-                }
-              }
-              *p0 = pack8(x);
-              *p1 = pack8(x + 8);
+            // packed float32 pairs: word w of a 16-byte chunk holds channels 2w, 2w + 1
+            const uint4 ua = *p0, ub = *p1;
+            const uint32_t wa[4] = {ua.x, ua.y, ua.z, ua.w}, wb[4] = {ub.x, ub.y, ub.z, ub.w};
+            f32x2 xa[4], xb[4];
+#pragma unroll
+            for (int z = 0; z < 4; ++z) {
+              xa[z] = f2_from_bf16x2(wa[z]);
+              xb[z] = f2_from_bf16x2(wb[z]);
             }
+            if (SEG && covered && at_source) {       // the correction lives at the source's positions: add, then rotate
+#pragma unroll
+              for (int z = 0; z < 4; ++z) {
+                xa[z] = f2_add(xa[z], f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
+                xb[z] = f2_add(xb[z], f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]));
+              }
+            }
+            if (rotate) {
+              const float4 c0 = *reinterpret_cast<const float4*>(csp + 8 * j), c1 = *reinterpret_cast<const float4*>(csp + 8 * j + 4);
+              const float4 s0 = *reinterpret_cast<const float4*>(snp + 8 * j), s1 = *reinterpret_cast<const float4*>(snp + 8 * j + 4);
+              const f32x2 cs[4] = {f2_pack(c0.x, c0.y), f2_pack(c0.z, c0.w), f2_pack(c1.x, c1.y), f2_pack(c1.z, c1.w)};
+              const f32x2 sn[4] = {f2_pack(s0.x, s0.y), f2_pack(s0.z, s0.w), f2_pack(s1.x, s1.y), f2_pack(s1.z, s1.w)};
+              const f32x2 nsn[4] = {f2_pack(-s0.x, -s0.y), f2_pack(-s0.z, -s0.w), f2_pack(-s1.x, -s1.y), f2_pack(-s1.z, -s1.w)};
+#pragma unroll
+              for (int z = 0; z < 4; ++z) {
+                const f32x2 u = xa[z], v = xb[z];
+                xa[z] = f2_fma(u, cs[z], f2_mul(v, nsn[z]));           // u cos - v sin
+                xb[z] = f2_fma(u, sn[z], f2_mul(v, cs[z]));            // u sin + v cos
+              }
+            }
+            if (covered && !(SEG && at_source)) {
+#pragma unroll
+              for (int z = 0; z < 4; ++z) {
+                xa[z] = f2_add(xa[z], f2_pack(a0[8 * jj + 2 * z], a0[8 * jj + 2 * z + 1]));
+                xb[z] = f2_add(xb[z], f2_pack(a1[8 * jj + 2 * z], a1[8 * jj + 2 * z + 1]));
+              }
+            }
+            *p0 = make_uint4(f2_to_bf16x2(xa[0]), f2_to_bf16x2(xa[1]), f2_to_bf16x2(xa[2]), f2_to_bf16x2(xa[3]));
+            *p1 = make_uint4(f2_to_bf16x2(xb[0]), f2_to_bf16x2(xb[1]), f2_to_bf16x2(xb[2]), f2_to_bf16x2(xb[3]));
           }
         } else {
           // interleaved pairs (2k, 2k+1): 32 consecutive channels 32cq .. 32cq+31
