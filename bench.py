@@ -40,7 +40,7 @@ HBM_FALLBACK_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one apply launch on the 8K workload, from an ncu
 # capture of the same kernel at L = 16 (811.95 MB read + 493.36 MB written per launch), scaled by 2
 # to L = 32 (traffic is proportional to the token-slabs processed).  None for other workloads.
-APPLY_TRAFFIC_BYTES_LLAMA8B_8K = 2 * (811_950_000 + 493_360_000)
+APPLY_TRAFFIC_BYTES_LLAMA8B_8K = 2 * (811_940_000 + 492_040_000)
 APPLY_TRAFFIC_SOURCE = "ncu dram__bytes_read.sum + dram__bytes_write.sum of apply_tc_kernel at L=16, scaled x2 to L=32 (not from this run)"
 HBM_NOMINAL_GBS = 8000.0
 
