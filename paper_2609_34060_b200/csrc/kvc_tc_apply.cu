@@ -909,9 +909,9 @@ static bool item_supported(const DevItem& it, int d) {
   return true;
 }
 
-// Does a launch run on a converter-warp kernel (see launch())?  Only those read page boxes: all but the kernels
-// with a segment table.
-static bool uses_cv_kernel(bool seg) { return !seg; }
+// Does a launch run on a converter-warp kernel (see launch())?  Only those read page boxes: all but the kernel
+// with a segment table and two rank blocks.
+static bool uses_cv_kernel(int max_r, bool seg) { return !(seg && max_r > 32); }
 
 static bool build_maps(const DevItem& it, ItemMaps* mp, bool page_boxes) {
   // paged pools on both sides with one page size (and all layers in one allocation): a box per page instead of one
@@ -972,8 +972,12 @@ static int launch(const ApplyTcLaunch& L, int max_r, bool paged, cudaStream_t s,
     if (sms <= 0) return KVC_E_CUDA;
     grid = (int)(L.total_tiles < sms ? L.total_tiles : sms);
   }
-  if (seg) {      // per-row tables: the paged ring depths (three coefficient slots) for one rank block
-    cudaError_t es = (max_r > 32) ? launch_seg_t<2, 4, 2>(L, *seg, grid, s) : launch_seg_t<1, 5, 3>(L, *seg, grid, s);
+  if (seg) {
+    // per-row tables: converter warps for one rank block (at the sustained clock 0.98 against 0.89 of the copy
+    // bandwidth on a contiguous source, 0.945 against 0.86 on a paged one, which also gets its page boxes); with two
+    // rank blocks the team keeps the conversions (0.89 / 0.87 against 0.885 / 0.84)
+    cudaError_t es = (max_r > 32) ? launch_seg_t<2, 4, 2>(L, *seg, grid, s)
+                                  : (paged ? launch_seg_t<1, 5, 3, true>(L, *seg, grid, s) : launch_seg_t<1, 5, 2, true>(L, *seg, grid, s));
     return es == cudaSuccess ? KVC_OK : KVC_E_CUDA;
   }
   // converter warps (CV) everywhere: with the SM clock where the power cap holds it in a long run (1.7-1.8 GHz)
@@ -1013,7 +1017,7 @@ int tc_apply_single(const DevItem& item, int d, int pairing, uint32_t* status, c
   memset(&L, 0, sizeof(L));
   L.one = item;
   L.one.tiles_per_slab = (item.src.T + tc::kTileTok - 1) / tc::kTileTok;
-  if (!tc::build_maps(L.one, &L.one_maps, tc::uses_cv_kernel(seg != nullptr))) return KVC_E_CUDA;
+  if (!tc::build_maps(L.one, &L.one_maps, tc::uses_cv_kernel(item.st.r, seg != nullptr))) return KVC_E_CUDA;
   L.n_items = 1;
   L.pairing = pairing;
   L.total_tiles = (int64_t)item.L * item.H * 2 * L.one.tiles_per_slab;
@@ -1112,7 +1116,7 @@ int tc_apply_batch(DevItem* tab, int64_t* prefix, int n_items, int n_table, int 
   tc::ItemMaps* maps = reinterpret_cast<tc::ItemMaps*>(stg + maps_off);
   for (int i = 0; i < n_items; ++i) {
     tab[i].tiles_per_slab = (tab[i].src.T + tc::kTileTok - 1) / tc::kTileTok;
-    if (!tc::build_maps(tab[i], &maps[i], tc::uses_cv_kernel(false))) return KVC_E_CUDA;
+    if (!tc::build_maps(tab[i], &maps[i], tc::uses_cv_kernel(tab[i].st.r, false))) return KVC_E_CUDA;
   }
 
   struct Plan {
