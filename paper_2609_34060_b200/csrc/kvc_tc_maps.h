@@ -51,6 +51,7 @@ inline bool encode_cache(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base,
 inline bool page_box_ok(const DevCache& c, int L) {
   if (!c.page_table) return false;
   const int page = c.page_mask + 1;
+  if ((int64_t)c.n_phys * L >= (int64_t)1 << 31) return false;      // the merged page coordinate is a 32-bit integer
   return page < 128 && (L == 1 || c.s_layer == (int64_t)c.n_phys * c.s_page);
 }
 inline bool encode_cache_page_box(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base, int L, int H) {
