@@ -161,7 +161,8 @@ def version() -> str:
 class Cache:
     """A cache descriptor over torch tensors (which it keeps alive).
 
-    contiguous: ``k``, ``v`` bf16 [L, H, T, d].
+    contiguous: ``k``, ``v`` bf16 [L, H, T, d]; ``token_major=True``: [L, T, H, d] (each token with all its
+                heads), described to the library through the strides.
     paged:      ``k``, ``v`` bf16 pools [L, P, H, page, d], ``page_table`` int32
                 [ceil(T/page)], ``T`` the logical length.  ``token_major=True``: the pools
                 are [L, P, page, H, d] (a page holds its tokens one after the other, each
@@ -175,8 +176,10 @@ class Cache:
         self.k, self.v, self.page_table = k, v, page_table
         self.token_major = bool(token_major)
         if page_table is None:
-            assert not token_major
-            self.L, self.H, self.T, self.d = (int(x) for x in k.shape)
+            if token_major:
+                self.L, self.T, self.H, self.d = (int(x) for x in k.shape)
+            else:
+                self.L, self.H, self.T, self.d = (int(x) for x in k.shape)
             self.page, self.P = 0, 0
         else:
             assert page_table.dtype == torch.int32 and page_table.is_contiguous() and T is not None
@@ -192,6 +195,9 @@ class Cache:
         s.L, s.H, s.T, s.d = self.L, self.H, self.T, self.d
         if self.page_table is None:
             s.layout = KVC_CONTIG
+            if self.token_major:
+                s.s_tok, s.s_head = self.H * self.d, self.d
+                s.s_layer = self.T * self.H * self.d
         else:
             s.layout = KVC_PAGED
             s.page_size, s.n_phys_pages = self.page, self.P
@@ -205,7 +211,7 @@ class Cache:
     def empty_like(self, page_table: Optional[torch.Tensor] = None, fill: Optional[float] = None) -> "Cache":
         mk = (lambda t: torch.empty_like(t)) if fill is None else (lambda t: torch.full_like(t, fill))
         if self.page_table is None:
-            return Cache(mk(self.k), mk(self.v))
+            return Cache(mk(self.k), mk(self.v), token_major=self.token_major)
         return Cache(mk(self.k), mk(self.v), T=self.T,
                      page_table=self.page_table if page_table is None else page_table, token_major=self.token_major)
 

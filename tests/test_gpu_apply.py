@@ -359,3 +359,33 @@ def test_token_major_pages_give_the_same_bits(cfg):
         kvc.kvc_apply_multi(src_t, states, None, None, 11, rope, mb, wsm)
         torch.cuda.synchronize()
         assert torch.equal(hm(mb.k), ma.k) and torch.equal(hm(mb.v), ma.v)
+
+
+def test_token_major_contiguous_cache_gives_the_same_bits():
+    """A contiguous cache held as [L, T, H, d] instead of [L, H, T, d], through the strides: one hop, the chain
+    and a projection give the same bits in the same logical places."""
+    cfg = CFG_8B_S
+    rope = kvc.Rope(cfg.theta)
+    src_cpu = hp.make_cache(cfg)
+    src = hp.to_dev(src_cpu, DEV)
+    tm = lambda t: t.permute(0, 2, 1, 3).contiguous()
+    src_t = kvc.Cache(tm(src.k), tm(src.v), token_major=True)
+    pl = wl.prefix_lengths(cfg)[:3]
+    states = [hp.state_to_dev(hp.make_state(cfg, a), DEV) for a in (1, 2)]
+    outs = [kvc.Cache(torch.zeros_like(src.k), torch.zeros_like(src.v)) for _ in range(2)]
+    outs_t = [kvc.Cache(torch.zeros_like(src_t.k), torch.zeros_like(src_t.v), token_major=True) for _ in range(2)]
+    kvc.kvc_chain(src, pl, states, rope, outs)
+    kvc.kvc_chain(src_t, pl, states, rope, outs_t)
+    torch.cuda.synchronize()
+    assert kvc.kvc_last_path() == kvc.KVC_PATH_TC
+    for a, b in zip(outs, outs_t):
+        assert torch.equal(tm(b.k), a.k) and torch.equal(tm(b.v), a.v)
+    # projection of the second agent's cache against the first, both layouts
+    sts = []
+    for s_, t_ in ((src, outs[0]), (src_t, outs_t[0])):
+        st = kvc.State(torch.zeros(cfg.L, cfg.H, cfg.T, cfg.r, device=DEV), torch.zeros(cfg.L, cfg.H, cfg.T, cfg.r, device=DEV),
+                       states[1].basis_k.clone(), states[1].basis_v.clone())
+        kvc.kvc_state_update(s_, t_, pl[1] - pl[0], rope, st, kvc.KVC_PROJECT)
+        sts.append(st)
+    torch.cuda.synchronize()
+    assert torch.equal(sts[0].coeff_k, sts[1].coeff_k) and torch.equal(sts[0].coeff_v, sts[1].coeff_v)
