@@ -397,8 +397,7 @@ __device__ __forceinline__ void apply_tc_body(const ApplyTcLaunch& p, const SegT
       if (!paged) {
         if (lane == 0) {
           mbar_expect_tx(bar, kBaseBytes);
-          tma_load_5d(st_base, smap, bar, 0, t.t0, t.h, 0, t.l);
-          tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t.t0, t.h, 0, t.l);
+          tma_load_5d(st_base, smap, bar, 0, t.t0, 0, t.h, t.l);      // both halves in one box
         }
       } else {
         const bool valid = lane < n_pages && (unsigned)id < (unsigned)it.src.n_phys;

@@ -161,8 +161,7 @@ __global__ void __launch_bounds__(kThreadsCv, 1) chain_tc_kernel(const __grid_co
       if (!paged) {
         if (lane == 0) {
           mbar_expect_tx(bar, kBaseBytes);
-          tma_load_5d(st_base, smap, bar, 0, t0, h, 0, l);
-          tma_load_5d(st_base + kHalfBytes, smap, bar, 64, t0, h, 0, l);
+          tma_load_5d(st_base, smap, bar, 0, t0, 0, h, l);            // both halves in one box
         }
       } else {
         const bool valid = lane < n_pages && (unsigned)id < (unsigned)p.src.n_phys;

@@ -27,11 +27,22 @@ inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 5-D view of a cache: (channel, token-in-unit, head, unit, layer); unit = page (paged) or the whole sequence.
+// 5-D view of a cache.  Paged: (channel, token-in-page, head, page, layer), a box per page and 64-channel half.
+// Contiguous: (channel-in-half, token, half, head, layer), ONE box of 64 x 128 x 2 per tile: it lands as
+// [half][128 rows][64 channels], the layout of two per-half boxes, and fetches whole 256-byte rows whatever the
+// distance between them ([L, H, T, d] or [L, T, H, d]).
 inline bool encode_cache(CUtensorMap* m, const DevCache& c, __nv_bfloat16* base, int L, int H) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const bool paged = c.page_table != nullptr;
+  if (!paged) {
+    const cuuint64_t dims[5] = {64, (cuuint64_t)c.T, 2, (cuuint64_t)H, (cuuint64_t)L};
+    const cuuint64_t strides[4] = {(cuuint64_t)c.s_tok * 2, 128, (cuuint64_t)c.s_head * 2, (cuuint64_t)c.s_layer * 2};
+    const cuuint32_t box[5] = {64, 128, 2, 1, 1};
+    const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  }
   const cuuint64_t rows = paged ? (cuuint64_t)(c.page_mask + 1) : (cuuint64_t)c.T;
   const cuuint64_t units = paged ? (cuuint64_t)c.n_phys : 1;
   const cuuint64_t dims[5] = {128, rows, (cuuint64_t)H, units, (cuuint64_t)L};

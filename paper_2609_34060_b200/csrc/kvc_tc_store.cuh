@@ -53,8 +53,7 @@ __device__ __forceinline__ void store_tile(const DevCache& dst, const CUtensorMa
   constexpr int kHalf = 128 * 128;                // bytes of one 64-channel half
   if (dst.page_table == nullptr) {
     if (lane == 0) {
-      tma_store_5d(dmap, st_base, 0, t0, h, 0, l);
-      tma_store_5d(dmap, st_base + kHalf, 64, t0, h, 0, l);
+      tma_store_5d(dmap, st_base, 0, t0, 0, h, l);                 // both halves in one box
     }
     return;
   }

@@ -128,8 +128,7 @@ __device__ __forceinline__ void tile_issue(const DevCache& c, const CUtensorMap*
                                            const PTile& t, int lane, int id, bool valid) {
   if (!valid) return;
   if (!c.page_table) {
-    tma_load_5d(dst, map, bar, 0, t.t0, t.h, 0, t.l);
-    tma_load_5d(dst + kHalfBytes, map, bar, 64, t.t0, t.h, 0, t.l);
+    tma_load_5d(dst, map, bar, 0, t.t0, 0, t.h, t.l);               // both halves in one box
   } else {
     const int page = c.page_mask + 1;
     tma_load_5d(dst + lane * page * 128, map, bar, 0, 0, t.h, id, t.l);
