@@ -318,7 +318,7 @@ def main():
         pe.record()
         torch.cuda.synchronize()
         est = dist_util.max_over_ranks(pb.elapsed_time(pe), dev)
-        repeats = int(min(25, max(1, round(1500.0 / max(est * args.steps, 1e-3)))))
+        repeats = int(min(201, max(1, round(1500.0 / max(est * args.steps, 1e-3)))))
         repeats += 1 - repeats % 2          # odd: the median is a measured block
     barrier()
     sampler = ClockSampler(local)
